@@ -1,0 +1,16 @@
+"""CPU oracle for the convolution forward path.  Test infrastructure only: imported by
+tests/, by the smoke check and by the bench's CPU-baseline leg, never by the product."""
+from .conv_oracle import (  # noqa: F401
+    ConvParams,
+    build,
+    conv_fast,
+    conv_naive,
+    conv_points,
+    double_to_half_bits,
+    half_bits_to_double,
+    num_threads,
+    out_dim,
+    nchw_to_nhwc,
+    nhwc_to_nchw,
+    repack_weights,
+)

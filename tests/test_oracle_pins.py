@@ -1,0 +1,322 @@
+"""Pins for the CPU oracle: hand-worked examples, closed forms, library restatements and
+invariants.  None of these calls the CUDA path; a dropped term, a wrong sign or index, a
+transposed operand or a narrow accumulator in the oracle fails at least one of them."""
+import json
+import os
+
+import numpy as np
+import pytest
+from hypothesis import given, settings, strategies as st
+from scipy.signal import correlate2d
+
+from paper_1901_00858_b200 import workloads
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+F16 = np.float16
+
+
+def _bits_list(hexes):
+    return np.array([int(h, 16) for h in hexes], dtype=np.uint16).view(F16)
+
+
+def _example_tensors(ex, P):
+    n, c, h, w = P.n, P.c, P.h, P.w
+    wshape = (P.k, P.c // P.group, P.r, P.s)
+    if "x_bits" in ex:
+        x = _bits_list(ex["x_bits"]).reshape(n, c, h, w)
+        wt = _bits_list(ex["w_bits"]).reshape(wshape)
+        b = _bits_list(ex["bias_bits"]) if ex.get("bias_bits") else None
+    elif "x_fill" in ex:
+        x = np.full((n, c, h, w), ex["x_fill"], dtype=F16)
+        wt = np.full(wshape, ex["w_fill"], dtype=F16)
+        b = None if ex.get("bias") is None else np.array(ex["bias"], dtype=F16)
+    else:
+        x = np.array(ex["x"], dtype=F16).reshape(n, c, h, w)
+        wt = np.array(ex["w"], dtype=F16).reshape(wshape)
+        b = None if ex.get("bias") is None else np.array(ex["bias"], dtype=F16)
+    return x, wt, b
+
+
+def load_hand_examples():
+    with open(os.path.join(GOLDEN, "hand_examples.json")) as f:
+        return json.load(f)["examples"]
+
+
+@pytest.mark.parametrize("ex", load_hand_examples(), ids=lambda e: e["id"])
+@pytest.mark.parametrize("impl", ["conv_naive", "conv_fast", "conv_points"])
+def test_hand_examples(oracle, ex, impl):
+    P = oracle.ConvParams(**ex["params"])
+    x, wt, b = _example_tensors(ex, P)
+    if impl == "conv_points":
+        shape = ex["out_shape"]
+        coords = np.stack(np.meshgrid(*[np.arange(d) for d in shape], indexing="ij"), -1).reshape(-1, 4)
+        y = oracle.conv_points(P, x, wt, b, ex["relu"], coords).reshape(shape)
+    else:
+        y = getattr(oracle, impl)(P, x, wt, b, ex["relu"])
+    assert list(y.shape) == ex["out_shape"]
+    if "expected_bits" in ex:
+        assert [format(v, "04x") for v in y.view(np.uint16).ravel()] == ex["expected_bits"]
+    else:
+        assert y.ravel().astype(np.float64).tolist() == [float(v) for v in ex["expected"]]
+
+
+def test_out_dim_golden(oracle):
+    with open(os.path.join(GOLDEN, "out_dims.json")) as f:
+        cases = json.load(f)["cases"]
+    for size, k, pad, stride, dil, want in cases:
+        assert oracle.out_dim(size, k, pad, stride, dil) == want, (size, k, pad, stride, dil)
+
+
+@settings(max_examples=300, deadline=None)
+@given(st.integers(1, 300), st.integers(1, 11), st.integers(0, 6), st.integers(1, 6), st.integers(1, 4))
+def test_out_dim_counts_valid_window_positions(oracle, size, k, pad, stride, dil):
+    """Brute force: count start positions t = -pad, -pad+stride, ... whose dilated window
+    [t, t + dil*(k-1)] ends inside the padded line."""
+    extent = dil * (k - 1) + 1
+    count = 0
+    t = -pad
+    while t + extent <= size + pad:
+        count += 1
+        t += stride
+    got = oracle.out_dim(size, k, pad, stride, dil)
+    assert (got if got > 0 else 0) == count
+
+
+def test_workload_planes_agree_with_formula(oracle):
+    for wl in workloads.all_workloads():
+        for l in wl.layers:
+            assert oracle.out_dim(l.h, l.r, l.pad, l.stride, l.dil) == l.out, (wl.name, l.name)
+
+
+# ---- binary16 conversion ---------------------------------------------------------------
+
+def test_half_to_double_all_patterns(oracle):
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    want = bits.view(F16).astype(np.float64)
+    got = np.array([oracle.half_bits_to_double(int(b)) for b in bits])
+    nan = np.isnan(want)
+    assert np.array_equal(np.isnan(got), nan)
+    assert np.array_equal(got[~nan], want[~nan])
+    assert np.array_equal(np.signbit(got[~nan]), np.signbit(want[~nan]))
+
+
+def test_double_to_half_roundtrip_midpoints_and_ties(oracle):
+    bits = np.arange(0x7c01, dtype=np.uint32).astype(np.uint16)   # +0 .. +inf
+    vals = bits.view(F16).astype(np.float64)
+    d2h = oracle.double_to_half_bits
+    for sgn, sbit in ((1.0, 0), (-1.0, 0x8000)):
+        for i in range(0, len(bits) - 1, 7):           # every 7th pattern: 4500 cases per sign
+            lo, hi = vals[i], vals[i + 1]
+            assert d2h(sgn * lo) == (int(bits[i]) | sbit)
+            if np.isinf(hi):
+                mid = 65520.0
+            else:
+                mid = (lo + hi) / 2                       # exact in fp64
+            even = int(bits[i]) if (bits[i] & 1) == 0 else int(bits[i + 1])
+            assert d2h(sgn * mid) == (even | sbit), (i, mid)
+            assert d2h(sgn * np.nextafter(mid, 0.0)) == (int(bits[i]) | sbit)
+            assert d2h(sgn * np.nextafter(mid, np.inf)) == (int(bits[i + 1]) | sbit)
+    assert d2h(65504.0) == 0x7bff and d2h(65519.99) == 0x7bff and d2h(65520.0) == 0x7c00
+    assert d2h(1e300) == 0x7c00 and d2h(-1e300) == 0xfc00
+    assert d2h(2.0 ** -25) == 0x0000            # tie between 0 and the smallest subnormal -> even
+    assert d2h(np.nextafter(2.0 ** -25, 1.0)) == 0x0001
+    assert d2h(-0.0) == 0x8000
+
+
+def test_double_to_half_matches_numpy_on_random_doubles(oracle):
+    rng = np.random.default_rng(7)
+    v = np.concatenate([rng.normal(0, 1, 4000), rng.normal(0, 1e-6, 2000), rng.normal(0, 3e4, 2000)])
+    want = v.astype(F16).view(np.uint16)
+    got = np.array([oracle.double_to_half_bits(float(t)) for t in v], dtype=np.uint16)
+    assert np.array_equal(got, want)
+
+
+# ---- invariants and restatements ---------------------------------------------------------
+
+def _dyadic(rng, shape, lo=-8, hi=8, scale=0.25):
+    """Small dyadic rationals: every product and partial sum below is exact in fp64 and the
+    results are exact in binary16, so equalities are bit-for-bit whatever the summation order."""
+    return (rng.integers(lo, hi + 1, size=shape) * scale).astype(F16)
+
+
+def test_1x1_conv_is_matmul(oracle):
+    rng = np.random.default_rng(1)
+    n, c, h, w, k = 2, 37, 5, 6, 19
+    x = _dyadic(rng, (n, c, h, w), -4, 4, 0.5)
+    wt = _dyadic(rng, (k, c, 1, 1), -4, 4, 0.5)
+    b = _dyadic(rng, (k,))
+    P = oracle.ConvParams(n, c, h, w, k, 1, 1)
+    y = oracle.conv_fast(P, x, wt, b, relu=False)
+    W = wt.reshape(k, c).astype(np.float64)
+    want = np.empty((n, k, h, w))
+    for i in range(n):
+        want[i] = (W @ x[i].reshape(c, h * w).astype(np.float64) + b.astype(np.float64)[:, None]).reshape(k, h, w)
+    assert np.abs(want).max() < 2048  # integers/halves below 2048 are exact in binary16
+    assert np.array_equal(y.astype(np.float64), want)
+    assert np.array_equal(oracle.conv_naive(P, x, wt, b, relu=False), y)
+
+
+@pytest.mark.parametrize("r,dil", [(1, 1), (3, 1), (3, 2), (5, 1), (5, 3), (7, 2)])
+def test_centred_delta_kernel_reproduces_input(oracle, r, dil):
+    rng = np.random.default_rng(r * 10 + dil)
+    n, c, h, w = 2, 3, 9, 11
+    x = rng.uniform(-1, 1, (n, c, h, w)).astype(F16)
+    wt = np.zeros((c, c, r, r), dtype=F16)
+    for ch in range(c):
+        wt[ch, ch, r // 2, r // 2] = 1
+    pad = (r - 1) // 2 * dil
+    P = oracle.ConvParams(n, c, h, w, c, r, r, pad, pad, 1, 1, dil, dil)
+    for fn in (oracle.conv_naive, oracle.conv_fast):
+        y = fn(P, x, wt)
+        assert np.array_equal(y.view(np.uint16), x.view(np.uint16))
+
+
+@pytest.mark.parametrize("r0,s0,pad,dil", [(0, 0, 1, 1), (2, 1, 1, 1), (0, 2, 0, 1), (2, 2, 2, 2), (1, 0, 3, 2)])
+def test_shifted_delta_shifts_input(oracle, r0, s0, pad, dil):
+    rng = np.random.default_rng(5)
+    h, w, r = 8, 9, 3
+    x = rng.uniform(-1, 1, (1, 1, h, w)).astype(F16)
+    wt = np.zeros((1, 1, r, r), dtype=F16)
+    wt[0, 0, r0, s0] = 1
+    P = oracle.ConvParams(1, 1, h, w, 1, r, r, pad, pad, 1, 1, dil, dil)
+    y = oracle.conv_fast(P, x, wt)
+    dy, dx = r0 * dil - pad, s0 * dil - pad     # y[p,q] = X[p+dy, q+dx]
+    want = np.zeros(y.shape, dtype=F16)
+    for p in range(y.shape[2]):
+        for q in range(y.shape[3]):
+            i, j = p + dy, q + dx
+            if 0 <= i < h and 0 <= j < w:
+                want[0, 0, p, q] = x[0, 0, i, j]
+    assert np.array_equal(y, want)
+    assert np.array_equal(oracle.conv_naive(P, x, wt), want)
+
+
+def test_linearity_in_x(oracle):
+    rng = np.random.default_rng(2)
+    n, c, h, w, k, r = 1, 4, 7, 8, 5, 3
+    x1 = _dyadic(rng, (n, c, h, w), -4, 4, 0.5)
+    x2 = _dyadic(rng, (n, c, h, w), -4, 4, 0.5)
+    wt = _dyadic(rng, (k, c, r, r), -2, 2, 0.5)
+    P = oracle.ConvParams(n, c, h, w, k, r, r, 1, 1, 2, 1, 1, 1)
+    a = 2.0
+    lhs = oracle.conv_fast(P, (a * x1.astype(np.float64) + x2.astype(np.float64)).astype(F16), wt)
+    rhs = a * oracle.conv_fast(P, x1, wt).astype(np.float64) + oracle.conv_fast(P, x2, wt).astype(np.float64)
+    assert np.array_equal(lhs.astype(np.float64), rhs)
+
+
+@pytest.mark.parametrize("group", [2, 3, 6])
+def test_groups_are_independent_convs_on_channel_slices(oracle, group):
+    rng = np.random.default_rng(group)
+    n, c, h, w, k, r = 2, 6, 6, 7, 12, 3
+    x, wt, b = workloads.random_layer_tensors(rng, n, c, h, w, k, r, r, group)
+    P = oracle.ConvParams(n, c, h, w, k, r, r, 1, 1, 1, 1, 1, 1, group)
+    y = oracle.conv_fast(P, x, wt, b, relu=True)
+    cg, kg = c // group, k // group
+    for gi in range(group):
+        Pg = oracle.ConvParams(n, cg, h, w, kg, r, r, 1, 1)
+        yg = oracle.conv_fast(Pg, x[:, gi * cg:(gi + 1) * cg], wt[gi * kg:(gi + 1) * kg], b[gi * kg:(gi + 1) * kg], relu=True)
+        assert np.array_equal(y[:, gi * kg:(gi + 1) * kg].view(np.uint16), yg.view(np.uint16))
+
+
+@pytest.mark.parametrize("stride", [2, 3])
+def test_stride_is_subsampling_of_stride_1(oracle, stride):
+    rng = np.random.default_rng(stride)
+    n, c, h, w, k, r = 1, 3, 11, 13, 4, 3
+    x, wt, b = workloads.random_layer_tensors(rng, n, c, h, w, k, r, r, 1)
+    y1 = oracle.conv_fast(oracle.ConvParams(n, c, h, w, k, r, r, 1, 1), x, wt, b)
+    ys = oracle.conv_fast(oracle.ConvParams(n, c, h, w, k, r, r, 1, 1, stride, stride), x, wt, b)
+    assert np.array_equal(ys.view(np.uint16), y1[:, :, ::stride, ::stride].view(np.uint16))
+
+
+@pytest.mark.parametrize("dil", [2, 3])
+def test_dilation_is_dense_conv_with_zero_stuffed_kernel(oracle, dil):
+    rng = np.random.default_rng(dil)
+    n, c, h, w, k, r = 1, 2, 12, 10, 3, 3
+    x, wt, b = workloads.random_layer_tensors(rng, n, c, h, w, k, r, r, 1)
+    ext = dil * (r - 1) + 1
+    stuffed = np.zeros((k, c, ext, ext), dtype=F16)
+    stuffed[:, :, ::dil, ::dil] = wt
+    yd = oracle.conv_fast(oracle.ConvParams(n, c, h, w, k, r, r, 2, 2, 1, 1, dil, dil), x, wt, b)
+    y1 = oracle.conv_fast(oracle.ConvParams(n, c, h, w, k, ext, ext, 2, 2), x, stuffed, b)
+    assert np.array_equal(yd.view(np.uint16), y1.view(np.uint16))
+
+
+@pytest.mark.parametrize("pad,stride", [(0, 1), (2, 1), (1, 2)])
+def test_against_scipy_correlate2d(oracle, pad, stride):
+    """Independent library restatement: per (k, c) plane correlation in float64, summed."""
+    rng = np.random.default_rng(11 + pad)
+    n, c, h, w, k, r, s = 2, 3, 9, 8, 4, 3, 2
+    x, wt, b = workloads.random_layer_tensors(rng, n, c, h, w, k, r, s, 1)
+    P = oracle.ConvParams(n, c, h, w, k, r, s, pad, pad, stride, stride)
+    y = oracle.conv_fast(P, x, wt, b, relu=True)
+    xp = np.pad(x.astype(np.float64), ((0, 0), (0, 0), (pad, pad), (pad, pad)))
+    want = np.empty(y.shape, dtype=F16)
+    for i in range(n):
+        for ko in range(k):
+            acc = sum(correlate2d(xp[i, ci], wt[ko, ci].astype(np.float64), mode="valid") for ci in range(c))
+            acc = acc[::stride, ::stride] + float(b[ko])
+            want[i, ko] = np.maximum(acc, 0).astype(F16)
+    # fp64 sums in another order: allow one binary16 step on rare ties, nothing more
+    diff = np.abs(y.astype(np.float64) - want.astype(np.float64))
+    assert np.all(diff <= np.spacing(np.abs(want).astype(F16)).astype(np.float64))
+    assert np.mean(y.view(np.uint16) == want.view(np.uint16)) > 0.999
+
+
+def test_pad_larger_than_kernel_gives_bias_border(oracle):
+    x = np.ones((1, 1, 2, 2), dtype=F16)
+    wt = np.ones((1, 1, 1, 1), dtype=F16)
+    b = np.array([0.25], dtype=F16)
+    y = oracle.conv_fast(oracle.ConvParams(1, 1, 2, 2, 1, 1, 1, 2, 3), x, wt, b)
+    assert y.shape == (1, 1, 6, 8)
+    want = np.full((6, 8), 0.25)
+    want[2:4, 3:5] = 1.25
+    assert np.array_equal(y[0, 0].astype(np.float64), want)
+
+
+def test_invalid_parameters_are_rejected(oracle):
+    x = np.zeros((1, 4, 4, 4), dtype=F16)
+    with pytest.raises(ValueError):
+        oracle.conv_fast(oracle.ConvParams(1, 4, 4, 4, 6, 3, 3, group=4), x, np.zeros((6, 1, 3, 3), dtype=F16))
+    with pytest.raises(ValueError):
+        oracle.conv_fast(oracle.ConvParams(1, 4, 4, 4, 4, 5, 5), x, np.zeros((4, 4, 5, 5), dtype=F16))
+
+
+_desc = st.tuples(
+    st.integers(1, 2), st.sampled_from([1, 2, 3, 4, 0]), st.integers(1, 6), st.integers(1, 6),
+    st.integers(1, 12), st.integers(1, 12), st.integers(1, 5), st.integers(1, 5),
+    st.integers(0, 3), st.integers(0, 3), st.integers(1, 4), st.integers(1, 4),
+    st.integers(1, 3), st.integers(1, 3), st.booleans(), st.booleans(), st.integers(0, 2 ** 31))
+
+
+@settings(max_examples=150, deadline=None)
+@given(_desc)
+def test_fast_is_bit_identical_to_naive(oracle, d):
+    n, g, cg, kg, h, w, r, s, ph, pw, sh, sw, dh, dw, relu, has_bias, seed = d
+    if g == 0:          # depthwise
+        g, cg = cg * 3, 1
+    c, k = g * cg, g * kg
+    if oracle.out_dim(h, r, ph, sh, dh) < 1 or oracle.out_dim(w, s, pw, sw, dw) < 1:
+        return
+    rng = np.random.default_rng(seed)
+    x, wt, b = workloads.random_layer_tensors(rng, n, c, h, w, k, r, s, g)
+    P = oracle.ConvParams(n, c, h, w, k, r, s, ph, pw, sh, sw, dh, dw, g)
+    bias = b if has_bias else None
+    y0 = oracle.conv_naive(P, x, wt, bias, relu)
+    y1 = oracle.conv_fast(P, x, wt, bias, relu)
+    assert np.array_equal(y0.view(np.uint16), y1.view(np.uint16))
+    coords = np.stack(np.meshgrid(*[np.arange(t) for t in y0.shape], indexing="ij"), -1).reshape(-1, 4)
+    y2 = oracle.conv_points(P, x, wt, bias, relu, coords)
+    assert np.array_equal(y2.view(np.uint16), y0.view(np.uint16).ravel())
+
+
+def test_layout_definitions_round_trip(oracle):
+    rng = np.random.default_rng(3)
+    x = rng.uniform(-1, 1, (2, 5, 3, 4)).astype(F16)
+    xp = oracle.nchw_to_nhwc(x, 8)
+    assert xp.shape == (2, 3, 4, 8) and np.all(xp[..., 5:] == 0)
+    assert xp[1, 2, 3, 4] == x[1, 4, 2, 3]
+    assert np.array_equal(oracle.nhwc_to_nchw(xp, 5), x)
+    wt = rng.uniform(-1, 1, (6, 2, 3, 3)).astype(F16)
+    wp = oracle.repack_weights(wt, 3, 8)
+    assert wp.shape == (3, 2, 3, 3, 8)
+    assert wp[2, 1, 0, 2, 1] == wt[5, 1, 0, 2] and np.all(wp[..., 2:] == 0)
