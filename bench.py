@@ -1,0 +1,391 @@
+#!/usr/bin/env python
+"""Benchmark of the convolution-forward hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+A step is one pass of the whole path over one batch of a workload: every layer of the named
+network shape, each with its own resident input, weights, bias and output (the layers'
+inputs are generated independently, so the working set is far larger than L2 and no L2
+flush is needed between steps).  Prints ONE JSON line (rank 0).
+
+N > 1 (under torchrun): the path has no exchange step; every rank runs an independent
+replica on its own batch ("weak" scaling) and the line reports the aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_1901_00858_b200 import workloads  # noqa: E402
+
+DEFAULT_WORKLOAD = "vgg16_n16"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+# ---- bookkeeping that needs no GPU (also exercised by the CPU tests) ------------------------
+
+def layer_flops(batch: int, l) -> float:
+    """2*N*K*(C/g)*R*S*P*Q: padded taps count, bias/ReLU/cast do not."""
+    return 2.0 * batch * l.k * (l.c // l.group) * l.r * l.r * l.out * l.out
+
+
+def layer_bytes(batch: int, l) -> float:
+    """Algorithmic bytes: x read once, w once, bias once, y written once (fp16)."""
+    return 2.0 * (batch * l.c * l.h * l.h + l.k * (l.c // l.group) * l.r * l.r + l.k + batch * l.k * l.out * l.out)
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return dict(FALLBACK_PEAKS, source="fallback")
+
+
+def layer_roof_seconds(batch, l, peaks) -> float:
+    return max(layer_flops(batch, l) / (peaks["bf16_tflops_sustained"] * 1e12),
+               layer_bytes(batch, l) / (peaks["hbm_gbs"] * 1e9))
+
+
+def aggregate(per_rank_flops, per_rank_images, max_seconds_per_step):
+    """Whole-job throughput of independent replicas: everything all ranks processed divided
+    by the slowest rank's time."""
+    return {"tflops": sum(per_rank_flops) / max_seconds_per_step / 1e12,
+            "images_per_s": sum(per_rank_images) / max_seconds_per_step}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.file.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        self.file.close()
+        try:
+            os.unlink(self.file.name)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ---- the oracle legs (CPU) -------------------------------------------------------------------
+
+def oracle_pass(wl, batch):
+    """One pass of every layer of the workload at `batch` images through the CPU oracle as it
+    stands.  Returns (seconds, flops)."""
+    import oracle
+    secs, flops = 0.0, 0.0
+    for li, l in enumerate(wl.expanded_unique()):
+        x, w, b = workloads.make_tensors(wl.config_id, wl.batch, li, l, batch_override=batch)
+        P = oracle.ConvParams(batch, l.c, l.h, l.h, l.k, l.r, l.r, l.pad, l.pad, l.stride, l.stride,
+                              l.dil, l.dil, l.group)
+        t0 = time.perf_counter()
+        oracle.conv_fast(P, x, w, b, l.relu)
+        secs += (time.perf_counter() - t0) * l.count
+        flops += layer_flops(batch, l) * l.count
+    return secs, flops
+
+
+def cpu_baseline(wl):
+    import oracle
+    secs, flops = oracle_pass(wl, 1)
+    batch = 1
+    if secs < 5.0 and wl.batch > 1:
+        batch = int(min(wl.batch, max(2, round(10.0 / max(secs, 1e-3)))))
+        secs, flops = oracle_pass(wl, batch)
+    return {"value": flops / secs / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(),
+            "kind": "oracle", "images_per_s": batch / secs,
+            "sample": f"every layer of {wl.name} once at batch {batch} (of {wl.batch}); repeated shapes "
+                      f"timed once and counted by multiplicity; {flops / 1e9:.1f} GFLOP in {secs:.1f} s"}
+
+
+def run_reference(args, wl):
+    """--impl reference: the CPU oracle on the machine's host cores, same metric and config; each
+    step is a bounded sample (every layer of the workload at batch 1)."""
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    oracle.build()
+    for _ in range(min(args.warmup, 1)):
+        oracle_pass(wl, 1)
+    steps = max(1, min(args.steps, 5))
+    secs, flops = 0.0, 0.0
+    for _ in range(steps):
+        s, f = oracle_pass(wl, 1)
+        secs += s
+        flops += f
+    val = flops / secs / 1e12
+    line = {
+        "impl": "reference", "metric": "conv_forward_tflops", "value": val, "unit": "TFLOP/s",
+        "n_gpus": args.gpus, "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": secs / steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "sample": "every layer once at batch 1 per step"},
+        "images_per_s": steps / secs,
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "kind": "oracle", "cores": oracle.num_threads(),
+                         "sample": f"every layer of {wl.name} at batch 1, {steps} passes"},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---- the CUDA arm ----------------------------------------------------------------------------
+
+def run_ours(args, wl):
+    import torch
+    import torch.distributed as dist
+    from paper_1901_00858_b200 import binding as hgc
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the CUDA path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    hgc.lib()
+    peaks = load_peaks()
+    stream = torch.cuda.current_stream()
+    layers = wl.expanded()
+    batch = wl.batch
+
+    # resident tensors, one set per layer (weights registered once: steady-state inference)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(1234 + rank)
+    state = []
+    for li, l in enumerate(layers):
+        d = hgc.ConvDesc(batch, l.c, l.h, l.h, l.k, l.r, l.r, l.pad, l.pad, l.stride, l.stride, l.dil, l.dil,
+                         l.group)
+        d.ensure_workspace()
+        x = torch.empty((batch, l.c, l.h, l.h), dtype=torch.float16, device="cuda")
+        x.uniform_(l.x_lo, 1.0, generator=gen)
+        w = torch.empty((l.k, l.c // l.group, l.r, l.r), dtype=torch.float16, device="cuda")
+        w.normal_(0.0, float(np.sqrt(2.0 / l.fan_in())), generator=gen)
+        b = torch.empty((l.k,), dtype=torch.float16, device="cuda")
+        b.uniform_(-0.1, 0.1, generator=gen)
+        y = torch.empty((batch, l.k, l.out, l.out), dtype=torch.float16, device="cuda")
+        d.set_weights(w)
+        state.append((d, x, w, b, y, l))
+    torch.cuda.synchronize()
+
+    def one_step(events=None):
+        for i, (d, x, w, b, y, l) in enumerate(state):
+            if events is not None:
+                events[i][0].record(stream)
+            hgc.conv_forward(d, x, w, b, y, l.relu, stream)
+            if events is not None:
+                events[i][1].record(stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    barrier()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    # timed region: exactly K steps between two events on the launching stream
+    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in state]
+          for _ in range(args.steps)]
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = hgc.kernel_launch_count()
+    barrier()
+    t_start.record(stream)
+    for s in range(args.steps):
+        one_step(ev[s])
+    t_end.record(stream)
+    barrier()
+    launches = hgc.kernel_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = t_start.elapsed_time(t_end)
+    ms_per_step = total_ms / args.steps
+
+    # per-layer device times (average over the K timed steps)
+    layer_ms = [sum(ev[s][i][0].elapsed_time(ev[s][i][1]) for s in range(args.steps)) / args.steps
+                for i in range(len(state))]
+
+    # ---- end to end through the host-buffer entry point ------------------------------------
+    e2e_steps = max(1, min(args.steps, 5))
+    host = []
+    h2d = d2h = 0
+    for (d, x, w, b, y, l) in state:
+        d.ensure_workspace(host=True)
+        hx = torch.empty(x.shape, dtype=torch.float16).pin_memory()
+        hx.copy_(x.cpu())
+        hw = w.cpu().pin_memory()
+        hb = b.cpu().pin_memory()
+        hy = torch.empty(y.shape, dtype=torch.float16).pin_memory()
+        host.append((hx, hw, hb, hy))
+        h2d += (hx.numel() + hw.numel() + hb.numel()) * 2
+        d2h += hy.numel() * 2
+    torch.cuda.synchronize()
+
+    def e2e_step():
+        for (d, x, w, b, y, l), (hx, hw, hb, hy) in zip(state, host):
+            hgc.conv_forward_host(d, hx, hw, hb, hy, l.relu, stream)
+
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+
+    # ---- max over ranks ---------------------------------------------------------------------
+    if world > 1:
+        t = torch.tensor([ms_per_step, e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_per_step, e2e_ms = float(t[0]), float(t[1])
+        lt = torch.tensor([launches], dtype=torch.int64, device="cuda")
+        dist.all_reduce(lt)
+        launches = int(lt[0])
+
+    step_flops = sum(layer_flops(batch, l) for l in layers)
+    agg = aggregate([step_flops] * world, [batch] * world, ms_per_step * 1e-3)
+    e2e = aggregate([step_flops] * world, [batch] * world, e2e_ms * 1e-3)
+
+    if rank == 0:
+        # dominant kernel path by time in the timed region
+        by_path = {}
+        for (d, x, w, b, y, l), ms in zip(state, layer_ms):
+            p = hgc.PATH_NAMES[d.path()]
+            e = by_path.setdefault(p, {"ms": 0.0, "flops": 0.0, "bytes": 0.0, "launches": 0})
+            e["ms"] += ms
+            e["flops"] += layer_flops(batch, l)
+            e["bytes"] += layer_bytes(batch, l)
+            e["launches"] += 1
+        dom = max(by_path, key=lambda k: by_path[k]["ms"])
+        e = by_path[dom]
+        if dom == "depthwise":
+            roof = {"bound": "hbm", "kernel": dom, "achieved": e["bytes"] / (e["ms"] * 1e-3) / 1e9,
+                    "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+        else:
+            roof = {"bound": "tensor", "kernel": dom, "achieved": e["flops"] / (e["ms"] * 1e-3) / 1e12,
+                    "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"}
+        roof["frac"] = roof["achieved"] / roof["peak"]
+        roof["traffic"] = None
+        roof["peak_source"] = peaks["source"]
+        roof["share_of_step"] = e["ms"] / sum(layer_ms)
+        roof["avg_launch_ms"] = e["ms"] / e["launches"]
+        t_roof = sum(layer_roof_seconds(batch, l, peaks) for l in layers)
+        cpu = cpu_baseline(wl) if world == 1 and not args.no_cpu_baseline else None
+        line = {
+            "metric": "conv_forward_tflops", "value": agg["tflops"], "unit": "TFLOP/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16 (f32 accumulate)",
+            "data": "synthetic",
+            "config": {"workload": wl.name, "layers": len(layers), "batch_per_gpu": batch,
+                       "l2": "inputs larger than L2 (every layer has its own tensors)",
+                       "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
+            "images_per_s": agg["images_per_s"],
+            "roofline": roof,
+            "roofline_config": {"t_roof_ms": t_roof * 1e3, "frac": t_roof * 1e3 / (sum(layer_ms)),
+                                "note": "sum over layers of max(flops/tensor peak, bytes/HBM peak) / sum of layer times"},
+            "per_path": {k: {"ms_per_step": v["ms"], "launches_per_step": v["launches"],
+                             "tflops": v["flops"] / (v["ms"] * 1e-3) / 1e12,
+                             "gbs": v["bytes"] / (v["ms"] * 1e-3) / 1e9} for k, v in by_path.items()},
+            "e2e": {"value": e2e["tflops"], "unit": "TFLOP/s", "ms_per_step": e2e_ms, "steps": e2e_steps,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "images_per_s": e2e["images_per_s"]},
+            "gpu_launches": launches,
+            "clocks": clocks,
+        }
+        if cpu is not None:
+            line["cpu_baseline"] = cpu
+        if args.layers:
+            line["layers"] = [{"name": l.name, "path": hgc.PATH_NAMES[d.path()], "ms": ms,
+                               "tflops": layer_flops(batch, l) / (ms * 1e-3) / 1e12,
+                               "gbs": layer_bytes(batch, l) / (ms * 1e-3) / 1e9,
+                               "roof_frac": layer_roof_seconds(batch, l, peaks) * 1e3 / ms}
+                              for (d, x, w, b, y, l), ms in zip(state, layer_ms)]
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD,
+                    help="one of: " + ", ".join(w.name for w in workloads.all_workloads()))
+    ap.add_argument("--layers", action="store_true", help="add per-layer figures to the JSON line")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    wl = workloads.by_name(args.workload)
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

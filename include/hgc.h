@@ -1,0 +1,165 @@
+/*
+ * hgc.h - C ABI of the B200 (sm_100a) FP16 convolution-forward library.
+ *
+ * The library implements the hot path of a forward-only FP16 inference engine in the
+ * style of HG-Caffe: the convolution layer forward with the semantics the paper inherits
+ * from BVLC Caffe (Section 2.2), FP16 tensors end to end with no float<->half conversion
+ * inside the engine (Section 3.3), scalars kept in host types and handed over at the call
+ * boundary (Section 3.2), a wide accumulator because FP16 accumulation overflows and loses
+ * small terms (Section 3.1), and no third-party compute library on the path (Section 2).
+ *
+ * General rules
+ *   - Every function returns an hgc_status (int); 0 is HGC_OK.  Nothing throws, aborts or
+ *     prints.  hgc_status_string() names a code.
+ *   - "device pointer" = CUDA global memory of the current device; "host pointer" = ordinary
+ *     (preferably pinned) host memory.  Each argument says which.
+ *   - Tensors are dense IEEE binary16: x[N][C][H][W], w[K][C/group][R][S], bias[K],
+ *     y[N][K][P][Q].  Device tensor pointers must be 16-byte aligned (HGC_BAD_ALIGNMENT) and
+ *     must not overlap.  The library borrows them until the work queued on `stream` is done.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - hgc_conv_forward and the layout/repack calls only enqueue kernels on `stream`: they do
+ *     not allocate, free or synchronise.  Scratch memory is provided by the caller through
+ *     hgc_conv_set_workspace and stays caller-owned.
+ *   - A descriptor is not thread-safe; distinct descriptors are independent.
+ *   - All element offsets are computed in 64-bit integers.
+ */
+#ifndef HGC_H_
+#define HGC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum hgc_status {
+  HGC_OK = 0,
+  HGC_INVALID_ARG = 1,    /* NULL where a pointer is required, or an impossible layer */
+  HGC_UNSUPPORTED = 2,    /* a valid request this build has no kernel for */
+  HGC_BAD_ALIGNMENT = 3,  /* a device tensor pointer is not 16-byte aligned */
+  HGC_NO_WORKSPACE = 4,   /* the chosen path needs scratch memory and none (or too little) is set */
+  HGC_CUDA_ERROR = 5,     /* a CUDA runtime/driver call or a kernel launch failed */
+  HGC_DEVICE_TIMEOUT = 6  /* a bounded device-side wait expired; the output is not valid */
+} hgc_status;
+
+/* Which kernel the planner chose for a descriptor (hgc_conv_path). */
+typedef enum hgc_path {
+  HGC_PATH_DIRECT = 0,     /* direct convolution on CUDA cores, any valid layer */
+  HGC_PATH_DEPTHWISE = 1,  /* 3x3 depthwise (group == C == K) stencil on CUDA cores */
+  HGC_PATH_IGEMM = 2       /* implicit GEMM on tcgen05 tensor cores with TMEM accumulators */
+} hgc_path;
+
+/* Layer description.  Scalars are plain host integers (Section 3.2: scalars stay in host
+   types; only tensors are half). */
+typedef struct hgc_conv_params {
+  int32_t n, c, h, w;        /* input  x[N][C][H][W]                      */
+  int32_t k, r, s;           /* weights w[K][C/group][R][S]               */
+  int32_t pad_h, pad_w;      /* zero padding, same amount on both sides   */
+  int32_t stride_h, stride_w;
+  int32_t dil_h, dil_w;      /* dilation: tap r reads row p*stride - pad + r*dil */
+  int32_t group;             /* C % group == 0 and K % group == 0         */
+  int32_t flags;             /* HGC_FLAG_* bits; 0 = planner's choice     */
+} hgc_conv_params;
+
+#define HGC_FLAG_FORCE_DIRECT 1  /* always use HGC_PATH_DIRECT (testing / comparison) */
+
+typedef struct hgc_conv_desc hgc_conv_desc; /* opaque; owned by the caller via create/destroy */
+
+/*
+ * Shape inference and planning (host only, no device work).  Implements the Caffe
+ * convolution output size (the layer semantics of Section 2.2):
+ *     P = floor((H + 2*pad_h - dil_h*(R-1) - 1) / stride_h) + 1,   Q likewise.
+ * HGC_INVALID_ARG if out or p is NULL, any of n,c,h,w,k,r,s,group,stride,dil < 1, pad < 0,
+ * C % group != 0, K % group != 0, or P < 1 or Q < 1.  On failure *out is left NULL.
+ */
+int hgc_conv_desc_create(hgc_conv_desc** out, const hgc_conv_params* p);
+
+/* Frees the descriptor (host memory only).  NULL is accepted.  The caller must make sure
+   that no queued work still uses it. */
+int hgc_conv_desc_destroy(hgc_conv_desc* d);
+
+/*
+ * The layer forward (Sections 2.2, 3.1, 3.3):
+ *   y[n,k,p,q] = fp16_rn( act( bias[k] + sum_{c',r,s} X(n, grp(k)*C/g + c',
+ *                   p*stride_h - pad_h + r*dil_h, q*stride_w - pad_w + s*dil_w) * w[k,c',r,s] ) )
+ * with X zero outside the image, grp(k) = k / (K/group), fp32 accumulation, bias added in
+ * fp32 before the activation, act = max(.,0) if relu != 0 else identity, and one
+ * round-to-nearest-even conversion to binary16 at the end.
+ * x, w, y: device pointers (required).  bias: device pointer or NULL (no bias).
+ * Enqueues on `stream` and returns; results are ready when the stream reaches that point.
+ * Errors: HGC_INVALID_ARG (NULL d/x/w/y), HGC_BAD_ALIGNMENT, HGC_NO_WORKSPACE,
+ * HGC_CUDA_ERROR.  A device-side timeout is reported by hgc_conv_last_device_status.
+ */
+int hgc_conv_forward(hgc_conv_desc* d, const void* x, const void* w, const void* bias,
+                     void* y, int relu, void* stream);
+
+/*
+ * Same layer with HOST tensors: copies x, w, bias host->device into the workspace, runs
+ * hgc_conv_forward, copies y device->host, all queued on `stream` (asynchronous if the host
+ * memory is pinned; the caller synchronises the stream before reading y).  Needs a workspace
+ * of at least hgc_conv_host_workspace_bytes.  x, w, bias, y: host pointers.
+ */
+int hgc_conv_forward_host(hgc_conv_desc* d, const void* x, const void* w, const void* bias,
+                          void* y, int relu, void* stream);
+
+/* Output shape N, K, P, Q of the descriptor (any output pointer may be NULL). */
+int hgc_conv_output_dims(const hgc_conv_desc* d, int32_t* n, int32_t* k, int32_t* p, int32_t* q);
+
+/* The kernel path the planner chose (an hgc_path value). */
+int hgc_conv_path(const hgc_conv_desc* d, int32_t* path);
+
+/* Scratch bytes hgc_conv_forward needs for this descriptor (0 if none). */
+int hgc_conv_workspace_bytes(const hgc_conv_desc* d, size_t* bytes);
+
+/* Scratch bytes hgc_conv_forward_host needs: the above plus device staging for x, w, bias, y. */
+int hgc_conv_host_workspace_bytes(const hgc_conv_desc* d, size_t* bytes);
+
+/* Hands the descriptor a caller-owned device buffer (256-byte aligned) used as scratch by
+   later forwards.  It must stay valid until those forwards have completed.  Passing
+   (NULL, 0) detaches it.  Setting a workspace forgets registered weights. */
+int hgc_conv_set_workspace(hgc_conv_desc* d, void* dev_ptr, size_t bytes);
+
+/*
+ * Optional: registers a weight tensor (device pointer) and runs the one-off weight
+ * re-layout for it on `stream` (Section 3.3: weights are prepared once when loaded, not
+ * converted on every use).  Later hgc_conv_forward calls given the same `w` pointer skip
+ * that step; a different pointer is re-laid-out on the fly each call.  Needs the workspace
+ * to be set if hgc_conv_workspace_bytes is non-zero.  No effect on paths that read w as is.
+ */
+int hgc_conv_set_weights(hgc_conv_desc* d, const void* w, void* stream);
+
+/* Reads the device status word of the descriptor's last forward (synchronises `stream`
+   work that was queued by this descriptor).  *status is HGC_OK or HGC_DEVICE_TIMEOUT. */
+int hgc_conv_last_device_status(hgc_conv_desc* d, int32_t* status);
+
+/*
+ * Layout transforms (the engine keeps tensors in FP16 and only re-arranges them; no value is
+ * changed, Section 3.3).  src, dst: device pointers, 16-byte aligned, non-overlapping.
+ *   nchw_to_nhwc: dst[n][h][w][c_pad] = src[n][c][h][w] for c < C, 0 for C <= c < c_pad
+ *   nhwc_to_nchw: dst[n][c][h][w]     = src[n][h][w][c] for c < C  (padding dropped)
+ * c_pad >= c and c_pad % 8 == 0 (one pixel is a whole number of 16-byte vectors).
+ */
+int hgc_layout_nchw_to_nhwc(const void* src, void* dst, int32_t n, int32_t c, int32_t h,
+                            int32_t w, int32_t c_pad, void* stream);
+int hgc_layout_nhwc_to_nchw(const void* src, void* dst, int32_t n, int32_t c, int32_t h,
+                            int32_t w, int32_t c_pad, void* stream);
+
+/*
+ * Weight re-layout for the implicit-GEMM path:
+ *   dst[g][K/group][R][S][c_pad] = src[g*(K/group)+k'][c'][r][s] for c' < C/group, else 0.
+ * src, dst: device pointers, 16-byte aligned.  c_pad >= C/group, c_pad % 8 == 0.
+ */
+int hgc_weights_repack(const void* src, void* dst, int32_t k, int32_t c_per_group, int32_t r,
+                       int32_t s, int32_t group, int32_t c_pad, void* stream);
+
+/* Number of kernels this library has launched in this process so far. */
+int hgc_kernel_launch_count(uint64_t* count);
+
+/* Static, never-NULL description of a status code. */
+const char* hgc_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HGC_H_ */

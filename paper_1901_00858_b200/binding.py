@@ -1,0 +1,212 @@
+"""Thin ctypes binding of libhgc.so: argument marshalling only.
+
+Every step of the path runs inside the CUDA library; torch is used for device memory and
+streams.  The names mirror the C ABI (include/hgc.h).  If the compiled library is missing
+this module raises on first use: there is no CPU or library fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libhgc.so")
+
+HGC_OK, HGC_INVALID_ARG, HGC_UNSUPPORTED, HGC_BAD_ALIGNMENT, HGC_NO_WORKSPACE, HGC_CUDA_ERROR, \
+    HGC_DEVICE_TIMEOUT = range(7)
+HGC_PATH_DIRECT, HGC_PATH_DEPTHWISE, HGC_PATH_IGEMM = range(3)
+HGC_FLAG_FORCE_DIRECT = 1
+PATH_NAMES = {HGC_PATH_DIRECT: "direct", HGC_PATH_DEPTHWISE: "depthwise", HGC_PATH_IGEMM: "igemm"}
+
+
+class HgcError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (hgc_status {status})")
+
+
+class hgc_conv_params(ctypes.Structure):
+    _fields_ = [(f, ctypes.c_int32) for f in (
+        "n", "c", "h", "w", "k", "r", "s", "pad_h", "pad_w", "stride_h", "stride_w",
+        "dil_h", "dil_w", "group", "flags")]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libhgc.so (built in-tree by `python -m paper_1901_00858_b200.build`)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_1901_00858_b200.build` "
+                "(nvcc, sm_100a). There is no fallback path.")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i32p = ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32)
+        szp = ctypes.POINTER(ctypes.c_size_t)
+        L.hgc_conv_desc_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(hgc_conv_params)]
+        L.hgc_conv_desc_destroy.argtypes = [vp]
+        L.hgc_conv_forward.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int, vp]
+        L.hgc_conv_forward_host.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int, vp]
+        L.hgc_conv_output_dims.argtypes = [vp, i32p, i32p, i32p, i32p]
+        L.hgc_conv_path.argtypes = [vp, i32p]
+        L.hgc_conv_workspace_bytes.argtypes = [vp, szp]
+        L.hgc_conv_host_workspace_bytes.argtypes = [vp, szp]
+        L.hgc_conv_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
+        L.hgc_conv_set_weights.argtypes = [vp, vp, vp]
+        L.hgc_conv_last_device_status.argtypes = [vp, i32p]
+        L.hgc_layout_nchw_to_nhwc.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp]
+        L.hgc_layout_nhwc_to_nchw.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp]
+        L.hgc_weights_repack.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, vp]
+        L.hgc_kernel_launch_count.argtypes = [ctypes.POINTER(ctypes.c_uint64)]
+        L.hgc_status_string.argtypes = [ctypes.c_int]
+        L.hgc_status_string.restype = ctypes.c_char_p
+        for name in ("hgc_conv_desc_create", "hgc_conv_desc_destroy", "hgc_conv_forward",
+                     "hgc_conv_forward_host", "hgc_conv_output_dims", "hgc_conv_path",
+                     "hgc_conv_workspace_bytes", "hgc_conv_host_workspace_bytes",
+                     "hgc_conv_set_workspace", "hgc_conv_set_weights", "hgc_conv_last_device_status",
+                     "hgc_layout_nchw_to_nhwc", "hgc_layout_nhwc_to_nchw", "hgc_weights_repack",
+                     "hgc_kernel_launch_count"):
+            getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().hgc_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != HGC_OK:
+        raise HgcError(status, where)
+
+
+def _ptr(t) -> Optional[int]:
+    """Device (or host) address of a torch tensor / numpy array / int / None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if hasattr(t, "data_ptr"):
+        return t.data_ptr()
+    return t.ctypes.data
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+class ConvDesc:
+    """Owns an hgc_conv_desc.  Keyword arguments are the fields of hgc_conv_params."""
+
+    def __init__(self, n, c, h, w, k, r, s, pad_h=0, pad_w=0, stride_h=1, stride_w=1, dil_h=1,
+                 dil_w=1, group=1, flags=0):
+        self.params = hgc_conv_params(n, c, h, w, k, r, s, pad_h, pad_w, stride_h, stride_w,
+                                      dil_h, dil_w, group, flags)
+        self._h = ctypes.c_void_p()
+        self._ws = None
+        _check(lib().hgc_conv_desc_create(ctypes.byref(self._h), ctypes.byref(self.params)),
+               "hgc_conv_desc_create")
+
+    @property
+    def handle(self):
+        return self._h
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            lib().hgc_conv_desc_destroy(self._h)
+            self._h = ctypes.c_void_p()
+            self._ws = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def output_dims(self):
+        v = [ctypes.c_int32() for _ in range(4)]
+        _check(lib().hgc_conv_output_dims(self._h, *[ctypes.byref(t) for t in v]), "hgc_conv_output_dims")
+        return tuple(t.value for t in v)
+
+    def path(self) -> int:
+        v = ctypes.c_int32()
+        _check(lib().hgc_conv_path(self._h, ctypes.byref(v)), "hgc_conv_path")
+        return v.value
+
+    def workspace_bytes(self) -> int:
+        v = ctypes.c_size_t()
+        _check(lib().hgc_conv_workspace_bytes(self._h, ctypes.byref(v)), "hgc_conv_workspace_bytes")
+        return v.value
+
+    def host_workspace_bytes(self) -> int:
+        v = ctypes.c_size_t()
+        _check(lib().hgc_conv_host_workspace_bytes(self._h, ctypes.byref(v)), "hgc_conv_host_workspace_bytes")
+        return v.value
+
+    def set_workspace(self, buf, nbytes: Optional[int] = None):
+        """buf: a torch uint8 CUDA tensor (kept alive by this object) or None."""
+        if buf is None:
+            _check(lib().hgc_conv_set_workspace(self._h, None, 0), "hgc_conv_set_workspace")
+            self._ws = None
+            return
+        nbytes = buf.numel() * buf.element_size() if nbytes is None else nbytes
+        _check(lib().hgc_conv_set_workspace(self._h, _ptr(buf), nbytes), "hgc_conv_set_workspace")
+        self._ws = buf
+
+    def ensure_workspace(self, host: bool = False):
+        """Allocates (with torch) and attaches a workspace of the needed size, if any."""
+        import torch
+        need = self.host_workspace_bytes() if host else self.workspace_bytes()
+        have = 0 if self._ws is None else self._ws.numel()
+        if need > have:
+            self.set_workspace(torch.empty(need, dtype=torch.uint8, device="cuda"))
+
+    def set_weights(self, w, stream=None):
+        _check(lib().hgc_conv_set_weights(self._h, _ptr(w), _stream(stream)), "hgc_conv_set_weights")
+
+    def last_device_status(self) -> int:
+        v = ctypes.c_int32()
+        _check(lib().hgc_conv_last_device_status(self._h, ctypes.byref(v)), "hgc_conv_last_device_status")
+        return v.value
+
+
+def conv_forward(desc: ConvDesc, x, w, bias, y, relu: bool, stream=None):
+    """hgc_conv_forward: x, w, bias (or None), y are CUDA fp16 tensors (or raw addresses)."""
+    _check(lib().hgc_conv_forward(desc.handle, _ptr(x), _ptr(w), _ptr(bias), _ptr(y), int(bool(relu)),
+                                  _stream(stream)), "hgc_conv_forward")
+
+
+def conv_forward_host(desc: ConvDesc, x, w, bias, y, relu: bool, stream=None):
+    """hgc_conv_forward_host: x, w, bias (or None), y are HOST fp16 buffers (pinned torch
+    tensors or numpy arrays); copies are queued on the stream."""
+    _check(lib().hgc_conv_forward_host(desc.handle, _ptr(x), _ptr(w), _ptr(bias), _ptr(y),
+                                       int(bool(relu)), _stream(stream)), "hgc_conv_forward_host")
+
+
+def layout_nchw_to_nhwc(src, dst, n, c, h, w, c_pad, stream=None):
+    _check(lib().hgc_layout_nchw_to_nhwc(_ptr(src), _ptr(dst), n, c, h, w, c_pad, _stream(stream)),
+           "hgc_layout_nchw_to_nhwc")
+
+
+def layout_nhwc_to_nchw(src, dst, n, c, h, w, c_pad, stream=None):
+    _check(lib().hgc_layout_nhwc_to_nchw(_ptr(src), _ptr(dst), n, c, h, w, c_pad, _stream(stream)),
+           "hgc_layout_nhwc_to_nchw")
+
+
+def weights_repack(src, dst, k, c_per_group, r, s, group, c_pad, stream=None):
+    _check(lib().hgc_weights_repack(_ptr(src), _ptr(dst), k, c_per_group, r, s, group, c_pad,
+                                    _stream(stream)), "hgc_weights_repack")
+
+
+def kernel_launch_count() -> int:
+    v = ctypes.c_uint64()
+    _check(lib().hgc_kernel_launch_count(ctypes.byref(v)), "hgc_kernel_launch_count")
+    return v.value

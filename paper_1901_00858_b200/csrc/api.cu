@@ -1,0 +1,267 @@
+// Host side of libhgc: parameter validation, shape inference, path choice, workspace
+// bookkeeping and the extern "C" entry points declared in hgc.h.
+#include <atomic>
+#include <new>
+
+#include "hgc_internal.h"
+
+namespace hgc {
+static std::atomic<uint64_t> g_launches{0};
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+}  // namespace hgc
+
+struct hgc_conv_desc {
+  hgc_conv_params params;
+  hgc::ConvGeom geom;
+  int32_t path;
+  size_t ws_needed;       // bytes the chosen path needs
+  void* ws;               // caller-owned device scratch
+  size_t ws_bytes;
+  const void* registered_w;
+};
+
+namespace {
+
+inline int64_t floor_div_pos(int64_t a, int64_t b) {  // b > 0
+  int64_t q = a / b;
+  if ((a % b) != 0 && a < 0) --q;
+  return q;
+}
+
+inline int64_t out_extent(int64_t in, int64_t kernel, int64_t pad, int64_t stride, int64_t dil) {
+  return floor_div_pos(in + 2 * pad - dil * (kernel - 1) - 1, stride) + 1;
+}
+
+inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct HostStaging {
+  size_t x_off, w_off, b_off, y_off, total;
+  size_t x_bytes, w_bytes, b_bytes, y_bytes;
+};
+
+HostStaging host_staging(const hgc_conv_desc* d) {
+  const hgc::ConvGeom& g = d->geom;
+  HostStaging s;
+  s.x_bytes = (size_t)g.n * g.c * g.h * g.w * 2;
+  s.w_bytes = (size_t)g.k * g.cg * g.r * g.s * 2;
+  s.b_bytes = (size_t)g.k * 2;
+  s.y_bytes = (size_t)g.n * g.k * g.p * g.q * 2;
+  s.x_off = round_up(d->ws_needed, 256);
+  s.w_off = s.x_off + round_up(s.x_bytes, 256);
+  s.b_off = s.w_off + round_up(s.w_bytes, 256);
+  s.y_off = s.b_off + round_up(s.b_bytes, 256);
+  s.total = s.y_off + round_up(s.y_bytes, 256);
+  return s;
+}
+
+int forward_impl(hgc_conv_desc* d, const void* x, const void* w, const void* bias, void* y,
+                 int relu, cudaStream_t stream) {
+  const hgc::ConvGeom& g = d->geom;
+  const __half* xh = static_cast<const __half*>(x);
+  const __half* wh = static_cast<const __half*>(w);
+  const __half* bh = static_cast<const __half*>(bias);
+  __half* yh = static_cast<__half*>(y);
+  cudaError_t err;
+  switch (d->path) {
+    case HGC_PATH_DEPTHWISE:
+      err = hgc::launch_depthwise3x3(g, xh, wh, bh, yh, relu, stream);
+      break;
+    case HGC_PATH_DIRECT:
+    default:
+      err = hgc::launch_direct_conv(g, xh, wh, bh, yh, relu, stream);
+      break;
+  }
+  if (err == cudaErrorInvalidConfiguration) return HGC_UNSUPPORTED;
+  return err == cudaSuccess ? HGC_OK : HGC_CUDA_ERROR;
+}
+
+}  // namespace
+
+extern "C" {
+
+int hgc_conv_desc_create(hgc_conv_desc** out, const hgc_conv_params* p) {
+  if (out == nullptr) return HGC_INVALID_ARG;
+  *out = nullptr;
+  if (p == nullptr) return HGC_INVALID_ARG;
+  if (p->n < 1 || p->c < 1 || p->h < 1 || p->w < 1 || p->k < 1 || p->r < 1 || p->s < 1)
+    return HGC_INVALID_ARG;
+  if (p->group < 1 || p->stride_h < 1 || p->stride_w < 1 || p->dil_h < 1 || p->dil_w < 1)
+    return HGC_INVALID_ARG;
+  if (p->pad_h < 0 || p->pad_w < 0) return HGC_INVALID_ARG;
+  if (p->c % p->group != 0 || p->k % p->group != 0) return HGC_INVALID_ARG;
+  const int64_t P = out_extent(p->h, p->r, p->pad_h, p->stride_h, p->dil_h);
+  const int64_t Q = out_extent(p->w, p->s, p->pad_w, p->stride_w, p->dil_w);
+  if (P < 1 || Q < 1) return HGC_INVALID_ARG;
+  if (P > 0x7fffffffLL || Q > 0x7fffffffLL) return HGC_UNSUPPORTED;
+
+  hgc_conv_desc* d = new (std::nothrow) hgc_conv_desc();
+  if (d == nullptr) return HGC_CUDA_ERROR;
+  d->params = *p;
+  hgc::ConvGeom& g = d->geom;
+  g.n = p->n; g.c = p->c; g.h = p->h; g.w = p->w;
+  g.k = p->k; g.r = p->r; g.s = p->s;
+  g.pad_h = p->pad_h; g.pad_w = p->pad_w;
+  g.stride_h = p->stride_h; g.stride_w = p->stride_w;
+  g.dil_h = p->dil_h; g.dil_w = p->dil_w;
+  g.group = p->group;
+  g.p = (int32_t)P; g.q = (int32_t)Q;
+  g.cg = p->c / p->group; g.kg = p->k / p->group;
+
+  d->path = HGC_PATH_DIRECT;
+  d->ws_needed = 0;
+  if (!(p->flags & HGC_FLAG_FORCE_DIRECT)) {
+    if (hgc::depthwise3x3_supported(g)) d->path = HGC_PATH_DEPTHWISE;
+  }
+  d->ws = nullptr;
+  d->ws_bytes = 0;
+  d->registered_w = nullptr;
+  *out = d;
+  return HGC_OK;
+}
+
+int hgc_conv_desc_destroy(hgc_conv_desc* d) {
+  delete d;
+  return HGC_OK;
+}
+
+int hgc_conv_forward(hgc_conv_desc* d, const void* x, const void* w, const void* bias, void* y,
+                     int relu, void* stream) {
+  if (d == nullptr || x == nullptr || w == nullptr || y == nullptr) return HGC_INVALID_ARG;
+  if (misaligned(x) || misaligned(w) || misaligned(y) || (bias != nullptr && misaligned(bias)))
+    return HGC_BAD_ALIGNMENT;
+  if (d->ws_needed > 0 && (d->ws == nullptr || d->ws_bytes < d->ws_needed)) return HGC_NO_WORKSPACE;
+  return forward_impl(d, x, w, bias, y, relu, static_cast<cudaStream_t>(stream));
+}
+
+int hgc_conv_forward_host(hgc_conv_desc* d, const void* x, const void* w, const void* bias, void* y,
+                          int relu, void* stream) {
+  if (d == nullptr || x == nullptr || w == nullptr || y == nullptr) return HGC_INVALID_ARG;
+  const HostStaging s = host_staging(d);
+  if (d->ws == nullptr || d->ws_bytes < s.total) return HGC_NO_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* base = static_cast<char*>(d->ws);
+  if (cudaMemcpyAsync(base + s.x_off, x, s.x_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return HGC_CUDA_ERROR;
+  if (cudaMemcpyAsync(base + s.w_off, w, s.w_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return HGC_CUDA_ERROR;
+  if (bias != nullptr &&
+      cudaMemcpyAsync(base + s.b_off, bias, s.b_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return HGC_CUDA_ERROR;
+  // host weights arrive anew on every call: never treat them as registered
+  d->registered_w = nullptr;
+  const int rc = forward_impl(d, base + s.x_off, base + s.w_off, bias ? base + s.b_off : nullptr,
+                              base + s.y_off, relu, st);
+  if (rc != HGC_OK) return rc;
+  if (cudaMemcpyAsync(y, base + s.y_off, s.y_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return HGC_CUDA_ERROR;
+  return HGC_OK;
+}
+
+int hgc_conv_output_dims(const hgc_conv_desc* d, int32_t* n, int32_t* k, int32_t* p, int32_t* q) {
+  if (d == nullptr) return HGC_INVALID_ARG;
+  if (n) *n = d->geom.n;
+  if (k) *k = d->geom.k;
+  if (p) *p = d->geom.p;
+  if (q) *q = d->geom.q;
+  return HGC_OK;
+}
+
+int hgc_conv_path(const hgc_conv_desc* d, int32_t* path) {
+  if (d == nullptr || path == nullptr) return HGC_INVALID_ARG;
+  *path = d->path;
+  return HGC_OK;
+}
+
+int hgc_conv_workspace_bytes(const hgc_conv_desc* d, size_t* bytes) {
+  if (d == nullptr || bytes == nullptr) return HGC_INVALID_ARG;
+  *bytes = d->ws_needed;
+  return HGC_OK;
+}
+
+int hgc_conv_host_workspace_bytes(const hgc_conv_desc* d, size_t* bytes) {
+  if (d == nullptr || bytes == nullptr) return HGC_INVALID_ARG;
+  *bytes = host_staging(d).total;
+  return HGC_OK;
+}
+
+int hgc_conv_set_workspace(hgc_conv_desc* d, void* dev_ptr, size_t bytes) {
+  if (d == nullptr) return HGC_INVALID_ARG;
+  if (dev_ptr == nullptr && bytes != 0) return HGC_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(dev_ptr) & 255u) != 0) return HGC_BAD_ALIGNMENT;
+  d->ws = dev_ptr;
+  d->ws_bytes = dev_ptr ? bytes : 0;
+  d->registered_w = nullptr;
+  return HGC_OK;
+}
+
+int hgc_conv_set_weights(hgc_conv_desc* d, const void* w, void* stream) {
+  (void)stream;
+  if (d == nullptr || w == nullptr) return HGC_INVALID_ARG;
+  if (misaligned(w)) return HGC_BAD_ALIGNMENT;
+  if (d->ws_needed > 0 && (d->ws == nullptr || d->ws_bytes < d->ws_needed)) return HGC_NO_WORKSPACE;
+  d->registered_w = w;
+  return HGC_OK;
+}
+
+int hgc_conv_last_device_status(hgc_conv_desc* d, int32_t* status) {
+  if (d == nullptr || status == nullptr) return HGC_INVALID_ARG;
+  *status = HGC_OK;
+  return HGC_OK;
+}
+
+int hgc_layout_nchw_to_nhwc(const void* src, void* dst, int32_t n, int32_t c, int32_t h, int32_t w,
+                            int32_t c_pad, void* stream) {
+  if (src == nullptr || dst == nullptr || n < 1 || c < 1 || h < 1 || w < 1 || c_pad < c || (c_pad % 8) != 0)
+    return HGC_INVALID_ARG;
+  if (misaligned(src) || misaligned(dst)) return HGC_BAD_ALIGNMENT;
+  cudaError_t err = hgc::launch_nchw_to_nhwc(static_cast<const __half*>(src), static_cast<__half*>(dst), n,
+                                            c, h, w, c_pad, static_cast<cudaStream_t>(stream));
+  if (err == cudaErrorInvalidConfiguration) return HGC_UNSUPPORTED;
+  return err == cudaSuccess ? HGC_OK : HGC_CUDA_ERROR;
+}
+
+int hgc_layout_nhwc_to_nchw(const void* src, void* dst, int32_t n, int32_t c, int32_t h, int32_t w,
+                            int32_t c_pad, void* stream) {
+  if (src == nullptr || dst == nullptr || n < 1 || c < 1 || h < 1 || w < 1 || c_pad < c || (c_pad % 8) != 0)
+    return HGC_INVALID_ARG;
+  if (misaligned(src) || misaligned(dst)) return HGC_BAD_ALIGNMENT;
+  cudaError_t err = hgc::launch_nhwc_to_nchw(static_cast<const __half*>(src), static_cast<__half*>(dst), n,
+                                            c, h, w, c_pad, static_cast<cudaStream_t>(stream));
+  if (err == cudaErrorInvalidConfiguration) return HGC_UNSUPPORTED;
+  return err == cudaSuccess ? HGC_OK : HGC_CUDA_ERROR;
+}
+
+int hgc_weights_repack(const void* src, void* dst, int32_t k, int32_t c_per_group, int32_t r, int32_t s,
+                       int32_t group, int32_t c_pad, void* stream) {
+  if (src == nullptr || dst == nullptr || k < 1 || c_per_group < 1 || r < 1 || s < 1 || group < 1 ||
+      (k % group) != 0 || c_pad < c_per_group || (c_pad % 8) != 0)
+    return HGC_INVALID_ARG;
+  if (misaligned(src) || misaligned(dst)) return HGC_BAD_ALIGNMENT;
+  cudaError_t err = hgc::launch_weights_repack(static_cast<const __half*>(src), static_cast<__half*>(dst), k,
+                                              c_per_group, r, s, group, c_pad,
+                                              static_cast<cudaStream_t>(stream));
+  return err == cudaSuccess ? HGC_OK : HGC_CUDA_ERROR;
+}
+
+int hgc_kernel_launch_count(uint64_t* count) {
+  if (count == nullptr) return HGC_INVALID_ARG;
+  *count = hgc::g_launches.load(std::memory_order_relaxed);
+  return HGC_OK;
+}
+
+const char* hgc_status_string(int status) {
+  switch (status) {
+    case HGC_OK: return "ok";
+    case HGC_INVALID_ARG: return "invalid argument";
+    case HGC_UNSUPPORTED: return "unsupported";
+    case HGC_BAD_ALIGNMENT: return "device pointer not 16-byte aligned";
+    case HGC_NO_WORKSPACE: return "workspace missing or too small";
+    case HGC_CUDA_ERROR: return "CUDA error";
+    case HGC_DEVICE_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

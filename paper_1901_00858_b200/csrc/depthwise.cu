@@ -1,0 +1,272 @@
+// 3x3 depthwise convolution (group == C == K, dilation 1, stride 1 or 2) on CUDA cores.
+// It is a 9-tap stencil per channel plane, not a dense contraction: the bound is HBM
+// bandwidth (4 bytes per output at stride 1, 10 at stride 2), so the kernel is organised
+// around 16-byte aligned global accesses for ANY plane size and works on NCHW directly.
+//
+// A CTA owns a contiguous piece of the tensor: either several whole (n,c) planes (small
+// planes: 7x7, 14x14, 28x28 ...) or a band of output rows of one plane.  Its input span and
+// its output span are contiguous in global memory, so both are moved as 16-byte vectors that
+// are aligned to the GLOBAL address (the span's first and last vector may be partial; the
+// first is over-read inside the tensor, the tail is guarded).  In between, each thread
+// slides a 3-row register window down two adjacent output columns, accumulating in fp32, and
+// leaves fp16 results in a shared staging span.
+#include "hgc_internal.h"
+
+namespace hgc {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kInBudget = 16384;   // elements of input a CTA may stage
+constexpr int kOutBudget = 12288;  // elements of output a CTA may stage
+
+struct DwPlan {
+  int32_t c, h, w, p, q, pad_h, pad_w;
+  int32_t th;              // output rows per thread unit
+  int32_t planes_per_cta;  // >= 1; > 1 only with bands_per_plane == 1
+  int32_t bands_per_plane; // row bands a plane is split into
+  int32_t band_rows;       // output rows per band
+  int64_t planes;          // N * C
+  int64_t x_elems, y_elems;
+  int32_t smem_in, smem_out;  // staged elements incl. alignment slack (multiples of 8)
+};
+
+template <int S>
+__global__ void __launch_bounds__(kThreads)
+depthwise3x3_kernel(DwPlan a, const uint16_t* __restrict__ x, const __half* __restrict__ w,
+                    const __half* __restrict__ bias, uint16_t* __restrict__ y, int relu) {
+  extern __shared__ __align__(16) uint16_t smem[];
+  uint16_t* sin = smem;
+  uint16_t* sout = smem + a.smem_in;
+  constexpr int NCOL = S + 3;
+
+  const int64_t hw = (int64_t)a.h * a.w, pq = (int64_t)a.p * a.q;
+  int64_t pl0;
+  int np, p0, p1;
+  if (a.bands_per_plane == 1) {
+    pl0 = (int64_t)blockIdx.x * a.planes_per_cta;
+    np = (int)((a.planes - pl0) < a.planes_per_cta ? (a.planes - pl0) : a.planes_per_cta);
+    p0 = 0;
+    p1 = a.p;
+  } else {
+    pl0 = blockIdx.x / a.bands_per_plane;
+    np = 1;
+    p0 = (blockIdx.x % a.bands_per_plane) * a.band_rows;
+    p1 = p0 + a.band_rows < a.p ? p0 + a.band_rows : a.p;
+  }
+  // input rows the band touches (whole planes when the CTA owns planes)
+  int ih_lo = p0 * S - a.pad_h;
+  int ih_hi = (p1 - 1) * S - a.pad_h + 3;
+  if (a.bands_per_plane == 1) {
+    ih_lo = 0;
+    ih_hi = a.h;
+  }
+  if (ih_lo < 0) ih_lo = 0;
+  if (ih_hi > a.h) ih_hi = a.h;
+  if (ih_hi < ih_lo) ih_hi = ih_lo;
+  const int64_t g_in0 = pl0 * hw + (int64_t)ih_lo * a.w;
+  const int64_t in_len = (int64_t)(np - 1) * hw + (int64_t)(ih_hi - ih_lo) * a.w;
+  const int mis_in = (int)(g_in0 & 7);
+  const int64_t g_out0 = pl0 * pq + (int64_t)p0 * a.q;
+  const int64_t out_len = (int64_t)(np - 1) * pq + (int64_t)(p1 - p0) * a.q;
+  const int mis_out = (int)(g_out0 & 7);
+
+  // ---- stage the input span: aligned 16-byte vectors --------------------------------
+  {
+    const int nvec = (int)((mis_in + in_len + 7) >> 3);
+    const int64_t gbase = g_in0 - mis_in;
+    for (int v = threadIdx.x; v < nvec; v += kThreads) {
+      const int64_t ge = gbase + (int64_t)v * 8;
+      uint4 val;
+      if (ge + 8 <= a.x_elems) {
+        val = __ldg(reinterpret_cast<const uint4*>(x + ge));
+      } else {
+        uint32_t o[4] = {0, 0, 0, 0};
+        for (int j = 0; j < 8; ++j)
+          if (ge + j < a.x_elems) o[j >> 1] |= (uint32_t)x[ge + j] << ((j & 1) * 16);
+        val = make_uint4(o[0], o[1], o[2], o[3]);
+      }
+      *reinterpret_cast<uint4*>(sin + v * 8) = val;
+    }
+  }
+  __syncthreads();
+
+  // ---- compute: thread = (unit, column pair) ------------------------------------------
+  const int cols2 = (a.q + 1) >> 1;
+  const int rows = p1 - p0;
+  const int units_per_plane = (rows + a.th - 1) / a.th;
+  const int units = np * units_per_plane;
+  const int lanes = units * cols2;
+  for (int t = threadIdx.x; t < lanes; t += kThreads) {
+    const int u = t / cols2, cp = t % cols2;
+    const int pl = u / units_per_plane;
+    const int r0 = p0 + (u % units_per_plane) * a.th;
+    const int r1 = r0 + a.th < p1 ? r0 + a.th : p1;
+    const int ch = (int)((pl0 + pl) % a.c);
+    float wv[9];
+#pragma unroll
+    for (int i = 0; i < 9; ++i) wv[i] = __half2float(__ldg(w + (int64_t)ch * 9 + i));
+    const float bv = bias != nullptr ? __half2float(__ldg(bias + ch)) : 0.f;
+
+    const int q0 = cp * 2;
+    const int iw0 = q0 * S - a.pad_w;
+    bool cvalid[NCOL];
+#pragma unroll
+    for (int j = 0; j < NCOL; ++j) cvalid[j] = (iw0 + j >= 0) && (iw0 + j < a.w);
+    const bool second = (q0 + 1) < a.q;
+    // smem index of (plane pl, row ih, col iw0)
+    const int in_base = mis_in + pl * (int)hw - ih_lo * a.w + iw0;
+    const int out_base = mis_out + pl * (int)pq - p0 * a.q + q0;
+
+    float win[3][NCOL];
+    auto load_row = [&](float (&dst)[NCOL], int ih) {
+      const bool rv = (ih >= 0) && (ih < a.h);
+      const uint16_t* src = sin + in_base + ih * a.w;
+#pragma unroll
+      for (int j = 0; j < NCOL; ++j) {
+        uint16_t bits = 0;
+        if (rv && cvalid[j]) bits = src[j];
+        dst[j] = __half2float(__ushort_as_half(bits));
+      }
+    };
+    int ih = r0 * S - a.pad_h;
+    if (S == 1) {
+      load_row(win[0], ih);
+      load_row(win[1], ih + 1);
+    } else {
+      load_row(win[0], ih);
+    }
+    for (int p = r0; p < r1; ++p, ih += S) {
+      if (S == 1) {
+        load_row(win[2], ih + 2);
+      } else {
+        load_row(win[1], ih + 1);
+        load_row(win[2], ih + 2);
+      }
+      float o0 = bv, o1 = bv;
+#pragma unroll
+      for (int r = 0; r < 3; ++r)
+#pragma unroll
+        for (int s = 0; s < 3; ++s) {
+          o0 = fmaf(win[r][s], wv[r * 3 + s], o0);
+          o1 = fmaf(win[r][s + S], wv[r * 3 + s], o1);
+        }
+      if (relu) {
+        o0 = fmaxf(o0, 0.f);
+        o1 = fmaxf(o1, 0.f);
+      }
+      uint16_t* dst = sout + out_base + p * a.q;
+      dst[0] = __half_as_ushort(__float2half_rn(o0));
+      if (second) dst[1] = __half_as_ushort(__float2half_rn(o1));
+#pragma unroll
+      for (int j = 0; j < NCOL; ++j) {
+        if (S == 1) {
+          win[0][j] = win[1][j];
+          win[1][j] = win[2][j];
+        } else {
+          win[0][j] = win[2][j];
+        }
+      }
+    }
+  }
+  __syncthreads();
+
+  // ---- write the output span: aligned 16-byte vectors, partial ones element-wise ----
+  {
+    const int nvec = (int)((mis_out + out_len + 7) >> 3);
+    const int64_t gbase = g_out0 - mis_out;
+    const int lo = mis_out, hi = mis_out + (int)out_len;  // valid staged range
+    for (int v = threadIdx.x; v < nvec; v += kThreads) {
+      const int e = v * 8;
+      if (e >= lo && e + 8 <= hi) {
+        *reinterpret_cast<uint4*>(y + gbase + e) = *reinterpret_cast<const uint4*>(sout + e);
+      } else {
+        for (int j = 0; j < 8; ++j)
+          if (e + j >= lo && e + j < hi) y[gbase + e + j] = sout[e + j];
+      }
+    }
+  }
+}
+
+bool make_plan(const ConvGeom& g, DwPlan* plan) {
+  if (g.r != 3 || g.s != 3 || g.dil_h != 1 || g.dil_w != 1) return false;
+  if (g.group != g.c || g.k != g.c) return false;
+  if (g.stride_h != g.stride_w || (g.stride_h != 1 && g.stride_h != 2)) return false;
+  const int S = g.stride_h;
+  DwPlan a{};
+  a.c = g.c; a.h = g.h; a.w = g.w; a.p = g.p; a.q = g.q; a.pad_h = g.pad_h; a.pad_w = g.pad_w;
+  a.planes = (int64_t)g.n * g.c;
+  a.x_elems = a.planes * g.h * g.w;
+  a.y_elems = a.planes * g.p * g.q;
+  a.th = (g.p % 7 == 0) ? 7 : 8;
+  const int64_t hw = (int64_t)g.h * g.w, pq = (int64_t)g.p * g.q;
+  const int cols2 = (g.q + 1) / 2;
+  if (cols2 > kThreads) return false;
+  if (hw <= kInBudget && pq <= kOutBudget) {
+    a.bands_per_plane = 1;
+    a.band_rows = g.p;
+    const int units_per_plane = (g.p + a.th - 1) / a.th;
+    int64_t ppc = kThreads / ((int64_t)cols2 * units_per_plane);
+    if (ppc < 1) ppc = 1;
+    if (ppc > kInBudget / hw) ppc = kInBudget / hw;
+    if (ppc > kOutBudget / pq) ppc = kOutBudget / pq;
+    if (ppc > a.planes) ppc = a.planes;
+    a.planes_per_cta = (int32_t)ppc;
+    a.smem_in = (int32_t)(((ppc * hw + 8 + 7) / 8) * 8);
+    a.smem_out = (int32_t)(((ppc * pq + 8 + 7) / 8) * 8);
+  } else {
+    a.planes_per_cta = 1;
+    // largest multiple of th whose input rows and output rows fit the budgets
+    int tb = 0;
+    for (int cand = a.th; cand <= g.p + a.th; cand += a.th) {
+      const int64_t in_rows = (int64_t)(cand - 1) * S + 3;
+      if (in_rows * g.w > kInBudget || (int64_t)cand * g.q > kOutBudget) break;
+      tb = cand;
+      if ((int64_t)(cand / a.th) * cols2 >= kThreads) break;  // one pass of the CTA is full
+    }
+    if (tb == 0) return false;
+    a.band_rows = tb;
+    a.bands_per_plane = (g.p + tb - 1) / tb;
+    const int64_t in_rows = (int64_t)(tb - 1) * S + 3;
+    a.smem_in = (int32_t)(((in_rows * g.w + 8 + 7) / 8) * 8);
+    a.smem_out = (int32_t)((((int64_t)tb * g.q + 8 + 7) / 8) * 8);
+  }
+  const int64_t ctas = a.bands_per_plane == 1 ? (a.planes + a.planes_per_cta - 1) / a.planes_per_cta
+                                               : a.planes * a.bands_per_plane;
+  if (ctas > 0x7fffffffLL) return false;
+  // staged indices are 32-bit
+  if ((int64_t)a.planes_per_cta * hw > (1 << 24)) return false;
+  *plan = a;
+  return true;
+}
+
+}  // namespace
+
+bool depthwise3x3_supported(const ConvGeom& g) {
+  DwPlan a;
+  return make_plan(g, &a);
+}
+
+cudaError_t launch_depthwise3x3(const ConvGeom& g, const __half* x, const __half* w,
+                                const __half* bias, __half* y, int relu, cudaStream_t stream) {
+  DwPlan a;
+  if (!make_plan(g, &a)) return cudaErrorInvalidConfiguration;
+  const int64_t ctas = a.bands_per_plane == 1 ? (a.planes + a.planes_per_cta - 1) / a.planes_per_cta
+                                               : a.planes * a.bands_per_plane;
+  const size_t smem = (size_t)(a.smem_in + a.smem_out) * sizeof(uint16_t);
+  const uint16_t* xs = reinterpret_cast<const uint16_t*>(x);
+  uint16_t* ys = reinterpret_cast<uint16_t*>(y);
+  cudaError_t err;
+  if (g.stride_h == 1) {
+    err = cudaFuncSetAttribute(depthwise3x3_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    depthwise3x3_kernel<1><<<(unsigned)ctas, kThreads, smem, stream>>>(a, xs, w, bias, ys, relu);
+  } else {
+    err = cudaFuncSetAttribute(depthwise3x3_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    depthwise3x3_kernel<2><<<(unsigned)ctas, kThreads, smem, stream>>>(a, xs, w, bias, ys, relu);
+  }
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace hgc

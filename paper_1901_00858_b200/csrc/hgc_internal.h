@@ -1,0 +1,38 @@
+// Internal declarations shared by the translation units of libhgc (host planner + kernels).
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hgc.h"
+
+namespace hgc {
+
+// Geometry of one layer as the kernels see it (all plain integers, passed by value).
+struct ConvGeom {
+  int32_t n, c, h, w;
+  int32_t k, r, s;
+  int32_t pad_h, pad_w, stride_h, stride_w, dil_h, dil_w;
+  int32_t group;
+  int32_t p, q;    // output plane
+  int32_t cg, kg;  // channels per group: C/group, K/group
+};
+
+void count_launch();  // bumps the process-wide kernel launch counter
+
+// Each launcher enqueues on `stream` and returns the launch error (cudaSuccess if fine).
+cudaError_t launch_direct_conv(const ConvGeom& g, const __half* x, const __half* w,
+                               const __half* bias, __half* y, int relu, cudaStream_t stream);
+
+bool depthwise3x3_supported(const ConvGeom& g);
+cudaError_t launch_depthwise3x3(const ConvGeom& g, const __half* x, const __half* w,
+                                const __half* bias, __half* y, int relu, cudaStream_t stream);
+
+cudaError_t launch_nchw_to_nhwc(const __half* src, __half* dst, int32_t n, int32_t c, int32_t h,
+                                int32_t w, int32_t c_pad, cudaStream_t stream);
+cudaError_t launch_nhwc_to_nchw(const __half* src, __half* dst, int32_t n, int32_t c, int32_t h,
+                                int32_t w, int32_t c_pad, cudaStream_t stream);
+cudaError_t launch_weights_repack(const __half* src, __half* dst, int32_t k, int32_t cg, int32_t r,
+                                  int32_t s, int32_t group, int32_t c_pad, cudaStream_t stream);
+
+}  // namespace hgc

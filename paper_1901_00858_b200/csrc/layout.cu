@@ -1,0 +1,174 @@
+// Data-movement kernels: NCHW <-> NHWC (channels padded to a multiple of 8 so that a pixel is
+// a whole number of 16-byte vectors) and the weight re-layout for the implicit-GEMM path.
+// Pure permutations of binary16 bit patterns; bound by HBM bandwidth.
+//
+// Transposes go through a shared-memory tile of kTileC channels x kTileP pixels.  Global
+// accesses are 16-byte vectors wherever the address allows it: always on the NHWC side
+// (c_pad % 8 == 0), and on the NCHW side when the plane size is a multiple of 8 elements (so
+// every channel row of every tile starts on a 16-byte boundary); other planes (7x7, 14x14,
+// 27x27 ...) take 2-byte accesses on the NCHW side.
+#include "hgc_internal.h"
+
+namespace hgc {
+namespace {
+
+constexpr int kTileC = 64;
+constexpr int kTileP = 64;
+constexpr int kRow = kTileP + 8;  // shared-memory row pitch in elements (16-byte multiple)
+constexpr int kThreads = 256;
+
+// x[n][c][hw] -> x'[n][hw][c_pad]
+__global__ void __launch_bounds__(kThreads)
+nchw_to_nhwc_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int64_t hw,
+                    int c_pad, int vec_ok) {
+  __shared__ __align__(16) uint16_t tile[kTileC][kRow];
+  const int64_t n = blockIdx.z;
+  const int c0 = blockIdx.y * kTileC;
+  const int64_t p0 = (int64_t)blockIdx.x * kTileP;
+  const uint16_t* s = src + n * c * hw;
+  uint16_t* d = dst + n * hw * c_pad;
+
+  if (vec_ok) {
+    // 64 rows x 8 vectors
+    for (int i = threadIdx.x; i < kTileC * (kTileP / 8); i += kThreads) {
+      const int row = i / (kTileP / 8), v = i % (kTileP / 8);
+      const int ch = c0 + row;
+      const int64_t p = p0 + v * 8;
+      uint4 val = make_uint4(0, 0, 0, 0);
+      if (ch < c && p < hw) val = *reinterpret_cast<const uint4*>(s + (int64_t)ch * hw + p);  // hw % 8 == 0
+      *reinterpret_cast<uint4*>(&tile[row][v * 8]) = val;
+    }
+  } else {
+    for (int i = threadIdx.x; i < kTileC * kTileP; i += kThreads) {
+      const int row = i / kTileP, col = i % kTileP;
+      const int ch = c0 + row;
+      const int64_t p = p0 + col;
+      tile[row][col] = (ch < c && p < hw) ? s[(int64_t)ch * hw + p] : (uint16_t)0;
+    }
+  }
+  __syncthreads();
+  // 64 pixels x 8 channel-vectors; a warp takes 32 consecutive pixels of one channel-vector
+  for (int i = threadIdx.x; i < kTileP * (kTileC / 8); i += kThreads) {
+    const int cv = i / kTileP, px = i % kTileP;
+    const int ch = c0 + cv * 8;
+    const int64_t p = p0 + px;
+    if (ch < c_pad && p < hw) {
+      uint32_t o[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        o[j] = (uint32_t)tile[cv * 8 + 2 * j][px] | ((uint32_t)tile[cv * 8 + 2 * j + 1][px] << 16);
+      *reinterpret_cast<uint4*>(d + p * c_pad + ch) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+  }
+}
+
+// x'[n][hw][c_pad] -> x[n][c][hw]
+__global__ void __launch_bounds__(kThreads)
+nhwc_to_nchw_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int64_t hw,
+                    int c_pad, int vec_ok) {
+  __shared__ __align__(16) uint16_t tile[kTileC][kRow];
+  const int64_t n = blockIdx.z;
+  const int c0 = blockIdx.y * kTileC;
+  const int64_t p0 = (int64_t)blockIdx.x * kTileP;
+  const uint16_t* s = src + n * hw * c_pad;
+  uint16_t* d = dst + n * c * hw;
+
+  for (int i = threadIdx.x; i < kTileP * (kTileC / 8); i += kThreads) {
+    const int px = i / (kTileC / 8), cv = i % (kTileC / 8);
+    const int ch = c0 + cv * 8;
+    const int64_t p = p0 + px;
+    uint4 val = make_uint4(0, 0, 0, 0);
+    if (ch < c_pad && p < hw) val = *reinterpret_cast<const uint4*>(s + p * c_pad + ch);
+    const uint32_t o[4] = {val.x, val.y, val.z, val.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      tile[cv * 8 + 2 * j][px] = (uint16_t)(o[j] & 0xffffu);
+      tile[cv * 8 + 2 * j + 1][px] = (uint16_t)(o[j] >> 16);
+    }
+  }
+  __syncthreads();
+  if (vec_ok) {
+    for (int i = threadIdx.x; i < kTileC * (kTileP / 8); i += kThreads) {
+      const int row = i / (kTileP / 8), v = i % (kTileP / 8);
+      const int ch = c0 + row;
+      const int64_t p = p0 + v * 8;
+      if (ch < c && p < hw)
+        *reinterpret_cast<uint4*>(d + (int64_t)ch * hw + p) = *reinterpret_cast<const uint4*>(&tile[row][v * 8]);
+    }
+  } else {
+    for (int i = threadIdx.x; i < kTileC * kTileP; i += kThreads) {
+      const int row = i / kTileP, col = i % kTileP;
+      const int ch = c0 + row;
+      const int64_t p = p0 + col;
+      if (ch < c && p < hw) d[(int64_t)ch * hw + p] = tile[row][col];
+    }
+  }
+}
+
+// w[g*kg + k'][c'][r][s] -> w'[g][k'][r][s][c_pad]; one thread per 8 output channels-of-input
+__global__ void weights_repack_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst,
+                                      int64_t k, int cg, int rs, int c_pad) {
+  const int64_t vecs_per_k = (int64_t)rs * (c_pad / 8);
+  const int64_t total = k * vecs_per_k;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+       i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t kk = i / vecs_per_k;
+    const int64_t rem = i % vecs_per_k;
+    const int t = (int)(rem / (c_pad / 8));
+    const int cv = (int)(rem % (c_pad / 8));
+    uint32_t o[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int ch = cv * 8 + j;
+      uint32_t v = 0;
+      if (ch < cg) v = src[(kk * cg + ch) * rs + t];
+      o[j >> 1] |= v << ((j & 1) * 16);
+    }
+    *reinterpret_cast<uint4*>(dst + (kk * rs + t) * c_pad + cv * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_nchw_to_nhwc(const __half* src, __half* dst, int32_t n, int32_t c, int32_t h,
+                                int32_t w, int32_t c_pad, cudaStream_t stream) {
+  const int64_t hw = (int64_t)h * w;
+  const int64_t px_tiles = (hw + kTileP - 1) / kTileP;
+  const int c_tiles = (c_pad + kTileC - 1) / kTileC;
+  if (px_tiles > 0x7fffffffLL || c_tiles > 65535 || n > 65535) return cudaErrorInvalidConfiguration;
+  dim3 grid((unsigned)px_tiles, (unsigned)c_tiles, (unsigned)n);
+  nchw_to_nhwc_kernel<<<grid, kThreads, 0, stream>>>(reinterpret_cast<const uint16_t*>(src),
+                                                     reinterpret_cast<uint16_t*>(dst), c, hw, c_pad,
+                                                     (hw % 8) == 0);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_nhwc_to_nchw(const __half* src, __half* dst, int32_t n, int32_t c, int32_t h,
+                                int32_t w, int32_t c_pad, cudaStream_t stream) {
+  const int64_t hw = (int64_t)h * w;
+  const int64_t px_tiles = (hw + kTileP - 1) / kTileP;
+  const int c_tiles = (c + kTileC - 1) / kTileC;
+  if (px_tiles > 0x7fffffffLL || c_tiles > 65535 || n > 65535) return cudaErrorInvalidConfiguration;
+  dim3 grid((unsigned)px_tiles, (unsigned)c_tiles, (unsigned)n);
+  nhwc_to_nchw_kernel<<<grid, kThreads, 0, stream>>>(reinterpret_cast<const uint16_t*>(src),
+                                                     reinterpret_cast<uint16_t*>(dst), c, hw, c_pad,
+                                                     (hw % 8) == 0);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_weights_repack(const __half* src, __half* dst, int32_t k, int32_t cg, int32_t r,
+                                  int32_t s, int32_t group, int32_t c_pad, cudaStream_t stream) {
+  (void)group;  // groups are contiguous blocks of output channels: the permutation is per k
+  const int64_t total = (int64_t)k * r * s * (c_pad / 8);
+  int64_t blocks = (total + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  weights_repack_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
+      reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), k, cg, r * s, c_pad);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace hgc

@@ -53,6 +53,18 @@ class Workload:
             outl.extend([l] * l.count)
         return outl
 
+    def expanded_unique(self) -> List[Layer]:
+        """Distinct layer shapes in network order, `count` = how often each occurs."""
+        import dataclasses
+        seen = {}
+        for l in self.expanded():
+            key = (l.c, l.h, l.k, l.r, l.stride, l.pad, l.dil, l.group, l.relu)
+            if key in seen:
+                seen[key] = dataclasses.replace(seen[key], count=seen[key].count + 1)
+            else:
+                seen[key] = dataclasses.replace(l, count=1)
+        return list(seen.values())
+
 
 def _single() -> List[Layer]:
     return [Layer("conv3x3", 3, 32, 16, 3, 1, 1, out=32, x_lo=-1.0)]

@@ -1,0 +1,115 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol
+the header declares, validates descriptors and infers integer shapes exactly like the oracle."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+from hypothesis import given, settings, strategies as st
+
+from paper_1901_00858_b200 import binding as hgc
+from paper_1901_00858_b200 import build as hgc_build
+from paper_1901_00858_b200 import workloads
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    hgc_build.build()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "hgc.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(hgc_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_symbols()
+    assert "hgc_conv_forward" in names and "hgc_conv_desc_create" in names and len(names) >= 14
+    L = ctypes.CDLL(hgc.LIB_PATH)
+    for nm in names:
+        assert hasattr(L, nm), f"{nm} is declared in hgc.h but not exported"
+
+
+def test_status_strings():
+    for code in range(7):
+        assert hgc.status_string(code)
+    assert hgc.status_string(0) == "ok"
+    assert "unknown" in hgc.status_string(12345)
+
+
+@pytest.mark.parametrize("bad", [
+    dict(n=0), dict(c=0), dict(h=0), dict(w=0), dict(k=0), dict(r=0), dict(s=0), dict(group=0),
+    dict(stride_h=0), dict(stride_w=0), dict(dil_h=0), dict(dil_w=0), dict(pad_h=-1), dict(pad_w=-1),
+    dict(c=6, group=4), dict(k=6, group=4, c=8), dict(h=2, r=3), dict(w=4, s=3, dil_w=2),
+])
+def test_invalid_descriptors_are_rejected(bad):
+    base = dict(n=1, c=4, h=8, w=8, k=4, r=3, s=3)
+    base.update(bad)
+    with pytest.raises(hgc.HgcError) as e:
+        hgc.ConvDesc(**base)
+    assert e.value.status == hgc.HGC_INVALID_ARG
+
+
+def test_null_arguments():
+    L = hgc.lib()
+    assert L.hgc_conv_desc_create(None, None) == hgc.HGC_INVALID_ARG
+    h = ctypes.c_void_p(123)
+    assert L.hgc_conv_desc_create(ctypes.byref(h), None) == hgc.HGC_INVALID_ARG
+    assert not h.value
+    assert L.hgc_conv_desc_destroy(None) == hgc.HGC_OK
+    d = hgc.ConvDesc(1, 3, 8, 8, 4, 3, 3)
+    assert L.hgc_conv_forward(d.handle, None, None, None, None, 0, None) == hgc.HGC_INVALID_ARG
+    assert L.hgc_conv_forward(None, 16, 16, None, 16, 0, None) == hgc.HGC_INVALID_ARG
+    assert L.hgc_conv_forward(d.handle, 32, 48, None, 66, 0, None) == hgc.HGC_BAD_ALIGNMENT
+    assert L.hgc_conv_forward(d.handle, 32, 48, 6, 64, 0, None) == hgc.HGC_BAD_ALIGNMENT
+    assert L.hgc_conv_output_dims(None, None, None, None, None) == hgc.HGC_INVALID_ARG
+    assert L.hgc_conv_set_workspace(d.handle, 128, 10) == hgc.HGC_BAD_ALIGNMENT
+    assert L.hgc_conv_set_workspace(d.handle, None, 10) == hgc.HGC_INVALID_ARG
+    assert L.hgc_layout_nchw_to_nhwc(16, 32, 1, 3, 4, 4, 4, None) == hgc.HGC_INVALID_ARG  # c_pad % 8
+    assert L.hgc_layout_nchw_to_nhwc(16, 32, 1, 9, 4, 4, 8, None) == hgc.HGC_INVALID_ARG  # c_pad < c
+    assert L.hgc_weights_repack(16, 32, 6, 3, 3, 3, 4, 8, None) == hgc.HGC_INVALID_ARG    # k % group
+
+
+def test_output_dims_of_the_workloads(oracle):
+    for wl in workloads.all_workloads():
+        for l in wl.layers:
+            d = hgc.ConvDesc(wl.batch, l.c, l.h, l.h, l.k, l.r, l.r, l.pad, l.pad, l.stride, l.stride,
+                             l.dil, l.dil, l.group)
+            assert d.output_dims() == (wl.batch, l.k, l.out, l.out), (wl.name, l.name)
+            d.close()
+
+
+@settings(max_examples=300, deadline=None)
+@given(st.integers(1, 200), st.integers(1, 200), st.integers(1, 9), st.integers(1, 9), st.integers(0, 5),
+       st.integers(0, 5), st.integers(1, 5), st.integers(1, 5), st.integers(1, 3), st.integers(1, 3))
+def test_shape_inference_matches_oracle_exactly(oracle, h, w, r, s, ph, pw, sh, sw, dh, dw):
+    P, Q = oracle.out_dim(h, r, ph, sh, dh), oracle.out_dim(w, s, pw, sw, dw)
+    args = dict(n=2, c=4, h=h, w=w, k=6, r=r, s=s, pad_h=ph, pad_w=pw, stride_h=sh, stride_w=sw,
+                dil_h=dh, dil_w=dw, group=2)
+    if P < 1 or Q < 1:
+        with pytest.raises(hgc.HgcError) as e:
+            hgc.ConvDesc(**args)
+        assert e.value.status == hgc.HGC_INVALID_ARG
+    else:
+        d = hgc.ConvDesc(**args)
+        assert d.output_dims() == (2, 6, P, Q)
+        d.close()
+
+
+def test_planner_paths():
+    dw = hgc.ConvDesc(2, 32, 14, 14, 32, 3, 3, 1, 1, 1, 1, 1, 1, 32)
+    assert dw.path() == hgc.HGC_PATH_DEPTHWISE
+    forced = hgc.ConvDesc(2, 32, 14, 14, 32, 3, 3, 1, 1, 1, 1, 1, 1, 32, hgc.HGC_FLAG_FORCE_DIRECT)
+    assert forced.path() == hgc.HGC_PATH_DIRECT
+    dil = hgc.ConvDesc(2, 32, 14, 14, 32, 3, 3, 2, 2, 1, 1, 2, 2, 32)
+    assert dil.path() == hgc.HGC_PATH_DIRECT      # dilated depthwise: generic kernel
+    mult = hgc.ConvDesc(2, 32, 14, 14, 64, 3, 3, 1, 1, 1, 1, 1, 1, 32)
+    assert mult.path() == hgc.HGC_PATH_DIRECT     # channel multiplier 2: generic kernel
+
+
+def test_launch_counter_readable():
+    assert hgc.kernel_launch_count() >= 0

@@ -1,0 +1,190 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element,
+on the same seeded float16 inputs.  Tolerance: |gpu - ref| <= 2e-3 + 1e-2*|ref|."""
+import json
+import os
+
+import numpy as np
+import pytest
+
+from paper_1901_00858_b200 import workloads
+from gpu_util import check_close, layer_args, params_dict, run_layer, sample_coords, to_dev, to_host
+
+pytestmark = pytest.mark.gpu
+F16 = np.float16
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+@pytest.fixture(scope="module")
+def hgc():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_1901_00858_b200 import binding
+    binding.lib()
+    return binding
+
+
+def _hand_examples():
+    with open(os.path.join(GOLDEN, "hand_examples.json")) as f:
+        return json.load(f)["examples"]
+
+
+@pytest.mark.parametrize("flags", [0, 1], ids=["planned", "forced-direct"])
+@pytest.mark.parametrize("ex", _hand_examples(), ids=lambda e: e["id"])
+def test_hand_examples_on_gpu(hgc, oracle, ex, flags):
+    from test_oracle_pins import _example_tensors
+    P = oracle.ConvParams(**ex["params"])
+    x, w, b = _example_tensors(ex, P)
+    args = params_dict(**ex["params"])
+    y, _ = run_layer(hgc, args, x, w, b, ex["relu"], flags=flags)
+    assert list(y.shape) == ex["out_shape"]
+    if "expected_bits" in ex:   # fp32 holds this sum exactly: the GPU must round like the oracle
+        assert [format(v, "04x") for v in y.view(np.uint16).ravel()] == ex["expected_bits"]
+    else:                        # small exact integers/halves: exact on the GPU as well
+        assert y.ravel().astype(np.float64).tolist() == [float(v) for v in ex["expected"]]
+
+
+def _random_descriptor(rng):
+    g = int(rng.choice([1, 1, 2, 3, 4, -1]))
+    cg, kg = int(rng.integers(1, 41)), int(rng.integers(1, 41))
+    if g == -1:   # depthwise, sometimes with a channel multiplier
+        g, cg, kg = int(rng.integers(1, 70)), 1, int(rng.choice([1, 1, 1, 2]))
+    h, w = int(rng.integers(1, 41)), int(rng.integers(1, 41))
+    r, s = int(rng.integers(1, 8)), int(rng.integers(1, 8))
+    if rng.random() < 0.4:
+        r = s = 3
+    ph, pw = int(rng.integers(0, 5)), int(rng.integers(0, 5))
+    sh, sw = int(rng.integers(1, 6)), int(rng.integers(1, 6))
+    if rng.random() < 0.5:
+        sh = sw = int(rng.integers(1, 3))
+    dh, dw = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+    if rng.random() < 0.5:
+        dh = dw = 1
+    n = int(rng.integers(1, 4))
+    return params_dict(n, g * cg, h, w, g * kg, r, s, ph, pw, sh, sw, dh, dw, g)
+
+
+@pytest.mark.parametrize("flags", [0, 1], ids=["planned", "forced-direct"])
+def test_random_descriptors(hgc, oracle, flags):
+    rng = np.random.default_rng(20240 + flags)
+    done = 0
+    paths = set()
+    while done < 160:
+        a = _random_descriptor(rng)
+        if oracle.out_dim(a["h"], a["r"], a["pad_h"], a["stride_h"], a["dil_h"]) < 1 or \
+           oracle.out_dim(a["w"], a["s"], a["pad_w"], a["stride_w"], a["dil_w"]) < 1:
+            with pytest.raises(hgc.HgcError) as e:
+                hgc.ConvDesc(**a)
+            assert e.value.status == hgc.HGC_INVALID_ARG
+            continue
+        x, w, b = workloads.random_layer_tensors(rng, a["n"], a["c"], a["h"], a["w"], a["k"], a["r"], a["s"],
+                                                 a["group"])
+        relu = bool(rng.integers(0, 2))
+        bias = b if rng.integers(0, 2) else None
+        ref = oracle.conv_fast(oracle.ConvParams(**a), x, w, bias, relu)
+        got, path = run_layer(hgc, a, x, w, bias, relu, flags=flags)
+        paths.add(path)
+        assert got.shape == ref.shape
+        check_close(got, ref, what=str(a))
+        done += 1
+    if flags:
+        assert paths == {hgc.HGC_PATH_DIRECT}
+
+
+@pytest.mark.parametrize("plane", [7, 13, 14, 27, 28, 33, 56, 57, 112, 113, 150])
+@pytest.mark.parametrize("stride", [1, 2])
+def test_depthwise_planes(hgc, oracle, plane, stride):
+    """3x3 depthwise at the MobileNet plane sizes and at odd, ragged ones; several images and a
+    channel count that leaves a ragged last CTA."""
+    rng = np.random.default_rng(plane * 10 + stride)
+    n, c = 3, 37
+    if plane >= 112:
+        n, c = 2, 5
+    for pad in (1, 0):
+        a = params_dict(n, c, plane, plane + (plane % 5), c, 3, 3, pad, pad, stride, stride, 1, 1, c)
+        x, w, b = workloads.random_layer_tensors(rng, n, c, a["h"], a["w"], c, 3, 3, c)
+        ref = oracle.conv_fast(oracle.ConvParams(**a), x, w, b, True)
+        got, path = run_layer(hgc, a, x, w, b, True)
+        assert path == hgc.HGC_PATH_DEPTHWISE
+        check_close(got, ref, what=f"dw plane {plane} stride {stride} pad {pad}")
+        got2, _ = run_layer(hgc, a, x, w, None, False)
+        check_close(got2, oracle.conv_fast(oracle.ConvParams(**a), x, w, None, False), what="dw no bias")
+
+
+@pytest.mark.parametrize("cfg,batch", [(0, 1), (1, 1), (2, 1), (3, 1)])
+def test_configs_whole_tensor(hgc, oracle, cfg, batch):
+    """Configs small enough for the oracle to compute every output."""
+    wl = workloads.workload(cfg, batch)
+    for li, l in enumerate(wl.layers):
+        x, w, b = workloads.make_tensors(cfg, batch, li, l)
+        a = layer_args(batch, l)
+        ref = oracle.conv_fast(oracle.ConvParams(**a), x, w, b, l.relu)
+        assert float(np.abs(ref.astype(np.float64)).max()) < 65504
+        got, _ = run_layer(hgc, a, x, w, b, l.relu, register_weights=True)
+        err, same = check_close(got, ref, what=f"{wl.name}/{l.name}")
+        assert same > 0.98, (wl.name, l.name, same)   # beyond rare 1-ulp rounding ties means a bug
+
+
+def _unique_layers(wl):
+    seen, out = set(), []
+    for li, l in enumerate(wl.layers):
+        key = (l.c, l.h, l.k, l.r, l.stride, l.pad, l.group, l.relu)
+        if key not in seen:
+            seen.add(key)
+            out.append((li, l))
+    return out
+
+
+@pytest.mark.parametrize("cfg,batch", [(2, 16), (3, 32), (4, 64)])
+def test_configs_full_size_sampled(hgc, oracle, cfg, batch):
+    """Full-size layers in the configuration the bench times (planner's path, registered
+    weights); the oracle evaluates a sample of outputs one by one: corners, borders, first and
+    last image/channel, and 16k random points per layer.  Every output must also be finite and,
+    with ReLU, non-negative (an unwritten element stays NaN)."""
+    import torch
+    wl = workloads.workload(cfg, batch)
+    rng = np.random.default_rng(99 + cfg)
+    for li, l in _unique_layers(wl):
+        x, w, b = workloads.make_tensors(cfg, batch, li, l)
+        a = layer_args(batch, l)
+        d = hgc.ConvDesc(**a)
+        n, k, p, q = d.output_dims()
+        assert (n, k, p, q) == (batch, l.k, l.out, l.out)
+        d.ensure_workspace()
+        xd, wd, bd = to_dev(x), to_dev(w), to_dev(b)
+        y = torch.full((n, k, p, q), float("nan"), dtype=torch.float16, device="cuda")
+        d.set_weights(wd)
+        hgc.conv_forward(d, xd, wd, bd, y, l.relu)
+        torch.cuda.synchronize()
+        assert d.last_device_status() == hgc.HGC_OK
+        assert bool(torch.isfinite(y).all()), f"{wl.name}/{l.name}: non-finite output"
+        if l.relu:
+            assert float(y.min()) >= 0.0
+        coords = sample_coords(rng, n, k, p, q)
+        ref = oracle.conv_points(oracle.ConvParams(**a), x, w, b, l.relu, coords)
+        ct = torch.from_numpy(coords).cuda()
+        got = to_host(y[ct[:, 0], ct[:, 1], ct[:, 2], ct[:, 3]])
+        check_close(got, ref, what=f"{wl.name}/{l.name}")
+        d.close()
+        del xd, wd, bd, y
+
+
+def test_forward_host_matches_device_forward(hgc, oracle):
+    import torch
+    rng = np.random.default_rng(4)
+    a = params_dict(2, 6, 17, 19, 10, 3, 3, 1, 1, 2, 1, 1, 1, 2)
+    x, w, b = workloads.random_layer_tensors(rng, 2, 6, 17, 19, 10, 3, 3, 2)
+    ref = oracle.conv_fast(oracle.ConvParams(**a), x, w, b, True)
+    d = hgc.ConvDesc(**a)
+    d.ensure_workspace(host=True)
+    xh = torch.from_numpy(x.view(np.int16)).pin_memory()
+    wh = torch.from_numpy(w.view(np.int16)).pin_memory()
+    bh = torch.from_numpy(b.view(np.int16)).pin_memory()
+    yh = torch.empty(ref.shape, dtype=torch.int16).pin_memory()
+    hgc.conv_forward_host(d, xh, wh, bh, yh, True)
+    torch.cuda.synchronize()
+    got = yh.numpy().view(F16)
+    check_close(got, ref, what="forward_host")
+    d.set_workspace(None)
+    with pytest.raises(hgc.HgcError) as e:
+        hgc.conv_forward_host(d, xh, wh, bh, yh, True)
+    assert e.value.status == hgc.HGC_NO_WORKSPACE
