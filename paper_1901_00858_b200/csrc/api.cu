@@ -18,6 +18,7 @@ struct hgc_conv_desc {
   void* ws;               // caller-owned device scratch
   size_t ws_bytes;
   const void* registered_w;
+  hgc::IgemmPlan igemm;
 };
 
 namespace {
@@ -65,6 +66,20 @@ int forward_impl(hgc_conv_desc* d, const void* x, const void* w, const void* bia
   __half* yh = static_cast<__half*>(y);
   cudaError_t err;
   switch (d->path) {
+    case HGC_PATH_IGEMM: {
+      char* ws = static_cast<char*>(d->ws);
+      const hgc::IgemmPlan& ip = d->igemm;
+      __half* wp = reinterpret_cast<__half*>(ws + ip.ws_w_off);
+      __half* xp = reinterpret_cast<__half*>(ws + ip.ws_x_off);
+      if (d->registered_w != w) {  // weights not prepared in advance: re-lay them out now
+        err = hgc::launch_weights_repack(wh, wp, g.k, g.cg, g.r, g.s, g.group, ip.cw, stream);
+        if (err != cudaSuccess) break;
+      }
+      err = hgc::launch_nchw_to_nhwc(xh, xp, g.n, g.c, g.h, g.w, ip.c_pad, stream);
+      if (err != cudaSuccess) break;
+      err = hgc::launch_igemm(g, ip, ws, bh, yh, relu, stream);
+      break;
+    }
     case HGC_PATH_DEPTHWISE:
       err = hgc::launch_depthwise3x3(g, xh, wh, bh, yh, relu, stream);
       break;
@@ -112,7 +127,12 @@ int hgc_conv_desc_create(hgc_conv_desc** out, const hgc_conv_params* p) {
   d->path = HGC_PATH_DIRECT;
   d->ws_needed = 0;
   if (!(p->flags & HGC_FLAG_FORCE_DIRECT)) {
-    if (hgc::depthwise3x3_supported(g)) d->path = HGC_PATH_DEPTHWISE;
+    if (hgc::depthwise3x3_supported(g)) {
+      d->path = HGC_PATH_DEPTHWISE;
+    } else if (hgc::igemm_make_plan(g, &d->igemm)) {
+      d->path = HGC_PATH_IGEMM;
+      d->ws_needed = d->igemm.ws_total;
+    }
   }
   d->ws = nullptr;
   d->ws_bytes = 0;
@@ -193,14 +213,27 @@ int hgc_conv_set_workspace(hgc_conv_desc* d, void* dev_ptr, size_t bytes) {
   d->ws = dev_ptr;
   d->ws_bytes = dev_ptr ? bytes : 0;
   d->registered_w = nullptr;
+  d->igemm.maps_ready = false;
+  if (d->path == HGC_PATH_IGEMM && dev_ptr != nullptr && bytes >= d->ws_needed) {
+    // the TMA descriptors point into the workspace: encode them now; clear the status word
+    if (!hgc::igemm_encode_maps(d->geom, &d->igemm, dev_ptr)) return HGC_CUDA_ERROR;
+    if (cudaMemset(static_cast<char*>(dev_ptr) + d->igemm.ws_status_off, 0, 256) != cudaSuccess)
+      return HGC_CUDA_ERROR;
+  }
   return HGC_OK;
 }
 
 int hgc_conv_set_weights(hgc_conv_desc* d, const void* w, void* stream) {
-  (void)stream;
   if (d == nullptr || w == nullptr) return HGC_INVALID_ARG;
   if (misaligned(w)) return HGC_BAD_ALIGNMENT;
   if (d->ws_needed > 0 && (d->ws == nullptr || d->ws_bytes < d->ws_needed)) return HGC_NO_WORKSPACE;
+  if (d->path == HGC_PATH_IGEMM) {
+    const hgc::ConvGeom& g = d->geom;
+    __half* wp = reinterpret_cast<__half*>(static_cast<char*>(d->ws) + d->igemm.ws_w_off);
+    if (hgc::launch_weights_repack(static_cast<const __half*>(w), wp, g.k, g.cg, g.r, g.s, g.group,
+                                   d->igemm.cw, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+      return HGC_CUDA_ERROR;
+  }
   d->registered_w = w;
   return HGC_OK;
 }
@@ -208,6 +241,15 @@ int hgc_conv_set_weights(hgc_conv_desc* d, const void* w, void* stream) {
 int hgc_conv_last_device_status(hgc_conv_desc* d, int32_t* status) {
   if (d == nullptr || status == nullptr) return HGC_INVALID_ARG;
   *status = HGC_OK;
+  if (d->path == HGC_PATH_IGEMM && d->ws != nullptr && d->ws_bytes >= d->ws_needed) {
+    int32_t word = 0;
+    char* sp = static_cast<char*>(d->ws) + d->igemm.ws_status_off;
+    if (cudaMemcpy(&word, sp, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return HGC_CUDA_ERROR;
+    if (word != 0) {
+      *status = word;
+      if (cudaMemset(sp, 0, sizeof(word)) != cudaSuccess) return HGC_CUDA_ERROR;
+    }
+  }
   return HGC_OK;
 }
 

@@ -1,5 +1,6 @@
 // Internal declarations shared by the translation units of libhgc (host planner + kernels).
 #pragma once
+#include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -34,5 +35,24 @@ cudaError_t launch_nhwc_to_nchw(const __half* src, __half* dst, int32_t n, int32
                                 int32_t w, int32_t c_pad, cudaStream_t stream);
 cudaError_t launch_weights_repack(const __half* src, __half* dst, int32_t k, int32_t cg, int32_t r,
                                   int32_t s, int32_t group, int32_t c_pad, cudaStream_t stream);
+
+// Plan of the tcgen05 implicit-GEMM path for one layer (host side).
+struct IgemmPlan {
+  int32_t kb, cblocks, cw, c_pad;
+  int32_t tn, th, tw, ncols;
+  int32_t tiles_h, tiles_n, mtiles;
+  int32_t stages, tmem_cols;
+  uint32_t a_bytes, b_bytes, b_alloc;
+  size_t smem_bytes;
+  size_t ws_status_off, ws_w_off, ws_x_off, ws_total;
+  bool maps_ready;
+  alignas(64) CUtensorMap tmA;
+  alignas(64) CUtensorMap tmB;
+};
+
+bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out);
+bool igemm_encode_maps(const ConvGeom& g, IgemmPlan* p, void* ws);
+cudaError_t launch_igemm(const ConvGeom& g, const IgemmPlan& p, void* ws, const __half* bias, __half* y,
+                         int relu, cudaStream_t stream);
 
 }  // namespace hgc
