@@ -207,7 +207,11 @@ def run_ours(args, wl):
     peaks = load_peaks()
     stream = torch.cuda.current_stream()
     layers = wl.expanded()
-    batch = wl.batch
+    if args.only:
+        layers = [l for l in layers if l.name in args.only.split(",")]
+        if not layers:
+            raise SystemExit(f"--only {args.only}: no such layer in {wl.name}")
+    batch = args.batch if args.batch else wl.batch
 
     # resident tensors, one set per layer (weights registered once: steady-state inference)
     gen = torch.Generator(device="cuda")
@@ -272,7 +276,7 @@ def run_ours(args, wl):
     e2e_steps = max(1, min(args.steps, 5))
     host = []
     h2d = d2h = 0
-    for (d, x, w, b, y, l) in state:
+    for (d, x, w, b, y, l) in (state if not args.no_e2e else []):
         d.ensure_workspace(host=True)
         hx = torch.empty(x.shape, dtype=torch.float16).pin_memory()
         hx.copy_(x.cpu())
@@ -288,15 +292,17 @@ def run_ours(args, wl):
         for (d, x, w, b, y, l), (hx, hw, hb, hy) in zip(state, host):
             hgc.conv_forward_host(d, hx, hw, hb, hy, l.relu, stream)
 
-    e2e_step()
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(e2e_steps):
+    e2e_ms = float("nan")
+    if not args.no_e2e:
         e2e_step()
-    e1.record(stream)
-    barrier()
-    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record(stream)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
     # ---- max over ranks ---------------------------------------------------------------------
     if world > 1:
@@ -341,7 +347,8 @@ def run_ours(args, wl):
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16 (f32 accumulate)",
             "data": "synthetic",
-            "config": {"workload": wl.name, "layers": len(layers), "batch_per_gpu": batch,
+            "config": {"workload": wl.name if not (args.only or args.batch) else f"{wl.name} (subset: only={args.only or 'all'}, batch={batch})",
+                       "layers": len(layers), "batch_per_gpu": batch,
                        "l2": "inputs larger than L2 (every layer has its own tensors)",
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
             "images_per_s": agg["images_per_s"],
@@ -379,6 +386,9 @@ def main():
                     help="one of: " + ", ".join(w.name for w in workloads.all_workloads()))
     ap.add_argument("--layers", action="store_true", help="add per-layer figures to the JSON line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
+    ap.add_argument("--only", default="", help="comma-separated layer names: run just these layers (profiling)")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling on a small case)")
     args = ap.parse_args()
     wl = workloads.by_name(args.workload)
     if args.impl == "reference":

@@ -109,6 +109,15 @@ int hgc_conv_output_dims(const hgc_conv_desc* d, int32_t* n, int32_t* k, int32_t
 /* The kernel path the planner chose (an hgc_path value). */
 int hgc_conv_path(const hgc_conv_desc* d, int32_t* path);
 
+/*
+ * Tiling the planner chose, for inspection and tests.  Writes up to `count` int32 values:
+ * [0] path, then for HGC_PATH_IGEMM: [1] channels per reduction block, [2] 1 if the taps of a
+ * kernel row share one activation tile (stride 1), [3] images per pixel tile, [4] rows per pixel
+ * tile, [5] accumulator columns per output row, [6] MMA N, [7] number of tiles, [8] weight-ring
+ * depth, [9] activation-ring depth; zeros for the other paths.  info: host pointer.
+ */
+int hgc_conv_plan_info(const hgc_conv_desc* d, int32_t* info, int32_t count);
+
 /* Scratch bytes hgc_conv_forward needs for this descriptor (0 if none). */
 int hgc_conv_workspace_bytes(const hgc_conv_desc* d, size_t* bytes);
 

@@ -52,6 +52,7 @@ def lib() -> ctypes.CDLL:
         L.hgc_conv_forward_host.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int, vp]
         L.hgc_conv_output_dims.argtypes = [vp, i32p, i32p, i32p, i32p]
         L.hgc_conv_path.argtypes = [vp, i32p]
+        L.hgc_conv_plan_info.argtypes = [vp, i32p, i32]
         L.hgc_conv_workspace_bytes.argtypes = [vp, szp]
         L.hgc_conv_host_workspace_bytes.argtypes = [vp, szp]
         L.hgc_conv_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
@@ -65,7 +66,7 @@ def lib() -> ctypes.CDLL:
         L.hgc_status_string.restype = ctypes.c_char_p
         for name in ("hgc_conv_desc_create", "hgc_conv_desc_destroy", "hgc_conv_forward",
                      "hgc_conv_forward_host", "hgc_conv_output_dims", "hgc_conv_path",
-                     "hgc_conv_workspace_bytes", "hgc_conv_host_workspace_bytes",
+                     "hgc_conv_workspace_bytes", "hgc_conv_host_workspace_bytes", "hgc_conv_plan_info",
                      "hgc_conv_set_workspace", "hgc_conv_set_weights", "hgc_conv_last_device_status",
                      "hgc_layout_nchw_to_nhwc", "hgc_layout_nhwc_to_nchw", "hgc_weights_repack",
                      "hgc_kernel_launch_count"):
@@ -140,6 +141,12 @@ class ConvDesc:
         v = ctypes.c_int32()
         _check(lib().hgc_conv_path(self._h, ctypes.byref(v)), "hgc_conv_path")
         return v.value
+
+    def plan_info(self) -> dict:
+        v = (ctypes.c_int32 * 10)()
+        _check(lib().hgc_conv_plan_info(self._h, v, 10), "hgc_conv_plan_info")
+        keys = ("path", "kb", "halo", "tn", "th", "pitch", "ncols", "tiles", "sa", "sb")
+        return dict(zip(keys, list(v)))
 
     def workspace_bytes(self) -> int:
         v = ctypes.c_size_t()

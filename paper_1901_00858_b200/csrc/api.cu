@@ -68,7 +68,7 @@ int forward_impl(hgc_conv_desc* d, const void* x, const void* w, const void* bia
   switch (d->path) {
     case HGC_PATH_IGEMM: {
       char* ws = static_cast<char*>(d->ws);
-      const hgc::IgemmPlan& ip = d->igemm;
+      hgc::IgemmPlan& ip = d->igemm;
       __half* wp = reinterpret_cast<__half*>(ws + ip.ws_w_off);
       __half* xp = reinterpret_cast<__half*>(ws + ip.ws_x_off);
       if (d->registered_w != w) {  // weights not prepared in advance: re-lay them out now
@@ -194,6 +194,18 @@ int hgc_conv_path(const hgc_conv_desc* d, int32_t* path) {
   return HGC_OK;
 }
 
+int hgc_conv_plan_info(const hgc_conv_desc* d, int32_t* info, int32_t count) {
+  if (d == nullptr || info == nullptr || count < 1) return HGC_INVALID_ARG;
+  int32_t v[10] = {d->path, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+  if (d->path == HGC_PATH_IGEMM) {
+    const hgc::IgemmPlan& p = d->igemm;
+    v[1] = p.kb; v[2] = p.halo; v[3] = p.tn; v[4] = p.th; v[5] = p.pitch; v[6] = p.ncols;
+    v[7] = p.total_tiles; v[8] = p.sa; v[9] = p.sb;
+  }
+  for (int i = 0; i < count && i < 10; ++i) info[i] = v[i];
+  return HGC_OK;
+}
+
 int hgc_conv_workspace_bytes(const hgc_conv_desc* d, size_t* bytes) {
   if (d == nullptr || bytes == nullptr) return HGC_INVALID_ARG;
   *bytes = d->ws_needed;
@@ -214,6 +226,7 @@ int hgc_conv_set_workspace(hgc_conv_desc* d, void* dev_ptr, size_t bytes) {
   d->ws_bytes = dev_ptr ? bytes : 0;
   d->registered_w = nullptr;
   d->igemm.maps_ready = false;
+  d->igemm.y_mapped = nullptr;
   if (d->path == HGC_PATH_IGEMM && dev_ptr != nullptr && bytes >= d->ws_needed) {
     // the TMA descriptors point into the workspace: encode them now; clear the status word
     if (!hgc::igemm_encode_maps(d->geom, &d->igemm, dev_ptr)) return HGC_CUDA_ERROR;

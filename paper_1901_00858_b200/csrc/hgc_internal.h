@@ -39,20 +39,25 @@ cudaError_t launch_weights_repack(const __half* src, __half* dst, int32_t k, int
 // Plan of the tcgen05 implicit-GEMM path for one layer (host side).
 struct IgemmPlan {
   int32_t kb, cblocks, cw, c_pad;
+  int32_t halo, pitch;
   int32_t tn, th, tw, ncols;
-  int32_t tiles_h, tiles_n, mtiles;
-  int32_t stages, tmem_cols;
+  int32_t tiles_h, tiles_n, mtiles, total_tiles;
+  int32_t sa, sb;
+  int32_t tma_store, rem;
+  void* y_mapped;  // output pointer tmY/tmYr were encoded for
   uint32_t a_bytes, b_bytes, b_alloc;
   size_t smem_bytes;
   size_t ws_status_off, ws_w_off, ws_x_off, ws_total;
   bool maps_ready;
   alignas(64) CUtensorMap tmA;
   alignas(64) CUtensorMap tmB;
+  alignas(64) CUtensorMap tmY;
+  alignas(64) CUtensorMap tmYr;
 };
 
 bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out);
 bool igemm_encode_maps(const ConvGeom& g, IgemmPlan* p, void* ws);
-cudaError_t launch_igemm(const ConvGeom& g, const IgemmPlan& p, void* ws, const __half* bias, __half* y,
+cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half* bias, __half* y,
                          int relu, cudaStream_t stream);
 
 }  // namespace hgc

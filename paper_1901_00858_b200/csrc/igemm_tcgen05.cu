@@ -23,12 +23,17 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
+#include <cstdlib>
+
 #include "hgc_internal.h"
 
 namespace hgc {
 namespace {
 
-constexpr int kIgemmThreads = 192;
+constexpr int kEpilogueWarps = 8;  // two per TMEM lane quarter
+constexpr int kIgemmThreads = 64 + 32 * kEpilogueWarps;
+constexpr int kPassElems = 64;               // output pixels per channel staged per TMA store
+constexpr uint32_t kStageBufBytes = 128u * kPassElems * 2u;  // 128 channels x 64 pixels, fp16
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -57,18 +62,38 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
   return ok;
 }
 
+__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+
 __device__ __forceinline__ uint64_t global_timer_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
 
-// Bounded wait: false if the limit expired or another role already gave up.
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// Bounded wait: false if the limit expired or another role already gave up.  `sleep_ns` > 0
+// makes a waiting warp yield its issue slots between polls (the epilogue warps wait for whole
+// tiles and must not compete with the single TMA and MMA issuing threads).
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                            uint32_t sleep_ns) {
   uint64_t t0 = 0;
   for (uint32_t i = 0;; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 63u) == 63u) {
+    // sleeping waiters use the suspending form; the TMA and MMA warps poll without suspending
+    // (a suspended thread is woken a few hundred cycles after the phase completes)
+    if (sleep_ns ? mbar_try_wait(bar, parity) : mbar_test_wait(bar, parity)) return true;
+    if (sleep_ns) __nanosleep(sleep_ns);
+    if ((i & 1023u) == 1023u) {
       if (*abort_flag) return false;
       const uint64_t t = global_timer_ns();
       if (t0 == 0) {
@@ -80,6 +105,36 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile i
     }
   }
 }
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          uint32_t sleep_ns = 0) {
+  if (mbar_test_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, sleep_ns);
+}
+
+// One lane of a converged warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "elect.sync _|p, 0xffffffff;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(pred));
+  return pred != 0;
+}
+
+// Position in a ring of mbarrier-guarded stages: index and the phase parity of the current lap.
+struct Ring {
+  uint32_t idx = 0, phase = 0;
+  __device__ __forceinline__ void advance(uint32_t depth) {
+    if (++idx == depth) {
+      idx = 0;
+      phase ^= 1u;
+    }
+  }
+};
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1,
                                             int c2) {
@@ -122,6 +177,118 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
       : "memory");
 }
 
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&v)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+               : "r"(taddr)
+               : "memory");
+}
+
+// two fp32 -> packed fp16x2 (round to nearest even), lo = first value; optional ReLU in the convert
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi, bool relu) {
+  uint32_t d;
+  if (relu)
+    asm("cvt.rn.relu.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  else
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* tm, uint32_t src, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(tm),
+               "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+               : "memory");
+}
+
+// Polls barrier `next_bar` (non-blocking), issues KSTEPS MMAs of one shared-memory stage from one
+// elected lane (16 channels per step: +32 bytes = +2 in the descriptors' address field), commits
+// them to `a_bar` (and to `b_bar` if release_b), and returns the poll's result.  Warp-collective.
+// The poll is issued first and its answer read last, so its latency hides behind the MMA issue.
+template <int KSTEPS>
+__device__ __forceinline__ uint32_t issue_stage(uint32_t next_bar, uint32_t next_parity, uint32_t d_tmem,
+                                                uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc,
+                                                uint32_t a_bar, uint32_t b_bar, uint32_t release_b,
+                                                uint32_t do_mma) {
+  uint32_t ready;
+#define HGC_STAGE_OPERANDS                                                                                   \
+  : "=r"(ready)                                                                                              \
+  : "r"(next_bar), "r"(next_parity), "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc), "r"(a_bar), \
+    "r"(b_bar), "r"(release_b), "r"(do_mma)                                                                  \
+  : "memory"
+  if (KSTEPS == 4) {
+    asm volatile(
+      "{\n"
+      ".reg .pred p_next, p_el, p_mma, p_acc, p_one, p_rel;\n"
+      ".reg .b64 da, db;\n"
+      "mbarrier.test_wait.parity.shared::cta.b64 p_next, [%1], %2;\n"
+      "elect.sync _|p_el, 0xffffffff;\n"
+      "setp.ne.b32 p_mma, %11, 0;\n"
+      "and.pred p_mma, p_mma, p_el;\n"
+      "setp.ne.b32 p_acc, %7, 0;\n"
+      "setp.eq.b32 p_one, 0, 0;\n"
+      "setp.ne.b32 p_rel, %10, 0;\n"
+      "and.pred p_rel, p_rel, p_el;\n"
+      "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], %4, %5, %6, p_acc;\n"
+      "add.u64 da, %4, 2;\n"
+      "add.u64 db, %5, 2;\n"
+      "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, p_one;\n"
+      "add.u64 da, %4, 4;\n"
+      "add.u64 db, %5, 4;\n"
+      "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, p_one;\n"
+      "add.u64 da, %4, 6;\n"
+      "add.u64 db, %5, 6;\n"
+      "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, p_one;\n"
+      "@p_el tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n"
+      "@p_rel tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n"
+      "selp.u32 %0, 1, 0, p_next;\n"
+      "}\n"
+        HGC_STAGE_OPERANDS);
+  } else if (KSTEPS == 2) {
+    asm volatile(
+      "{\n"
+      ".reg .pred p_next, p_el, p_mma, p_acc, p_one, p_rel;\n"
+      ".reg .b64 da, db;\n"
+      "mbarrier.test_wait.parity.shared::cta.b64 p_next, [%1], %2;\n"
+      "elect.sync _|p_el, 0xffffffff;\n"
+      "setp.ne.b32 p_mma, %11, 0;\n"
+      "and.pred p_mma, p_mma, p_el;\n"
+      "setp.ne.b32 p_acc, %7, 0;\n"
+      "setp.eq.b32 p_one, 0, 0;\n"
+      "setp.ne.b32 p_rel, %10, 0;\n"
+      "and.pred p_rel, p_rel, p_el;\n"
+      "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], %4, %5, %6, p_acc;\n"
+      "add.u64 da, %4, 2;\n"
+      "add.u64 db, %5, 2;\n"
+      "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, p_one;\n"
+      "@p_el tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n"
+      "@p_rel tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n"
+      "selp.u32 %0, 1, 0, p_next;\n"
+      "}\n"
+        HGC_STAGE_OPERANDS);
+  } else {
+    asm volatile(
+      "{\n"
+      ".reg .pred p_next, p_el, p_mma, p_acc, p_one, p_rel;\n"
+      ".reg .b64 da, db;\n"
+      "mbarrier.test_wait.parity.shared::cta.b64 p_next, [%1], %2;\n"
+      "elect.sync _|p_el, 0xffffffff;\n"
+      "setp.ne.b32 p_mma, %11, 0;\n"
+      "and.pred p_mma, p_mma, p_el;\n"
+      "setp.ne.b32 p_acc, %7, 0;\n"
+      "setp.eq.b32 p_one, 0, 0;\n"
+      "setp.ne.b32 p_rel, %10, 0;\n"
+      "and.pred p_rel, p_rel, p_el;\n"
+      "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], %4, %5, %6, p_acc;\n"
+      "@p_el tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n"
+      "@p_rel tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n"
+      "selp.u32 %0, 1, 0, p_next;\n"
+      "}\n"
+        HGC_STAGE_OPERANDS);
+  }
+#undef HGC_STAGE_OPERANDS
+  return ready;
+}
+
 struct IgemmArgs {
   int32_t N, K, P, Q;
   int32_t kg, group;
@@ -129,57 +296,72 @@ struct IgemmArgs {
   int32_t kb;        // channels per reduction block (64 / 32 / 16)
   int32_t cblocks;   // blocks per tap
   int32_t cw;        // channels per tap in w' (cblocks * kb)
-  int32_t tn, th, tw;  // pixel tile: images x rows x full width (tw == Q)
-  int32_t ncols;     // MMA N: tn*th*tw rounded up to 16
+  int32_t halo;      // 1: one B load per kernel row r serves its S taps (stride 1); 0: one B load per tap
+  int32_t tn, th;    // pixel tile: images x rows (full output width)
+  int32_t pitch;     // accumulator columns per output row (Q + (S-1)*dil in halo mode, else Q)
+  int32_t ncols;     // MMA N
   int32_t tiles_h;   // row tiles per plane
+  int32_t tiles_px;  // pixel tiles in total
   int32_t mtiles;    // 128-channel tiles per group
-  int32_t stages;
-  int32_t tmem_cols; // power of two >= ncols
-  uint32_t a_bytes, b_bytes, b_alloc;  // TMA bytes of A and B per stage, smem reserved for B
+  int32_t total_tiles;
+  int32_t sa, sb;    // ring depths of A and B
+  uint32_t a_bytes, b_bytes, b_alloc;  // TMA bytes of A and B per load, smem reserved per B stage
   uint32_t idesc;
   uint64_t desc_hi;  // shared-memory descriptor bits other than the start address
   int32_t relu;
+  int32_t tma_store;  // 1: the epilogue stages fp16 tiles in shared memory and stores them with TMA
+  int32_t rem;        // (th*Q) % 64: width of the last staged pass of a full tile (0 = none)
+  int32_t debug;      // timing experiments only (results are wrong): 1 = no TMA loads, 2 = no MMAs
 };
 
+constexpr int kMaxStages = 8;
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// Persistent kernel: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...; the two TMEM
+// accumulators alternate so that the epilogue of one tile overlaps the MMAs of the next.
+template <int KB, bool HALO>
 __global__ void __launch_bounds__(kIgemmThreads, 1)
 igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+             const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmYr,
              const IgemmArgs a, const __half* __restrict__ bias, __half* __restrict__ y, int* status) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t full_bar[8];
-  __shared__ __align__(8) uint64_t empty_bar[8];
-  __shared__ __align__(8) uint64_t acc_bar;
+  __shared__ __align__(8) uint64_t a_full[kMaxStages], a_empty[kMaxStages];
+  __shared__ __align__(8) uint64_t b_full[kMaxStages], b_empty[kMaxStages];
+  __shared__ __align__(8) uint64_t acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int abort_flag;
 
-  // a CTA of an earlier wave gave up: do not start new work on a path that is not progressing
+  // an earlier CTA gave up: do not start new work on a path that is not progressing
   if (status != nullptr && *reinterpret_cast<volatile int*>(status) != 0) return;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t stage_bytes = a.a_bytes + a.b_alloc;
-
-  // tile coordinates
-  const int tile_n = blockIdx.x / a.tiles_h;
-  const int tile_h = blockIdx.x % a.tiles_h;
-  const int n0 = tile_n * a.tn;
-  const int p0 = tile_h * a.th;
-  const int grp = blockIdx.y / a.mtiles;
-  const int m0 = (blockIdx.y % a.mtiles) * 128;
-  const int niter = a.R * a.S * a.cblocks;
+  const uint32_t a_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t b_base = a_base + (uint32_t)a.sa * a.a_bytes;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < a.stages; ++s) {
-      mbar_init(smem_u32(&full_bar[s]), 1);
-      mbar_init(smem_u32(&empty_bar[s]), 1);
+    for (int s = 0; s < a.sa; ++s) {
+      mbar_init(smem_u32(&a_full[s]), 1);
+      mbar_init(smem_u32(&a_empty[s]), 1);
     }
-    mbar_init(smem_u32(&acc_bar), 1);
+    for (int s = 0; s < a.sb; ++s) {
+      mbar_init(smem_u32(&b_full[s]), 1);
+      mbar_init(smem_u32(&b_empty[s]), 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(smem_u32(&acc_full[s]), 1);
+      mbar_init(smem_u32(&acc_empty[s]), kEpilogueWarps);  // one arrival per epilogue warp
+    }
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
+    // the whole TMEM (512 columns): the kernel's shared-memory request keeps it alone on the SM
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
-                 "r"((uint32_t)a.tmem_cols)
+                 "r"(512u)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -190,34 +372,79 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
-    if (lane == 0) {
-      int issued = 0;
-      int r = 0, s = 0, cb = 0;
-      for (int it = 0; it < niter; ++it) {
-        const int st = it % a.stages;
-        const uint32_t ph = (uint32_t)(it / a.stages) & 1u;
-        if (!mbar_wait(smem_u32(&empty_bar[st]), ph ^ 1u, &abort_flag)) break;
-        const uint32_t fb = smem_u32(&full_bar[st]);
-        mbar_expect_tx(fb, a.a_bytes + a.b_bytes);
-        const uint32_t sa = tiles_base + (uint32_t)st * stage_bytes;
-        tma_load_3d(sa, &tmA, fb, (r * a.S + s) * a.cw + cb * a.kb, m0, grp);
-        tma_load_5d(sa + a.a_bytes, &tmB, fb, cb * a.kb, grp, s * a.dil_w - a.pad_w,
-                    p0 * a.stride_h - a.pad_h + r * a.dil_h, n0);
-        issued = it + 1;
-        if (++cb == a.cblocks) {
-          cb = 0;
-          if (++s == a.S) {
-            s = 0;
-            ++r;
+    // The whole warp walks the loop (warp-uniform control flow keeps addresses, coordinates and
+    // barrier operands in uniform registers); one elected lane issues the copies.
+    Ring ra, rb;              // next stage to fill in each ring
+    uint32_t ia = 0, ib = 0;  // loads issued so far into each ring
+    bool ok = true;
+    const uint32_t sa_n = (uint32_t)a.sa, sb_n = (uint32_t)a.sb;
+    const int mgn = a.mtiles * a.group;
+    // an mbarrier poll takes a couple of hundred cycles even when it succeeds: the poll for the
+    // next stage is issued before the work of the current one and its result used afterwards
+    uint32_t a_free = mbar_test_wait(smem_u32(&a_empty[0]), 1u);
+    uint32_t b_free = mbar_test_wait(smem_u32(&b_empty[0]), 1u);
+    for (int tile = blockIdx.x; tile < a.total_tiles && ok; tile += gridDim.x) {
+      const int px = tile / mgn;
+      const int mg = tile - px * mgn;
+      const int grp = mg / a.mtiles;
+      const int m0 = (mg - grp * a.mtiles) * 128;
+      const int n0 = (px / a.tiles_h) * a.tn;
+      const int p0 = (px % a.tiles_h) * a.th;
+      const int h_base = p0 * a.stride_h - a.pad_h;
+      for (int cb = 0; cb < a.cblocks && ok; ++cb) {
+        int acol = cb * KB;  // column of w' for tap (r, s): (r*S + s)*cw + cb*KB
+        for (int r = 0; r < a.R && ok; ++r) {
+          for (int s = 0; s < a.S; ++s, acol += a.cw) {
+            if (s == 0 || !HALO) {
+              if (!b_free && !mbar_wait(smem_u32(&b_empty[rb.idx]), rb.phase ^ 1u, &abort_flag)) {
+                ok = false;
+                break;
+              }
+              if (elect_one()) {
+                const uint32_t fb = smem_u32(&b_full[rb.idx]);
+                if (a.debug & 1) {
+                  mbar_arrive(fb);
+                } else {
+                  mbar_expect_tx(fb, a.b_bytes);
+                  tma_load_5d(b_base + rb.idx * a.b_alloc, &tmB, fb, cb * KB, grp,
+                              (HALO ? 0 : s * a.dil_w) - a.pad_w, h_base + r * a.dil_h, n0);
+                }
+              }
+              __syncwarp();
+              rb.advance(sb_n);
+              ++ib;
+              b_free = mbar_test_wait(smem_u32(&b_empty[rb.idx]), rb.phase ^ 1u);  // poll ahead
+            }
+            if (!a_free && !mbar_wait(smem_u32(&a_empty[ra.idx]), ra.phase ^ 1u, &abort_flag)) {
+              ok = false;
+              break;
+            }
+            if (elect_one()) {
+              const uint32_t fa = smem_u32(&a_full[ra.idx]);
+              if (a.debug & 1) {
+                mbar_arrive(fa);
+              } else {
+                mbar_expect_tx(fa, a.a_bytes);
+                tma_load_3d(a_base + ra.idx * a.a_bytes, &tmA, fa, acol, m0, grp);
+              }
+            }
+            __syncwarp();
+            ra.advance(sa_n);
+            ++ia;
+            a_free = mbar_test_wait(smem_u32(&a_empty[ra.idx]), ra.phase ^ 1u);  // poll ahead
           }
         }
       }
-      if (abort_flag) {
-        // let the copies that were issued land before the CTA's shared memory goes away
-        const int first = issued > a.stages ? issued - a.stages : 0;
-        for (int it = first; it < issued; ++it) {
-          uint64_t t0 = global_timer_ns();
-          while (!mbar_try_wait(smem_u32(&full_bar[it % a.stages]), (uint32_t)(it / a.stages) & 1u)) {
+    }
+    if (abort_flag && lane == 0) {
+      // let the copies that were issued land before the CTA's shared memory goes away
+      for (int ring = 0; ring < 2; ++ring) {
+        const uint32_t issued = ring ? ib : ia, depth = (uint32_t)(ring ? a.sb : a.sa);
+        const uint32_t first = issued > depth ? issued - depth : 0;
+        for (uint32_t it = first; it < issued; ++it) {
+          const uint32_t bar = smem_u32(ring ? &b_full[it % depth] : &a_full[it % depth]);
+          const uint64_t t0 = global_timer_ns();
+          while (!mbar_try_wait(bar, (it / depth) & 1u)) {
             if (global_timer_ns() - t0 > kWaitLimitNs) break;
           }
         }
@@ -226,100 +453,255 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     __syncwarp();
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
-    if (lane == 0) {
-      bool ok = true;
-      const int ksteps = a.kb / 16;
-      for (int it = 0; it < niter; ++it) {
-        const int st = it % a.stages;
-        const uint32_t ph = (uint32_t)(it / a.stages) & 1u;
-        if (!mbar_wait(smem_u32(&full_bar[st]), ph, &abort_flag)) {
-          ok = false;
-          break;
-        }
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t sa = tiles_base + (uint32_t)st * stage_bytes;
-        const uint32_t sb = sa + a.a_bytes;
-        const uint64_t adesc = a.desc_hi | (uint64_t)((sa & 0x3FFFFu) >> 4);
-        const uint64_t bdesc = a.desc_hi | (uint64_t)((sb & 0x3FFFFu) >> 4);
-        for (int k = 0; k < ksteps; ++k) {
-          // 16 channels = 32 bytes further along the swizzled row: +2 in the address field
-          umma_f16(tmem_base, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), a.idesc,
-                   (it > 0 || k > 0) ? 1u : 0u);
-        }
-        umma_commit(smem_u32(&empty_bar[st]));  // frees the stage when these MMAs have read it
+    // Warp-uniform loop; one elected lane issues tcgen05.mma and tcgen05.commit (always the same
+    // lane: a commit tracks the MMAs of the thread that executes it).
+    Ring ra, rb;
+    uint32_t lt = 0;
+    bool ok = true;
+    constexpr int ksteps = KB / 16;
+    constexpr uint32_t row_bytes = (uint32_t)KB * 2u;
+    const uint32_t sa_n = (uint32_t)a.sa, sb_n = (uint32_t)a.sb;
+    const uint32_t tap_step = (uint32_t)a.dil_w * row_bytes;  // halo mode: tap s starts s*dil pixels in
+    const uint64_t desc_hi = a.desc_hi;
+    const uint32_t idesc = a.idesc;
+    uint32_t a_ready = mbar_test_wait(smem_u32(&a_full[0]), 0u);
+    uint32_t b_ready = mbar_test_wait(smem_u32(&b_full[0]), 0u);
+    long long m_acc = 0, m_a = 0, m_b = 0;
+    const long long m_start = clock64();
+    for (int tile = blockIdx.x; tile < a.total_tiles && ok; tile += gridDim.x, ++lt) {
+      const uint32_t buf = lt & 1u;
+      // the epilogue must have drained this accumulator (two tiles ago)
+      const long long tm0 = clock64();
+      if (!mbar_wait(smem_u32(&acc_empty[buf]), ((lt >> 1) & 1u) ^ 1u, &abort_flag)) {
+        ok = false;
+        break;
       }
-      if (ok) umma_commit(smem_u32(&acc_bar));  // accumulator complete
-    }
-    __syncwarp();
-  } else {
-    // ---------------- epilogue (warps 2..5) ----------------
-    const int quarter = warp & 3;  // the TMEM lane quarter this warp may read
-    const int row = quarter * 32 + lane;
-    const int kin = m0 + row;
-    const bool kvalid = kin < a.kg;
-    const int k = grp * a.kg + (kvalid ? kin : 0);
-    const float bv = (bias != nullptr && kvalid) ? __half2float(__ldg(bias + k)) : 0.f;
-    const bool ok = mbar_wait(smem_u32(&acc_bar), 0, &abort_flag);
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (ok) {
-      const int64_t pq = (int64_t)a.P * a.Q;
-      const int plane_tile = a.th * a.tw;
-      const int ntile = a.tn * plane_tile;
-      const int64_t plane_off0 = (int64_t)p0 * a.Q;
-      uint16_t* yb = reinterpret_cast<uint16_t*>(y);
-      for (int col0 = 0; col0 < a.ncols; col0 += 16) {
-        uint32_t v[16];
-        tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)col0, v);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-        for (int h8 = 0; h8 < 2; ++h8) {
-          const int j = col0 + h8 * 8;
-          if (j >= ntile || !kvalid) continue;
-          uint32_t o[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            float f0 = __uint_as_float(v[h8 * 8 + 2 * e]) + bv;
-            float f1 = __uint_as_float(v[h8 * 8 + 2 * e + 1]) + bv;
-            if (a.relu) {
-              f0 = fmaxf(f0, 0.f);
-              f1 = fmaxf(f1, 0.f);
+      m_acc += clock64() - tm0;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t d_tmem = tmem_base + buf * 256u;
+      uint32_t acc = 0;
+      for (int cb = 0; cb < a.cblocks && ok; ++cb) {
+        for (int r = 0; r < a.R && ok; ++r) {
+          uint32_t sb_addr = 0, b_bar = 0;
+          for (int s = 0; s < a.S; ++s) {
+            if (s == 0 || !HALO) {
+              if (!b_ready) {
+                const long long t_ = clock64();
+                if (!mbar_wait(smem_u32(&b_full[rb.idx]), rb.phase, &abort_flag)) {
+                  ok = false;
+                  break;
+                }
+                m_b += clock64() - t_;
+              }
+              sb_addr = b_base + rb.idx * a.b_alloc;
+              b_bar = smem_u32(&b_empty[rb.idx]);
+              rb.advance(sb_n);
+              b_ready = mbar_test_wait(smem_u32(&b_full[rb.idx]), rb.phase);  // poll ahead
             }
-            o[e] = (uint32_t)__half_as_ushort(__float2half_rn(f0)) |
-                   ((uint32_t)__half_as_ushort(__float2half_rn(f1)) << 16);
+            if (!a_ready) {
+              const long long t_ = clock64();
+              if (!mbar_wait(smem_u32(&a_full[ra.idx]), ra.phase, &abort_flag)) {
+                ok = false;
+                break;
+              }
+              m_a += clock64() - t_;
+            }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t sa_addr = a_base + ra.idx * a.a_bytes;
+            const uint64_t adesc = desc_hi | (uint64_t)((sa_addr & 0x3FFFFu) >> 4);
+            const uint64_t bdesc = desc_hi | (uint64_t)((sb_addr & 0x3FFFFu) >> 4);
+            const uint32_t a_bar = smem_u32(&a_empty[ra.idx]);
+            const bool release_b = (s == a.S - 1) || !HALO;
+            ra.advance(sa_n);
+            // One instruction stream for the warp: poll the NEXT stage's barrier, let the elected
+            // lane issue this stage's MMAs and commits, and only then read the poll's answer, so
+            // that the poll's latency hides behind the MMA issue.
+            a_ready = issue_stage<ksteps>(smem_u32(&a_full[ra.idx]), ra.phase, d_tmem, adesc, bdesc, idesc, acc, a_bar,
+                                          b_bar, release_b ? 1u : 0u, (a.debug & 2) ? 0u : 1u);
+            acc = 1;
+            if (HALO) sb_addr += tap_step;
           }
-          const int in = j / plane_tile;
-          const int rem = j - in * plane_tile;
-          const int n = n0 + in;
-          const int64_t off = plane_off0 + rem;
-          uint16_t* dst = yb + ((int64_t)n * a.K + k) * pq + off;
-          if (rem + 7 < plane_tile && n < a.N && off + 7 < pq && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
-            *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
-          } else {
+        }
+      }
+      if (ok) {
+        if (elect_one()) umma_commit(smem_u32(&acc_full[buf]));  // accumulator complete
+        __syncwarp();
+      }
+    }
+    if ((a.debug & 128) && blockIdx.x == 0 && status != nullptr && lane == 0) {
+      long long* dbg = reinterpret_cast<long long*>(status) + 8;
+      dbg[0] = clock64() - m_start; dbg[1] = m_a; dbg[2] = m_b; dbg[3] = m_acc; dbg[4] = lt;
+    }
+  } else {
+    // ---------------- epilogue (warps 2..9) ----------------
+    // Warp w may read TMEM lanes 32*(w%4)..+31; the two warps of a lane quarter split the columns.
+    const int ew = warp - 2;
+    const int quarter = warp & 3;
+    const int half = ew >> 2;
+    const int row = quarter * 32 + lane;  // accumulator lane = output channel within the tile
+    const int64_t pq = (int64_t)a.P * a.Q;
+    uint16_t* yb = reinterpret_cast<uint16_t*>(y);
+    const uint32_t stage_base = b_base + (uint32_t)a.sb * a.b_alloc;
+    const bool issuer = (ew == 0 && lane == 0);
+    const bool relu = a.relu != 0;
+    const int mgn = a.mtiles * a.group;
+    uint32_t lt = 0, pass_ctr = 0;
+    long long e_wait = 0;
+    const long long e_start = clock64();
+    for (int tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x, ++lt) {
+      const int px = tile / mgn;
+      const int mg = tile - px * mgn;
+      const int grp = mg / a.mtiles;
+      const int m0 = (mg - grp * a.mtiles) * 128;
+      const int n0 = (px / a.tiles_h) * a.tn;
+      const int p0 = (px % a.tiles_h) * a.th;
+      const int kin = m0 + row;
+      const bool kvalid = kin < a.kg;
+      const int k = grp * a.kg + (kvalid ? kin : 0);
+      const float bv = (bias != nullptr && kvalid) ? __half2float(__ldg(bias + k)) : 0.f;
+      const uint32_t buf = lt & 1u;
+      const long long tw0 = clock64();
+      mbar_wait(smem_u32(&acc_full[buf]), (lt >> 1) & 1u, &abort_flag, 256);
+      // all epilogue warps take the same decision: a warp that gave up has raised the flag
+      asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpilogueWarps) : "memory");
+      const long long tw1 = clock64();
+      e_wait += tw1 - tw0;
+      if (abort_flag) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t t_addr = tmem_base + buf * 256u + ((uint32_t)(quarter * 32) << 16);
+
+      if (a.tma_store) {
+        // ---- staged epilogue: TMEM -> registers -> swizzled fp16 tile in smem -> TMA store ----
+        // (taken when Q % 8 == 0, P*Q % 8 == 0 and a tile holds one image: every staged run of
+        //  pixels then starts on a 16-byte boundary of y)
+        const int rows_valid = (a.P - p0) < a.th ? (a.P - p0) : a.th;
+        const int e_valid = rows_valid * a.Q;  // output pixels of one channel in this tile
+        const int npass = (e_valid + kPassElems - 1) / kPassElems;
+        const bool last_row_tile = p0 + a.th >= a.P;
+        for (int pass = 0; pass < npass; ++pass, ++pass_ctr) {
+          const uint32_t sbuf = stage_base + (pass_ctr & 1u) * kStageBufBytes;
+          const int e_lo = pass * kPassElems;
+          const int e_hi = e_lo + kPassElems < e_valid ? e_lo + kPassElems : e_valid;
+          const int e0 = e_lo + half * (kPassElems / 2);
+          const int e1 = e0 + kPassElems / 2 < e_hi ? e0 + kPassElems / 2 : e_hi;
+          if (e0 < e1) {
+            int hr = e0 / a.Q;
+            int wc = e0 - hr * a.Q;
+            uint32_t col = (uint32_t)(hr * a.pitch + wc);
+            for (int e = e0; e < e1; e += 8) {
+              uint32_t v[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+              if (!(a.debug & 16)) {
+                tmem_ld8(t_addr + col, v);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+              }
+              uint32_t o[4];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              const int jj = j + e;
-              if (jj < ntile) {
-                const int in2 = jj / plane_tile;
-                const int rem2 = jj - in2 * plane_tile;
-                const int n2 = n0 + in2;
-                const int64_t off2 = plane_off0 + rem2;
-                if (n2 < a.N && off2 < pq)
-                  yb[((int64_t)n2 * a.K + k) * pq + off2] = (uint16_t)((o[e >> 1] >> ((e & 1) * 16)) & 0xffffu);
+              for (int i = 0; i < 4; ++i)
+                o[i] = pack_f16x2(__uint_as_float(v[2 * i]) + bv, __uint_as_float(v[2 * i + 1]) + bv, relu);
+              const uint32_t chunk = (uint32_t)(e - e_lo) >> 3;
+              const uint32_t dst = sbuf + (uint32_t)row * 128u + ((chunk ^ ((uint32_t)row & 7u)) << 4);
+              if (!(a.debug & 32))
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]),
+                             "r"(o[3])
+                             : "memory");
+              wc += 8;
+              col += 8;
+              if (wc == a.Q) {  // next output row: skip the junk columns of the pitch
+                wc = 0;
+                col += (uint32_t)(a.pitch - a.Q);
               }
             }
           }
+          if (pass == npass - 1) asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          // the other staging buffer is free again once the store issued from it has been read
+          if (issuer) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpilogueWarps) : "memory");
+          if (pass == npass - 1 && lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
+          if (issuer && !(a.debug & 64)) {
+            const bool full_box = (e_hi - e_lo == kPassElems) || last_row_tile;  // past P*Q the store is clipped
+            tma_store_4d(full_box ? &tmY : &tmYr, sbuf, p0 * a.Q + e_lo, m0, grp, n0);
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          }
         }
-        __syncwarp();  // tcgen05.ld is warp-collective: reconverge before the next one
+      } else {
+        // ---- direct epilogue: each thread stores runs of its own channel plane ----
+        if (half == 0) {
+          // running position of column j: image `img`, tile row `hr`, column `wc` within the pitch
+          int img = 0, hr = 0, wc = 0;
+          for (int col0 = 0; col0 < a.ncols; col0 += 16) {
+            uint32_t v[16];
+            tmem_ld16(t_addr + (uint32_t)col0, v);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+            for (int h8 = 0; h8 < 2; ++h8) {
+              uint32_t o[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e)
+                o[e] = pack_f16x2(__uint_as_float(v[h8 * 8 + 2 * e]) + bv, __uint_as_float(v[h8 * 8 + 2 * e + 1]) + bv,
+                                  relu);
+              const int n = n0 + img, p = p0 + hr;
+              const bool rowvalid = kvalid && img < a.tn && n < a.N && p < a.P;
+              uint16_t* dst = yb + ((int64_t)n * a.K + k) * pq + (int64_t)p * a.Q + wc;
+              if (wc + 8 <= a.Q) {
+                // the 8 columns are 8 consecutive output pixels of one row
+                if (rowvalid) {
+                  const uintptr_t ad = reinterpret_cast<uintptr_t>(dst);
+                  if ((ad & 15u) == 0) {
+                    *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
+                  } else if ((ad & 3u) == 0) {
+                    uint32_t* d32 = reinterpret_cast<uint32_t*>(dst);
+                    d32[0] = o[0]; d32[1] = o[1]; d32[2] = o[2]; d32[3] = o[3];
+                  } else {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) dst[e] = (uint16_t)((o[e >> 1] >> ((e & 1) * 16)) & 0xffffu);
+                  }
+                }
+                wc += 8;
+                if (wc >= a.pitch) {  // only when pitch == Q and Q % 8 == 0
+                  wc = 0;
+                  if (++hr == a.th) { hr = 0; ++img; }
+                }
+              } else {
+                // the chunk runs over the end of a row (junk columns and/or the next row)
+                int im2 = img, hr2 = hr, wc2 = wc;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                  const int n2 = n0 + im2, p2 = p0 + hr2;
+                  if (kvalid && wc2 < a.Q && im2 < a.tn && n2 < a.N && p2 < a.P)
+                    yb[((int64_t)n2 * a.K + k) * pq + (int64_t)p2 * a.Q + wc2] =
+                        (uint16_t)((o[e >> 1] >> ((e & 1) * 16)) & 0xffffu);
+                  if (++wc2 == a.pitch) {
+                    wc2 = 0;
+                    if (++hr2 == a.th) { hr2 = 0; ++im2; }
+                  }
+                }
+                img = im2; hr = hr2; wc = wc2;
+              }
+            }
+            __syncwarp();  // tcgen05.ld is warp-collective: reconverge before the next one
+          }
+        }
+        // this warp has read its lanes of the accumulator: hand the buffer back to the MMA issuer
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
       }
     }
+    if ((a.debug & 128) && blockIdx.x == 0 && status != nullptr && lane == 0 && ew < 2) {
+      long long* dbg = reinterpret_cast<long long*>(status) + 2 + 3 * ew;
+      dbg[0] = clock64() - e_start; dbg[1] = e_wait; dbg[2] = lt;
+    }
+    // the shared-memory tiles of outstanding stores must stay intact until they have been read,
+    // and the stores themselves must be complete before the kernel ends
+    if (issuer) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)a.tmem_cols)
-                 : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
   }
   if (threadIdx.x == 0 && abort_flag && status != nullptr) atomicExch(status, (int)HGC_DEVICE_TIMEOUT);
 }
@@ -344,6 +726,19 @@ inline size_t round_up_sz(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 }  // namespace
 
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+      n = v;
+    else
+      return 148;  // B200; not cached so that a later call can still query the device
+  }
+  return n;
+}
+
 bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   IgemmPlan p{};
   if (g.cg < 9) return false;                         // too few channels per tap for a K=16 MMA step
@@ -352,37 +747,75 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   p.cblocks = (g.cg + p.kb - 1) / p.kb;
   p.cw = p.cblocks * p.kb;
   p.c_pad = (g.c + 7) / 8 * 8;
-  // pixel tile: full output width, as many rows (then images) as fit 256 columns
-  if (g.q > 256 || (int64_t)g.q * g.stride_w > 256) return false;
+  // stride 1: the S taps of a kernel row read one shared tile, shifted by s*dil pixels
+  p.halo = (g.stride_h == 1 && g.stride_w == 1) ? 1 : 0;
+  p.pitch = p.halo ? g.q + (g.s - 1) * g.dil_w : g.q;
   p.tw = g.q;
-  const int th_max = 256 / g.q;
-  if (th_max >= g.p) {
-    p.th = g.p;
-    p.tiles_h = 1;
-    int tn_max = 256 / (g.p * g.q);
-    if (tn_max > g.n) tn_max = g.n;
-    const int nt = (g.n + tn_max - 1) / tn_max;
-    p.tn = (g.n + nt - 1) / nt;
-  } else {
-    p.tiles_h = (g.p + th_max - 1) / th_max;
-    p.th = (g.p + p.tiles_h - 1) / p.tiles_h;
-    p.tn = 1;
-  }
-  if ((int64_t)p.th * g.stride_h > 256) return false;
-  p.tiles_n = (g.n + p.tn - 1) / p.tn;
-  p.ncols = (p.tn * p.th * p.tw + 15) / 16 * 16;
+  const int box_w = p.halo ? p.pitch : g.q * g.stride_w;
+  if (p.pitch > 256 || box_w > 256) return false;
   p.mtiles = (g.kg + 127) / 128;
-  if ((int64_t)p.tiles_n * p.tiles_h > 0x7fffffffLL || (int64_t)p.mtiles * g.group > 65535) return false;
+  const int64_t mg = (int64_t)p.mtiles * g.group;
+  // pixel tile = tn images x th rows; accumulator columns = tn*th*pitch (<= 256).  Among the
+  // feasible shapes pick the one with the least estimated time: waves over the SMs x (columns
+  // + a per-tile overhead), preferring larger tiles on ties.
+  const int sms = sm_count();
+  const int junk = p.pitch - g.q;
+  double best = 1e300;
+  int best_th = 0, best_tn = 0;
+  for (int th = 1; th <= g.p; ++th) {
+    if ((int64_t)th * p.pitch - junk > 256 || (int64_t)th * g.stride_h > 256) break;
+    const int tn_hi = th == g.p ? g.n : 1;  // several images only when a tile holds whole planes
+    for (int tn = 1; tn <= tn_hi; ++tn) {
+      const int64_t cols = (int64_t)tn * th * p.pitch - junk;
+      if (cols > 256 || tn > 256) break;
+      const int64_t tiles = (int64_t)((g.n + tn - 1) / tn) * ((g.p + th - 1) / th) * mg;
+      const int64_t waves = (tiles + sms - 1) / sms;
+      const double ncols = (double)((cols + 15) / 16 * 16);
+      // covered columns (incl. ragged last tiles) matter when there are many waves; whole waves
+      // when there are few
+      // an MMA step costs about max(N, 64 + N/2) column-times (narrow tiles re-read the weight
+      // stage from shared memory too often to keep the tensor pipe busy)
+      const double mma = ncols > 64.0 + 0.5 * ncols ? ncols : 64.0 + 0.5 * ncols;
+      const double cost = (double)waves * (mma + 40.0) + 1e-3 * (double)tiles;
+      if (cost < best - 1e-9 || (cost < best + 1e-9 && (int64_t)tn * th > (int64_t)best_tn * best_th)) {
+        best = cost;
+        best_th = th;
+        best_tn = tn;
+      }
+    }
+  }
+  if (best_th == 0) return false;
+  p.th = best_th;
+  p.tn = best_tn;
+  p.tiles_h = (g.p + p.th - 1) / p.th;
+  p.tiles_n = (g.n + p.tn - 1) / p.tn;
+  p.ncols = (p.tn * p.th * p.pitch - junk + 15) / 16 * 16;
+  const int64_t total = (int64_t)p.tiles_n * p.tiles_h * mg;
+  if (total > 0x7fffffffLL) return false;
+  p.total_tiles = (int32_t)total;
   p.a_bytes = 128u * p.kb * 2u;
-  p.b_bytes = (uint32_t)(p.tn * p.th * p.tw) * p.kb * 2u;
-  p.b_alloc = (uint32_t)round_up_sz((size_t)p.ncols * p.kb * 2u, 1024);
-  const size_t stage = p.a_bytes + p.b_alloc;
-  int stages = (int)((220u * 1024u) / stage);
-  if (stages > 8) stages = 8;
-  if (stages < 2) return false;
-  p.stages = stages;
-  p.smem_bytes = stage * stages + 1024;
-  p.tmem_cols = p.ncols <= 32 ? 32 : p.ncols <= 64 ? 64 : p.ncols <= 128 ? 128 : 256;
+  const uint32_t box_rows = (uint32_t)(p.tn * p.th * p.pitch);
+  p.b_bytes = box_rows * p.kb * 2u;
+  // rows the MMA may touch: the last tap starts (S-1)*dil rows in and reads ncols rows
+  uint32_t rows = (uint32_t)(p.halo ? (g.s - 1) * g.dil_w : 0) + (uint32_t)p.ncols;
+  if (rows < box_rows) rows = box_rows;
+  p.b_alloc = (uint32_t)round_up_sz((size_t)rows * p.kb * 2u, 1024);
+  // the epilogue stages fp16 tiles for TMA stores when every staged run of pixels starts on a
+  // 16-byte boundary of y: Q % 8 == 0 (so P*Q % 8 == 0 too) and one image per tile
+  p.tma_store = ((g.q % 8) == 0 && p.tn == 1) ? 1 : 0;
+  p.rem = (p.th * g.q) % kPassElems;
+  // rings: B two or three deep, A with what is left (each A stage feeds kb/16 MMAs).  227 KB per
+  // CTA minus alignment slack, static barriers and the two epilogue staging buffers.
+  const size_t budget = 232448u - 1024u - 512u - 2u * kStageBufBytes;
+  p.sb = p.halo ? 3 : 4;
+  while (p.sb > 2 && (size_t)p.sb * p.b_alloc + 4u * p.a_bytes > budget) --p.sb;
+  if ((size_t)p.sb * p.b_alloc + 2u * p.a_bytes > budget) return false;
+  p.sa = (int)((budget - (size_t)p.sb * p.b_alloc) / p.a_bytes);
+  if (p.sa > 8) p.sa = 8;
+  p.smem_bytes = (size_t)p.sa * p.a_bytes + (size_t)p.sb * p.b_alloc + 2u * kStageBufBytes + 1024;
+  // more than half of an SM's shared memory: at most one CTA per SM, so that the kernel can take
+  // all 512 TMEM columns without ever waiting for another CTA to free them
+  if (p.smem_bytes < 120u * 1024u) p.smem_bytes = 120u * 1024u;
   // workspace: status word, re-laid-out weights, NHWC input
   p.ws_status_off = 0;
   p.ws_w_off = 256;
@@ -416,8 +849,8 @@ bool igemm_encode_maps(const ConvGeom& g, IgemmPlan* p, void* ws) {
     const cuuint64_t pix = (cuuint64_t)p->c_pad * 2;
     cuuint64_t dims[5] = {cdim, (cuuint64_t)g.group, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.n};
     cuuint64_t strides[4] = {g.group > 1 ? (cuuint64_t)g.cg * 2 : pix, pix, pix * g.w, pix * g.w * g.h};
-    cuuint32_t box[5] = {(cuuint32_t)p->kb, 1, (cuuint32_t)(p->tw * g.stride_w), (cuuint32_t)(p->th * g.stride_h),
-                         (cuuint32_t)p->tn};
+    const cuuint32_t box_w = p->halo ? (cuuint32_t)p->pitch : (cuuint32_t)(p->tw * g.stride_w);
+    cuuint32_t box[5] = {(cuuint32_t)p->kb, 1, box_w, (cuuint32_t)(p->th * g.stride_h), (cuuint32_t)p->tn};
     cuuint32_t es[5] = {1, 1, (cuuint32_t)g.stride_w, (cuuint32_t)g.stride_h, 1};
     if (enc(&p->tmB, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, base + p->ws_x_off, dims, strides, box, es,
             CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -428,17 +861,39 @@ bool igemm_encode_maps(const ConvGeom& g, IgemmPlan* p, void* ws) {
   return true;
 }
 
-cudaError_t launch_igemm(const ConvGeom& g, const IgemmPlan& p, void* ws, const __half* bias, __half* y,
+// Tensor maps of the output y[N][K][P*Q] seen as (pixels, channels of a group, groups, images):
+// one with a 64-pixel box and one with the narrower box of a tile's last staged pass.
+bool igemm_encode_y_maps(const ConvGeom& g, IgemmPlan* p, void* y) {
+  PFN_cuTensorMapEncodeTiled_v12000 enc = encode_fn();
+  if (enc == nullptr) return false;
+  const cuuint64_t pq = (cuuint64_t)g.p * g.q;
+  cuuint64_t dims[4] = {pq, (cuuint64_t)g.kg, (cuuint64_t)g.group, (cuuint64_t)g.n};
+  cuuint64_t strides[3] = {pq * 2, pq * 2 * (cuuint64_t)g.kg, pq * 2 * (cuuint64_t)g.k};
+  cuuint32_t es[4] = {1, 1, 1, 1};
+  for (int i = 0; i < 2; ++i) {
+    cuuint32_t box[4] = {(cuuint32_t)((i == 0 || p->rem == 0) ? kPassElems : p->rem), 128, 1, 1};
+    if (enc(i == 0 ? &p->tmY : &p->tmYr, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, y, dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return false;
+  }
+  p->y_mapped = y;
+  return true;
+}
+
+cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half* bias, __half* y,
                          int relu, cudaStream_t stream) {
   if (!p.maps_ready) return cudaErrorInvalidValue;
+  if (p.tma_store && p.y_mapped != y && !igemm_encode_y_maps(g, &p, y)) return cudaErrorInvalidValue;
   IgemmArgs a{};
   a.N = g.n; a.K = g.k; a.P = g.p; a.Q = g.q;
   a.kg = g.kg; a.group = g.group;
   a.R = g.r; a.S = g.s; a.pad_h = g.pad_h; a.pad_w = g.pad_w;
   a.stride_h = g.stride_h; a.stride_w = g.stride_w; a.dil_h = g.dil_h; a.dil_w = g.dil_w;
   a.kb = p.kb; a.cblocks = p.cblocks; a.cw = p.cw;
-  a.tn = p.tn; a.th = p.th; a.tw = p.tw; a.ncols = p.ncols;
-  a.tiles_h = p.tiles_h; a.mtiles = p.mtiles; a.stages = p.stages; a.tmem_cols = p.tmem_cols;
+  a.halo = p.halo; a.tn = p.tn; a.th = p.th; a.pitch = p.pitch; a.ncols = p.ncols;
+  a.tiles_h = p.tiles_h; a.tiles_px = p.tiles_h * p.tiles_n; a.mtiles = p.mtiles;
+  a.total_tiles = p.total_tiles; a.sa = p.sa; a.sb = p.sb;
   a.a_bytes = p.a_bytes; a.b_bytes = p.b_bytes; a.b_alloc = p.b_alloc;
   // instruction descriptor: D = f32, A = B = f16, both K-major, N >> 3 at bit 17, M >> 4 at bit 24
   a.idesc = (1u << 4) | ((uint32_t)(p.ncols >> 3) << 17) | ((128u >> 4) << 24);
@@ -448,12 +903,33 @@ cudaError_t launch_igemm(const ConvGeom& g, const IgemmPlan& p, void* ws, const 
   const uint64_t layout = p.kb == 64 ? 2 : (p.kb == 32 ? 4 : 6);
   a.desc_hi = (1ull << 16) | (sbo << 32) | (1ull << 46) | (layout << 61);
   a.relu = relu;
-  cudaError_t err = cudaFuncSetAttribute(igemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)p.smem_bytes);
-  if (err != cudaSuccess) return err;
-  dim3 grid((unsigned)(p.tiles_n * p.tiles_h), (unsigned)(p.mtiles * g.group));
+  a.tma_store = p.tma_store;
+  a.rem = p.rem;
+  {
+    static const char* dbg = getenv("HGC_IGEMM_DEBUG");
+    a.debug = dbg ? atoi(dbg) : 0;
+  }
+  const int sms = sm_count();
+  dim3 grid((unsigned)(p.total_tiles < sms ? p.total_tiles : sms));
   int* status = reinterpret_cast<int*>(static_cast<char*>(ws) + p.ws_status_off);
-  igemm_kernel<<<grid, kIgemmThreads, p.smem_bytes, stream>>>(p.tmA, p.tmB, a, bias, y, status);
+  cudaError_t err = cudaSuccess;
+#define HGC_LAUNCH_IGEMM(KBV, HALOV)                                                                     \
+  do {                                                                                                   \
+    err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV>, cudaFuncAttributeMaxDynamicSharedMemorySize,    \
+                               (int)p.smem_bytes);                                                       \
+    if (err == cudaSuccess)                                                                              \
+      igemm_kernel<KBV, HALOV><<<grid, kIgemmThreads, p.smem_bytes, stream>>>(p.tmA, p.tmB, p.tmY, p.tmYr, a,   \
+                                                                              bias, y, status);          \
+  } while (0)
+  if (p.kb == 64) {
+    if (p.halo) HGC_LAUNCH_IGEMM(64, true); else HGC_LAUNCH_IGEMM(64, false);
+  } else if (p.kb == 32) {
+    if (p.halo) HGC_LAUNCH_IGEMM(32, true); else HGC_LAUNCH_IGEMM(32, false);
+  } else {
+    if (p.halo) HGC_LAUNCH_IGEMM(16, true); else HGC_LAUNCH_IGEMM(16, false);
+  }
+#undef HGC_LAUNCH_IGEMM
+  if (err != cudaSuccess) return err;
   count_launch();
   return cudaGetLastError();
 }
