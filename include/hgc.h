@@ -113,8 +113,8 @@ int hgc_conv_path(const hgc_conv_desc* d, int32_t* path);
  * Tiling the planner chose, for inspection and tests.  Writes up to `count` int32 values:
  * [0] path, then for HGC_PATH_IGEMM: [1] channels per reduction block, [2] 1 if the taps of a
  * kernel row share one activation tile (stride 1), [3] images per pixel tile, [4] rows per pixel
- * tile, [5] accumulator columns per output row, [6] MMA N, [7] number of tiles, [8] weight-ring
- * depth, [9] activation-ring depth; zeros for the other paths.  info: host pointer.
+ * tile, [5] accumulator columns per output row, [6] MMA N, [7] number of tiles, [8] depth of the
+ * shared-memory ring, [9] weight tiles (taps) per ring stage; zeros for the other paths.  info: host pointer.
  */
 int hgc_conv_plan_info(const hgc_conv_desc* d, int32_t* info, int32_t count);
 

@@ -145,7 +145,7 @@ class ConvDesc:
     def plan_info(self) -> dict:
         v = (ctypes.c_int32 * 10)()
         _check(lib().hgc_conv_plan_info(self._h, v, 10), "hgc_conv_plan_info")
-        keys = ("path", "kb", "halo", "tn", "th", "pitch", "ncols", "tiles", "sa", "sb")
+        keys = ("path", "kb", "halo", "tn", "th", "pitch", "ncols", "tiles", "stages", "taps")
         return dict(zip(keys, list(v)))
 
     def workspace_bytes(self) -> int:

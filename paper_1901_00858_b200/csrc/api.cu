@@ -200,7 +200,7 @@ int hgc_conv_plan_info(const hgc_conv_desc* d, int32_t* info, int32_t count) {
   if (d->path == HGC_PATH_IGEMM) {
     const hgc::IgemmPlan& p = d->igemm;
     v[1] = p.kb; v[2] = p.halo; v[3] = p.tn; v[4] = p.th; v[5] = p.pitch; v[6] = p.ncols;
-    v[7] = p.total_tiles; v[8] = p.sa; v[9] = p.sb;
+    v[7] = p.total_tiles; v[8] = p.stages; v[9] = p.taps;
   }
   for (int i = 0; i < count && i < 10; ++i) info[i] = v[i];
   return HGC_OK;

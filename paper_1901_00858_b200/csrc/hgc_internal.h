@@ -42,7 +42,8 @@ struct IgemmPlan {
   int32_t halo, pitch;
   int32_t tn, th, tw, ncols;
   int32_t tiles_h, tiles_n, mtiles, total_tiles;
-  int32_t sa, sb;
+  int32_t stages, taps;
+  uint32_t stage_bytes;
   int32_t tma_store, rem;
   void* y_mapped;  // output pointer tmY/tmYr were encoded for
   uint32_t a_bytes, b_bytes, b_alloc;

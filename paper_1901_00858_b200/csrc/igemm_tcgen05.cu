@@ -85,7 +85,7 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 // Bounded wait: false if the limit expired or another role already gave up.  `sleep_ns` > 0
 // makes a waiting warp yield its issue slots between polls (the epilogue warps wait for whole
 // tiles and must not compete with the single TMA and MMA issuing threads).
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                             uint32_t sleep_ns) {
   uint64_t t0 = 0;
   for (uint32_t i = 0;; ++i) {
@@ -289,6 +289,66 @@ __device__ __forceinline__ uint32_t issue_stage(uint32_t next_bar, uint32_t next
   return ready;
 }
 
+// KSTEPS MMAs of one weight tile against one activation tile, issued by one elected lane.
+template <int KSTEPS>
+__device__ __forceinline__ void issue_mmas(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                           uint32_t acc, uint32_t do_mma) {
+#define HGC_MMA_OPERANDS ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc), "r"(do_mma) : "memory"
+  if (KSTEPS == 4) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p_el, p_mma, p_acc, p_one;\n"
+        ".reg .b64 da, db;\n"
+        "elect.sync _|p_el, 0xffffffff;\n"
+        "setp.ne.b32 p_mma, %5, 0;\n"
+        "and.pred p_mma, p_mma, p_el;\n"
+        "setp.ne.b32 p_acc, %4, 0;\n"
+        "setp.eq.b32 p_one, 0, 0;\n"
+        "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p_acc;\n"
+        "add.u64 da, %1, 2;\n"
+        "add.u64 db, %2, 2;\n"
+        "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p_one;\n"
+        "add.u64 da, %1, 4;\n"
+        "add.u64 db, %2, 4;\n"
+        "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p_one;\n"
+        "add.u64 da, %1, 6;\n"
+        "add.u64 db, %2, 6;\n"
+        "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p_one;\n"
+        "}\n"
+        HGC_MMA_OPERANDS);
+  } else if (KSTEPS == 2) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p_el, p_mma, p_acc, p_one;\n"
+        ".reg .b64 da, db;\n"
+        "elect.sync _|p_el, 0xffffffff;\n"
+        "setp.ne.b32 p_mma, %5, 0;\n"
+        "and.pred p_mma, p_mma, p_el;\n"
+        "setp.ne.b32 p_acc, %4, 0;\n"
+        "setp.eq.b32 p_one, 0, 0;\n"
+        "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p_acc;\n"
+        "add.u64 da, %1, 2;\n"
+        "add.u64 db, %2, 2;\n"
+        "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p_one;\n"
+        "}\n"
+        HGC_MMA_OPERANDS);
+  } else {
+    asm volatile(
+        "{\n"
+        ".reg .pred p_el, p_mma, p_acc, p_one;\n"
+        ".reg .b64 da, db;\n"
+        "elect.sync _|p_el, 0xffffffff;\n"
+        "setp.ne.b32 p_mma, %5, 0;\n"
+        "and.pred p_mma, p_mma, p_el;\n"
+        "setp.ne.b32 p_acc, %4, 0;\n"
+        "setp.eq.b32 p_one, 0, 0;\n"
+        "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p_acc;\n"
+        "}\n"
+        HGC_MMA_OPERANDS);
+  }
+#undef HGC_MMA_OPERANDS
+}
+
 struct IgemmArgs {
   int32_t N, K, P, Q;
   int32_t kg, group;
@@ -304,7 +364,9 @@ struct IgemmArgs {
   int32_t tiles_px;  // pixel tiles in total
   int32_t mtiles;    // 128-channel tiles per group
   int32_t total_tiles;
-  int32_t sa, sb;    // ring depths of A and B
+  int32_t stages;    // ring depth
+  int32_t taps;      // weight tiles per stage: S in halo mode, else 1
+  uint32_t stage_bytes;
   uint32_t a_bytes, b_bytes, b_alloc;  // TMA bytes of A and B per load, smem reserved per B stage
   uint32_t idesc;
   uint64_t desc_hi;  // shared-memory descriptor bits other than the start address
@@ -328,8 +390,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
              const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmYr,
              const IgemmArgs a, const __half* __restrict__ bias, __half* __restrict__ y, int* status) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t a_full[kMaxStages], a_empty[kMaxStages];
-  __shared__ __align__(8) uint64_t b_full[kMaxStages], b_empty[kMaxStages];
+  __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages];
   __shared__ __align__(8) uint64_t acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int abort_flag;
@@ -339,17 +400,13 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const uint32_t a_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t b_base = a_base + (uint32_t)a.sa * a.a_bytes;
+  // ring of stages; a stage holds one activation tile followed by `taps` weight tiles
+  const uint32_t ring_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < a.sa; ++s) {
-      mbar_init(smem_u32(&a_full[s]), 1);
-      mbar_init(smem_u32(&a_empty[s]), 1);
-    }
-    for (int s = 0; s < a.sb; ++s) {
-      mbar_init(smem_u32(&b_full[s]), 1);
-      mbar_init(smem_u32(&b_empty[s]), 1);
+    for (int s = 0; s < a.stages; ++s) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), 1);
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(smem_u32(&acc_full[s]), 1);
@@ -373,16 +430,16 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     // The whole warp walks the loop (warp-uniform control flow keeps addresses, coordinates and
-    // barrier operands in uniform registers); one elected lane issues the copies.
-    Ring ra, rb;              // next stage to fill in each ring
-    uint32_t ia = 0, ib = 0;  // loads issued so far into each ring
+    // barrier operands in uniform registers); one elected lane issues the copies.  A stage is
+    // the activation tile of one kernel row (or one tap when taps cannot share it) plus the
+    // weight tiles of its `taps` taps, all completing on one barrier: the MMA warp then pays the
+    // barrier handshake once per taps*KB/16 MMAs.
+    Ring ring;
+    uint32_t issued = 0;
     bool ok = true;
-    const uint32_t sa_n = (uint32_t)a.sa, sb_n = (uint32_t)a.sb;
+    const uint32_t depth = (uint32_t)a.stages;
     const int mgn = a.mtiles * a.group;
-    // an mbarrier poll takes a couple of hundred cycles even when it succeeds: the poll for the
-    // next stage is issued before the work of the current one and its result used afterwards
-    uint32_t a_free = mbar_test_wait(smem_u32(&a_empty[0]), 1u);
-    uint32_t b_free = mbar_test_wait(smem_u32(&b_empty[0]), 1u);
+    const int groups_per_row = a.S / a.taps;  // 1 in halo mode (taps == S), S otherwise (taps == 1)
     for (int tile = blockIdx.x; tile < a.total_tiles && ok; tile += gridDim.x) {
       const int px = tile / mgn;
       const int mg = tile - px * mgn;
@@ -394,59 +451,40 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       for (int cb = 0; cb < a.cblocks && ok; ++cb) {
         int acol = cb * KB;  // column of w' for tap (r, s): (r*S + s)*cw + cb*KB
         for (int r = 0; r < a.R && ok; ++r) {
-          for (int s = 0; s < a.S; ++s, acol += a.cw) {
-            if (s == 0 || !HALO) {
-              if (!b_free && !mbar_wait(smem_u32(&b_empty[rb.idx]), rb.phase ^ 1u, &abort_flag)) {
-                ok = false;
-                break;
-              }
-              if (elect_one()) {
-                const uint32_t fb = smem_u32(&b_full[rb.idx]);
-                if (a.debug & 1) {
-                  mbar_arrive(fb);
-                } else {
-                  mbar_expect_tx(fb, a.b_bytes);
-                  tma_load_5d(b_base + rb.idx * a.b_alloc, &tmB, fb, cb * KB, grp,
-                              (HALO ? 0 : s * a.dil_w) - a.pad_w, h_base + r * a.dil_h, n0);
-                }
-              }
-              __syncwarp();
-              rb.advance(sb_n);
-              ++ib;
-              b_free = mbar_test_wait(smem_u32(&b_empty[rb.idx]), rb.phase ^ 1u);  // poll ahead
-            }
-            if (!a_free && !mbar_wait(smem_u32(&a_empty[ra.idx]), ra.phase ^ 1u, &abort_flag)) {
+          for (int sg = 0; sg < groups_per_row; ++sg) {
+            if (!mbar_wait(smem_u32(&empty_bar[ring.idx]), ring.phase ^ 1u, &abort_flag, 32)) {
               ok = false;
               break;
             }
+            const uint32_t fb = smem_u32(&full_bar[ring.idx]);
+            const uint32_t sbase = ring_base + ring.idx * a.stage_bytes;
             if (elect_one()) {
-              const uint32_t fa = smem_u32(&a_full[ra.idx]);
               if (a.debug & 1) {
-                mbar_arrive(fa);
+                mbar_arrive(fb);
               } else {
-                mbar_expect_tx(fa, a.a_bytes);
-                tma_load_3d(a_base + ra.idx * a.a_bytes, &tmA, fa, acol, m0, grp);
+                mbar_expect_tx(fb, a.b_bytes + (uint32_t)a.taps * a.a_bytes);
+                tma_load_5d(sbase, &tmB, fb, cb * KB, grp, (HALO ? 0 : sg * a.dil_w) - a.pad_w,
+                            h_base + r * a.dil_h, n0);
+                for (int t = 0; t < a.taps; ++t)
+                  tma_load_3d(sbase + a.b_alloc + (uint32_t)t * a.a_bytes, &tmA, fb, acol + t * a.cw, m0, grp);
               }
             }
             __syncwarp();
-            ra.advance(sa_n);
-            ++ia;
-            a_free = mbar_test_wait(smem_u32(&a_empty[ra.idx]), ra.phase ^ 1u);  // poll ahead
+            acol += a.taps * a.cw;
+            ring.advance(depth);
+            ++issued;
           }
         }
       }
     }
     if (abort_flag && lane == 0) {
       // let the copies that were issued land before the CTA's shared memory goes away
-      for (int ring = 0; ring < 2; ++ring) {
-        const uint32_t issued = ring ? ib : ia, depth = (uint32_t)(ring ? a.sb : a.sa);
-        const uint32_t first = issued > depth ? issued - depth : 0;
-        for (uint32_t it = first; it < issued; ++it) {
-          const uint32_t bar = smem_u32(ring ? &b_full[it % depth] : &a_full[it % depth]);
-          const uint64_t t0 = global_timer_ns();
-          while (!mbar_try_wait(bar, (it / depth) & 1u)) {
-            if (global_timer_ns() - t0 > kWaitLimitNs) break;
-          }
+      const uint32_t first = issued > depth ? issued - depth : 0;
+      for (uint32_t it = first; it < issued; ++it) {
+        const uint32_t bar = smem_u32(&full_bar[it % depth]);
+        const uint64_t t0 = global_timer_ns();
+        while (!mbar_try_wait(bar, (it / depth) & 1u)) {
+          if (global_timer_ns() - t0 > kWaitLimitNs) break;
         }
       }
     }
@@ -455,82 +493,57 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     // ---------------- MMA issuer ----------------
     // Warp-uniform loop; one elected lane issues tcgen05.mma and tcgen05.commit (always the same
     // lane: a commit tracks the MMAs of the thread that executes it).
-    Ring ra, rb;
+    Ring ring;
     uint32_t lt = 0;
     bool ok = true;
     constexpr int ksteps = KB / 16;
     constexpr uint32_t row_bytes = (uint32_t)KB * 2u;
-    const uint32_t sa_n = (uint32_t)a.sa, sb_n = (uint32_t)a.sb;
+    const uint32_t depth = (uint32_t)a.stages;
     const uint32_t tap_step = (uint32_t)a.dil_w * row_bytes;  // halo mode: tap s starts s*dil pixels in
     const uint64_t desc_hi = a.desc_hi;
     const uint32_t idesc = a.idesc;
-    uint32_t a_ready = mbar_test_wait(smem_u32(&a_full[0]), 0u);
-    uint32_t b_ready = mbar_test_wait(smem_u32(&b_full[0]), 0u);
-    long long m_acc = 0, m_a = 0, m_b = 0;
-    const long long m_start = clock64();
+    const uint32_t do_mma = (a.debug & 2) ? 0u : 1u;
+    const int groups_per_row = a.S / a.taps;
+    const int groups_per_tile = a.cblocks * a.R * groups_per_row;
+    uint32_t ready = mbar_test_wait(smem_u32(&full_bar[0]), 0u);
     for (int tile = blockIdx.x; tile < a.total_tiles && ok; tile += gridDim.x, ++lt) {
       const uint32_t buf = lt & 1u;
       // the epilogue must have drained this accumulator (two tiles ago)
-      const long long tm0 = clock64();
       if (!mbar_wait(smem_u32(&acc_empty[buf]), ((lt >> 1) & 1u) ^ 1u, &abort_flag)) {
         ok = false;
         break;
       }
-      m_acc += clock64() - tm0;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t d_tmem = tmem_base + buf * 256u;
       uint32_t acc = 0;
-      for (int cb = 0; cb < a.cblocks && ok; ++cb) {
-        for (int r = 0; r < a.R && ok; ++r) {
-          uint32_t sb_addr = 0, b_bar = 0;
-          for (int s = 0; s < a.S; ++s) {
-            if (s == 0 || !HALO) {
-              if (!b_ready) {
-                const long long t_ = clock64();
-                if (!mbar_wait(smem_u32(&b_full[rb.idx]), rb.phase, &abort_flag)) {
-                  ok = false;
-                  break;
-                }
-                m_b += clock64() - t_;
-              }
-              sb_addr = b_base + rb.idx * a.b_alloc;
-              b_bar = smem_u32(&b_empty[rb.idx]);
-              rb.advance(sb_n);
-              b_ready = mbar_test_wait(smem_u32(&b_full[rb.idx]), rb.phase);  // poll ahead
-            }
-            if (!a_ready) {
-              const long long t_ = clock64();
-              if (!mbar_wait(smem_u32(&a_full[ra.idx]), ra.phase, &abort_flag)) {
-                ok = false;
-                break;
-              }
-              m_a += clock64() - t_;
-            }
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t sa_addr = a_base + ra.idx * a.a_bytes;
-            const uint64_t adesc = desc_hi | (uint64_t)((sa_addr & 0x3FFFFu) >> 4);
-            const uint64_t bdesc = desc_hi | (uint64_t)((sb_addr & 0x3FFFFu) >> 4);
-            const uint32_t a_bar = smem_u32(&a_empty[ra.idx]);
-            const bool release_b = (s == a.S - 1) || !HALO;
-            ra.advance(sa_n);
-            // One instruction stream for the warp: poll the NEXT stage's barrier, let the elected
-            // lane issue this stage's MMAs and commits, and only then read the poll's answer, so
-            // that the poll's latency hides behind the MMA issue.
-            a_ready = issue_stage<ksteps>(smem_u32(&a_full[ra.idx]), ra.phase, d_tmem, adesc, bdesc, idesc, acc, a_bar,
-                                          b_bar, release_b ? 1u : 0u, (a.debug & 2) ? 0u : 1u);
-            acc = 1;
-            if (HALO) sb_addr += tap_step;
-          }
+      for (int gi = 0; gi < groups_per_tile; ++gi) {
+        if (!ready && !mbar_wait(smem_u32(&full_bar[ring.idx]), ring.phase, &abort_flag)) {
+          ok = false;
+          break;
         }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t sbase = ring_base + ring.idx * a.stage_bytes;
+        const uint32_t e_bar = smem_u32(&empty_bar[ring.idx]);
+        uint64_t bdesc = desc_hi | (uint64_t)((sbase & 0x3FFFFu) >> 4);
+        uint64_t adesc = desc_hi | (uint64_t)(((sbase + a.b_alloc) & 0x3FFFFu) >> 4);
+        ring.advance(depth);
+        // all taps but the last: MMAs only
+        for (int t = 0; t + 1 < a.taps; ++t) {
+          issue_mmas<ksteps>(d_tmem, adesc, bdesc, idesc, acc, do_mma);
+          acc = 1;
+          adesc += (uint64_t)(a.a_bytes >> 4);
+          bdesc += (uint64_t)(tap_step >> 4);
+        }
+        // last tap: poll the NEXT stage's barrier first and read the answer after the MMAs and the
+        // commit have been issued, so that the poll's latency hides behind them
+        ready = issue_stage<ksteps>(smem_u32(&full_bar[ring.idx]), ring.phase, d_tmem, adesc, bdesc, idesc, acc, e_bar,
+                                    e_bar, 0u, do_mma);
+        acc = 1;
       }
       if (ok) {
         if (elect_one()) umma_commit(smem_u32(&acc_full[buf]));  // accumulator complete
         __syncwarp();
       }
-    }
-    if ((a.debug & 128) && blockIdx.x == 0 && status != nullptr && lane == 0) {
-      long long* dbg = reinterpret_cast<long long*>(status) + 8;
-      dbg[0] = clock64() - m_start; dbg[1] = m_a; dbg[2] = m_b; dbg[3] = m_acc; dbg[4] = lt;
     }
   } else {
     // ---------------- epilogue (warps 2..9) ----------------
@@ -541,7 +554,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const int row = quarter * 32 + lane;  // accumulator lane = output channel within the tile
     const int64_t pq = (int64_t)a.P * a.Q;
     uint16_t* yb = reinterpret_cast<uint16_t*>(y);
-    const uint32_t stage_base = b_base + (uint32_t)a.sb * a.b_alloc;
+    const uint32_t stage_base = ring_base + (uint32_t)a.stages * a.stage_bytes;
     const bool issuer = (ew == 0 && lane == 0);
     const bool relu = a.relu != 0;
     const int mgn = a.mtiles * a.group;
@@ -549,6 +562,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     long long e_wait = 0;
     const long long e_start = clock64();
     for (int tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x, ++lt) {
+      if (a.debug & 1024) break;  // timing experiment: no epilogue at all
       const int px = tile / mgn;
       const int mg = tile - px * mgn;
       const int grp = mg / a.mtiles;
@@ -807,12 +821,26 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   // rings: B two or three deep, A with what is left (each A stage feeds kb/16 MMAs).  227 KB per
   // CTA minus alignment slack, static barriers and the two epilogue staging buffers.
   const size_t budget = 232448u - 1024u - 512u - 2u * kStageBufBytes;
-  p.sb = p.halo ? 3 : 4;
-  while (p.sb > 2 && (size_t)p.sb * p.b_alloc + 4u * p.a_bytes > budget) --p.sb;
-  if ((size_t)p.sb * p.b_alloc + 2u * p.a_bytes > budget) return false;
-  p.sa = (int)((budget - (size_t)p.sb * p.b_alloc) / p.a_bytes);
-  if (p.sa > 8) p.sa = 8;
-  p.smem_bytes = (size_t)p.sa * p.a_bytes + (size_t)p.sb * p.b_alloc + 2u * kStageBufBytes + 1024;
+  // ring of stages: one activation tile + `taps` weight tiles each, at least two deep; if the
+  // S taps of a kernel row do not fit twice, fall back to one tap (and its own tile) per stage
+  for (;;) {
+    p.taps = p.halo ? g.s : 1;
+    p.pitch = p.halo ? g.q + (g.s - 1) * g.dil_w : g.q;
+    const uint32_t box_rows2 = (uint32_t)(p.tn * p.th * p.pitch);
+    p.b_bytes = box_rows2 * p.kb * 2u;
+    uint32_t rows2 = (uint32_t)(p.halo ? (g.s - 1) * g.dil_w : 0) + (uint32_t)p.ncols;
+    if (rows2 < box_rows2) rows2 = box_rows2;
+    p.b_alloc = (uint32_t)round_up_sz((size_t)rows2 * p.kb * 2u, 1024);
+    p.stage_bytes = p.b_alloc + (uint32_t)p.taps * p.a_bytes;
+    p.stages = (int)(budget / p.stage_bytes);
+    if (p.stages > 8) p.stages = 8;
+    if (p.stages >= 2) break;
+    if (!p.halo) return false;
+    // without sharing, the accumulator pitch is Q again: the tile found above still fits
+    p.halo = 0;
+    p.ncols = (p.tn * p.th * g.q + 15) / 16 * 16;
+  }
+  p.smem_bytes = (size_t)p.stages * p.stage_bytes + 2u * kStageBufBytes + 1024;
   // more than half of an SM's shared memory: at most one CTA per SM, so that the kernel can take
   // all 512 TMEM columns without ever waiting for another CTA to free them
   if (p.smem_bytes < 120u * 1024u) p.smem_bytes = 120u * 1024u;
@@ -893,7 +921,7 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
   a.kb = p.kb; a.cblocks = p.cblocks; a.cw = p.cw;
   a.halo = p.halo; a.tn = p.tn; a.th = p.th; a.pitch = p.pitch; a.ncols = p.ncols;
   a.tiles_h = p.tiles_h; a.tiles_px = p.tiles_h * p.tiles_n; a.mtiles = p.mtiles;
-  a.total_tiles = p.total_tiles; a.sa = p.sa; a.sb = p.sb;
+  a.total_tiles = p.total_tiles; a.stages = p.stages; a.taps = p.taps; a.stage_bytes = p.stage_bytes;
   a.a_bytes = p.a_bytes; a.b_bytes = p.b_bytes; a.b_alloc = p.b_alloc;
   // instruction descriptor: D = f32, A = B = f16, both K-major, N >> 3 at bit 17, M >> 4 at bit 24
   a.idesc = (1u << 4) | ((uint32_t)(p.ncols >> 3) << 17) | ((128u >> 4) << 24);
