@@ -103,6 +103,40 @@ int hgc_conv_forward(hgc_conv_desc* d, const void* x, const void* w, const void*
 int hgc_conv_forward_host(hgc_conv_desc* d, const void* x, const void* w, const void* bias,
                           void* y, int relu, void* stream);
 
+/*
+ * The same layer for callers that cannot allocate device memory.  (The paper has no counterpart
+ * to this entry point; it exists for deployment.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a host process whose
+ * memory pool is owned and fully reserved by another framework, in a plug-in that is forbidden
+ * to grow the process's device footprint after start-up, or between the begin and end of a
+ * region that must not call the allocator.  Such a caller has tensors to read and write but no
+ * way to obtain the scratch buffer that hgc_conv_set_workspace wants.
+ *
+ * What it does: runs the tensor-core path (HGC_PATH_IGEMM) of hgc_conv_forward with its scratch
+ * (status word, re-laid-out weights, NHWC copy of x) in a 32 MiB array that is part of the
+ * library image: every device that loads the library holds those 32 MiB until the process exits.
+ * It takes the layer description directly; no descriptor object, no workspace, no weight
+ * registration (the weights are re-laid-out on every call).  x, w, y: device pointers (required),
+ * bias: device pointer or NULL, all 16-byte aligned; everything is queued on `stream`.
+ *
+ * It calls no cudaMalloc, cudaFree or other allocating routine.  The first call on each device
+ * looks up the array's device address (cudaGetSymbolAddress, with that device current); make
+ * that first call outside any stream capture.
+ *
+ * Limits and errors: HGC_UNSUPPORTED if the layer is not one the tensor-core path takes (fewer
+ * than 9 channels per group, very wide rows ...: use hgc_conv_forward); HGC_NO_WORKSPACE if the
+ * layer needs more than the 32 MiB (256 B + K*R*S*c_w*2 + N*H*W*c_pad*2 bytes, channels rounded
+ * up); HGC_INVALID_ARG / HGC_BAD_ALIGNMENT as for hgc_conv_forward; HGC_CUDA_ERROR.  A
+ * device-side timeout cannot be read back through this entry point.
+ *
+ * All calls on a device share the one array, and it keeps the previous call's contents (the
+ * call clears the part that must start at zero).  Two calls whose GPU work overlaps - different
+ * streams, or different host threads - race on it: serialise them on one stream.
+ */
+int hgc_conv_forward_static(const hgc_conv_params* p, const void* x, const void* w, const void* bias,
+                            void* y, int relu, void* stream);
+
 /* Output shape N, K, P, Q of the descriptor (any output pointer may be NULL). */
 int hgc_conv_output_dims(const hgc_conv_desc* d, int32_t* n, int32_t* k, int32_t* p, int32_t* q);
 

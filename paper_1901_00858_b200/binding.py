@@ -50,6 +50,7 @@ def lib() -> ctypes.CDLL:
         L.hgc_conv_desc_destroy.argtypes = [vp]
         L.hgc_conv_forward.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int, vp]
         L.hgc_conv_forward_host.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int, vp]
+        L.hgc_conv_forward_static.argtypes = [ctypes.POINTER(hgc_conv_params), vp, vp, vp, vp, ctypes.c_int, vp]
         L.hgc_conv_output_dims.argtypes = [vp, i32p, i32p, i32p, i32p]
         L.hgc_conv_path.argtypes = [vp, i32p]
         L.hgc_conv_plan_info.argtypes = [vp, i32p, i32]
@@ -65,7 +66,7 @@ def lib() -> ctypes.CDLL:
         L.hgc_status_string.argtypes = [ctypes.c_int]
         L.hgc_status_string.restype = ctypes.c_char_p
         for name in ("hgc_conv_desc_create", "hgc_conv_desc_destroy", "hgc_conv_forward",
-                     "hgc_conv_forward_host", "hgc_conv_output_dims", "hgc_conv_path",
+                     "hgc_conv_forward_host", "hgc_conv_forward_static", "hgc_conv_output_dims", "hgc_conv_path",
                      "hgc_conv_workspace_bytes", "hgc_conv_host_workspace_bytes", "hgc_conv_plan_info",
                      "hgc_conv_set_workspace", "hgc_conv_set_weights", "hgc_conv_last_device_status",
                      "hgc_layout_nchw_to_nhwc", "hgc_layout_nhwc_to_nchw", "hgc_weights_repack",
@@ -196,6 +197,14 @@ def conv_forward_host(desc: ConvDesc, x, w, bias, y, relu: bool, stream=None):
     tensors or numpy arrays); copies are queued on the stream."""
     _check(lib().hgc_conv_forward_host(desc.handle, _ptr(x), _ptr(w), _ptr(bias), _ptr(y),
                                        int(bool(relu)), _stream(stream)), "hgc_conv_forward_host")
+
+
+def conv_forward_static(params: hgc_conv_params, x, w, bias, y, relu: bool, stream=None):
+    """hgc_conv_forward_static: the tensor-core layer with its scratch in the library's own fixed
+    device array, for callers that may not allocate device memory.  `params` is an
+    hgc_conv_params; x, w, bias (or None), y are CUDA fp16 tensors (or raw addresses)."""
+    _check(lib().hgc_conv_forward_static(ctypes.byref(params), _ptr(x), _ptr(w), _ptr(bias), _ptr(y),
+                                         int(bool(relu)), _stream(stream)), "hgc_conv_forward_static")
 
 
 def layout_nchw_to_nhwc(src, dst, n, c, h, w, c_pad, stream=None):
