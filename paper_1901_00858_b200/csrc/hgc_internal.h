@@ -33,6 +33,10 @@ cudaError_t launch_nchw_to_nhwc(const __half* src, __half* dst, int32_t n, int32
                                 int32_t w, int32_t c_pad, cudaStream_t stream);
 cudaError_t launch_nhwc_to_nchw(const __half* src, __half* dst, int32_t n, int32_t c, int32_t h,
                                 int32_t w, int32_t c_pad, cudaStream_t stream);
+cudaError_t launch_nchw_to_nhwc8_bordered(const __half* src, __half* dst, int32_t n, int32_t c, int32_t h, int32_t w,
+                                          int32_t pad_h, int32_t pad_w, int32_t hp, int32_t wp, cudaStream_t stream);
+cudaError_t launch_weights_repack_window(const __half* src, __half* dst, int32_t k, int32_t c, int32_t r, int32_t s,
+                                         int32_t kw_pix, cudaStream_t stream);
 cudaError_t launch_weights_repack(const __half* src, __half* dst, int32_t k, int32_t cg, int32_t r,
                                   int32_t s, int32_t group, int32_t c_pad, cudaStream_t stream);
 
@@ -40,6 +44,8 @@ cudaError_t launch_weights_repack(const __half* src, __half* dst, int32_t k, int
 struct IgemmPlan {
   int32_t kb, cblocks, cw, c_pad;
   int32_t halo, pitch;
+  int32_t window, kw_pix, hp, wp;                // few-channel layers: windows over a zero-bordered NHWC8 copy
+  int32_t eff_r, eff_s, eff_pad_h, eff_pad_w;    // the convolution as the kernel sees it
   int32_t tn, th, tw, ncols;
   int32_t tiles_h, tiles_n, mtiles, total_tiles;
   int32_t stages, taps;

@@ -755,17 +755,38 @@ int sm_count() {
 
 bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   IgemmPlan p{};
-  if (g.cg < 9) return false;                         // too few channels per tap for a K=16 MMA step
   if (g.group > 1 && (g.cg % 8) != 0) return false;  // group stride of x' must be 16-byte aligned
-  p.kb = g.cg > 32 ? 64 : (g.cg > 16 ? 32 : 16);
-  p.cblocks = (g.cg + p.kb - 1) / p.kb;
-  p.cw = p.cblocks * p.kb;
-  p.c_pad = (g.c + 7) / 8 * 8;
-  // stride 1: the S taps of a kernel row read one shared tile, shifted by s*dil pixels
-  p.halo = (g.stride_h == 1 && g.stride_w == 1) ? 1 : 0;
+  // Few input channels (image stems, C <= 8): a tap alone is too short for a K=16 MMA step.
+  // The input is copied to a zero-bordered NHWC buffer with 8 channels per pixel; the S taps of
+  // a kernel row are then S*8 CONTIGUOUS elements, read as one "window" per output pixel through
+  // a tensor map whose pixel stride (stride_w pixels) is smaller than the window.  The kernel
+  // sees a convolution with R taps (one per kernel row), no padding and kw_pix*8 channels.
+  p.window = (g.cg <= 8 && g.group == 1 && g.dil_w == 1) ? 1 : 0;
+  if (!p.window && g.cg < 9) return false;
+  if (p.window) {
+    const int kelems = g.s * 8 <= 16 ? 16 : g.s * 8 <= 32 ? 32 : (g.s * 8 + 63) / 64 * 64;
+    p.kw_pix = kelems / 8;
+    p.kb = kelems >= 64 ? 64 : kelems;
+    p.cblocks = kelems / p.kb;
+    p.cw = kelems;
+    p.c_pad = 8;
+    p.hp = g.h + 2 * g.pad_h;
+    p.wp = g.w + 2 * g.pad_w;
+    if (p.wp < (g.q - 1) * g.stride_w + p.kw_pix) p.wp = (g.q - 1) * g.stride_w + p.kw_pix;
+    p.eff_r = g.r; p.eff_s = 1; p.eff_pad_h = 0; p.eff_pad_w = 0;
+    p.halo = 0;
+  } else {
+    p.kb = g.cg > 32 ? 64 : (g.cg > 16 ? 32 : 16);
+    p.cblocks = (g.cg + p.kb - 1) / p.kb;
+    p.cw = p.cblocks * p.kb;
+    p.c_pad = (g.c + 7) / 8 * 8;
+    p.eff_r = g.r; p.eff_s = g.s; p.eff_pad_h = g.pad_h; p.eff_pad_w = g.pad_w;
+    // stride 1: the S taps of a kernel row read one shared tile, shifted by s*dil pixels
+    p.halo = (g.stride_h == 1 && g.stride_w == 1) ? 1 : 0;
+  }
   p.pitch = p.halo ? g.q + (g.s - 1) * g.dil_w : g.q;
   p.tw = g.q;
-  const int box_w = p.halo ? p.pitch : g.q * g.stride_w;
+  const int box_w = p.halo ? p.pitch : (p.window ? g.q : g.q * g.stride_w);
   if (p.pitch > 256 || box_w > 256) return false;
   p.mtiles = (g.kg + 127) / 128;
   const int64_t mg = (int64_t)p.mtiles * g.group;
@@ -824,7 +845,7 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   // ring of stages: one activation tile + `taps` weight tiles each, at least two deep; if the
   // S taps of a kernel row do not fit twice, fall back to one tap (and its own tile) per stage
   for (;;) {
-    p.taps = p.halo ? g.s : 1;
+    p.taps = p.halo ? p.eff_s : 1;
     p.pitch = p.halo ? g.q + (g.s - 1) * g.dil_w : g.q;
     const uint32_t box_rows2 = (uint32_t)(p.tn * p.th * p.pitch);
     p.b_bytes = box_rows2 * p.kb * 2u;
@@ -847,8 +868,9 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   // workspace: status word, re-laid-out weights, NHWC input
   p.ws_status_off = 0;
   p.ws_w_off = 256;
-  p.ws_x_off = p.ws_w_off + round_up_sz((size_t)g.k * g.r * g.s * p.cw * 2, 256);
-  p.ws_total = p.ws_x_off + round_up_sz((size_t)g.n * g.h * g.w * p.c_pad * 2, 256);
+  p.ws_x_off = p.ws_w_off + round_up_sz((size_t)g.k * p.eff_r * p.eff_s * p.cw * 2, 256);
+  p.ws_total = p.ws_x_off + round_up_sz(p.window ? (size_t)g.n * p.hp * p.wp * 16 + 256
+                                                 : (size_t)g.n * g.h * g.w * p.c_pad * 2, 256);
   *out = p;
   return true;
 }
@@ -862,7 +884,7 @@ bool igemm_encode_maps(const ConvGeom& g, IgemmPlan* p, void* ws) {
                                : p->kb == 32 ? CU_TENSOR_MAP_SWIZZLE_64B
                                              : CU_TENSOR_MAP_SWIZZLE_32B;
   {
-    const cuuint64_t kred = (cuuint64_t)g.r * g.s * p->cw;
+    const cuuint64_t kred = (cuuint64_t)p->eff_r * p->eff_s * p->cw;
     cuuint64_t dims[3] = {kred, (cuuint64_t)g.kg, (cuuint64_t)g.group};
     cuuint64_t strides[2] = {kred * 2, kred * 2 * (cuuint64_t)g.kg};
     cuuint32_t box[3] = {(cuuint32_t)p->kb, 128, 1};
@@ -872,7 +894,20 @@ bool igemm_encode_maps(const ConvGeom& g, IgemmPlan* p, void* ws) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return false;
   }
-  {
+  if (p->window) {
+    // (window element, -, output column, padded input row, image): the column stride is stride_w
+    // pixels of 16 bytes, i.e. consecutive windows overlap
+    const cuuint64_t pix = 16;
+    cuuint64_t dims[5] = {(cuuint64_t)p->cw, 1, (cuuint64_t)g.q, (cuuint64_t)p->hp, (cuuint64_t)g.n};
+    cuuint64_t strides[4] = {pix, pix * (cuuint64_t)g.stride_w, pix * (cuuint64_t)p->wp,
+                             pix * (cuuint64_t)p->wp * (cuuint64_t)p->hp};
+    cuuint32_t box[5] = {(cuuint32_t)p->kb, 1, (cuuint32_t)p->tw, (cuuint32_t)(p->th * g.stride_h), (cuuint32_t)p->tn};
+    cuuint32_t es[5] = {1, 1, 1, (cuuint32_t)g.stride_h, 1};
+    if (enc(&p->tmB, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, base + p->ws_x_off, dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return false;
+  } else {
     const cuuint64_t cdim = g.group > 1 ? (cuuint64_t)g.cg : (cuuint64_t)p->c_pad;
     const cuuint64_t pix = (cuuint64_t)p->c_pad * 2;
     cuuint64_t dims[5] = {cdim, (cuuint64_t)g.group, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.n};
@@ -916,7 +951,7 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
   IgemmArgs a{};
   a.N = g.n; a.K = g.k; a.P = g.p; a.Q = g.q;
   a.kg = g.kg; a.group = g.group;
-  a.R = g.r; a.S = g.s; a.pad_h = g.pad_h; a.pad_w = g.pad_w;
+  a.R = p.eff_r; a.S = p.eff_s; a.pad_h = p.eff_pad_h; a.pad_w = p.eff_pad_w;
   a.stride_h = g.stride_h; a.stride_w = g.stride_w; a.dil_h = g.dil_h; a.dil_w = g.dil_w;
   a.kb = p.kb; a.cblocks = p.cblocks; a.cw = p.cw;
   a.halo = p.halo; a.tn = p.tn; a.th = p.th; a.pitch = p.pitch; a.ncols = p.ncols;

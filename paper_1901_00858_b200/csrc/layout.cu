@@ -128,7 +128,71 @@ __global__ void weights_repack_kernel(const uint16_t* __restrict__ src, uint16_t
   }
 }
 
+// x[n][c][h][w] (c <= 8) -> x'[n][hp][wp][8]: pixel (h, w) lands at (h + pad_h, w + pad_w); the
+// border, the extra columns and channels c..7 are zero.  One thread per output pixel (16 bytes).
+__global__ void __launch_bounds__(256)
+nchw_to_nhwc8_bordered_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int h, int w,
+                              int pad_h, int pad_w, int hp, int wp, int64_t total) {
+  const int64_t hw = (int64_t)h * w;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int ow = (int)(i % wp);
+    const int64_t t = i / wp;
+    const int oh = (int)(t % hp);
+    const int64_t n = t / hp;
+    const int ih = oh - pad_h, iw = ow - pad_w;
+    uint32_t o[4] = {0, 0, 0, 0};
+    if (ih >= 0 && ih < h && iw >= 0 && iw < w) {
+      const uint16_t* s = src + n * c * hw + (int64_t)ih * w + iw;
+#pragma unroll
+      for (int ch = 0; ch < 8; ++ch)
+        if (ch < c) o[ch >> 1] |= (uint32_t)s[ch * hw] << ((ch & 1) * 16);
+    }
+    *reinterpret_cast<uint4*>(dst + i * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
+// w[k][c][r][s] (c <= 8) -> w'[k][r][kw_pix][8]: tap s, channel ch at [s][ch]; zeros elsewhere.
+__global__ void weights_repack_window_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst,
+                                             int64_t k, int c, int r, int s, int kw_pix) {
+  const int64_t total = k * r * kw_pix;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int sp = (int)(i % kw_pix);
+    const int64_t t = i / kw_pix;
+    const int rr = (int)(t % r);
+    const int64_t kk = t / r;
+    uint32_t o[4] = {0, 0, 0, 0};
+    if (sp < s) {
+#pragma unroll
+      for (int ch = 0; ch < 8; ++ch)
+        if (ch < c) o[ch >> 1] |= (uint32_t)src[((kk * c + ch) * r + rr) * s + sp] << ((ch & 1) * 16);
+    }
+    *reinterpret_cast<uint4*>(dst + i * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_nchw_to_nhwc8_bordered(const __half* src, __half* dst, int32_t n, int32_t c, int32_t h, int32_t w,
+                                          int32_t pad_h, int32_t pad_w, int32_t hp, int32_t wp, cudaStream_t stream) {
+  const int64_t total = (int64_t)n * hp * wp;
+  int64_t blocks = (total + 255) / 256;
+  if (blocks > 148 * 32) blocks = 148 * 32;
+  nchw_to_nhwc8_bordered_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
+      reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), c, h, w, pad_h, pad_w, hp, wp, total);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_weights_repack_window(const __half* src, __half* dst, int32_t k, int32_t c, int32_t r, int32_t s,
+                                         int32_t kw_pix, cudaStream_t stream) {
+  const int64_t total = (int64_t)k * r * kw_pix;
+  int64_t blocks = (total + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  weights_repack_window_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
+      reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), k, c, r, s, kw_pix);
+  count_launch();
+  return cudaGetLastError();
+}
 
 cudaError_t launch_nchw_to_nhwc(const __half* src, __half* dst, int32_t n, int32_t c, int32_t h,
                                 int32_t w, int32_t c_pad, cudaStream_t stream) {

@@ -56,8 +56,9 @@ def test_static_scratch_matches_ordinary_entry_point_twice_in_a_row(hgc):
 def test_static_scratch_rejects_what_it_cannot_hold(hgc):
     import torch
     dummy = torch.zeros(64, dtype=torch.float16, device="cuda")
-    # 3 input channels: not a tensor-core layer, this entry point has no variant for it
-    small = hgc.hgc_conv_params(1, 3, 8, 8, 4, 3, 3, 1, 1, 1, 1, 1, 1, 1, 0)
+    # two groups of 3 channels: not a layer the tensor-core path takes, so this entry point has
+    # no variant for it
+    small = hgc.hgc_conv_params(1, 6, 8, 8, 4, 3, 3, 1, 1, 1, 1, 1, 1, 2, 0)
     with pytest.raises(hgc.HgcError) as e:
         hgc.conv_forward_static(small, dummy, dummy, None, dummy, False)
     assert e.value.status == hgc.HGC_UNSUPPORTED
