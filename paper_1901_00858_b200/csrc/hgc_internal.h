@@ -50,7 +50,7 @@ struct IgemmPlan {
   int32_t tiles_h, tiles_n, mtiles, total_tiles;
   int32_t stages, taps;
   uint32_t stage_bytes;
-  int32_t tma_store, rem;
+  int32_t tma_store, rem, nbuf;
   void* y_mapped;  // output pointer tmY/tmYr were encoded for
   uint32_t a_bytes, b_bytes, b_alloc;
   size_t smem_bytes;

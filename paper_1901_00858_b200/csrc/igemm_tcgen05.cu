@@ -23,7 +23,6 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
-#include <cstdlib>
 
 #include "hgc_internal.h"
 
@@ -33,7 +32,8 @@ namespace {
 constexpr int kEpilogueWarps = 8;  // two per TMEM lane quarter
 constexpr int kIgemmThreads = 64 + 32 * kEpilogueWarps;
 constexpr int kPassElems = 64;               // output pixels per channel staged per TMA store
-constexpr uint32_t kStageBufBytes = 128u * kPassElems * 2u;  // 128 channels x 64 pixels, fp16
+constexpr uint32_t kWarpStageBytes = 32u * kPassElems * 2u;  // one warp's staging tile: 32 channels x 64 pixels
+constexpr uint32_t kStageBufBytes = kEpilogueWarps * kWarpStageBytes;  // one such tile per epilogue warp
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -76,6 +76,12 @@ __device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity
   return ok;
 }
 
+__device__ __forceinline__ long long clk() {
+  long long t;
+  asm volatile("mov.u64 %0, %%clock64;" : "=l"(t)::"memory");
+  return t;
+}
+
 __device__ __forceinline__ uint64_t global_timer_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -85,13 +91,13 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 // Bounded wait: false if the limit expired or another role already gave up.  `sleep_ns` > 0
 // makes a waiting warp yield its issue slots between polls (the epilogue warps wait for whole
 // tiles and must not compete with the single TMA and MMA issuing threads).
-__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                             uint32_t sleep_ns) {
   uint64_t t0 = 0;
   for (uint32_t i = 0;; ++i) {
-    // sleeping waiters use the suspending form; the TMA and MMA warps poll without suspending
-    // (a suspended thread is woken a few hundred cycles after the phase completes)
-    if (sleep_ns ? mbar_try_wait(bar, parity) : mbar_test_wait(bar, parity)) return true;
+    // the suspending form: a waiting warp must not burn issue slots or shared-memory bandwidth
+    // that the working warps need
+    if (mbar_try_wait(bar, parity)) return true;
     if (sleep_ns) __nanosleep(sleep_ns);
     if ((i & 1023u) == 1023u) {
       if (*abort_flag) return false;
@@ -349,6 +355,69 @@ __device__ __forceinline__ void issue_mmas(uint32_t d_tmem, uint64_t adesc, uint
 #undef HGC_MMA_OPERANDS
 }
 
+// Direct epilogue (shapes the staged TMA-store epilogue does not take): one warp reads its 32
+// accumulator lanes 16 columns at a time and every thread stores the runs of its own channel
+// plane.  Kept out of line: it is long, and the hot loops of the kernel should stay compact in
+// the instruction cache.
+__device__ __noinline__ void epilogue_direct(uint32_t t_addr, int ncols, int tn, int th, int pitch, int N, int K,
+                                             int P, int Q, int n0, int p0, int k, bool kvalid, float bv, bool relu,
+                                             uint16_t* yb) {
+  const int64_t pq = (int64_t)P * Q;
+  // running position of column j: image `img`, tile row `hr`, column `wc` within the pitch
+  int img = 0, hr = 0, wc = 0;
+#pragma unroll 1
+  for (int col0 = 0; col0 < ncols; col0 += 16) {
+    uint32_t v[16];
+    tmem_ld16(t_addr + (uint32_t)col0, v);
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int h8 = 0; h8 < 2; ++h8) {
+      uint32_t o[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        o[e] = pack_f16x2(__uint_as_float(v[h8 * 8 + 2 * e]) + bv, __uint_as_float(v[h8 * 8 + 2 * e + 1]) + bv, relu);
+      const int n = n0 + img, p = p0 + hr;
+      const bool rowvalid = kvalid && img < tn && n < N && p < P;
+      uint16_t* dst = yb + ((int64_t)n * K + k) * pq + (int64_t)p * Q + wc;
+      if (wc + 8 <= Q) {
+        // the 8 columns are 8 consecutive output pixels of one row
+        if (rowvalid) {
+          const uintptr_t ad = reinterpret_cast<uintptr_t>(dst);
+          if ((ad & 15u) == 0) {
+            *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
+          } else if ((ad & 3u) == 0) {
+            uint32_t* d32 = reinterpret_cast<uint32_t*>(dst);
+            d32[0] = o[0]; d32[1] = o[1]; d32[2] = o[2]; d32[3] = o[3];
+          } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) dst[e] = (uint16_t)((o[e >> 1] >> ((e & 1) * 16)) & 0xffffu);
+          }
+        }
+        wc += 8;
+        if (wc >= pitch) {  // only when pitch == Q and Q % 8 == 0
+          wc = 0;
+          if (++hr == th) { hr = 0; ++img; }
+        }
+      } else {
+        // the chunk runs over the end of a row (junk columns and/or the next row)
+        int im2 = img, hr2 = hr, wc2 = wc;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int n2 = n0 + im2, p2 = p0 + hr2;
+          if (kvalid && wc2 < Q && im2 < tn && n2 < N && p2 < P)
+            yb[((int64_t)n2 * K + k) * pq + (int64_t)p2 * Q + wc2] = (uint16_t)((o[e >> 1] >> ((e & 1) * 16)) & 0xffffu);
+          if (++wc2 == pitch) {
+            wc2 = 0;
+            if (++hr2 == th) { hr2 = 0; ++im2; }
+          }
+        }
+        img = im2; hr = hr2; wc = wc2;
+      }
+    }
+    __syncwarp();  // tcgen05.ld is warp-collective: reconverge before the next one
+  }
+}
+
 struct IgemmArgs {
   int32_t N, K, P, Q;
   int32_t kg, group;
@@ -373,7 +442,7 @@ struct IgemmArgs {
   int32_t relu;
   int32_t tma_store;  // 1: the epilogue stages fp16 tiles in shared memory and stores them with TMA
   int32_t rem;        // (th*Q) % 64: width of the last staged pass of a full tile (0 = none)
-  int32_t debug;      // timing experiments only (results are wrong): 1 = no TMA loads, 2 = no MMAs
+  int32_t nbuf;       // staging tiles per epilogue warp (1 or 2)
 };
 
 constexpr int kMaxStages = 8;
@@ -452,22 +521,18 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         int acol = cb * KB;  // column of w' for tap (r, s): (r*S + s)*cw + cb*KB
         for (int r = 0; r < a.R && ok; ++r) {
           for (int sg = 0; sg < groups_per_row; ++sg) {
-            if (!mbar_wait(smem_u32(&empty_bar[ring.idx]), ring.phase ^ 1u, &abort_flag, 32)) {
+            if (!mbar_wait(smem_u32(&empty_bar[ring.idx]), ring.phase ^ 1u, &abort_flag, 64)) {
               ok = false;
               break;
             }
             const uint32_t fb = smem_u32(&full_bar[ring.idx]);
             const uint32_t sbase = ring_base + ring.idx * a.stage_bytes;
             if (elect_one()) {
-              if (a.debug & 1) {
-                mbar_arrive(fb);
-              } else {
-                mbar_expect_tx(fb, a.b_bytes + (uint32_t)a.taps * a.a_bytes);
-                tma_load_5d(sbase, &tmB, fb, cb * KB, grp, (HALO ? 0 : sg * a.dil_w) - a.pad_w,
-                            h_base + r * a.dil_h, n0);
-                for (int t = 0; t < a.taps; ++t)
-                  tma_load_3d(sbase + a.b_alloc + (uint32_t)t * a.a_bytes, &tmA, fb, acol + t * a.cw, m0, grp);
-              }
+              mbar_expect_tx(fb, a.b_bytes + (uint32_t)a.taps * a.a_bytes);
+              tma_load_5d(sbase, &tmB, fb, cb * KB, grp, (HALO ? 0 : sg * a.dil_w) - a.pad_w, h_base + r * a.dil_h,
+                          n0);
+              for (int t = 0; t < a.taps; ++t)
+                tma_load_3d(sbase + a.b_alloc + (uint32_t)t * a.a_bytes, &tmA, fb, acol + t * a.cw, m0, grp);
             }
             __syncwarp();
             acol += a.taps * a.cw;
@@ -502,14 +567,14 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const uint32_t tap_step = (uint32_t)a.dil_w * row_bytes;  // halo mode: tap s starts s*dil pixels in
     const uint64_t desc_hi = a.desc_hi;
     const uint32_t idesc = a.idesc;
-    const uint32_t do_mma = (a.debug & 2) ? 0u : 1u;
+    const uint32_t do_mma = 1u;
     const int groups_per_row = a.S / a.taps;
     const int groups_per_tile = a.cblocks * a.R * groups_per_row;
     uint32_t ready = mbar_test_wait(smem_u32(&full_bar[0]), 0u);
     for (int tile = blockIdx.x; tile < a.total_tiles && ok; tile += gridDim.x, ++lt) {
       const uint32_t buf = lt & 1u;
       // the epilogue must have drained this accumulator (two tiles ago)
-      if (!mbar_wait(smem_u32(&acc_empty[buf]), ((lt >> 1) & 1u) ^ 1u, &abort_flag)) {
+      if (!mbar_wait(smem_u32(&acc_empty[buf]), ((lt >> 1) & 1u) ^ 1u, &abort_flag, 64)) {
         ok = false;
         break;
       }
@@ -552,17 +617,16 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const int quarter = warp & 3;
     const int half = ew >> 2;
     const int row = quarter * 32 + lane;  // accumulator lane = output channel within the tile
-    const int64_t pq = (int64_t)a.P * a.Q;
     uint16_t* yb = reinterpret_cast<uint16_t*>(y);
     const uint32_t stage_base = ring_base + (uint32_t)a.stages * a.stage_bytes;
-    const bool issuer = (ew == 0 && lane == 0);
     const bool relu = a.relu != 0;
+    // this warp's own staging tiles: 32 channel rows of 128 bytes each, 128-byte swizzled
+    const uint32_t my_stage = stage_base + (uint32_t)ew * (uint32_t)a.nbuf * kWarpStageBytes;
+    const uint32_t row_off = (uint32_t)lane * 128u + (((uint32_t)lane & 7u) << 4);
+    uint32_t unit_ctr = 0;
     const int mgn = a.mtiles * a.group;
-    uint32_t lt = 0, pass_ctr = 0;
-    long long e_wait = 0;
-    const long long e_start = clock64();
+    uint32_t lt = 0;
     for (int tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x, ++lt) {
-      if (a.debug & 1024) break;  // timing experiment: no epilogue at all
       const int px = tile / mgn;
       const int mg = tile - px * mgn;
       const int grp = mg / a.mtiles;
@@ -574,141 +638,97 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       const int k = grp * a.kg + (kvalid ? kin : 0);
       const float bv = (bias != nullptr && kvalid) ? __half2float(__ldg(bias + k)) : 0.f;
       const uint32_t buf = lt & 1u;
-      const long long tw0 = clock64();
-      mbar_wait(smem_u32(&acc_full[buf]), (lt >> 1) & 1u, &abort_flag, 256);
-      // all epilogue warps take the same decision: a warp that gave up has raised the flag
-      asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpilogueWarps) : "memory");
-      const long long tw1 = clock64();
-      e_wait += tw1 - tw0;
-      if (abort_flag) break;
+      if (!mbar_wait(smem_u32(&acc_full[buf]), (lt >> 1) & 1u, &abort_flag, 256)) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t t_addr = tmem_base + buf * 256u + ((uint32_t)(quarter * 32) << 16);
+      const bool quarter_live = m0 + quarter * 32 < a.kg;  // any real output channel in this warp's lanes?
 
       if (a.tma_store) {
         // ---- staged epilogue: TMEM -> registers -> swizzled fp16 tile in smem -> TMA store ----
-        // (taken when Q % 8 == 0, P*Q % 8 == 0 and a tile holds one image: every staged run of
-        //  pixels then starts on a 16-byte boundary of y)
-        const int rows_valid = (a.P - p0) < a.th ? (a.P - p0) : a.th;
-        const int e_valid = rows_valid * a.Q;  // output pixels of one channel in this tile
-        const int npass = (e_valid + kPassElems - 1) / kPassElems;
-        const bool last_row_tile = p0 + a.th >= a.P;
-        for (int pass = 0; pass < npass; ++pass, ++pass_ctr) {
-          const uint32_t sbuf = stage_base + (pass_ctr & 1u) * kStageBufBytes;
-          const int e_lo = pass * kPassElems;
-          const int e_hi = e_lo + kPassElems < e_valid ? e_lo + kPassElems : e_valid;
-          const int e0 = e_lo + half * (kPassElems / 2);
-          const int e1 = e0 + kPassElems / 2 < e_hi ? e0 + kPassElems / 2 : e_hi;
-          if (e0 < e1) {
-            int hr = e0 / a.Q;
-            int wc = e0 - hr * a.Q;
-            uint32_t col = (uint32_t)(hr * a.pitch + wc);
-            for (int e = e0; e < e1; e += 8) {
-              uint32_t v[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-              if (!(a.debug & 16)) {
-                tmem_ld8(t_addr + col, v);
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        // (taken when Q % 8 == 0, hence P*Q % 8 == 0, and a tile holds one image: every staged run
+        //  of pixels then starts on a 16-byte boundary of y).  A unit of work is 32 channels (this
+        //  warp's TMEM lanes) x 64 consecutive output pixels; the two warps of a lane quarter take
+        //  alternate units.  Each warp owns its staging tiles and issues its own stores, so the
+        //  epilogue warps never wait for one another.
+        if (quarter_live) {
+          const int rows_valid = (a.P - p0) < a.th ? (a.P - p0) : a.th;
+          const int e_valid = rows_valid * a.Q;  // output pixels of one channel in this tile
+          const bool last_row_tile = p0 + a.th >= a.P;
+          // (row, column) of the unit's first pixel, kept up to date without divisions
+          int hr = 0, wc = half * kPassElems;
+          while (wc >= a.Q) { wc -= a.Q; ++hr; }
+          for (int e_lo = half * kPassElems; e_lo < e_valid; e_lo += 2 * kPassElems, ++unit_ctr) {
+            const int e_hi = e_lo + kPassElems < e_valid ? e_lo + kPassElems : e_valid;
+            const uint32_t sbuf = my_stage + (unit_ctr % (uint32_t)a.nbuf) * kWarpStageBytes;
+            int uh = hr, uw = wc;  // walks through this unit
+#pragma unroll 1
+            for (int g = 0; g < 2; ++g) {
+              const int e0 = e_lo + g * 32;
+              if (e0 >= e_hi) break;
+              const int nchunks = (e_hi - e0) >= 32 ? 4 : (e_hi - e0) >> 3;
+              uint32_t cols[4];
+#pragma unroll
+              for (int c = 0; c < 4; ++c) {
+                cols[c] = (uint32_t)(uh * a.pitch + uw);
+                uw += 8;
+                if (uw == a.Q) { uw = 0; ++uh; }  // next output row: the junk columns of the pitch are skipped
               }
-              uint32_t o[4];
+              uint32_t v[4][8];
 #pragma unroll
-              for (int i = 0; i < 4; ++i)
-                o[i] = pack_f16x2(__uint_as_float(v[2 * i]) + bv, __uint_as_float(v[2 * i + 1]) + bv, relu);
-              const uint32_t chunk = (uint32_t)(e - e_lo) >> 3;
-              const uint32_t dst = sbuf + (uint32_t)row * 128u + ((chunk ^ ((uint32_t)row & 7u)) << 4);
-              if (!(a.debug & 32))
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]),
-                             "r"(o[3])
-                             : "memory");
-              wc += 8;
-              col += 8;
-              if (wc == a.Q) {  // next output row: skip the junk columns of the pitch
-                wc = 0;
-                col += (uint32_t)(a.pitch - a.Q);
+              for (int c = 0; c < 4; ++c)
+                if (c < nchunks) tmem_ld8(t_addr + cols[c], v[c]);
+              if (g == 0) {
+                // this buffer's previous store must have been read out of shared memory
+                if (lane == 0) {
+                  if (a.nbuf == 1) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                  else asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                }
+                __syncwarp();
               }
-            }
-          }
-          if (pass == npass - 1) asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          // the other staging buffer is free again once the store issued from it has been read
-          if (issuer) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-          asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpilogueWarps) : "memory");
-          if (pass == npass - 1 && lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
-          if (issuer && !(a.debug & 64)) {
-            const bool full_box = (e_hi - e_lo == kPassElems) || last_row_tile;  // past P*Q the store is clipped
-            tma_store_4d(full_box ? &tmY : &tmYr, sbuf, p0 * a.Q + e_lo, m0, grp, n0);
-            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-          }
-        }
-      } else {
-        // ---- direct epilogue: each thread stores runs of its own channel plane ----
-        if (half == 0) {
-          // running position of column j: image `img`, tile row `hr`, column `wc` within the pitch
-          int img = 0, hr = 0, wc = 0;
-          for (int col0 = 0; col0 < a.ncols; col0 += 16) {
-            uint32_t v[16];
-            tmem_ld16(t_addr + (uint32_t)col0, v);
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+              asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-            for (int h8 = 0; h8 < 2; ++h8) {
-              uint32_t o[4];
+              for (int c = 0; c < 4; ++c) {
+                if (c < nchunks) {
+                  uint32_t o[4];
 #pragma unroll
-              for (int e = 0; e < 4; ++e)
-                o[e] = pack_f16x2(__uint_as_float(v[h8 * 8 + 2 * e]) + bv, __uint_as_float(v[h8 * 8 + 2 * e + 1]) + bv,
-                                  relu);
-              const int n = n0 + img, p = p0 + hr;
-              const bool rowvalid = kvalid && img < a.tn && n < a.N && p < a.P;
-              uint16_t* dst = yb + ((int64_t)n * a.K + k) * pq + (int64_t)p * a.Q + wc;
-              if (wc + 8 <= a.Q) {
-                // the 8 columns are 8 consecutive output pixels of one row
-                if (rowvalid) {
-                  const uintptr_t ad = reinterpret_cast<uintptr_t>(dst);
-                  if ((ad & 15u) == 0) {
-                    *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
-                  } else if ((ad & 3u) == 0) {
-                    uint32_t* d32 = reinterpret_cast<uint32_t*>(dst);
-                    d32[0] = o[0]; d32[1] = o[1]; d32[2] = o[2]; d32[3] = o[3];
-                  } else {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) dst[e] = (uint16_t)((o[e >> 1] >> ((e & 1) * 16)) & 0xffffu);
-                  }
+                  for (int i = 0; i < 4; ++i)
+                    o[i] = pack_f16x2(__uint_as_float(v[c][2 * i]) + bv, __uint_as_float(v[c][2 * i + 1]) + bv, relu);
+                  const uint32_t dst = sbuf + (row_off ^ ((uint32_t)(g * 4 + c) << 4));
+                  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]),
+                               "r"(o[3])
+                               : "memory");
                 }
-                wc += 8;
-                if (wc >= a.pitch) {  // only when pitch == Q and Q % 8 == 0
-                  wc = 0;
-                  if (++hr == a.th) { hr = 0; ++img; }
-                }
-              } else {
-                // the chunk runs over the end of a row (junk columns and/or the next row)
-                int im2 = img, hr2 = hr, wc2 = wc;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                  const int n2 = n0 + im2, p2 = p0 + hr2;
-                  if (kvalid && wc2 < a.Q && im2 < a.tn && n2 < a.N && p2 < a.P)
-                    yb[((int64_t)n2 * a.K + k) * pq + (int64_t)p2 * a.Q + wc2] =
-                        (uint16_t)((o[e >> 1] >> ((e & 1) * 16)) & 0xffffu);
-                  if (++wc2 == a.pitch) {
-                    wc2 = 0;
-                    if (++hr2 == a.th) { hr2 = 0; ++im2; }
-                  }
-                }
-                img = im2; hr = hr2; wc = wc2;
               }
             }
-            __syncwarp();  // tcgen05.ld is warp-collective: reconverge before the next one
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+              const bool full_box = (e_hi - e_lo == kPassElems) || last_row_tile;  // past P*Q the store is clipped
+              tma_store_4d(full_box ? &tmY : &tmYr, sbuf, p0 * a.Q + e_lo, m0 + quarter * 32, grp, n0);
+              asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            }
+            // first pixel of this warp's next unit: two units further on
+            wc += 2 * kPassElems;
+            while (wc >= a.Q) { wc -= a.Q; ++hr; }
           }
         }
         // this warp has read its lanes of the accumulator: hand the buffer back to the MMA issuer
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
+      } else {
+        // ---- direct epilogue: each thread stores runs of its own channel plane ----
+        if (half == 0)
+          epilogue_direct(t_addr, a.ncols, a.tn, a.th, a.pitch, a.N, a.K, a.P, a.Q, n0, p0, k, kvalid, bv, relu, yb);
+        // this warp has read its lanes of the accumulator: hand the buffer back to the MMA issuer
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
       }
-    }
-    if ((a.debug & 128) && blockIdx.x == 0 && status != nullptr && lane == 0 && ew < 2) {
-      long long* dbg = reinterpret_cast<long long*>(status) + 2 + 3 * ew;
-      dbg[0] = clock64() - e_start; dbg[1] = e_wait; dbg[2] = lt;
     }
     // the shared-memory tiles of outstanding stores must stay intact until they have been read,
     // and the stores themselves must be complete before the kernel ends
-    if (issuer) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -841,7 +861,8 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   p.rem = (p.th * g.q) % kPassElems;
   // rings: B two or three deep, A with what is left (each A stage feeds kb/16 MMAs).  227 KB per
   // CTA minus alignment slack, static barriers and the two epilogue staging buffers.
-  const size_t budget = 232448u - 1024u - 512u - 2u * kStageBufBytes;
+  const size_t budget_all = 232448u - 1024u - 512u;
+  const size_t budget = budget_all - kStageBufBytes;
   // ring of stages: one activation tile + `taps` weight tiles each, at least two deep; if the
   // S taps of a kernel row do not fit twice, fall back to one tap (and its own tile) per stage
   for (;;) {
@@ -861,7 +882,9 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
     p.halo = 0;
     p.ncols = (p.tn * p.th * g.q + 15) / 16 * 16;
   }
-  p.smem_bytes = (size_t)p.stages * p.stage_bytes + 2u * kStageBufBytes + 1024;
+  // a second staging tile per epilogue warp (its store overlaps the next unit) if memory is left
+  p.nbuf = ((size_t)p.stages * p.stage_bytes + 2u * kStageBufBytes <= budget_all) ? 2 : 1;
+  p.smem_bytes = (size_t)p.stages * p.stage_bytes + (size_t)p.nbuf * kStageBufBytes + 1024;
   // more than half of an SM's shared memory: at most one CTA per SM, so that the kernel can take
   // all 512 TMEM columns without ever waiting for another CTA to free them
   if (p.smem_bytes < 120u * 1024u) p.smem_bytes = 120u * 1024u;
@@ -934,7 +957,7 @@ bool igemm_encode_y_maps(const ConvGeom& g, IgemmPlan* p, void* y) {
   cuuint64_t strides[3] = {pq * 2, pq * 2 * (cuuint64_t)g.kg, pq * 2 * (cuuint64_t)g.k};
   cuuint32_t es[4] = {1, 1, 1, 1};
   for (int i = 0; i < 2; ++i) {
-    cuuint32_t box[4] = {(cuuint32_t)((i == 0 || p->rem == 0) ? kPassElems : p->rem), 128, 1, 1};
+    cuuint32_t box[4] = {(cuuint32_t)((i == 0 || p->rem == 0) ? kPassElems : p->rem), 32, 1, 1};
     if (enc(i == 0 ? &p->tmY : &p->tmYr, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, y, dims, strides, box, es,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -968,10 +991,7 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
   a.relu = relu;
   a.tma_store = p.tma_store;
   a.rem = p.rem;
-  {
-    static const char* dbg = getenv("HGC_IGEMM_DEBUG");
-    a.debug = dbg ? atoi(dbg) : 0;
-  }
+  a.nbuf = p.nbuf;
   const int sms = sm_count();
   dim3 grid((unsigned)(p.total_tiles < sms ? p.total_tiles : sms));
   int* status = reinterpret_cast<int*>(static_cast<char*>(ws) + p.ws_status_off);
