@@ -57,6 +57,21 @@ def load_peaks():
     return dict(FALLBACK_PEAKS, source="fallback")
 
 
+def measured_traffic(workload: str, kernel: str, subset: bool):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu capture of this
+    workload (profiles/traffic.txt: `workload kernel bytes_per_launch`), or None."""
+    if subset:
+        return None
+    path = os.path.join(ROOT, "profiles", "traffic.txt")
+    if not os.path.exists(path):
+        return None
+    for line in open(path):
+        parts = line.split()
+        if len(parts) >= 3 and not line.startswith("#") and parts[0] == workload and parts[1] == kernel:
+            return float(parts[2])
+    return None
+
+
 def layer_roof_seconds(batch, l, peaks) -> float:
     return max(layer_flops(batch, l) / (peaks["bf16_tflops_sustained"] * 1e12),
                layer_bytes(batch, l) / (peaks["hbm_gbs"] * 1e9))
@@ -71,7 +86,7 @@ def aggregate(per_rank_flops, per_rank_images, max_seconds_per_step):
 
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -85,13 +100,16 @@ class ClockSampler:
             self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=self.file, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    def stop(self, window=None):
+        """window = (t0, t1) host epoch seconds of the timed region: only samples inside it are
+        used if there are at least three, else every sample taken while the bench ran."""
+        import datetime
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "window": "timed region"}
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -101,20 +119,25 @@ class ClockSampler:
             self.proc.kill()
         self.file.flush()
         self.file.seek(0)
-        sm, smax, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = []
         for line in self.file.read().splitlines():
             parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 8:
+            if len(parts) < 9:
                 continue
             try:
-                sm.append(float(parts[0]))
-                smax.append(float(parts[1]))
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(parts[1]), float(parts[2]),
+                             [nm for nm, v in zip(names, parts[5:9]) if v.lower().startswith("active")]))
             except ValueError:
                 continue
-            for nm, v in zip(names, parts[4:8]):
-                if v.lower().startswith("active"):
-                    reasons.add(nm)
+        inside = [r for r in rows if window and window[0] <= r[0] <= window[1]]
+        if len(inside) < 3:
+            inside = rows
+            out["window"] = "whole bench run (timed region shorter than three samples)"
+        sm = [r[1] for r in inside]
+        smax = [r[2] for r in inside]
+        reasons = set(x for r in inside for x in r[3])
         self.file.close()
         try:
             os.unlink(self.file.name)
@@ -245,26 +268,27 @@ def run_ours(args, wl):
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
     for _ in range(max(args.warmup, 3)):
         one_step()
     barrier()
 
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     # timed region: exactly K steps between two events on the launching stream
     ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in state]
           for _ in range(args.steps)]
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches0 = hgc.kernel_launch_count()
     barrier()
+    host_t0 = time.time()
     t_start.record(stream)
     for s in range(args.steps):
         one_step(ev[s])
     t_end.record(stream)
     barrier()
+    host_t1 = time.time()
     launches = hgc.kernel_launch_count() - launches0
-    clocks = sampler.stop() if rank == 0 else None
     total_ms = t_start.elapsed_time(t_end)
     ms_per_step = total_ms / args.steps
 
@@ -304,6 +328,33 @@ def run_ours(args, wl):
         barrier()
         e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
+    # ---- the same step replayed as one CUDA graph (no per-launch host cost) -------------------
+    graph_ms = None
+    if not args.no_graph:
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(g, stream=side):
+                    for (d, x, w, b, y, l) in state:
+                        hgc.conv_forward(d, x, w, b, y, l.relu, side)
+            torch.cuda.synchronize()
+            for _ in range(3):
+                g.replay()
+            barrier()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            g0.record()
+            for _ in range(args.steps):
+                g.replay()
+            g1.record()
+            barrier()
+            graph_ms = g0.elapsed_time(g1) / args.steps
+        except Exception as exc:  # capture not possible: report why, keep the main numbers
+            graph_ms = None
+            graph_err = repr(exc)
+    clocks = sampler.stop((host_t0, host_t1)) if rank == 0 else None
+
     # ---- max over ranks ---------------------------------------------------------------------
     if world > 1:
         t = torch.tensor([ms_per_step, e2e_ms], dtype=torch.float64, device="cuda")
@@ -329,14 +380,15 @@ def run_ours(args, wl):
             e["launches"] += 1
         dom = max(by_path, key=lambda k: by_path[k]["ms"])
         e = by_path[dom]
-        if dom == "depthwise":
+        hbm_bound = e["bytes"] / (peaks["hbm_gbs"] * 1e9) > e["flops"] / (peaks["bf16_tflops_sustained"] * 1e12)
+        if dom == "depthwise" or hbm_bound:
             roof = {"bound": "hbm", "kernel": dom, "achieved": e["bytes"] / (e["ms"] * 1e-3) / 1e9,
                     "peak": peaks["hbm_gbs"], "unit": "GB/s"}
         else:
             roof = {"bound": "tensor", "kernel": dom, "achieved": e["flops"] / (e["ms"] * 1e-3) / 1e12,
                     "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"}
         roof["frac"] = roof["achieved"] / roof["peak"]
-        roof["traffic"] = None
+        roof["traffic"] = measured_traffic(wl.name, dom, bool(args.only or args.batch))
         roof["peak_source"] = peaks["source"]
         roof["share_of_step"] = e["ms"] / sum(layer_ms)
         roof["avg_launch_ms"] = e["ms"] / e["launches"]
@@ -363,6 +415,10 @@ def run_ours(args, wl):
             "gpu_launches": launches,
             "clocks": clocks,
         }
+        if graph_ms is not None:
+            line["graph_replay"] = {"ms_per_step": graph_ms, "tflops": step_flops / (graph_ms * 1e-3) / 1e12,
+                                    "images_per_s": batch / (graph_ms * 1e-3),
+                                    "note": "same step captured once and replayed as a CUDA graph, this rank"}
         if cpu is not None:
             line["cpu_baseline"] = cpu
         if args.layers:
@@ -379,13 +435,14 @@ def run_ours(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD,
                     help="one of: " + ", ".join(w.name for w in workloads.all_workloads()))
     ap.add_argument("--layers", action="store_true", help="add per-layer figures to the JSON line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     ap.add_argument("--only", default="", help="comma-separated layer names: run just these layers (profiling)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling on a small case)")
