@@ -102,9 +102,11 @@ depthwise3x3_kernel(DwPlan a, const uint16_t* __restrict__ x, const __half* __re
     const int r0 = p0 + (u % units_per_plane) * a.th;
     const int r1 = r0 + a.th < p1 ? r0 + a.th : p1;
     const int ch = (int)((pl0 + pl) % a.c);
-    float wv[9];
+    // weights and window stay binary16; products and sums use the mixed-precision FMA
+    // (f16 x f16 + f32 -> f32), so nothing is converted on the way in
+    uint16_t wv[9];
 #pragma unroll
-    for (int i = 0; i < 9; ++i) wv[i] = __half2float(__ldg(w + (int64_t)ch * 9 + i));
+    for (int i = 0; i < 9; ++i) wv[i] = __half_as_ushort(__ldg(w + (int64_t)ch * 9 + i));
     const float bv = bias != nullptr ? __half2float(__ldg(bias + ch)) : 0.f;
 
     const int q0 = cp * 2;
@@ -117,15 +119,15 @@ depthwise3x3_kernel(DwPlan a, const uint16_t* __restrict__ x, const __half* __re
     const int in_base = mis_in + pl * (int)hw - ih_lo * a.w + iw0;
     const int out_base = mis_out + pl * (int)pq - p0 * a.q + q0;
 
-    float win[3][NCOL];
-    auto load_row = [&](float (&dst)[NCOL], int ih) {
+    uint16_t win[3][NCOL];
+    auto load_row = [&](uint16_t (&dst)[NCOL], int ih) {
       const bool rv = (ih >= 0) && (ih < a.h);
       const uint16_t* src = sin + in_base + ih * a.w;
 #pragma unroll
       for (int j = 0; j < NCOL; ++j) {
         uint16_t bits = 0;
         if (rv && cvalid[j]) bits = src[j];
-        dst[j] = __half2float(__ushort_as_half(bits));
+        dst[j] = bits;
       }
     };
     int ih = r0 * S - a.pad_h;
@@ -147,8 +149,8 @@ depthwise3x3_kernel(DwPlan a, const uint16_t* __restrict__ x, const __half* __re
       for (int r = 0; r < 3; ++r)
 #pragma unroll
         for (int s = 0; s < 3; ++s) {
-          o0 = fmaf(win[r][s], wv[r * 3 + s], o0);
-          o1 = fmaf(win[r][s + S], wv[r * 3 + s], o1);
+          asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(o0) : "h"(win[r][s]), "h"(wv[r * 3 + s]));
+          asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(o1) : "h"(win[r][s + S]), "h"(wv[r * 3 + s]));
         }
       if (relu) {
         o0 = fmaxf(o0, 0.f);
@@ -185,6 +187,150 @@ depthwise3x3_kernel(DwPlan a, const uint16_t* __restrict__ x, const __half* __re
       }
     }
   }
+}
+
+
+// ---- row-vector kernel: planes whose rows are whole 16-byte vectors (W % 8 == 0) -----------------
+//
+// No shared memory and no block-wide synchronisation: a thread owns one 16-byte vector column (8
+// output pixels) of a strip of TH output rows.  It reads each input row it needs as one (stride 1)
+// or two (stride 2) aligned 16-byte vectors straight from global memory (consecutive lanes read
+// consecutive vectors), fetches the single halo pixel on its left (and right, at stride 1) from
+// the neighbouring lanes with warp shuffles, keeps a sliding window of three converted rows in
+// registers and writes one aligned 16-byte vector per output row.  Rows shared between strips are
+// re-read through L2.
+template <int S, int TH>
+__global__ void __launch_bounds__(256, 4)
+depthwise3x3_rowvec_kernel(const uint16_t* __restrict__ x, const __half* __restrict__ w,
+                           const __half* __restrict__ bias, uint16_t* __restrict__ y, int c, int h, int wd,
+                           int p, int q, int relu, int64_t total_items, int vec_per_row, int strips) {
+  // item = (plane, strip, vector); the vectors of a row are consecutive lanes.  32-bit index
+  // arithmetic (the launcher checks that the item count fits).
+  const uint32_t item = blockIdx.x * blockDim.x + threadIdx.x;
+  const bool live = item < (uint32_t)total_items;
+  const uint32_t it = live ? item : (uint32_t)total_items - 1u;
+  const int v = (int)(it % (uint32_t)vec_per_row);
+  const uint32_t t = it / (uint32_t)vec_per_row;
+  const int strip = (int)(t % (uint32_t)strips);
+  const int64_t plane = (int64_t)(t / (uint32_t)strips);
+  const int ch = (int)((uint32_t)(t / (uint32_t)strips) % (uint32_t)c);
+  const int lane = threadIdx.x & 31;
+
+  // weights stay binary16: the stencil uses the mixed-precision FMA of sm_100 (f16 x f16 + f32),
+  // so no input value is ever converted (the half->float converts run at a quarter of the FMA rate
+  // and were the bottleneck of this kernel)
+  uint16_t wv[9];
+#pragma unroll
+  for (int i = 0; i < 9; ++i) wv[i] = __half_as_ushort(__ldg(w + (int64_t)ch * 9 + i));
+  const float bv = bias != nullptr ? __half2float(__ldg(bias + ch)) : 0.f;
+
+  const uint16_t* xp = x + plane * (int64_t)h * wd;
+  uint16_t* yp = y + plane * (int64_t)p * q;
+  const int p_lo = strip * TH;
+  // neighbours inside the same row of vectors? (lanes of a warp run over consecutive items)
+  const bool has_left = v > 0 && lane > 0;
+  const bool has_right = v + 1 < vec_per_row && lane < 31;
+
+  // All input rows of the strip are requested up front (TH*S + 2 rows, one or two 16-byte vectors
+  // each): with only a few warps per SM the kernel lives on memory-level parallelism.
+  constexpr int NR = TH * S + 2 - (S - 1);  // stride 1: TH + 2 rows; stride 2: 2*TH + 1 rows
+  constexpr int NE = 8 * S + 2;             // converted row: elements [-1 .. 8*S] around the 8 outputs
+  uint4 ra[NR], rb[S == 2 ? NR : 1];
+  uint32_t left[NR], right[NR];
+  const int ih0 = p_lo * S - 1;  // pad == 1 (required by the launcher)
+#pragma unroll
+  for (int i = 0; i < NR; ++i) {
+    const int ih = ih0 + i;
+    const bool rv = ih >= 0 && ih < h;
+    ra[i] = make_uint4(0, 0, 0, 0);
+    if (S == 2) rb[i] = make_uint4(0, 0, 0, 0);
+    if (rv) {
+      const uint4* src = reinterpret_cast<const uint4*>(xp + (int64_t)ih * wd) + (int64_t)v * S;
+      ra[i] = __ldg(src);
+      if (S == 2 && (v * 2 + 1) * 8 < wd) rb[i] = __ldg(src + 1);  // the row may end after the first vector
+    }
+    // halo pixels that no neighbouring lane holds (warp boundary inside a row)
+    left[i] = 0;
+    right[i] = 0;
+    if (rv && !has_left && v > 0) left[i] = xp[(int64_t)ih * wd + (int64_t)v * 8 * S - 1];
+    if (S == 1 && rv && !has_right && v + 1 < vec_per_row) right[i] = xp[(int64_t)ih * wd + (int64_t)(v + 1) * 8];
+  }
+  // halo from the neighbouring lanes: last element of the left vector(s), first of the right one
+#pragma unroll
+  for (int i = 0; i < NR; ++i) {
+    const uint32_t my_last = (S == 2 ? rb[i].w : ra[i].w) >> 16;
+    const uint32_t my_first = ra[i].x & 0xffffu;
+    const uint32_t l = __shfl_up_sync(0xffffffffu, my_last, 1);
+    const uint32_t r = __shfl_down_sync(0xffffffffu, my_first, 1);
+    if (has_left) left[i] = l;
+    if (S == 1 && has_right) right[i] = r;
+  }
+
+  // one input row as 16-bit lanes: elements [-1 .. 8*S] around the 8 outputs
+  auto unpack_row = [&](uint16_t (&dst)[NE], int i) {
+    dst[0] = (uint16_t)left[i];
+    const uint32_t wa[4] = {ra[i].x, ra[i].y, ra[i].z, ra[i].w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      asm("mov.b32 {%0, %1}, %2;" : "=h"(dst[1 + 2 * e]), "=h"(dst[2 + 2 * e]) : "r"(wa[e]));
+    if (S == 2) {
+      const uint32_t wb[4] = {rb[i].x, rb[i].y, rb[i].z, rb[i].w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        asm("mov.b32 {%0, %1}, %2;" : "=h"(dst[9 + 2 * e]), "=h"(dst[10 + 2 * e]) : "r"(wb[e]));
+      dst[NE - 1] = 0;
+    } else {
+      dst[9] = (uint16_t)right[i];
+    }
+  };
+
+  uint16_t win[3][NE];
+#pragma unroll
+  for (int r = 0; r < TH; ++r) {
+    const int pr = p_lo + r;
+#pragma unroll
+    for (int rr = 0; rr < 3; ++rr) unpack_row(win[rr], r * S + rr);  // rows r*S .. r*S+2 of the strip
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float f[2];
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int col = (2 * j + e) * S;  // window index of the tap s = 0
+        float acc = bv;
+#pragma unroll
+        for (int rr = 0; rr < 3; ++rr)
+#pragma unroll
+          for (int ss = 0; ss < 3; ++ss)
+            asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(acc) : "h"(win[rr][col + ss]), "h"(wv[rr * 3 + ss]));
+        f[e] = acc;
+      }
+      // two results -> one packed pair, ReLU folded into the convert
+      if (relu)
+        asm("cvt.rn.relu.f16x2.f32 %0, %1, %2;" : "=r"(o[j]) : "f"(f[1]), "f"(f[0]));
+      else
+        asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(o[j]) : "f"(f[1]), "f"(f[0]));
+    }
+    if (live && pr < p) {
+      uint16_t* dst = yp + (int64_t)pr * q + (int64_t)v * 8;
+      if ((q & 7) == 0) {
+        *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
+      } else {  // q % 8 == 4: rows are 8-byte aligned and the last vector of a row is half full
+        reinterpret_cast<uint2*>(dst)[0] = make_uint2(o[0], o[1]);
+        if (v * 8 + 8 <= q) reinterpret_cast<uint2*>(dst)[1] = make_uint2(o[2], o[3]);
+      }
+    }
+  }
+}
+
+// shapes the row-vector kernel takes: pad 1, W % 8 == 0, whole output vectors per row
+bool rowvec_ok(const ConvGeom& g) {
+  if (g.pad_h != 1 || g.pad_w != 1) return false;
+  if ((g.w & 7) != 0) return false;
+  const int S = g.stride_h;
+  if (g.q * S != g.w) return false;               // stride 1: Q == W; stride 2: Q == W/2
+  if ((g.q & 7) != 0 && (g.q & 7) != 4) return false;  // output rows: whole 16-byte or 8-byte vectors
+  return true;
 }
 
 bool make_plan(const ConvGeom& g, DwPlan* plan) {
@@ -250,6 +396,25 @@ cudaError_t launch_depthwise3x3(const ConvGeom& g, const __half* x, const __half
                                 const __half* bias, __half* y, int relu, cudaStream_t stream) {
   DwPlan a;
   if (!make_plan(g, &a)) return cudaErrorInvalidConfiguration;
+  if (rowvec_ok(g)) {
+    const int TH = g.stride_h == 1 ? 4 : 2;  // output rows per thread (bounded by registers: all input rows are prefetched)
+    const int vec_per_row = (g.q + 7) / 8;
+    const int strips = (g.p + TH - 1) / TH;
+    const int64_t items = (int64_t)g.n * g.c * strips * vec_per_row;
+    const int64_t blocks = (items + 255) / 256;
+    if (items < 0x7fffffffLL) {
+      const uint16_t* xs0 = reinterpret_cast<const uint16_t*>(x);
+      uint16_t* ys0 = reinterpret_cast<uint16_t*>(y);
+      if (g.stride_h == 1)
+        depthwise3x3_rowvec_kernel<1, 4><<<(unsigned)blocks, 256, 0, stream>>>(xs0, w, bias, ys0, g.c, g.h, g.w, g.p,
+                                                                               g.q, relu, items, vec_per_row, strips);
+      else
+        depthwise3x3_rowvec_kernel<2, 2><<<(unsigned)blocks, 256, 0, stream>>>(xs0, w, bias, ys0, g.c, g.h, g.w, g.p,
+                                                                               g.q, relu, items, vec_per_row, strips);
+      count_launch();
+      return cudaGetLastError();
+    }
+  }
   const int64_t ctas = a.bands_per_plane == 1 ? (a.planes + a.planes_per_cta - 1) / a.planes_per_cta
                                                : a.planes * a.bands_per_plane;
   const size_t smem = (size_t)(a.smem_in + a.smem_out) * sizeof(uint16_t);

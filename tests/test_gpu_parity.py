@@ -110,6 +110,22 @@ def test_depthwise_planes(hgc, oracle, plane, stride):
         check_close(got2, oracle.conv_fast(oracle.ConvParams(**a), x, w, None, False), what="dw no bias")
 
 
+@pytest.mark.parametrize("h,w,stride", [(56, 56, 1), (112, 112, 1), (24, 40, 1), (9, 8, 1), (56, 56, 2), (112, 112, 2),
+                                        (40, 24, 2), (16, 8, 2), (30, 72, 2)])
+def test_depthwise_row_vector_shapes(hgc, oracle, h, w, stride):
+    """Planes whose rows are whole 16-byte vectors take the shuffle-based kernel: cover warp
+    boundaries inside rows, half-full last vectors (Q % 8 == 4) and ragged last strips."""
+    rng = np.random.default_rng(h * 7 + w + stride)
+    n, c = 2, 19
+    a = params_dict(n, c, h, w, c, 3, 3, 1, 1, stride, stride, 1, 1, c)
+    x, wt, b = workloads.random_layer_tensors(rng, n, c, h, w, c, 3, 3, c)
+    for relu, bias in ((True, b), (False, None)):
+        ref = oracle.conv_fast(oracle.ConvParams(**a), x, wt, bias, relu)
+        got, path = run_layer(hgc, a, x, wt, bias, relu)
+        assert path == hgc.HGC_PATH_DEPTHWISE
+        check_close(got, ref, what=f"dw rowvec {h}x{w} s{stride}")
+
+
 @pytest.mark.parametrize("cfg,batch", [(0, 1), (1, 1), (2, 1), (3, 1)])
 def test_configs_whole_tensor(hgc, oracle, cfg, batch):
     """Configs small enough for the oracle to compute every output."""
