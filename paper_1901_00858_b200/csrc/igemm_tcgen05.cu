@@ -32,7 +32,9 @@ namespace {
 constexpr int kEpilogueWarps = 8;  // two per TMEM lane quarter
 constexpr int kIgemmThreads = 64 + 32 * kEpilogueWarps;
 constexpr int kPassElems = 64;               // output pixels per channel staged per TMA store
-constexpr uint32_t kWarpStageBytes = 32u * kPassElems * 2u;  // one warp's staging tile: 32 channels x 64 pixels
+// one warp's staging tile: 32 channels x 64 pixels for the TMA-store epilogue (4 KB, 1024-byte
+// aligned), or 32 rows of 144 bytes for the row epilogue (4.5 KB)
+constexpr uint32_t kWarpStageBytes = 5120u;
 constexpr uint32_t kStageBufBytes = kEpilogueWarps * kWarpStageBytes;  // one such tile per epilogue warp
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
@@ -355,67 +357,125 @@ __device__ __forceinline__ void issue_mmas(uint32_t d_tmem, uint64_t adesc, uint
 #undef HGC_MMA_OPERANDS
 }
 
-// Direct epilogue (shapes the staged TMA-store epilogue does not take): one warp reads its 32
-// accumulator lanes 16 columns at a time and every thread stores the runs of its own channel
-// plane.  Kept out of line: it is long, and the hot loops of the kernel should stay compact in
-// the instruction cache.
-__device__ __noinline__ void epilogue_direct(uint32_t t_addr, int ncols, int tn, int th, int pitch, int N, int K,
-                                             int P, int Q, int n0, int p0, int k, bool kvalid, float bv, bool relu,
-                                             uint16_t* yb) {
-  const int64_t pq = (int64_t)P * Q;
-  // running position of column j: image `img`, tile row `hr`, column `wc` within the pitch
-  int img = 0, hr = 0, wc = 0;
-#pragma unroll 1
-  for (int col0 = 0; col0 < ncols; col0 += 16) {
-    uint32_t v[16];
-    tmem_ld16(t_addr + (uint32_t)col0, v);
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+// Row epilogue (every shape the TMA-store epilogue does not take: planes whose rows or sizes
+// are not multiples of 8 pixels, several images per tile).  A thread owns one output channel
+// (its TMEM lane); the pixels of one image that it holds are one contiguous run of y.  It
+// converts them 8 columns at a time into its own 144-byte row of shared memory, placed at the
+// same offset modulo 16 as the run has in global memory, and copies the row out with aligned
+// 16-byte stores (the ragged head and tail pixel by pixel).  Only the thread itself touches its
+// row, so no synchronisation is needed.  Kept out of line: the hot loops of the kernel should
+// stay compact in the instruction cache.
+constexpr int kRowRunElems = 56;     // pixels staged per flush (112 bytes + up to 14 bytes of phase)
+constexpr uint32_t kRowPitch = 144;  // bytes between the rows of neighbouring lanes (bank spread)
+
+__device__ __forceinline__ void flush_row(uint32_t srow, uint16_t* gdst, int len) {
+  // gdst: global address of the run's first pixel; the run starts at byte (gdst & 15) of srow
+  const uint32_t phase = (uint32_t)(reinterpret_cast<uintptr_t>(gdst) & 15u);
+  char* gbase = reinterpret_cast<char*>(gdst) - phase;
+  const uint32_t end = phase + 2u * (uint32_t)len;
+  for (uint32_t off = 0; off < end; off += 16) {
+    uint32_t v0, v1, v2, v3;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3) : "r"(srow + off));
+    if (off >= phase && off + 16 <= end) {
+      *reinterpret_cast<uint4*>(gbase + off) = make_uint4(v0, v1, v2, v3);
+    } else {
+      const uint32_t w[4] = {v0, v1, v2, v3};
 #pragma unroll
-    for (int h8 = 0; h8 < 2; ++h8) {
-      uint32_t o[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e)
-        o[e] = pack_f16x2(__uint_as_float(v[h8 * 8 + 2 * e]) + bv, __uint_as_float(v[h8 * 8 + 2 * e + 1]) + bv, relu);
-      const int n = n0 + img, p = p0 + hr;
-      const bool rowvalid = kvalid && img < tn && n < N && p < P;
-      uint16_t* dst = yb + ((int64_t)n * K + k) * pq + (int64_t)p * Q + wc;
-      if (wc + 8 <= Q) {
-        // the 8 columns are 8 consecutive output pixels of one row
-        if (rowvalid) {
-          const uintptr_t ad = reinterpret_cast<uintptr_t>(dst);
-          if ((ad & 15u) == 0) {
-            *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
-          } else if ((ad & 3u) == 0) {
-            uint32_t* d32 = reinterpret_cast<uint32_t*>(dst);
-            d32[0] = o[0]; d32[1] = o[1]; d32[2] = o[2]; d32[3] = o[3];
-          } else {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) dst[e] = (uint16_t)((o[e >> 1] >> ((e & 1) * 16)) & 0xffffu);
-          }
-        }
-        wc += 8;
-        if (wc >= pitch) {  // only when pitch == Q and Q % 8 == 0
-          wc = 0;
-          if (++hr == th) { hr = 0; ++img; }
-        }
-      } else {
-        // the chunk runs over the end of a row (junk columns and/or the next row)
-        int im2 = img, hr2 = hr, wc2 = wc;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const int n2 = n0 + im2, p2 = p0 + hr2;
-          if (kvalid && wc2 < Q && im2 < tn && n2 < N && p2 < P)
-            yb[((int64_t)n2 * K + k) * pq + (int64_t)p2 * Q + wc2] = (uint16_t)((o[e >> 1] >> ((e & 1) * 16)) & 0xffffu);
-          if (++wc2 == pitch) {
-            wc2 = 0;
-            if (++hr2 == th) { hr2 = 0; ++im2; }
-          }
-        }
-        img = im2; hr = hr2; wc = wc2;
+      for (int e = 0; e < 8; ++e) {
+        const uint32_t b = off + 2u * e;
+        if (b >= phase && b < end) *reinterpret_cast<uint16_t*>(gbase + b) = (uint16_t)((w[e >> 1] >> ((e & 1) * 16)) & 0xffffu);
       }
     }
-    __syncwarp();  // tcgen05.ld is warp-collective: reconverge before the next one
   }
+}
+
+__device__ __noinline__ void epilogue_rows(uint32_t t_addr, int col_begin, int col_end, int tn, int th, int pitch,
+                                           int N, int K, int P, int Q, int n0, int p0, int k, bool kvalid, float bv,
+                                           bool relu, uint16_t* yb, uint32_t srow) {
+  const int64_t pq = (int64_t)P * Q;
+  // walk the tile rows that intersect this warp's column range
+  int rowi = col_begin / pitch;
+  int wc = col_begin - rowi * pitch;  // column within the pitch (>= Q: junk)
+  int img = rowi / th;
+  int hr = rowi - img * th;
+  uint16_t* run = nullptr;  // global address of the first staged pixel of the current run
+  int fill = 0;             // pixels staged so far
+  uint32_t wpos = 0;        // byte position in srow of the next pixel
+  int col = col_begin;
+#pragma unroll 1
+  while (col < col_end && img < tn) {
+    // control flow below is the same for all lanes of the warp (the TMEM loads are
+    // warp-collective); a lane without a real channel only skips its stores
+    const bool row_ok = (n0 + img) < N && (p0 + hr) < P;
+    if (wc >= Q || !row_ok) {
+      // junk columns / rows past the plane: skip to the next tile row
+      col += pitch - wc;
+      wc = 0;
+      if (++hr == th) {
+        hr = 0;
+        ++img;
+        if (fill) {  // the next image is not contiguous
+          if (kvalid) flush_row(srow, run, fill);
+          fill = 0;
+        }
+      }
+      continue;
+    }
+    int cnt = Q - wc;
+    if (cnt > 8) cnt = 8;
+    if (cnt > col_end - col) cnt = col_end - col;
+    uint32_t v[8];
+    __syncwarp();
+    tmem_ld8(t_addr + (uint32_t)col, v);
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+    uint32_t o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      o[i] = pack_f16x2(__uint_as_float(v[2 * i]) + bv, __uint_as_float(v[2 * i + 1]) + bv, relu);
+    if (fill == 0) {
+      run = yb + ((int64_t)(n0 + img) * K + k) * pq + (int64_t)(p0 + hr) * Q + wc;
+      wpos = (uint32_t)(reinterpret_cast<uintptr_t>(run) & 15u);
+    }
+    const uint32_t dst = srow + wpos;
+    if (!kvalid) {
+      // nothing to stage for a lane beyond the group's last channel
+    } else if (cnt == 8 && (wpos & 15u) == 0) {
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+    } else if (cnt == 8 && (wpos & 7u) == 0) {
+      asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(dst), "r"(o[0]), "r"(o[1]) : "memory");
+      asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(dst + 8), "r"(o[2]), "r"(o[3]) : "memory");
+    } else if (cnt == 8 && (wpos & 3u) == 0) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst + 4 * i), "r"(o[i]) : "memory");
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        if (e < cnt)
+          asm volatile("st.shared.b16 [%0], %1;" ::"r"(dst + 2 * e), "h"((uint16_t)((o[e >> 1] >> ((e & 1) * 16)) & 0xffffu))
+                       : "memory");
+    }
+    fill += cnt;
+    wpos += 2u * (uint32_t)cnt;
+    col += cnt;
+    wc += cnt;
+    if (wc == pitch) {  // pitch == Q: straight on to the next row
+      wc = 0;
+      if (++hr == th) {
+        hr = 0;
+        ++img;
+        if (fill) {
+          if (kvalid) flush_row(srow, run, fill);
+          fill = 0;
+        }
+      }
+    }
+    if (fill > kRowRunElems - 8) {  // no room for another chunk
+      if (kvalid) flush_row(srow, run, fill);
+      fill = 0;
+    }
+  }
+  if (fill && kvalid) flush_row(srow, run, fill);
+  __syncwarp();
 }
 
 struct IgemmArgs {
@@ -718,8 +778,13 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
       } else {
         // ---- direct epilogue: each thread stores runs of its own channel plane ----
-        if (half == 0)
-          epilogue_direct(t_addr, a.ncols, a.tn, a.th, a.pitch, a.N, a.K, a.P, a.Q, n0, p0, k, kvalid, bv, relu, yb);
+        {
+          // the two warps of a lane quarter take the first and the second half of the columns
+          const int split = ((a.ncols >> 1) + 15) & ~15;
+          if (quarter_live)
+            epilogue_rows(t_addr, half ? split : 0, half ? a.ncols : split, a.tn, a.th, a.pitch, a.N, a.K, a.P, a.Q, n0,
+                          p0, k, kvalid, bv, relu, yb, my_stage + (uint32_t)lane * kRowPitch);
+        }
         // this warp has read its lanes of the accumulator: hand the buffer back to the MMA issuer
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncwarp();

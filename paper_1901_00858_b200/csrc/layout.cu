@@ -62,6 +62,38 @@ nchw_to_nhwc_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst
   }
 }
 
+// x[n][c][hw] -> x'[n][hw][c_pad] for SMALL planes whose size is not a multiple of 8 (7x7, 14x14,
+// 13x13 ...): the rows of such planes are not 16-byte aligned, but 64 consecutive channel planes
+// of one image are one contiguous, 16-byte aligned span (when C*hw % 8 == 0).  A CTA copies that
+// span into shared memory with 16-byte vectors and writes whole-pixel 16-byte vectors out.
+__global__ void __launch_bounds__(kThreads)
+nchw_to_nhwc_smallplane_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int hw,
+                               int c_pad) {
+  extern __shared__ __align__(16) uint16_t flat[];  // [kTileC][hw]
+  const int64_t n = blockIdx.y;
+  const int c0 = blockIdx.x * kTileC;
+  const int nch = c - c0 < kTileC ? c - c0 : kTileC;   // real channels in this tile (may be <= 0)
+  const int span = nch > 0 ? nch * hw : 0;             // elements to copy
+  const uint16_t* s = src + (n * c + c0) * (int64_t)hw;
+  const int nvec = span >> 3;
+  for (int v = threadIdx.x; v < nvec; v += kThreads)
+    reinterpret_cast<uint4*>(flat)[v] = __ldg(reinterpret_cast<const uint4*>(s) + v);
+  for (int e = (nvec << 3) + threadIdx.x; e < span; e += kThreads) flat[e] = s[e];
+  __syncthreads();
+  uint16_t* d = dst + n * (int64_t)hw * c_pad;
+  const int cvecs = (c_pad - c0 < kTileC ? c_pad - c0 : kTileC) >> 3;  // 16-byte vectors per pixel in this tile
+  for (int i = threadIdx.x; i < hw * cvecs; i += kThreads) {
+    const int cv = i % cvecs, px = i / cvecs;
+    uint32_t o[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int ch = cv * 8 + j;
+      if (ch < nch) o[j >> 1] |= (uint32_t)flat[ch * hw + px] << ((j & 1) * 16);
+    }
+    *reinterpret_cast<uint4*>(d + (int64_t)px * c_pad + c0 + cv * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
 // x'[n][hw][c_pad] -> x[n][c][hw]
 __global__ void __launch_bounds__(kThreads)
 nhwc_to_nchw_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int64_t hw,
@@ -200,6 +232,18 @@ cudaError_t launch_nchw_to_nhwc(const __half* src, __half* dst, int32_t n, int32
   const int64_t px_tiles = (hw + kTileP - 1) / kTileP;
   const int c_tiles = (c_pad + kTileC - 1) / kTileC;
   if (px_tiles > 0x7fffffffLL || c_tiles > 65535 || n > 65535) return cudaErrorInvalidConfiguration;
+  if ((hw % 8) != 0 && hw <= 640 && ((int64_t)c * hw) % 8 == 0 && (kTileC * hw) % 8 == 0) {
+    // small odd plane: contiguous 64-channel spans (at most 80 KB of shared memory)
+    const size_t smem = (size_t)kTileC * hw * sizeof(uint16_t);
+    cudaError_t err = cudaFuncSetAttribute(nchw_to_nhwc_smallplane_kernel,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    dim3 grid2((unsigned)c_tiles, (unsigned)n);
+    nchw_to_nhwc_smallplane_kernel<<<grid2, kThreads, smem, stream>>>(reinterpret_cast<const uint16_t*>(src),
+                                                                      reinterpret_cast<uint16_t*>(dst), c, (int)hw, c_pad);
+    count_launch();
+    return cudaGetLastError();
+  }
   dim3 grid((unsigned)px_tiles, (unsigned)c_tiles, (unsigned)n);
   nchw_to_nhwc_kernel<<<grid, kThreads, 0, stream>>>(reinterpret_cast<const uint16_t*>(src),
                                                      reinterpret_cast<uint16_t*>(dst), c, hw, c_pad,
