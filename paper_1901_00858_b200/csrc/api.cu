@@ -76,11 +76,13 @@ int forward_impl(hgc_conv_desc* d, const void* x, const void* w, const void* bia
                         : hgc::launch_weights_repack(wh, wp, g.k, g.cg, g.r, g.s, g.group, ip.cw, stream);
         if (err != cudaSuccess) break;
       }
-      err = ip.window ? hgc::launch_nchw_to_nhwc8_bordered(xh, xp, g.n, g.c, g.h, g.w, g.pad_h, g.pad_w, ip.hp, ip.wp,
-                                                           stream)
-                      : hgc::launch_nchw_to_nhwc(xh, xp, g.n, g.c, g.h, g.w, ip.c_pad, stream);
-      if (err != cudaSuccess) break;
-      err = hgc::launch_igemm(g, ip, ws, bh, yh, relu, stream);
+      if (!ip.nchw) {
+        err = ip.window ? hgc::launch_nchw_to_nhwc8_bordered(xh, xp, g.n, g.c, g.h, g.w, g.pad_h, g.pad_w, ip.hp,
+                                                             ip.wp, stream)
+                        : hgc::launch_nchw_to_nhwc(xh, xp, g.n, g.c, g.h, g.w, ip.c_pad, stream);
+        if (err != cudaSuccess) break;
+      }
+      err = hgc::launch_igemm(g, ip, ws, xh, bh, yh, relu, stream);
       break;
     }
     case HGC_PATH_DEPTHWISE:
@@ -230,6 +232,7 @@ int hgc_conv_set_workspace(hgc_conv_desc* d, void* dev_ptr, size_t bytes) {
   d->registered_w = nullptr;
   d->igemm.maps_ready = false;
   d->igemm.y_mapped = nullptr;
+  d->igemm.x_mapped = nullptr;
   if (d->path == HGC_PATH_IGEMM && dev_ptr != nullptr && bytes >= d->ws_needed) {
     // the TMA descriptors point into the workspace: encode them now; clear the status word
     if (!hgc::igemm_encode_maps(d->geom, &d->igemm, dev_ptr)) return HGC_CUDA_ERROR;

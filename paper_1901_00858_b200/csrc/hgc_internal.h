@@ -44,6 +44,8 @@ cudaError_t launch_weights_repack(const __half* src, __half* dst, int32_t k, int
 struct IgemmPlan {
   int32_t kb, cblocks, cw, c_pad;
   int32_t halo, pitch;
+  int32_t nchw, nblk;                            // 1x1 layers reading x (NCHW) directly
+  const void* x_mapped;                          // input pointer tmB was encoded for (nchw)
   int32_t window, kw_pix, hp, wp;                // few-channel layers: windows over a zero-bordered NHWC8 copy
   int32_t eff_r, eff_s, eff_pad_h, eff_pad_w;    // the convolution as the kernel sees it
   int32_t tn, th, tw, ncols;
@@ -64,7 +66,7 @@ struct IgemmPlan {
 
 bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out);
 bool igemm_encode_maps(const ConvGeom& g, IgemmPlan* p, void* ws);
-cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half* bias, __half* y,
+cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half* x, const __half* bias, __half* y,
                          int relu, cudaStream_t stream);
 
 }  // namespace hgc

@@ -216,18 +216,20 @@ template <int KSTEPS>
 __device__ __forceinline__ uint32_t issue_stage(uint32_t next_bar, uint32_t next_parity, uint32_t d_tmem,
                                                 uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc,
                                                 uint32_t a_bar, uint32_t b_bar, uint32_t release_b,
-                                                uint32_t do_mma) {
+                                                uint32_t do_mma, uint64_t b_step) {
   uint32_t ready;
 #define HGC_STAGE_OPERANDS                                                                                   \
   : "=r"(ready)                                                                                              \
   : "r"(next_bar), "r"(next_parity), "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc), "r"(a_bar), \
-    "r"(b_bar), "r"(release_b), "r"(do_mma)                                                                  \
+    "r"(b_bar), "r"(release_b), "r"(do_mma), "l"(b_step)                                                     \
   : "memory"
   if (KSTEPS == 4) {
     asm volatile(
       "{\n"
       ".reg .pred p_next, p_el, p_mma, p_acc, p_one, p_rel;\n"
       ".reg .b64 da, db;\n"
+      "mov.b64 da, %4;\n"
+      "mov.b64 db, %5;\n"
       "mbarrier.test_wait.parity.shared::cta.b64 p_next, [%1], %2;\n"
       "elect.sync _|p_el, 0xffffffff;\n"
       "setp.ne.b32 p_mma, %11, 0;\n"
@@ -237,14 +239,14 @@ __device__ __forceinline__ uint32_t issue_stage(uint32_t next_bar, uint32_t next
       "setp.ne.b32 p_rel, %10, 0;\n"
       "and.pred p_rel, p_rel, p_el;\n"
       "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], %4, %5, %6, p_acc;\n"
-      "add.u64 da, %4, 2;\n"
-      "add.u64 db, %5, 2;\n"
+      "add.u64 da, da, 2;\n"
+      "add.u64 db, db, %12;\n"
       "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, p_one;\n"
-      "add.u64 da, %4, 4;\n"
-      "add.u64 db, %5, 4;\n"
+      "add.u64 da, da, 2;\n"
+      "add.u64 db, db, %12;\n"
       "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, p_one;\n"
-      "add.u64 da, %4, 6;\n"
-      "add.u64 db, %5, 6;\n"
+      "add.u64 da, da, 2;\n"
+      "add.u64 db, db, %12;\n"
       "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, p_one;\n"
       "@p_el tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n"
       "@p_rel tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n"
@@ -256,6 +258,8 @@ __device__ __forceinline__ uint32_t issue_stage(uint32_t next_bar, uint32_t next
       "{\n"
       ".reg .pred p_next, p_el, p_mma, p_acc, p_one, p_rel;\n"
       ".reg .b64 da, db;\n"
+      "mov.b64 da, %4;\n"
+      "mov.b64 db, %5;\n"
       "mbarrier.test_wait.parity.shared::cta.b64 p_next, [%1], %2;\n"
       "elect.sync _|p_el, 0xffffffff;\n"
       "setp.ne.b32 p_mma, %11, 0;\n"
@@ -265,8 +269,8 @@ __device__ __forceinline__ uint32_t issue_stage(uint32_t next_bar, uint32_t next
       "setp.ne.b32 p_rel, %10, 0;\n"
       "and.pred p_rel, p_rel, p_el;\n"
       "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], %4, %5, %6, p_acc;\n"
-      "add.u64 da, %4, 2;\n"
-      "add.u64 db, %5, 2;\n"
+      "add.u64 da, da, 2;\n"
+      "add.u64 db, db, %12;\n"
       "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, p_one;\n"
       "@p_el tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n"
       "@p_rel tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n"
@@ -278,6 +282,8 @@ __device__ __forceinline__ uint32_t issue_stage(uint32_t next_bar, uint32_t next
       "{\n"
       ".reg .pred p_next, p_el, p_mma, p_acc, p_one, p_rel;\n"
       ".reg .b64 da, db;\n"
+      "mov.b64 da, %4;\n"
+      "mov.b64 db, %5;\n"
       "mbarrier.test_wait.parity.shared::cta.b64 p_next, [%1], %2;\n"
       "elect.sync _|p_el, 0xffffffff;\n"
       "setp.ne.b32 p_mma, %11, 0;\n"
@@ -300,27 +306,29 @@ __device__ __forceinline__ uint32_t issue_stage(uint32_t next_bar, uint32_t next
 // KSTEPS MMAs of one weight tile against one activation tile, issued by one elected lane.
 template <int KSTEPS>
 __device__ __forceinline__ void issue_mmas(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                           uint32_t acc, uint32_t do_mma) {
-#define HGC_MMA_OPERANDS ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc), "r"(do_mma) : "memory"
+                                           uint32_t acc, uint32_t do_mma, uint64_t b_step) {
+#define HGC_MMA_OPERANDS ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc), "r"(do_mma), "l"(b_step) : "memory"
   if (KSTEPS == 4) {
     asm volatile(
         "{\n"
         ".reg .pred p_el, p_mma, p_acc, p_one;\n"
         ".reg .b64 da, db;\n"
+        "mov.b64 da, %1;\n"
+        "mov.b64 db, %2;\n"
         "elect.sync _|p_el, 0xffffffff;\n"
         "setp.ne.b32 p_mma, %5, 0;\n"
         "and.pred p_mma, p_mma, p_el;\n"
         "setp.ne.b32 p_acc, %4, 0;\n"
         "setp.eq.b32 p_one, 0, 0;\n"
         "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p_acc;\n"
-        "add.u64 da, %1, 2;\n"
-        "add.u64 db, %2, 2;\n"
+        "add.u64 da, da, 2;\n"
+        "add.u64 db, db, %6;\n"
         "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p_one;\n"
-        "add.u64 da, %1, 4;\n"
-        "add.u64 db, %2, 4;\n"
+        "add.u64 da, da, 2;\n"
+        "add.u64 db, db, %6;\n"
         "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p_one;\n"
-        "add.u64 da, %1, 6;\n"
-        "add.u64 db, %2, 6;\n"
+        "add.u64 da, da, 2;\n"
+        "add.u64 db, db, %6;\n"
         "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p_one;\n"
         "}\n"
         HGC_MMA_OPERANDS);
@@ -329,14 +337,16 @@ __device__ __forceinline__ void issue_mmas(uint32_t d_tmem, uint64_t adesc, uint
         "{\n"
         ".reg .pred p_el, p_mma, p_acc, p_one;\n"
         ".reg .b64 da, db;\n"
+        "mov.b64 da, %1;\n"
+        "mov.b64 db, %2;\n"
         "elect.sync _|p_el, 0xffffffff;\n"
         "setp.ne.b32 p_mma, %5, 0;\n"
         "and.pred p_mma, p_mma, p_el;\n"
         "setp.ne.b32 p_acc, %4, 0;\n"
         "setp.eq.b32 p_one, 0, 0;\n"
         "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p_acc;\n"
-        "add.u64 da, %1, 2;\n"
-        "add.u64 db, %2, 2;\n"
+        "add.u64 da, da, 2;\n"
+        "add.u64 db, db, %6;\n"
         "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p_one;\n"
         "}\n"
         HGC_MMA_OPERANDS);
@@ -345,6 +355,8 @@ __device__ __forceinline__ void issue_mmas(uint32_t d_tmem, uint64_t adesc, uint
         "{\n"
         ".reg .pred p_el, p_mma, p_acc, p_one;\n"
         ".reg .b64 da, db;\n"
+        "mov.b64 da, %1;\n"
+        "mov.b64 db, %2;\n"
         "elect.sync _|p_el, 0xffffffff;\n"
         "setp.ne.b32 p_mma, %5, 0;\n"
         "and.pred p_mma, p_mma, p_el;\n"
@@ -498,7 +510,12 @@ struct IgemmArgs {
   uint32_t stage_bytes;
   uint32_t a_bytes, b_bytes, b_alloc;  // TMA bytes of A and B per load, smem reserved per B stage
   uint32_t idesc;
-  uint64_t desc_hi;  // shared-memory descriptor bits other than the start address
+  uint64_t desc_hi;    // shared-memory descriptor bits other than the start address (weights; activations too unless nchw)
+  uint64_t desc_hi_b;  // the same for the activation operand
+  uint64_t b_kstep;    // address-field increment of the activation descriptor per 16-channel MMA step
+  int32_t nchw;        // 1: 1x1 layer reading x as it is (NCHW): pixel-major activation tiles of 64-pixel blocks
+  int32_t nblk;        // 64-pixel blocks per activation tile (nchw)
+  int32_t cg;          // channels per group (nchw: channel coordinate of the tile)
   int32_t relu;
   int32_t tma_store;  // 1: the epilogue stages fp16 tiles in shared memory and stores them with TMA
   int32_t rem;        // (th*Q) % 64: width of the last staged pass of a full tile (0 = none)
@@ -589,8 +606,15 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             const uint32_t sbase = ring_base + ring.idx * a.stage_bytes;
             if (elect_one()) {
               mbar_expect_tx(fb, a.b_bytes + (uint32_t)a.taps * a.a_bytes);
-              tma_load_5d(sbase, &tmB, fb, cb * KB, grp, (HALO ? 0 : sg * a.dil_w) - a.pad_w, h_base + r * a.dil_h,
-                          n0);
+              if (a.nchw) {
+                // x itself, (pixel, channel, image): blocks of 64 pixels x KB channels, pixels contiguous
+                for (int j = 0; j < a.nblk; ++j)
+                  tma_load_3d(sbase + (uint32_t)j * (uint32_t)(KB * 128), &tmB, fb, p0 * a.Q + 64 * j,
+                              grp * a.cg + cb * KB, n0);
+              } else {
+                tma_load_5d(sbase, &tmB, fb, cb * KB, grp, (HALO ? 0 : sg * a.dil_w) - a.pad_w,
+                            h_base + r * a.dil_h, n0);
+              }
               for (int t = 0; t < a.taps; ++t)
                 tma_load_3d(sbase + a.b_alloc + (uint32_t)t * a.a_bytes, &tmA, fb, acol + t * a.cw, m0, grp);
             }
@@ -649,12 +673,12 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t sbase = ring_base + ring.idx * a.stage_bytes;
         const uint32_t e_bar = smem_u32(&empty_bar[ring.idx]);
-        uint64_t bdesc = desc_hi | (uint64_t)((sbase & 0x3FFFFu) >> 4);
+        uint64_t bdesc = a.desc_hi_b | (uint64_t)((sbase & 0x3FFFFu) >> 4);
         uint64_t adesc = desc_hi | (uint64_t)(((sbase + a.b_alloc) & 0x3FFFFu) >> 4);
         ring.advance(depth);
         // all taps but the last: MMAs only
         for (int t = 0; t + 1 < a.taps; ++t) {
-          issue_mmas<ksteps>(d_tmem, adesc, bdesc, idesc, acc, do_mma);
+          issue_mmas<ksteps>(d_tmem, adesc, bdesc, idesc, acc, do_mma, a.b_kstep);
           acc = 1;
           adesc += (uint64_t)(a.a_bytes >> 4);
           bdesc += (uint64_t)(tap_step >> 4);
@@ -662,7 +686,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         // last tap: poll the NEXT stage's barrier first and read the answer after the MMAs and the
         // commit have been issued, so that the poll's latency hides behind them
         ready = issue_stage<ksteps>(smem_u32(&full_bar[ring.idx]), ring.phase, d_tmem, adesc, bdesc, idesc, acc, e_bar,
-                                    e_bar, 0u, do_mma);
+                                    e_bar, 0u, do_mma, a.b_kstep);
         acc = 1;
       }
       if (ok) {
@@ -869,6 +893,12 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
     // stride 1: the S taps of a kernel row read one shared tile, shifted by s*dil pixels
     p.halo = (g.stride_h == 1 && g.stride_w == 1) ? 1 : 0;
   }
+  // 1x1, stride 1, unpadded layers on planes of a multiple of 8 pixels read x as it is (no NHWC
+  // copy): the activation operand is then pixel-major ("MN-major") in shared memory
+  p.nchw = (!p.window && g.r == 1 && g.s == 1 && g.stride_h == 1 && g.stride_w == 1 && g.pad_h == 0 &&
+            g.pad_w == 0 && g.group == 1 && ((int64_t)g.h * g.w) % 8 == 0)
+               ? 1
+               : 0;
   p.pitch = p.halo ? g.q + (g.s - 1) * g.dil_w : g.q;
   p.tw = g.q;
   const int box_w = p.halo ? p.pitch : (p.window ? g.q : g.q * g.stride_w);
@@ -884,7 +914,8 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   int best_th = 0, best_tn = 0;
   for (int th = 1; th <= g.p; ++th) {
     if ((int64_t)th * p.pitch - junk > 256 || (int64_t)th * g.stride_h > 256) break;
-    const int tn_hi = th == g.p ? g.n : 1;  // several images only when a tile holds whole planes
+    if (p.nchw && th != g.p && ((int64_t)th * g.q) % 8 != 0) continue;  // tiles must start on 16-byte boundaries of x
+    const int tn_hi = (th == g.p && !p.nchw) ? g.n : 1;  // several images only when a tile holds whole planes
     for (int tn = 1; tn <= tn_hi; ++tn) {
       const int64_t cols = (int64_t)tn * th * p.pitch - junk;
       if (cols > 256 || tn > 256) break;
@@ -938,6 +969,11 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
     uint32_t rows2 = (uint32_t)(p.halo ? (g.s - 1) * g.dil_w : 0) + (uint32_t)p.ncols;
     if (rows2 < box_rows2) rows2 = box_rows2;
     p.b_alloc = (uint32_t)round_up_sz((size_t)rows2 * p.kb * 2u, 1024);
+    if (p.nchw) {
+      p.nblk = (p.ncols + 63) / 64;
+      p.b_bytes = (uint32_t)p.nblk * (uint32_t)p.kb * 128u;
+      p.b_alloc = p.b_bytes;
+    }
     p.stage_bytes = p.b_alloc + (uint32_t)p.taps * p.a_bytes;
     p.stages = (int)(budget / p.stage_bytes);
     if (p.stages > 8) p.stages = 8;
@@ -957,8 +993,9 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   p.ws_status_off = 0;
   p.ws_w_off = 256;
   p.ws_x_off = p.ws_w_off + round_up_sz((size_t)g.k * p.eff_r * p.eff_s * p.cw * 2, 256);
-  p.ws_total = p.ws_x_off + round_up_sz(p.window ? (size_t)g.n * p.hp * p.wp * 16 + 256
-                                                 : (size_t)g.n * g.h * g.w * p.c_pad * 2, 256);
+  p.ws_total = p.ws_x_off + (p.nchw ? 0
+                                    : round_up_sz(p.window ? (size_t)g.n * p.hp * p.wp * 16 + 256
+                                                           : (size_t)g.n * g.h * g.w * p.c_pad * 2, 256));
   *out = p;
   return true;
 }
@@ -982,7 +1019,9 @@ bool igemm_encode_maps(const ConvGeom& g, IgemmPlan* p, void* ws) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return false;
   }
-  if (p->window) {
+  if (p->nchw) {
+    // the activation map is over the caller's x and is encoded when x is known (igemm_encode_x_map)
+  } else if (p->window) {
     // (window element, -, output column, padded input row, image): the column stride is stride_w
     // pixels of 16 bytes, i.e. consecutive windows overlap
     const cuuint64_t pix = 16;
@@ -1012,6 +1051,24 @@ bool igemm_encode_maps(const ConvGeom& g, IgemmPlan* p, void* ws) {
   return true;
 }
 
+// 1x1 layers that read x directly: x[N][C][H*W] seen as (pixel, channel, image), 64 pixels x kb
+// channels per box, 128-byte swizzle (pixel-major operand tiles).
+bool igemm_encode_x_map(const ConvGeom& g, IgemmPlan* p, const void* x) {
+  PFN_cuTensorMapEncodeTiled_v12000 enc = encode_fn();
+  if (enc == nullptr) return false;
+  const cuuint64_t hw = (cuuint64_t)g.h * g.w;
+  cuuint64_t dims[3] = {hw, (cuuint64_t)g.c, (cuuint64_t)g.n};
+  cuuint64_t strides[2] = {hw * 2, hw * 2 * (cuuint64_t)g.c};
+  cuuint32_t box[3] = {64, (cuuint32_t)p->kb, 1};
+  cuuint32_t es[3] = {1, 1, 1};
+  if (enc(&p->tmB, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(x), dims, strides, box, es,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return false;
+  p->x_mapped = x;
+  return true;
+}
+
 // Tensor maps of the output y[N][K][P*Q] seen as (pixels, channels of a group, groups, images):
 // one with a 64-pixel box and one with the narrower box of a tile's last staged pass.
 bool igemm_encode_y_maps(const ConvGeom& g, IgemmPlan* p, void* y) {
@@ -1032,9 +1089,10 @@ bool igemm_encode_y_maps(const ConvGeom& g, IgemmPlan* p, void* y) {
   return true;
 }
 
-cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half* bias, __half* y,
+cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half* x, const __half* bias, __half* y,
                          int relu, cudaStream_t stream) {
   if (!p.maps_ready) return cudaErrorInvalidValue;
+  if (p.nchw && p.x_mapped != x && !igemm_encode_x_map(g, &p, x)) return cudaErrorInvalidValue;
   if (p.tma_store && p.y_mapped != y && !igemm_encode_y_maps(g, &p, y)) return cudaErrorInvalidValue;
   IgemmArgs a{};
   a.N = g.n; a.K = g.k; a.P = g.p; a.Q = g.q;
@@ -1048,11 +1106,22 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
   a.a_bytes = p.a_bytes; a.b_bytes = p.b_bytes; a.b_alloc = p.b_alloc;
   // instruction descriptor: D = f32, A = B = f16, both K-major, N >> 3 at bit 17, M >> 4 at bit 24
   a.idesc = (1u << 4) | ((uint32_t)(p.ncols >> 3) << 17) | ((128u >> 4) << 24);
+  if (p.nchw) a.idesc |= 1u << 16;  // activation operand is pixel-major (MN-major)
   // shared-memory descriptor: 8-row groups are 8 * row bytes apart; descriptor version 1;
   // swizzle mode 2 = 128 B, 4 = 64 B, 6 = 32 B
   const uint64_t sbo = (uint64_t)(8 * p.kb * 2) >> 4;
   const uint64_t layout = p.kb == 64 ? 2 : (p.kb == 32 ? 4 : 6);
   a.desc_hi = (1ull << 16) | (sbo << 32) | (1ull << 46) | (layout << 61);
+  a.desc_hi_b = a.desc_hi;
+  a.b_kstep = 2;  // 16 channels = 32 bytes along a swizzled K-major row
+  a.nchw = p.nchw; a.nblk = p.nblk; a.cg = g.cg;
+  if (p.nchw) {
+    // pixel-major tile: 64-pixel blocks of kb channel rows (128 bytes each, 128-byte swizzle):
+    // leading offset = one block, stride offset = 8 channel rows; 16 channels = 2048 bytes
+    const uint64_t lbo = (uint64_t)(p.kb * 128) >> 4;
+    a.desc_hi_b = (lbo << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+    a.b_kstep = 2048 >> 4;
+  }
   a.relu = relu;
   a.tma_store = p.tma_store;
   a.rem = p.rem;
