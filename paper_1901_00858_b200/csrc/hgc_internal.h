@@ -64,6 +64,9 @@ struct IgemmPlan {
   alignas(64) CUtensorMap tmYr;
 };
 
+// number of SMs of the current device (148 if it cannot be queried)
+int sm_count();
+
 bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out);
 bool igemm_encode_maps(const ConvGeom& g, IgemmPlan* p, void* ws);
 cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half* x, const __half* bias, __half* y,
