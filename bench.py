@@ -6,7 +6,9 @@
 A step is one pass of the whole path over one batch of a workload: every layer of the named
 network shape, each with its own resident input, weights, bias and output (the layers'
 inputs are generated independently, so the working set is far larger than L2 and no L2
-flush is needed between steps).  Prints ONE JSON line (rank 0).
+flush is needed between steps).  The step is captured once as a CUDA graph and the K timed
+steps replay it (--no-graph: eager launches); per-layer times come from a separate eager pass
+with an event pair around every layer.  Prints ONE JSON line (rank 0).
 
 N > 1 (under torchrun): the path has no exchange step; every rank runs an independent
 replica on its own batch ("weak" scaling) and the line reports the aggregate.
@@ -275,25 +277,67 @@ def run_ours(args, wl):
         one_step()
     barrier()
 
+    # The step is launch-bound in places (layers of 10-40 us behind a ctypes call each), so the
+    # whole step is captured once as a CUDA graph and the timed steps replay it: same kernels,
+    # same arguments, same order, no per-launch host cost.  --no-graph times eager launches.
+    graph = None
+    graph_err = None
+    side = torch.cuda.Stream()
+    launches_per_step = None
+    if not args.no_graph:
+        try:
+            side.wait_stream(stream)
+            graph = torch.cuda.CUDAGraph()
+            c0 = hgc.kernel_launch_count()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(graph, stream=side):
+                    for (d, x, w, b, y, l) in state:
+                        hgc.conv_forward(d, x, w, b, y, l.relu, side)
+            launches_per_step = hgc.kernel_launch_count() - c0
+            torch.cuda.synchronize()
+            with torch.cuda.stream(side):
+                for _ in range(3):
+                    graph.replay()
+            torch.cuda.synchronize()
+        except Exception as exc:  # capture not possible: say why and time eager launches
+            graph = None
+            graph_err = repr(exc)
+
     # timed region: exactly K steps between two events on the launching stream
-    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in state]
-          for _ in range(args.steps)]
+    tstream = side if graph is not None else stream
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches0 = hgc.kernel_launch_count()
     barrier()
     host_t0 = time.time()
-    t_start.record(stream)
-    for s in range(args.steps):
-        one_step(ev[s])
-    t_end.record(stream)
+    with torch.cuda.stream(tstream):
+        t_start.record(tstream)
+        for s in range(args.steps):
+            if graph is not None:
+                graph.replay()
+            else:
+                one_step()
+        t_end.record(tstream)
     barrier()
     host_t1 = time.time()
-    launches = hgc.kernel_launch_count() - launches0
+    launches = (launches_per_step * args.steps) if graph is not None else hgc.kernel_launch_count() - launches0
     total_ms = t_start.elapsed_time(t_end)
     ms_per_step = total_ms / args.steps
 
-    # per-layer device times (average over the K timed steps)
-    layer_ms = [sum(ev[s][i][0].elapsed_time(ev[s][i][1]) for s in range(args.steps)) / args.steps
+    # per-layer device times: a separate pass of eager launches with an event pair around every
+    # layer (average over its steps).  Short layers include some launch latency here, so the
+    # per-kernel roofline fractions derived from them are on the low side.
+    lsteps = max(1, min(args.steps, 20))
+    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in state]
+          for _ in range(lsteps)]
+    e_start, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e_start.record(stream)
+    for s in range(lsteps):
+        one_step(ev[s])
+    e_end.record(stream)
+    barrier()
+    eager_ms = e_start.elapsed_time(e_end) / lsteps
+    layer_ms = [sum(ev[s][i][0].elapsed_time(ev[s][i][1]) for s in range(lsteps)) / lsteps
                 for i in range(len(state))]
 
     # ---- end to end through the host-buffer entry point ------------------------------------
@@ -328,31 +372,6 @@ def run_ours(args, wl):
         barrier()
         e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
-    # ---- the same step replayed as one CUDA graph (no per-launch host cost) -------------------
-    graph_ms = None
-    if not args.no_graph:
-        try:
-            side = torch.cuda.Stream()
-            side.wait_stream(stream)
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.stream(side):
-                with torch.cuda.graph(g, stream=side):
-                    for (d, x, w, b, y, l) in state:
-                        hgc.conv_forward(d, x, w, b, y, l.relu, side)
-            torch.cuda.synchronize()
-            for _ in range(3):
-                g.replay()
-            barrier()
-            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            g0.record()
-            for _ in range(args.steps):
-                g.replay()
-            g1.record()
-            barrier()
-            graph_ms = g0.elapsed_time(g1) / args.steps
-        except Exception as exc:  # capture not possible: report why, keep the main numbers
-            graph_ms = None
-            graph_err = repr(exc)
     clocks = sampler.stop((host_t0, host_t1)) if rank == 0 else None
 
     # ---- max over ranks ---------------------------------------------------------------------
@@ -402,6 +421,7 @@ def run_ours(args, wl):
             "config": {"workload": wl.name if not (args.only or args.batch) else f"{wl.name} (subset: only={args.only or 'all'}, batch={batch})",
                        "layers": len(layers), "batch_per_gpu": batch,
                        "l2": "inputs larger than L2 (every layer has its own tensors)",
+                       "launch": "cuda_graph" if graph is not None else "eager",
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
             "images_per_s": agg["images_per_s"],
             "roofline": roof,
@@ -415,10 +435,12 @@ def run_ours(args, wl):
             "gpu_launches": launches,
             "clocks": clocks,
         }
-        if graph_ms is not None:
-            line["graph_replay"] = {"ms_per_step": graph_ms, "tflops": step_flops / (graph_ms * 1e-3) / 1e12,
-                                    "images_per_s": batch / (graph_ms * 1e-3),
-                                    "note": "same step captured once and replayed as a CUDA graph, this rank"}
+        line["eager"] = {"ms_per_step": eager_ms, "tflops": step_flops / (eager_ms * 1e-3) / 1e12,
+                         "steps": lsteps,
+                         "note": "the same step as eager launches with an event pair around every layer "
+                                 "(source of the per-layer and per-kernel times), this rank"}
+        if graph_err is not None:
+            line["graph_error"] = graph_err
         if cpu is not None:
             line["cpu_baseline"] = cpu
         if args.layers:
@@ -435,14 +457,14 @@ def run_ours(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD,
                     help="one of: " + ", ".join(w.name for w in workloads.all_workloads()))
     ap.add_argument("--layers", action="store_true", help="add per-layer figures to the JSON line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay leg")
+    ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of replaying the step as a CUDA graph")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     ap.add_argument("--only", default="", help="comma-separated layer names: run just these layers (profiling)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling on a small case)")
