@@ -78,12 +78,6 @@ __device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity
   return ok;
 }
 
-__device__ __forceinline__ long long clk() {
-  long long t;
-  asm volatile("mov.u64 %0, %%clock64;" : "=l"(t)::"memory");
-  return t;
-}
-
 __device__ __forceinline__ uint64_t global_timer_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -160,29 +154,9 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm,
       : "memory");
 }
 
-__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                         uint32_t accumulate) {
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "setp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
-      "}\n" ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-      : "r"(taddr)
-      : "memory");
 }
 
 __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&v)[8]) {
@@ -886,6 +860,10 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
     p.halo = 0;
   } else {
     p.kb = g.cg > 32 ? 64 : (g.cg > 16 ? 32 : 16);
+    // stride-1 layers with three or more taps per kernel row and at least two 64-channel blocks:
+    // 32-channel stages halve a stage (one activation tile + S weight tiles) so that the ring
+    // is four or five deep instead of two; measured 3-5 % faster on 3x3 layers of 128-512 channels
+    if (p.kb == 64 && g.stride_h == 1 && g.stride_w == 1 && g.s >= 3 && g.cg >= 128) p.kb = 32;
     p.cblocks = (g.cg + p.kb - 1) / p.kb;
     p.cw = p.cblocks * p.kb;
     p.c_pad = (g.c + 7) / 8 * 8;
@@ -906,10 +884,33 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   p.mtiles = (g.kg + 127) / 128;
   const int64_t mg = (int64_t)p.mtiles * g.group;
   // pixel tile = tn images x th rows; accumulator columns = tn*th*pitch (<= 256).  Among the
-  // feasible shapes pick the one with the least estimated time: waves over the SMs x (columns
-  // + a per-tile overhead), preferring larger tiles on ties.
+  // feasible shapes pick the one with the least estimated time: waves over the SMs x the
+  // estimated clocks of one tile.
   const int sms = sm_count();
   const int junk = p.pitch - g.q;
+  // An MMA step (128 channels x ncols pixels x 16 reduction elements) is bounded by
+  //   the tensor pipe:     ncols / 2 clocks,
+  //   L2 -> shared memory  (about 30 bytes per clock and SM, measured): its 4 KB slice of the
+  //                        weights plus its share of the activation tile, which the taps and
+  //                        16-channel steps of a stage share,
+  //   the issuing thread:  about 45 clocks per MMA plus about 400 per barrier hand-shake;
+  // the epilogue of the previous tile runs beside the main loop and bounds short main loops.
+  const int taps_est = p.halo ? p.eff_s : 1;
+  const double mps = (double)taps_est * (p.kb / 16.0);                       // MMAs per stage
+  const double mpt = (double)p.cblocks * p.eff_r * p.eff_s * (p.kb / 16.0);  // MMAs per tile
+  const double a_bytes_mma = 32.0 * (g.kg < 128 ? g.kg : 128);
+  auto tile_clk = [&](int64_t brow, int64_t cols) {
+    const double ncols = (double)((cols + 15) / 16 * 16);
+    const double brows = p.nchw ? (double)((cols + 63) / 64 * 64) : (double)brow;
+    const double t_l2 = (a_bytes_mma + brows * p.kb * 2.0 / mps) / 30.0;
+    const double t_tensor = ncols / 2.0;
+    const double t_issue = 45.0 + 400.0 / mps;
+    double t = t_tensor > t_l2 ? t_tensor : t_l2;
+    if (t_issue > t) t = t_issue;
+    const double main_loop = mpt * t;
+    const double epilogue = 600.0 + 10.0 * ncols;
+    return (main_loop > epilogue ? main_loop : epilogue) + 300.0;
+  };
   double best = 1e300;
   int best_th = 0, best_tn = 0;
   for (int th = 1; th <= g.p; ++th) {
@@ -921,13 +922,7 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
       if (cols > 256 || tn > 256) break;
       const int64_t tiles = (int64_t)((g.n + tn - 1) / tn) * ((g.p + th - 1) / th) * mg;
       const int64_t waves = (tiles + sms - 1) / sms;
-      const double ncols = (double)((cols + 15) / 16 * 16);
-      // covered columns (incl. ragged last tiles) matter when there are many waves; whole waves
-      // when there are few
-      // an MMA step costs about max(N, 64 + N/2) column-times (narrow tiles re-read the weight
-      // stage from shared memory too often to keep the tensor pipe busy)
-      const double mma = ncols > 64.0 + 0.5 * ncols ? ncols : 64.0 + 0.5 * ncols;
-      const double cost = (double)waves * (mma + 40.0) + 1e-3 * (double)tiles;
+      const double cost = (double)waves * tile_clk((int64_t)tn * th * p.pitch, cols) + 1e-3 * (double)tiles;
       if (cost < best - 1e-9 || (cost < best + 1e-9 && (int64_t)tn * th > (int64_t)best_tn * best_th)) {
         best = cost;
         best_th = th;
