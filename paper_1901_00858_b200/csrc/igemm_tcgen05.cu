@@ -343,124 +343,94 @@ __device__ __forceinline__ void issue_mmas(uint32_t d_tmem, uint64_t adesc, uint
 #undef HGC_MMA_OPERANDS
 }
 
-// Row epilogue (every shape the TMA-store epilogue does not take: planes whose rows or sizes
-// are not multiples of 8 pixels, several images per tile).  A thread owns one output channel
-// (its TMEM lane); the pixels of one image that it holds are one contiguous run of y.  It
-// converts them 8 columns at a time into its own 144-byte row of shared memory, placed at the
-// same offset modulo 16 as the run has in global memory, and copies the row out with aligned
-// 16-byte stores (the ragged head and tail pixel by pixel).  Only the thread itself touches its
-// row, so no synchronisation is needed.  Kept out of line: the hot loops of the kernel should
+// Copy epilogue (every shape the TMA-store epilogue does not take: planes whose size is not a
+// multiple of 8 pixels, tiles with junk columns between their rows, several images per tile).
+// A unit of work is this warp's 32 channels (its TMEM lanes) x up to 64 accumulator columns of
+// one image.  The warp converts the unit into its own staging tile in shared memory (32 rows of
+// 128 bytes, one per channel, 16-byte chunks XOR-swizzled by the row so that the 16-byte stores
+// of 8 lanes fall into 8 different bank groups), then copies it out with the roles turned: a
+// lane owns one or two COLUMNS and walks the 32 channel rows, so that every store instruction
+// writes consecutive pixels of one channel plane (64 or 128 contiguous bytes).  The two warps
+// of a lane quarter take alternate units.  Kept out of line: the hot loops of the kernel should
 // stay compact in the instruction cache.
-constexpr int kRowRunElems = 56;     // pixels staged per flush (112 bytes + up to 14 bytes of phase)
-constexpr uint32_t kRowPitch = 144;  // bytes between the rows of neighbouring lanes (bank spread)
-
-__device__ __forceinline__ void flush_row(uint32_t srow, uint16_t* gdst, int len) {
-  // gdst: global address of the run's first pixel; the run starts at byte (gdst & 15) of srow
-  const uint32_t phase = (uint32_t)(reinterpret_cast<uintptr_t>(gdst) & 15u);
-  char* gbase = reinterpret_cast<char*>(gdst) - phase;
-  const uint32_t end = phase + 2u * (uint32_t)len;
-  for (uint32_t off = 0; off < end; off += 16) {
-    uint32_t v0, v1, v2, v3;
-    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3) : "r"(srow + off));
-    if (off >= phase && off + 16 <= end) {
-      *reinterpret_cast<uint4*>(gbase + off) = make_uint4(v0, v1, v2, v3);
-    } else {
-      const uint32_t w[4] = {v0, v1, v2, v3};
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const uint32_t b = off + 2u * e;
-        if (b >= phase && b < end) *reinterpret_cast<uint16_t*>(gbase + b) = (uint16_t)((w[e >> 1] >> ((e & 1) * 16)) & 0xffffu);
-      }
-    }
-  }
-}
-
-__device__ __noinline__ void epilogue_rows(uint32_t t_addr, int col_begin, int col_end, int tn, int th, int pitch,
-                                           int N, int K, int P, int Q, int n0, int p0, int k, bool kvalid, float bv,
-                                           bool relu, uint16_t* yb, uint32_t srow) {
+__device__ __noinline__ void epilogue_copy(uint32_t t_addr, uint32_t sbuf, int first_unit, int unit_step, int tn, int th,
+                                           int pitch, int N, int K, int P, int Q, int n0, int p0, int k0,
+                                           int kvalid_rows, float bv, bool relu, uint16_t* yb) {
+  const int lane = threadIdx.x & 31;
   const int64_t pq = (int64_t)P * Q;
-  // walk the tile rows that intersect this warp's column range
-  int rowi = col_begin / pitch;
-  int wc = col_begin - rowi * pitch;  // column within the pitch (>= Q: junk)
-  int img = rowi / th;
-  int hr = rowi - img * th;
-  uint16_t* run = nullptr;  // global address of the first staged pixel of the current run
-  int fill = 0;             // pixels staged so far
-  uint32_t wpos = 0;        // byte position in srow of the next pixel
-  int col = col_begin;
+  const int rows_valid = (P - p0) < th ? (P - p0) : th;
+  const int cols_need = (rows_valid - 1) * pitch + Q;  // columns of one image up to its last real pixel
+  const int img_cols = th * pitch;
+  // pairs of columns can be copied as 4-byte words when columns are pixels (no junk) and every
+  // image's first pixel and every channel plane start on a 4-byte boundary
+  const bool words = pitch == Q && (pq & 1) == 0 && ((p0 * Q) & 1) == 0 && (cols_need & 1) == 0;
+  const uint32_t row_off = (uint32_t)lane * 128u;
+  int unit = 0;
+  for (int img = 0; img < tn; ++img) {
+    if (n0 + img >= N) break;
+    uint16_t* yimg = yb + ((int64_t)(n0 + img) * K + k0) * pq;  // this warp's first channel plane
+    for (int c0 = 0; c0 < cols_need; c0 += 64, ++unit) {
+      if (unit % unit_step != first_unit) continue;
+      const int ncol = cols_need - c0 < 64 ? cols_need - c0 : 64;
+      const uint32_t tcol = t_addr + (uint32_t)(img * img_cols + c0);
+      // ---- accumulators -> fp16 staging tile (lane = channel) ----
+      __syncwarp();  // the previous unit has been copied out
 #pragma unroll 1
-  while (col < col_end && img < tn) {
-    // control flow below is the same for all lanes of the warp (the TMEM loads are
-    // warp-collective); a lane without a real channel only skips its stores
-    const bool row_ok = (n0 + img) < N && (p0 + hr) < P;
-    if (wc >= Q || !row_ok) {
-      // junk columns / rows past the plane: skip to the next tile row
-      col += pitch - wc;
-      wc = 0;
-      if (++hr == th) {
-        hr = 0;
-        ++img;
-        if (fill) {  // the next image is not contiguous
-          if (kvalid) flush_row(srow, run, fill);
-          fill = 0;
+      for (int g = 0; g < 2; ++g) {
+        if (g * 32 >= ncol) break;
+        uint32_t v[4][8];
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          if (g * 32 + c * 8 < ncol) tmem_ld8(tcol + (uint32_t)(g * 32 + c * 8), v[c]);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          if (g * 32 + c * 8 < ncol) {
+            uint32_t o[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              o[i] = pack_f16x2(__uint_as_float(v[c][2 * i]) + bv, __uint_as_float(v[c][2 * i + 1]) + bv, relu);
+            const uint32_t dst = sbuf + row_off + ((uint32_t)((g * 4 + c) ^ (lane & 7)) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3])
+                         : "memory");
+          }
         }
       }
-      continue;
-    }
-    int cnt = Q - wc;
-    if (cnt > 8) cnt = 8;
-    if (cnt > col_end - col) cnt = col_end - col;
-    uint32_t v[8];
-    __syncwarp();
-    tmem_ld8(t_addr + (uint32_t)col, v);
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-    uint32_t o[4];
+      __syncwarp();
+      // ---- staging tile -> y (lane = column) ----
+      if (words) {
+        const int col = 2 * lane;  // columns col, col + 1 of the unit
+        if (col < ncol) {          // ncol is even here
+          uint16_t* dst = yimg + (int64_t)p0 * Q + c0 + col;
+          const uint32_t chunk = (uint32_t)col >> 3, within = ((uint32_t)col & 7u) * 2u;
+#pragma unroll 4
+          for (int r = 0; r < kvalid_rows; ++r) {
+            uint32_t w;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w) : "r"(sbuf + (uint32_t)r * 128u + ((chunk ^ ((uint32_t)r & 7u)) << 4) + within));
+            *reinterpret_cast<uint32_t*>(dst + (int64_t)r * pq) = w;
+          }
+        }
+      } else {
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
-      o[i] = pack_f16x2(__uint_as_float(v[2 * i]) + bv, __uint_as_float(v[2 * i + 1]) + bv, relu);
-    if (fill == 0) {
-      run = yb + ((int64_t)(n0 + img) * K + k) * pq + (int64_t)(p0 + hr) * Q + wc;
-      wpos = (uint32_t)(reinterpret_cast<uintptr_t>(run) & 15u);
-    }
-    const uint32_t dst = srow + wpos;
-    if (!kvalid) {
-      // nothing to stage for a lane beyond the group's last channel
-    } else if (cnt == 8 && (wpos & 15u) == 0) {
-      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
-    } else if (cnt == 8 && (wpos & 7u) == 0) {
-      asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(dst), "r"(o[0]), "r"(o[1]) : "memory");
-      asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(dst + 8), "r"(o[2]), "r"(o[3]) : "memory");
-    } else if (cnt == 8 && (wpos & 3u) == 0) {
-#pragma unroll
-      for (int i = 0; i < 4; ++i) asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst + 4 * i), "r"(o[i]) : "memory");
-    } else {
-#pragma unroll
-      for (int e = 0; e < 8; ++e)
-        if (e < cnt)
-          asm volatile("st.shared.b16 [%0], %1;" ::"r"(dst + 2 * e), "h"((uint16_t)((o[e >> 1] >> ((e & 1) * 16)) & 0xffffu))
-                       : "memory");
-    }
-    fill += cnt;
-    wpos += 2u * (uint32_t)cnt;
-    col += cnt;
-    wc += cnt;
-    if (wc == pitch) {  // pitch == Q: straight on to the next row
-      wc = 0;
-      if (++hr == th) {
-        hr = 0;
-        ++img;
-        if (fill) {
-          if (kvalid) flush_row(srow, run, fill);
-          fill = 0;
+        for (int hcol = 0; hcol < 2; ++hcol) {
+          const int col = lane + 32 * hcol;
+          const int cabs = c0 + col;
+          const int hr = cabs / pitch;
+          const int wc = cabs - hr * pitch;
+          if (col < ncol && wc < Q) {
+            uint16_t* dst = yimg + (int64_t)(p0 + hr) * Q + wc;
+            const uint32_t chunk = (uint32_t)col >> 3, within = ((uint32_t)col & 7u) * 2u;
+#pragma unroll 4
+            for (int r = 0; r < kvalid_rows; ++r) {
+              uint16_t w;
+              asm volatile("ld.shared.b16 %0, [%1];" : "=h"(w) : "r"(sbuf + (uint32_t)r * 128u + ((chunk ^ ((uint32_t)r & 7u)) << 4) + within));
+              dst[(int64_t)r * pq] = w;
+            }
+          }
         }
       }
-    }
-    if (fill > kRowRunElems - 8) {  // no room for another chunk
-      if (kvalid) flush_row(srow, run, fill);
-      fill = 0;
     }
   }
-  if (fill && kvalid) flush_row(srow, run, fill);
   __syncwarp();
 }
 
@@ -713,8 +683,9 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           const int e_valid = rows_valid * a.Q;  // output pixels of one channel in this tile
           const bool last_row_tile = p0 + a.th >= a.P;
           // (row, column) of the unit's first pixel, kept up to date without divisions
+          const bool linear = a.pitch == a.Q;  // no junk columns: accumulator columns are consecutive pixels
           int hr = 0, wc = half * kPassElems;
-          while (wc >= a.Q) { wc -= a.Q; ++hr; }
+          while (!linear && wc >= a.Q) { wc -= a.Q; ++hr; }
           for (int e_lo = half * kPassElems; e_lo < e_valid; e_lo += 2 * kPassElems, ++unit_ctr) {
             const int e_hi = e_lo + kPassElems < e_valid ? e_lo + kPassElems : e_valid;
             const uint32_t sbuf = my_stage + (unit_ctr % (uint32_t)a.nbuf) * kWarpStageBytes;
@@ -727,9 +698,13 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
               uint32_t cols[4];
 #pragma unroll
               for (int c = 0; c < 4; ++c) {
-                cols[c] = (uint32_t)(uh * a.pitch + uw);
-                uw += 8;
-                if (uw == a.Q) { uw = 0; ++uh; }  // next output row: the junk columns of the pitch are skipped
+                if (linear) {
+                  cols[c] = (uint32_t)(e0 + 8 * c);  // columns are pixels
+                } else {
+                  cols[c] = (uint32_t)(uh * a.pitch + uw);
+                  uw += 8;
+                  if (uw == a.Q) { uw = 0; ++uh; }  // next output row: the junk columns of the pitch are skipped
+                }
               }
               uint32_t v[4][8];
 #pragma unroll
@@ -767,7 +742,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             }
             // first pixel of this warp's next unit: two units further on
             wc += 2 * kPassElems;
-            while (wc >= a.Q) { wc -= a.Q; ++hr; }
+            while (!linear && wc >= a.Q) { wc -= a.Q; ++hr; }
           }
         }
         // this warp has read its lanes of the accumulator: hand the buffer back to the MMA issuer
@@ -777,11 +752,12 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       } else {
         // ---- direct epilogue: each thread stores runs of its own channel plane ----
         {
-          // the two warps of a lane quarter take the first and the second half of the columns
-          const int split = ((a.ncols >> 1) + 15) & ~15;
-          if (quarter_live)
-            epilogue_rows(t_addr, half ? split : 0, half ? a.ncols : split, a.tn, a.th, a.pitch, a.N, a.K, a.P, a.Q, n0,
-                          p0, k, kvalid, bv, relu, yb, my_stage + (uint32_t)lane * kRowPitch);
+          // the two warps of a lane quarter take alternate units
+          if (quarter_live) {
+            const int kleft = a.kg - (m0 + quarter * 32);
+            epilogue_copy(t_addr, my_stage, half, 2, a.tn, a.th, a.pitch, a.N, a.K, a.P, a.Q, n0, p0,
+                          grp * a.kg + m0 + quarter * 32, kleft < 32 ? kleft : 32, bv, relu, yb);
+          }
         }
         // this warp has read its lanes of the accumulator: hand the buffer back to the MMA issuer
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -919,7 +895,9 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
     const int tn_hi = (th == g.p && !p.nchw) ? g.n : 1;  // several images only when a tile holds whole planes
     for (int tn = 1; tn <= tn_hi; ++tn) {
       const int64_t cols = (int64_t)tn * th * p.pitch - junk;
-      if (cols > 256 || tn > 256) break;
+      // several images per tile: image boundaries need not fall on multiples of 8 columns, and an
+      // 8-column accumulator read that starts in the tile must end inside the 256-column buffer
+      if (cols > (tn > 1 ? 248 : 256) || tn > 256) break;
       const int64_t tiles = (int64_t)((g.n + tn - 1) / tn) * ((g.p + th - 1) / th) * mg;
       const int64_t waves = (tiles + sms - 1) / sms;
       const double cost = (double)waves * tile_clk((int64_t)tn * th * p.pitch, cols) + 1e-3 * (double)tiles;
@@ -948,7 +926,11 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   p.b_alloc = (uint32_t)round_up_sz((size_t)rows * p.kb * 2u, 1024);
   // the epilogue stages fp16 tiles for TMA stores when every staged run of pixels starts on a
   // 16-byte boundary of y: Q % 8 == 0 (so P*Q % 8 == 0 too) and one image per tile
-  p.tma_store = ((g.q % 8) == 0 && p.tn == 1) ? 1 : 0;
+  // (or, when the tile has no junk columns, plane and tile sizes are multiples of 8 pixels)
+  p.tma_store = (p.tn == 1 && ((g.q % 8) == 0 || (p.pitch == g.q && ((int64_t)g.p * g.q) % 8 == 0 &&
+                                                  ((int64_t)p.th * g.q) % 8 == 0)))
+                    ? 1
+                    : 0;
   p.rem = (p.th * g.q) % kPassElems;
   // rings: B two or three deep, A with what is left (each A stage feeds kb/16 MMAs).  227 KB per
   // CTA minus alignment slack, static barriers and the two epilogue staging buffers.
