@@ -62,18 +62,19 @@ nchw_to_nhwc_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst
   }
 }
 
-// x[n][c][hw] -> x'[n][hw][c_pad] for planes of a multiple of 8 pixels, without shared memory.
-// A thread owns 8 channels x 8 consecutive pixels: eight 16-byte loads (one per channel), an
-// 8x8 transpose of the binary16 values in registers (byte permutes), eight 16-byte stores (one
-// per pixel).  In a warp, lane % CH picks the 8-channel chunk and lane / CH the 8-pixel group,
-// so that a store instruction writes CH*16 contiguous bytes per pixel (whole 32-byte sectors)
-// and a load instruction reads (32/CH)*16 contiguous bytes per channel.  A warp's unit of work
-// is CH*8 channels x (32/CH)*8 pixels of one image.
-template <int CH>
+// x[n][c][hw] -> x'[n][hw][c_pad] for planes of a multiple of PX (8 or 4) pixels, without shared
+// memory.  A thread owns 8 channels x PX consecutive pixels: eight 16- or 8-byte loads (one per
+// channel), a transpose of the binary16 values in registers (byte permutes), PX 16-byte stores
+// (one per pixel).  In a warp, lane % CH picks the 8-channel chunk and lane / CH the pixel
+// group, so that a store instruction writes CH*16 contiguous bytes per pixel (whole 32-byte
+// sectors) and a load instruction reads (32/CH)*PX*2 contiguous bytes per channel.  A warp's
+// unit of work is CH*8 channels x (32/CH)*PX pixels of one image.
+template <int CH, int PX>
 __global__ void __launch_bounds__(kThreads)
 nchw_to_nhwc_regs_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int64_t hw,
                          int c_pad, int64_t units_p, int units_c, int64_t total_units) {
   constexpr int PG = 32 / CH;
+  constexpr int W32 = PX / 2;  // 32-bit words per channel
   const int lane = threadIdx.x & 31;
   const int c8 = lane % CH, pg = lane / CH;
   const int64_t warp0 = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
@@ -85,27 +86,32 @@ nchw_to_nhwc_regs_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict_
     const int uc = (int)(t % units_c);
     const int64_t n = t / units_c;
     const int ch = (uc * CH + c8) * 8;
-    const int64_t p = (up * PG + pg) * 8;
+    const int64_t p = (up * PG + pg) * PX;
     if (ch >= c_pad || p >= hw) continue;
     const uint16_t* s = src + (n * c + ch) * hw + p;
-    uint4 v[8];
+    uint32_t v[8][W32];
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
-      v[i] = (ch + i < c) ? __ldcs(reinterpret_cast<const uint4*>(s + (int64_t)i * hw)) : make_uint4(0u, 0u, 0u, 0u);
+    for (int i = 0; i < 8; ++i) {
+      if (ch + i < c) {
+        if constexpr (PX == 8) {
+          const uint4 q = __ldcs(reinterpret_cast<const uint4*>(s + (int64_t)i * hw));
+          v[i][0] = q.x; v[i][1] = q.y; v[i][2] = q.z; v[i][3] = q.w;
+        } else {
+          const uint2 q = __ldcs(reinterpret_cast<const uint2*>(s + (int64_t)i * hw));
+          v[i][0] = q.x; v[i][1] = q.y;
+        }
+      } else {
+#pragma unroll
+        for (int w = 0; w < W32; ++w) v[i][w] = 0u;
+      }
+    }
     uint16_t* d = dst + (n * hw + p) * c_pad + ch;
 #pragma unroll
-    for (int q = 0; q < 8; ++q) {
+    for (int q = 0; q < PX; ++q) {
       const uint32_t sel = (q & 1) ? 0x7632u : 0x5410u;
       uint32_t o[4];
 #pragma unroll
-      for (int m = 0; m < 4; ++m) {
-        const uint32_t lo = (q >> 1) == 0 ? v[2 * m].x : (q >> 1) == 1 ? v[2 * m].y : (q >> 1) == 2 ? v[2 * m].z : v[2 * m].w;
-        const uint32_t hi = (q >> 1) == 0   ? v[2 * m + 1].x
-                            : (q >> 1) == 1 ? v[2 * m + 1].y
-                            : (q >> 1) == 2 ? v[2 * m + 1].z
-                                            : v[2 * m + 1].w;
-        o[m] = __byte_perm(lo, hi, sel);
-      }
+      for (int m = 0; m < 4; ++m) o[m] = __byte_perm(v[2 * m][q >> 1], v[2 * m + 1][q >> 1], sel);
       *reinterpret_cast<uint4*>(d + (int64_t)q * c_pad) = make_uint4(o[0], o[1], o[2], o[3]);
     }
   }
@@ -281,6 +287,32 @@ cudaError_t launch_nchw_to_nhwc(const __half* src, __half* dst, int32_t n, int32
   const int64_t px_tiles = (hw + kTileP - 1) / kTileP;
   const int c_tiles = (c_pad + kTileC - 1) / kTileC;
   if (px_tiles > 0x7fffffffLL || c_tiles > 65535 || n > 65535) return cudaErrorInvalidConfiguration;
+  if ((hw % 4) == 0) {
+    // planes of a multiple of 8 (or 4) pixels: every channel row starts on a 16- (8-) byte
+    // boundary: register transpose, 8 or 4 channel chunks per pixel per warp
+    const int px = (hw % 8) == 0 ? 8 : 4;
+    const int ch_per = c_pad >= 64 ? 8 : 4;
+    const int64_t units_p = (hw / px + (32 / ch_per) - 1) / (32 / ch_per);
+    const int units_c = (c_pad / 8 + ch_per - 1) / ch_per;
+    const int64_t total_units = units_p * units_c * n;
+    int64_t blocks = (total_units + (kThreads / 32) - 1) / (kThreads / 32);
+    const int64_t cap = (int64_t)sm_count() * 8 * 4;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    const uint16_t* s16 = reinterpret_cast<const uint16_t*>(src);
+    uint16_t* d16 = reinterpret_cast<uint16_t*>(dst);
+    const unsigned gb = (unsigned)blocks;
+    if (px == 8 && ch_per == 8)
+      nchw_to_nhwc_regs_kernel<8, 8><<<gb, kThreads, 0, stream>>>(s16, d16, c, hw, c_pad, units_p, units_c, total_units);
+    else if (px == 8)
+      nchw_to_nhwc_regs_kernel<4, 8><<<gb, kThreads, 0, stream>>>(s16, d16, c, hw, c_pad, units_p, units_c, total_units);
+    else if (ch_per == 8)
+      nchw_to_nhwc_regs_kernel<8, 4><<<gb, kThreads, 0, stream>>>(s16, d16, c, hw, c_pad, units_p, units_c, total_units);
+    else
+      nchw_to_nhwc_regs_kernel<4, 4><<<gb, kThreads, 0, stream>>>(s16, d16, c, hw, c_pad, units_p, units_c, total_units);
+    count_launch();
+    return cudaGetLastError();
+  }
   if ((hw % 8) != 0 && hw <= 640 && ((int64_t)c * hw) % 8 == 0 && (kTileC * hw) % 8 == 0) {
     // small odd plane: contiguous 64-channel spans (at most 80 KB of shared memory)
     const size_t smem = (size_t)kTileC * hw * sizeof(uint16_t);
@@ -290,27 +322,6 @@ cudaError_t launch_nchw_to_nhwc(const __half* src, __half* dst, int32_t n, int32
     dim3 grid2((unsigned)c_tiles, (unsigned)n);
     nchw_to_nhwc_smallplane_kernel<<<grid2, kThreads, smem, stream>>>(reinterpret_cast<const uint16_t*>(src),
                                                                       reinterpret_cast<uint16_t*>(dst), c, (int)hw, c_pad);
-    count_launch();
-    return cudaGetLastError();
-  }
-  if ((hw % 8) == 0) {
-    // planes of a multiple of 8 pixels: register transpose, 8 or 4 channel chunks per pixel per warp
-    const int ch_per = c_pad >= 64 ? 8 : 4;
-    const int64_t units_p = (hw / 8 + (32 / ch_per) - 1) / (32 / ch_per);
-    const int units_c = (c_pad / 8 + ch_per - 1) / ch_per;
-    const int64_t total_units = units_p * units_c * n;
-    int64_t blocks = (total_units + (kThreads / 32) - 1) / (kThreads / 32);
-    const int64_t cap = (int64_t)sm_count() * 8 * 4;
-    if (blocks > cap) blocks = cap;
-    if (blocks < 1) blocks = 1;
-    if (ch_per == 8)
-      nchw_to_nhwc_regs_kernel<8><<<(unsigned)blocks, kThreads, 0, stream>>>(
-          reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), c, hw, c_pad, units_p, units_c,
-          total_units);
-    else
-      nchw_to_nhwc_regs_kernel<4><<<(unsigned)blocks, kThreads, 0, stream>>>(
-          reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), c, hw, c_pad, units_p, units_c,
-          total_units);
     count_launch();
     return cudaGetLastError();
   }
