@@ -323,6 +323,85 @@ depthwise3x3_rowvec_kernel(const uint16_t* __restrict__ x, const __half* __restr
   }
 }
 
+// Small planes (W = 28, 14, 7; pad 1): rows are shorter than a 16-byte vector pattern can use, so
+// a thread owns one whole output row of one plane.  It reads its three input rows straight from
+// global memory (4-byte words when W is even, else 2-byte elements; consecutive lanes read
+// consecutive rows, so a warp's loads cover one contiguous span, and the rows shared with the
+// neighbouring lanes come from L1), keeps them in registers with a zero halo on both sides,
+// accumulates with the mixed-precision FMA and writes its output row the same way.  No shared
+// memory, no synchronisation (staging the span in shared memory first was measured slower).
+template <int W, int S>
+__global__ void __launch_bounds__(256)
+depthwise3x3_smallrow_kernel(const uint16_t* __restrict__ x, const __half* __restrict__ w,
+                             const __half* __restrict__ bias, uint16_t* __restrict__ y, int c, int h, int p, int relu,
+                             int64_t total_rows) {
+  constexpr int Q = (W - 1) / S + 1;  // kernel 3, pad 1
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total_rows) return;
+  const int64_t plane = idx / p;
+  const int pr = (int)(idx - plane * p);
+  const int ch = (int)(plane % c);
+  uint16_t wv[9];
+#pragma unroll
+  for (int i = 0; i < 9; ++i) wv[i] = __half_as_ushort(__ldg(w + (int64_t)ch * 9 + i));
+  const float bv = bias != nullptr ? __half2float(__ldg(bias + ch)) : 0.f;
+
+  uint16_t in[3][W + 2];  // element e of a row at [e + 1]; [0] and [W + 1] are the zero padding
+#pragma unroll
+  for (int rr = 0; rr < 3; ++rr) {
+    const int ih = pr * S - 1 + rr;
+    const bool rv = ih >= 0 && ih < h;
+    const uint16_t* xr = x + (plane * h + (rv ? ih : 0)) * W;
+    in[rr][0] = 0;
+    in[rr][W + 1] = 0;
+    if constexpr ((W & 1) == 0) {
+#pragma unroll
+      for (int e = 0; e < W / 2; ++e) {
+        const uint32_t v = rv ? __ldg(reinterpret_cast<const uint32_t*>(xr) + e) : 0u;
+        asm("mov.b32 {%0, %1}, %2;" : "=h"(in[rr][1 + 2 * e]), "=h"(in[rr][2 + 2 * e]) : "r"(v));
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < W; ++e) in[rr][1 + e] = rv ? __ldg(xr + e) : (uint16_t)0;
+    }
+  }
+  float f[Q + 1];
+#pragma unroll
+  for (int j = 0; j < Q; ++j) {
+    float acc = bv;
+#pragma unroll
+    for (int rr = 0; rr < 3; ++rr)
+#pragma unroll
+      for (int ss = 0; ss < 3; ++ss)
+        asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(acc) : "h"(in[rr][j * S + ss]), "h"(wv[rr * 3 + ss]));
+    f[j] = acc;
+  }
+  f[Q] = 0.f;
+  uint16_t* yr = y + (plane * p + pr) * Q;
+#pragma unroll
+  for (int j = 0; j < Q; j += 2) {
+    uint32_t o;
+    if (relu)
+      asm("cvt.rn.relu.f16x2.f32 %0, %1, %2;" : "=r"(o) : "f"(f[j + 1]), "f"(f[j]));
+    else
+      asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(o) : "f"(f[j + 1]), "f"(f[j]));
+    if constexpr ((Q & 1) == 0) {
+      reinterpret_cast<uint32_t*>(yr)[j >> 1] = o;
+    } else {
+      yr[j] = (uint16_t)(o & 0xffffu);
+      if (j + 1 < Q) yr[j + 1] = (uint16_t)(o >> 16);
+    }
+  }
+}
+
+// shapes the small-row kernel takes
+bool smallrow_ok(const ConvGeom& g) {
+  if (g.pad_h != 1 || g.pad_w != 1) return false;
+  if (g.w != 28 && g.w != 14 && g.w != 7) return false;
+  if (g.stride_h != g.stride_w) return false;
+  return g.q == (g.w - 1) / g.stride_w + 1;
+}
+
 // shapes the row-vector kernel takes: pad 1, W % 8 == 0, whole output vectors per row
 bool rowvec_ok(const ConvGeom& g) {
   if (g.pad_h != 1 || g.pad_w != 1) return false;
@@ -411,6 +490,26 @@ cudaError_t launch_depthwise3x3(const ConvGeom& g, const __half* x, const __half
       else
         depthwise3x3_rowvec_kernel<2, 2><<<(unsigned)blocks, 256, 0, stream>>>(xs0, w, bias, ys0, g.c, g.h, g.w, g.p,
                                                                                g.q, relu, items, vec_per_row, strips);
+      count_launch();
+      return cudaGetLastError();
+    }
+  }
+  if (smallrow_ok(g)) {
+    const int64_t rows = (int64_t)g.n * g.c * g.p;
+    const int64_t blocks = (rows + 255) / 256;
+    if (blocks < 0x7fffffffLL) {
+      const uint16_t* xs0 = reinterpret_cast<const uint16_t*>(x);
+      uint16_t* ys0 = reinterpret_cast<uint16_t*>(y);
+      const unsigned gb = (unsigned)blocks;
+#define HGC_DW_SMALLROW(WV, SV) \
+  depthwise3x3_smallrow_kernel<WV, SV><<<gb, 256, 0, stream>>>(xs0, w, bias, ys0, g.c, g.h, g.p, relu, rows)
+      if (g.w == 28 && g.stride_h == 1) HGC_DW_SMALLROW(28, 1);
+      else if (g.w == 28) HGC_DW_SMALLROW(28, 2);
+      else if (g.w == 14 && g.stride_h == 1) HGC_DW_SMALLROW(14, 1);
+      else if (g.w == 14) HGC_DW_SMALLROW(14, 2);
+      else if (g.stride_h == 1) HGC_DW_SMALLROW(7, 1);
+      else HGC_DW_SMALLROW(7, 2);
+#undef HGC_DW_SMALLROW
       count_launch();
       return cudaGetLastError();
     }
