@@ -72,16 +72,11 @@ int forward_impl(hgc_conv_desc* d, const void* x, const void* w, const void* bia
       __half* wp = reinterpret_cast<__half*>(ws + ip.ws_w_off);
       __half* xp = reinterpret_cast<__half*>(ws + ip.ws_x_off);
       if (d->registered_w != w) {  // weights not prepared in advance: re-lay them out now
-        err = ip.window ? hgc::launch_weights_repack_window(wh, wp, g.k, g.c, g.r, g.s, ip.kw_pix, stream)
-                        : hgc::launch_weights_repack(wh, wp, g.k, g.cg, g.r, g.s, g.group, ip.cw, stream);
+        err = hgc::launch_igemm_weights(g, ip, wh, wp, stream);
         if (err != cudaSuccess) break;
       }
-      if (!ip.nchw) {
-        err = ip.window ? hgc::launch_nchw_to_nhwc8_bordered(xh, xp, g.n, g.c, g.h, g.w, g.pad_h, g.pad_w, ip.hp,
-                                                             ip.wp, stream)
-                        : hgc::launch_nchw_to_nhwc(xh, xp, g.n, g.c, g.h, g.w, ip.c_pad, stream);
-        if (err != cudaSuccess) break;
-      }
+      err = hgc::launch_igemm_input(g, ip, xh, xp, stream);
+      if (err != cudaSuccess) break;
       err = hgc::launch_igemm(g, ip, ws, xh, bh, yh, relu, stream);
       break;
     }
@@ -249,11 +244,8 @@ int hgc_conv_set_weights(hgc_conv_desc* d, const void* w, void* stream) {
   if (d->path == HGC_PATH_IGEMM) {
     const hgc::ConvGeom& g = d->geom;
     __half* wp = reinterpret_cast<__half*>(static_cast<char*>(d->ws) + d->igemm.ws_w_off);
-    const cudaError_t err =
-        d->igemm.window ? hgc::launch_weights_repack_window(static_cast<const __half*>(w), wp, g.k, g.c, g.r, g.s,
-                                                            d->igemm.kw_pix, static_cast<cudaStream_t>(stream))
-                        : hgc::launch_weights_repack(static_cast<const __half*>(w), wp, g.k, g.cg, g.r, g.s, g.group,
-                                                     d->igemm.cw, static_cast<cudaStream_t>(stream));
+    const cudaError_t err = hgc::launch_igemm_weights(g, d->igemm, static_cast<const __half*>(w), wp,
+                                                      static_cast<cudaStream_t>(stream));
     if (err != cudaSuccess) return HGC_CUDA_ERROR;
   }
   d->registered_w = w;

@@ -47,6 +47,7 @@ struct IgemmPlan {
   int32_t nchw, nblk;                            // 1x1 layers reading x (NCHW) directly
   const void* x_mapped;                          // input pointer tmB was encoded for (nchw)
   int32_t window, kw_pix, hp, wp;                // few-channel layers: windows over a zero-bordered NHWC8 copy
+  int32_t patch;                                 // tiny receptive fields: 1x1 conv over an im2col copy of x
   int32_t eff_r, eff_s, eff_pad_h, eff_pad_w;    // the convolution as the kernel sees it
   int32_t tn, th, tw, ncols;
   int32_t tiles_h, tiles_n, mtiles, total_tiles;
@@ -63,6 +64,12 @@ struct IgemmPlan {
   alignas(64) CUtensorMap tmY;
   alignas(64) CUtensorMap tmYr;
 };
+
+// the weight re-layout and the input preparation of the tensor-core path, by plan mode
+cudaError_t launch_igemm_weights(const ConvGeom& g, const IgemmPlan& p, const __half* w, __half* wp,
+                                 cudaStream_t stream);
+cudaError_t launch_igemm_input(const ConvGeom& g, const IgemmPlan& p, const __half* x, __half* xp,
+                               cudaStream_t stream);
 
 // number of SMs of the current device (148 if it cannot be queried)
 int sm_count();

@@ -159,7 +159,22 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
                : "memory");
 }
 
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&v)[8]) {
+// 32 consecutive accumulator columns of this warp's 32 lanes in one instruction: a TMEM load
+// costs the issuing warp about 100 cycles whatever its width (measured), so wide loads matter
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t* v) {
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
                : "r"(taddr)
@@ -378,10 +393,14 @@ __device__ __noinline__ void epilogue_copy(uint32_t t_addr, uint32_t sbuf, int f
 #pragma unroll 1
       for (int g = 0; g < 2; ++g) {
         if (g * 32 >= ncol) break;
-        uint32_t v[4][8];
+        uint32_t v[32];
+        if (g * 32 + 32 <= ncol) {
+          tmem_ld32(tcol + (uint32_t)(g * 32), v);
+        } else {
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
-          if (g * 32 + c * 8 < ncol) tmem_ld8(tcol + (uint32_t)(g * 32 + c * 8), v[c]);
+          for (int c = 0; c < 4; ++c)
+            if (g * 32 + c * 8 < ncol) tmem_ld8(tcol + (uint32_t)(g * 32 + c * 8), &v[8 * c]);
+        }
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
@@ -389,7 +408,7 @@ __device__ __noinline__ void epilogue_copy(uint32_t t_addr, uint32_t sbuf, int f
             uint32_t o[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-              o[i] = pack_f16x2(__uint_as_float(v[c][2 * i]) + bv, __uint_as_float(v[c][2 * i + 1]) + bv, relu);
+              o[i] = pack_f16x2(__uint_as_float(v[8 * c + 2 * i]) + bv, __uint_as_float(v[8 * c + 2 * i + 1]) + bv, relu);
             const uint32_t dst = sbuf + row_off + ((uint32_t)((g * 4 + c) ^ (lane & 7)) << 4);
             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3])
                          : "memory");
@@ -466,6 +485,53 @@ struct IgemmArgs {
   int32_t nbuf;       // staging tiles per epilogue warp (1 or 2)
 };
 
+// The tiles of one CTA: blockIdx.x, blockIdx.x + gridDim.x, ...  Tile t = (pixel tile px, channel
+// tile mg) with mg fastest, px = (image tile, row tile).  The decomposition is kept up to date
+// by additions (a handful of divisions once per kernel instead of five per tile and role).
+struct TileIter {
+  int tile, mg, pt, ph;  // current tile, its channel tile, image tile and row tile
+  int stride, d_mg, d_pt, d_ph;
+  __device__ __forceinline__ void init(const IgemmArgs& a) {
+    const int mgn = a.mtiles * a.group;
+    tile = blockIdx.x;
+    const int px = tile / mgn;
+    mg = tile - px * mgn;
+    pt = px / a.tiles_h;
+    ph = px - pt * a.tiles_h;
+    stride = gridDim.x;
+    const int d_px = stride / mgn;
+    d_mg = stride - d_px * mgn;
+    d_pt = d_px / a.tiles_h;
+    d_ph = d_px - d_pt * a.tiles_h;
+  }
+  __device__ __forceinline__ bool valid(const IgemmArgs& a) const { return tile < a.total_tiles; }
+  __device__ __forceinline__ void next(const IgemmArgs& a) {
+    const int mgn = a.mtiles * a.group;
+    tile += stride;
+    mg += d_mg;
+    ph += d_ph;
+    pt += d_pt;
+    if (mg >= mgn) {
+      mg -= mgn;
+      ++ph;
+    }
+    if (ph >= a.tiles_h) {
+      ph -= a.tiles_h;
+      ++pt;
+    }
+  }
+  // group and first output channel (within the group) of the channel tile
+  __device__ __forceinline__ void channel_tile(const IgemmArgs& a, int& grp, int& m0) const {
+    if (a.group == 1) {
+      grp = 0;
+      m0 = mg * 128;
+    } else {
+      grp = mg / a.mtiles;
+      m0 = (mg - grp * a.mtiles) * 128;
+    }
+  }
+};
+
 constexpr int kMaxStages = 8;
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
@@ -528,15 +594,13 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     uint32_t issued = 0;
     bool ok = true;
     const uint32_t depth = (uint32_t)a.stages;
-    const int mgn = a.mtiles * a.group;
     const int groups_per_row = a.S / a.taps;  // 1 in halo mode (taps == S), S otherwise (taps == 1)
-    for (int tile = blockIdx.x; tile < a.total_tiles && ok; tile += gridDim.x) {
-      const int px = tile / mgn;
-      const int mg = tile - px * mgn;
-      const int grp = mg / a.mtiles;
-      const int m0 = (mg - grp * a.mtiles) * 128;
-      const int n0 = (px / a.tiles_h) * a.tn;
-      const int p0 = (px % a.tiles_h) * a.th;
+    TileIter it;
+    for (it.init(a); it.valid(a) && ok; it.next(a)) {
+      int grp, m0;
+      it.channel_tile(a, grp, m0);
+      const int n0 = it.pt * a.tn;
+      const int p0 = it.ph * a.th;
       const int h_base = p0 * a.stride_h - a.pad_h;
       for (int cb = 0; cb < a.cblocks && ok; ++cb) {
         int acol = cb * KB;  // column of w' for tap (r, s): (r*S + s)*cw + cb*KB
@@ -599,7 +663,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const int groups_per_row = a.S / a.taps;
     const int groups_per_tile = a.cblocks * a.R * groups_per_row;
     uint32_t ready = mbar_test_wait(smem_u32(&full_bar[0]), 0u);
-    for (int tile = blockIdx.x; tile < a.total_tiles && ok; tile += gridDim.x, ++lt) {
+    for (int tile = blockIdx.x; tile < a.total_tiles && ok; tile += gridDim.x, ++lt) {  // only the count matters here
       const uint32_t buf = lt & 1u;
       // the epilogue must have drained this accumulator (two tiles ago)
       if (!mbar_wait(smem_u32(&acc_empty[buf]), ((lt >> 1) & 1u) ^ 1u, &abort_flag, 64)) {
@@ -651,16 +715,14 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     // this warp's own staging tiles: 32 channel rows of 128 bytes each, 128-byte swizzled
     const uint32_t my_stage = stage_base + (uint32_t)ew * (uint32_t)a.nbuf * kWarpStageBytes;
     const uint32_t row_off = (uint32_t)lane * 128u + (((uint32_t)lane & 7u) << 4);
-    uint32_t unit_ctr = 0;
-    const int mgn = a.mtiles * a.group;
+    uint32_t unit_ctr = 0, stage_sel = 0;
     uint32_t lt = 0;
-    for (int tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x, ++lt) {
-      const int px = tile / mgn;
-      const int mg = tile - px * mgn;
-      const int grp = mg / a.mtiles;
-      const int m0 = (mg - grp * a.mtiles) * 128;
-      const int n0 = (px / a.tiles_h) * a.tn;
-      const int p0 = (px % a.tiles_h) * a.th;
+    TileIter it;
+    for (it.init(a); it.valid(a); it.next(a), ++lt) {
+      int grp, m0;
+      it.channel_tile(a, grp, m0);
+      const int n0 = it.pt * a.tn;
+      const int p0 = it.ph * a.th;
       const int kin = m0 + row;
       const bool kvalid = kin < a.kg;
       const int k = grp * a.kg + (kvalid ? kin : 0);
@@ -688,28 +750,37 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           while (!linear && wc >= a.Q) { wc -= a.Q; ++hr; }
           for (int e_lo = half * kPassElems; e_lo < e_valid; e_lo += 2 * kPassElems, ++unit_ctr) {
             const int e_hi = e_lo + kPassElems < e_valid ? e_lo + kPassElems : e_valid;
-            const uint32_t sbuf = my_stage + (unit_ctr % (uint32_t)a.nbuf) * kWarpStageBytes;
+            const uint32_t sbuf = my_stage + stage_sel * kWarpStageBytes;
+            stage_sel = a.nbuf == 2 ? stage_sel ^ 1u : 0u;
             int uh = hr, uw = wc;  // walks through this unit
 #pragma unroll 1
             for (int g = 0; g < 2; ++g) {
               const int e0 = e_lo + g * 32;
               if (e0 >= e_hi) break;
               const int nchunks = (e_hi - e0) >= 32 ? 4 : (e_hi - e0) >> 3;
-              uint32_t cols[4];
+              uint32_t v[32];
+              // 32 pixels: one wide accumulator load when they are 32 consecutive columns (always
+              // when columns are pixels; else when the row does not end inside them)
+              if (nchunks == 4 && (linear || uw + 32 <= a.Q)) {
+                tmem_ld32(t_addr + (uint32_t)(linear ? e0 : uh * a.pitch + uw), v);
+                if (!linear) {
+                  uw += 32;
+                  if (uw == a.Q) { uw = 0; ++uh; }
+                }
+              } else {
 #pragma unroll
-              for (int c = 0; c < 4; ++c) {
-                if (linear) {
-                  cols[c] = (uint32_t)(e0 + 8 * c);  // columns are pixels
-                } else {
-                  cols[c] = (uint32_t)(uh * a.pitch + uw);
-                  uw += 8;
-                  if (uw == a.Q) { uw = 0; ++uh; }  // next output row: the junk columns of the pitch are skipped
+                for (int c = 0; c < 4; ++c) {
+                  uint32_t col;
+                  if (linear) {
+                    col = (uint32_t)(e0 + 8 * c);  // columns are pixels
+                  } else {
+                    col = (uint32_t)(uh * a.pitch + uw);
+                    uw += 8;
+                    if (uw == a.Q) { uw = 0; ++uh; }  // next output row: the junk columns of the pitch are skipped
+                  }
+                  if (c < nchunks) tmem_ld8(t_addr + col, &v[8 * c]);
                 }
               }
-              uint32_t v[4][8];
-#pragma unroll
-              for (int c = 0; c < 4; ++c)
-                if (c < nchunks) tmem_ld8(t_addr + cols[c], v[c]);
               if (g == 0) {
                 // this buffer's previous store must have been read out of shared memory
                 if (lane == 0) {
@@ -725,7 +796,8 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                   uint32_t o[4];
 #pragma unroll
                   for (int i = 0; i < 4; ++i)
-                    o[i] = pack_f16x2(__uint_as_float(v[c][2 * i]) + bv, __uint_as_float(v[c][2 * i + 1]) + bv, relu);
+                    o[i] = pack_f16x2(__uint_as_float(v[8 * c + 2 * i]) + bv, __uint_as_float(v[8 * c + 2 * i + 1]) + bv,
+                                      relu);
                   const uint32_t dst = sbuf + (row_off ^ ((uint32_t)(g * 4 + c) << 4));
                   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]),
                                "r"(o[3])

@@ -257,6 +257,109 @@ __global__ void weights_repack_window_kernel(const uint16_t* __restrict__ src, u
   }
 }
 
+// Patch mode (layers whose whole receptive field R*S*C is at most 64 elements: image stems).
+// x[n][c][h][w] -> x''[n][p][q][kelems]: for every OUTPUT pixel the R*S*C input values under the
+// kernel, element (r*S + s)*C + ch, zero where the tap falls into the padding and from R*S*C up
+// to kelems.  The convolution then is a 1x1 convolution over x'' with kelems channels.
+// One thread per output pixel; the specialised form has every index known at compile time.
+template <int R, int S, int C>
+__global__ void __launch_bounds__(256)
+patch_im2col_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int h, int w, int p, int q,
+                    int pad_h, int pad_w, int stride_h, int stride_w, int dil_h, int dil_w, int kelems,
+                    int64_t total) {
+  constexpr int E = R * S * C;
+  constexpr int EW = (E + 1) / 2;  // 32-bit words that hold real elements
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const int oq = (int)(i % q);
+  const int64_t t = i / q;
+  const int op = (int)(t % p);
+  const int64_t n = t / p;
+  const int64_t hw = (int64_t)h * w;
+  const uint16_t* xn = src + n * C * hw;
+  uint32_t o[EW];
+#pragma unroll
+  for (int e = 0; e < EW; ++e) o[e] = 0u;
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const int ih = op * stride_h - pad_h + r * dil_h;
+#pragma unroll
+    for (int sx = 0; sx < S; ++sx) {
+      const int iw = oq * stride_w - pad_w + sx * dil_w;
+      const bool ok = ih >= 0 && ih < h && iw >= 0 && iw < w;
+#pragma unroll
+      for (int ch = 0; ch < C; ++ch) {
+        const int e = (r * S + sx) * C + ch;
+        const uint32_t v = ok ? (uint32_t)__ldg(xn + ch * hw + (int64_t)ih * w + iw) : 0u;
+        o[e >> 1] |= v << ((e & 1) * 16);
+      }
+    }
+  }
+  uint4* d = reinterpret_cast<uint4*>(dst + i * kelems);
+  const int vecs = kelems >> 3;
+#pragma unroll
+  for (int v = 0; v < 8; ++v) {
+    if (v < vecs) {
+      uint32_t a[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) a[j] = (4 * v + j) < EW ? o[(4 * v + j) < EW ? 4 * v + j : 0] : 0u;
+      d[v] = make_uint4(a[0], a[1], a[2], a[3]);
+    }
+  }
+}
+
+// any R, S, C with R*S*C <= 64: one thread per 8-element chunk of an output pixel's patch
+__global__ void __launch_bounds__(256)
+patch_im2col_generic_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int h, int w,
+                            int p, int q, int r, int s, int pad_h, int pad_w, int stride_h, int stride_w,
+                            int dil_h, int dil_w, int kelems, int64_t total_chunks) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total_chunks) return;
+  const int vecs = kelems >> 3;
+  const int v = (int)(i % vecs);
+  const int64_t pix = i / vecs;
+  const int oq = (int)(pix % q);
+  const int64_t t = pix / q;
+  const int op = (int)(t % p);
+  const int64_t n = t / p;
+  const int64_t hw = (int64_t)h * w;
+  const uint16_t* xn = src + n * c * hw;
+  const int rsc = r * s * c;
+  uint32_t o[4] = {0, 0, 0, 0};
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int e = v * 8 + j;
+    if (e < rsc) {
+      const int ch = e % c;
+      const int tap = e / c;
+      const int sx = tap % s, rr = tap / s;
+      const int ih = op * stride_h - pad_h + rr * dil_h;
+      const int iw = oq * stride_w - pad_w + sx * dil_w;
+      if (ih >= 0 && ih < h && iw >= 0 && iw < w)
+        o[j >> 1] |= (uint32_t)__ldg(xn + ch * hw + (int64_t)ih * w + iw) << ((j & 1) * 16);
+    }
+  }
+  *reinterpret_cast<uint4*>(dst + i * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// w[k][c][r][s] -> w'[k][kelems], element (r*S + s)*C + ch; zeros from R*S*C on
+__global__ void weights_repack_patch_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int64_t k,
+                                            int c, int r, int s, int kelems) {
+  const int64_t total = k * kelems;
+  const int rsc = r * s * c;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int e = (int)(i % kelems);
+    const int64_t kk = i / kelems;
+    uint16_t v = 0;
+    if (e < rsc) {
+      const int ch = e % c;
+      const int tap = e / c;
+      v = src[(kk * c + ch) * (r * s) + tap];
+    }
+    dst[i] = v;
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_nchw_to_nhwc8_bordered(const __half* src, __half* dst, int32_t n, int32_t c, int32_t h, int32_t w,
@@ -358,6 +461,62 @@ cudaError_t launch_weights_repack(const __half* src, __half* dst, int32_t k, int
       reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), k, cg, r * s, c_pad);
   count_launch();
   return cudaGetLastError();
+}
+
+cudaError_t launch_patch_im2col(const ConvGeom& g, const __half* src, __half* dst, int32_t kelems,
+                                cudaStream_t stream) {
+  const uint16_t* s16 = reinterpret_cast<const uint16_t*>(src);
+  uint16_t* d16 = reinterpret_cast<uint16_t*>(dst);
+  const int64_t pixels = (int64_t)g.n * g.p * g.q;
+  if (g.r == 3 && g.s == 3 && (g.c == 3 || g.c == 1 || g.c == 4)) {
+    const int64_t blocks = (pixels + 255) / 256;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+#define HGC_PATCH(CV)                                                                                         \
+  patch_im2col_kernel<3, 3, CV><<<(unsigned)blocks, 256, 0, stream>>>(s16, d16, g.h, g.w, g.p, g.q, g.pad_h, \
+                                                                      g.pad_w, g.stride_h, g.stride_w, g.dil_h, \
+                                                                      g.dil_w, kelems, pixels)
+    if (g.c == 3) HGC_PATCH(3);
+    else if (g.c == 1) HGC_PATCH(1);
+    else HGC_PATCH(4);
+#undef HGC_PATCH
+  } else {
+    const int64_t chunks = pixels * (kelems / 8);
+    const int64_t blocks = (chunks + 255) / 256;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    patch_im2col_generic_kernel<<<(unsigned)blocks, 256, 0, stream>>>(s16, d16, g.c, g.h, g.w, g.p, g.q, g.r, g.s,
+                                                                      g.pad_h, g.pad_w, g.stride_h, g.stride_w,
+                                                                      g.dil_h, g.dil_w, kelems, chunks);
+  }
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_weights_repack_patch(const __half* src, __half* dst, int32_t k, int32_t c, int32_t r, int32_t s,
+                                        int32_t kelems, cudaStream_t stream) {
+  const int64_t total = (int64_t)k * kelems;
+  int64_t blocks = (total + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  weights_repack_patch_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
+      reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), k, c, r, s, kelems);
+  count_launch();
+  return cudaGetLastError();
+}
+
+// The two preparation steps of the tensor-core path, dispatched on the plan's mode.
+cudaError_t launch_igemm_weights(const ConvGeom& g, const IgemmPlan& p, const __half* w, __half* wp,
+                                 cudaStream_t stream) {
+  if (p.patch) return launch_weights_repack_patch(w, wp, g.k, g.c, g.r, g.s, p.cw, stream);
+  if (p.window) return launch_weights_repack_window(w, wp, g.k, g.c, g.r, g.s, p.kw_pix, stream);
+  return launch_weights_repack(w, wp, g.k, g.cg, g.r, g.s, g.group, p.cw, stream);
+}
+
+cudaError_t launch_igemm_input(const ConvGeom& g, const IgemmPlan& p, const __half* x, __half* xp,
+                               cudaStream_t stream) {
+  if (p.nchw) return cudaSuccess;  // the kernel reads x itself
+  if (p.patch) return launch_patch_im2col(g, x, xp, p.cw, stream);
+  if (p.window) return launch_nchw_to_nhwc8_bordered(x, xp, g.n, g.c, g.h, g.w, g.pad_h, g.pad_w, p.hp, p.wp, stream);
+  return launch_nchw_to_nhwc(x, xp, g.n, g.c, g.h, g.w, p.c_pad, stream);
 }
 
 }  // namespace hgc

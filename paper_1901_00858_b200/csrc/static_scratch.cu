@@ -84,14 +84,8 @@ extern "C" int hgc_conv_forward_static(const hgc_conv_params* p, const void* x, 
   const __half* wh = static_cast<const __half*>(w);
   __half* wp = reinterpret_cast<__half*>(ws + plan.ws_w_off);
   __half* xp = reinterpret_cast<__half*>(ws + plan.ws_x_off);
-  if ((plan.window ? hgc::launch_weights_repack_window(wh, wp, g.k, g.c, g.r, g.s, plan.kw_pix, st)
-                   : hgc::launch_weights_repack(wh, wp, g.k, g.cg, g.r, g.s, g.group, plan.cw, st)) != cudaSuccess)
-    return HGC_CUDA_ERROR;
-  if (!plan.nchw &&
-      (plan.window
-           ? hgc::launch_nchw_to_nhwc8_bordered(xh, xp, g.n, g.c, g.h, g.w, g.pad_h, g.pad_w, plan.hp, plan.wp, st)
-           : hgc::launch_nchw_to_nhwc(xh, xp, g.n, g.c, g.h, g.w, plan.c_pad, st)) != cudaSuccess)
-    return HGC_CUDA_ERROR;
+  if (hgc::launch_igemm_weights(g, plan, wh, wp, st) != cudaSuccess) return HGC_CUDA_ERROR;
+  if (hgc::launch_igemm_input(g, plan, xh, xp, st) != cudaSuccess) return HGC_CUDA_ERROR;
   if (hgc::launch_igemm(g, plan, ws, xh, static_cast<const __half*>(bias), static_cast<__half*>(y), relu, st) !=
       cudaSuccess)
     return HGC_CUDA_ERROR;
