@@ -148,7 +148,12 @@ int hgc_conv_path(const hgc_conv_desc* d, int32_t* path);
  * [0] path, then for HGC_PATH_IGEMM: [1] channels per reduction block, [2] 1 if the taps of a
  * kernel row share one activation tile (stride 1), [3] images per pixel tile, [4] rows per pixel
  * tile, [5] accumulator columns per output row, [6] MMA N, [7] number of tiles, [8] depth of the
- * shared-memory ring, [9] weight tiles (taps) per ring stage; zeros for the other paths.  info: host pointer.
+ * shared-memory ring, [9] weight tiles (taps) per ring stage, [10] where the kernel's activation
+ * tiles come from: 0 = an NHWC copy of x made by the layout pass, 1 = x itself, read as
+ * pixel-major tiles (1x1 layers), 2 = a zero-bordered 8-channel NHWC copy read through
+ * overlapping windows (few input channels), 3 = an expanded copy holding, per output pixel, the
+ * values under the kernel (few input channels, strided); zeros for the other paths.
+ * info: host pointer.
  */
 int hgc_conv_plan_info(const hgc_conv_desc* d, int32_t* info, int32_t count);
 

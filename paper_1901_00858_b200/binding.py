@@ -144,9 +144,9 @@ class ConvDesc:
         return v.value
 
     def plan_info(self) -> dict:
-        v = (ctypes.c_int32 * 10)()
-        _check(lib().hgc_conv_plan_info(self._h, v, 10), "hgc_conv_plan_info")
-        keys = ("path", "kb", "halo", "tn", "th", "pitch", "ncols", "tiles", "stages", "taps")
+        v = (ctypes.c_int32 * 11)()
+        _check(lib().hgc_conv_plan_info(self._h, v, 11), "hgc_conv_plan_info")
+        keys = ("path", "kb", "halo", "tn", "th", "pitch", "ncols", "tiles", "stages", "taps", "x_source")
         return dict(zip(keys, list(v)))
 
     def workspace_bytes(self) -> int:
