@@ -182,13 +182,34 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t* v) {
 }
 
 // two fp32 -> packed fp16x2 (round to nearest even), lo = first value; optional ReLU in the convert
-__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi, bool relu) {
+template <bool RELU>
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
   uint32_t d;
-  if (relu)
+  if (RELU)
     asm("cvt.rn.relu.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
   else
     asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
   return d;
+}
+
+// `nchunks` (<= 4) chunks of 8 accumulator columns (+ bias, optional ReLU) -> 16-byte fp16 chunks
+// at dst0 ^ (chunk << 4) (the swizzled staging row of this lane).  The ReLU choice is a template
+// parameter: a run-time test around every convert costs more than the convert.
+template <bool RELU>
+__device__ __forceinline__ void convert_store(const uint32_t (&v)[32], int nchunks, float bv, uint32_t dst0,
+                                              uint32_t chunk0) {
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    if (c < nchunks) {
+      uint32_t o[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        o[i] = pack_f16x2<RELU>(__uint_as_float(v[8 * c + 2 * i]) + bv, __uint_as_float(v[8 * c + 2 * i + 1]) + bv);
+      const uint32_t dst = dst0 ^ ((chunk0 + (uint32_t)c) << 4);
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3])
+                   : "memory");
+    }
+  }
 }
 
 __device__ __forceinline__ void tma_store_4d(const CUtensorMap* tm, uint32_t src, int c0, int c1, int c2, int c3) {
@@ -402,17 +423,11 @@ __device__ __noinline__ void epilogue_copy(uint32_t t_addr, uint32_t sbuf, int f
             if (g * 32 + c * 8 < ncol) tmem_ld8(tcol + (uint32_t)(g * 32 + c * 8), &v[8 * c]);
         }
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          if (g * 32 + c * 8 < ncol) {
-            uint32_t o[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-              o[i] = pack_f16x2(__uint_as_float(v[8 * c + 2 * i]) + bv, __uint_as_float(v[8 * c + 2 * i + 1]) + bv, relu);
-            const uint32_t dst = sbuf + row_off + ((uint32_t)((g * 4 + c) ^ (lane & 7)) << 4);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3])
-                         : "memory");
-          }
+        {
+          const int nch = (ncol - g * 32 + 7) >> 3;  // chunks with real columns in this batch
+          const uint32_t dst0 = sbuf + row_off + (((uint32_t)lane & 7u) << 4);
+          if (relu) convert_store<true>(v, nch < 4 ? nch : 4, bv, dst0, (uint32_t)(g * 4));
+          else convert_store<false>(v, nch < 4 ? nch : 4, bv, dst0, (uint32_t)(g * 4));
         }
       }
       __syncwarp();
@@ -790,20 +805,8 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 __syncwarp();
               }
               asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-              for (int c = 0; c < 4; ++c) {
-                if (c < nchunks) {
-                  uint32_t o[4];
-#pragma unroll
-                  for (int i = 0; i < 4; ++i)
-                    o[i] = pack_f16x2(__uint_as_float(v[8 * c + 2 * i]) + bv, __uint_as_float(v[8 * c + 2 * i + 1]) + bv,
-                                      relu);
-                  const uint32_t dst = sbuf + (row_off ^ ((uint32_t)(g * 4 + c) << 4));
-                  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]),
-                               "r"(o[3])
-                               : "memory");
-                }
-              }
+              if (relu) convert_store<true>(v, nchunks, bv, sbuf + row_off, (uint32_t)(g * 4));
+              else convert_store<false>(v, nchunks, bv, sbuf + row_off, (uint32_t)(g * 4));
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
