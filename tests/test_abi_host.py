@@ -111,5 +111,31 @@ def test_planner_paths():
     assert mult.path() == hgc.HGC_PATH_DIRECT     # channel multiplier 2: generic kernel
 
 
+def test_plan_info_reports_tiling_and_activation_source():
+    """The planner runs on the host: its choices can be checked without a GPU."""
+    keys = {"path", "kb", "halo", "tn", "th", "pitch", "ncols", "tiles", "stages", "taps", "x_source"}
+    cases = [
+        # (n, c, h, w, k, r, s, pad, stride), x_source
+        ((16, 256, 56, 56, 256, 3, 3, 1, 1), 0),   # NHWC copy of x
+        ((64, 64, 56, 56, 256, 1, 1, 0, 1), 1),    # 1x1 on a plane of a multiple of 8 pixels: x itself
+        ((64, 1024, 14, 14, 256, 1, 1, 0, 1), 0),  # 196 pixels: rows of x are not 16-byte aligned
+        ((16, 3, 224, 224, 64, 3, 3, 1, 1), 2),    # stride-1 stem: overlapping windows
+        ((32, 3, 224, 224, 32, 3, 3, 1, 2), 3),    # strided stem: expanded copy
+    ]
+    for (n, c, h, w, k, r, s, pad, stride), source in cases:
+        d = hgc.ConvDesc(n, c, h, w, k, r, s, pad, pad, stride, stride, 1, 1, 1)
+        assert d.path() == hgc.HGC_PATH_IGEMM
+        info = d.plan_info()
+        assert set(info) == keys
+        assert info["x_source"] == source, info
+        assert info["kb"] in (16, 32, 64) and 16 <= info["ncols"] <= 256 and info["ncols"] % 16 == 0
+        assert info["tn"] >= 1 and info["th"] >= 1 and info["stages"] >= 2 and info["tiles"] >= 1
+        # an accumulator tile never holds more than 256 columns
+        assert info["tn"] * info["th"] * info["pitch"] - (info["pitch"] - d.output_dims()[3]) <= 256
+        d.close()
+    dw = hgc.ConvDesc(2, 32, 14, 14, 32, 3, 3, 1, 1, 1, 1, 1, 1, 32)
+    assert dw.plan_info()["kb"] == 0   # not the tensor-core path: zeros
+
+
 def test_launch_counter_readable():
     assert hgc.kernel_launch_count() >= 0

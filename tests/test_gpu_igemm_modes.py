@@ -1,0 +1,90 @@
+"""GPU parity of the tensor-core path, one case per way it can feed and drain the MMA: where the
+activation tiles come from (NHWC copy, x itself for 1x1 layers, overlapping windows or an
+expanded copy for few-channel stems), which epilogue writes y (TMA store, copy), tile shapes with
+several images, ragged last tiles and partially filled channel tiles.  Every case is compared
+with the CPU oracle element by element; outputs are NaN-filled before the call."""
+import zlib
+
+import numpy as np
+import pytest
+
+from paper_1901_00858_b200 import workloads
+from gpu_util import check_close, params_dict, run_layer
+
+pytestmark = pytest.mark.gpu
+
+X_NHWC_COPY, X_DIRECT, X_WINDOWS, X_PATCHES = 0, 1, 2, 3
+
+
+@pytest.fixture(scope="module")
+def hgc():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_1901_00858_b200 import binding
+    binding.lib()
+    return binding
+
+
+CASES = [
+    # (id, params, expected activation source or None)
+    ("1x1 direct 56x56 k256", params_dict(2, 64, 56, 56, 256, 1, 1), X_DIRECT),
+    ("1x1 direct 28x28 k200 (tile rows in whole 8-pixel steps)", params_dict(3, 128, 28, 28, 200, 1, 1), X_DIRECT),
+    ("1x1 direct 8x8 single tile", params_dict(1, 64, 8, 8, 128, 1, 1), X_DIRECT),
+    ("1x1 direct c40 (channel tail in the block)", params_dict(2, 40, 16, 24, 48, 1, 1), X_DIRECT),
+    ("1x1 14x14 (copy epilogue, 4-byte words)", params_dict(5, 256, 14, 14, 136, 1, 1), X_NHWC_COPY),
+    ("1x1 7x7 several images per tile", params_dict(9, 512, 7, 7, 130, 1, 1), X_NHWC_COPY),
+    ("1x1 stride 2", params_dict(2, 64, 28, 28, 96, 1, 1, 0, 0, 2, 2), X_NHWC_COPY),
+    ("1x1 grouped", params_dict(2, 64, 12, 12, 64, 1, 1, 0, 0, 1, 1, 1, 1, 4), X_NHWC_COPY),
+    ("3x3 224 wide rows k64", params_dict(1, 64, 20, 224, 64, 3, 3, 1, 1), X_NHWC_COPY),
+    ("3x3 c256 32-channel stages", params_dict(2, 256, 24, 24, 160, 3, 3, 1, 1), X_NHWC_COPY),
+    ("3x3 13x13 odd plane (copy epilogue with junk columns)", params_dict(3, 96, 13, 13, 72, 3, 3, 1, 1), X_NHWC_COPY),
+    ("3x3 7x7 several images per tile", params_dict(7, 64, 7, 7, 40, 3, 3, 1, 1), X_NHWC_COPY),
+    ("3x3 stride 2", params_dict(2, 96, 15, 15, 200, 3, 3, 1, 1, 2, 2), X_NHWC_COPY),
+    ("5x5 grouped pad 2", params_dict(1, 96, 27, 27, 256, 5, 5, 2, 2, 1, 1, 1, 1, 2), X_NHWC_COPY),
+    ("3x3 dilation 2", params_dict(2, 24, 20, 18, 30, 3, 3, 2, 2, 1, 1, 2, 2), X_NHWC_COPY),
+    ("3x1 and unpadded rows", params_dict(2, 40, 10, 40, 16, 3, 1, 1, 0), X_NHWC_COPY),
+    ("stem 3x3 c3 stride 1 (windows)", params_dict(2, 3, 32, 40, 16, 3, 3, 1, 1), X_WINDOWS),
+    ("stem 7x7 c3 stride 2 (windows)", params_dict(2, 3, 64, 64, 64, 7, 7, 3, 3, 2, 2), X_WINDOWS),
+    ("stem 11x11 c3 stride 4 (windows)", params_dict(1, 3, 67, 67, 96, 11, 11, 0, 0, 4, 4), X_WINDOWS),
+    ("stem 3x3 c3 stride 2 (patches)", params_dict(2, 3, 64, 48, 32, 3, 3, 1, 1, 2, 2), X_PATCHES),
+    ("stem 3x3 c1 stride 2 (patches)", params_dict(3, 1, 33, 31, 24, 3, 3, 1, 1, 2, 2), X_PATCHES),
+    ("stem 3x3 c4 stride 2 dilated (patches)", params_dict(2, 4, 30, 30, 20, 3, 3, 2, 2, 2, 2, 2, 2), X_PATCHES),
+    ("stem 5x5 c2 stride 3 (patches, generic expansion)", params_dict(2, 2, 29, 35, 20, 5, 5, 2, 2, 3, 3), X_PATCHES),
+    ("stem 1x1 c8 stride 2 (patches)", params_dict(2, 8, 18, 18, 16, 1, 1, 0, 0, 2, 2), X_PATCHES),
+]
+
+
+@pytest.mark.parametrize("name,a,source", CASES, ids=[c[0] for c in CASES])
+def test_igemm_mode(hgc, oracle, name, a, source):
+    rng = np.random.default_rng(zlib.crc32(name.encode()))
+    x, w, b = workloads.random_layer_tensors(rng, a["n"], a["c"], a["h"], a["w"], a["k"], a["r"], a["s"], a["group"])
+    P = oracle.ConvParams(**a)
+    d = hgc.ConvDesc(**a)
+    assert d.path() == hgc.HGC_PATH_IGEMM, name
+    if source is not None:
+        assert d.plan_info()["x_source"] == source, (name, d.plan_info())
+    d.close()
+    for relu, bias, registered in ((True, b, True), (False, None, False)):
+        ref = oracle.conv_fast(P, x, w, bias, relu)
+        got, path = run_layer(hgc, a, x, w, bias, relu, register_weights=registered)
+        assert path == hgc.HGC_PATH_IGEMM
+        check_close(got, ref, what=f"{name} relu={relu}")
+
+
+def test_same_descriptor_new_tensors(hgc, oracle):
+    """A descriptor keeps tensor maps over x and y between calls: new pointers must re-encode them."""
+    import torch
+    from gpu_util import to_dev, to_host
+    a = params_dict(2, 64, 16, 16, 128, 1, 1)
+    rng = np.random.default_rng(5)
+    d = hgc.ConvDesc(**a)
+    d.ensure_workspace()
+    P = oracle.ConvParams(**a)
+    for rep in range(3):
+        x, w, b = workloads.random_layer_tensors(rng, a["n"], a["c"], a["h"], a["w"], a["k"], 1, 1, 1)
+        xd, wd, bd = to_dev(x), to_dev(w), to_dev(b)
+        y = torch.full((2, 128, 16, 16), float("nan"), dtype=torch.float16, device="cuda")
+        hgc.conv_forward(d, xd, wd, bd, y, True)
+        torch.cuda.synchronize()
+        check_close(to_host(y), oracle.conv_fast(P, x, w, b, True), what=f"rep {rep}")
+    d.close()
