@@ -81,6 +81,11 @@ def _load():
         lib.ref_conv_points.argtypes = [pp, u16p, u16p, u16p, ctypes.c_int,
                                         ctypes.POINTER(ctypes.c_int64), ctypes.c_int64, u16p]
         lib.ref_num_threads.restype = ctypes.c_int
+        lib.ref_cast_f32_to_f16.restype = ctypes.c_int64
+        lib.ref_cast_f32_to_f16.argtypes = [ctypes.POINTER(ctypes.c_float), u16p, ctypes.c_int64]
+        lib.ref_inner_product.restype = None
+        lib.ref_inner_product.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, u16p, u16p, u16p, u16p,
+                                          ctypes.c_int]
         _lib = lib
     return _lib
 
@@ -169,6 +174,29 @@ def conv_points(p: ConvParams, x, w, bias, relu, coords) -> np.ndarray:
 
 
 # ---- data-movement steps: their definitions are permutations ----------------------------
+
+def cast_f32_to_f16(src: np.ndarray):
+    """(float16 array, number of finite inputs that became infinite): the converter's cast."""
+    lib = _load()
+    a = np.ascontiguousarray(src, dtype=np.float32)
+    out = np.empty(a.shape, dtype=np.uint16)
+    n_over = lib.ref_cast_f32_to_f16(a.ctypes.data_as(ctypes.POINTER(ctypes.c_float)),
+                                     out.ctypes.data_as(ctypes.POINTER(ctypes.c_uint16)), a.size)
+    return out.view(np.float16), int(n_over)
+
+
+def inner_product(x, w, bias=None, relu=False) -> np.ndarray:
+    """x [N,C], w [K,C], bias [K] or None (float16) -> y [N,K] float16."""
+    lib = _load()
+    xb, wb = _bits(x), _bits(w)
+    n, c = xb.shape
+    k = wb.shape[0]
+    assert wb.shape == (k, c)
+    bb = None if bias is None else _bits(bias, (k,))
+    y = np.empty((n, k), dtype=np.uint16)
+    lib.ref_inner_product(n, c, k, _u16(xb), _u16(wb), None if bb is None else _u16(bb), _u16(y), int(bool(relu)))
+    return y.view(np.float16)
+
 
 def nchw_to_nhwc(x: np.ndarray, c_pad: int) -> np.ndarray:
     """x[n][c][h][w] -> x'[n][h][w][c], channels zero-filled up to c_pad."""

@@ -31,6 +31,12 @@
  *                    (sampled checks on problems too large to compute whole)
  *   ref_out_dim      the output-size formula
  *   ref_half_to_double / ref_double_to_half   binary16 conversion used above
+ *   ref_cast_f32_to_f16   the weight-file converter's arithmetic (Section 3.4): every binary32
+ *                    value rounded to the nearest binary16, ties to even; counts the finite
+ *                    inputs that no finite binary16 can hold (they become infinities)
+ *   ref_inner_product  the inner-product (fully connected) layer, named in Section 3.1 as
+ *                    the other layer whose long sums overflow FP16:
+ *                    y[n,k] = round( relu?( bias[k] + sum_c x[n,c] * w[k,c] ) ), fp64 sum
  *
  * Parity pins: every function here is pinned by the CPU tests (hand-worked
  * examples, closed forms, matmul / correlate2d restatements, invariants).
@@ -249,6 +255,36 @@ int ref_conv_fast(const ref_conv_params* p, const uint16_t* x, const uint16_t* w
   }
   free(xf);
   return fail ? 2 : 0;
+}
+
+/* ---- FP32 -> FP16 cast (the converter's arithmetic, Section 3.4) --------- */
+
+/* dst[i] = binary16 nearest to src[i] (ties to even; |v| >= 65520 -> inf; NaN -> a quiet NaN
+   of the same sign).  Returns the number of FINITE inputs whose result is infinite. */
+int64_t ref_cast_f32_to_f16(const float* src, uint16_t* dst, int64_t count) {
+  int64_t overflow = 0;
+  for (int64_t i = 0; i < count; ++i) {
+    const double v = (double)src[i];  /* exact */
+    const uint16_t h = ref_double_to_half(v);
+    dst[i] = h;
+    if (isfinite(v) && (h & 0x7fffu) == 0x7c00u) ++overflow;
+  }
+  return overflow;
+}
+
+/* ---- inner product (fully connected) layer ------------------------------ */
+
+/* x[N][C], w[K][C], bias[K] or NULL, y[N][K]; the sum runs bias first, then c ascending */
+void ref_inner_product(int64_t n, int64_t c, int64_t k, const uint16_t* x, const uint16_t* w,
+                       const uint16_t* bias, uint16_t* y, int relu) {
+  for (int64_t in = 0; in < n; ++in) {
+    for (int64_t ik = 0; ik < k; ++ik) {
+      double acc = bias ? ref_half_to_double(bias[ik]) : 0.0;
+      for (int64_t ic = 0; ic < c; ++ic)
+        acc += ref_half_to_double(x[in * c + ic]) * ref_half_to_double(w[ik * c + ic]);
+      y[in * k + ik] = finish(acc, relu);
+    }
+  }
 }
 
 int ref_num_threads(void) {

@@ -320,3 +320,76 @@ def test_layout_definitions_round_trip(oracle):
     wp = oracle.repack_weights(wt, 3, 8)
     assert wp.shape == (3, 2, 3, 3, 8)
     assert wp[2, 1, 0, 2, 1] == wt[5, 1, 0, 2] and np.all(wp[..., 2:] == 0)
+
+
+# ---- the converter's cast and the inner-product layer (oracle functions added for the next rows) ----
+
+def test_cast_matches_numpy_on_every_class_of_value(oracle):
+    """ref_cast_f32_to_f16 against numpy's float32 -> float16 conversion (an independent
+    implementation of IEEE round-to-nearest-even): normals, subnormals, ties, overflow, signed
+    zeros, infinities; NaN stays NaN."""
+    rng = np.random.default_rng(11)
+    parts = [
+        rng.normal(0, 1, 20000), rng.normal(0, 300, 20000), rng.uniform(-70000, 70000, 20000),
+        rng.uniform(-1e-4, 1e-4, 20000), rng.uniform(-1e-7, 1e-7, 20000),   # fp16 subnormals and below
+        np.array([0.0, -0.0, np.inf, -np.inf, 65504.0, 65519.996, 65520.0, -65520.0, 65536.0, 1e30, -1e30,
+                  2.0 ** -24, 2.0 ** -25, 2.0 ** -25 * 1.0000001, 3 * 2.0 ** -25, 2.0 ** -14, 2.0 ** -14 - 2.0 ** -25]),
+        # exact ties between neighbouring fp16 values in several binades: (m + 0.5) * 2^(e-10)
+        np.array([(1024 + m + 0.5) * 2.0 ** (e - 10) for e in (-14, -3, 0, 7, 15) for m in (0, 1, 2, 511, 1022)]),
+    ]
+    src = np.concatenate(parts).astype(np.float32)
+    got, n_over = oracle.cast_f32_to_f16(src)
+    with np.errstate(over="ignore"):
+        want = src.astype(np.float16)
+    assert np.array_equal(got.view(np.uint16), want.view(np.uint16))
+    finite_in = np.isfinite(src)
+    assert n_over == int(np.count_nonzero(finite_in & np.isinf(want)))
+    assert n_over > 0
+    nan_out, n2 = oracle.cast_f32_to_f16(np.array([np.nan, -np.nan, 1.0], dtype=np.float32))
+    assert np.isnan(nan_out[0]) and np.isnan(nan_out[1]) and nan_out[2] == 1.0 and n2 == 0
+
+
+def test_cast_is_the_identity_on_values_that_are_already_fp16(oracle):
+    bits = np.arange(0, 0x10000, dtype=np.uint32).astype(np.uint16)
+    h = bits.view(np.float16)
+    keep = ~np.isnan(h)
+    got, n_over = oracle.cast_f32_to_f16(h[keep].astype(np.float32))
+    assert np.array_equal(got.view(np.uint16), bits[keep]) and n_over == 0
+
+
+def test_inner_product_matches_float64_matmul(oracle):
+    """y = x W^T + b in float64 (numpy matmul), rounded once: the oracle's loop must agree
+    bit for bit wherever the float64 sums agree, i.e. within one fp16 ulp everywhere and
+    exactly on small integer-valued data where no rounding happens at all."""
+    rng = np.random.default_rng(3)
+    x = rng.integers(-4, 5, size=(7, 33)).astype(F16)
+    w = rng.integers(-3, 4, size=(11, 33)).astype(F16)
+    b = rng.integers(-5, 6, size=(11,)).astype(F16)
+    want = (x.astype(np.float64) @ w.astype(np.float64).T + b.astype(np.float64))
+    for relu in (False, True):
+        ref = np.maximum(want, 0) if relu else want
+        got = oracle.inner_product(x, w, b, relu)
+        assert np.array_equal(got.astype(np.float64), ref)     # integers < 2048: exact in fp16
+    xr = rng.uniform(-1, 1, size=(5, 400)).astype(F16)
+    wr = rng.normal(0, 0.07, size=(9, 400)).astype(F16)
+    got = oracle.inner_product(xr, wr, None, False).astype(np.float64)
+    want = xr.astype(np.float64) @ wr.astype(np.float64).T
+    assert np.all(np.abs(got - want) <= np.abs(want) * 2.0 ** -11 + 2.0 ** -25)   # half an ulp of fp16
+
+
+def test_inner_product_is_a_1x1_convolution_on_a_1x1_plane(oracle):
+    rng = np.random.default_rng(4)
+    x = rng.uniform(-1, 1, size=(6, 50)).astype(F16)
+    w = rng.normal(0, 0.2, size=(13, 50)).astype(F16)
+    b = rng.uniform(-0.1, 0.1, size=(13,)).astype(F16)
+    P = oracle.ConvParams(6, 50, 1, 1, 13, 1, 1, 0, 0, 1, 1, 1, 1, 1)
+    conv = oracle.conv_naive(P, x.reshape(6, 50, 1, 1), w.reshape(13, 50, 1, 1), b, True)
+    fc = oracle.inner_product(x, w, b, True)
+    assert np.array_equal(conv.reshape(6, 13).view(np.uint16), fc.view(np.uint16))
+
+
+def test_wide_accumulation_in_the_inner_product(oracle):
+    """4096 ones times ones: a sum carried in FP16 stalls at 2048; the layer must give 4096."""
+    x = np.ones((1, 4096), dtype=F16)
+    w = np.ones((2, 4096), dtype=F16)
+    assert np.array_equal(oracle.inner_product(x, w, None, False), np.full((1, 2), 4096, dtype=F16))
