@@ -454,12 +454,100 @@ def run_ours(args, wl):
         dist.destroy_process_group()
 
 
+# ---- the two layers next to the convolution path (not part of the default run) ----------------
+
+def run_side_op(args):
+    """--op cast: FP32 -> FP16 cast of 64 Mi values (HBM bound, 6 bytes per element).
+    --op fc: the three inner-product layers of a VGG-16 classifier at batch 64 (25088->4096,
+    4096->4096, 4096->1000; weight-streaming, HBM bound).  One JSON line each, same keys."""
+    import torch
+    from paper_1901_00858_b200 import binding as hgc
+    import oracle
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the CUDA path has no CPU fallback")
+    hgc.lib()
+    peaks = load_peaks()
+    stream = torch.cuda.current_stream()
+    steps, warm = args.steps, max(args.warmup, 3)
+    if args.op == "cast":
+        count = 64 << 20
+        nbuf = 3   # rotate buffers: 1.1 GB footprint, far larger than L2
+        srcs = [torch.randn(count, dtype=torch.float32, device="cuda") for _ in range(nbuf)]
+        dsts = [torch.empty(count, dtype=torch.float16, device="cuda") for _ in range(nbuf)]
+        over = torch.zeros(1, dtype=torch.int64, device="cuda")
+        step = lambda i: hgc.cast_f32_to_f16(srcs[i % nbuf], dsts[i % nbuf], overflow_count=over, stream=stream)
+        step_bytes, step_flops = 6.0 * count, 0.0
+        metric, unit, workload = "cast_f32_to_f16_gbs", "GB/s", "cast_64Mi"
+        sample = np.random.default_rng(0).normal(0, 1, 16 << 20).astype(np.float32)
+        t0 = time.perf_counter(); oracle.cast_f32_to_f16(sample); dt = time.perf_counter() - t0
+        cpu = {"value": 6.0 * sample.size / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+               "sample": f"{sample.size} values once ({dt:.2f} s)"}
+    else:
+        n = 64
+        shapes = [(25088, 4096), (4096, 4096), (4096, 1000)]
+        layers = []
+        for c, k in shapes:
+            d = hgc.ConvDesc.inner_product(n, c, k)
+            d.ensure_workspace()
+            x = torch.rand((n, c), dtype=torch.float16, device="cuda")
+            w = torch.randn((k, c), dtype=torch.float16, device="cuda") * float(np.sqrt(2.0 / c))
+            b = torch.zeros(k, dtype=torch.float16, device="cuda")
+            y = torch.empty((n, k), dtype=torch.float16, device="cuda")
+            d.set_weights(w)
+            layers.append((d, x, w, b, y))
+        def step(i):
+            for d, x, w, b, y in layers:
+                hgc.conv_forward(d, x, w, b, y, True, stream)
+        step_flops = sum(2.0 * n * c * k for c, k in shapes)
+        step_bytes = sum(2.0 * (n * c + c * k + k + n * k) for c, k in shapes)
+        metric, unit, workload = "inner_product_tflops", "TFLOP/s", "vgg16_classifier_n64"
+        rng = np.random.default_rng(0)
+        t0 = time.perf_counter()
+        oracle.inner_product(rng.uniform(-1, 1, (4, 4096)).astype(np.float16),
+                             rng.normal(0, 0.02, (1000, 4096)).astype(np.float16), None, True)
+        dt = time.perf_counter() - t0
+        cpu = {"value": 2.0 * 4 * 4096 * 1000 / dt / 1e12, "unit": "TFLOP/s", "cores": 1, "kind": "oracle",
+               "sample": f"4096->1000 at batch 4 once ({dt:.2f} s)"}
+    sampler = ClockSampler(0)
+    sampler.start()
+    for i in range(warm):
+        step(i)
+    torch.cuda.synchronize()
+    c0 = hgc.kernel_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    host_t0 = time.time()
+    e0.record(stream)
+    for i in range(steps):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    host_t1 = time.time()
+    ms = e0.elapsed_time(e1) / steps
+    gbs = step_bytes / (ms * 1e-3) / 1e9
+    value = gbs if args.op == "cast" else step_flops / (ms * 1e-3) / 1e12
+    line = {"metric": metric, "value": value, "unit": unit, "n_gpus": 1, "steps": steps, "warmup": warm,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32 -> f16" if args.op == "cast" else "f16 (f32 accumulate)", "data": "synthetic",
+            "config": {"workload": workload, "l2": "buffers rotate over a footprint larger than L2" if args.op == "cast"
+                       else "weights (278 MB) larger than L2", "launch": "eager"},
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]},
+            "cpu_baseline": cpu, "gpu_launches": hgc.kernel_launch_count() - c0,
+            "e2e": {"value": None, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                    "note": "side operation: device-resident timing only"},
+            "clocks": sampler.stop((host_t0, host_t1))}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--op", choices=["conv", "cast", "fc"], default="conv",
+                    help="conv: the convolution path (default); cast / fc: the FP32->FP16 cast and the "
+                         "inner-product layer, measured on their own")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD,
                     help="one of: " + ", ".join(w.name for w in workloads.all_workloads()))
     ap.add_argument("--layers", action="store_true", help="add per-layer figures to the JSON line")
@@ -469,6 +557,10 @@ def main():
     ap.add_argument("--only", default="", help="comma-separated layer names: run just these layers (profiling)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling on a small case)")
     args = ap.parse_args()
+    if args.op != "conv":
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_side_op(args)
+        return
     wl = workloads.by_name(args.workload)
     if args.impl == "reference":
         run_reference(args, wl)

@@ -201,6 +201,28 @@ int hgc_layout_nhwc_to_nchw(const void* src, void* dst, int32_t n, int32_t c, in
 int hgc_weights_repack(const void* src, void* dst, int32_t k, int32_t c_per_group, int32_t r,
                        int32_t s, int32_t group, int32_t c_pad, void* stream);
 
+/*
+ * Inner-product (fully connected) layer, the other layer the paper names as overflowing in FP16
+ * because of its long sums (Section 3.1):  y[n][k] = relu?( bias[k] + sum_c x[n][c] * w[k][c] ),
+ * FP16 storage, FP32 accumulation, one rounding.  It is the convolution of this library on a 1x1
+ * plane with a 1x1 kernel: this call creates exactly that descriptor (x: [n][c], w: [k][c],
+ * y: [n][k], all dense FP16), to be used with hgc_conv_forward and the other descriptor calls.
+ * n, c, k >= 1.  Errors as hgc_conv_desc_create.
+ */
+int hgc_inner_product_desc_create(hgc_conv_desc** out, int32_t n, int32_t c, int32_t k);
+
+/*
+ * FP32 -> FP16 cast, the arithmetic of a weight-file converter (Section 3.4: models are stored
+ * in FP32 and converted once to an FP16 copy): dst[i] = the binary16 value nearest to src[i],
+ * ties to even; magnitudes >= 65520 become infinities, NaNs stay NaNs.
+ * src: `count` floats, dst: `count` binary16 values, device pointers, 16-byte aligned, not
+ * overlapping.  overflow_count: device pointer to a 64-bit counter or NULL; the kernel ADDS the
+ * number of finite inputs that became infinite (zero it first; read it after the stream has
+ * finished).  Queued on `stream`; nothing is allocated.  count == 0 is a no-op.
+ * Errors: HGC_INVALID_ARG (NULL src/dst, count < 0), HGC_BAD_ALIGNMENT, HGC_CUDA_ERROR.
+ */
+int hgc_cast_f32_to_f16(const void* src, void* dst, int64_t count, uint64_t* overflow_count, void* stream);
+
 /* Number of kernels this library has launched in this process so far. */
 int hgc_kernel_launch_count(uint64_t* count);
 

@@ -51,6 +51,8 @@ def lib() -> ctypes.CDLL:
         L.hgc_conv_forward.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int, vp]
         L.hgc_conv_forward_host.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int, vp]
         L.hgc_conv_forward_static.argtypes = [ctypes.POINTER(hgc_conv_params), vp, vp, vp, vp, ctypes.c_int, vp]
+        L.hgc_inner_product_desc_create.argtypes = [ctypes.POINTER(ctypes.c_void_p), i32, i32, i32]
+        L.hgc_cast_f32_to_f16.argtypes = [vp, vp, ctypes.c_int64, vp, vp]
         L.hgc_conv_output_dims.argtypes = [vp, i32p, i32p, i32p, i32p]
         L.hgc_conv_path.argtypes = [vp, i32p]
         L.hgc_conv_plan_info.argtypes = [vp, i32p, i32]
@@ -70,7 +72,7 @@ def lib() -> ctypes.CDLL:
                      "hgc_conv_workspace_bytes", "hgc_conv_host_workspace_bytes", "hgc_conv_plan_info",
                      "hgc_conv_set_workspace", "hgc_conv_set_weights", "hgc_conv_last_device_status",
                      "hgc_layout_nchw_to_nhwc", "hgc_layout_nhwc_to_nchw", "hgc_weights_repack",
-                     "hgc_kernel_launch_count"):
+                     "hgc_kernel_launch_count", "hgc_inner_product_desc_create", "hgc_cast_f32_to_f16"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -116,6 +118,17 @@ class ConvDesc:
         self._ws = None
         _check(lib().hgc_conv_desc_create(ctypes.byref(self._h), ctypes.byref(self.params)),
                "hgc_conv_desc_create")
+
+    @classmethod
+    def inner_product(cls, n, c, k):
+        """hgc_inner_product_desc_create: the fully connected layer x[n][c] . w[k][c]^T + bias as
+        the 1x1 convolution on a 1x1 plane; use with conv_forward (x, y may be 2-D tensors)."""
+        self = cls.__new__(cls)
+        self.params = hgc_conv_params(n, c, 1, 1, k, 1, 1, 0, 0, 1, 1, 1, 1, 1, 0)
+        self._h = ctypes.c_void_p()
+        self._ws = None
+        _check(lib().hgc_inner_product_desc_create(ctypes.byref(self._h), n, c, k), "hgc_inner_product_desc_create")
+        return self
 
     @property
     def handle(self):
@@ -205,6 +218,14 @@ def conv_forward_static(params: hgc_conv_params, x, w, bias, y, relu: bool, stre
     hgc_conv_params; x, w, bias (or None), y are CUDA fp16 tensors (or raw addresses)."""
     _check(lib().hgc_conv_forward_static(ctypes.byref(params), _ptr(x), _ptr(w), _ptr(bias), _ptr(y),
                                          int(bool(relu)), _stream(stream)), "hgc_conv_forward_static")
+
+
+def cast_f32_to_f16(src, dst, count=None, overflow_count=None, stream=None):
+    """hgc_cast_f32_to_f16: src float32 -> dst float16 CUDA tensors (round to nearest even);
+    overflow_count: a 1-element int64 CUDA tensor that the kernel adds to, or None."""
+    n = src.numel() if count is None else count
+    _check(lib().hgc_cast_f32_to_f16(_ptr(src), _ptr(dst), n, _ptr(overflow_count), _stream(stream)),
+           "hgc_cast_f32_to_f16")
 
 
 def layout_nchw_to_nhwc(src, dst, n, c, h, w, c_pad, stream=None):

@@ -302,6 +302,25 @@ int hgc_weights_repack(const void* src, void* dst, int32_t k, int32_t c_per_grou
   return err == cudaSuccess ? HGC_OK : HGC_CUDA_ERROR;
 }
 
+int hgc_inner_product_desc_create(hgc_conv_desc** out, int32_t n, int32_t c, int32_t k) {
+  hgc_conv_params p{};
+  p.n = n; p.c = c; p.h = 1; p.w = 1; p.k = k; p.r = 1; p.s = 1;
+  p.pad_h = 0; p.pad_w = 0; p.stride_h = 1; p.stride_w = 1; p.dil_h = 1; p.dil_w = 1; p.group = 1; p.flags = 0;
+  return hgc_conv_desc_create(out, &p);
+}
+
+int hgc_cast_f32_to_f16(const void* src, void* dst, int64_t count, uint64_t* overflow_count, void* stream) {
+  if (count < 0 || (count > 0 && (src == nullptr || dst == nullptr))) return HGC_INVALID_ARG;
+  if (count == 0) return HGC_OK;
+  if (misaligned(src) || misaligned(dst) || (reinterpret_cast<uintptr_t>(overflow_count) & 7u) != 0)
+    return HGC_BAD_ALIGNMENT;
+  const cudaError_t err =
+      hgc::launch_cast_f32_to_f16(static_cast<const float*>(src), static_cast<__half*>(dst), count,
+                                  reinterpret_cast<unsigned long long*>(overflow_count),
+                                  static_cast<cudaStream_t>(stream));
+  return err == cudaSuccess ? HGC_OK : HGC_CUDA_ERROR;
+}
+
 int hgc_kernel_launch_count(uint64_t* count) {
   if (count == nullptr) return HGC_INVALID_ARG;
   *count = hgc::g_launches.load(std::memory_order_relaxed);

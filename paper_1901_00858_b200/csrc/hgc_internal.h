@@ -40,6 +40,9 @@ cudaError_t launch_weights_repack_window(const __half* src, __half* dst, int32_t
 cudaError_t launch_weights_repack(const __half* src, __half* dst, int32_t k, int32_t cg, int32_t r,
                                   int32_t s, int32_t group, int32_t c_pad, cudaStream_t stream);
 
+cudaError_t launch_cast_f32_to_f16(const float* src, __half* dst, int64_t count, unsigned long long* overflow,
+                                   cudaStream_t stream);
+
 // Plan of the tcgen05 implicit-GEMM path for one layer (host side).
 struct IgemmPlan {
   int32_t kb, cblocks, cw, c_pad;
