@@ -59,6 +59,7 @@ struct IgemmPlan {
   int32_t tma_store, rem, nbuf;
   void* y_mapped;  // output pointer tmY/tmYr were encoded for
   uint32_t a_bytes, b_bytes, b_alloc;
+  int32_t a_rows;  // rows of a weight tile in shared memory (128, or 64 for layers of <= 64 channels per group)
   size_t smem_bytes;
   size_t ws_status_off, ws_w_off, ws_x_off, ws_total;
   bool maps_ready;

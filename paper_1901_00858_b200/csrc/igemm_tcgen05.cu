@@ -1009,7 +1009,11 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   const int64_t total = (int64_t)p.tiles_n * p.tiles_h * mg;
   if (total > 0x7fffffffLL) return false;
   p.total_tiles = (int32_t)total;
-  p.a_bytes = 128u * p.kb * 2u;
+  // weight tile rows: 128, or 64 when the layer has at most 64 output channels per group (the MMA
+  // still reads 128 rows: the upper 64 come from whatever follows in shared memory and land in
+  // accumulator lanes that no epilogue warp reads; half the tile bytes, one more ring stage)
+  p.a_rows = g.kg <= 64 ? 64 : 128;
+  p.a_bytes = (uint32_t)p.a_rows * p.kb * 2u;
   const uint32_t box_rows = (uint32_t)(p.tn * p.th * p.pitch);
   p.b_bytes = box_rows * p.kb * 2u;
   // rows the MMA may touch: the last tap starts (S-1)*dil rows in and reads ncols rows
@@ -1082,7 +1086,7 @@ bool igemm_encode_maps(const ConvGeom& g, IgemmPlan* p, void* ws) {
     const cuuint64_t kred = (cuuint64_t)p->eff_r * p->eff_s * p->cw;
     cuuint64_t dims[3] = {kred, (cuuint64_t)g.kg, (cuuint64_t)g.group};
     cuuint64_t strides[2] = {kred * 2, kred * 2 * (cuuint64_t)g.kg};
-    cuuint32_t box[3] = {(cuuint32_t)p->kb, 128, 1};
+    cuuint32_t box[3] = {(cuuint32_t)p->kb, (cuuint32_t)p->a_rows, 1};
     cuuint32_t es[3] = {1, 1, 1};
     if (enc(&p->tmA, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, base + p->ws_w_off, dims, strides, box, es,
             CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
