@@ -57,6 +57,7 @@ struct IgemmPlan {
   int32_t stages, taps;
   uint32_t stage_bytes;
   int32_t tma_store, rem, nbuf;
+  int32_t epi_warps;  // epilogue warps of the launch: 8, or 16 for tiles bound by the epilogue
   void* y_mapped;  // output pointer tmY/tmYr were encoded for
   uint32_t a_bytes, b_bytes, b_alloc;
   int32_t a_rows;  // rows of a weight tile in shared memory (128, or 64 for layers of <= 64 channels per group)

@@ -29,13 +29,12 @@
 namespace hgc {
 namespace {
 
-constexpr int kEpilogueWarps = 8;  // two per TMEM lane quarter
-constexpr int kIgemmThreads = 64 + 32 * kEpilogueWarps;
+constexpr int kEpilogueWarps = 8;       // two per TMEM lane quarter (the default)
+constexpr int kEpilogueWarpsWide = 16;  // four per quarter: layers whose tiles are bound by the epilogue
 constexpr int kPassElems = 64;               // output pixels per channel staged per TMA store
 // one warp's staging tile: 32 channels x 64 pixels for the TMA-store epilogue (4 KB, 1024-byte
 // aligned), or 32 rows of 144 bytes for the row epilogue (4.5 KB)
 constexpr uint32_t kWarpStageBytes = 5120u;
-constexpr uint32_t kStageBufBytes = kEpilogueWarps * kWarpStageBytes;  // one such tile per epilogue warp
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -555,8 +554,8 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 
 // Persistent kernel: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...; the two TMEM
 // accumulators alternate so that the epilogue of one tile overlaps the MMAs of the next.
-template <int KB, bool HALO>
-__global__ void __launch_bounds__(kIgemmThreads, 1)
+template <int KB, bool HALO, int EW>
+__global__ void __launch_bounds__(64 + 32 * EW, 1)
 igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
              const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmYr,
              const IgemmArgs a, const __half* __restrict__ bias, __half* __restrict__ y, int* status) {
@@ -581,7 +580,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(smem_u32(&acc_full[s]), 1);
-      mbar_init(smem_u32(&acc_empty[s]), kEpilogueWarps);  // one arrival per epilogue warp
+      mbar_init(smem_u32(&acc_empty[s]), EW);  // one arrival per epilogue warp
     }
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -719,10 +718,12 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     }
   } else {
     // ---------------- epilogue (warps 2..9) ----------------
-    // Warp w may read TMEM lanes 32*(w%4)..+31; the two warps of a lane quarter split the columns.
+    // Warp w may read TMEM lanes 32*(w%4)..+31; the EW/4 warps of a lane quarter take the units of
+    // a tile in turn.
+    constexpr int kPerQuarter = EW / 4;
     const int ew = warp - 2;
     const int quarter = warp & 3;
-    const int half = ew >> 2;
+    const int half = ew >> 2;  // which of the quarter's warps this is
     const int row = quarter * 32 + lane;  // accumulator lane = output channel within the tile
     uint16_t* yb = reinterpret_cast<uint16_t*>(y);
     const uint32_t stage_base = ring_base + (uint32_t)a.stages * a.stage_bytes;
@@ -763,7 +764,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           const bool linear = a.pitch == a.Q;  // no junk columns: accumulator columns are consecutive pixels
           int hr = 0, wc = half * kPassElems;
           while (!linear && wc >= a.Q) { wc -= a.Q; ++hr; }
-          for (int e_lo = half * kPassElems; e_lo < e_valid; e_lo += 2 * kPassElems, ++unit_ctr) {
+          for (int e_lo = half * kPassElems; e_lo < e_valid; e_lo += kPerQuarter * kPassElems, ++unit_ctr) {
             const int e_hi = e_lo + kPassElems < e_valid ? e_lo + kPassElems : e_valid;
             const uint32_t sbuf = my_stage + stage_sel * kWarpStageBytes;
             stage_sel = a.nbuf == 2 ? stage_sel ^ 1u : 0u;
@@ -815,8 +816,8 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
               tma_store_4d(full_box ? &tmY : &tmYr, sbuf, p0 * a.Q + e_lo, m0 + quarter * 32, grp, n0);
               asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             }
-            // first pixel of this warp's next unit: two units further on
-            wc += 2 * kPassElems;
+            // first pixel of this warp's next unit
+            wc += kPerQuarter * kPassElems;
             while (!linear && wc >= a.Q) { wc -= a.Q; ++hr; }
           }
         }
@@ -827,11 +828,14 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       } else {
         // ---- direct epilogue: each thread stores runs of its own channel plane ----
         {
-          // the two warps of a lane quarter take alternate units
-          if (quarter_live) {
-            const int kleft = a.kg - (m0 + quarter * 32);
-            epilogue_copy(t_addr, my_stage, half, 2, a.tn, a.th, a.pitch, a.N, a.K, a.P, a.Q, n0, p0,
-                          grp * a.kg + m0 + quarter * 32, kleft < 32 ? kleft : 32, bv, relu, yb);
+          // the warps of a lane quarter take alternate units (the wide variant is only launched
+          // for layers that take the TMA-store epilogue: it must fit 96 registers per thread)
+          if constexpr (EW == kEpilogueWarps) {
+            if (quarter_live) {
+              const int kleft = a.kg - (m0 + quarter * 32);
+              epilogue_copy(t_addr, my_stage, half, kPerQuarter, a.tn, a.th, a.pitch, a.N, a.K, a.P, a.Q, n0, p0,
+                            grp * a.kg + m0 + quarter * 32, kleft < 32 ? kleft : 32, bv, relu, yb);
+            }
           }
         }
         // this warp has read its lanes of the accumulator: hand the buffer back to the MMA issuer
@@ -1028,10 +1032,16 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
                     ? 1
                     : 0;
   p.rem = (p.th * g.q) % kPassElems;
+  // epilogue warps: 16 when the main loop of a tile is shorter than its epilogue (1x1 layers of
+  // few input channels, stems) and the layer takes the TMA-store epilogue, else 8
+  p.epi_warps = kEpilogueWarps;
+  if (p.tma_store && mpt * 130.0 < 600.0 + 10.0 * p.ncols && (p.th * g.q) > 2 * kPassElems)
+    p.epi_warps = kEpilogueWarpsWide;
+  const size_t stage_buf_bytes = (size_t)p.epi_warps * kWarpStageBytes;
   // rings: B two or three deep, A with what is left (each A stage feeds kb/16 MMAs).  227 KB per
   // CTA minus alignment slack, static barriers and the two epilogue staging buffers.
   const size_t budget_all = 232448u - 1024u - 512u;
-  const size_t budget = budget_all - kStageBufBytes;
+  const size_t budget = budget_all - stage_buf_bytes;
   // ring of stages: one activation tile + `taps` weight tiles each, at least two deep; if the
   // S taps of a kernel row do not fit twice, fall back to one tap (and its own tile) per stage
   for (;;) {
@@ -1057,8 +1067,8 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
     p.ncols = (p.tn * p.th * g.q + 15) / 16 * 16;
   }
   // a second staging tile per epilogue warp (its store overlaps the next unit) if memory is left
-  p.nbuf = ((size_t)p.stages * p.stage_bytes + 2u * kStageBufBytes <= budget_all) ? 2 : 1;
-  p.smem_bytes = (size_t)p.stages * p.stage_bytes + (size_t)p.nbuf * kStageBufBytes + 1024;
+  p.nbuf = ((size_t)p.stages * p.stage_bytes + 2u * stage_buf_bytes <= budget_all) ? 2 : 1;
+  p.smem_bytes = (size_t)p.stages * p.stage_bytes + (size_t)p.nbuf * stage_buf_bytes + 1024;
   // more than half of an SM's shared memory: at most one CTA per SM, so that the kernel can take
   // all 512 TMEM columns without ever waiting for another CTA to free them
   if (p.smem_bytes < 120u * 1024u) p.smem_bytes = 120u * 1024u;
@@ -1216,13 +1226,18 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
   dim3 grid((unsigned)(p.total_tiles < sms ? p.total_tiles : sms));
   int* status = reinterpret_cast<int*>(static_cast<char*>(ws) + p.ws_status_off);
   cudaError_t err = cudaSuccess;
-#define HGC_LAUNCH_IGEMM(KBV, HALOV)                                                                     \
+#define HGC_LAUNCH_IGEMM_EW(KBV, HALOV, EWV)                                                             \
   do {                                                                                                   \
-    err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV>, cudaFuncAttributeMaxDynamicSharedMemorySize,    \
+    err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV, EWV>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                (int)p.smem_bytes);                                                       \
     if (err == cudaSuccess)                                                                              \
-      igemm_kernel<KBV, HALOV><<<grid, kIgemmThreads, p.smem_bytes, stream>>>(p.tmA, p.tmB, p.tmY, p.tmYr, a,   \
-                                                                              bias, y, status);          \
+      igemm_kernel<KBV, HALOV, EWV><<<grid, 64 + 32 * EWV, p.smem_bytes, stream>>>(p.tmA, p.tmB, p.tmY,   \
+                                                                                  p.tmYr, a, bias, y, status); \
+  } while (0)
+#define HGC_LAUNCH_IGEMM(KBV, HALOV)                                              \
+  do {                                                                            \
+    if (p.epi_warps == kEpilogueWarpsWide) HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 16);   \
+    else HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 8);                                      \
   } while (0)
   if (p.kb == 64) {
     if (p.halo) HGC_LAUNCH_IGEMM(64, true); else HGC_LAUNCH_IGEMM(64, false);
@@ -1231,6 +1246,7 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
   } else {
     if (p.halo) HGC_LAUNCH_IGEMM(16, true); else HGC_LAUNCH_IGEMM(16, false);
   }
+#undef HGC_LAUNCH_IGEMM_EW
 #undef HGC_LAUNCH_IGEMM
   if (err != cudaSuccess) return err;
   count_launch();
