@@ -223,6 +223,18 @@ int hgc_inner_product_desc_create(hgc_conv_desc** out, int32_t n, int32_t c, int
  */
 int hgc_cast_f32_to_f16(const void* src, void* dst, int64_t count, uint64_t* overflow_count, void* stream);
 
+/*
+ * Launch overlap (off by default).  With enabled != 0 the library launches its kernels with the
+ * programmatic stream serialization attribute: a kernel may be scheduled while the previous
+ * kernel of the stream is still draining, and waits, before it touches global memory, until that
+ * kernel has completed.  Results are the same either way.  Measured on B200: with eager launches
+ * the gap between dependent kernels shrinks (a VGG-16 step 0.776 -> 0.757 ms, ResNet-50 1.76 ->
+ * 1.69 ms); a step replayed as a CUDA graph gets slower with programmatic edges (0.657 -> 0.737
+ * ms), which is why it is off unless asked for.  Applies to all later launches of this process.
+ * Always returns HGC_OK.
+ */
+int hgc_set_launch_overlap(int enabled);
+
 /* Number of kernels this library has launched in this process so far. */
 int hgc_kernel_launch_count(uint64_t* count);
 

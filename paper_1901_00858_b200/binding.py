@@ -65,6 +65,7 @@ def lib() -> ctypes.CDLL:
         L.hgc_layout_nhwc_to_nchw.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp]
         L.hgc_weights_repack.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, vp]
         L.hgc_kernel_launch_count.argtypes = [ctypes.POINTER(ctypes.c_uint64)]
+        L.hgc_set_launch_overlap.argtypes = [ctypes.c_int]
         L.hgc_status_string.argtypes = [ctypes.c_int]
         L.hgc_status_string.restype = ctypes.c_char_p
         for name in ("hgc_conv_desc_create", "hgc_conv_desc_destroy", "hgc_conv_forward",
@@ -72,7 +73,8 @@ def lib() -> ctypes.CDLL:
                      "hgc_conv_workspace_bytes", "hgc_conv_host_workspace_bytes", "hgc_conv_plan_info",
                      "hgc_conv_set_workspace", "hgc_conv_set_weights", "hgc_conv_last_device_status",
                      "hgc_layout_nchw_to_nhwc", "hgc_layout_nhwc_to_nchw", "hgc_weights_repack",
-                     "hgc_kernel_launch_count", "hgc_inner_product_desc_create", "hgc_cast_f32_to_f16"):
+                     "hgc_kernel_launch_count", "hgc_inner_product_desc_create", "hgc_cast_f32_to_f16",
+                     "hgc_set_launch_overlap"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -241,6 +243,11 @@ def layout_nhwc_to_nchw(src, dst, n, c, h, w, c_pad, stream=None):
 def weights_repack(src, dst, k, c_per_group, r, s, group, c_pad, stream=None):
     _check(lib().hgc_weights_repack(_ptr(src), _ptr(dst), k, c_per_group, r, s, group, c_pad,
                                     _stream(stream)), "hgc_weights_repack")
+
+
+def set_launch_overlap(enabled: bool) -> None:
+    """hgc_set_launch_overlap: programmatic dependent launch of the library's kernels on/off."""
+    _check(lib().hgc_set_launch_overlap(int(bool(enabled))), "hgc_set_launch_overlap")
 
 
 def kernel_launch_count() -> int:

@@ -8,6 +8,9 @@
 namespace hgc {
 static std::atomic<uint64_t> g_launches{0};
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+static std::atomic<bool> g_launch_overlap{false};
+bool launch_overlap_enabled() { return g_launch_overlap.load(std::memory_order_relaxed); }
+void set_launch_overlap(bool on) { g_launch_overlap.store(on, std::memory_order_relaxed); }
 }  // namespace hgc
 
 struct hgc_conv_desc {
@@ -319,6 +322,11 @@ int hgc_cast_f32_to_f16(const void* src, void* dst, int64_t count, uint64_t* ove
                                   reinterpret_cast<unsigned long long*>(overflow_count),
                                   static_cast<cudaStream_t>(stream));
   return err == cudaSuccess ? HGC_OK : HGC_CUDA_ERROR;
+}
+
+int hgc_set_launch_overlap(int enabled) {
+  hgc::set_launch_overlap(enabled != 0);
+  return HGC_OK;
 }
 
 int hgc_kernel_launch_count(uint64_t* count) {

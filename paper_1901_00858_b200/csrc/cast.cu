@@ -22,6 +22,7 @@ __device__ __forceinline__ int overflows(float v) { return fabsf(v) >= 65520.f &
 __global__ void __launch_bounds__(256)
 cast_f32_to_f16_kernel(const float* __restrict__ src, uint16_t* __restrict__ dst, int64_t count,
                        unsigned long long* __restrict__ overflow) {
+  grid_dependency_wait();
   const int64_t groups = count >> 3;
   int over = 0;
   for (int64_t gidx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; gidx < groups;
@@ -57,7 +58,7 @@ cudaError_t launch_cast_f32_to_f16(const float* src, __half* dst, int64_t count,
   const int64_t cap = (int64_t)sm_count() * 16;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
-  cast_f32_to_f16_kernel<<<(unsigned)blocks, 256, 0, stream>>>(src, reinterpret_cast<uint16_t*>(dst), count, overflow);
+  launch_kernel(cast_f32_to_f16_kernel, dim3((unsigned)blocks), dim3(256), 0, stream, src, reinterpret_cast<uint16_t*>(dst), count, overflow);
   count_launch();
   return cudaGetLastError();
 }

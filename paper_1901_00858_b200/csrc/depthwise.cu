@@ -34,6 +34,7 @@ template <int S>
 __global__ void __launch_bounds__(kThreads)
 depthwise3x3_kernel(DwPlan a, const uint16_t* __restrict__ x, const __half* __restrict__ w,
                     const __half* __restrict__ bias, uint16_t* __restrict__ y, int relu) {
+  grid_dependency_wait();
   extern __shared__ __align__(16) uint16_t smem[];
   uint16_t* sin = smem;
   uint16_t* sout = smem + a.smem_in;
@@ -204,6 +205,7 @@ __global__ void __launch_bounds__(256, 4)
 depthwise3x3_rowvec_kernel(const uint16_t* __restrict__ x, const __half* __restrict__ w,
                            const __half* __restrict__ bias, uint16_t* __restrict__ y, int c, int h, int wd,
                            int p, int q, int relu, int64_t total_items, int vec_per_row, int strips) {
+  grid_dependency_wait();
   // item = (plane, strip, vector); the vectors of a row are consecutive lanes.  32-bit index
   // arithmetic (the launcher checks that the item count fits).
   const uint32_t item = blockIdx.x * blockDim.x + threadIdx.x;
@@ -335,6 +337,7 @@ __global__ void __launch_bounds__(256)
 depthwise3x3_smallrow_kernel(const uint16_t* __restrict__ x, const __half* __restrict__ w,
                              const __half* __restrict__ bias, uint16_t* __restrict__ y, int c, int h, int p, int relu,
                              int64_t total_rows) {
+  grid_dependency_wait();
   constexpr int Q = (W - 1) / S + 1;  // kernel 3, pad 1
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= total_rows) return;
@@ -485,10 +488,10 @@ cudaError_t launch_depthwise3x3(const ConvGeom& g, const __half* x, const __half
       const uint16_t* xs0 = reinterpret_cast<const uint16_t*>(x);
       uint16_t* ys0 = reinterpret_cast<uint16_t*>(y);
       if (g.stride_h == 1)
-        depthwise3x3_rowvec_kernel<1, 4><<<(unsigned)blocks, 256, 0, stream>>>(xs0, w, bias, ys0, g.c, g.h, g.w, g.p,
+        launch_kernel(depthwise3x3_rowvec_kernel<1, 4>, dim3((unsigned)blocks), dim3(256), 0, stream, xs0, w, bias, ys0, g.c, g.h, g.w, g.p,
                                                                                g.q, relu, items, vec_per_row, strips);
       else
-        depthwise3x3_rowvec_kernel<2, 2><<<(unsigned)blocks, 256, 0, stream>>>(xs0, w, bias, ys0, g.c, g.h, g.w, g.p,
+        launch_kernel(depthwise3x3_rowvec_kernel<2, 2>, dim3((unsigned)blocks), dim3(256), 0, stream, xs0, w, bias, ys0, g.c, g.h, g.w, g.p,
                                                                                g.q, relu, items, vec_per_row, strips);
       count_launch();
       return cudaGetLastError();
@@ -502,7 +505,7 @@ cudaError_t launch_depthwise3x3(const ConvGeom& g, const __half* x, const __half
       uint16_t* ys0 = reinterpret_cast<uint16_t*>(y);
       const unsigned gb = (unsigned)blocks;
 #define HGC_DW_SMALLROW(WV, SV) \
-  depthwise3x3_smallrow_kernel<WV, SV><<<gb, 256, 0, stream>>>(xs0, w, bias, ys0, g.c, g.h, g.p, relu, rows)
+  launch_kernel(depthwise3x3_smallrow_kernel<WV, SV>, dim3(gb), dim3(256), 0, stream, xs0, w, bias, ys0, g.c, g.h, g.p, relu, rows)
       if (g.w == 28 && g.stride_h == 1) HGC_DW_SMALLROW(28, 1);
       else if (g.w == 28) HGC_DW_SMALLROW(28, 2);
       else if (g.w == 14 && g.stride_h == 1) HGC_DW_SMALLROW(14, 1);
@@ -523,11 +526,11 @@ cudaError_t launch_depthwise3x3(const ConvGeom& g, const __half* x, const __half
   if (g.stride_h == 1) {
     err = cudaFuncSetAttribute(depthwise3x3_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
-    depthwise3x3_kernel<1><<<(unsigned)ctas, kThreads, smem, stream>>>(a, xs, w, bias, ys, relu);
+    launch_kernel(depthwise3x3_kernel<1>, dim3((unsigned)ctas), dim3(kThreads), smem, stream, a, xs, w, bias, ys, relu);
   } else {
     err = cudaFuncSetAttribute(depthwise3x3_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
-    depthwise3x3_kernel<2><<<(unsigned)ctas, kThreads, smem, stream>>>(a, xs, w, bias, ys, relu);
+    launch_kernel(depthwise3x3_kernel<2>, dim3((unsigned)ctas), dim3(kThreads), smem, stream, a, xs, w, bias, ys, relu);
   }
   count_launch();
   return cudaGetLastError();

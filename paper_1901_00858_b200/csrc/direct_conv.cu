@@ -18,6 +18,7 @@ template <int KT>
 __global__ void __launch_bounds__(kThreads)
 direct_conv_kernel(ConvGeom g, const __half* __restrict__ x, const __half* __restrict__ w,
                    const __half* __restrict__ bias, __half* __restrict__ y, int relu) {
+  grid_dependency_wait();
   __shared__ float ws[KT][kChunk];
 
   // blockIdx.x = (n * ktiles + ktile) * px_tiles + px_tile
@@ -107,9 +108,9 @@ cudaError_t launch_direct_conv(const ConvGeom& g, const __half* x, const __half*
   if (total > 2147483647.0) return cudaErrorInvalidConfiguration;
   dim3 grid((unsigned)(px_tiles * ktiles * g.n));
   if (kt == 8)
-    direct_conv_kernel<8><<<grid, kThreads, 0, stream>>>(g, x, w, bias, y, relu);
+    launch_kernel(direct_conv_kernel<8>, dim3(grid), dim3(kThreads), 0, stream, g, x, w, bias, y, relu);
   else
-    direct_conv_kernel<1><<<grid, kThreads, 0, stream>>>(g, x, w, bias, y, relu);
+    launch_kernel(direct_conv_kernel<1>, dim3(grid), dim3(kThreads), 0, stream, g, x, w, bias, y, relu);
   count_launch();
   return cudaGetLastError();
 }

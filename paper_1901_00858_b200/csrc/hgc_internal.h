@@ -21,6 +21,45 @@ struct ConvGeom {
 
 void count_launch();  // bumps the process-wide kernel launch counter
 
+// Programmatic dependent launch: a kernel launched with this helper may be scheduled while the
+// kernel before it in the stream is still draining; every kernel of this library therefore
+// executes grid_dependency_wait() before its first access to global memory (it returns when the
+// preceding kernel has completed and its writes are visible; a no-op for a kernel launched
+// without the attribute), so only launch latency and on-chip set-up overlap.  Off by default
+// (hgc_set_launch_overlap): it helps eager launches by a few per cent and slows a step replayed
+// as a CUDA graph down.
+bool launch_overlap_enabled();
+void set_launch_overlap(bool on);
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                 Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = launch_overlap_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+#ifdef __CUDACC__
+// see launch_kernel: call before the first global-memory access of a kernel
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel of the stream be scheduled as soon as every CTA of this grid has called
+// this (or exited).  Only the persistent tensor-core kernel calls it: its CTAs hold a whole SM, so
+// the next kernel's CTAs start exactly where one of them has finished.  The many-block copy and
+// depthwise kernels do not: CTAs of a following tensor-core kernel that became resident early
+// would pin most of an SM's registers while they wait and starve the blocks still to run.
+__device__ __forceinline__ void grid_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+#endif
+
 // Each launcher enqueues on `stream` and returns the launch error (cudaSuccess if fine).
 cudaError_t launch_direct_conv(const ConvGeom& g, const __half* x, const __half* w,
                                const __half* bias, __half* y, int relu, cudaStream_t stream);

@@ -565,9 +565,6 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int abort_flag;
 
-  // an earlier CTA gave up: do not start new work on a path that is not progressing
-  if (status != nullptr && *reinterpret_cast<volatile int*>(status) != 0) return;
-
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   // ring of stages; a stage holds one activation tile followed by `taps` weight tiles
@@ -597,7 +594,16 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = tmem_slot;
 
-  if (warp == 0) {
+  // everything above touched only this CTA's shared and tensor memory and may overlap the tail of
+  // the previous kernel in the stream; from here on global memory is read and written
+  grid_dependency_wait();
+  grid_launch_dependents();
+  // an earlier CTA gave up: do not start new work on a path that is not progressing
+  const bool skip = status != nullptr && *reinterpret_cast<volatile int*>(status) != 0;
+
+  if (skip) {
+    // fall through to the release of the tensor memory
+  } else if (warp == 0) {
     // ---------------- TMA producer ----------------
     // The whole warp walks the loop (warp-uniform control flow keeps addresses, coordinates and
     // barrier operands in uniform registers); one elected lane issues the copies.  A stage is
@@ -1231,8 +1237,8 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
     err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV, EWV>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                (int)p.smem_bytes);                                                       \
     if (err == cudaSuccess)                                                                              \
-      igemm_kernel<KBV, HALOV, EWV><<<grid, 64 + 32 * EWV, p.smem_bytes, stream>>>(p.tmA, p.tmB, p.tmY,   \
-                                                                                  p.tmYr, a, bias, y, status); \
+      err = launch_kernel(igemm_kernel<KBV, HALOV, EWV>, grid, dim3(64 + 32 * EWV), p.smem_bytes, stream, p.tmA, \
+                          p.tmB, p.tmY, p.tmYr, a, bias, y, status);                                     \
   } while (0)
 #define HGC_LAUNCH_IGEMM(KBV, HALOV)                                              \
   do {                                                                            \

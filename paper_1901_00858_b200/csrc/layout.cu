@@ -21,6 +21,7 @@ constexpr int kThreads = 256;
 __global__ void __launch_bounds__(kThreads)
 nchw_to_nhwc_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int64_t hw,
                     int c_pad, int vec_ok) {
+  grid_dependency_wait();
   __shared__ __align__(16) uint16_t tile[kTileC][kRow];
   const int64_t n = blockIdx.z;
   const int c0 = blockIdx.y * kTileC;
@@ -73,6 +74,7 @@ template <int CH, int PX>
 __global__ void __launch_bounds__(kThreads)
 nchw_to_nhwc_regs_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int64_t hw,
                          int c_pad, int64_t units_p, int units_c, int64_t total_units) {
+  grid_dependency_wait();
   constexpr int PG = 32 / CH;
   constexpr int W32 = PX / 2;  // 32-bit words per channel
   const int lane = threadIdx.x & 31;
@@ -124,6 +126,7 @@ nchw_to_nhwc_regs_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict_
 __global__ void __launch_bounds__(kThreads)
 nchw_to_nhwc_smallplane_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int hw,
                                int c_pad) {
+  grid_dependency_wait();
   extern __shared__ __align__(16) uint16_t flat[];  // [kTileC][hw]
   const int64_t n = blockIdx.y;
   const int c0 = blockIdx.x * kTileC;
@@ -153,6 +156,7 @@ nchw_to_nhwc_smallplane_kernel(const uint16_t* __restrict__ src, uint16_t* __res
 __global__ void __launch_bounds__(kThreads)
 nhwc_to_nchw_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int64_t hw,
                     int c_pad, int vec_ok) {
+  grid_dependency_wait();
   __shared__ __align__(16) uint16_t tile[kTileC][kRow];
   const int64_t n = blockIdx.z;
   const int c0 = blockIdx.y * kTileC;
@@ -195,6 +199,7 @@ nhwc_to_nchw_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst
 // w[g*kg + k'][c'][r][s] -> w'[g][k'][r][s][c_pad]; one thread per 8 output channels-of-input
 __global__ void weights_repack_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst,
                                       int64_t k, int cg, int rs, int c_pad) {
+  grid_dependency_wait();
   const int64_t vecs_per_k = (int64_t)rs * (c_pad / 8);
   const int64_t total = k * vecs_per_k;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
@@ -220,6 +225,7 @@ __global__ void weights_repack_kernel(const uint16_t* __restrict__ src, uint16_t
 __global__ void __launch_bounds__(256)
 nchw_to_nhwc8_bordered_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int h, int w,
                               int pad_h, int pad_w, int hp, int wp, int64_t total) {
+  grid_dependency_wait();
   const int64_t hw = (int64_t)h * w;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int ow = (int)(i % wp);
@@ -241,6 +247,7 @@ nchw_to_nhwc8_bordered_kernel(const uint16_t* __restrict__ src, uint16_t* __rest
 // w[k][c][r][s] (c <= 8) -> w'[k][r][kw_pix][8]: tap s, channel ch at [s][ch]; zeros elsewhere.
 __global__ void weights_repack_window_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst,
                                              int64_t k, int c, int r, int s, int kw_pix) {
+  grid_dependency_wait();
   const int64_t total = k * r * kw_pix;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int sp = (int)(i % kw_pix);
@@ -267,6 +274,7 @@ __global__ void __launch_bounds__(256)
 patch_im2col_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int h, int w, int p, int q,
                     int pad_h, int pad_w, int stride_h, int stride_w, int dil_h, int dil_w, int kelems,
                     int64_t total) {
+  grid_dependency_wait();
   constexpr int E = R * S * C;
   constexpr int EW = (E + 1) / 2;  // 32-bit words that hold real elements
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -313,6 +321,7 @@ __global__ void __launch_bounds__(256)
 patch_im2col_generic_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int h, int w,
                             int p, int q, int r, int s, int pad_h, int pad_w, int stride_h, int stride_w,
                             int dil_h, int dil_w, int kelems, int64_t total_chunks) {
+  grid_dependency_wait();
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total_chunks) return;
   const int vecs = kelems >> 3;
@@ -345,6 +354,7 @@ patch_im2col_generic_kernel(const uint16_t* __restrict__ src, uint16_t* __restri
 // w[k][c][r][s] -> w'[k][kelems], element (r*S + s)*C + ch; zeros from R*S*C on
 __global__ void weights_repack_patch_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int64_t k,
                                             int c, int r, int s, int kelems) {
+  grid_dependency_wait();
   const int64_t total = k * kelems;
   const int rsc = r * s * c;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
@@ -367,7 +377,7 @@ cudaError_t launch_nchw_to_nhwc8_bordered(const __half* src, __half* dst, int32_
   const int64_t total = (int64_t)n * hp * wp;
   int64_t blocks = (total + 255) / 256;
   if (blocks > 148 * 32) blocks = 148 * 32;
-  nchw_to_nhwc8_bordered_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
+  launch_kernel(nchw_to_nhwc8_bordered_kernel, dim3((unsigned)blocks), dim3(256), 0, stream, 
       reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), c, h, w, pad_h, pad_w, hp, wp, total);
   count_launch();
   return cudaGetLastError();
@@ -378,7 +388,7 @@ cudaError_t launch_weights_repack_window(const __half* src, __half* dst, int32_t
   const int64_t total = (int64_t)k * r * kw_pix;
   int64_t blocks = (total + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
-  weights_repack_window_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
+  launch_kernel(weights_repack_window_kernel, dim3((unsigned)blocks), dim3(256), 0, stream, 
       reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), k, c, r, s, kw_pix);
   count_launch();
   return cudaGetLastError();
@@ -406,13 +416,13 @@ cudaError_t launch_nchw_to_nhwc(const __half* src, __half* dst, int32_t n, int32
     uint16_t* d16 = reinterpret_cast<uint16_t*>(dst);
     const unsigned gb = (unsigned)blocks;
     if (px == 8 && ch_per == 8)
-      nchw_to_nhwc_regs_kernel<8, 8><<<gb, kThreads, 0, stream>>>(s16, d16, c, hw, c_pad, units_p, units_c, total_units);
+      launch_kernel(nchw_to_nhwc_regs_kernel<8, 8>, dim3(gb), dim3(kThreads), 0, stream, s16, d16, c, hw, c_pad, units_p, units_c, total_units);
     else if (px == 8)
-      nchw_to_nhwc_regs_kernel<4, 8><<<gb, kThreads, 0, stream>>>(s16, d16, c, hw, c_pad, units_p, units_c, total_units);
+      launch_kernel(nchw_to_nhwc_regs_kernel<4, 8>, dim3(gb), dim3(kThreads), 0, stream, s16, d16, c, hw, c_pad, units_p, units_c, total_units);
     else if (ch_per == 8)
-      nchw_to_nhwc_regs_kernel<8, 4><<<gb, kThreads, 0, stream>>>(s16, d16, c, hw, c_pad, units_p, units_c, total_units);
+      launch_kernel(nchw_to_nhwc_regs_kernel<8, 4>, dim3(gb), dim3(kThreads), 0, stream, s16, d16, c, hw, c_pad, units_p, units_c, total_units);
     else
-      nchw_to_nhwc_regs_kernel<4, 4><<<gb, kThreads, 0, stream>>>(s16, d16, c, hw, c_pad, units_p, units_c, total_units);
+      launch_kernel(nchw_to_nhwc_regs_kernel<4, 4>, dim3(gb), dim3(kThreads), 0, stream, s16, d16, c, hw, c_pad, units_p, units_c, total_units);
     count_launch();
     return cudaGetLastError();
   }
@@ -423,13 +433,13 @@ cudaError_t launch_nchw_to_nhwc(const __half* src, __half* dst, int32_t n, int32
                                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     dim3 grid2((unsigned)c_tiles, (unsigned)n);
-    nchw_to_nhwc_smallplane_kernel<<<grid2, kThreads, smem, stream>>>(reinterpret_cast<const uint16_t*>(src),
+    launch_kernel(nchw_to_nhwc_smallplane_kernel, dim3(grid2), dim3(kThreads), smem, stream, reinterpret_cast<const uint16_t*>(src),
                                                                       reinterpret_cast<uint16_t*>(dst), c, (int)hw, c_pad);
     count_launch();
     return cudaGetLastError();
   }
   dim3 grid((unsigned)px_tiles, (unsigned)c_tiles, (unsigned)n);
-  nchw_to_nhwc_kernel<<<grid, kThreads, 0, stream>>>(reinterpret_cast<const uint16_t*>(src),
+  launch_kernel(nchw_to_nhwc_kernel, dim3(grid), dim3(kThreads), 0, stream, reinterpret_cast<const uint16_t*>(src),
                                                      reinterpret_cast<uint16_t*>(dst), c, hw, c_pad,
                                                      (hw % 8) == 0);
   count_launch();
@@ -443,7 +453,7 @@ cudaError_t launch_nhwc_to_nchw(const __half* src, __half* dst, int32_t n, int32
   const int c_tiles = (c + kTileC - 1) / kTileC;
   if (px_tiles > 0x7fffffffLL || c_tiles > 65535 || n > 65535) return cudaErrorInvalidConfiguration;
   dim3 grid((unsigned)px_tiles, (unsigned)c_tiles, (unsigned)n);
-  nhwc_to_nchw_kernel<<<grid, kThreads, 0, stream>>>(reinterpret_cast<const uint16_t*>(src),
+  launch_kernel(nhwc_to_nchw_kernel, dim3(grid), dim3(kThreads), 0, stream, reinterpret_cast<const uint16_t*>(src),
                                                      reinterpret_cast<uint16_t*>(dst), c, hw, c_pad,
                                                      (hw % 8) == 0);
   count_launch();
@@ -457,7 +467,7 @@ cudaError_t launch_weights_repack(const __half* src, __half* dst, int32_t k, int
   int64_t blocks = (total + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
   if (blocks < 1) blocks = 1;
-  weights_repack_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
+  launch_kernel(weights_repack_kernel, dim3((unsigned)blocks), dim3(256), 0, stream, 
       reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), k, cg, r * s, c_pad);
   count_launch();
   return cudaGetLastError();
@@ -472,7 +482,7 @@ cudaError_t launch_patch_im2col(const ConvGeom& g, const __half* src, __half* ds
     const int64_t blocks = (pixels + 255) / 256;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
 #define HGC_PATCH(CV)                                                                                         \
-  patch_im2col_kernel<3, 3, CV><<<(unsigned)blocks, 256, 0, stream>>>(s16, d16, g.h, g.w, g.p, g.q, g.pad_h, \
+  launch_kernel(patch_im2col_kernel<3, 3, CV>, dim3((unsigned)blocks), dim3(256), 0, stream, s16, d16, g.h, g.w, g.p, g.q, g.pad_h, \
                                                                       g.pad_w, g.stride_h, g.stride_w, g.dil_h, \
                                                                       g.dil_w, kelems, pixels)
     if (g.c == 3) HGC_PATCH(3);
@@ -483,7 +493,7 @@ cudaError_t launch_patch_im2col(const ConvGeom& g, const __half* src, __half* ds
     const int64_t chunks = pixels * (kelems / 8);
     const int64_t blocks = (chunks + 255) / 256;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    patch_im2col_generic_kernel<<<(unsigned)blocks, 256, 0, stream>>>(s16, d16, g.c, g.h, g.w, g.p, g.q, g.r, g.s,
+    launch_kernel(patch_im2col_generic_kernel, dim3((unsigned)blocks), dim3(256), 0, stream, s16, d16, g.c, g.h, g.w, g.p, g.q, g.r, g.s,
                                                                       g.pad_h, g.pad_w, g.stride_h, g.stride_w,
                                                                       g.dil_h, g.dil_w, kelems, chunks);
   }
@@ -497,7 +507,7 @@ cudaError_t launch_weights_repack_patch(const __half* src, __half* dst, int32_t 
   int64_t blocks = (total + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
   if (blocks < 1) blocks = 1;
-  weights_repack_patch_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
+  launch_kernel(weights_repack_patch_kernel, dim3((unsigned)blocks), dim3(256), 0, stream, 
       reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), k, c, r, s, kelems);
   count_launch();
   return cudaGetLastError();

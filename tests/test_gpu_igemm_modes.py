@@ -88,3 +88,37 @@ def test_same_descriptor_new_tensors(hgc, oracle):
         torch.cuda.synchronize()
         check_close(to_host(y), oracle.conv_fast(P, x, w, b, True), what=f"rep {rep}")
     d.close()
+
+
+def test_launch_overlap_gives_the_same_results(hgc, oracle):
+    """With programmatic dependent launch on, a chain of dependent kernels (layout pass ->
+    tensor-core kernel, twice on the same descriptor and workspace, then a depthwise layer) must
+    still see every predecessor's writes."""
+    import torch
+    from gpu_util import to_dev, to_host
+    a = params_dict(2, 96, 20, 20, 72, 3, 3, 1, 1)
+    rng = np.random.default_rng(77)
+    P = oracle.ConvParams(**a)
+    d = hgc.ConvDesc(**a)
+    d.ensure_workspace()
+    dw_a = params_dict(2, 72, 20, 20, 72, 3, 3, 1, 1, 1, 1, 1, 1, 72)
+    dw = hgc.ConvDesc(**dw_a)
+    hgc.set_launch_overlap(True)
+    try:
+        for rep in range(3):
+            x, w, b = workloads.random_layer_tensors(rng, 2, 96, 20, 20, 72, 3, 3, 1)
+            _, w2, b2 = workloads.random_layer_tensors(rng, 2, 72, 20, 20, 72, 3, 3, 72)
+            xd, wd, bd, w2d, b2d = to_dev(x), to_dev(w), to_dev(b), to_dev(w2), to_dev(b2)
+            y = torch.full((2, 72, 20, 20), float("nan"), dtype=torch.float16, device="cuda")
+            z = torch.full((2, 72, 20, 20), float("nan"), dtype=torch.float16, device="cuda")
+            hgc.conv_forward(d, xd, wd, bd, y, True)
+            hgc.conv_forward(dw, y, w2d, b2d, z, False)     # reads what the kernel before wrote
+            torch.cuda.synchronize()
+            ref_y = oracle.conv_fast(P, x, w, b, True)
+            check_close(to_host(y), ref_y, what=f"overlap rep {rep} conv")
+            ref_z = oracle.conv_fast(oracle.ConvParams(**dw_a), to_host(y), w2, b2, False)
+            check_close(to_host(z), ref_z, what=f"overlap rep {rep} depthwise")
+    finally:
+        hgc.set_launch_overlap(False)
+    d.close()
+    dw.close()
