@@ -4,19 +4,27 @@
 //   M (TMEM lanes)   = 128 output channels of the group
 //   N (TMEM columns) = a tile of output pixels: tn images x th rows x the full output width
 //   K (reduction)    = taps (r,s) x channel blocks of kb = 64 / 32 / 16 channels
-// Both operands are K-major in shared memory (channels innermost):
-//   A = re-laid-out weights  w'[g][K/g][R][S][cw]        (TMA, 3-D map, box kb x 128 x 1)
-//   B = NHWC copy of the input x'[N][H][W][c_pad]        (TMA, 5-D map (c, g, w, h, n),
-//       box kb x 1 x tw*stride x th*stride x tn with element strides = conv stride; the
-//       start coordinate (q0*stride - pad + s*dil, p0*stride - pad + r*dil) may lie outside the
-//       image: TMA zero-fills, which IS the zero padding)
-// TMA writes the 128/64/32-byte swizzled layout the UMMA shared-memory descriptors name.
+// Operands in shared memory (written by TMA in the 128/64/32-byte swizzled layouts that the UMMA
+// shared-memory descriptors name):
+//   A = re-laid-out weights  w'[g][K/g][R][S][cw], K-major   (3-D map, box kb x 128 (or 64) x 1)
+//   B = activations, one of
+//       - the NHWC copy x'[N][H][W][c_pad], K-major (5-D map (c, g, w, h, n), box kb x 1 x
+//         tw*stride x th*stride x tn with element strides = conv stride; the start coordinate
+//         (q0*stride - pad + s*dil, p0*stride - pad + r*dil) may lie outside the image: TMA
+//         zero-fills, which IS the zero padding).  At stride 1 the S taps of a kernel row share one
+//         tile: tap s starts s*dil pixel rows further in (a descriptor start offset);
+//       - x itself for 1x1 layers (3-D map (pixel, channel, image), boxes of 64 pixels x kb
+//         channels): pixel-major ("MN-major") tiles, no copy of x at all;
+//       - for few-channel stems, overlapping windows of a zero-bordered 8-channel copy, or an
+//         expanded copy holding the values under the kernel per output pixel.
 //
-// One CTA computes one 128 x N tile:  warp 0 = TMA producer, warp 1 = TMEM allocator and MMA
-// issuer (one elected lane issues tcgen05.mma; tcgen05.commit releases smem stages through
-// mbarriers), warps 2..5 = epilogue: tcgen05.ld of the fp32 accumulators (lane = output
-// channel, so a thread owns a run of consecutive pixels of one NCHW channel plane), + bias,
-// ReLU, cvt.rn.f16, 16-byte stores straight into y (no NHWC->NCHW pass for the output).
+// One persistent CTA per SM walks its tiles:  warp 0 = TMA producer (a ring stage = one
+// activation tile + the weight tiles of its taps, one mbarrier), warp 1 = TMEM allocator and MMA
+// issuer (one elected lane issues tcgen05.mma; tcgen05.commit releases ring stages and hands
+// accumulators over through mbarriers; two 256-column accumulators alternate), warps 2.. =
+// epilogue, two (or four) per TMEM lane quarter: tcgen05.ld of the fp32 accumulators (lane =
+// output channel), + bias, ReLU, cvt.rn.f16x2, staged as fp16 in shared memory and written to
+// NCHW y either by TMA stores or by coalesced plain stores (no NHWC->NCHW pass for the output).
 //
 // Every wait on an mbarrier is bounded by wall-clock time; on expiry the CTA raises a status
 // word, lets its outstanding copies land, frees its TMEM and returns.
