@@ -475,6 +475,30 @@ __device__ __noinline__ void epilogue_copy(uint32_t t_addr, uint32_t sbuf, int f
   __syncwarp();
 }
 
+// Epilogue of the inner-product layer (1x1 output plane: a column is an image).  y[n][k] has the
+// channels of one image contiguous, so the lanes (channels) of a warp write 64 contiguous bytes
+// per column straight from registers.
+__device__ __noinline__ void epilogue_columns(uint32_t t_addr, int first_unit, int unit_step, int nimg, int K, int n0,
+                                              int k0, int kvalid_rows, float bv, bool relu, uint16_t* yb) {
+  const int lane = threadIdx.x & 31;
+  for (int c0 = first_unit * 32; c0 < nimg; c0 += unit_step * 32) {
+    uint32_t v[32];
+    tmem_ld32(t_addr + (uint32_t)c0, v);  // columns past the tile's last image are read and dropped
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+    if (lane < kvalid_rows) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        if (c0 + j < nimg) {
+          float f = __uint_as_float(v[j]) + bv;
+          if (relu) f = fmaxf(f, 0.f);
+          yb[(int64_t)(n0 + c0 + j) * K + k0 + lane] = __half_as_ushort(__float2half_rn(f));
+        }
+      }
+    }
+  }
+  __syncwarp();
+}
+
 struct IgemmArgs {
   int32_t N, K, P, Q;
   int32_t kg, group;
@@ -845,7 +869,12 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           // the warps of a lane quarter take alternate units (the wide variant is only launched
           // for layers that take the TMA-store epilogue: it must fit 96 registers per thread)
           if constexpr (EW == kEpilogueWarps) {
-            if (quarter_live) {
+            if (quarter_live && a.P * a.Q == 1) {
+              const int kleft = a.kg - (m0 + quarter * 32);
+              const int nimg = a.N - n0 < a.tn ? a.N - n0 : a.tn;
+              epilogue_columns(t_addr, half, kPerQuarter, nimg, a.K, n0, grp * a.kg + m0 + quarter * 32,
+                               kleft < 32 ? kleft : 32, bv, relu, yb);
+            } else if (quarter_live) {
               const int kleft = a.kg - (m0 + quarter * 32);
               epilogue_copy(t_addr, my_stage, half, kPerQuarter, a.tn, a.th, a.pitch, a.N, a.K, a.P, a.Q, n0, p0,
                             grp * a.kg + m0 + quarter * 32, kleft < 32 ? kleft : 32, bv, relu, yb);
