@@ -586,7 +586,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 
 // Persistent kernel: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...; the two TMEM
 // accumulators alternate so that the epilogue of one tile overlaps the MMAs of the next.
-template <int KB, bool HALO, int EW>
+template <int KB, bool HALO, int EW, bool COPY>
 __global__ void __launch_bounds__(64 + 32 * EW, 1)
 igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
              const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmYr,
@@ -787,7 +787,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       const uint32_t t_addr = tmem_base + buf * 256u + ((uint32_t)(quarter * 32) << 16);
       const bool quarter_live = m0 + quarter * 32 < a.kg;  // any real output channel in this warp's lanes?
 
-      if (a.tma_store) {
+      if constexpr (!COPY) {
         // ---- staged epilogue: TMEM -> registers -> swizzled fp16 tile in smem -> TMA store ----
         // (taken when Q % 8 == 0, hence P*Q % 8 == 0, and a tile holds one image: every staged run
         //  of pixels then starts on a 16-byte boundary of y).  A unit of work is 32 channels (this
@@ -866,9 +866,8 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       } else {
         // ---- direct epilogue: each thread stores runs of its own channel plane ----
         {
-          // the warps of a lane quarter take alternate units (the wide variant is only launched
-          // for layers that take the TMA-store epilogue: it must fit 96 registers per thread)
-          if constexpr (EW == kEpilogueWarps) {
+          // the warps of a lane quarter take alternate units
+          {
             if (quarter_live && a.P * a.Q == 1) {
               const int kleft = a.kg - (m0 + quarter * 32);
               const int nimg = a.N - n0 < a.tn ? a.N - n0 : a.tn;
@@ -1269,18 +1268,22 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
   dim3 grid((unsigned)(p.total_tiles < sms ? p.total_tiles : sms));
   int* status = reinterpret_cast<int*>(static_cast<char*>(ws) + p.ws_status_off);
   cudaError_t err = cudaSuccess;
-#define HGC_LAUNCH_IGEMM_EW(KBV, HALOV, EWV)                                                             \
-  do {                                                                                                   \
-    err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV, EWV>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                               (int)p.smem_bytes);                                                       \
-    if (err == cudaSuccess)                                                                              \
-      err = launch_kernel(igemm_kernel<KBV, HALOV, EWV>, grid, dim3(64 + 32 * EWV), p.smem_bytes, stream, p.tmA, \
-                          p.tmB, p.tmY, p.tmYr, a, bias, y, status);                                     \
+  // three instantiations per (kb, halo): TMA-store epilogue with 8 or 16 epilogue warps, copy
+  // epilogue with 8 (each kernel carries only the epilogue it runs: the hot loops are sensitive to
+  // the size of the code around them)
+#define HGC_LAUNCH_IGEMM_EW(KBV, HALOV, EWV, COPYV)                                                         \
+  do {                                                                                                     \
+    err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV, EWV, COPYV>,                                        \
+                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);            \
+    if (err == cudaSuccess)                                                                                \
+      err = launch_kernel(igemm_kernel<KBV, HALOV, EWV, COPYV>, grid, dim3(64 + 32 * EWV), p.smem_bytes,    \
+                          stream, p.tmA, p.tmB, p.tmY, p.tmYr, a, bias, y, status);                        \
   } while (0)
-#define HGC_LAUNCH_IGEMM(KBV, HALOV)                                              \
-  do {                                                                            \
-    if (p.epi_warps == kEpilogueWarpsWide) HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 16);   \
-    else HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 8);                                      \
+#define HGC_LAUNCH_IGEMM(KBV, HALOV)                                                       \
+  do {                                                                                     \
+    if (!p.tma_store) HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 8, true);                            \
+    else if (p.epi_warps == kEpilogueWarpsWide) HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 16, false); \
+    else HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 8, false);                                        \
   } while (0)
   if (p.kb == 64) {
     if (p.halo) HGC_LAUNCH_IGEMM(64, true); else HGC_LAUNCH_IGEMM(64, false);
