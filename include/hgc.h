@@ -152,8 +152,10 @@ int hgc_conv_path(const hgc_conv_desc* d, int32_t* path);
  * tiles come from: 0 = an NHWC copy of x made by the layout pass, 1 = x itself, read as
  * pixel-major tiles (1x1 layers), 2 = a zero-bordered 8-channel NHWC copy read through
  * overlapping windows (few input channels), 3 = an expanded copy holding, per output pixel, the
- * values under the kernel (few input channels, strided); zeros for the other paths.
- * info: host pointer.
+ * values under the kernel (few input channels, strided), [11] the number of CTAs that share
+ * the reduction of one tile (1, or 2 / 4 / 8 for layers with very few tiles, e.g. inner products:
+ * each CTA writes fp32 partial sums and a second kernel adds them in a fixed order); zeros for
+ * the other paths.  info: host pointer.
  */
 int hgc_conv_plan_info(const hgc_conv_desc* d, int32_t* info, int32_t count);
 

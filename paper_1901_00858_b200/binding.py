@@ -159,9 +159,10 @@ class ConvDesc:
         return v.value
 
     def plan_info(self) -> dict:
-        v = (ctypes.c_int32 * 11)()
-        _check(lib().hgc_conv_plan_info(self._h, v, 11), "hgc_conv_plan_info")
-        keys = ("path", "kb", "halo", "tn", "th", "pitch", "ncols", "tiles", "stages", "taps", "x_source")
+        v = (ctypes.c_int32 * 12)()
+        _check(lib().hgc_conv_plan_info(self._h, v, 12), "hgc_conv_plan_info")
+        keys = ("path", "kb", "halo", "tn", "th", "pitch", "ncols", "tiles", "stages", "taps", "x_source",
+                "k_slices")
         return dict(zip(keys, list(v)))
 
     def workspace_bytes(self) -> int:

@@ -199,14 +199,15 @@ int hgc_conv_path(const hgc_conv_desc* d, int32_t* path) {
 
 int hgc_conv_plan_info(const hgc_conv_desc* d, int32_t* info, int32_t count) {
   if (d == nullptr || info == nullptr || count < 1) return HGC_INVALID_ARG;
-  int32_t v[11] = {d->path, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+  int32_t v[12] = {d->path, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
   if (d->path == HGC_PATH_IGEMM) {
     const hgc::IgemmPlan& p = d->igemm;
     v[1] = p.kb; v[2] = p.halo; v[3] = p.tn; v[4] = p.th; v[5] = p.pitch; v[6] = p.ncols;
     v[7] = p.total_tiles; v[8] = p.stages; v[9] = p.taps;
     v[10] = p.nchw ? 1 : (p.window ? 2 : (p.patch ? 3 : 0));
+    v[11] = 1 << p.ks_log2;
   }
-  for (int i = 0; i < count && i < 11; ++i) info[i] = v[i];
+  for (int i = 0; i < count && i < 12; ++i) info[i] = v[i];
   return HGC_OK;
 }
 

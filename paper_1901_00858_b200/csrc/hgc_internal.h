@@ -101,7 +101,8 @@ struct IgemmPlan {
   uint32_t a_bytes, b_bytes, b_alloc;
   int32_t a_rows;  // rows of a weight tile in shared memory (128, or 64 for layers of <= 64 channels per group)
   size_t smem_bytes;
-  size_t ws_status_off, ws_w_off, ws_x_off, ws_total;
+  int32_t ks_log2;  // log2 of the number of reduction slices a tile is split into (0 = none)
+  size_t ws_status_off, ws_w_off, ws_x_off, ws_part_off, ws_total;
   bool maps_ready;
   alignas(64) CUtensorMap tmA;
   alignas(64) CUtensorMap tmB;

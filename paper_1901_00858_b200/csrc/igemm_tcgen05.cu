@@ -499,6 +499,96 @@ __device__ __noinline__ void epilogue_columns(uint32_t t_addr, int first_unit, i
   __syncwarp();
 }
 
+// Epilogue of a reduction slice: the fp32 accumulators go, unrounded, to this slice's copy of
+// the output (same [n][k][p][q] order as y).  Same two-phase scheme as epilogue_copy with 4-byte
+// elements: a unit is 32 channels x 32 columns; lane = channel stages its row of 32 floats
+// (128 bytes, swizzled), then lane = column walks the 32 rows, so a store instruction writes 32
+// consecutive floats of one channel plane.  On a 1x1 plane (inner product) a column is an image
+// and the lanes' channels are contiguous: straight from registers.
+__device__ __noinline__ void epilogue_partial(uint32_t t_addr, uint32_t sbuf, int first_unit, int unit_step, int tn,
+                                              int th, int pitch, int N, int K, int P, int Q, int n0, int p0, int k0,
+                                              int kvalid_rows, float* part) {
+  const int lane = threadIdx.x & 31;
+  const int64_t pq = (int64_t)P * Q;
+  if (pq == 1) {
+    const int nimg = N - n0 < tn ? N - n0 : tn;
+    for (int c0 = first_unit * 32; c0 < nimg; c0 += unit_step * 32) {
+      uint32_t v[32];
+      tmem_ld32(t_addr + (uint32_t)c0, v);  // columns past the tile's last image are read and dropped
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      if (lane < kvalid_rows) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (c0 + j < nimg) part[(int64_t)(n0 + c0 + j) * K + k0 + lane] = __uint_as_float(v[j]);
+      }
+    }
+    __syncwarp();
+    return;
+  }
+  const int rows_valid = (P - p0) < th ? (P - p0) : th;
+  const int cols_need = (rows_valid - 1) * pitch + Q;
+  const int img_cols = th * pitch;
+  const uint32_t row_off = (uint32_t)lane * 128u;
+  int unit = 0;
+  for (int img = 0; img < tn; ++img) {
+    if (n0 + img >= N) break;
+    float* pimg = part + ((int64_t)(n0 + img) * K + k0) * pq;
+    for (int c0 = 0; c0 < cols_need; c0 += 32, ++unit) {
+      if (unit % unit_step != first_unit) continue;
+      const int ncol = cols_need - c0 < 32 ? cols_need - c0 : 32;
+      const uint32_t tcol = t_addr + (uint32_t)(img * img_cols + c0);
+      __syncwarp();  // the previous unit has been copied out
+      uint32_t v[32];
+      if (ncol == 32) {
+        tmem_ld32(tcol, v);
+      } else {
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          if (c * 8 < ncol) tmem_ld8(tcol + (uint32_t)(c * 8), &v[8 * c]);
+      }
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        if (c * 4 < ncol) {
+          const uint32_t dst = sbuf + row_off + ((uint32_t)(c ^ (lane & 7)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v[4 * c]), "r"(v[4 * c + 1]),
+                       "r"(v[4 * c + 2]), "r"(v[4 * c + 3])
+                       : "memory");
+        }
+      }
+      __syncwarp();
+      const int cabs = c0 + lane;
+      const int hr = cabs / pitch;
+      const int wc = cabs - hr * pitch;
+      if (lane < ncol && wc < Q) {
+        float* dst = pimg + (int64_t)(p0 + hr) * Q + wc;
+        const uint32_t chunk = (uint32_t)lane >> 2, within = ((uint32_t)lane & 3u) * 4u;
+#pragma unroll 4
+        for (int r = 0; r < kvalid_rows; ++r) {
+          uint32_t w;
+          asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w) : "r"(sbuf + (uint32_t)r * 128u + ((chunk ^ ((uint32_t)r & 7u)) << 4) + within));
+          dst[(int64_t)r * pq] = __uint_as_float(w);
+        }
+      }
+    }
+  }
+  __syncwarp();
+}
+
+// y = round( relu?( bias[k] + partial[0] + partial[1] + ... ) ): the slices are added in a fixed
+// order, so the result does not depend on which CTA finished first
+__global__ void __launch_bounds__(256)
+splitk_finish_kernel(const float* __restrict__ part, int slices, int64_t stride, const __half* __restrict__ bias,
+                     uint16_t* __restrict__ y, int K, int64_t pq, int64_t total, int relu) {
+  grid_dependency_wait();
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    float acc = bias != nullptr ? __half2float(__ldg(bias + (int)((i / pq) % K))) : 0.f;
+    for (int sidx = 0; sidx < slices; ++sidx) acc += __ldcs(part + sidx * stride + i);
+    if (relu) acc = fmaxf(acc, 0.f);
+    y[i] = __half_as_ushort(__float2half_rn(acc));
+  }
+}
+
 struct IgemmArgs {
   int32_t N, K, P, Q;
   int32_t kg, group;
@@ -529,16 +619,24 @@ struct IgemmArgs {
   int32_t tma_store;  // 1: the epilogue stages fp16 tiles in shared memory and stores them with TMA
   int32_t rem;        // (th*Q) % 64: width of the last staged pass of a full tile (0 = none)
   int32_t nbuf;       // staging tiles per epilogue warp (1 or 2)
+  // split reduction (its own kernel instantiation): the channel blocks of a tile are dealt out to
+  // 2^ks_log2 CTAs, each of which writes its fp32 partial sums to its own slice of `partials`; a
+  // second kernel adds the slices in a fixed order (+ bias, ReLU, rounding)
+  int32_t ks_log2;
+  int64_t part_stride;  // elements between two slices: N * K * P * Q
 };
 
 // The tiles of one CTA: blockIdx.x, blockIdx.x + gridDim.x, ...  Tile t = (pixel tile px, channel
 // tile mg) with mg fastest, px = (image tile, row tile).  The decomposition is kept up to date
 // by additions (a handful of divisions once per kernel instead of five per tile and role).
+template <bool SPLIT>
 struct TileIter {
   int tile, mg, pt, ph;  // current tile, its channel tile, image tile and row tile
   int stride, d_mg, d_pt, d_ph;
+  // with a split reduction the slices of a tile are the fastest index
+  __device__ __forceinline__ int ks(const IgemmArgs& a) const { return SPLIT ? a.ks_log2 : 0; }
   __device__ __forceinline__ void init(const IgemmArgs& a) {
-    const int mgn = a.mtiles * a.group;
+    const int mgn = (a.mtiles * a.group) << ks(a);
     tile = blockIdx.x;
     const int px = tile / mgn;
     mg = tile - px * mgn;
@@ -550,9 +648,9 @@ struct TileIter {
     d_pt = d_px / a.tiles_h;
     d_ph = d_px - d_pt * a.tiles_h;
   }
-  __device__ __forceinline__ bool valid(const IgemmArgs& a) const { return tile < a.total_tiles; }
+  __device__ __forceinline__ bool valid(const IgemmArgs& a) const { return tile < (a.total_tiles << ks(a)); }
   __device__ __forceinline__ void next(const IgemmArgs& a) {
-    const int mgn = a.mtiles * a.group;
+    const int mgn = (a.mtiles * a.group) << ks(a);
     tile += stride;
     mg += d_mg;
     ph += d_ph;
@@ -568,12 +666,25 @@ struct TileIter {
   }
   // group and first output channel (within the group) of the channel tile
   __device__ __forceinline__ void channel_tile(const IgemmArgs& a, int& grp, int& m0) const {
+    const int mgc = mg >> ks(a);
     if (a.group == 1) {
       grp = 0;
-      m0 = mg * 128;
+      m0 = mgc * 128;
     } else {
-      grp = mg / a.mtiles;
-      m0 = (mg - grp * a.mtiles) * 128;
+      grp = mgc / a.mtiles;
+      m0 = (mgc - grp * a.mtiles) * 128;
+    }
+  }
+  // reduction slice of this unit and its range of channel blocks
+  __device__ __forceinline__ int slice(const IgemmArgs& a) const { return SPLIT ? (mg & ((1 << a.ks_log2) - 1)) : 0; }
+  __device__ __forceinline__ void block_range(const IgemmArgs& a, int& cb0, int& cb1) const {
+    if (SPLIT) {
+      const int sl = slice(a);
+      cb0 = (sl * a.cblocks) >> a.ks_log2;
+      cb1 = ((sl + 1) * a.cblocks) >> a.ks_log2;
+    } else {
+      cb0 = 0;
+      cb1 = a.cblocks;
     }
   }
 };
@@ -586,11 +697,12 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 
 // Persistent kernel: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...; the two TMEM
 // accumulators alternate so that the epilogue of one tile overlaps the MMAs of the next.
-template <int KB, bool HALO, int EW, bool COPY>
+template <int KB, bool HALO, int EW, bool COPY, bool SPLIT>
 __global__ void __launch_bounds__(64 + 32 * EW, 1)
 igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
              const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmYr,
-             const IgemmArgs a, const __half* __restrict__ bias, __half* __restrict__ y, int* status) {
+             const IgemmArgs a, const __half* __restrict__ bias, __half* __restrict__ y, float* __restrict__ partials,
+             int* status) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages];
   __shared__ __align__(8) uint64_t acc_full[2], acc_empty[2];
@@ -647,14 +759,16 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     bool ok = true;
     const uint32_t depth = (uint32_t)a.stages;
     const int groups_per_row = a.S / a.taps;  // 1 in halo mode (taps == S), S otherwise (taps == 1)
-    TileIter it;
+    TileIter<SPLIT> it;
     for (it.init(a); it.valid(a) && ok; it.next(a)) {
       int grp, m0;
       it.channel_tile(a, grp, m0);
       const int n0 = it.pt * a.tn;
       const int p0 = it.ph * a.th;
       const int h_base = p0 * a.stride_h - a.pad_h;
-      for (int cb = 0; cb < a.cblocks && ok; ++cb) {
+      int cb0, cb1;
+      it.block_range(a, cb0, cb1);
+      for (int cb = cb0; cb < cb1 && ok; ++cb) {
         int acol = cb * KB;  // column of w' for tap (r, s): (r*S + s)*cw + cb*KB
         for (int r = 0; r < a.R && ok; ++r) {
           for (int sg = 0; sg < groups_per_row; ++sg) {
@@ -713,9 +827,14 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const uint32_t idesc = a.idesc;
     const uint32_t do_mma = 1u;
     const int groups_per_row = a.S / a.taps;
-    const int groups_per_tile = a.cblocks * a.R * groups_per_row;
     uint32_t ready = mbar_test_wait(smem_u32(&full_bar[0]), 0u);
-    for (int tile = blockIdx.x; tile < a.total_tiles && ok; tile += gridDim.x, ++lt) {  // only the count matters here
+    const int units = SPLIT ? (a.total_tiles << a.ks_log2) : a.total_tiles;
+    for (int unit = blockIdx.x; unit < units && ok; unit += gridDim.x, ++lt) {  // only count and slice matter here
+      int groups_per_tile = a.cblocks * a.R * groups_per_row;
+      if constexpr (SPLIT) {  // the slice is the fastest index of a unit
+        const int sl = unit & ((1 << a.ks_log2) - 1);
+        groups_per_tile = ((((sl + 1) * a.cblocks) >> a.ks_log2) - ((sl * a.cblocks) >> a.ks_log2)) * a.R * groups_per_row;
+      }
       const uint32_t buf = lt & 1u;
       // the epilogue must have drained this accumulator (two tiles ago)
       if (!mbar_wait(smem_u32(&acc_empty[buf]), ((lt >> 1) & 1u) ^ 1u, &abort_flag, 64)) {
@@ -771,7 +890,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const uint32_t row_off = (uint32_t)lane * 128u + (((uint32_t)lane & 7u) << 4);
     uint32_t unit_ctr = 0, stage_sel = 0;
     uint32_t lt = 0;
-    TileIter it;
+    TileIter<SPLIT> it;
     for (it.init(a); it.valid(a); it.next(a), ++lt) {
       int grp, m0;
       it.channel_tile(a, grp, m0);
@@ -867,7 +986,14 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         // ---- direct epilogue: each thread stores runs of its own channel plane ----
         {
           // the warps of a lane quarter take alternate units
-          {
+          if constexpr (SPLIT) {
+            if (quarter_live) {
+              const int kleft = a.kg - (m0 + quarter * 32);
+              epilogue_partial(t_addr, my_stage, half, kPerQuarter, a.tn, a.th, a.pitch, a.N, a.K, a.P, a.Q, n0, p0,
+                               grp * a.kg + m0 + quarter * 32, kleft < 32 ? kleft : 32,
+                               partials + (int64_t)it.slice(a) * a.part_stride);
+            }
+          } else {
             if (quarter_live && a.P * a.Q == 1) {
               const int kleft = a.kg - (m0 + quarter * 32);
               const int nimg = a.N - n0 < a.tn ? a.N - n0 : a.tn;
@@ -1013,7 +1139,9 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   const double mps = (double)taps_est * (p.kb / 16.0);                       // MMAs per stage
   const double mpt = (double)p.cblocks * p.eff_r * p.eff_s * (p.kb / 16.0);  // MMAs per tile
   const double a_bytes_mma = 32.0 * (g.kg < 128 ? g.kg : 128);
-  auto tile_clk = [&](int64_t brow, int64_t cols) {
+  // ks: log2 of the number of CTAs that share the reduction of a tile (each then writes fp32
+  // partial sums, added by a second kernel): main loop / 2^ks, an epilogue of twice the bytes
+  auto tile_clk = [&](int64_t brow, int64_t cols, int ks) {
     const double ncols = (double)((cols + 15) / 16 * 16);
     const double brows = p.nchw ? (double)((cols + 63) / 64 * 64) : (double)brow;
     const double t_l2 = (a_bytes_mma + brows * p.kb * 2.0 / mps) / 30.0;
@@ -1021,12 +1149,20 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
     const double t_issue = 45.0 + 400.0 / mps;
     double t = t_tensor > t_l2 ? t_tensor : t_l2;
     if (t_issue > t) t = t_issue;
-    const double main_loop = mpt * t;
-    const double epilogue = 600.0 + 10.0 * ncols;
+    const double main_loop = mpt / (double)(1 << ks) * t;
+    const double epilogue = (600.0 + 10.0 * ncols) * (ks > 0 ? 2.0 : 1.0);
     return (main_loop > epilogue ? main_loop : epilogue) + 300.0;
   };
+  // the second kernel of a split reduction: a launch plus reading the slices and writing y
+  auto finish_clk = [&](int ks) {
+    if (ks == 0) return 0.0;
+    const double elems = (double)g.n * g.k * g.p * g.q;
+    return 8000.0 + elems * (4.0 * (1 << ks) + 2.0) / 3000.0;
+  };
+  // the split kernel exists for 64-channel stages of stride-1 layers without the direct-x mode
+  const bool can_split = p.kb == 64 && p.halo && !p.nchw;
   double best = 1e300;
-  int best_th = 0, best_tn = 0;
+  int best_th = 0, best_tn = 0, best_ks = 0;
   for (int th = 1; th <= g.p; ++th) {
     if ((int64_t)th * p.pitch - junk > 256 || (int64_t)th * (p.patch ? 1 : g.stride_h) > 256) break;
     if (p.nchw && th != g.p && ((int64_t)th * g.q) % 8 != 0) continue;  // tiles must start on 16-byte boundaries of x
@@ -1037,12 +1173,22 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
       // 8-column accumulator read that starts in the tile must end inside the 256-column buffer
       if (cols > (tn > 1 ? 248 : 256) || tn > 256) break;
       const int64_t tiles = (int64_t)((g.n + tn - 1) / tn) * ((g.p + th - 1) / th) * mg;
-      const int64_t waves = (tiles + sms - 1) / sms;
-      const double cost = (double)waves * tile_clk((int64_t)tn * th * p.pitch, cols) + 1e-3 * (double)tiles;
-      if (cost < best - 1e-9 || (cost < best + 1e-9 && (int64_t)tn * th > (int64_t)best_tn * best_th)) {
-        best = cost;
-        best_th = th;
-        best_tn = tn;
+      for (int ks = 0; ks <= 3; ++ks) {
+        // a slice keeps at least two channel blocks and a main loop of 24 MMAs; only layers whose
+        // tiles leave three quarters of the SMs idle are split (inner products, tiny planes): on
+        // a 14x14 layer of 128 tiles the second pass costs what the split gains (measured)
+        if (ks > 0 && (!can_split || (p.cblocks >> ks) < 2 || mpt / (1 << ks) < 24.0 || 4 * tiles > sms)) break;
+        const int64_t units = tiles << ks;
+        const int64_t waves = (units + sms - 1) / sms;
+        const double cost = (double)waves * tile_clk((int64_t)tn * th * p.pitch, cols, ks) + finish_clk(ks) +
+                            1e-3 * (double)units;
+        if (cost < best - 1e-9 ||
+            (cost < best + 1e-9 && ks == best_ks && (int64_t)tn * th > (int64_t)best_tn * best_th)) {
+          best = cost;
+          best_th = th;
+          best_tn = tn;
+          best_ks = ks;
+        }
       }
     }
   }
@@ -1079,6 +1225,12 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   p.epi_warps = kEpilogueWarps;
   if (p.tma_store && mpt * 130.0 < 600.0 + 10.0 * p.ncols && (p.th * g.q) > 2 * kPassElems)
     p.epi_warps = kEpilogueWarpsWide;
+  // split reduction (chosen with the tile shape above): fp32 partials, copy-style epilogue
+  p.ks_log2 = best_ks;
+  if (p.ks_log2 > 0) {
+    p.epi_warps = kEpilogueWarps;
+    p.tma_store = 0;
+  }
   const size_t stage_buf_bytes = (size_t)p.epi_warps * kWarpStageBytes;
   // rings: B two or three deep, A with what is left (each A stage feeds kb/16 MMAs).  227 KB per
   // CTA minus alignment slack, static barriers and the two epilogue staging buffers.
@@ -1118,10 +1270,15 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   p.ws_status_off = 0;
   p.ws_w_off = 256;
   p.ws_x_off = p.ws_w_off + round_up_sz((size_t)g.k * p.eff_r * p.eff_s * p.cw * 2, 256);
+  p.ws_part_off = 0;
   p.ws_total = p.ws_x_off + (p.nchw ? 0
                                     : round_up_sz(p.patch    ? (size_t)g.n * g.p * g.q * p.cw * 2
                                                   : p.window ? (size_t)g.n * p.hp * p.wp * 16 + 256
                                                            : (size_t)g.n * g.h * g.w * p.c_pad * 2, 256));
+  if (p.ks_log2 > 0) {
+    p.ws_part_off = p.ws_total;
+    p.ws_total += round_up_sz(((size_t)g.n * g.k * g.p * g.q * 4) << p.ks_log2, 256);
+  }
   *out = p;
   return true;
 }
@@ -1264,27 +1421,34 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
   a.tma_store = p.tma_store;
   a.rem = p.rem;
   a.nbuf = p.nbuf;
+  a.ks_log2 = p.ks_log2;
+  a.part_stride = (int64_t)g.n * g.k * g.p * g.q;
+  float* partials = p.ks_log2 > 0 ? reinterpret_cast<float*>(static_cast<char*>(ws) + p.ws_part_off) : nullptr;
   const int sms = sm_count();
-  dim3 grid((unsigned)(p.total_tiles < sms ? p.total_tiles : sms));
+  const int64_t units = (int64_t)p.total_tiles << p.ks_log2;
+  dim3 grid((unsigned)(units < sms ? units : sms));
   int* status = reinterpret_cast<int*>(static_cast<char*>(ws) + p.ws_status_off);
   cudaError_t err = cudaSuccess;
   // three instantiations per (kb, halo): TMA-store epilogue with 8 or 16 epilogue warps, copy
   // epilogue with 8 (each kernel carries only the epilogue it runs: the hot loops are sensitive to
   // the size of the code around them)
-#define HGC_LAUNCH_IGEMM_EW(KBV, HALOV, EWV, COPYV)                                                         \
+#define HGC_LAUNCH_IGEMM_EW(KBV, HALOV, EWV, COPYV, SPLITV)                                                 \
   do {                                                                                                     \
-    err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV, EWV, COPYV>,                                        \
+    err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV, EWV, COPYV, SPLITV>,                                \
                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);            \
     if (err == cudaSuccess)                                                                                \
-      err = launch_kernel(igemm_kernel<KBV, HALOV, EWV, COPYV>, grid, dim3(64 + 32 * EWV), p.smem_bytes,    \
-                          stream, p.tmA, p.tmB, p.tmY, p.tmYr, a, bias, y, status);                        \
+      err = launch_kernel(igemm_kernel<KBV, HALOV, EWV, COPYV, SPLITV>, grid, dim3(64 + 32 * EWV),          \
+                          p.smem_bytes, stream, p.tmA, p.tmB, p.tmY, p.tmYr, a, bias, y, partials, status); \
   } while (0)
-#define HGC_LAUNCH_IGEMM(KBV, HALOV)                                                       \
-  do {                                                                                     \
-    if (!p.tma_store) HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 8, true);                            \
-    else if (p.epi_warps == kEpilogueWarpsWide) HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 16, false); \
-    else HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 8, false);                                        \
+#define HGC_LAUNCH_IGEMM(KBV, HALOV)                                                              \
+  do {                                                                                            \
+    if (!p.tma_store) HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 8, true, false);                            \
+    else if (p.epi_warps == kEpilogueWarpsWide) HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 16, false, false); \
+    else HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 8, false, false);                                        \
   } while (0)
+  if (p.ks_log2 > 0) {
+    HGC_LAUNCH_IGEMM_EW(64, true, 8, true, true);  // the one instantiation with a split reduction
+  } else
   if (p.kb == 64) {
     if (p.halo) HGC_LAUNCH_IGEMM(64, true); else HGC_LAUNCH_IGEMM(64, false);
   } else if (p.kb == 32) {
@@ -1296,6 +1460,16 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
 #undef HGC_LAUNCH_IGEMM
   if (err != cudaSuccess) return err;
   count_launch();
+  if (p.ks_log2 > 0) {
+    const int64_t total = a.part_stride;
+    int64_t blocks = (total + 255) / 256;
+    if (blocks > (int64_t)sms * 16) blocks = (int64_t)sms * 16;
+    err = launch_kernel(splitk_finish_kernel, dim3((unsigned)blocks), dim3(256), 0, stream, (const float*)partials,
+                        1 << p.ks_log2, a.part_stride, bias, reinterpret_cast<uint16_t*>(y), g.k,
+                        (int64_t)g.p * g.q, total, relu);
+    if (err != cudaSuccess) return err;
+    count_launch();
+  }
   return cudaGetLastError();
 }
 

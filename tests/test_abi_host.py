@@ -113,7 +113,7 @@ def test_planner_paths():
 
 def test_plan_info_reports_tiling_and_activation_source():
     """The planner runs on the host: its choices can be checked without a GPU."""
-    keys = {"path", "kb", "halo", "tn", "th", "pitch", "ncols", "tiles", "stages", "taps", "x_source"}
+    keys = {"path", "kb", "halo", "tn", "th", "pitch", "ncols", "tiles", "stages", "taps", "x_source", "k_slices"}
     cases = [
         # (n, c, h, w, k, r, s, pad, stride), x_source
         ((16, 256, 56, 56, 256, 3, 3, 1, 1), 0),   # NHWC copy of x
@@ -130,9 +130,13 @@ def test_plan_info_reports_tiling_and_activation_source():
         assert info["x_source"] == source, info
         assert info["kb"] in (16, 32, 64) and 16 <= info["ncols"] <= 256 and info["ncols"] % 16 == 0
         assert info["tn"] >= 1 and info["th"] >= 1 and info["stages"] >= 2 and info["tiles"] >= 1
+        assert info["k_slices"] == 1
         # an accumulator tile never holds more than 256 columns
         assert info["tn"] * info["th"] * info["pitch"] - (info["pitch"] - d.output_dims()[3]) <= 256
         d.close()
+    fc = hgc.ConvDesc.inner_product(64, 4096, 4096)
+    assert fc.plan_info()["k_slices"] in (2, 4, 8) and fc.plan_info()["tn"] == 64   # few tiles: split reduction
+    fc.close()
     dw = hgc.ConvDesc(2, 32, 14, 14, 32, 3, 3, 1, 1, 1, 1, 1, 1, 32)
     assert dw.plan_info()["kb"] == 0   # not the tensor-core path: zeros
 

@@ -43,6 +43,9 @@ CASES = [
     ("5x5 grouped pad 2", params_dict(1, 96, 27, 27, 256, 5, 5, 2, 2, 1, 1, 1, 1, 2), X_NHWC_COPY),
     ("3x3 dilation 2", params_dict(2, 24, 20, 18, 30, 3, 3, 2, 2, 1, 1, 2, 2), X_NHWC_COPY),
     ("3x1 and unpadded rows", params_dict(2, 40, 10, 40, 16, 3, 1, 1, 0), X_NHWC_COPY),
+    ("1x1 5x5 c4096 k96: reduction split over several CTAs, ragged channel tile", params_dict(3, 4096, 5, 5, 96, 1, 1), X_NHWC_COPY),
+    ("1x1 7x7 c2048 k200: reduction split, one-row tiles", params_dict(2, 2048, 7, 7, 200, 1, 1), X_NHWC_COPY),
+    ("1x1 3x5 c4096 k64: reduction split, several images per tile", params_dict(4, 4096, 3, 5, 64, 1, 1), X_NHWC_COPY),
     ("stem 3x3 c3 stride 1 (windows)", params_dict(2, 3, 32, 40, 16, 3, 3, 1, 1), X_WINDOWS),
     ("stem 7x7 c3 stride 2 (windows)", params_dict(2, 3, 64, 64, 64, 7, 7, 3, 3, 2, 2), X_WINDOWS),
     ("stem 11x11 c3 stride 4 (windows)", params_dict(1, 3, 67, 67, 96, 11, 11, 0, 0, 4, 4), X_WINDOWS),
@@ -63,6 +66,8 @@ def test_igemm_mode(hgc, oracle, name, a, source):
     assert d.path() == hgc.HGC_PATH_IGEMM, name
     if source is not None:
         assert d.plan_info()["x_source"] == source, (name, d.plan_info())
+    if "reduction split" in name:
+        assert d.plan_info()["k_slices"] > 1, d.plan_info()
     d.close()
     for relu, bias, registered in ((True, b, True), (False, None, False)):
         ref = oracle.conv_fast(P, x, w, bias, relu)
