@@ -340,6 +340,53 @@ def run_ours(args, wl):
     layer_ms = [sum(ev[s][i][0].elapsed_time(ev[s][i][1]) for s in range(lsteps)) / lsteps
                 for i in range(len(state))]
 
+    # ---- the same step with channels-last activations (HGC_FLAG_X_NHWC / HGC_FLAG_Y_NHWC) --------
+    # Not the headline (the metric is NCHW in, NCHW out): what a stack of layers that keeps its
+    # activations channels-last between layers pays per step.  Layers that cannot take a flag
+    # (3-channel stems on the input side, depthwise layers) keep NCHW on that side.
+    nhwc = None
+    if not args.no_graph:
+        try:
+            nstate, n_in, n_out = [], 0, 0
+            for (d0, x, w, b, y, l) in state:
+                geo = (batch, l.c, l.h, l.h, l.k, l.r, l.r, l.pad, l.pad, l.stride, l.stride, l.dil, l.dil, l.group)
+                d = None
+                for fl in (hgc.HGC_FLAG_X_NHWC | hgc.HGC_FLAG_Y_NHWC, hgc.HGC_FLAG_Y_NHWC, 0):
+                    try:
+                        d = hgc.ConvDesc(*geo, fl)
+                        break
+                    except hgc.HgcError:
+                        continue
+                d.ensure_workspace()
+                d.set_weights(w)
+                n_in += 1 if fl & hgc.HGC_FLAG_X_NHWC else 0
+                n_out += 1 if fl & hgc.HGC_FLAG_Y_NHWC else 0
+                nstate.append((d, x, w, b, y, l))   # same buffers: only the interpretation of x and y changes
+            gl = torch.cuda.CUDAGraph()
+            for (d, x, w, b, y, l) in nstate:
+                hgc.conv_forward(d, x, w, b, y, l.relu, side)
+            torch.cuda.synchronize()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(gl, stream=side):
+                    for (d, x, w, b, y, l) in nstate:
+                        hgc.conv_forward(d, x, w, b, y, l.relu, side)
+                torch.cuda.synchronize()
+                for _ in range(3):
+                    gl.replay()
+                n0, n1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                n0.record(side)
+                for _ in range(args.steps):
+                    gl.replay()
+                n1.record(side)
+            torch.cuda.synchronize()
+            nms = n0.elapsed_time(n1) / args.steps
+            nhwc = {"ms_per_step": nms, "layers_with_channels_last_input": n_in,
+                    "layers_with_channels_last_output": n_out, "layers": len(nstate),
+                    "note": "same layers, activations channels-last where the layer takes the flag; this rank"}
+        except Exception as exc:
+            nhwc = {"error": repr(exc)}
+
     # ---- end to end through the host-buffer entry point ------------------------------------
     e2e_steps = max(1, min(args.steps, 5))
     host = []
@@ -441,6 +488,10 @@ def run_ours(args, wl):
                                  "(source of the per-layer and per-kernel times), this rank"}
         if graph_err is not None:
             line["graph_error"] = graph_err
+        if nhwc is not None:
+            if "ms_per_step" in nhwc:
+                nhwc["tflops"] = step_flops / (nhwc["ms_per_step"] * 1e-3) / 1e12
+            line["channels_last"] = nhwc
         if cpu is not None:
             line["cpu_baseline"] = cpu
         if args.layers:

@@ -17,6 +17,8 @@ HGC_OK, HGC_INVALID_ARG, HGC_UNSUPPORTED, HGC_BAD_ALIGNMENT, HGC_NO_WORKSPACE, H
     HGC_DEVICE_TIMEOUT = range(7)
 HGC_PATH_DIRECT, HGC_PATH_DEPTHWISE, HGC_PATH_IGEMM = range(3)
 HGC_FLAG_FORCE_DIRECT = 1
+HGC_FLAG_X_NHWC = 2
+HGC_FLAG_Y_NHWC = 4
 PATH_NAMES = {HGC_PATH_DIRECT: "direct", HGC_PATH_DEPTHWISE: "depthwise", HGC_PATH_IGEMM: "igemm"}
 
 

@@ -126,16 +126,23 @@ int hgc_conv_desc_create(hgc_conv_desc** out, const hgc_conv_params* p) {
   g.group = p->group;
   g.p = (int32_t)P; g.q = (int32_t)Q;
   g.cg = p->c / p->group; g.kg = p->k / p->group;
+  g.x_nhwc = (p->flags & HGC_FLAG_X_NHWC) ? 1 : 0;
+  g.y_nhwc = (p->flags & HGC_FLAG_Y_NHWC) ? 1 : 0;
+  const bool channels_last = g.x_nhwc || g.y_nhwc;
 
   d->path = HGC_PATH_DIRECT;
   d->ws_needed = 0;
   if (!(p->flags & HGC_FLAG_FORCE_DIRECT)) {
-    if (hgc::depthwise3x3_supported(g)) {
+    if (!channels_last && hgc::depthwise3x3_supported(g)) {
       d->path = HGC_PATH_DEPTHWISE;
     } else if (hgc::igemm_make_plan(g, &d->igemm)) {
       d->path = HGC_PATH_IGEMM;
       d->ws_needed = d->igemm.ws_total;
     }
+  }
+  if (channels_last && d->path != HGC_PATH_IGEMM) {  // only the tensor-core path takes channels-last tensors
+    delete d;
+    return HGC_UNSUPPORTED;
   }
   d->ws = nullptr;
   d->ws_bytes = 0;

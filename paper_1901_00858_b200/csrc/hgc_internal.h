@@ -17,6 +17,7 @@ struct ConvGeom {
   int32_t group;
   int32_t p, q;    // output plane
   int32_t cg, kg;  // channels per group: C/group, K/group
+  int32_t x_nhwc, y_nhwc;  // channels-last input / output (tensor-core path only)
 };
 
 void count_launch();  // bumps the process-wide kernel launch counter
@@ -74,10 +75,11 @@ cudaError_t launch_nhwc_to_nchw(const __half* src, __half* dst, int32_t n, int32
                                 int32_t w, int32_t c_pad, cudaStream_t stream);
 cudaError_t launch_nchw_to_nhwc8_bordered(const __half* src, __half* dst, int32_t n, int32_t c, int32_t h, int32_t w,
                                           int32_t pad_h, int32_t pad_w, int32_t hp, int32_t wp, cudaStream_t stream);
+// perm: rows of every block of 32 output channels interleaved (see row_channel in layout.cu)
 cudaError_t launch_weights_repack_window(const __half* src, __half* dst, int32_t k, int32_t c, int32_t r, int32_t s,
-                                         int32_t kw_pix, cudaStream_t stream);
+                                         int32_t kw_pix, cudaStream_t stream, int perm = 0);
 cudaError_t launch_weights_repack(const __half* src, __half* dst, int32_t k, int32_t cg, int32_t r,
-                                  int32_t s, int32_t group, int32_t c_pad, cudaStream_t stream);
+                                  int32_t s, int32_t group, int32_t c_pad, cudaStream_t stream, int perm = 0);
 
 cudaError_t launch_cast_f32_to_f16(const float* src, __half* dst, int64_t count, unsigned long long* overflow,
                                    cudaStream_t stream);
@@ -87,7 +89,10 @@ struct IgemmPlan {
   int32_t kb, cblocks, cw, c_pad;
   int32_t halo, pitch;
   int32_t nchw, nblk;                            // 1x1 layers reading x (NCHW) directly
-  const void* x_mapped;                          // input pointer tmB was encoded for (nchw)
+  const void* x_mapped;                          // input pointer tmB was encoded for (nchw, x_nhwc)
+  int32_t x_nhwc, y_nhwc;                        // channels-last input (no layout pass) / output
+  int32_t y_rpu, y_full_w;                       // channels-last stores: tile rows and pixels per store
+  int32_t y_perm;                                // weight rows interleaved for the staged channels-last epilogue
   int32_t window, kw_pix, hp, wp;                // few-channel layers: windows over a zero-bordered NHWC8 copy
   int32_t patch;                                 // tiny receptive fields: 1x1 conv over an im2col copy of x
   int32_t eff_r, eff_s, eff_pad_h, eff_pad_w;    // the convolution as the kernel sees it

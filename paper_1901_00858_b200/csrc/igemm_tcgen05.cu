@@ -589,6 +589,71 @@ splitk_finish_kernel(const float* __restrict__ part, int slices, int64_t stride,
   }
 }
 
+// Channels-last epilogue (y[N][P][Q][K]): a lane owns a channel, so for every output pixel the 32
+// lanes of a warp write 32 consecutive channels (64 contiguous bytes) straight from registers.
+// A unit of work is one tile row x up to 32 pixels; the warps of a lane quarter take units in turn.
+__device__ __noinline__ void epilogue_nhwc(uint32_t t_addr, int first_unit, int unit_step, int tn, int th, int pitch,
+                                           int N, int K, int P, int Q, int n0, int p0, int k, bool kvalid, float bv,
+                                           bool relu, uint16_t* yb) {
+  const int rows_valid = (P - p0) < th ? (P - p0) : th;
+  int unit = 0;
+  for (int img = 0; img < tn; ++img) {
+    if (n0 + img >= N) break;
+    for (int hr = 0; hr < rows_valid; ++hr) {
+      for (int wc0 = 0; wc0 < Q; wc0 += 32, ++unit) {
+        if (unit % unit_step != first_unit) continue;
+        const int ncol = Q - wc0 < 32 ? Q - wc0 : 32;
+        const uint32_t tcol = t_addr + (uint32_t)((img * th + hr) * pitch + wc0);
+        uint32_t v[32];
+        if (ncol == 32) {
+          tmem_ld32(tcol, v);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+            if (c * 8 < ncol) tmem_ld8(tcol + (uint32_t)(c * 8), &v[8 * c]);
+        }
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        uint16_t* dst = yb + (((int64_t)(n0 + img) * P + (p0 + hr)) * Q + wc0) * K + k;
+#pragma unroll
+        for (int j = 0; j < 32; j += 2) {
+          if (j < ncol) {
+            const float f0 = __uint_as_float(v[j]) + bv, f1 = __uint_as_float(v[j + 1]) + bv;
+            const uint32_t o = relu ? pack_f16x2<true>(f0, f1) : pack_f16x2<false>(f0, f1);
+            if (kvalid) {
+              dst[(int64_t)j * K] = (uint16_t)(o & 0xffffu);
+              if (j + 1 < ncol) dst[(int64_t)(j + 1) * K] = (uint16_t)(o >> 16);
+            }
+          }
+        }
+      }
+    }
+  }
+  __syncwarp();
+}
+
+// Channels-last staging: up to 32 accumulator columns (pixels) of this lane's channel -> fp16
+// pairs -> a dense [pixel][32 channels] tile in shared memory (64 bytes per pixel).  Each group of
+// 8 pixels is four 8x8 matrices (one per pixel pair) spread over the warp's registers; a
+// transposing matrix store writes them as 16-byte rows of eight channels of one pixel.  That needs
+// the lanes to hold the channels interleaved (lane 4*b + a = channel 8*a + b of the warp's 32),
+// which the weight re-layout arranges.  `dst` is this lane's row address for the first 8 pixels:
+// lane T addresses pixel 2*(T/8) + T%2, channels 8*((T%8)/2)...
+template <bool RELU>
+__device__ __forceinline__ void convert_store_pixels(const uint32_t (&v)[32], int npix, float bv, uint32_t dst) {
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    if (c * 8 < npix) {
+      const uint32_t o0 = pack_f16x2<RELU>(__uint_as_float(v[8 * c + 0]) + bv, __uint_as_float(v[8 * c + 1]) + bv);
+      const uint32_t o1 = pack_f16x2<RELU>(__uint_as_float(v[8 * c + 2]) + bv, __uint_as_float(v[8 * c + 3]) + bv);
+      const uint32_t o2 = pack_f16x2<RELU>(__uint_as_float(v[8 * c + 4]) + bv, __uint_as_float(v[8 * c + 5]) + bv);
+      const uint32_t o3 = pack_f16x2<RELU>(__uint_as_float(v[8 * c + 6]) + bv, __uint_as_float(v[8 * c + 7]) + bv);
+      asm volatile("stmatrix.sync.aligned.m8n8.x4.trans.shared.b16 [%0], {%1, %2, %3, %4};" ::"r"(dst + (uint32_t)c * 512u),
+                   "r"(o0), "r"(o1), "r"(o2), "r"(o3)
+                   : "memory");
+    }
+  }
+}
+
 struct IgemmArgs {
   int32_t N, K, P, Q;
   int32_t kg, group;
@@ -624,6 +689,9 @@ struct IgemmArgs {
   // second kernel adds the slices in a fixed order (+ bias, ReLU, rounding)
   int32_t ks_log2;
   int64_t part_stride;  // elements between two slices: N * K * P * Q
+  int32_t y_tma;        // channels-last output staged for TMA stores (else plain stores)
+  int32_t y_full_w;     // pixels of a full channels-last store
+  int32_t y_rpu;        // tile rows per channels-last store (rows of at most 32 pixels are batched)
 };
 
 // The tiles of one CTA: blockIdx.x, blockIdx.x + gridDim.x, ...  Tile t = (pixel tile px, channel
@@ -697,7 +765,8 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 
 // Persistent kernel: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...; the two TMEM
 // accumulators alternate so that the epilogue of one tile overlaps the MMAs of the next.
-template <int KB, bool HALO, int EW, bool COPY, bool SPLIT>
+// EPI: 0 = TMA-store epilogue, 1 = copy epilogue (NCHW, any shape), 2 = channels-last output
+template <int KB, bool HALO, int EW, int EPI, bool SPLIT>
 __global__ void __launch_bounds__(64 + 32 * EW, 1)
 igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
              const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmYr,
@@ -881,7 +950,9 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const int ew = warp - 2;
     const int quarter = warp & 3;
     const int half = ew >> 2;  // which of the quarter's warps this is
-    const int row = quarter * 32 + lane;  // accumulator lane = output channel within the tile
+    // accumulator lane = output channel within the tile (interleaved within the warp's 32 when the
+    // staged channels-last epilogue runs: see convert_store_pixels)
+    const int row = quarter * 32 + ((EPI == 2 && a.y_tma) ? ((lane & 3) << 3) + (lane >> 2) : lane);
     uint16_t* yb = reinterpret_cast<uint16_t*>(y);
     const uint32_t stage_base = ring_base + (uint32_t)a.stages * a.stage_bytes;
     const bool relu = a.relu != 0;
@@ -906,7 +977,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       const uint32_t t_addr = tmem_base + buf * 256u + ((uint32_t)(quarter * 32) << 16);
       const bool quarter_live = m0 + quarter * 32 < a.kg;  // any real output channel in this warp's lanes?
 
-      if constexpr (!COPY) {
+      if constexpr (EPI == 0) {
         // ---- staged epilogue: TMEM -> registers -> swizzled fp16 tile in smem -> TMA store ----
         // (taken when Q % 8 == 0, hence P*Q % 8 == 0, and a tile holds one image: every staged run
         //  of pixels then starts on a 16-byte boundary of y).  A unit of work is 32 channels (this
@@ -986,7 +1057,75 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         // ---- direct epilogue: each thread stores runs of its own channel plane ----
         {
           // the warps of a lane quarter take alternate units
-          if constexpr (SPLIT) {
+          if constexpr (EPI == 2) {
+            if (quarter_live && a.y_tma) {
+              // staged channels-last epilogue (output channels per group a multiple of 8: every
+              // pixel's run of channels starts on a 16-byte boundary of y).  A unit of work is this
+              // warp's 32 channels x up to 64 consecutive output pixels: a piece of a tile row, or
+              // several whole rows when rows are at most 32 pixels wide; one TMA store per unit,
+              // clipped at the last channel of the group and at the end of the image.
+              const uint32_t lane_off = (2u * ((uint32_t)lane >> 3) + ((uint32_t)lane & 1u)) * 64u +
+                                        (((uint32_t)lane & 7u) >> 1) * 16u;
+              const int rows_valid = (a.P - p0) < a.th ? (a.P - p0) : a.th;
+              const int cpu = a.Q > kPassElems ? kPassElems : a.Q;  // columns per unit
+              int unit = 0;
+              for (int img = 0; img < a.tn; ++img) {
+                if (n0 + img >= a.N) break;
+                for (int hr0 = 0; hr0 < rows_valid; hr0 += a.y_rpu) {
+                  for (int wc0 = 0; wc0 < a.Q; wc0 += cpu, ++unit) {
+                    if (unit % kPerQuarter != half) continue;
+                    const int nrows = rows_valid - hr0 < a.y_rpu ? rows_valid - hr0 : a.y_rpu;
+                    const int ncol = a.Q - wc0 < cpu ? a.Q - wc0 : cpu;
+                    const uint32_t sbuf = my_stage + stage_sel * kWarpStageBytes;
+                    stage_sel = a.nbuf == 2 ? stage_sel ^ 1u : 0u;
+                    bool first = true;
+#pragma unroll 1
+                    for (int r = 0; r < nrows; ++r) {
+#pragma unroll 1
+                      for (int g = 0; g < 2; ++g) {
+                        const int rem = ncol - g * 32;
+                        if (rem <= 0) break;
+                        const uint32_t tcol = t_addr + (uint32_t)((img * a.th + hr0 + r) * a.pitch + wc0 + g * 32);
+                        uint32_t v[32];
+                        if (rem >= 32) {
+                          tmem_ld32(tcol, v);
+                        } else {
+#pragma unroll
+                          for (int c = 0; c < 4; ++c)
+                            if (c * 8 < rem) tmem_ld8(tcol + (uint32_t)(c * 8), &v[8 * c]);
+                        }
+                        if (first) {
+                          // this buffer's previous store must have been read out of shared memory
+                          if (lane == 0) {
+                            if (a.nbuf == 1) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                            else asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                          }
+                          __syncwarp();
+                          first = false;
+                        }
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                        const uint32_t dst = sbuf + (uint32_t)(r * ncol + g * 32) * 64u + lane_off;
+                        if (relu) convert_store_pixels<true>(v, rem, bv, dst);
+                        else convert_store_pixels<false>(v, rem, bv, dst);
+                      }
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                      // a short unit at the end of the image takes the full box: the rest is clipped
+                      const bool image_end = p0 + hr0 + nrows == a.P && wc0 + ncol == a.Q;
+                      tma_store_4d((nrows * ncol == a.y_full_w || image_end) ? &tmY : &tmYr, sbuf, m0 + quarter * 32, grp,
+                                   (p0 + hr0) * a.Q + wc0, n0 + img);
+                      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    }
+                  }
+                }
+              }
+            }
+            else if (EW == 8 && quarter_live)  // (16 epilogue warps only ever run the staged form)
+              epilogue_nhwc(t_addr, half, kPerQuarter, a.tn, a.th, a.pitch, a.N, a.K, a.P, a.Q, n0, p0, k, kvalid, bv,
+                            relu, yb);
+          } else if constexpr (SPLIT) {
             if (quarter_live) {
               const int kleft = a.kg - (m0 + quarter * 32);
               epilogue_partial(t_addr, my_stage, half, kPerQuarter, a.tn, a.th, a.pitch, a.N, a.K, a.P, a.Q, n0, p0,
@@ -1062,6 +1201,10 @@ int sm_count() {
 bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   IgemmPlan p{};
   if (g.group > 1 && (g.cg % 8) != 0) return false;  // group stride of x' must be 16-byte aligned
+  p.x_nhwc = g.x_nhwc;
+  p.y_nhwc = g.y_nhwc;
+  // channels-last input: x is used as x' (a pixel must be a whole number of 16-byte vectors)
+  if (p.x_nhwc && ((g.c % 8) != 0 || g.cg < 9)) return false;
   // Few input channels (image stems, C <= 8): a tap alone is too short for a K=16 MMA step.
   // The input is copied to a zero-bordered NHWC buffer with 8 channels per pixel; the S taps of
   // a kernel row are then S*8 CONTIGUOUS elements, read as one "window" per output pixel through
@@ -1075,8 +1218,8 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   // (measured: 3x3 stride-2 stem 50.6 us against 56.8 us in window mode; at stride 1 the window
   // mode wins, 74.7 us against 82.5 us, because the expansion pass writes 64 bytes per pixel).
   const int64_t rsc = (int64_t)g.r * g.s * g.cg;
-  p.patch = (g.group == 1 && rsc <= 64 && (g.stride_h > 1 || g.stride_w > 1) && g.cg <= 8) ? 1 : 0;
-  p.window = (!p.patch && g.cg <= 8 && g.group == 1 && g.dil_w == 1) ? 1 : 0;
+  p.patch = (!p.x_nhwc && g.group == 1 && rsc <= 64 && (g.stride_h > 1 || g.stride_w > 1) && g.cg <= 8) ? 1 : 0;
+  p.window = (!p.x_nhwc && !p.patch && g.cg <= 8 && g.group == 1 && g.dil_w == 1) ? 1 : 0;
   if (!p.window && !p.patch && g.cg < 9) return false;
   if (p.patch) {
     const int kelems = rsc <= 16 ? 16 : (rsc <= 32 ? 32 : 64);
@@ -1113,7 +1256,7 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   }
   // 1x1, stride 1, unpadded layers on planes of a multiple of 8 pixels read x as it is (no NHWC
   // copy): the activation operand is then pixel-major ("MN-major") in shared memory
-  p.nchw = (!p.window && !p.patch && g.r == 1 && g.s == 1 && g.stride_h == 1 && g.stride_w == 1 && g.pad_h == 0 &&
+  p.nchw = (!p.x_nhwc && !p.window && !p.patch && g.r == 1 && g.s == 1 && g.stride_h == 1 && g.stride_w == 1 && g.pad_h == 0 &&
             g.pad_w == 0 && g.group == 1 && ((int64_t)g.h * g.w) % 8 == 0)
                ? 1
                : 0;
@@ -1160,7 +1303,7 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
     return 8000.0 + elems * (4.0 * (1 << ks) + 2.0) / 3000.0;
   };
   // the split kernel exists for 64-channel stages of stride-1 layers without the direct-x mode
-  const bool can_split = p.kb == 64 && p.halo && !p.nchw;
+  const bool can_split = p.kb == 64 && p.halo && !p.nchw && !p.y_nhwc;
   double best = 1e300;
   int best_th = 0, best_tn = 0, best_ks = 0;
   for (int th = 1; th <= g.p; ++th) {
@@ -1225,6 +1368,19 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   p.epi_warps = kEpilogueWarps;
   if (p.tma_store && mpt * 130.0 < 600.0 + 10.0 * p.ncols && (p.th * g.q) > 2 * kPassElems)
     p.epi_warps = kEpilogueWarpsWide;
+  if (p.y_nhwc) {
+    // channels-last output: up to 64 pixels x 32 channels staged for TMA stores when the groups
+    // have whole blocks of 32 output channels (the weight rows are then interleaved for the
+    // transposing staging stores), else plain stores (any shape)
+    p.tma_store = (g.kg % 32) == 0 ? 1 : 0;
+    p.y_perm = p.tma_store;
+    p.y_rpu = g.q > 32 ? 1 : (kPassElems / g.q < p.th ? kPassElems / g.q : p.th);
+    p.y_full_w = g.q > kPassElems ? kPassElems : p.y_rpu * g.q;
+    p.rem = g.q > kPassElems ? g.q % kPassElems : (p.th % p.y_rpu) * g.q;
+    p.epi_warps = kEpilogueWarps;
+    if (p.tma_store && mpt * 130.0 < 600.0 + 10.0 * p.ncols && p.tn * p.th * ((g.q + kPassElems - 1) / kPassElems) > 2)
+      p.epi_warps = kEpilogueWarpsWide;
+  }
   // split reduction (chosen with the tile shape above): fp32 partials, copy-style epilogue
   p.ks_log2 = best_ks;
   if (p.ks_log2 > 0) {
@@ -1271,7 +1427,7 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   p.ws_w_off = 256;
   p.ws_x_off = p.ws_w_off + round_up_sz((size_t)g.k * p.eff_r * p.eff_s * p.cw * 2, 256);
   p.ws_part_off = 0;
-  p.ws_total = p.ws_x_off + (p.nchw ? 0
+  p.ws_total = p.ws_x_off + ((p.nchw || p.x_nhwc) ? 0
                                     : round_up_sz(p.patch    ? (size_t)g.n * g.p * g.q * p.cw * 2
                                                   : p.window ? (size_t)g.n * p.hp * p.wp * 16 + 256
                                                            : (size_t)g.n * g.h * g.w * p.c_pad * 2, 256));
@@ -1281,6 +1437,25 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   }
   *out = p;
   return true;
+}
+
+// The 5-D map (channel in group, group, W, H, N) over a channels-last activation tensor at `base`:
+// the NHWC copy in the workspace, or the caller's x itself when it is channels-last already.
+bool encode_nhwc_map(const ConvGeom& g, IgemmPlan* p, void* base) {
+  PFN_cuTensorMapEncodeTiled_v12000 enc = encode_fn();
+  if (enc == nullptr) return false;
+  const CUtensorMapSwizzle sw = p->kb == 64 ? CU_TENSOR_MAP_SWIZZLE_128B
+                               : p->kb == 32 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                             : CU_TENSOR_MAP_SWIZZLE_32B;
+  const cuuint64_t cdim = g.group > 1 ? (cuuint64_t)g.cg : (cuuint64_t)p->c_pad;
+  const cuuint64_t pix = (cuuint64_t)p->c_pad * 2;
+  cuuint64_t dims[5] = {cdim, (cuuint64_t)g.group, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.n};
+  cuuint64_t strides[4] = {g.group > 1 ? (cuuint64_t)g.cg * 2 : pix, pix, pix * g.w, pix * g.w * g.h};
+  const cuuint32_t box_w = p->halo ? (cuuint32_t)p->pitch : (cuuint32_t)(p->tw * g.stride_w);
+  cuuint32_t box[5] = {(cuuint32_t)p->kb, 1, box_w, (cuuint32_t)(p->th * g.stride_h), (cuuint32_t)p->tn};
+  cuuint32_t es[5] = {1, 1, (cuuint32_t)g.stride_w, (cuuint32_t)g.stride_h, 1};
+  return enc(&p->tmB, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // Encodes the two tensor maps over the workspace tensors.  Returns false on failure.
@@ -1328,18 +1503,10 @@ bool igemm_encode_maps(const ConvGeom& g, IgemmPlan* p, void* ws) {
             CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return false;
-  } else {
-    const cuuint64_t cdim = g.group > 1 ? (cuuint64_t)g.cg : (cuuint64_t)p->c_pad;
-    const cuuint64_t pix = (cuuint64_t)p->c_pad * 2;
-    cuuint64_t dims[5] = {cdim, (cuuint64_t)g.group, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.n};
-    cuuint64_t strides[4] = {g.group > 1 ? (cuuint64_t)g.cg * 2 : pix, pix, pix * g.w, pix * g.w * g.h};
-    const cuuint32_t box_w = p->halo ? (cuuint32_t)p->pitch : (cuuint32_t)(p->tw * g.stride_w);
-    cuuint32_t box[5] = {(cuuint32_t)p->kb, 1, box_w, (cuuint32_t)(p->th * g.stride_h), (cuuint32_t)p->tn};
-    cuuint32_t es[5] = {1, 1, (cuuint32_t)g.stride_w, (cuuint32_t)g.stride_h, 1};
-    if (enc(&p->tmB, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, base + p->ws_x_off, dims, strides, box, es,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return false;
+  } else if (p->x_nhwc) {
+    // the activation map is over the caller's x (channels-last) and is encoded when x is known
+  } else if (!encode_nhwc_map(g, p, base + p->ws_x_off)) {
+    return false;
   }
   p->maps_ready = true;
   return true;
@@ -1369,6 +1536,22 @@ bool igemm_encode_y_maps(const ConvGeom& g, IgemmPlan* p, void* y) {
   PFN_cuTensorMapEncodeTiled_v12000 enc = encode_fn();
   if (enc == nullptr) return false;
   const cuuint64_t pq = (cuuint64_t)g.p * g.q;
+  if (p->y_nhwc) {
+    // y[N][P*Q][group][kg]: a store is up to 64 pixels of one row x 32 channels, dense in smem
+    cuuint64_t dims[4] = {(cuuint64_t)g.kg, (cuuint64_t)g.group, pq, (cuuint64_t)g.n};
+    cuuint64_t strides[3] = {(cuuint64_t)g.kg * 2, (cuuint64_t)g.k * 2, pq * 2 * (cuuint64_t)g.k};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    const cuuint32_t full_w = (cuuint32_t)p->y_full_w;
+    for (int i = 0; i < 2; ++i) {
+      cuuint32_t box[4] = {32, 1, (i == 0 || p->rem == 0) ? full_w : (cuuint32_t)p->rem, 1};
+      if (enc(i == 0 ? &p->tmY : &p->tmYr, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, y, dims, strides, box, es,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    }
+    p->y_mapped = y;
+    return true;
+  }
   cuuint64_t dims[4] = {pq, (cuuint64_t)g.kg, (cuuint64_t)g.group, (cuuint64_t)g.n};
   cuuint64_t strides[3] = {pq * 2, pq * 2 * (cuuint64_t)g.kg, pq * 2 * (cuuint64_t)g.k};
   cuuint32_t es[4] = {1, 1, 1, 1};
@@ -1387,6 +1570,10 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
                          int relu, cudaStream_t stream) {
   if (!p.maps_ready) return cudaErrorInvalidValue;
   if (p.nchw && p.x_mapped != x && !igemm_encode_x_map(g, &p, x)) return cudaErrorInvalidValue;
+  if (p.x_nhwc && p.x_mapped != x) {
+    if (!encode_nhwc_map(g, &p, const_cast<__half*>(x))) return cudaErrorInvalidValue;
+    p.x_mapped = x;
+  }
   if (p.tma_store && p.y_mapped != y && !igemm_encode_y_maps(g, &p, y)) return cudaErrorInvalidValue;
   IgemmArgs a{};
   a.N = g.n; a.K = g.k; a.P = g.p; a.Q = g.q;
@@ -1423,31 +1610,36 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
   a.nbuf = p.nbuf;
   a.ks_log2 = p.ks_log2;
   a.part_stride = (int64_t)g.n * g.k * g.p * g.q;
+  a.y_tma = (p.y_nhwc && p.tma_store) ? 1 : 0;
+  a.y_full_w = p.y_full_w;
+  a.y_rpu = p.y_rpu > 0 ? p.y_rpu : 1;
   float* partials = p.ks_log2 > 0 ? reinterpret_cast<float*>(static_cast<char*>(ws) + p.ws_part_off) : nullptr;
   const int sms = sm_count();
   const int64_t units = (int64_t)p.total_tiles << p.ks_log2;
   dim3 grid((unsigned)(units < sms ? units : sms));
   int* status = reinterpret_cast<int*>(static_cast<char*>(ws) + p.ws_status_off);
   cudaError_t err = cudaSuccess;
-  // three instantiations per (kb, halo): TMA-store epilogue with 8 or 16 epilogue warps, copy
-  // epilogue with 8 (each kernel carries only the epilogue it runs: the hot loops are sensitive to
+  // four instantiations per (kb, halo): TMA-store epilogue with 8 or 16 epilogue warps, copy
+  // epilogue and channels-last epilogue with 8 (each kernel carries only the epilogue it runs: the hot loops are sensitive to
   // the size of the code around them)
-#define HGC_LAUNCH_IGEMM_EW(KBV, HALOV, EWV, COPYV, SPLITV)                                                 \
+#define HGC_LAUNCH_IGEMM_EW(KBV, HALOV, EWV, EPIV, SPLITV)                                                 \
   do {                                                                                                     \
-    err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV, EWV, COPYV, SPLITV>,                                \
+    err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV, EWV, EPIV, SPLITV>,                                \
                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);            \
     if (err == cudaSuccess)                                                                                \
-      err = launch_kernel(igemm_kernel<KBV, HALOV, EWV, COPYV, SPLITV>, grid, dim3(64 + 32 * EWV),          \
+      err = launch_kernel(igemm_kernel<KBV, HALOV, EWV, EPIV, SPLITV>, grid, dim3(64 + 32 * EWV),          \
                           p.smem_bytes, stream, p.tmA, p.tmB, p.tmY, p.tmYr, a, bias, y, partials, status); \
   } while (0)
 #define HGC_LAUNCH_IGEMM(KBV, HALOV)                                                              \
   do {                                                                                            \
-    if (!p.tma_store) HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 8, true, false);                            \
-    else if (p.epi_warps == kEpilogueWarpsWide) HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 16, false, false); \
-    else HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 8, false, false);                                        \
+    if (p.y_nhwc && p.epi_warps == kEpilogueWarpsWide) HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 16, 2, false); \
+    else if (p.y_nhwc) HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 8, 2, false);                              \
+    else if (!p.tma_store) HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 8, 1, false);                          \
+    else if (p.epi_warps == kEpilogueWarpsWide) HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 16, 0, false);    \
+    else HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 8, 0, false);                                            \
   } while (0)
   if (p.ks_log2 > 0) {
-    HGC_LAUNCH_IGEMM_EW(64, true, 8, true, true);  // the one instantiation with a split reduction
+    HGC_LAUNCH_IGEMM_EW(64, true, 8, 1, true);  // the one instantiation with a split reduction
   } else
   if (p.kb == 64) {
     if (p.halo) HGC_LAUNCH_IGEMM(64, true); else HGC_LAUNCH_IGEMM(64, false);

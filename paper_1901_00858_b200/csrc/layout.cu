@@ -196,9 +196,20 @@ nhwc_to_nchw_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst
   }
 }
 
+// Output channel held by row `row` of the re-laid-out weights.  Normally the row itself; with
+// `perm` (layers that write y channels-last through the staged epilogue) the rows of every block
+// of 32 are interleaved, row 4*b + a holding channel 8*a + b of the block: the accumulator lanes
+// of an epilogue warp then hold the channels in the order in which a transposing matrix store
+// writes eight consecutive channels of one pixel as one 16-byte row.
+__device__ __forceinline__ int64_t row_channel(int64_t row, int perm) {
+  if (!perm) return row;
+  const int64_t in = row & 31;
+  return (row & ~(int64_t)31) + 8 * (in & 3) + (in >> 2);
+}
+
 // w[g*kg + k'][c'][r][s] -> w'[g][k'][r][s][c_pad]; one thread per 8 output channels-of-input
 __global__ void weights_repack_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst,
-                                      int64_t k, int cg, int rs, int c_pad) {
+                                      int64_t k, int cg, int rs, int c_pad, int perm) {
   grid_dependency_wait();
   const int64_t vecs_per_k = (int64_t)rs * (c_pad / 8);
   const int64_t total = k * vecs_per_k;
@@ -213,7 +224,7 @@ __global__ void weights_repack_kernel(const uint16_t* __restrict__ src, uint16_t
     for (int j = 0; j < 8; ++j) {
       const int ch = cv * 8 + j;
       uint32_t v = 0;
-      if (ch < cg) v = src[(kk * cg + ch) * rs + t];
+      if (ch < cg) v = src[(row_channel(kk, perm) * cg + ch) * rs + t];
       o[j >> 1] |= v << ((j & 1) * 16);
     }
     *reinterpret_cast<uint4*>(dst + (kk * rs + t) * c_pad + cv * 8) = make_uint4(o[0], o[1], o[2], o[3]);
@@ -246,7 +257,7 @@ nchw_to_nhwc8_bordered_kernel(const uint16_t* __restrict__ src, uint16_t* __rest
 
 // w[k][c][r][s] (c <= 8) -> w'[k][r][kw_pix][8]: tap s, channel ch at [s][ch]; zeros elsewhere.
 __global__ void weights_repack_window_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst,
-                                             int64_t k, int c, int r, int s, int kw_pix) {
+                                             int64_t k, int c, int r, int s, int kw_pix, int perm) {
   grid_dependency_wait();
   const int64_t total = k * r * kw_pix;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
@@ -258,7 +269,8 @@ __global__ void weights_repack_window_kernel(const uint16_t* __restrict__ src, u
     if (sp < s) {
 #pragma unroll
       for (int ch = 0; ch < 8; ++ch)
-        if (ch < c) o[ch >> 1] |= (uint32_t)src[((kk * c + ch) * r + rr) * s + sp] << ((ch & 1) * 16);
+        if (ch < c)
+          o[ch >> 1] |= (uint32_t)src[((row_channel(kk, perm) * c + ch) * r + rr) * s + sp] << ((ch & 1) * 16);
     }
     *reinterpret_cast<uint4*>(dst + i * 8) = make_uint4(o[0], o[1], o[2], o[3]);
   }
@@ -353,7 +365,7 @@ patch_im2col_generic_kernel(const uint16_t* __restrict__ src, uint16_t* __restri
 
 // w[k][c][r][s] -> w'[k][kelems], element (r*S + s)*C + ch; zeros from R*S*C on
 __global__ void weights_repack_patch_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int64_t k,
-                                            int c, int r, int s, int kelems) {
+                                            int c, int r, int s, int kelems, int perm) {
   grid_dependency_wait();
   const int64_t total = k * kelems;
   const int rsc = r * s * c;
@@ -364,7 +376,7 @@ __global__ void weights_repack_patch_kernel(const uint16_t* __restrict__ src, ui
     if (e < rsc) {
       const int ch = e % c;
       const int tap = e / c;
-      v = src[(kk * c + ch) * (r * s) + tap];
+      v = src[(row_channel(kk, perm) * c + ch) * (r * s) + tap];
     }
     dst[i] = v;
   }
@@ -384,12 +396,12 @@ cudaError_t launch_nchw_to_nhwc8_bordered(const __half* src, __half* dst, int32_
 }
 
 cudaError_t launch_weights_repack_window(const __half* src, __half* dst, int32_t k, int32_t c, int32_t r, int32_t s,
-                                         int32_t kw_pix, cudaStream_t stream) {
+                                         int32_t kw_pix, cudaStream_t stream, int perm) {
   const int64_t total = (int64_t)k * r * kw_pix;
   int64_t blocks = (total + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
   launch_kernel(weights_repack_window_kernel, dim3((unsigned)blocks), dim3(256), 0, stream, 
-      reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), k, c, r, s, kw_pix);
+      reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), k, c, r, s, kw_pix, perm);
   count_launch();
   return cudaGetLastError();
 }
@@ -461,14 +473,14 @@ cudaError_t launch_nhwc_to_nchw(const __half* src, __half* dst, int32_t n, int32
 }
 
 cudaError_t launch_weights_repack(const __half* src, __half* dst, int32_t k, int32_t cg, int32_t r,
-                                  int32_t s, int32_t group, int32_t c_pad, cudaStream_t stream) {
+                                  int32_t s, int32_t group, int32_t c_pad, cudaStream_t stream, int perm) {
   (void)group;  // groups are contiguous blocks of output channels: the permutation is per k
   const int64_t total = (int64_t)k * r * s * (c_pad / 8);
   int64_t blocks = (total + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
   if (blocks < 1) blocks = 1;
   launch_kernel(weights_repack_kernel, dim3((unsigned)blocks), dim3(256), 0, stream, 
-      reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), k, cg, r * s, c_pad);
+      reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), k, cg, r * s, c_pad, perm);
   count_launch();
   return cudaGetLastError();
 }
@@ -502,13 +514,13 @@ cudaError_t launch_patch_im2col(const ConvGeom& g, const __half* src, __half* ds
 }
 
 cudaError_t launch_weights_repack_patch(const __half* src, __half* dst, int32_t k, int32_t c, int32_t r, int32_t s,
-                                        int32_t kelems, cudaStream_t stream) {
+                                        int32_t kelems, cudaStream_t stream, int perm) {
   const int64_t total = (int64_t)k * kelems;
   int64_t blocks = (total + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
   if (blocks < 1) blocks = 1;
   launch_kernel(weights_repack_patch_kernel, dim3((unsigned)blocks), dim3(256), 0, stream, 
-      reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), k, c, r, s, kelems);
+      reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), k, c, r, s, kelems, perm);
   count_launch();
   return cudaGetLastError();
 }
@@ -516,14 +528,14 @@ cudaError_t launch_weights_repack_patch(const __half* src, __half* dst, int32_t 
 // The two preparation steps of the tensor-core path, dispatched on the plan's mode.
 cudaError_t launch_igemm_weights(const ConvGeom& g, const IgemmPlan& p, const __half* w, __half* wp,
                                  cudaStream_t stream) {
-  if (p.patch) return launch_weights_repack_patch(w, wp, g.k, g.c, g.r, g.s, p.cw, stream);
-  if (p.window) return launch_weights_repack_window(w, wp, g.k, g.c, g.r, g.s, p.kw_pix, stream);
-  return launch_weights_repack(w, wp, g.k, g.cg, g.r, g.s, g.group, p.cw, stream);
+  if (p.patch) return launch_weights_repack_patch(w, wp, g.k, g.c, g.r, g.s, p.cw, stream, p.y_perm);
+  if (p.window) return launch_weights_repack_window(w, wp, g.k, g.c, g.r, g.s, p.kw_pix, stream, p.y_perm);
+  return launch_weights_repack(w, wp, g.k, g.cg, g.r, g.s, g.group, p.cw, stream, p.y_perm);
 }
 
 cudaError_t launch_igemm_input(const ConvGeom& g, const IgemmPlan& p, const __half* x, __half* xp,
                                cudaStream_t stream) {
-  if (p.nchw) return cudaSuccess;  // the kernel reads x itself
+  if (p.nchw || p.x_nhwc) return cudaSuccess;  // the kernel reads x itself
   if (p.patch) return launch_patch_im2col(g, x, xp, p.cw, stream);
   if (p.window) return launch_nchw_to_nhwc8_bordered(x, xp, g.n, g.c, g.h, g.w, g.pad_h, g.pad_w, p.hp, p.wp, stream);
   return launch_nchw_to_nhwc(x, xp, g.n, g.c, g.h, g.w, p.c_pad, stream);

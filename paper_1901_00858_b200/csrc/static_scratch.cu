@@ -56,6 +56,7 @@ int make_geom(const hgc_conv_params* p, hgc::ConvGeom* g) {
   g->group = p->group;
   g->p = (int32_t)P; g->q = (int32_t)Q;
   g->cg = p->c / p->group; g->kg = p->k / p->group;
+  g->x_nhwc = 0; g->y_nhwc = 0;  // this entry point takes NCHW tensors only
   return HGC_OK;
 }
 

@@ -127,3 +127,54 @@ def test_launch_overlap_gives_the_same_results(hgc, oracle):
         hgc.set_launch_overlap(False)
     d.close()
     dw.close()
+
+
+NHWC_CASES = [
+    # (id, params, x channels-last, y channels-last)
+    ("3x3 c64 k128 both channels-last", params_dict(2, 64, 20, 24, 128, 3, 3, 1, 1), True, True),
+    ("3x3 c256 k72 odd plane both", params_dict(3, 256, 13, 13, 72, 3, 3, 1, 1), True, True),
+    ("1x1 c128 k200 28x28 both", params_dict(2, 128, 28, 28, 200, 1, 1), True, True),
+    ("1x1 c512 7x7 several images per tile both", params_dict(9, 512, 7, 7, 130, 1, 1), True, True),
+    ("3x3 stride 2 c96 both", params_dict(2, 96, 15, 15, 200, 3, 3, 1, 1, 2, 2), True, True),
+    ("grouped 5x5 both", params_dict(1, 96, 27, 27, 256, 5, 5, 2, 2, 1, 1, 1, 1, 2), True, True),
+    ("stem c3: NCHW in, channels-last out", params_dict(2, 3, 32, 40, 16, 3, 3, 1, 1), False, True),
+    ("last layer: channels-last in, NCHW out", params_dict(2, 64, 16, 16, 40, 3, 3, 1, 1), True, False),
+    ("wide rows 224 channels-last out", params_dict(1, 64, 6, 224, 64, 3, 3, 1, 1), True, True),
+    ("rows of 100: a full and a ragged store per row", params_dict(2, 32, 5, 100, 48, 3, 3, 1, 1), True, True),
+    ("k = 100: channel runs not 16-byte aligned, plain stores", params_dict(2, 64, 14, 14, 100, 3, 3, 1, 1), True, True),
+    ("4 groups of 24 output channels", params_dict(2, 64, 12, 12, 96, 3, 3, 1, 1, 1, 1, 1, 1, 4), True, True),
+    ("1x1 c64 k256 56x56: wide epilogue", params_dict(2, 64, 56, 56, 256, 1, 1), True, True),
+]
+
+
+@pytest.mark.parametrize("name,a,xl,yl", NHWC_CASES, ids=[c[0] for c in NHWC_CASES])
+def test_channels_last_flags(hgc, oracle, name, a, xl, yl):
+    import torch
+    from gpu_util import to_dev, to_host
+    rng = np.random.default_rng(zlib.crc32(name.encode()))
+    x, w, b = workloads.random_layer_tensors(rng, a["n"], a["c"], a["h"], a["w"], a["k"], a["r"], a["s"], a["group"])
+    ref = oracle.conv_fast(oracle.ConvParams(**a), x, w, b, True)          # NCHW
+    flags = (hgc.HGC_FLAG_X_NHWC if xl else 0) | (hgc.HGC_FLAG_Y_NHWC if yl else 0)
+    d = hgc.ConvDesc(flags=flags, **a)
+    assert d.path() == hgc.HGC_PATH_IGEMM
+    n, k, p, q = d.output_dims()
+    d.ensure_workspace()
+    xin = np.ascontiguousarray(x.transpose(0, 2, 3, 1)) if xl else x
+    xd, wd, bd = to_dev(xin), to_dev(w), to_dev(b)
+    yshape = (n, p, q, k) if yl else (n, k, p, q)
+    y = torch.full(yshape, float("nan"), dtype=torch.float16, device="cuda")
+    hgc.conv_forward(d, xd, wd, bd, y, True)
+    torch.cuda.synchronize()
+    assert d.last_device_status() == hgc.HGC_OK
+    got = to_host(y)
+    if yl:
+        got = np.ascontiguousarray(got.transpose(0, 3, 1, 2))
+    check_close(got, ref, what=name)
+    d.close()
+
+
+def test_channels_last_flags_are_refused_where_they_cannot_apply(hgc):
+    with pytest.raises(hgc.HgcError):     # depthwise layers have no channels-last variant
+        hgc.ConvDesc(2, 32, 14, 14, 32, 3, 3, 1, 1, 1, 1, 1, 1, 32, flags=hgc.HGC_FLAG_Y_NHWC)
+    with pytest.raises(hgc.HgcError):     # 3 input channels are not a whole number of 16-byte vectors
+        hgc.ConvDesc(2, 3, 14, 14, 32, 3, 3, 1, 1, flags=hgc.HGC_FLAG_X_NHWC)
