@@ -144,6 +144,13 @@ NHWC_CASES = [
     ("k = 100: channel runs not 16-byte aligned, plain stores", params_dict(2, 64, 14, 14, 100, 3, 3, 1, 1), True, True),
     ("4 groups of 24 output channels", params_dict(2, 64, 12, 12, 96, 3, 3, 1, 1, 1, 1, 1, 1, 4), True, True),
     ("1x1 c64 k256 56x56: wide epilogue", params_dict(2, 64, 56, 56, 256, 1, 1), True, True),
+    ("7x7 planes: nine rows per store, several images per tile", params_dict(9, 512, 7, 7, 128, 1, 1), True, True),
+    ("14x14 planes k256: four rows per store", params_dict(3, 256, 14, 14, 256, 3, 3, 1, 1), True, True),
+    ("28x28 planes k64: two rows per store, ragged last tile", params_dict(2, 128, 28, 28, 64, 3, 3, 1, 1), True, True),
+    ("15x15 odd rows k96: junk pixel slots between rows", params_dict(2, 64, 15, 15, 96, 3, 3, 1, 1), True, True),
+    ("stem c3 k64 windows, channels-last out", params_dict(2, 3, 24, 40, 64, 3, 3, 1, 1), False, True),
+    ("stem 7x7 stride 2 c3 k64 patches, channels-last out", params_dict(2, 3, 38, 38, 64, 7, 7, 3, 3, 2, 2), False, True),
+    ("grouped: 2 groups of 64 output channels", params_dict(2, 64, 12, 20, 128, 3, 3, 1, 1, 1, 1, 1, 1, 2), True, True),
 ]
 
 
@@ -178,3 +185,44 @@ def test_channels_last_flags_are_refused_where_they_cannot_apply(hgc):
         hgc.ConvDesc(2, 32, 14, 14, 32, 3, 3, 1, 1, 1, 1, 1, 1, 32, flags=hgc.HGC_FLAG_Y_NHWC)
     with pytest.raises(hgc.HgcError):     # 3 input channels are not a whole number of 16-byte vectors
         hgc.ConvDesc(2, 3, 14, 14, 32, 3, 3, 1, 1, flags=hgc.HGC_FLAG_X_NHWC)
+
+
+def test_channels_last_chain_with_registered_weights(hgc, oracle):
+    """Four layers that hand their activations on channels-last: NCHW enters the first layer and
+    leaves the last, nothing is converted in between (y of one layer is x of the next).  Weights
+    are registered once per layer.  Compared with the same chain through the oracle, every
+    intermediate rounded to fp16 exactly where the layers do."""
+    import torch
+    from gpu_util import to_dev, to_host
+    rng = np.random.default_rng(77)
+    n = 2
+    chain = [  # (params, flags)
+        (params_dict(n, 3, 30, 36, 32, 3, 3, 1, 1), hgc.HGC_FLAG_Y_NHWC),
+        (params_dict(n, 32, 30, 36, 64, 3, 3, 1, 1), hgc.HGC_FLAG_X_NHWC | hgc.HGC_FLAG_Y_NHWC),
+        (params_dict(n, 64, 30, 36, 64, 1, 1), hgc.HGC_FLAG_X_NHWC | hgc.HGC_FLAG_Y_NHWC),
+        (params_dict(n, 64, 30, 36, 40, 3, 3, 1, 1, 2, 2), hgc.HGC_FLAG_X_NHWC),
+    ]
+    x0 = rng.uniform(0.0, 1.0, (n, 3, 30, 36)).astype(np.float16)
+    ref = x0
+    cur = to_dev(x0)
+    keep = []
+    for a, fl in chain:
+        _, w, b = workloads.random_layer_tensors(rng, a["n"], a["c"], a["h"], a["w"], a["k"], a["r"], a["s"], a["group"])
+        ref = oracle.conv_fast(oracle.ConvParams(**a), ref, w, b, True)
+        d = hgc.ConvDesc(flags=fl, **a)
+        assert d.path() == hgc.HGC_PATH_IGEMM
+        d.ensure_workspace()
+        wd, bd = to_dev(w), to_dev(b)
+        d.set_weights(wd)
+        nn, k, p, q = d.output_dims()
+        shape = (nn, p, q, k) if fl & hgc.HGC_FLAG_Y_NHWC else (nn, k, p, q)
+        y = torch.full(shape, float("nan"), dtype=torch.float16, device="cuda")
+        hgc.conv_forward(d, cur, wd, bd, y, True)
+        keep.append((d, wd, bd, cur))
+        cur = y
+    torch.cuda.synchronize()
+    for d, *_ in keep:
+        assert d.last_device_status() == hgc.HGC_OK
+    check_close(to_host(cur), ref, what="channels-last chain")
+    for d, *_ in keep:
+        d.close()
