@@ -2,6 +2,8 @@
 tests/, by the smoke check and by the bench's CPU-baseline leg, never by the product."""
 from .conv_oracle import (  # noqa: F401
     ConvParams,
+    batchnorm,
+    bn_fold,
     build,
     cast_f32_to_f16,
     conv_fast,

@@ -86,6 +86,13 @@ def _load():
         lib.ref_inner_product.restype = None
         lib.ref_inner_product.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, u16p, u16p, u16p, u16p,
                                           ctypes.c_int]
+        f64p = ctypes.POINTER(ctypes.c_double)
+        lib.ref_batchnorm.restype = None
+        lib.ref_batchnorm.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, u16p, ctypes.c_double,
+                                      ctypes.c_int, f64p, f64p, u16p]
+        lib.ref_bn_fold.restype = None
+        lib.ref_bn_fold.argtypes = [ctypes.c_int64, ctypes.c_int64, u16p, u16p, f64p, f64p, f64p, f64p,
+                                    ctypes.c_double, u16p, u16p]
         _lib = lib
     return _lib
 
@@ -196,6 +203,52 @@ def inner_product(x, w, bias=None, relu=False) -> np.ndarray:
     y = np.empty((n, k), dtype=np.uint16)
     lib.ref_inner_product(n, c, k, _u16(xb), _u16(wb), None if bb is None else _u16(bb), _u16(y), int(bool(relu)))
     return y.view(np.float16)
+
+
+def _f64(a):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_double))
+
+
+def batchnorm(x, eps, mean=None, var=None):
+    """Batch norm of x [N,C,H,W] (float16), Section 3.1: per channel over N*H*W,
+    y = (x - mean) / sqrt(var + eps) with the biased variance.  mean/var None: computed from x;
+    else the stored statistics (float64 [C]).  Returns (y float16, mean float64, var float64)."""
+    lib = _load()
+    xb = _bits(x)
+    n, c = xb.shape[0], xb.shape[1]
+    hw = int(np.prod(xb.shape[2:], dtype=np.int64))
+    stored = mean is not None
+    if stored != (var is not None):
+        raise ValueError("give both mean and var, or neither")
+    m = np.ascontiguousarray(mean, dtype=np.float64).copy() if stored else np.zeros(c, dtype=np.float64)
+    v = np.ascontiguousarray(var, dtype=np.float64).copy() if stored else np.zeros(c, dtype=np.float64)
+    if m.shape != (c,) or v.shape != (c,):
+        raise ValueError("mean and var have one entry per channel")
+    y = np.empty(xb.shape, dtype=np.uint16)
+    lib.ref_batchnorm(n, c, hw, _u16(xb), float(eps), int(stored), _f64(m), _f64(v), _u16(y))
+    return y.view(np.float16), m, v
+
+
+def bn_fold(w, bias, mean, var, eps, gamma=None, beta=None):
+    """Stored statistics (and an optional per-channel scale gamma / shift beta) folded into the
+    convolution before the batch norm: returns (w' float16 like w, b' float16 [K])."""
+    lib = _load()
+    wb = _bits(w)
+    k = wb.shape[0]
+    per_k = int(np.prod(wb.shape[1:], dtype=np.int64))
+    bb = None if bias is None else _bits(bias, (k,))
+    m = np.ascontiguousarray(mean, dtype=np.float64)
+    v = np.ascontiguousarray(var, dtype=np.float64)
+    ga = None if gamma is None else np.ascontiguousarray(gamma, dtype=np.float64)
+    be = None if beta is None else np.ascontiguousarray(beta, dtype=np.float64)
+    for a in (m, v, ga, be):
+        if a is not None and a.shape != (k,):
+            raise ValueError("per-channel vectors have K entries")
+    wo = np.empty(wb.shape, dtype=np.uint16)
+    bo = np.empty(k, dtype=np.uint16)
+    lib.ref_bn_fold(k, per_k, _u16(wb), None if bb is None else _u16(bb), _f64(m), _f64(v),
+                    None if ga is None else _f64(ga), None if be is None else _f64(be), float(eps), _u16(wo), _u16(bo))
+    return wo.view(np.float16), bo.view(np.float16)
 
 
 def nchw_to_nhwc(x: np.ndarray, c_pad: int) -> np.ndarray:

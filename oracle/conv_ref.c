@@ -37,6 +37,14 @@
  *   ref_inner_product  the inner-product (fully connected) layer, named in Section 3.1 as
  *                    the other layer whose long sums overflow FP16:
  *                    y[n,k] = round( relu?( bias[k] + sum_c x[n,c] * w[k,c] ) ), fp64 sum
+ *   ref_batchnorm    the batch-norm layer of Section 3.1 as its plain definition: per channel
+ *                    over the N*H*W values, mean = sum x / M, var = sum (x - mean)^2 / M (the
+ *                    biased variance), y = round( (x - mean) / sqrt(var + eps) ), all in fp64
+ *                    (the grouped mean and the shift before squaring that the section describes
+ *                    are ways of reaching these same numbers in narrow arithmetic); with stored
+ *                    statistics the mean and variance are inputs
+ *   ref_bn_fold      stored statistics and an optional per-channel scale and shift folded into
+ *                    the weights and bias of the convolution before the batch norm
  *
  * Parity pins: every function here is pinned by the CPU tests (hand-worked
  * examples, closed forms, matmul / correlate2d restatements, invariants).
@@ -284,6 +292,53 @@ void ref_inner_product(int64_t n, int64_t c, int64_t k, const uint16_t* x, const
         acc += ref_half_to_double(x[in * c + ic]) * ref_half_to_double(w[ik * c + ic]);
       y[in * k + ik] = finish(acc, relu);
     }
+  }
+}
+
+/* ---- batch norm (Section 3.1) -------------------------------------------- */
+
+/* x[N][C][HW] -> y of the same shape.  use_stored == 0: mean[c] and var[c] are computed from x
+   and written; otherwise they are read.  No scale or shift (Caffe keeps those in a separate
+   layer). */
+void ref_batchnorm(int64_t n, int64_t c, int64_t hw, const uint16_t* x, double eps, int use_stored,
+                   double* mean, double* var, uint16_t* y) {
+  const double m = (double)(n * hw);
+  for (int64_t ic = 0; ic < c; ++ic) {
+    if (!use_stored) {
+      double sum = 0.0;
+      for (int64_t in = 0; in < n; ++in)
+        for (int64_t i = 0; i < hw; ++i) sum += ref_half_to_double(x[(in * c + ic) * hw + i]);
+      mean[ic] = sum / m;
+      double sq = 0.0;
+      for (int64_t in = 0; in < n; ++in)
+        for (int64_t i = 0; i < hw; ++i) {
+          const double d = ref_half_to_double(x[(in * c + ic) * hw + i]) - mean[ic];
+          sq += d * d;
+        }
+      var[ic] = sq / m;
+    }
+    const double inv = 1.0 / sqrt(var[ic] + eps);
+    for (int64_t in = 0; in < n; ++in)
+      for (int64_t i = 0; i < hw; ++i) {
+        const int64_t at = (in * c + ic) * hw + i;
+        y[at] = ref_double_to_half((ref_half_to_double(x[at]) - mean[ic]) * inv);
+      }
+  }
+}
+
+/* a_k = gamma_k / sqrt(var_k + eps) (gamma = 1 if NULL); w'[k][j] = round(w[k][j] * a_k);
+   b'[k] = round((b[k] - mean_k) * a_k + beta_k) (b = 0 if bias is NULL, beta = 0 if NULL):
+   conv(x, w') + b' equals gamma * (conv(x, w) + b - mean) / sqrt(var + eps) + beta up to the
+   rounding of w' and b'. */
+void ref_bn_fold(int64_t k, int64_t per_k, const uint16_t* w, const uint16_t* bias, const double* mean,
+                 const double* var, const double* gamma, const double* beta, double eps, uint16_t* w_out,
+                 uint16_t* b_out) {
+  for (int64_t ik = 0; ik < k; ++ik) {
+    const double a = (gamma ? gamma[ik] : 1.0) / sqrt(var[ik] + eps);
+    for (int64_t j = 0; j < per_k; ++j)
+      w_out[ik * per_k + j] = ref_double_to_half(ref_half_to_double(w[ik * per_k + j]) * a);
+    const double b = bias ? ref_half_to_double(bias[ik]) : 0.0;
+    b_out[ik] = ref_double_to_half((b - mean[ik]) * a + (beta ? beta[ik] : 0.0));
   }
 }
 

@@ -393,3 +393,111 @@ def test_wide_accumulation_in_the_inner_product(oracle):
     x = np.ones((1, 4096), dtype=F16)
     w = np.ones((2, 4096), dtype=F16)
     assert np.array_equal(oracle.inner_product(x, w, None, False), np.full((1, 2), 4096, dtype=F16))
+
+
+# ---- batch norm (Section 3.1) ------------------------------------------------------------------
+
+def test_batchnorm_hand_examples(oracle):
+    """{1,2,3,4}: mean 5/2, variance 5/4, outputs -+3/sqrt(5) and -+1/sqrt(5).  Two images of one
+    pixel {0, 2}: mean 1, variance 1, outputs -1 and 1 (the statistics run over images too)."""
+    y, m, v = oracle.batchnorm(np.array([[[[1, 2], [3, 4]]]], dtype=F16), 0.0)
+    assert m[0] == 2.5 and v[0] == 1.25
+    want = np.array([-3, -1, 1, 3], dtype=np.float64) / np.sqrt(5.0)
+    assert np.array_equal(y.ravel(), want.astype(F16))
+    y, m, v = oracle.batchnorm(np.array([[[[0]]], [[[2]]]], dtype=F16), 0.0)
+    assert (m[0], v[0]) == (1.0, 1.0) and y.ravel().tolist() == [-1.0, 1.0]
+    # eps enters under the root: {0, 2} with eps = 3 gives -+1/2
+    y, _, _ = oracle.batchnorm(np.array([[[[0]]], [[[2]]]], dtype=F16), 3.0)
+    assert y.ravel().tolist() == [-0.5, 0.5]
+
+
+def test_batchnorm_matches_float64_numpy_per_channel(oracle):
+    rng = np.random.default_rng(11)
+    x = (rng.normal(0, 1, size=(3, 5, 7, 6)) * np.array([1, 4, 0.25, 10, 1]).reshape(1, 5, 1, 1)
+         + np.array([0, 3, -1, 20, 0.5]).reshape(1, 5, 1, 1)).astype(F16)
+    eps = 1e-5
+    y, m, v = oracle.batchnorm(x, eps)
+    xd = x.astype(np.float64)
+    mean = xd.mean(axis=(0, 2, 3))
+    var = xd.var(axis=(0, 2, 3))          # biased, like the layer
+    assert np.allclose(m, mean, rtol=1e-13, atol=1e-15) and np.allclose(v, var, rtol=1e-12, atol=0)
+    want = (xd - mean.reshape(1, 5, 1, 1)) / np.sqrt(var.reshape(1, 5, 1, 1) + eps)
+    # both are fp64 before the one rounding; different summation orders can flip a rare tie
+    err = np.abs(y.astype(np.float64) - want)
+    assert np.all(err <= np.abs(want) * 2.0 ** -11 + 2.0 ** -25)
+    assert np.mean(y.view(np.uint16) == want.astype(F16).view(np.uint16)) > 0.999
+
+
+def test_batchnorm_output_has_zero_mean_and_unit_variance(oracle):
+    rng = np.random.default_rng(12)
+    x = rng.uniform(0, 255, size=(4, 3, 16, 16)).astype(F16)
+    y, _, _ = oracle.batchnorm(x, 0.0)
+    yd = y.astype(np.float64)
+    assert np.all(np.abs(yd.mean(axis=(0, 2, 3))) < 2e-4)
+    assert np.all(np.abs(yd.var(axis=(0, 2, 3)) - 1.0) < 2e-3)
+
+
+def test_batchnorm_ignores_exact_shifts_and_positive_scales(oracle):
+    """x + 16 and 4 * x are exact in fp16 for multiples of 1/64 in [0, 8): the normalised output
+    has the same bits (eps = 0)."""
+    rng = np.random.default_rng(13)
+    x = (rng.integers(0, 512, size=(2, 4, 9, 5)) / 64.0).astype(F16)
+    base, _, _ = oracle.batchnorm(x, 0.0)
+    shifted, ms, _ = oracle.batchnorm((x.astype(np.float64) + 16.0).astype(F16), 0.0)
+    scaled, _, vs = oracle.batchnorm((x.astype(np.float64) * 4.0).astype(F16), 0.0)
+    assert np.array_equal(base.view(np.uint16), shifted.view(np.uint16))
+    assert np.array_equal(base.view(np.uint16), scaled.view(np.uint16))
+    # a negative scale mirrors the output
+    neg, _, _ = oracle.batchnorm((-x.astype(np.float64)).astype(F16), 0.0)
+    assert np.array_equal((-base).view(np.uint16), neg.view(np.uint16))
+
+
+def test_batchnorm_image_valued_data_does_not_overflow(oracle):
+    """The case the section names: pixel values 0..255, many of them.  Every value 0..255 equally
+    often: mean 255/2, variance (256^2 - 1)/12.  (A sum, or a square, carried in FP16 would have
+    left the finite range after a few hundred values.)"""
+    x = np.tile(np.arange(256, dtype=np.float64), 64).reshape(4, 1, 64, 64).astype(F16)
+    y, m, v = oracle.batchnorm(x, 0.0)
+    assert m[0] == 127.5 and v[0] == (256.0 ** 2 - 1.0) / 12.0
+    assert np.all(np.isfinite(y.astype(np.float64)))
+    assert y.ravel()[0] == F16(-127.5 / np.sqrt(v[0])) and y.ravel()[255] == F16(127.5 / np.sqrt(v[0]))
+
+
+def test_batchnorm_with_stored_statistics(oracle):
+    rng = np.random.default_rng(14)
+    x = rng.normal(2, 3, size=(2, 6, 5, 5)).astype(F16)
+    y0, m, v = oracle.batchnorm(x, 1e-3)
+    y1, m1, v1 = oracle.batchnorm(x, 1e-3, m, v)          # its own statistics handed back in
+    assert np.array_equal(y0.view(np.uint16), y1.view(np.uint16)) and np.array_equal(m, m1) and np.array_equal(v, v1)
+    mean = rng.normal(0, 1, 6)
+    var = rng.uniform(0.5, 2, 6)
+    y2, _, _ = oracle.batchnorm(x, 1e-3, mean, var)
+    want = (x.astype(np.float64) - mean.reshape(1, 6, 1, 1)) / np.sqrt(var.reshape(1, 6, 1, 1) + 1e-3)
+    assert np.array_equal(y2.view(np.uint16), want.astype(F16).view(np.uint16))
+
+
+def test_bn_fold_restates_the_formula_and_commutes_with_a_1x1_convolution(oracle):
+    rng = np.random.default_rng(15)
+    k, c = 7, 24
+    w = rng.normal(0, 0.2, size=(k, c, 1, 1)).astype(F16)
+    b = rng.uniform(-0.5, 0.5, size=k).astype(F16)
+    mean, var = rng.normal(0, 1, k), rng.uniform(0.25, 4, k)
+    gamma, beta = rng.uniform(0.5, 2, k), rng.normal(0, 1, k)
+    eps = 1e-5
+    wf, bf = oracle.bn_fold(w, b, mean, var, eps, gamma, beta)
+    a = gamma / np.sqrt(var + eps)
+    assert np.array_equal(wf.view(np.uint16), (w.astype(np.float64) * a.reshape(k, 1, 1, 1)).astype(F16).view(np.uint16))
+    assert np.array_equal(bf.view(np.uint16), ((b.astype(np.float64) - mean) * a + beta).astype(F16).view(np.uint16))
+    # defaults: gamma = 1, beta = 0, no bias
+    wf1, bf1 = oracle.bn_fold(w, None, mean, var, eps)
+    a1 = 1.0 / np.sqrt(var + eps)
+    assert np.array_equal(wf1.view(np.uint16), (w.astype(np.float64) * a1.reshape(k, 1, 1, 1)).astype(F16).view(np.uint16))
+    assert np.array_equal(bf1.view(np.uint16), (-mean * a1).astype(F16).view(np.uint16))
+    # the folded layer computes what conv -> batch norm (stored statistics) -> scale/shift computes
+    x = rng.uniform(-1, 1, size=(3, c, 4, 4)).astype(F16)
+    P = oracle.ConvParams(3, c, 4, 4, k, 1, 1, 0, 0, 1, 1, 1, 1, 1)
+    folded = oracle.conv_naive(P, x, wf, bf, False).astype(np.float64)
+    conv = np.einsum("nchw,kc->nkhw", x.astype(np.float64), w.astype(np.float64).reshape(k, c)) + \
+        b.astype(np.float64).reshape(1, k, 1, 1)
+    want = (conv - mean.reshape(1, k, 1, 1)) * a.reshape(1, k, 1, 1) + beta.reshape(1, k, 1, 1)
+    assert np.all(np.abs(folded - want) <= 2e-3 + 1e-2 * np.abs(want))
