@@ -238,6 +238,47 @@ int hgc_inner_product_desc_create(hgc_conv_desc** out, int32_t n, int32_t c, int
 int hgc_cast_f32_to_f16(const void* src, void* dst, int64_t count, uint64_t* overflow_count, void* stream);
 
 /*
+ * Batch norm forward (Section 3.1), x and y [n][c][hw] dense FP16 (hw = H*W):
+ *     y = (x - mean_c) / sqrt(var_c + eps),   one rounding to FP16,
+ * mean_c and var_c (the biased variance) taken per channel over its n*hw values.  The statistics
+ * are computed the way the section describes: the values of a channel are partitioned into groups
+ * (one image, at most 2048 consecutive pixels), the mean of each group is taken, then the mean
+ * of the group means weighted by the group sizes; the centred values are multiplied by
+ * 2^shift_log2 before they are squared (the section's 1/32 for large data is -5, its 32 for
+ * small data is 5, 0 is no shift) and the variance is shifted back.  All sums are FP32, so the
+ * result does not depend on shift_log2 (|shift_log2| <= 8).
+ * use_stored == 0: mean and var (device, `c` floats each) are WRITTEN; `workspace` must hold
+ * hgc_batchnorm_workspace_bytes(n, c, hw) bytes of device memory (16-byte aligned; contents
+ * irrelevant before, undefined after).  use_stored != 0: mean and var are READ (stored
+ * statistics, e.g. a trained model's), workspace may be NULL.  No scale/shift parameters: Caffe
+ * keeps them in a separate layer (see hgc_bn_fold for inference).
+ * x, y: device pointers, 16-byte aligned, not overlapping.  Queued on `stream` (three kernels, or
+ * one with stored statistics); nothing is allocated, nothing synchronises.
+ * Errors: HGC_INVALID_ARG (NULL pointers, n/c/hw < 1, eps < 0, shift out of range),
+ * HGC_UNSUPPORTED (c > 65535 or more than 2^31-1 groups), HGC_BAD_ALIGNMENT, HGC_NO_WORKSPACE
+ * (workspace NULL when statistics are to be computed), HGC_CUDA_ERROR.
+ */
+size_t hgc_batchnorm_workspace_bytes(int32_t n, int32_t c, int64_t hw);
+int hgc_batchnorm_forward(const void* x, void* y, int32_t n, int32_t c, int64_t hw, float eps, int32_t shift_log2,
+                          int32_t use_stored, float* mean, float* var, void* workspace, void* stream);
+
+/*
+ * Inference-time folding of a batch norm with stored statistics (and an optional per-channel
+ * scale gamma and shift beta) into the convolution in front of it:
+ *     a_k = gamma_k / sqrt(var_k + eps),  w_out[k][j] = w[k][j] * a_k,
+ *     b_out[k] = (bias[k] - mean_k) * a_k + beta_k,
+ * computed in FP32, rounded once to FP16.  conv(x, w_out) + b_out then equals
+ * gamma * (conv(x, w) + bias - mean) / sqrt(var + eps) + beta up to the rounding of w_out and
+ * b_out, so the normalisation costs nothing at run time (it rides in the conv epilogue's bias).
+ * w, w_out: [k][per_k] FP16 (per_k = (C/group)*R*S); bias: [k] FP16 or NULL (zeros); mean, var:
+ * [k] floats; gamma, beta: [k] floats or NULL (ones / zeros); b_out: [k] FP16.  Device pointers;
+ * w_out may equal w.  Errors: HGC_INVALID_ARG (NULL required pointer, k or per_k < 1, eps < 0),
+ * HGC_CUDA_ERROR.
+ */
+int hgc_bn_fold(const void* w, const void* bias, const float* mean, const float* var, const float* gamma,
+                const float* beta, float eps, int32_t k, int64_t per_k, void* w_out, void* b_out, void* stream);
+
+/*
  * Launch overlap (off by default).  With enabled != 0 the library launches its kernels with the
  * programmatic stream serialization attribute: a kernel may be scheduled while the previous
  * kernel of the stream is still draining, and waits, before it touches global memory, until that

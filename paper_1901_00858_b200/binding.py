@@ -55,6 +55,10 @@ def lib() -> ctypes.CDLL:
         L.hgc_conv_forward_static.argtypes = [ctypes.POINTER(hgc_conv_params), vp, vp, vp, vp, ctypes.c_int, vp]
         L.hgc_inner_product_desc_create.argtypes = [ctypes.POINTER(ctypes.c_void_p), i32, i32, i32]
         L.hgc_cast_f32_to_f16.argtypes = [vp, vp, ctypes.c_int64, vp, vp]
+        L.hgc_batchnorm_workspace_bytes.argtypes = [i32, i32, ctypes.c_int64]
+        L.hgc_batchnorm_workspace_bytes.restype = ctypes.c_size_t
+        L.hgc_batchnorm_forward.argtypes = [vp, vp, i32, i32, ctypes.c_int64, ctypes.c_float, i32, i32, vp, vp, vp, vp]
+        L.hgc_bn_fold.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, i32, ctypes.c_int64, vp, vp, vp]
         L.hgc_conv_output_dims.argtypes = [vp, i32p, i32p, i32p, i32p]
         L.hgc_conv_path.argtypes = [vp, i32p]
         L.hgc_conv_plan_info.argtypes = [vp, i32p, i32]
@@ -76,7 +80,7 @@ def lib() -> ctypes.CDLL:
                      "hgc_conv_set_workspace", "hgc_conv_set_weights", "hgc_conv_last_device_status",
                      "hgc_layout_nchw_to_nhwc", "hgc_layout_nhwc_to_nchw", "hgc_weights_repack",
                      "hgc_kernel_launch_count", "hgc_inner_product_desc_create", "hgc_cast_f32_to_f16",
-                     "hgc_set_launch_overlap"):
+                     "hgc_set_launch_overlap", "hgc_batchnorm_forward", "hgc_bn_fold"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -231,6 +235,30 @@ def cast_f32_to_f16(src, dst, count=None, overflow_count=None, stream=None):
     n = src.numel() if count is None else count
     _check(lib().hgc_cast_f32_to_f16(_ptr(src), _ptr(dst), n, _ptr(overflow_count), _stream(stream)),
            "hgc_cast_f32_to_f16")
+
+
+def batchnorm_workspace_bytes(n: int, c: int, hw: int) -> int:
+    return int(lib().hgc_batchnorm_workspace_bytes(n, c, hw))
+
+
+def batchnorm_forward(x, y, eps, mean, var, workspace=None, shift_log2=0, use_stored=False, stream=None):
+    """hgc_batchnorm_forward: x, y [N,C,...] float16 CUDA tensors; mean, var float32 [C] CUDA
+    tensors (written, or read with use_stored); workspace: a CUDA tensor of at least
+    batchnorm_workspace_bytes(...) bytes (not needed with use_stored)."""
+    n, c = int(x.shape[0]), int(x.shape[1])
+    hw = x.numel() // (n * c)
+    _check(lib().hgc_batchnorm_forward(_ptr(x), _ptr(y), n, c, hw, float(eps), int(shift_log2), int(bool(use_stored)),
+                                       _ptr(mean), _ptr(var), _ptr(workspace), _stream(stream)),
+           "hgc_batchnorm_forward")
+
+
+def bn_fold(w, bias, mean, var, eps, w_out, b_out, gamma=None, beta=None, stream=None):
+    """hgc_bn_fold: stored statistics (float32 [K]) and optional gamma/beta folded into conv
+    weights w [K,...] and bias [K] (or None); results in w_out, b_out (float16)."""
+    k = int(w.shape[0])
+    per_k = w.numel() // k
+    _check(lib().hgc_bn_fold(_ptr(w), _ptr(bias), _ptr(mean), _ptr(var), _ptr(gamma), _ptr(beta), float(eps), k,
+                             per_k, _ptr(w_out), _ptr(b_out), _stream(stream)), "hgc_bn_fold")
 
 
 def layout_nchw_to_nhwc(src, dst, n, c, h, w, c_pad, stream=None):

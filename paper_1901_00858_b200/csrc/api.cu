@@ -332,6 +332,37 @@ int hgc_cast_f32_to_f16(const void* src, void* dst, int64_t count, uint64_t* ove
   return err == cudaSuccess ? HGC_OK : HGC_CUDA_ERROR;
 }
 
+size_t hgc_batchnorm_workspace_bytes(int32_t n, int32_t c, int64_t hw) {
+  if (n < 1 || c < 1 || hw < 1) return 0;
+  return hgc::batchnorm_workspace_bytes(n, c, hw);
+}
+
+int hgc_batchnorm_forward(const void* x, void* y, int32_t n, int32_t c, int64_t hw, float eps, int32_t shift_log2,
+                          int32_t use_stored, float* mean, float* var, void* workspace, void* stream) {
+  if (x == nullptr || y == nullptr || mean == nullptr || var == nullptr) return HGC_INVALID_ARG;
+  if (n < 1 || c < 1 || hw < 1 || !(eps >= 0.f) || shift_log2 < -8 || shift_log2 > 8) return HGC_INVALID_ARG;
+  const int64_t chunks = (hw + 2047) / 2048;
+  if (c > 65535 || (int64_t)n * chunks > 0x7fffffffLL) return HGC_UNSUPPORTED;
+  if (misaligned(x) || misaligned(y) || (workspace != nullptr && misaligned(workspace))) return HGC_BAD_ALIGNMENT;
+  if ((reinterpret_cast<uintptr_t>(mean) & 3u) != 0 || (reinterpret_cast<uintptr_t>(var) & 3u) != 0)
+    return HGC_BAD_ALIGNMENT;
+  if (!use_stored && workspace == nullptr) return HGC_NO_WORKSPACE;
+  const cudaError_t err =
+      hgc::launch_batchnorm(static_cast<const __half*>(x), static_cast<__half*>(y), n, c, hw, eps, shift_log2,
+                            use_stored != 0, mean, var, workspace, static_cast<cudaStream_t>(stream));
+  return err == cudaSuccess ? HGC_OK : HGC_CUDA_ERROR;
+}
+
+int hgc_bn_fold(const void* w, const void* bias, const float* mean, const float* var, const float* gamma,
+                const float* beta, float eps, int32_t k, int64_t per_k, void* w_out, void* b_out, void* stream) {
+  if (w == nullptr || mean == nullptr || var == nullptr || w_out == nullptr || b_out == nullptr) return HGC_INVALID_ARG;
+  if (k < 1 || per_k < 1 || !(eps >= 0.f)) return HGC_INVALID_ARG;
+  const cudaError_t err = hgc::launch_bn_fold(static_cast<const __half*>(w), static_cast<const __half*>(bias), mean,
+                                              var, gamma, beta, eps, k, per_k, static_cast<__half*>(w_out),
+                                              static_cast<__half*>(b_out), static_cast<cudaStream_t>(stream));
+  return err == cudaSuccess ? HGC_OK : HGC_CUDA_ERROR;
+}
+
 int hgc_set_launch_overlap(int enabled) {
   hgc::set_launch_overlap(enabled != 0);
   return HGC_OK;

@@ -84,6 +84,14 @@ cudaError_t launch_weights_repack(const __half* src, __half* dst, int32_t k, int
 cudaError_t launch_cast_f32_to_f16(const float* src, __half* dst, int64_t count, unsigned long long* overflow,
                                    cudaStream_t stream);
 
+size_t batchnorm_workspace_bytes(int32_t n, int32_t c, int64_t hw);
+cudaError_t launch_batchnorm(const __half* x, __half* y, int32_t n, int32_t c, int64_t hw, float eps,
+                             int32_t shift_log2, int32_t use_stored, float* mean, float* var, void* ws,
+                             cudaStream_t stream);
+cudaError_t launch_bn_fold(const __half* w, const __half* bias, const float* mean, const float* var,
+                           const float* gamma, const float* beta, float eps, int32_t k, int64_t per_k, __half* w_out,
+                           __half* b_out, cudaStream_t stream);
+
 // Plan of the tcgen05 implicit-GEMM path for one layer (host side).
 struct IgemmPlan {
   int32_t kb, cblocks, cw, c_pad;

@@ -143,3 +143,30 @@ def test_plan_info_reports_tiling_and_activation_source():
 
 def test_launch_counter_readable():
     assert hgc.kernel_launch_count() >= 0
+
+
+def test_batchnorm_entry_points_validate_their_arguments():
+    """No launch: every call below must be refused on the host."""
+    import ctypes
+    L = hgc.lib()
+    ok_ptr = ctypes.c_void_p(0x10000)           # never dereferenced: the calls fail before any launch
+    f = ctypes.c_void_p(0x20000)
+    assert hgc.batchnorm_workspace_bytes(16, 64, 224 * 224) == 2 * 64 * 16 * 25 * 4   # 25 groups of <= 2048 per plane
+    assert hgc.batchnorm_workspace_bytes(2, 3, 2048) == 2 * 3 * 2 * 1 * 4
+    assert hgc.batchnorm_workspace_bytes(0, 3, 10) == 0
+    bad = [
+        (None, ok_ptr, 1, 1, 10, 0.0, 0, 0, f, f, ok_ptr, hgc.HGC_INVALID_ARG),      # x NULL
+        (ok_ptr, ok_ptr, 0, 1, 10, 0.0, 0, 0, f, f, ok_ptr, hgc.HGC_INVALID_ARG),    # n < 1
+        (ok_ptr, ok_ptr, 1, 1, 0, 0.0, 0, 0, f, f, ok_ptr, hgc.HGC_INVALID_ARG),     # hw < 1
+        (ok_ptr, ok_ptr, 1, 1, 10, -1.0, 0, 0, f, f, ok_ptr, hgc.HGC_INVALID_ARG),   # eps < 0
+        (ok_ptr, ok_ptr, 1, 1, 10, 0.0, 9, 0, f, f, ok_ptr, hgc.HGC_INVALID_ARG),    # shift out of range
+        (ok_ptr, ok_ptr, 1, 1, 10, 0.0, 0, 0, None, f, ok_ptr, hgc.HGC_INVALID_ARG),  # mean NULL
+        (ok_ptr, ok_ptr, 1, 70000, 10, 0.0, 0, 0, f, f, ok_ptr, hgc.HGC_UNSUPPORTED),  # too many channels
+        (ctypes.c_void_p(0x10002), ok_ptr, 1, 1, 10, 0.0, 0, 0, f, f, ok_ptr, hgc.HGC_BAD_ALIGNMENT),
+        (ok_ptr, ok_ptr, 1, 1, 10, 0.0, 0, 0, f, f, None, hgc.HGC_NO_WORKSPACE),     # statistics need scratch
+    ]
+    for *args, want in bad:
+        assert L.hgc_batchnorm_forward(*args, None) == want, args
+    assert L.hgc_bn_fold(None, None, f, f, None, None, 0.0, 4, 9, ok_ptr, ok_ptr, None) == hgc.HGC_INVALID_ARG
+    assert L.hgc_bn_fold(ok_ptr, None, f, f, None, None, 0.0, 0, 9, ok_ptr, ok_ptr, None) == hgc.HGC_INVALID_ARG
+    assert L.hgc_bn_fold(ok_ptr, None, f, f, None, None, -1.0, 4, 9, ok_ptr, ok_ptr, None) == hgc.HGC_INVALID_ARG
