@@ -509,6 +509,8 @@ def run_ours(args, wl):
 
 def run_side_op(args):
     """--op cast: FP32 -> FP16 cast of 64 Mi values (HBM bound, 6 bytes per element).
+    --op bn: batch norm with batch statistics on two VGG-16 activation tensors (HBM bound, 8 bytes
+    per element: three reads of x, one write of y).
     --op fc: the three inner-product layers of a VGG-16 classifier at batch 64 (25088->4096,
     4096->4096, 4096->1000; weight-streaming, HBM bound).  One JSON line each, same keys."""
     import torch
@@ -532,6 +534,30 @@ def run_side_op(args):
         sample = np.random.default_rng(0).normal(0, 1, 16 << 20).astype(np.float32)
         t0 = time.perf_counter(); oracle.cast_f32_to_f16(sample); dt = time.perf_counter() - t0
         cpu = {"value": 6.0 * sample.size / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+               "sample": f"{sample.size} values once ({dt:.2f} s)"}
+    elif args.op == "bn":
+        # the output of VGG-16's first block at batch 16 (16 x 64 x 224 x 224, 103 MB) and of its
+        # second (16 x 128 x 112 x 112, 51 MB), alternating: 308 MB touched per pair, larger than L2
+        shapes_bn = [(16, 64, 224, 224), (16, 128, 112, 112)]
+        bufs = []
+        for shp in shapes_bn:
+            n_, c_ = shp[0], shp[1]
+            hw_ = shp[2] * shp[3]
+            x = (torch.rand(shp, device="cuda") * 255.0).to(torch.float16)
+            y = torch.empty_like(x)
+            mean = torch.empty(c_, dtype=torch.float32, device="cuda")
+            var = torch.empty(c_, dtype=torch.float32, device="cuda")
+            ws = torch.empty(hgc.batchnorm_workspace_bytes(n_, c_, hw_), dtype=torch.uint8, device="cuda")
+            bufs.append((x, y, mean, var, ws))
+        def step(i):
+            for x, y, mean, var, ws in bufs:
+                hgc.batchnorm_forward(x, y, 1e-5, mean, var, ws, shift_log2=-5, stream=stream)
+        elems = sum(b[0].numel() for b in bufs)
+        step_bytes, step_flops = 8.0 * elems, 0.0   # x read three times, y written once
+        metric, unit, workload = "batchnorm_gbs", "GB/s", "vgg16_block1_block2_n16"
+        sample = (np.random.default_rng(0).integers(0, 256, (8, 64, 224, 224))).astype(np.float16)
+        t0 = time.perf_counter(); oracle.batchnorm(sample, 1e-5); dt = time.perf_counter() - t0
+        cpu = {"value": 8.0 * sample.size / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
                "sample": f"{sample.size} values once ({dt:.2f} s)"}
     else:
         n = 64
@@ -575,12 +601,13 @@ def run_side_op(args):
     host_t1 = time.time()
     ms = e0.elapsed_time(e1) / steps
     gbs = step_bytes / (ms * 1e-3) / 1e9
-    value = gbs if args.op == "cast" else step_flops / (ms * 1e-3) / 1e12
+    value = gbs if args.op in ("cast", "bn") else step_flops / (ms * 1e-3) / 1e12
     line = {"metric": metric, "value": value, "unit": unit, "n_gpus": 1, "steps": steps, "warmup": warm,
             "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32 -> f16" if args.op == "cast" else "f16 (f32 accumulate)", "data": "synthetic",
             "config": {"workload": workload, "l2": "buffers rotate over a footprint larger than L2" if args.op == "cast"
-                       else "weights (278 MB) larger than L2", "launch": "eager"},
+                       else ("two tensors alternate, 308 MB touched per step" if args.op == "bn"
+                             else "weights (278 MB) larger than L2"), "launch": "eager"},
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]},
             "cpu_baseline": cpu, "gpu_launches": hgc.kernel_launch_count() - c0,
@@ -596,9 +623,9 @@ def main():
     ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--op", choices=["conv", "cast", "fc"], default="conv",
-                    help="conv: the convolution path (default); cast / fc: the FP32->FP16 cast and the "
-                         "inner-product layer, measured on their own")
+    ap.add_argument("--op", choices=["conv", "cast", "fc", "bn"], default="conv",
+                    help="conv: the convolution path (default); cast / fc / bn: the FP32->FP16 cast, the "
+                         "inner-product layer and the batch-norm layer, measured on their own")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD,
                     help="one of: " + ", ".join(w.name for w in workloads.all_workloads()))
     ap.add_argument("--layers", action="store_true", help="add per-layer figures to the JSON line")
