@@ -42,24 +42,33 @@ __device__ __forceinline__ float group_sum(const uint16_t* __restrict__ p, int c
   const int lane = (int)(threadIdx.x & 31u);
   float acc = 0.f;
   int done = 0;
-  if (vec) {
-    const int nvec = count >> 3;
-    const uint4* pv = reinterpret_cast<const uint4*>(p);
-    for (int i = lane; i < nvec; i += 32) {
-      const uint4 q = __ldg(pv + i);
-      const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+  auto add = [&](const uint4& q) {
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        float a = h_lo(w[j]), b = h_hi(w[j]);
-        if (SQ) {
-          a = (a - mean) * shift;
-          b = (b - mean) * shift;
-          acc += a * a + b * b;
-        } else {
-          acc += a + b;
-        }
+    for (int j = 0; j < 4; ++j) {
+      float a = h_lo(w[j]), b = h_hi(w[j]);
+      if (SQ) {
+        a = (a - mean) * shift;
+        b = (b - mean) * shift;
+        acc += a * a + b * b;
+      } else {
+        acc += a + b;
       }
     }
+  };
+  if (vec) {
+    const uint4* pv = reinterpret_cast<const uint4*>(p);
+    if (count == kBnGroup) {
+      // a full group: the lane's eight loads are issued before the first is used
+      uint4 q[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) q[j] = __ldg(pv + lane + 32 * j);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) add(q[j]);
+      return warp_sum(acc);
+    }
+    const int nvec = count >> 3;
+    for (int i = lane; i < nvec; i += 32) add(__ldg(pv + i));
     done = nvec << 3;
   }
   for (int i = done + lane; i < count; i += 32) {
@@ -150,11 +159,9 @@ bn_apply_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, const 
     const int64_t base = ((int64_t)img * C + c) * hw + start;
     int done = 0;
     if (vec) {
-      const int nvec = count >> 3;
       const uint4* pv = reinterpret_cast<const uint4*>(x + base);
       uint4* py = reinterpret_cast<uint4*>(y + base);
-      for (int i = lane; i < nvec; i += 32) {
-        const uint4 q = __ldcs(pv + i);
+      auto norm = [&](const uint4& q) {
         const uint32_t w[4] = {q.x, q.y, q.z, q.w};
         uint32_t o[4];
 #pragma unroll
@@ -162,8 +169,18 @@ bn_apply_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, const 
           const __half2 h = __floats2half2_rn((h_lo(w[j]) - mean) * inv, (h_hi(w[j]) - mean) * inv);
           o[j] = *reinterpret_cast<const uint32_t*>(&h);
         }
-        py[i] = make_uint4(o[0], o[1], o[2], o[3]);
+        return make_uint4(o[0], o[1], o[2], o[3]);
+      };
+      if (count == kBnGroup) {
+        uint4 q[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) q[j] = __ldcs(pv + lane + 32 * j);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) py[lane + 32 * j] = norm(q[j]);
+        continue;
       }
+      const int nvec = count >> 3;
+      for (int i = lane; i < nvec; i += 32) py[i] = norm(__ldcs(pv + i));
       done = nvec << 3;
     }
     for (int i = done + lane; i < count; i += 32) {
@@ -204,9 +221,10 @@ cudaError_t launch_batchnorm(const __half* x, __half* y, int32_t n, int32_t c, i
                              cudaStream_t stream) {
   const int chunks = bn_chunks(hw);
   const int64_t G = (int64_t)n * chunks;
-  // blocks per channel: enough to fill the GPU a few times over, never more than the groups need
+  // blocks per channel: one group per warp unless that would be far more blocks than the GPU can
+  // hold several times over
   int64_t bx = (G + kBnWarps - 1) / kBnWarps;
-  const int64_t cap = ((int64_t)sm_count() * 16 + c - 1) / c;
+  const int64_t cap = ((int64_t)sm_count() * 64 + c - 1) / c;
   if (bx > cap) bx = cap;
   if (bx < 1) bx = 1;
   const dim3 grid((unsigned)bx, (unsigned)c);
