@@ -184,6 +184,44 @@ def test_configs_full_size_sampled(hgc, oracle, cfg, batch):
         del xd, wd, bd, y
 
 
+@pytest.mark.parametrize("cfg,batch", [(2, 16), (4, 64)])
+def test_configs_full_size_channels_last_sampled(hgc, oracle, cfg, batch):
+    """The bench's channels-last leg at full size: every layer that takes the flags reads
+    x[N][H][W][C] and writes y[N][P][Q][K]; sampled outputs against the oracle as above."""
+    import torch
+    wl = workloads.workload(cfg, batch)
+    rng = np.random.default_rng(199 + cfg)
+    for li, l in _unique_layers(wl):
+        a = layer_args(batch, l)
+        d, fl = None, 0
+        for fl in (hgc.HGC_FLAG_X_NHWC | hgc.HGC_FLAG_Y_NHWC, hgc.HGC_FLAG_Y_NHWC):
+            try:
+                d = hgc.ConvDesc(flags=fl, **a)
+                break
+            except hgc.HgcError:
+                d = None
+        if d is None:
+            continue
+        x, w, b = workloads.make_tensors(cfg, batch, li, l)
+        n, k, p, q = d.output_dims()
+        d.ensure_workspace()
+        xin = np.ascontiguousarray(x.transpose(0, 2, 3, 1)) if fl & hgc.HGC_FLAG_X_NHWC else x
+        xd, wd, bd = to_dev(xin), to_dev(w), to_dev(b)
+        y = torch.full((n, p, q, k), float("nan"), dtype=torch.float16, device="cuda")
+        d.set_weights(wd)
+        hgc.conv_forward(d, xd, wd, bd, y, l.relu)
+        torch.cuda.synchronize()
+        assert d.last_device_status() == hgc.HGC_OK
+        assert bool(torch.isfinite(y).all()), f"{wl.name}/{l.name}: non-finite output"
+        coords = sample_coords(rng, n, k, p, q)
+        ref = oracle.conv_points(oracle.ConvParams(**a), x, w, b, l.relu, coords)
+        ct = torch.from_numpy(coords).cuda()
+        got = to_host(y[ct[:, 0], ct[:, 2], ct[:, 3], ct[:, 1]])
+        check_close(got, ref, what=f"{wl.name}/{l.name} channels-last")
+        d.close()
+        del xd, wd, bd, y
+
+
 def test_forward_host_matches_device_forward(hgc, oracle):
     import torch
     rng = np.random.default_rng(4)
