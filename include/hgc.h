@@ -68,7 +68,8 @@ typedef struct hgc_conv_params {
  * (the paper's rule "convert only at the input and the output", Section 3.3, applied to the
  * layout): with HGC_FLAG_X_NHWC the input is x[N][H][W][C] and the layout pass is skipped; with
  * HGC_FLAG_Y_NHWC the output is written as y[N][P][Q][K].  Both are taken by the tensor-core path
- * only (HGC_FLAG_X_NHWC also needs C, and C/group for grouped layers, to be multiples of 8);
+ * (HGC_FLAG_X_NHWC also needs C, and C/group for grouped layers, to be multiples of 8) and, when
+ * given together, by 3x3 depthwise layers of C % 8 == 0 channels (stride 1 or 2, dilation 1);
  * hgc_conv_desc_create returns HGC_UNSUPPORTED otherwise.  Weights and bias are as always.
  * Channels-last output is staged in shared memory and written by TMA when K/group is a multiple
  * of 32 (as fast as the NCHW epilogue); other channel counts are written with plain 2-byte stores.

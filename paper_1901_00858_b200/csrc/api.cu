@@ -84,7 +84,8 @@ int forward_impl(hgc_conv_desc* d, const void* x, const void* w, const void* bia
       break;
     }
     case HGC_PATH_DEPTHWISE:
-      err = hgc::launch_depthwise3x3(g, xh, wh, bh, yh, relu, stream);
+      err = g.x_nhwc ? hgc::launch_depthwise3x3_nhwc(g, xh, wh, bh, yh, relu, stream)
+                     : hgc::launch_depthwise3x3(g, xh, wh, bh, yh, relu, stream);
       break;
     case HGC_PATH_DIRECT:
     default:
@@ -135,12 +136,15 @@ int hgc_conv_desc_create(hgc_conv_desc** out, const hgc_conv_params* p) {
   if (!(p->flags & HGC_FLAG_FORCE_DIRECT)) {
     if (!channels_last && hgc::depthwise3x3_supported(g)) {
       d->path = HGC_PATH_DEPTHWISE;
+    } else if (g.x_nhwc && g.y_nhwc && hgc::depthwise3x3_nhwc_supported(g)) {
+      d->path = HGC_PATH_DEPTHWISE;  // channels-last on both sides: its own kernel
     } else if (hgc::igemm_make_plan(g, &d->igemm)) {
       d->path = HGC_PATH_IGEMM;
       d->ws_needed = d->igemm.ws_total;
     }
   }
-  if (channels_last && d->path != HGC_PATH_IGEMM) {  // only the tensor-core path takes channels-last tensors
+  // channels-last tensors: the tensor-core path, or a depthwise layer with both sides channels-last
+  if (channels_last && d->path != HGC_PATH_IGEMM && !(d->path == HGC_PATH_DEPTHWISE && g.x_nhwc && g.y_nhwc)) {
     delete d;
     return HGC_UNSUPPORTED;
   }

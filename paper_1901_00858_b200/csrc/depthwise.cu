@@ -397,6 +397,103 @@ depthwise3x3_smallrow_kernel(const uint16_t* __restrict__ x, const __half* __res
   }
 }
 
+// Channels-last depthwise 3x3 (x[N][H][W][C], y[N][P][Q][C], C % 8 == 0; any padding, stride 1
+// or 2): a thread owns 8 consecutive channels (one 16-byte vector per pixel) and TQ consecutive
+// output pixels of one output row.  It issues all its input vectors (3 rows x (TQ-1)*S+3 columns)
+// before using the first, keeps its 72 weights in registers, accumulates with the mixed-precision
+// FMA and writes one 16-byte vector per output pixel.  Consecutive lanes take consecutive channel
+// octets, so a warp's loads and stores are contiguous runs of channels (and of pixels, when a
+// pixel has fewer than 32 octets).  Neighbouring threads share input columns through L1.
+template <int S, int TQ>
+__global__ void __launch_bounds__(256)
+depthwise3x3_nhwc_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w,
+                         const uint16_t* __restrict__ bias, uint16_t* __restrict__ y, int c, int h, int wd, int p,
+                         int q, int pad_h, int pad_w, int relu, int strips, int64_t items) {
+  grid_dependency_wait();
+  constexpr int COLS = (TQ - 1) * S + 3;
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= items) return;
+  const int octets = c >> 3;
+  const int oc = (int)(idx % octets);
+  int64_t t = idx / octets;
+  const int strip = (int)(t % strips);
+  t /= strips;
+  const int pr = (int)(t % p);
+  const int64_t img = t / p;
+  const int q0 = strip * TQ;
+
+  // input window: rows pr*S - pad_h .. +2, columns q0*S - pad_w .. + COLS-1; zero outside the image
+  uint4 in[3][COLS];
+  const int ih0 = pr * S - pad_h, iw0 = q0 * S - pad_w;
+#pragma unroll
+  for (int rr = 0; rr < 3; ++rr) {
+    const int ih = ih0 + rr;
+    const bool rv = ih >= 0 && ih < h;
+#pragma unroll
+    for (int cc = 0; cc < COLS; ++cc) {
+      const int iw = iw0 + cc;
+      const bool v = rv && iw >= 0 && iw < wd;
+      in[rr][cc] = v ? __ldg(reinterpret_cast<const uint4*>(x + ((img * h + ih) * wd + iw) * c) + oc)
+                     : make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
+  // weights w[ch][9] of the 8 channels: 144 contiguous bytes, element ch*9 + tap
+  uint16_t wv[72];
+  {
+    const uint4* wp = reinterpret_cast<const uint4*>(w + (int64_t)oc * 72);
+#pragma unroll
+    for (int i = 0; i < 9; ++i) {
+      const uint4 v = __ldg(wp + i);
+      const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) asm("mov.b32 {%0, %1}, %2;" : "=h"(wv[8 * i + 2 * j]), "=h"(wv[8 * i + 2 * j + 1]) : "r"(u[j]));
+    }
+  }
+  float bv[8];
+  if (bias != nullptr) {
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(bias) + oc);
+    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      bv[2 * j] = __half2float(__ushort_as_half((uint16_t)(u[j] & 0xffffu)));
+      bv[2 * j + 1] = __half2float(__ushort_as_half((uint16_t)(u[j] >> 16)));
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) bv[j] = 0.f;
+  }
+#pragma unroll
+  for (int o = 0; o < TQ; ++o) {
+    if (q0 + o >= q) break;
+    float acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = bv[e];
+#pragma unroll
+    for (int rr = 0; rr < 3; ++rr)
+#pragma unroll
+      for (int ss = 0; ss < 3; ++ss) {
+        const uint4 v = in[rr][o * S + ss];
+        const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          uint16_t lo, hi;
+          asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(u[j]));
+          asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(acc[2 * j]) : "h"(lo), "h"(wv[(2 * j) * 9 + rr * 3 + ss]));
+          asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(acc[2 * j + 1]) : "h"(hi), "h"(wv[(2 * j + 1) * 9 + rr * 3 + ss]));
+        }
+      }
+    uint32_t ov[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (relu)
+        asm("cvt.rn.relu.f16x2.f32 %0, %1, %2;" : "=r"(ov[j]) : "f"(acc[2 * j + 1]), "f"(acc[2 * j]));
+      else
+        asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(ov[j]) : "f"(acc[2 * j + 1]), "f"(acc[2 * j]));
+    }
+    reinterpret_cast<uint4*>(y + ((img * p + pr) * q + q0 + o) * c)[oc] = make_uint4(ov[0], ov[1], ov[2], ov[3]);
+  }
+}
+
 // shapes the small-row kernel takes
 bool smallrow_ok(const ConvGeom& g) {
   if (g.pad_h != 1 || g.pad_w != 1) return false;
@@ -468,6 +565,38 @@ bool make_plan(const ConvGeom& g, DwPlan* plan) {
 }
 
 }  // namespace
+
+bool depthwise3x3_nhwc_supported(const ConvGeom& g) {
+  if (g.r != 3 || g.s != 3 || g.dil_h != 1 || g.dil_w != 1) return false;
+  if (g.group != g.c || g.k != g.c || (g.c & 7) != 0) return false;
+  if (g.stride_h != g.stride_w || (g.stride_h != 1 && g.stride_h != 2)) return false;
+  const int tq = g.stride_h == 1 ? 4 : 2;
+  const int64_t items = (int64_t)g.n * g.p * ((g.q + tq - 1) / tq) * (g.c / 8);
+  return (items + 255) / 256 < 0x7fffffffLL;
+}
+
+cudaError_t launch_depthwise3x3_nhwc(const ConvGeom& g, const __half* x, const __half* w, const __half* bias,
+                                     __half* y, int relu, cudaStream_t stream) {
+  if (!depthwise3x3_nhwc_supported(g)) return cudaErrorInvalidConfiguration;
+  const int tq = g.stride_h == 1 ? 4 : 2;
+  const int strips = (g.q + tq - 1) / tq;
+  const int64_t items = (int64_t)g.n * g.p * strips * (g.c / 8);
+  const unsigned blocks = (unsigned)((items + 255) / 256);
+  const uint16_t* xs = reinterpret_cast<const uint16_t*>(x);
+  const uint16_t* ws = reinterpret_cast<const uint16_t*>(w);
+  const uint16_t* bs = reinterpret_cast<const uint16_t*>(bias);
+  uint16_t* ys = reinterpret_cast<uint16_t*>(y);
+  cudaError_t err;
+  if (g.stride_h == 1)
+    err = launch_kernel(depthwise3x3_nhwc_kernel<1, 4>, dim3(blocks), dim3(256), 0, stream, xs, ws, bs, ys, g.c, g.h, g.w,
+                        g.p, g.q, g.pad_h, g.pad_w, relu, strips, items);
+  else
+    err = launch_kernel(depthwise3x3_nhwc_kernel<2, 2>, dim3(blocks), dim3(256), 0, stream, xs, ws, bs, ys, g.c, g.h, g.w,
+                        g.p, g.q, g.pad_h, g.pad_w, relu, strips, items);
+  if (err != cudaSuccess) return err;
+  count_launch();
+  return cudaGetLastError();
+}
 
 bool depthwise3x3_supported(const ConvGeom& g) {
   DwPlan a;

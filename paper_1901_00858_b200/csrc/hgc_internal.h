@@ -69,6 +69,11 @@ bool depthwise3x3_supported(const ConvGeom& g);
 cudaError_t launch_depthwise3x3(const ConvGeom& g, const __half* x, const __half* w,
                                 const __half* bias, __half* y, int relu, cudaStream_t stream);
 
+// channels-last variant (x and y [N][H][W][C], C % 8 == 0)
+bool depthwise3x3_nhwc_supported(const ConvGeom& g);
+cudaError_t launch_depthwise3x3_nhwc(const ConvGeom& g, const __half* x, const __half* w, const __half* bias,
+                                     __half* y, int relu, cudaStream_t stream);
+
 cudaError_t launch_nchw_to_nhwc(const __half* src, __half* dst, int32_t n, int32_t c, int32_t h,
                                 int32_t w, int32_t c_pad, cudaStream_t stream);
 cudaError_t launch_nhwc_to_nchw(const __half* src, __half* dst, int32_t n, int32_t c, int32_t h,

@@ -180,9 +180,43 @@ def test_channels_last_flags(hgc, oracle, name, a, xl, yl):
     d.close()
 
 
+DW_NHWC_CASES = [
+    ("112x112 c32", params_dict(2, 32, 112, 112, 32, 3, 3, 1, 1, 1, 1, 1, 1, 32)),
+    ("56x56 c128 stride 2", params_dict(2, 128, 56, 56, 128, 3, 3, 1, 1, 2, 2, 1, 1, 128)),
+    ("14x14 c512", params_dict(3, 512, 14, 14, 512, 3, 3, 1, 1, 1, 1, 1, 1, 512)),
+    ("7x7 c1024", params_dict(2, 1024, 7, 7, 1024, 3, 3, 1, 1, 1, 1, 1, 1, 1024)),
+    ("odd plane 13x9 c24, ragged strips", params_dict(2, 24, 13, 9, 24, 3, 3, 1, 1, 1, 1, 1, 1, 24)),
+    ("15x15 stride 2 c40", params_dict(1, 40, 15, 15, 40, 3, 3, 1, 1, 2, 2, 1, 1, 40)),
+    ("no padding 10x12 c16", params_dict(2, 16, 10, 12, 16, 3, 3, 0, 0, 1, 1, 1, 1, 16)),
+    ("padding 2, stride 2, 9x11 c8", params_dict(2, 8, 9, 11, 8, 3, 3, 2, 2, 2, 2, 1, 1, 8)),
+]
+
+
+@pytest.mark.parametrize("name,a", DW_NHWC_CASES, ids=[c[0] for c in DW_NHWC_CASES])
+def test_depthwise_channels_last(hgc, oracle, name, a):
+    import torch
+    from gpu_util import to_dev, to_host
+    rng = np.random.default_rng(zlib.crc32(name.encode()))
+    x, w, b = workloads.random_layer_tensors(rng, a["n"], a["c"], a["h"], a["w"], a["k"], 3, 3, a["group"])
+    d = hgc.ConvDesc(flags=hgc.HGC_FLAG_X_NHWC | hgc.HGC_FLAG_Y_NHWC, **a)
+    assert d.path() == hgc.HGC_PATH_DEPTHWISE
+    n, k, p, q = d.output_dims()
+    xd, wd, bd = to_dev(np.ascontiguousarray(x.transpose(0, 2, 3, 1))), to_dev(w), to_dev(b)
+    for relu, bias, bias_d in ((True, b, bd), (False, None, None)):
+        ref = oracle.conv_fast(oracle.ConvParams(**a), x, w, bias, relu)
+        y = torch.full((n, p, q, k), float("nan"), dtype=torch.float16, device="cuda")
+        hgc.conv_forward(d, xd, wd, bias_d, y, relu)
+        torch.cuda.synchronize()
+        check_close(np.ascontiguousarray(to_host(y).transpose(0, 3, 1, 2)), ref, what=f"{name} relu={relu}")
+    d.close()
+
+
 def test_channels_last_flags_are_refused_where_they_cannot_apply(hgc):
-    with pytest.raises(hgc.HgcError):     # depthwise layers have no channels-last variant
+    with pytest.raises(hgc.HgcError):     # a depthwise layer takes the flags only together
         hgc.ConvDesc(2, 32, 14, 14, 32, 3, 3, 1, 1, 1, 1, 1, 1, 32, flags=hgc.HGC_FLAG_Y_NHWC)
+    with pytest.raises(hgc.HgcError):     # and only with whole 16-byte vectors of channels
+        hgc.ConvDesc(2, 12, 14, 14, 12, 3, 3, 1, 1, 1, 1, 1, 1, 12,
+                     flags=hgc.HGC_FLAG_X_NHWC | hgc.HGC_FLAG_Y_NHWC)
     with pytest.raises(hgc.HgcError):     # 3 input channels are not a whole number of 16-byte vectors
         hgc.ConvDesc(2, 3, 14, 14, 32, 3, 3, 1, 1, flags=hgc.HGC_FLAG_X_NHWC)
 
