@@ -151,6 +151,9 @@ NHWC_CASES = [
     ("stem c3 k64 windows, channels-last out", params_dict(2, 3, 24, 40, 64, 3, 3, 1, 1), False, True),
     ("stem 7x7 stride 2 c3 k64 patches, channels-last out", params_dict(2, 3, 38, 38, 64, 7, 7, 3, 3, 2, 2), False, True),
     ("grouped: 2 groups of 64 output channels", params_dict(2, 64, 12, 20, 128, 3, 3, 1, 1, 1, 1, 1, 1, 2), True, True),
+    ("7x7 c2048 k128: channels-last in, few tiles (split reduction), NCHW out", params_dict(2, 2048, 7, 7, 128, 3, 3, 1, 1), True, False),
+    ("7x7 c2048 k128: both channels-last (no split)", params_dict(2, 2048, 7, 7, 128, 3, 3, 1, 1), True, True),
+    ("dilated 3x3 c64 k64 channels-last", params_dict(2, 64, 20, 20, 64, 3, 3, 2, 2, 1, 1, 2, 2), True, True),
 ]
 
 
