@@ -162,8 +162,9 @@ int hgc_conv_path(const hgc_conv_desc* d, int32_t* path);
  * kernel row share one activation tile (stride 1), [3] images per pixel tile, [4] rows per pixel
  * tile, [5] accumulator columns per output row, [6] MMA N, [7] number of tiles, [8] depth of the
  * shared-memory ring, [9] weight tiles (taps) per ring stage, [10] where the kernel's activation
- * tiles come from: 0 = an NHWC copy of x made by the layout pass, 1 = x itself, read as
- * pixel-major tiles (1x1 layers), 2 = a zero-bordered 8-channel NHWC copy read through
+ * tiles come from: 0 = an NHWC copy of x made by the layout pass, 1 = x itself (1x1 layers read
+ * as pixel-major tiles; channels-last x, which includes every input with a 1x1 plane), 2 = a
+ * zero-bordered 8-channel NHWC copy read through
  * overlapping windows (few input channels), 3 = an expanded copy holding, per output pixel, the
  * values under the kernel (few input channels, strided), [11] the number of CTAs that share
  * the reduction of one tile (1, or 2 / 4 / 8 for layers with very few tiles, e.g. inner products:

@@ -215,7 +215,7 @@ int hgc_conv_plan_info(const hgc_conv_desc* d, int32_t* info, int32_t count) {
     const hgc::IgemmPlan& p = d->igemm;
     v[1] = p.kb; v[2] = p.halo; v[3] = p.tn; v[4] = p.th; v[5] = p.pitch; v[6] = p.ncols;
     v[7] = p.total_tiles; v[8] = p.stages; v[9] = p.taps;
-    v[10] = p.nchw ? 1 : (p.window ? 2 : (p.patch ? 3 : 0));
+    v[10] = (p.nchw || p.x_nhwc) ? 1 : (p.window ? 2 : (p.patch ? 3 : 0));
     v[11] = 1 << p.ks_log2;
   }
   for (int i = 0; i < count && i < 12; ++i) info[i] = v[i];

@@ -1205,6 +1205,8 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   p.y_nhwc = g.y_nhwc;
   // channels-last input: x is used as x' (a pixel must be a whole number of 16-byte vectors)
   if (p.x_nhwc && ((g.c % 8) != 0 || g.cg < 9)) return false;
+  // a 1x1 input plane (inner products) is channels-last as it stands: no layout pass
+  if (g.h == 1 && g.w == 1 && (g.c % 8) == 0 && g.cg >= 9) p.x_nhwc = 1;
   // Few input channels (image stems, C <= 8): a tap alone is too short for a K=16 MMA step.
   // The input is copied to a zero-bordered NHWC buffer with 8 channels per pixel; the S taps of
   // a kernel row are then S*8 CONTIGUOUS elements, read as one "window" per output pixel through
