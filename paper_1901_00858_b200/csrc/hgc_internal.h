@@ -107,6 +107,8 @@ struct IgemmPlan {
   int32_t y_rpu, y_full_w;                       // channels-last stores: tile rows and pixels per store
   int32_t y_perm;                                // weight rows interleaved for the staged channels-last epilogue
   int32_t window, kw_pix, hp, wp;                // few-channel layers: windows over a zero-bordered NHWC8 copy
+  int32_t dense_rows;                            // window mode at stride 1: whole rows loaded, windows read in place
+  int32_t vhalo;                                 // ... and the R kernel rows share one tile of th + R - 1 rows
   int32_t patch;                                 // tiny receptive fields: 1x1 conv over an im2col copy of x
   int32_t eff_r, eff_s, eff_pad_h, eff_pad_w;    // the convolution as the kernel sees it
   int32_t tn, th, tw, ncols;

@@ -1241,8 +1241,25 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
     p.hp = g.h + 2 * g.pad_h;
     p.wp = g.w + 2 * g.pad_w;
     if (p.wp < (g.q - 1) * g.stride_w + p.kw_pix) p.wp = (g.q - 1) * g.stride_w + p.kw_pix;
+    // Stride 1 along W: the window of output pixel q is the kw_pix pixels from q on, so whole rows
+    // of the bordered copy (a multiple of 8 pixels wide) are loaded densely, 128 bytes per TMA
+    // request instead of one request per window, and the MMA reads the overlapping windows
+    // straight out of them: an unswizzled K-major operand whose rows are 16 bytes (one pixel)
+    // apart and whose 16-byte K chunks are also 16 bytes apart.  The accumulator then has one
+    // column per pixel of the padded row (pitch wp, junk columns at the end of each tile row).
+    p.dense_rows = (g.stride_w == 1 && p.cblocks == 1 && (p.wp + 7) / 8 * 8 <= 256) ? 1 : 0;
+    if (p.dense_rows) p.wp = (p.wp + 7) / 8 * 8;
     p.eff_r = g.r; p.eff_s = 1; p.eff_pad_h = 0; p.eff_pad_w = 0;
     p.halo = 0;
+    // ... and with stride 1 along H too, the R kernel rows share one tile of th + R - 1 dense rows
+    // (the mechanism of the shared taps of a kernel row, turned by 90 degrees: tap r starts r
+    // image rows = r * wp pixels further in shared memory): one pipeline stage per tile
+    if (p.dense_rows && g.stride_h == 1 && g.dil_h == 1) {
+      p.vhalo = 1;
+      p.halo = 1;
+      p.eff_r = 1;
+      p.eff_s = g.r;
+    }
   } else {
     p.kb = g.cg > 32 ? 64 : (g.cg > 16 ? 32 : 16);
     // stride-1 layers with three or more taps per kernel row and at least two 64-channel blocks:
@@ -1262,9 +1279,9 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
             g.pad_w == 0 && g.group == 1 && ((int64_t)g.h * g.w) % 8 == 0)
                ? 1
                : 0;
-  p.pitch = p.halo ? g.q + (g.s - 1) * g.dil_w : g.q;
+  p.pitch = p.dense_rows ? p.wp : (p.halo ? g.q + (g.s - 1) * g.dil_w : g.q);
   p.tw = g.q;
-  const int box_w = p.halo ? p.pitch : ((p.window || p.patch) ? g.q : g.q * g.stride_w);
+  const int box_w = (p.halo && !p.vhalo) ? p.pitch : ((p.window || p.patch) ? g.q : g.q * g.stride_w);
   if (p.pitch > 256 || box_w > 256) return false;
   p.mtiles = (g.kg + 127) / 128;
   const int64_t mg = (int64_t)p.mtiles * g.group;
@@ -1311,7 +1328,7 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   for (int th = 1; th <= g.p; ++th) {
     if ((int64_t)th * p.pitch - junk > 256 || (int64_t)th * (p.patch ? 1 : g.stride_h) > 256) break;
     if (p.nchw && th != g.p && ((int64_t)th * g.q) % 8 != 0) continue;  // tiles must start on 16-byte boundaries of x
-    const int tn_hi = (th == g.p && !p.nchw) ? g.n : 1;  // several images only when a tile holds whole planes
+    const int tn_hi = (th == g.p && !p.nchw && !p.vhalo) ? g.n : 1;  // several images only when a tile holds whole planes
     for (int tn = 1; tn <= tn_hi; ++tn) {
       const int64_t cols = (int64_t)tn * th * p.pitch - junk;
       // several images per tile: image boundaries need not fall on multiples of 8 columns, and an
@@ -1398,12 +1415,18 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   // S taps of a kernel row do not fit twice, fall back to one tap (and its own tile) per stage
   for (;;) {
     p.taps = p.halo ? p.eff_s : 1;
-    p.pitch = p.halo ? g.q + (g.s - 1) * g.dil_w : g.q;
-    const uint32_t box_rows2 = (uint32_t)(p.tn * p.th * p.pitch);
+    p.pitch = p.dense_rows ? p.wp : (p.halo ? g.q + (g.s - 1) * g.dil_w : g.q);
+    const uint32_t box_rows2 = (uint32_t)(p.tn * (p.th + (p.vhalo ? g.r - 1 : 0)) * p.pitch);
     p.b_bytes = box_rows2 * p.kb * 2u;
     uint32_t rows2 = (uint32_t)(p.halo ? (g.s - 1) * g.dil_w : 0) + (uint32_t)p.ncols;
     if (rows2 < box_rows2) rows2 = box_rows2;
     p.b_alloc = (uint32_t)round_up_sz((size_t)rows2 * p.kb * 2u, 1024);
+    if (p.dense_rows) {
+      // 16 bytes per pixel of the tile's rows; the last window read starts at column ncols - 1
+      p.b_bytes = box_rows2 * 16u;
+      const size_t reach = ((size_t)(p.vhalo ? (g.r - 1) * p.wp : 0) + p.ncols + p.kw_pix) * 16u;
+      p.b_alloc = (uint32_t)round_up_sz(reach > p.b_bytes ? reach : (size_t)p.b_bytes, 1024);
+    }
     if (p.nchw) {
       p.nblk = (p.ncols + 63) / 64;
       p.b_bytes = (uint32_t)p.nblk * (uint32_t)p.kb * 128u;
@@ -1490,6 +1513,19 @@ bool igemm_encode_maps(const ConvGeom& g, IgemmPlan* p, void* ws) {
     cuuint32_t es[5] = {1, 1, 1, 1, 1};
     if (enc(&p->tmB, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, base + p->ws_x_off, dims, strides, box, es,
             CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return false;
+  } else if (p->window && p->dense_rows) {
+    // (8 pixels x 8 channels = 128 bytes, block of 8 pixels, -, padded input row, image): whole
+    // rows of the bordered copy, dense in shared memory
+    cuuint64_t dims[5] = {64, (cuuint64_t)(p->wp / 8), 1, (cuuint64_t)p->hp, (cuuint64_t)g.n};
+    cuuint64_t strides[4] = {128, 128 * (cuuint64_t)(p->wp / 8), 16 * (cuuint64_t)p->wp,
+                             16 * (cuuint64_t)p->wp * (cuuint64_t)p->hp};
+    cuuint32_t box[5] = {64, (cuuint32_t)(p->wp / 8), 1,
+                         (cuuint32_t)(p->vhalo ? p->th + g.r - 1 : p->th * g.stride_h), (cuuint32_t)p->tn};
+    cuuint32_t es[5] = {1, 1, 1, (cuuint32_t)g.stride_h, 1};
+    if (enc(&p->tmB, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, base + p->ws_x_off, dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return false;
   } else if (p->window) {
@@ -1605,6 +1641,15 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
     const uint64_t lbo = (uint64_t)(p.kb * 128) >> 4;
     a.desc_hi_b = (lbo << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
     a.b_kstep = 2048 >> 4;
+  }
+  if (p.dense_rows) {
+    // unswizzled K-major tile of overlapping windows: a row (pixel) every 16 bytes, the next 16-byte
+    // K chunk (the next pixel of the window) 16 bytes on, the next 8 rows 128 bytes on
+    a.desc_hi_b = (1ull << 16) | (8ull << 32) | (1ull << 46);
+    a.b_kstep = 2;  // 16 window elements = two pixels
+    // shared kernel rows: the kernel advances the activation descriptor by dil_w rows of kb
+    // elements per tap; one image row is wp pixels of 8 elements
+    if (p.vhalo) a.dil_w = p.wp * 8 / p.kb;
   }
   a.relu = relu;
   a.tma_store = p.tma_store;
