@@ -79,10 +79,11 @@ cudaError_t launch_nchw_to_nhwc(const __half* src, __half* dst, int32_t n, int32
 cudaError_t launch_nhwc_to_nchw(const __half* src, __half* dst, int32_t n, int32_t c, int32_t h,
                                 int32_t w, int32_t c_pad, cudaStream_t stream);
 cudaError_t launch_nchw_to_nhwc8_bordered(const __half* src, __half* dst, int32_t n, int32_t c, int32_t h, int32_t w,
-                                          int32_t pad_h, int32_t pad_w, int32_t hp, int32_t wp, cudaStream_t stream);
+                                          int32_t pad_h, int32_t pad_w, int32_t hp, int32_t wp, cudaStream_t stream,
+                                          int px_ch = 8);  // channels per pixel of the copy: 8 or 4
 // perm: rows of every block of 32 output channels interleaved (see row_channel in layout.cu)
 cudaError_t launch_weights_repack_window(const __half* src, __half* dst, int32_t k, int32_t c, int32_t r, int32_t s,
-                                         int32_t kw_pix, cudaStream_t stream, int perm = 0);
+                                         int32_t kw_pix, cudaStream_t stream, int perm = 0, int px_ch = 8);
 cudaError_t launch_weights_repack(const __half* src, __half* dst, int32_t k, int32_t cg, int32_t r,
                                   int32_t s, int32_t group, int32_t c_pad, cudaStream_t stream, int perm = 0);
 
@@ -107,7 +108,8 @@ struct IgemmPlan {
   int32_t y_rpu, y_full_w;                       // channels-last stores: tile rows and pixels per store
   int32_t y_perm;                                // weight rows interleaved for the staged channels-last epilogue
   int32_t window, kw_pix, hp, wp;                // few-channel layers: windows over a zero-bordered NHWC8 copy
-  int32_t dense_rows;                            // window mode at stride 1: whole rows loaded, windows read in place
+  int32_t px_ch;                                 // channels per pixel of the bordered copy: 8, or 4 (strided stems)
+  int32_t dense_rows, dense_pitch;               // windows 16 bytes apart: whole rows loaded, windows read in place
   int32_t vhalo;                                 // ... and the R kernel rows share one tile of th + R - 1 rows
   int32_t patch;                                 // tiny receptive fields: 1x1 conv over an im2col copy of x
   int32_t eff_r, eff_s, eff_pad_h, eff_pad_w;    // the convolution as the kernel sees it

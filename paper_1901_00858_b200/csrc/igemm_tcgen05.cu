@@ -1232,29 +1232,49 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
     p.eff_r = 1; p.eff_s = 1; p.eff_pad_h = 0; p.eff_pad_w = 0;
     p.halo = 0;
   } else if (p.window) {
-    const int kelems = g.s * 8 <= 16 ? 16 : g.s * 8 <= 32 ? 32 : (g.s * 8 + 63) / 64 * 64;
-    p.kw_pix = kelems / 8;
-    p.kb = kelems >= 64 ? 64 : kelems;
-    p.cblocks = kelems / p.kb;
-    p.cw = kelems;
-    p.c_pad = 8;
-    p.hp = g.h + 2 * g.pad_h;
-    p.wp = g.w + 2 * g.pad_w;
-    if (p.wp < (g.q - 1) * g.stride_w + p.kw_pix) p.wp = (g.q - 1) * g.stride_w + p.kw_pix;
-    // Stride 1 along W: the window of output pixel q is the kw_pix pixels from q on, so whole rows
-    // of the bordered copy (a multiple of 8 pixels wide) are loaded densely, 128 bytes per TMA
-    // request instead of one request per window, and the MMA reads the overlapping windows
-    // straight out of them: an unswizzled K-major operand whose rows are 16 bytes (one pixel)
-    // apart and whose 16-byte K chunks are also 16 bytes apart.  The accumulator then has one
-    // column per pixel of the padded row (pitch wp, junk columns at the end of each tile row).
-    p.dense_rows = (g.stride_w == 1 && p.cblocks == 1 && (p.wp + 7) / 8 * 8 <= 256) ? 1 : 0;
-    if (p.dense_rows) p.wp = (p.wp + 7) / 8 * 8;
+    // Pixels of the bordered copy hold 8 channels (16 bytes), or 4 (8 bytes) for layers of at most
+    // 4 channels with stride 2 along W: consecutive windows then start 2 pixels = 16 bytes apart,
+    // which lets them take the dense form below too, at half the reduction length.
+    p.px_ch = (g.cg <= 4 && g.stride_w == 2 && g.s * 4 <= 64) ? 4 : 8;
+    for (;;) {
+      const int elems = g.s * p.px_ch;
+      const int kelems = elems <= 16 ? 16 : elems <= 32 ? 32 : (elems + 63) / 64 * 64;
+      p.kw_pix = kelems / p.px_ch;
+      p.kb = kelems >= 64 ? 64 : kelems;
+      p.cblocks = kelems / p.kb;
+      p.cw = kelems;
+      p.c_pad = p.px_ch;
+      p.hp = g.h + 2 * g.pad_h;
+      p.wp = g.w + 2 * g.pad_w;
+      if (p.wp < (g.q - 1) * g.stride_w + p.kw_pix) p.wp = (g.q - 1) * g.stride_w + p.kw_pix;
+      // Windows that start 16 bytes apart (stride 1 with 8-channel pixels, stride 2 with 4-channel
+      // pixels) are not fetched one by one: whole rows of the bordered copy (a multiple of 128 bytes
+      // wide) are loaded densely, 128 bytes per TMA request, and the MMA reads the overlapping
+      // windows straight out of them: an unswizzled K-major operand whose rows (windows) are 16
+      // bytes apart and whose 16-byte K chunks are also 16 bytes apart.  The accumulator then has
+      // one column per 16 bytes of the padded row (junk columns at the end of each tile row).
+      const int per128 = 64 / p.px_ch;  // pixels per 128 bytes
+      const int wp_dense = (p.wp + per128 - 1) / per128 * per128;
+      const int pitch_dense = wp_dense * p.px_ch / 8;
+      p.dense_rows = (g.stride_w * p.px_ch == 8 && p.cblocks == 1 && pitch_dense <= 256) ? 1 : 0;
+      if (p.dense_rows) {
+        p.wp = wp_dense;
+        p.dense_pitch = pitch_dense;
+      }
+      if (p.px_ch == 4 && !p.dense_rows) {  // 4-channel pixels only pay in the dense form
+        p.px_ch = 8;
+        continue;
+      }
+      break;
+    }
     p.eff_r = g.r; p.eff_s = 1; p.eff_pad_h = 0; p.eff_pad_w = 0;
     p.halo = 0;
     // ... and with stride 1 along H too, the R kernel rows share one tile of th + R - 1 dense rows
     // (the mechanism of the shared taps of a kernel row, turned by 90 degrees: tap r starts r
     // image rows = r * wp pixels further in shared memory): one pipeline stage per tile
-    if (p.dense_rows && g.stride_h == 1 && g.dil_h == 1) {
+    // (with a stride along H the tile is one output row: rows of a taller tile would be
+    // stride_h image rows apart, more accumulator columns than there are)
+    if (p.dense_rows && g.dil_h == 1) {
       p.vhalo = 1;
       p.halo = 1;
       p.eff_r = 1;
@@ -1279,7 +1299,7 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
             g.pad_w == 0 && g.group == 1 && ((int64_t)g.h * g.w) % 8 == 0)
                ? 1
                : 0;
-  p.pitch = p.dense_rows ? p.wp : (p.halo ? g.q + (g.s - 1) * g.dil_w : g.q);
+  p.pitch = p.dense_rows ? p.dense_pitch : (p.halo ? g.q + (g.s - 1) * g.dil_w : g.q);
   p.tw = g.q;
   const int box_w = (p.halo && !p.vhalo) ? p.pitch : ((p.window || p.patch) ? g.q : g.q * g.stride_w);
   if (p.pitch > 256 || box_w > 256) return false;
@@ -1327,6 +1347,7 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   int best_th = 0, best_tn = 0, best_ks = 0;
   for (int th = 1; th <= g.p; ++th) {
     if ((int64_t)th * p.pitch - junk > 256 || (int64_t)th * (p.patch ? 1 : g.stride_h) > 256) break;
+    if (p.vhalo && g.stride_h > 1 && th > 1) break;
     if (p.nchw && th != g.p && ((int64_t)th * g.q) % 8 != 0) continue;  // tiles must start on 16-byte boundaries of x
     const int tn_hi = (th == g.p && !p.nchw && !p.vhalo) ? g.n : 1;  // several images only when a tile holds whole planes
     for (int tn = 1; tn <= tn_hi; ++tn) {
@@ -1415,8 +1436,8 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   // S taps of a kernel row do not fit twice, fall back to one tap (and its own tile) per stage
   for (;;) {
     p.taps = p.halo ? p.eff_s : 1;
-    p.pitch = p.dense_rows ? p.wp : (p.halo ? g.q + (g.s - 1) * g.dil_w : g.q);
-    const uint32_t box_rows2 = (uint32_t)(p.tn * (p.th + (p.vhalo ? g.r - 1 : 0)) * p.pitch);
+    p.pitch = p.dense_rows ? p.dense_pitch : (p.halo ? g.q + (g.s - 1) * g.dil_w : g.q);
+    const uint32_t box_rows2 = (uint32_t)(p.tn * (p.vhalo ? (p.th - 1) * g.stride_h + g.r : p.th) * p.pitch);
     p.b_bytes = box_rows2 * p.kb * 2u;
     uint32_t rows2 = (uint32_t)(p.halo ? (g.s - 1) * g.dil_w : 0) + (uint32_t)p.ncols;
     if (rows2 < box_rows2) rows2 = box_rows2;
@@ -1424,7 +1445,7 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
     if (p.dense_rows) {
       // 16 bytes per pixel of the tile's rows; the last window read starts at column ncols - 1
       p.b_bytes = box_rows2 * 16u;
-      const size_t reach = ((size_t)(p.vhalo ? (g.r - 1) * p.wp : 0) + p.ncols + p.kw_pix) * 16u;
+      const size_t reach = ((size_t)(p.vhalo ? (g.r - 1) * p.pitch : 0) + p.ncols + p.cw / 8) * 16u;
       p.b_alloc = (uint32_t)round_up_sz(reach > p.b_bytes ? reach : (size_t)p.b_bytes, 1024);
     }
     if (p.nchw) {
@@ -1439,7 +1460,13 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
     if (!p.halo) return false;
     // without sharing, the accumulator pitch is Q again: the tile found above still fits
     p.halo = 0;
-    p.ncols = (p.tn * p.th * g.q + 15) / 16 * 16;
+    if (p.vhalo) {  // dense rows: the kernel rows take a stage each again, same columns
+      p.vhalo = 0;
+      p.eff_r = g.r;
+      p.eff_s = 1;
+    } else {
+      p.ncols = (p.tn * p.th * g.q + 15) / 16 * 16;
+    }
   }
   // a second staging tile per epilogue warp (its store overlaps the next unit) if memory is left
   p.nbuf = ((size_t)p.stages * p.stage_bytes + 2u * stage_buf_bytes <= budget_all) ? 2 : 1;
@@ -1454,7 +1481,7 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   p.ws_part_off = 0;
   p.ws_total = p.ws_x_off + ((p.nchw || p.x_nhwc) ? 0
                                     : round_up_sz(p.patch    ? (size_t)g.n * g.p * g.q * p.cw * 2
-                                                  : p.window ? (size_t)g.n * p.hp * p.wp * 16 + 256
+                                                  : p.window ? (size_t)g.n * p.hp * p.wp * p.px_ch * 2 + 256
                                                            : (size_t)g.n * g.h * g.w * p.c_pad * 2, 256));
   if (p.ks_log2 > 0) {
     p.ws_part_off = p.ws_total;
@@ -1518,12 +1545,14 @@ bool igemm_encode_maps(const ConvGeom& g, IgemmPlan* p, void* ws) {
   } else if (p->window && p->dense_rows) {
     // (8 pixels x 8 channels = 128 bytes, block of 8 pixels, -, padded input row, image): whole
     // rows of the bordered copy, dense in shared memory
-    cuuint64_t dims[5] = {64, (cuuint64_t)(p->wp / 8), 1, (cuuint64_t)p->hp, (cuuint64_t)g.n};
-    cuuint64_t strides[4] = {128, 128 * (cuuint64_t)(p->wp / 8), 16 * (cuuint64_t)p->wp,
-                             16 * (cuuint64_t)p->wp * (cuuint64_t)p->hp};
-    cuuint32_t box[5] = {64, (cuuint32_t)(p->wp / 8), 1,
-                         (cuuint32_t)(p->vhalo ? p->th + g.r - 1 : p->th * g.stride_h), (cuuint32_t)p->tn};
-    cuuint32_t es[5] = {1, 1, 1, (cuuint32_t)g.stride_h, 1};
+    const cuuint64_t row_bytes = (cuuint64_t)p->wp * p->px_ch * 2;
+    const cuuint32_t blocks = (cuuint32_t)(row_bytes / 128);
+    cuuint64_t dims[5] = {64, blocks, 1, (cuuint64_t)p->hp, (cuuint64_t)g.n};
+    cuuint64_t strides[4] = {128, row_bytes, row_bytes, row_bytes * (cuuint64_t)p->hp};
+    cuuint32_t box[5] = {64, blocks, 1,
+                         (cuuint32_t)(p->vhalo ? (p->th - 1) * g.stride_h + g.r : p->th * g.stride_h),
+                         (cuuint32_t)p->tn};
+    cuuint32_t es[5] = {1, 1, 1, (cuuint32_t)(p->vhalo ? 1 : g.stride_h), 1};
     if (enc(&p->tmB, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, base + p->ws_x_off, dims, strides, box, es,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -1649,7 +1678,7 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
     a.b_kstep = 2;  // 16 window elements = two pixels
     // shared kernel rows: the kernel advances the activation descriptor by dil_w rows of kb
     // elements per tap; one image row is wp pixels of 8 elements
-    if (p.vhalo) a.dil_w = p.wp * 8 / p.kb;
+    if (p.vhalo) a.dil_w = p.pitch * 8 / p.kb;
   }
   a.relu = relu;
   a.tma_store = p.tma_store;

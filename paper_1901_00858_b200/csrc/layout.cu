@@ -233,6 +233,7 @@ __global__ void weights_repack_kernel(const uint16_t* __restrict__ src, uint16_t
 
 // x[n][c][h][w] (c <= 8) -> x'[n][hp][wp][8]: pixel (h, w) lands at (h + pad_h, w + pad_w); the
 // border, the extra columns and channels c..7 are zero.  One thread per output pixel (16 bytes).
+template <int PC>  // channels per pixel of the copy: 8 (16 bytes) or 4 (8 bytes)
 __global__ void __launch_bounds__(256)
 nchw_to_nhwc8_bordered_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int h, int w,
                               int pad_h, int pad_w, int hp, int wp, int64_t total) {
@@ -248,14 +249,16 @@ nchw_to_nhwc8_bordered_kernel(const uint16_t* __restrict__ src, uint16_t* __rest
     if (ih >= 0 && ih < h && iw >= 0 && iw < w) {
       const uint16_t* s = src + n * c * hw + (int64_t)ih * w + iw;
 #pragma unroll
-      for (int ch = 0; ch < 8; ++ch)
+      for (int ch = 0; ch < PC; ++ch)
         if (ch < c) o[ch >> 1] |= (uint32_t)s[ch * hw] << ((ch & 1) * 16);
     }
-    *reinterpret_cast<uint4*>(dst + i * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+    if (PC == 8) *reinterpret_cast<uint4*>(dst + i * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+    else *reinterpret_cast<uint2*>(dst + i * 4) = make_uint2(o[0], o[1]);
   }
 }
 
 // w[k][c][r][s] (c <= 8) -> w'[k][r][kw_pix][8]: tap s, channel ch at [s][ch]; zeros elsewhere.
+template <int PC>  // channels per pixel of the window: 8 or 4
 __global__ void weights_repack_window_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst,
                                              int64_t k, int c, int r, int s, int kw_pix, int perm) {
   grid_dependency_wait();
@@ -268,11 +271,12 @@ __global__ void weights_repack_window_kernel(const uint16_t* __restrict__ src, u
     uint32_t o[4] = {0, 0, 0, 0};
     if (sp < s) {
 #pragma unroll
-      for (int ch = 0; ch < 8; ++ch)
+      for (int ch = 0; ch < PC; ++ch)
         if (ch < c)
           o[ch >> 1] |= (uint32_t)src[((row_channel(kk, perm) * c + ch) * r + rr) * s + sp] << ((ch & 1) * 16);
     }
-    *reinterpret_cast<uint4*>(dst + i * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+    if (PC == 8) *reinterpret_cast<uint4*>(dst + i * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+    else *reinterpret_cast<uint2*>(dst + i * 4) = make_uint2(o[0], o[1]);
   }
 }
 
@@ -385,22 +389,31 @@ __global__ void weights_repack_patch_kernel(const uint16_t* __restrict__ src, ui
 }  // namespace
 
 cudaError_t launch_nchw_to_nhwc8_bordered(const __half* src, __half* dst, int32_t n, int32_t c, int32_t h, int32_t w,
-                                          int32_t pad_h, int32_t pad_w, int32_t hp, int32_t wp, cudaStream_t stream) {
+                                          int32_t pad_h, int32_t pad_w, int32_t hp, int32_t wp, cudaStream_t stream,
+                                          int px_ch) {
   const int64_t total = (int64_t)n * hp * wp;
   int64_t blocks = (total + 255) / 256;
   if (blocks > 148 * 32) blocks = 148 * 32;
-  launch_kernel(nchw_to_nhwc8_bordered_kernel, dim3((unsigned)blocks), dim3(256), 0, stream, 
+  if (px_ch == 4)
+    launch_kernel(nchw_to_nhwc8_bordered_kernel<4>, dim3((unsigned)blocks), dim3(256), 0, stream,
+        reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), c, h, w, pad_h, pad_w, hp, wp, total);
+  else
+  launch_kernel(nchw_to_nhwc8_bordered_kernel<8>, dim3((unsigned)blocks), dim3(256), 0, stream, 
       reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), c, h, w, pad_h, pad_w, hp, wp, total);
   count_launch();
   return cudaGetLastError();
 }
 
 cudaError_t launch_weights_repack_window(const __half* src, __half* dst, int32_t k, int32_t c, int32_t r, int32_t s,
-                                         int32_t kw_pix, cudaStream_t stream, int perm) {
+                                         int32_t kw_pix, cudaStream_t stream, int perm, int px_ch) {
   const int64_t total = (int64_t)k * r * kw_pix;
   int64_t blocks = (total + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
-  launch_kernel(weights_repack_window_kernel, dim3((unsigned)blocks), dim3(256), 0, stream, 
+  if (px_ch == 4)
+    launch_kernel(weights_repack_window_kernel<4>, dim3((unsigned)blocks), dim3(256), 0, stream,
+        reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), k, c, r, s, kw_pix, perm);
+  else
+  launch_kernel(weights_repack_window_kernel<8>, dim3((unsigned)blocks), dim3(256), 0, stream, 
       reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), k, c, r, s, kw_pix, perm);
   count_launch();
   return cudaGetLastError();
@@ -529,7 +542,7 @@ cudaError_t launch_weights_repack_patch(const __half* src, __half* dst, int32_t 
 cudaError_t launch_igemm_weights(const ConvGeom& g, const IgemmPlan& p, const __half* w, __half* wp,
                                  cudaStream_t stream) {
   if (p.patch) return launch_weights_repack_patch(w, wp, g.k, g.c, g.r, g.s, p.cw, stream, p.y_perm);
-  if (p.window) return launch_weights_repack_window(w, wp, g.k, g.c, g.r, g.s, p.kw_pix, stream, p.y_perm);
+  if (p.window) return launch_weights_repack_window(w, wp, g.k, g.c, g.r, g.s, p.kw_pix, stream, p.y_perm, p.px_ch);
   return launch_weights_repack(w, wp, g.k, g.cg, g.r, g.s, g.group, p.cw, stream, p.y_perm);
 }
 
@@ -537,7 +550,7 @@ cudaError_t launch_igemm_input(const ConvGeom& g, const IgemmPlan& p, const __ha
                                cudaStream_t stream) {
   if (p.nchw || p.x_nhwc) return cudaSuccess;  // the kernel reads x itself
   if (p.patch) return launch_patch_im2col(g, x, xp, p.cw, stream);
-  if (p.window) return launch_nchw_to_nhwc8_bordered(x, xp, g.n, g.c, g.h, g.w, g.pad_h, g.pad_w, p.hp, p.wp, stream);
+  if (p.window) return launch_nchw_to_nhwc8_bordered(x, xp, g.n, g.c, g.h, g.w, g.pad_h, g.pad_w, p.hp, p.wp, stream, p.px_ch);
   return launch_nchw_to_nhwc(x, xp, g.n, g.c, g.h, g.w, p.c_pad, stream);
 }
 

@@ -49,6 +49,17 @@ CASES = [
     ("stem 3x3 c3 stride 1 (windows)", params_dict(2, 3, 32, 40, 16, 3, 3, 1, 1), X_WINDOWS),
     ("stem 7x7 c3 stride 2 (windows)", params_dict(2, 3, 64, 64, 64, 7, 7, 3, 3, 2, 2), X_WINDOWS),
     ("stem 11x11 c3 stride 4 (windows)", params_dict(1, 3, 67, 67, 96, 11, 11, 0, 0, 4, 4), X_WINDOWS),
+    ("stem 7x7 c3 stride 2, 224 wide (dense rows of 4-channel pixels, two rows per tile)",
+     params_dict(2, 3, 20, 224, 64, 7, 7, 3, 3, 2, 2), X_WINDOWS),
+    ("stem 5x5 c4 stride 2 (dense rows of 4-channel pixels)", params_dict(2, 4, 37, 45, 40, 5, 5, 2, 2, 2, 2), X_WINDOWS),
+    ("stem 7x7 c3 stride 1 along H, 2 along W", params_dict(2, 3, 30, 50, 24, 7, 7, 3, 3, 1, 2), X_WINDOWS),
+    ("stem 7x7 c1 stride 1 along H, 2 along W (49 values under the kernel: patches)",
+     params_dict(2, 1, 30, 50, 24, 7, 7, 3, 3, 1, 2), X_PATCHES),
+    ("stem 9x9 c3 stride 2 (64-element windows)", params_dict(1, 3, 41, 41, 32, 9, 9, 4, 4, 2, 2), X_WINDOWS),
+    ("stem 5x5 c5 stride 2 (8-channel pixels: one request per window)", params_dict(2, 5, 33, 33, 16, 5, 5, 2, 2, 2, 2), X_WINDOWS),
+    ("stem 5x5 c3 stride 1 (dense rows, shared kernel rows)", params_dict(2, 3, 30, 70, 48, 5, 5, 2, 2), X_WINDOWS),
+    ("stem 3x3 c8 stride 1, 250 wide (dense rows at the column limit)", params_dict(1, 8, 9, 250, 16, 3, 3, 1, 1), X_WINDOWS),
+    ("stem 3x3 c3 stride 1, 256 wide (rows too wide for the dense form)", params_dict(1, 3, 6, 256, 16, 3, 3, 1, 1), X_WINDOWS),
     ("stem 3x3 c3 stride 2 (patches)", params_dict(2, 3, 64, 48, 32, 3, 3, 1, 1, 2, 2), X_PATCHES),
     ("stem 3x3 c1 stride 2 (patches)", params_dict(3, 1, 33, 31, 24, 3, 3, 1, 1, 2, 2), X_PATCHES),
     ("stem 3x3 c4 stride 2 dilated (patches)", params_dict(2, 4, 30, 30, 20, 3, 3, 2, 2, 2, 2, 2, 2), X_PATCHES),
