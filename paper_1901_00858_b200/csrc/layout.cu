@@ -257,6 +257,59 @@ nchw_to_nhwc8_bordered_kernel(const uint16_t* __restrict__ src, uint16_t* __rest
   }
 }
 
+// The same copy for rows that are whole 16-byte vectors (w % 8 == 0): a thread takes 8 consecutive
+// pixels of one input row, one 16-byte load per channel, transposes them in registers and writes
+// the 8 pixels (PC * 2 bytes each, contiguous); the last slot of every output row writes the zero
+// columns left and right of the image, and slots of rows above and below the image write zeros.
+// 8x the bytes in flight per thread of the one-pixel form, which is bound by latency.
+template <int PC>
+__global__ void __launch_bounds__(256)
+nchw_to_nhwc8_bordered_vec_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int h, int w,
+                                  int pad_h, int pad_w, int hp, int wp, int64_t items) {
+  grid_dependency_wait();
+  const int slots = w / 8 + 1;
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= items) return;
+  const int slot = (int)(i % slots);
+  const int64_t t = i / slots;
+  const int oh = (int)(t % hp);
+  const int64_t n = t / hp;
+  uint16_t* drow = dst + (n * hp + oh) * (int64_t)wp * PC;
+  auto store_px = [&](int ow, uint32_t o0, uint32_t o1, uint32_t o2, uint32_t o3) {
+    if (PC == 8) *reinterpret_cast<uint4*>(drow + (int64_t)ow * 8) = make_uint4(o0, o1, o2, o3);
+    else *reinterpret_cast<uint2*>(drow + (int64_t)ow * 4) = make_uint2(o0, o1);
+  };
+  if (slot == slots - 1) {  // the zero columns of this row
+    for (int ow = 0; ow < pad_w; ++ow) store_px(ow, 0u, 0u, 0u, 0u);
+    for (int ow = pad_w + w; ow < wp; ++ow) store_px(ow, 0u, 0u, 0u, 0u);
+    return;
+  }
+  const int ih = oh - pad_h;
+  const int ow0 = pad_w + slot * 8;
+  if (ih < 0 || ih >= h) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) store_px(ow0 + j, 0u, 0u, 0u, 0u);
+    return;
+  }
+  uint4 v[PC];
+#pragma unroll
+  for (int ch = 0; ch < PC; ++ch)
+    v[ch] = ch < c ? __ldcs(reinterpret_cast<const uint4*>(src + ((n * c + ch) * h + ih) * (int64_t)w) + slot)
+                   : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    uint32_t o[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int k = 0; k < PC / 2; ++k) {
+      const uint4 a4 = v[2 * k], b4 = v[2 * k + 1];
+      const uint32_t a = (j >> 1) == 0 ? a4.x : ((j >> 1) == 1 ? a4.y : ((j >> 1) == 2 ? a4.z : a4.w));
+      const uint32_t b = (j >> 1) == 0 ? b4.x : ((j >> 1) == 1 ? b4.y : ((j >> 1) == 2 ? b4.z : b4.w));
+      o[k] = __byte_perm(a, b, (j & 1) ? 0x7632 : 0x5410);
+    }
+    store_px(ow0 + j, o[0], o[1], o[2], o[3]);
+  }
+}
+
 // w[k][c][r][s] (c <= 8) -> w'[k][r][kw_pix][8]: tap s, channel ch at [s][ch]; zeros elsewhere.
 template <int PC>  // channels per pixel of the window: 8 or 4
 __global__ void weights_repack_window_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst,
@@ -392,6 +445,22 @@ cudaError_t launch_nchw_to_nhwc8_bordered(const __half* src, __half* dst, int32_
                                           int32_t pad_h, int32_t pad_w, int32_t hp, int32_t wp, cudaStream_t stream,
                                           int px_ch) {
   const int64_t total = (int64_t)n * hp * wp;
+  if ((w % 8) == 0) {
+    const int64_t items = (int64_t)n * hp * (w / 8 + 1);
+    const int64_t vblocks = (items + 255) / 256;
+    if (vblocks <= 0x7fffffffLL) {
+      const uint16_t* s16 = reinterpret_cast<const uint16_t*>(src);
+      uint16_t* d16 = reinterpret_cast<uint16_t*>(dst);
+      if (px_ch == 4)
+        launch_kernel(nchw_to_nhwc8_bordered_vec_kernel<4>, dim3((unsigned)vblocks), dim3(256), 0, stream, s16, d16, c,
+                      h, w, pad_h, pad_w, hp, wp, items);
+      else
+        launch_kernel(nchw_to_nhwc8_bordered_vec_kernel<8>, dim3((unsigned)vblocks), dim3(256), 0, stream, s16, d16, c,
+                      h, w, pad_h, pad_w, hp, wp, items);
+      count_launch();
+      return cudaGetLastError();
+    }
+  }
   int64_t blocks = (total + 255) / 256;
   if (blocks > 148 * 32) blocks = 148 * 32;
   if (px_ch == 4)
