@@ -494,6 +494,96 @@ depthwise3x3_nhwc_kernel(const uint16_t* __restrict__ x, const uint16_t* __restr
   }
 }
 
+// 28x28 and 14x14 planes (pad 1, stride 1 or 2): a lane owns one 4-byte column word (two pixels) of
+// one plane and walks down its rows; 32 / (W/2) planes share a warp, so every load and store
+// instruction of a warp covers whole contiguous rows (the one-row-per-thread form above reads with
+// a stride of one row between lanes, which costs an L1 wavefront per lane or two).  All H words of
+// the column are loaded up front; the pixel left of the word and the pixel right of it come from
+// the neighbouring lanes by shuffle (zero at the plane's edge).
+template <int W, int S>
+__global__ void __launch_bounds__(256)
+depthwise3x3_colword_kernel(const uint16_t* __restrict__ x, const __half* __restrict__ w,
+                            const __half* __restrict__ bias, uint16_t* __restrict__ y, int c, int relu,
+                            int64_t planes) {
+  grid_dependency_wait();
+  constexpr int WORDS = W / 2;         // column words per row
+  constexpr int PPW = 32 / WORDS;      // planes per warp
+  constexpr int H = W;
+  const int lane = (int)(threadIdx.x & 31u);
+  const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int pl = lane / WORDS, e = lane - pl * WORDS;
+  const int64_t plane = warp * PPW + pl;
+  const bool live = pl < PPW && plane < planes;
+  const int ch = live ? (int)(plane % c) : 0;
+  uint16_t wv[9];
+#pragma unroll
+  for (int i = 0; i < 9; ++i) wv[i] = __half_as_ushort(__ldg(w + (int64_t)ch * 9 + i));
+  const float bv = bias != nullptr ? __half2float(__ldg(bias + ch)) : 0.f;
+  const uint32_t* xp = reinterpret_cast<const uint32_t*>(x) + (live ? plane : 0) * (H * WORDS) + e;
+  uint32_t v[H];
+#pragma unroll
+  for (int r = 0; r < H; ++r) v[r] = live ? __ldg(xp + r * WORDS) : 0u;
+  // per row: (pixel left of the word, pixel right of it)
+  uint32_t lr[H];
+#pragma unroll
+  for (int r = 0; r < H; ++r) {
+    const uint32_t up = __shfl_up_sync(0xffffffffu, v[r], 1);
+    const uint32_t dn = __shfl_down_sync(0xffffffffu, v[r], 1);
+    const uint32_t left = e > 0 ? (up >> 16) : 0u;
+    const uint32_t right = e < WORDS - 1 ? (dn & 0xffffu) : 0u;
+    lr[r] = left | (right << 16);
+  }
+  if constexpr (S == 2) {
+    // stride 2: the lane's word holds input columns 2e and 2e+1, so it owns output column e
+    // (columns 2e-1, 2e, 2e+1) of output rows p (input rows 2p-1, 2p, 2p+1); 2-byte stores
+    constexpr int Q = W / 2;
+    uint16_t* yh = y + (live ? plane : 0) * (Q * Q) + e;
+#pragma unroll
+    for (int p = 0; p < Q; ++p) {
+      float a0 = bv;
+#pragma unroll
+      for (int rr = 0; rr < 3; ++rr) {
+        const int r = 2 * p - 1 + rr;
+        if (r < 0 || r >= H) continue;
+        uint16_t lo, hi, lf, rt;
+        asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(v[r]));
+        asm("mov.b32 {%0, %1}, %2;" : "=h"(lf), "=h"(rt) : "r"(lr[r]));
+        asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(a0) : "h"(lf), "h"(wv[rr * 3 + 0]));
+        asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(a0) : "h"(lo), "h"(wv[rr * 3 + 1]));
+        asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(a0) : "h"(hi), "h"(wv[rr * 3 + 2]));
+      }
+      if (relu) a0 = fmaxf(a0, 0.f);
+      if (live) yh[p * Q] = __half_as_ushort(__float2half_rn(a0));
+    }
+    return;
+  }
+  uint32_t* yp = reinterpret_cast<uint32_t*>(y) + (live ? plane : 0) * (H * WORDS) + e;
+#pragma unroll
+  for (int p = 0; p < H; ++p) {
+    float a0 = bv, a1 = bv;
+#pragma unroll
+    for (int rr = 0; rr < 3; ++rr) {
+      const int r = p - 1 + rr;
+      if (r < 0 || r >= H) continue;
+      uint16_t lo, hi, lf, rt;
+      asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(v[r]));
+      asm("mov.b32 {%0, %1}, %2;" : "=h"(lf), "=h"(rt) : "r"(lr[r]));
+      asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(a0) : "h"(lf), "h"(wv[rr * 3 + 0]));
+      asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(a0) : "h"(lo), "h"(wv[rr * 3 + 1]));
+      asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(a0) : "h"(hi), "h"(wv[rr * 3 + 2]));
+      asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(a1) : "h"(lo), "h"(wv[rr * 3 + 0]));
+      asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(a1) : "h"(hi), "h"(wv[rr * 3 + 1]));
+      asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(a1) : "h"(rt), "h"(wv[rr * 3 + 2]));
+    }
+    uint32_t o;
+    if (relu)
+      asm("cvt.rn.relu.f16x2.f32 %0, %1, %2;" : "=r"(o) : "f"(a1), "f"(a0));
+    else
+      asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(o) : "f"(a1), "f"(a0));
+    if (live) yp[p * WORDS] = o;
+  }
+}
+
 // shapes the small-row kernel takes
 bool smallrow_ok(const ConvGeom& g) {
   if (g.pad_h != 1 || g.pad_w != 1) return false;
@@ -622,6 +712,26 @@ cudaError_t launch_depthwise3x3(const ConvGeom& g, const __half* x, const __half
       else
         launch_kernel(depthwise3x3_rowvec_kernel<2, 2>, dim3((unsigned)blocks), dim3(256), 0, stream, xs0, w, bias, ys0, g.c, g.h, g.w, g.p,
                                                                                g.q, relu, items, vec_per_row, strips);
+      count_launch();
+      return cudaGetLastError();
+    }
+  }
+  if (smallrow_ok(g) && (g.w == 28 || g.w == 14) && g.h == g.w) {
+    const int64_t planes = (int64_t)g.n * g.c;
+    const int ppw = g.w == 28 ? 2 : 4;
+    const int64_t warps = (planes + ppw - 1) / ppw;
+    const int64_t blocks = (warps + 7) / 8;
+    if (blocks < 0x7fffffffLL) {
+      const uint16_t* xs0 = reinterpret_cast<const uint16_t*>(x);
+      uint16_t* ys0 = reinterpret_cast<uint16_t*>(y);
+#define HGC_DW_COLWORD(WV, SV)                                                                                   \
+  launch_kernel(depthwise3x3_colword_kernel<WV, SV>, dim3((unsigned)blocks), dim3(256), 0, stream, xs0, w, bias, ys0, \
+                g.c, relu, planes)
+      if (g.w == 28 && g.stride_h == 1) HGC_DW_COLWORD(28, 1);
+      else if (g.w == 28) HGC_DW_COLWORD(28, 2);
+      else if (g.stride_h == 1) HGC_DW_COLWORD(14, 1);
+      else HGC_DW_COLWORD(14, 2);
+#undef HGC_DW_COLWORD
       count_launch();
       return cudaGetLastError();
     }

@@ -110,6 +110,22 @@ def test_depthwise_planes(hgc, oracle, plane, stride):
         check_close(got2, oracle.conv_fast(oracle.ConvParams(**a), x, w, None, False), what="dw no bias")
 
 
+@pytest.mark.parametrize("plane", [14, 28])
+@pytest.mark.parametrize("stride", [1, 2])
+def test_depthwise_square_small_planes(hgc, oracle, plane, stride):
+    """The 28x28 and 14x14 planes of MobileNet (one column word per lane, several planes per
+    warp): a plane count that leaves the last warp partly filled, with and without bias/ReLU."""
+    rng = np.random.default_rng(500 + plane + stride)
+    n, c = 3, 37
+    a = params_dict(n, c, plane, plane, c, 3, 3, 1, 1, stride, stride, 1, 1, c)
+    x, w, b = workloads.random_layer_tensors(rng, n, c, plane, plane, c, 3, 3, c)
+    for relu, bias in ((True, b), (False, None), (False, b)):
+        ref = oracle.conv_fast(oracle.ConvParams(**a), x, w, bias, relu)
+        got, path = run_layer(hgc, a, x, w, bias, relu)
+        assert path == hgc.HGC_PATH_DEPTHWISE
+        check_close(got, ref, what=f"dw square {plane} stride {stride} relu={relu}")
+
+
 @pytest.mark.parametrize("h,w,stride", [(56, 56, 1), (112, 112, 1), (24, 40, 1), (9, 8, 1), (56, 56, 2), (112, 112, 2),
                                         (40, 24, 2), (16, 8, 2), (30, 72, 2)])
 def test_depthwise_row_vector_shapes(hgc, oracle, h, w, stride):
