@@ -242,9 +242,23 @@ def run_ours(args, wl):
     gen = torch.Generator(device="cuda")
     gen.manual_seed(1234 + rank)
     state = []
+    n_cl_in = n_cl_out = 0
     for li, l in enumerate(layers):
-        d = hgc.ConvDesc(batch, l.c, l.h, l.h, l.k, l.r, l.r, l.pad, l.pad, l.stride, l.stride, l.dil, l.dil,
-                         l.group)
+        geo = (batch, l.c, l.h, l.h, l.k, l.r, l.r, l.pad, l.pad, l.stride, l.stride, l.dil, l.dil, l.group)
+        if args.layout == "channels_last":
+            # every layer that can takes both flags; a layer that cannot read channels-last input
+            # (3-channel stems) takes the output flag alone; the buffers keep their sizes
+            d = None
+            for fl in (hgc.HGC_FLAG_X_NHWC | hgc.HGC_FLAG_Y_NHWC, hgc.HGC_FLAG_Y_NHWC, 0):
+                try:
+                    d = hgc.ConvDesc(*geo, fl)
+                    break
+                except hgc.HgcError:
+                    continue
+            n_cl_in += 1 if fl & hgc.HGC_FLAG_X_NHWC else 0
+            n_cl_out += 1 if fl & hgc.HGC_FLAG_Y_NHWC else 0
+        else:
+            d = hgc.ConvDesc(*geo)
         d.ensure_workspace()
         x = torch.empty((batch, l.c, l.h, l.h), dtype=torch.float16, device="cuda")
         x.uniform_(l.x_lo, 1.0, generator=gen)
@@ -345,7 +359,7 @@ def run_ours(args, wl):
     # activations channels-last between layers pays per step.  Layers that cannot take a flag
     # (3-channel stems on the input side, depthwise layers) keep NCHW on that side.
     nhwc = None
-    if not args.no_graph:
+    if not args.no_graph and args.layout == "nchw":
         try:
             nstate, n_in, n_out = [], 0, 0
             for (d0, x, w, b, y, l) in state:
@@ -469,7 +483,9 @@ def run_ours(args, wl):
                        "layers": len(layers), "batch_per_gpu": batch,
                        "l2": "inputs larger than L2 (every layer has its own tensors)",
                        "launch": "cuda_graph" if graph is not None else "eager",
-                       "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
+                       "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                       **({"layout": f"channels_last ({n_cl_in} of {len(layers)} layers read, {n_cl_out} write "
+                                     "channels-last activations)"} if args.layout == "channels_last" else {})},
             "images_per_s": agg["images_per_s"],
             "roofline": roof,
             "roofline_config": {"t_roof_ms": t_roof * 1e3, "frac": t_roof * 1e3 / (sum(layer_ms)),
@@ -628,6 +644,9 @@ def main():
                          "inner-product layer and the batch-norm layer, measured on their own")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD,
                     help="one of: " + ", ".join(w.name for w in workloads.all_workloads()))
+    ap.add_argument("--layout", choices=["nchw", "channels_last"], default="nchw",
+                    help="nchw: the metric's configuration (default). channels_last: the same layers with "
+                         "HGC_FLAG_X_NHWC / HGC_FLAG_Y_NHWC where a layer takes them (a chained stack)")
     ap.add_argument("--layers", action="store_true", help="add per-layer figures to the JSON line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of replaying the step as a CUDA graph")
