@@ -84,7 +84,9 @@ int forward_impl(hgc_conv_desc* d, const void* x, const void* w, const void* bia
       break;
     }
     case HGC_PATH_DEPTHWISE:
-      err = g.x_nhwc ? hgc::launch_depthwise3x3_nhwc(g, xh, wh, bh, yh, relu, stream)
+      err = g.x_nhwc ? (hgc::depthwise3x3_nhwc_tma_supported(g)
+                            ? hgc::launch_depthwise3x3_nhwc_tma(g, xh, wh, bh, yh, relu, stream)
+                            : hgc::launch_depthwise3x3_nhwc(g, xh, wh, bh, yh, relu, stream))
                      : hgc::launch_depthwise3x3(g, xh, wh, bh, yh, relu, stream);
       break;
     case HGC_PATH_DIRECT:
@@ -279,6 +281,12 @@ int hgc_conv_last_device_status(hgc_conv_desc* d, int32_t* status) {
       *status = word;
       if (cudaMemset(sp, 0, sizeof(word)) != cudaSuccess) return HGC_CUDA_ERROR;
     }
+  }
+  // the TMA-fed channels-last depthwise kernel keeps one status word per process
+  if (d->path == HGC_PATH_DEPTHWISE && d->geom.x_nhwc && hgc::depthwise3x3_nhwc_tma_supported(d->geom)) {
+    const int v = hgc::depthwise_nhwc_tma_status();
+    if (v < 0) return HGC_CUDA_ERROR;
+    if (v != 0) *status = HGC_DEVICE_TIMEOUT;
   }
   return HGC_OK;
 }

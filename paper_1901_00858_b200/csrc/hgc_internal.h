@@ -74,6 +74,13 @@ bool depthwise3x3_nhwc_supported(const ConvGeom& g);
 cudaError_t launch_depthwise3x3_nhwc(const ConvGeom& g, const __half* x, const __half* w, const __half* bias,
                                      __half* y, int relu, cudaStream_t stream);
 
+// ... and its TMA-fed form (stride 1, C % 32 == 0); the status is 0, or 1 after a copy that never
+// arrived (reading it synchronises with the device and clears it)
+bool depthwise3x3_nhwc_tma_supported(const ConvGeom& g);
+cudaError_t launch_depthwise3x3_nhwc_tma(const ConvGeom& g, const __half* x, const __half* w, const __half* bias,
+                                         __half* y, int relu, cudaStream_t stream);
+int depthwise_nhwc_tma_status();
+
 cudaError_t launch_nchw_to_nhwc(const __half* src, __half* dst, int32_t n, int32_t c, int32_t h,
                                 int32_t w, int32_t c_pad, cudaStream_t stream);
 cudaError_t launch_nhwc_to_nchw(const __half* src, __half* dst, int32_t n, int32_t c, int32_t h,

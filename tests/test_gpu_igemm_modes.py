@@ -202,6 +202,10 @@ DW_NHWC_CASES = [
     ("odd plane 13x9 c24, ragged strips", params_dict(2, 24, 13, 9, 24, 3, 3, 1, 1, 1, 1, 1, 1, 24)),
     ("15x15 stride 2 c40", params_dict(1, 40, 15, 15, 40, 3, 3, 1, 1, 2, 2, 1, 1, 40)),
     ("no padding 10x12 c16", params_dict(2, 16, 10, 12, 16, 3, 3, 0, 0, 1, 1, 1, 1, 16)),
+    ("c64 odd plane 37x21 (TMA-fed, ragged tiles)", params_dict(2, 64, 37, 21, 64, 3, 3, 1, 1, 1, 1, 1, 1, 64)),
+    ("c96 no padding 20x50 (TMA-fed, three 32-channel blocks)", params_dict(3, 96, 20, 50, 96, 3, 3, 0, 0, 1, 1, 1, 1, 96)),
+    ("c128 padding 2, 33x40 (TMA-fed)", params_dict(1, 128, 33, 40, 128, 3, 3, 2, 2, 1, 1, 1, 1, 128)),
+    ("c32 56x56 many tiles per block (TMA-fed)", params_dict(8, 32, 56, 56, 32, 3, 3, 1, 1, 1, 1, 1, 1, 32)),
     ("padding 2, stride 2, 9x11 c8", params_dict(2, 8, 9, 11, 8, 3, 3, 2, 2, 2, 2, 1, 1, 8)),
 ]
 
@@ -222,6 +226,7 @@ def test_depthwise_channels_last(hgc, oracle, name, a):
         hgc.conv_forward(d, xd, wd, bias_d, y, relu)
         torch.cuda.synchronize()
         check_close(np.ascontiguousarray(to_host(y).transpose(0, 3, 1, 2)), ref, what=f"{name} relu={relu}")
+    assert d.last_device_status() == hgc.HGC_OK
     d.close()
 
 
