@@ -194,7 +194,9 @@ int hgc_conv_set_workspace(hgc_conv_desc* d, void* dev_ptr, size_t bytes);
 int hgc_conv_set_weights(hgc_conv_desc* d, const void* w, void* stream);
 
 /* Reads the device status word of the descriptor's last forward (synchronises `stream`
-   work that was queued by this descriptor).  *status is HGC_OK or HGC_DEVICE_TIMEOUT. */
+   work that was queued by this descriptor).  *status is HGC_OK or HGC_DEVICE_TIMEOUT.
+   Channels-last depthwise layers share one status word per process (set by any of them,
+   cleared when read). */
 int hgc_conv_last_device_status(hgc_conv_desc* d, int32_t* status);
 
 /*
