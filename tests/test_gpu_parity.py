@@ -238,6 +238,51 @@ def test_configs_full_size_channels_last_sampled(hgc, oracle, cfg, batch):
         del xd, wd, bd, y
 
 
+@pytest.mark.parametrize("kind", ["tensor cores", "channels-last", "depthwise", "depthwise channels-last",
+                                  "1x1 reading x in place"])
+def test_tensors_of_more_than_2_31_elements(hgc, oracle, kind):
+    """Maximum sizes: 700 (1400) images of 224x224, x and y of 2.25 G elements (4.5 GB) each, so every
+    flat index beyond the first 2^31 elements needs 64-bit arithmetic.  Inputs are generated on the
+    device; the oracle evaluates sampled outputs including the last ones."""
+    import torch
+    n, c, k, r, pad, group = 700, 64, 64, 3, 1, 1
+    if kind.startswith("depthwise"):
+        group = 64
+    if kind.startswith("1x1"):
+        n, c, k, r, pad = 1400, 32, 32, 1, 0
+    cl = "channels-last" in kind
+    a = params_dict(n, c, 224, 224, k, r, r, pad, pad, 1, 1, 1, 1, group)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(11)
+    x = torch.empty((n, c, 224, 224), dtype=torch.float16, device="cuda").uniform_(0, 1, generator=g)
+    w = (torch.randn((k, c // group, r, r), device="cuda", generator=g) * float(np.sqrt(2.0 / (c // group * r * r)))).to(torch.float16)
+    b = torch.empty(k, dtype=torch.float16, device="cuda").uniform_(-0.1, 0.1, generator=g)
+    assert x.numel() > 2 ** 31
+    d = hgc.ConvDesc(flags=(hgc.HGC_FLAG_X_NHWC | hgc.HGC_FLAG_Y_NHWC) if cl else 0, **a)
+    assert d.path() == (hgc.HGC_PATH_DEPTHWISE if group > 1 else hgc.HGC_PATH_IGEMM)
+    d.ensure_workspace()
+    nn, kk, p, q = d.output_dims()
+    y = torch.full((nn, p, q, kk) if cl else (nn, kk, p, q), float("nan"), dtype=torch.float16, device="cuda")
+    xin = x.permute(0, 2, 3, 1).contiguous() if cl else x
+    hgc.conv_forward(d, xin, w, b, y, True)
+    torch.cuda.synchronize()
+    del xin
+    assert d.last_device_status() == hgc.HGC_OK
+    assert bool(torch.isfinite(y).all())
+    rng = np.random.default_rng(5)
+    pts = np.stack([rng.integers(0, nn, 4000), rng.integers(0, kk, 4000), rng.integers(0, p, 4000),
+                    rng.integers(0, q, 4000)], 1).astype(np.int64)
+    pts[:6] = [[nn - 1, kk - 1, p - 1, q - 1], [nn - 1, 0, 0, 0], [0, kk - 1, p - 1, 0], [nn - 1, kk - 1, 0, q - 1],
+               [nn // 2 + 1, kk // 2, p // 2, q // 2], [0, 0, 0, 0]]
+    ref = oracle.conv_points(oracle.ConvParams(**a), x.cpu().numpy(), w.cpu().numpy(), b.cpu().numpy(), True, pts)
+    ct = torch.from_numpy(pts).cuda()
+    got = y[ct[:, 0], ct[:, 2], ct[:, 3], ct[:, 1]] if cl else y[ct[:, 0], ct[:, 1], ct[:, 2], ct[:, 3]]
+    check_close(to_host(got), ref, what=f"2^31 elements, {kind}")
+    d.close()
+    del x, y
+    torch.cuda.empty_cache()
+
+
 def test_forward_host_matches_device_forward(hgc, oracle):
     import torch
     rng = np.random.default_rng(4)
