@@ -156,3 +156,39 @@ def test_fold_matches_oracle_and_the_folded_convolution_normalises(hgc, oracle):
     # the folded weights carry one extra FP16 rounding each: a slightly wider band than a plain layer
     assert np.all(np.abs(got - want) <= 4e-3 + 1e-2 * np.abs(want))
     d.close()
+
+
+def test_batchnorm_on_more_than_2_31_elements(hgc, oracle):
+    """700 x 64 x 224 x 224 (2.25 G elements).  Every plane holds every value 0..255 equally
+    often, so the statistics have the closed form the oracle is pinned to (mean 255/2, variance
+    (256^2 - 1)/12) and every output is one of 256 values, which the oracle computes from those
+    statistics."""
+    import torch
+    n, c, h, w = 700, 64, 224, 224
+    hw = h * w
+    assert hw % 256 == 0 and n * c * hw > 2 ** 31
+    plane = (torch.arange(hw, device="cuda") % 256).to(torch.float16)
+    x = plane.expand(n, c, hw).contiguous().view(n, c, h, w)
+    y = torch.empty_like(x)
+    mean = torch.empty(c, dtype=torch.float32, device="cuda")
+    var = torch.empty(c, dtype=torch.float32, device="cuda")
+    ws = torch.empty(hgc.batchnorm_workspace_bytes(n, c, hw), dtype=torch.uint8, device="cuda")
+    hgc.batchnorm_forward(x, y, 1e-5, mean, var, ws, shift_log2=-5)
+    torch.cuda.synchronize()
+    m, v = mean.cpu().numpy().astype(np.float64), var.cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(m - 127.5) <= 127.5e-5) and np.all(np.abs(v - (256.0 ** 2 - 1) / 12) <= 2e-5 * 5461.25)
+    # the 256 possible outputs, from the oracle with the closed-form statistics
+    vals = np.arange(256, dtype=np.float64).reshape(1, 1, 16, 16).astype(np.float16)
+    table, _, _ = oracle.batchnorm(vals, 1e-5, np.array([127.5]), np.array([(256.0 ** 2 - 1) / 12]))
+    table = torch.from_numpy(table.reshape(256).view(np.int16)).cuda().view(torch.float16).float()
+    # sampled outputs, including the very last ones
+    g = torch.Generator(device="cuda")
+    g.manual_seed(3)
+    idx = torch.randint(0, n * c * hw, (200000,), device="cuda", generator=g)
+    idx[:4] = torch.tensor([n * c * hw - 1, n * c * hw - 2, 2 ** 31 + 5, 0], device="cuda")
+    got = y.view(-1)[idx].float()
+    ref = table[(idx % hw) % 256]
+    err = (got - ref).abs()
+    assert bool((err <= 2e-3 + 1e-2 * ref.abs()).all()), float(err.max())
+    del x, y
+    torch.cuda.empty_cache()
