@@ -103,3 +103,28 @@ def test_inner_product_keeps_a_wide_sum(hgc, oracle):
     torch.cuda.synchronize()
     assert torch.all(y == 4096).item()
     d.close()
+
+
+def test_cast_of_more_than_2_31_values(hgc, oracle):
+    """2^31 + 12345 values (8.6 GB in, 4.3 GB out): a sample of a million positions, the last ones
+    included, must carry exactly the oracle's bits (the tail after the last group of 8 too)."""
+    import torch
+    count = 2 ** 31 + 12345
+    g = torch.Generator(device="cuda")
+    g.manual_seed(9)
+    src = torch.empty(count, dtype=torch.float32, device="cuda").normal_(0, 300.0, generator=g)
+    src[-1] = 70000.0          # a finite value that overflows, at the very end
+    dst = torch.zeros(count, dtype=torch.float16, device="cuda")
+    over = torch.zeros(1, dtype=torch.int64, device="cuda")
+    hgc.cast_f32_to_f16(src, dst, overflow_count=over)
+    torch.cuda.synchronize()
+    idx = torch.randint(0, count, (1 << 20,), device="cuda", generator=g)
+    idx[:5] = torch.tensor([count - 1, count - 2, count - 9, 2 ** 31, 0], device="cuda")
+    sample = src[idx].cpu().numpy()
+    ref, _ = oracle.cast_f32_to_f16(sample)
+    got = dst[idx].cpu().numpy()
+    assert np.array_equal(got.view(np.uint16), ref.view(np.uint16))
+    assert int(over.item()) >= 1
+    assert bool(torch.isinf(dst[-1]))
+    del src, dst
+    torch.cuda.empty_cache()
