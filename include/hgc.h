@@ -76,6 +76,22 @@ typedef struct hgc_conv_params {
  */
 #define HGC_FLAG_X_NHWC 2
 #define HGC_FLAG_Y_NHWC 4
+/*
+ * Scheduling choices of the tensor-core path, off by default, for measurement and tests (the
+ * result is the same layer within the tolerance; the summation order over the input channels
+ * changes).  Both were built to lift what looked like the limits of the single-CTA kernel; on the
+ * measured layers, which run under the board's power cap, neither made a layer faster by more
+ * than a few per cent, so the planner does not choose them by itself.
+ * HGC_FLAG_CTA_PAIRS: layers with more than 128 output channels per group may be launched as CTA
+ * pairs (clusters of two SMs that share tiles of 256 output channels through tcgen05
+ * cta_group::2: each CTA fetches its own 128 weight rows and half of the activation tile).
+ * HGC_FLAG_SHARED_TILES: the ring stages of all tiles are dealt out in equal contiguous ranges,
+ * so that every CTA (or pair) gets the same amount of work; a tile that straddles a boundary is
+ * reduced by several CTAs inside the one launch (fp32 hand-over through the workspace, added in
+ * a fixed order: deterministic).  Such a launch is cooperative.
+ */
+#define HGC_FLAG_CTA_PAIRS 8
+#define HGC_FLAG_SHARED_TILES 16
 
 typedef struct hgc_conv_desc hgc_conv_desc; /* opaque; owned by the caller via create/destroy */
 
@@ -168,8 +184,14 @@ int hgc_conv_path(const hgc_conv_desc* d, int32_t* path);
  * overlapping windows (few input channels), 3 = an expanded copy holding, per output pixel, the
  * values under the kernel (few input channels, strided), [11] the number of CTAs that share
  * the reduction of one tile (1, or 2 / 4 / 8 for layers with very few tiles, e.g. inner products:
- * each CTA writes fp32 partial sums and a second kernel adds them in a fixed order); zeros for
- * the other paths.  info: host pointer.
+ * each CTA writes fp32 partial sums and a second kernel adds them in a fixed order), [12] the
+ * number of CTAs of the launch when the ring stages of all tiles are dealt out as contiguous
+ * ranges (0 with reduction slices), [13] 1 if those ranges are equal, so that a tile straddling a
+ * boundary is reduced by several CTAs inside the one launch (the CTA holding the tile's first
+ * stage adds the others' fp32 accumulators in a fixed order), 0 if every CTA takes whole tiles,
+ * [14] 1 if the launch consists of CTA pairs (clusters of two that share tiles of 256 output
+ * channels; [3], [4] then describe one CTA's pixel sub-tile, [6] the MMA N of the pair, [7] the
+ * number of pair tiles, [12] the number of pairs); zeros for the other paths.  info: host pointer.
  */
 int hgc_conv_plan_info(const hgc_conv_desc* d, int32_t* info, int32_t count);
 

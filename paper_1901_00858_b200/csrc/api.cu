@@ -131,6 +131,8 @@ int hgc_conv_desc_create(hgc_conv_desc** out, const hgc_conv_params* p) {
   g.cg = p->c / p->group; g.kg = p->k / p->group;
   g.x_nhwc = (p->flags & HGC_FLAG_X_NHWC) ? 1 : 0;
   g.y_nhwc = (p->flags & HGC_FLAG_Y_NHWC) ? 1 : 0;
+  g.no_pair = (p->flags & HGC_FLAG_CTA_PAIRS) ? 0 : 1;
+  g.no_split = (p->flags & HGC_FLAG_SHARED_TILES) ? 0 : 1;
   const bool channels_last = g.x_nhwc || g.y_nhwc;
 
   d->path = HGC_PATH_DIRECT;
@@ -212,15 +214,18 @@ int hgc_conv_path(const hgc_conv_desc* d, int32_t* path) {
 
 int hgc_conv_plan_info(const hgc_conv_desc* d, int32_t* info, int32_t count) {
   if (d == nullptr || info == nullptr || count < 1) return HGC_INVALID_ARG;
-  int32_t v[12] = {d->path, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+  int32_t v[15] = {d->path, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
   if (d->path == HGC_PATH_IGEMM) {
     const hgc::IgemmPlan& p = d->igemm;
     v[1] = p.kb; v[2] = p.halo; v[3] = p.tn; v[4] = p.th; v[5] = p.pitch; v[6] = p.ncols;
     v[7] = p.total_tiles; v[8] = p.stages; v[9] = p.taps;
     v[10] = (p.nchw || p.x_nhwc) ? 1 : (p.window ? 2 : (p.patch ? 3 : 0));
     v[11] = 1 << p.ks_log2;
+    v[12] = p.ks_log2 > 0 ? 0 : ((p.pair && p.pair_fit > 0 && p.pair_fit < p.grid) ? p.pair_fit : p.grid);
+    v[13] = p.sk_split;
+    v[14] = p.pair;
   }
-  for (int i = 0; i < count && i < 12; ++i) info[i] = v[i];
+  for (int i = 0; i < count && i < 15; ++i) info[i] = v[i];
   return HGC_OK;
 }
 
@@ -249,7 +254,7 @@ int hgc_conv_set_workspace(hgc_conv_desc* d, void* dev_ptr, size_t bytes) {
   if (d->path == HGC_PATH_IGEMM && dev_ptr != nullptr && bytes >= d->ws_needed) {
     // the TMA descriptors point into the workspace: encode them now; clear the status word
     if (!hgc::igemm_encode_maps(d->geom, &d->igemm, dev_ptr)) return HGC_CUDA_ERROR;
-    if (cudaMemset(static_cast<char*>(dev_ptr) + d->igemm.ws_status_off, 0, 256) != cudaSuccess)
+    if (cudaMemset(static_cast<char*>(dev_ptr) + d->igemm.ws_status_off, 0, hgc::kWsHeaderBytes) != cudaSuccess)
       return HGC_CUDA_ERROR;
   }
   return HGC_OK;
@@ -279,7 +284,8 @@ int hgc_conv_last_device_status(hgc_conv_desc* d, int32_t* status) {
     if (cudaMemcpy(&word, sp, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return HGC_CUDA_ERROR;
     if (word != 0) {
       *status = word;
-      if (cudaMemset(sp, 0, sizeof(word)) != cudaSuccess) return HGC_CUDA_ERROR;
+      // the launch that gave up may have left hand-over flags raised: clear the whole header
+      if (cudaMemset(sp, 0, hgc::kWsHeaderBytes) != cudaSuccess) return HGC_CUDA_ERROR;
     }
   }
   // the TMA-fed channels-last depthwise kernel keeps one status word per process

@@ -18,7 +18,15 @@ struct ConvGeom {
   int32_t p, q;    // output plane
   int32_t cg, kg;  // channels per group: C/group, K/group
   int32_t x_nhwc, y_nhwc;  // channels-last input / output (tensor-core path only)
+  int32_t no_split;        // 1: never let several CTAs share the reduction of a tile (no scratch for it)
+  int32_t no_pair;         // 1: never pair CTAs on 256-channel tiles
 };
+
+// First bytes of the tensor-core path's workspace: the device status word (int at byte 0) and,
+// from byte 256 on, one hand-over flag per CTA for tiles whose reduction several CTAs share.
+constexpr size_t kWsHeaderBytes = 1024;
+constexpr size_t kWsFlagsOff = 256;
+constexpr int kMaxGrid = 192;
 
 void count_launch();  // bumps the process-wide kernel launch counter
 
@@ -45,6 +53,25 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = launch_overlap_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// The same with the cooperative attribute when `cooperative` is set: the launch waits until every
+// CTA of the grid can be resident at once (kernels whose CTAs wait for one another).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel_coop(bool cooperative, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                      cudaStream_t stream, Args... args) {
+  if (!cooperative) return launch_kernel(kernel, grid, block, smem, stream, args...);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
@@ -131,7 +158,16 @@ struct IgemmPlan {
   int32_t a_rows;  // rows of a weight tile in shared memory (128, or 64 for layers of <= 64 channels per group)
   size_t smem_bytes;
   int32_t ks_log2;  // log2 of the number of reduction slices a tile is split into (0 = none)
-  size_t ws_status_off, ws_w_off, ws_x_off, ws_part_off, ws_total;
+  // work distribution of the kernels without reduction slices: `grid` CTAs take contiguous ranges
+  // of the ring stages of all tiles; sk_split = 1: equal ranges, a tile that straddles a boundary
+  // is reduced by several CTAs (fp32 hand-over through the workspace, sk_cols32 * 32 columns)
+  int32_t ts, grid, sk_split, sk_cols32;
+  // CTA pairs (clusters of two sharing 256-channel tiles): th/tn/tiles_h/tiles_n describe one
+  // CTA's pixel sub-tile, ncols = 2 * ncols_sub, grid counts pairs; pair_fit = pairs that can be
+  // resident at once (asked of the runtime at the first launch)
+  int32_t pair, ncols_sub, pair_fit;
+  double est_clk;  // the cost model's estimate for the launch, in SM clocks
+  size_t ws_status_off, ws_w_off, ws_x_off, ws_part_off, ws_sk_off, ws_total;
   bool maps_ready;
   alignas(64) CUtensorMap tmA;
   alignas(64) CUtensorMap tmB;

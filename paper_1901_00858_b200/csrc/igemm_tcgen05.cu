@@ -40,9 +40,9 @@ namespace {
 constexpr int kEpilogueWarps = 8;       // two per TMEM lane quarter (the default)
 constexpr int kEpilogueWarpsWide = 16;  // four per quarter: layers whose tiles are bound by the epilogue
 constexpr int kPassElems = 64;               // output pixels per channel staged per TMA store
-// one warp's staging tile: 32 channels x 64 pixels for the TMA-store epilogue (4 KB, 1024-byte
-// aligned), or 32 rows of 144 bytes for the row epilogue (4.5 KB)
-constexpr uint32_t kWarpStageBytes = 5120u;
+// one warp's staging tile: 32 channels x 64 pixels (or 64 pixels x 32 channels, or 32 rows of 32
+// floats): 4 KB, 1024-byte aligned
+constexpr uint32_t kWarpStageBytes = 4096u;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -153,11 +153,60 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
       : "memory");
 }
 
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1,
+                                            int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+      : "memory");
+}
+
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1,
                                             int c2, int c3, int c4) {
   asm volatile(
       "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
       ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
+      : "memory");
+}
+
+// The same copies issued by a CTA of a pair: the data lands in the issuing CTA's shared memory,
+// the bytes are counted on a barrier that may live in the other CTA of the pair (`bar` is a
+// shared::cluster address).  No multicast: every CTA fetches its own tiles.
+__device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1,
+                                                 int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tma_load_5d_pair(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1,
+                                                 int c2, int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+      ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
+      : "memory");
+}
+
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t cluster_addr(uint32_t local, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+  return r;
+}
+
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+      "h"((uint16_t)3)
       : "memory");
 }
 
@@ -186,6 +235,91 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t* v) {
                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
                : "r"(taddr)
                : "memory");
+}
+
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
+        "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
+        "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+      : "memory");
+}
+
+// Meeting point of the epilogue warps (one arrival per warp on an mbarrier initialised to their
+// number), with a bounded wait: false if it ran out or another role already gave up.  A plain
+// named barrier would hang the warps that reach it after others have left on a timeout.
+__device__ __forceinline__ bool epi_sync(uint32_t bar, uint32_t& phase, volatile int* abort_flag) {
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+  const bool ok = mbar_wait(bar, phase, abort_flag, 32);
+  phase ^= 1u;
+  __syncwarp();
+  return ok;
+}
+
+// A tile reduced by several CTAs (IgemmArgs::sk_split).  The accumulators travel as fp32 in the
+// order [column][128 lanes]: a warp's 32 lanes are 128 contiguous bytes per column.
+// sk_hand_over: this warp's lane quarter, column chunks `first`, `first + step`, ... -> slot.
+__device__ __noinline__ void sk_hand_over(uint32_t t_addr, int quarter, int first, int step, int cols32, float* slot) {
+  const int lane = threadIdx.x & 31;
+  float* dst = slot + quarter * 32 + lane;
+  for (int c = first; c < cols32; c += step) {
+    uint32_t v[32];
+    tmem_ld32(t_addr + (uint32_t)(c * 32), v);
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int j = 0; j < 32; ++j) __stcg(dst + (size_t)(c * 32 + j) * 128, __uint_as_float(v[j]));
+  }
+}
+
+// sk_take_over: adds the slots of CTAs first_cta, first_cta + cta_step, ... (count of them, in that
+// order: the sum does not depend on timing) to this CTA's accumulator, in place.  The tile is the
+// CTA's last piece of work, so the operand ring is idle: each slot is fetched into it with bulk
+// copies (pieces of `piece32` 32-column chunks, as many as the ring holds) and added from there.
+// Called by all epilogue warps, which meet on `meet_bar`; `leader` issues the copies.  False after a
+// wait that ran out.
+__device__ __noinline__ bool sk_take_over(uint32_t t_addr, int quarter, int first, int step, int cols32, bool live,
+                                          const float* slots, size_t slot_elems, int first_cta, int cta_step, int count,
+                                          uint32_t ring, int piece32, uint32_t copy_bar, uint32_t& copy_phase,
+                                          uint32_t meet_bar, uint32_t& meet_phase, bool leader, volatile int* abort_flag) {
+  const int lane = threadIdx.x & 31;
+  for (int i = 0; i < count; ++i) {
+    const float* slot = slots + (size_t)(first_cta + i * cta_step) * slot_elems;
+    for (int c0 = 0; c0 < cols32; c0 += piece32) {
+      const int nc = cols32 - c0 < piece32 ? cols32 - c0 : piece32;
+      // the previous piece has been added by everybody before it is overwritten
+      if (!epi_sync(meet_bar, meet_phase, abort_flag)) return false;
+      if (leader) {
+        const uint32_t bytes = (uint32_t)nc * 32u * 128u * 4u;
+        mbar_expect_tx(copy_bar, bytes);
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(ring),
+                     "l"(slot + (size_t)c0 * 32 * 128), "r"(bytes), "r"(copy_bar)
+                     : "memory");
+      }
+      if (!mbar_wait(copy_bar, copy_phase, abort_flag, 32)) return false;
+      copy_phase ^= 1u;
+      if (live) {
+        for (int c = first; c < nc; c += step) {
+          uint32_t v[32];
+          tmem_ld32(t_addr + (uint32_t)((c0 + c) * 32), v);
+          const uint32_t src = ring + (uint32_t)(c * 32 * 128 + quarter * 32 + lane) * 4u;
+          float add[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) asm volatile("ld.shared.f32 %0, [%1];" : "=f"(add[j]) : "r"(src + (uint32_t)j * 512u));
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + add[j]);
+          tmem_st32(t_addr + (uint32_t)((c0 + c) * 32), v);
+        }
+      }
+    }
+  }
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+  return true;
 }
 
 // two fp32 -> packed fp16x2 (round to nearest even), lo = first value; optional ReLU in the convert
@@ -229,7 +363,38 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap* tm, uint32_t src
 // elected lane (16 channels per step: +32 bytes = +2 in the descriptors' address field), commits
 // them to `a_bar` (and to `b_bar` if release_b), and returns the poll's result.  Warp-collective.
 // The poll is issued first and its answer read last, so its latency hides behind the MMA issue.
-template <int KSTEPS>
+// PAIR: the MMAs are those of a CTA pair (cta_group::2: 256 output channels, each CTA's tensor
+// core reads its own 128 weight rows and both halves of the activation tile) and the commits
+// arrive on the barriers at the same offsets in both CTAs.
+#define HGC_MMA_FIRST(CG) "@p_mma tcgen05.mma.cta_group::" CG ".kind::f16 [%3], %4, %5, %6, p_acc;\n"
+#define HGC_MMA_NEXT(CG)      \
+  "add.u64 da, da, 2;\n"      \
+  "add.u64 db, db, %12;\n"    \
+  "@p_mma tcgen05.mma.cta_group::" CG ".kind::f16 [%3], da, db, %6, p_one;\n"
+#define HGC_COMMITS_1                                                                      \
+  "@p_el tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n"    \
+  "@p_rel tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n"
+#define HGC_COMMITS_2                                                                                            \
+  "@p_el tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%8], cm;\n"   \
+  "@p_rel tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%9], cm;\n"
+#define HGC_STAGE_HEAD                                                  \
+  "{\n"                                                                 \
+  ".reg .pred p_next, p_el, p_mma, p_acc, p_one, p_rel;\n"              \
+  ".reg .b64 da, db;\n"                                                 \
+  ".reg .b16 cm;\n"                                                     \
+  "mov.b16 cm, 3;\n"                                                    \
+  "mov.b64 da, %4;\n"                                                   \
+  "mov.b64 db, %5;\n"                                                   \
+  "mbarrier.test_wait.parity.shared::cta.b64 p_next, [%1], %2;\n"       \
+  "elect.sync _|p_el, 0xffffffff;\n"                                    \
+  "setp.ne.b32 p_mma, %11, 0;\n"                                        \
+  "and.pred p_mma, p_mma, p_el;\n"                                      \
+  "setp.ne.b32 p_acc, %7, 0;\n"                                         \
+  "setp.eq.b32 p_one, 0, 0;\n"                                          \
+  "setp.ne.b32 p_rel, %10, 0;\n"                                        \
+  "and.pred p_rel, p_rel, p_el;\n"
+#define HGC_STAGE_TAIL "selp.u32 %0, 1, 0, p_next;\n}\n"
+template <int KSTEPS, bool PAIR>
 __device__ __forceinline__ uint32_t issue_stage(uint32_t next_bar, uint32_t next_parity, uint32_t d_tmem,
                                                 uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc,
                                                 uint32_t a_bar, uint32_t b_bar, uint32_t release_b,
@@ -240,148 +405,66 @@ __device__ __forceinline__ uint32_t issue_stage(uint32_t next_bar, uint32_t next
   : "r"(next_bar), "r"(next_parity), "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc), "r"(a_bar), \
     "r"(b_bar), "r"(release_b), "r"(do_mma), "l"(b_step)                                                     \
   : "memory"
-  if (KSTEPS == 4) {
-    asm volatile(
-      "{\n"
-      ".reg .pred p_next, p_el, p_mma, p_acc, p_one, p_rel;\n"
-      ".reg .b64 da, db;\n"
-      "mov.b64 da, %4;\n"
-      "mov.b64 db, %5;\n"
-      "mbarrier.test_wait.parity.shared::cta.b64 p_next, [%1], %2;\n"
-      "elect.sync _|p_el, 0xffffffff;\n"
-      "setp.ne.b32 p_mma, %11, 0;\n"
-      "and.pred p_mma, p_mma, p_el;\n"
-      "setp.ne.b32 p_acc, %7, 0;\n"
-      "setp.eq.b32 p_one, 0, 0;\n"
-      "setp.ne.b32 p_rel, %10, 0;\n"
-      "and.pred p_rel, p_rel, p_el;\n"
-      "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], %4, %5, %6, p_acc;\n"
-      "add.u64 da, da, 2;\n"
-      "add.u64 db, db, %12;\n"
-      "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, p_one;\n"
-      "add.u64 da, da, 2;\n"
-      "add.u64 db, db, %12;\n"
-      "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, p_one;\n"
-      "add.u64 da, da, 2;\n"
-      "add.u64 db, db, %12;\n"
-      "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, p_one;\n"
-      "@p_el tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n"
-      "@p_rel tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n"
-      "selp.u32 %0, 1, 0, p_next;\n"
-      "}\n"
-        HGC_STAGE_OPERANDS);
-  } else if (KSTEPS == 2) {
-    asm volatile(
-      "{\n"
-      ".reg .pred p_next, p_el, p_mma, p_acc, p_one, p_rel;\n"
-      ".reg .b64 da, db;\n"
-      "mov.b64 da, %4;\n"
-      "mov.b64 db, %5;\n"
-      "mbarrier.test_wait.parity.shared::cta.b64 p_next, [%1], %2;\n"
-      "elect.sync _|p_el, 0xffffffff;\n"
-      "setp.ne.b32 p_mma, %11, 0;\n"
-      "and.pred p_mma, p_mma, p_el;\n"
-      "setp.ne.b32 p_acc, %7, 0;\n"
-      "setp.eq.b32 p_one, 0, 0;\n"
-      "setp.ne.b32 p_rel, %10, 0;\n"
-      "and.pred p_rel, p_rel, p_el;\n"
-      "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], %4, %5, %6, p_acc;\n"
-      "add.u64 da, da, 2;\n"
-      "add.u64 db, db, %12;\n"
-      "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], da, db, %6, p_one;\n"
-      "@p_el tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n"
-      "@p_rel tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n"
-      "selp.u32 %0, 1, 0, p_next;\n"
-      "}\n"
-        HGC_STAGE_OPERANDS);
+  if constexpr (!PAIR) {
+    if (KSTEPS == 4) {
+      asm volatile(HGC_STAGE_HEAD HGC_MMA_FIRST("1") HGC_MMA_NEXT("1") HGC_MMA_NEXT("1") HGC_MMA_NEXT("1") HGC_COMMITS_1
+                       HGC_STAGE_TAIL HGC_STAGE_OPERANDS);
+    } else if (KSTEPS == 2) {
+      asm volatile(HGC_STAGE_HEAD HGC_MMA_FIRST("1") HGC_MMA_NEXT("1") HGC_COMMITS_1 HGC_STAGE_TAIL HGC_STAGE_OPERANDS);
+    } else {
+      asm volatile(HGC_STAGE_HEAD HGC_MMA_FIRST("1") HGC_COMMITS_1 HGC_STAGE_TAIL HGC_STAGE_OPERANDS);
+    }
   } else {
-    asm volatile(
-      "{\n"
-      ".reg .pred p_next, p_el, p_mma, p_acc, p_one, p_rel;\n"
-      ".reg .b64 da, db;\n"
-      "mov.b64 da, %4;\n"
-      "mov.b64 db, %5;\n"
-      "mbarrier.test_wait.parity.shared::cta.b64 p_next, [%1], %2;\n"
-      "elect.sync _|p_el, 0xffffffff;\n"
-      "setp.ne.b32 p_mma, %11, 0;\n"
-      "and.pred p_mma, p_mma, p_el;\n"
-      "setp.ne.b32 p_acc, %7, 0;\n"
-      "setp.eq.b32 p_one, 0, 0;\n"
-      "setp.ne.b32 p_rel, %10, 0;\n"
-      "and.pred p_rel, p_rel, p_el;\n"
-      "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%3], %4, %5, %6, p_acc;\n"
-      "@p_el tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n"
-      "@p_rel tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n"
-      "selp.u32 %0, 1, 0, p_next;\n"
-      "}\n"
-        HGC_STAGE_OPERANDS);
+    if (KSTEPS == 4) {
+      asm volatile(HGC_STAGE_HEAD HGC_MMA_FIRST("2") HGC_MMA_NEXT("2") HGC_MMA_NEXT("2") HGC_MMA_NEXT("2") HGC_COMMITS_2
+                       HGC_STAGE_TAIL HGC_STAGE_OPERANDS);
+    } else if (KSTEPS == 2) {
+      asm volatile(HGC_STAGE_HEAD HGC_MMA_FIRST("2") HGC_MMA_NEXT("2") HGC_COMMITS_2 HGC_STAGE_TAIL HGC_STAGE_OPERANDS);
+    } else {
+      asm volatile(HGC_STAGE_HEAD HGC_MMA_FIRST("2") HGC_COMMITS_2 HGC_STAGE_TAIL HGC_STAGE_OPERANDS);
+    }
   }
 #undef HGC_STAGE_OPERANDS
   return ready;
 }
 
 // KSTEPS MMAs of one weight tile against one activation tile, issued by one elected lane.
-template <int KSTEPS>
+#define HGC_MMAS_HEAD                             \
+  "{\n"                                           \
+  ".reg .pred p_el, p_mma, p_acc, p_one;\n"       \
+  ".reg .b64 da, db;\n"                           \
+  "mov.b64 da, %1;\n"                             \
+  "mov.b64 db, %2;\n"                             \
+  "elect.sync _|p_el, 0xffffffff;\n"              \
+  "setp.ne.b32 p_mma, %5, 0;\n"                   \
+  "and.pred p_mma, p_mma, p_el;\n"                \
+  "setp.ne.b32 p_acc, %4, 0;\n"                   \
+  "setp.eq.b32 p_one, 0, 0;\n"
+#define HGC_MMAS_FIRST(CG) "@p_mma tcgen05.mma.cta_group::" CG ".kind::f16 [%0], %1, %2, %3, p_acc;\n"
+#define HGC_MMAS_NEXT(CG)    \
+  "add.u64 da, da, 2;\n"     \
+  "add.u64 db, db, %6;\n"    \
+  "@p_mma tcgen05.mma.cta_group::" CG ".kind::f16 [%0], da, db, %3, p_one;\n"
+template <int KSTEPS, bool PAIR>
 __device__ __forceinline__ void issue_mmas(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                            uint32_t acc, uint32_t do_mma, uint64_t b_step) {
 #define HGC_MMA_OPERANDS ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc), "r"(do_mma), "l"(b_step) : "memory"
-  if (KSTEPS == 4) {
-    asm volatile(
-        "{\n"
-        ".reg .pred p_el, p_mma, p_acc, p_one;\n"
-        ".reg .b64 da, db;\n"
-        "mov.b64 da, %1;\n"
-        "mov.b64 db, %2;\n"
-        "elect.sync _|p_el, 0xffffffff;\n"
-        "setp.ne.b32 p_mma, %5, 0;\n"
-        "and.pred p_mma, p_mma, p_el;\n"
-        "setp.ne.b32 p_acc, %4, 0;\n"
-        "setp.eq.b32 p_one, 0, 0;\n"
-        "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p_acc;\n"
-        "add.u64 da, da, 2;\n"
-        "add.u64 db, db, %6;\n"
-        "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p_one;\n"
-        "add.u64 da, da, 2;\n"
-        "add.u64 db, db, %6;\n"
-        "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p_one;\n"
-        "add.u64 da, da, 2;\n"
-        "add.u64 db, db, %6;\n"
-        "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p_one;\n"
-        "}\n"
-        HGC_MMA_OPERANDS);
-  } else if (KSTEPS == 2) {
-    asm volatile(
-        "{\n"
-        ".reg .pred p_el, p_mma, p_acc, p_one;\n"
-        ".reg .b64 da, db;\n"
-        "mov.b64 da, %1;\n"
-        "mov.b64 db, %2;\n"
-        "elect.sync _|p_el, 0xffffffff;\n"
-        "setp.ne.b32 p_mma, %5, 0;\n"
-        "and.pred p_mma, p_mma, p_el;\n"
-        "setp.ne.b32 p_acc, %4, 0;\n"
-        "setp.eq.b32 p_one, 0, 0;\n"
-        "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p_acc;\n"
-        "add.u64 da, da, 2;\n"
-        "add.u64 db, db, %6;\n"
-        "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p_one;\n"
-        "}\n"
-        HGC_MMA_OPERANDS);
+  if constexpr (!PAIR) {
+    if (KSTEPS == 4) {
+      asm volatile(HGC_MMAS_HEAD HGC_MMAS_FIRST("1") HGC_MMAS_NEXT("1") HGC_MMAS_NEXT("1") HGC_MMAS_NEXT("1") "}\n" HGC_MMA_OPERANDS);
+    } else if (KSTEPS == 2) {
+      asm volatile(HGC_MMAS_HEAD HGC_MMAS_FIRST("1") HGC_MMAS_NEXT("1") "}\n" HGC_MMA_OPERANDS);
+    } else {
+      asm volatile(HGC_MMAS_HEAD HGC_MMAS_FIRST("1") "}\n" HGC_MMA_OPERANDS);
+    }
   } else {
-    asm volatile(
-        "{\n"
-        ".reg .pred p_el, p_mma, p_acc, p_one;\n"
-        ".reg .b64 da, db;\n"
-        "mov.b64 da, %1;\n"
-        "mov.b64 db, %2;\n"
-        "elect.sync _|p_el, 0xffffffff;\n"
-        "setp.ne.b32 p_mma, %5, 0;\n"
-        "and.pred p_mma, p_mma, p_el;\n"
-        "setp.ne.b32 p_acc, %4, 0;\n"
-        "setp.eq.b32 p_one, 0, 0;\n"
-        "@p_mma tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p_acc;\n"
-        "}\n"
-        HGC_MMA_OPERANDS);
+    if (KSTEPS == 4) {
+      asm volatile(HGC_MMAS_HEAD HGC_MMAS_FIRST("2") HGC_MMAS_NEXT("2") HGC_MMAS_NEXT("2") HGC_MMAS_NEXT("2") "}\n" HGC_MMA_OPERANDS);
+    } else if (KSTEPS == 2) {
+      asm volatile(HGC_MMAS_HEAD HGC_MMAS_FIRST("2") HGC_MMAS_NEXT("2") "}\n" HGC_MMA_OPERANDS);
+    } else {
+      asm volatile(HGC_MMAS_HEAD HGC_MMAS_FIRST("2") "}\n" HGC_MMA_OPERANDS);
+    }
   }
 #undef HGC_MMA_OPERANDS
 }
@@ -692,6 +775,23 @@ struct IgemmArgs {
   int32_t y_tma;        // channels-last output staged for TMA stores (else plain stores)
   int32_t y_full_w;     // pixels of a full channels-last store
   int32_t y_rpu;        // tile rows per channels-last store (rows of at most 32 pixels are batched)
+  // Work distribution (kernels without a split reduction): the ring stages of all tiles form one
+  // sequence (tile, channel block, kernel row, tap group); CTA i takes a contiguous range of it.
+  // sk_split = 0: ranges end on tile boundaries (whole tiles, at most one tile apart between CTAs).
+  // sk_split = 1: equal ranges; a tile that straddles a boundary is reduced by two or more CTAs:
+  // the CTA that holds the tile's first stage finishes it, the others hand over their fp32
+  // accumulators through `sk_part` (one slot per CTA, [column][128 lanes]) and raise `sk_flags`.
+  int32_t ts;           // ring stages per tile: cblocks * R * (S / taps)
+  // CTA pairs (clusters of two, tcgen05 cta_group::2): a tile is 256 output channels x two pixel
+  // sub-tiles of tn x th; CTA r of the pair fetches weight rows r*128.. and pixel sub-tile r, its
+  // tensor memory receives output channels r*128.. of BOTH sub-tiles (sub-tile j at column
+  // j * ncols_sub).  tiles_h / tiles_px then count sub-tiles, total_tiles counts pair tiles.
+  int32_t pair;         // 0 / 1 (also the shift between CTA index and work-unit index)
+  int32_t ncols_sub;    // accumulator columns of one sub-tile (MMA N = 2 * ncols_sub)
+  int32_t sk_split;
+  int32_t sk_cols32;    // accumulator columns handed over, in units of 32
+  float* sk_part;
+  int* sk_flags;
 };
 
 // The tiles of one CTA: blockIdx.x, blockIdx.x + gridDim.x, ...  Tile t = (pixel tile px, channel
@@ -755,7 +855,96 @@ struct TileIter {
       cb1 = a.cblocks;
     }
   }
+  // the same as a range of ring stages of the tile
+  __device__ __forceinline__ void stage_range(const IgemmArgs& a, int& s0, int& s1) const {
+    int cb0, cb1;
+    block_range(a, cb0, cb1);
+    const int per_block = a.ts / a.cblocks;
+    s0 = cb0 * per_block;
+    s1 = cb1 * per_block;
+  }
+  __device__ __forceinline__ int kind(const IgemmArgs&) const { return 0; }
+  __device__ __forceinline__ bool sub_tile(const IgemmArgs&, int, int&, int&) const { return true; }  // (no CTA pairs here)
 };
+
+// The work items of one CTA when the stages of all tiles are dealt out as contiguous ranges (see
+// IgemmArgs::sk_split): item = (tile, stages [s0, s1) of it).  Only the first item of a CTA can
+// start inside a tile and only the last one can end inside a tile.
+struct SegIter {
+  int tile, mg, px, pt, ph;  // px: pixel tile (pair of sub-tiles for CTA pairs); pt, ph: its image and row tile (single CTAs)
+  int s0, s1;
+  int64_t g, g_end;  // position in the global stage sequence, end of this unit's range
+  // work units: CTAs, or CTA pairs
+  __device__ __forceinline__ static int unit(const IgemmArgs& a) { return (int)blockIdx.x >> a.pair; }
+  __device__ __forceinline__ static int units(const IgemmArgs& a) { return (int)gridDim.x >> a.pair; }
+  __device__ __forceinline__ static int64_t range_start(const IgemmArgs& a, int u) {
+    if (a.sk_split) return (int64_t)a.total_tiles * a.ts * u / units(a);
+    return ((int64_t)a.total_tiles * u / units(a)) * a.ts;
+  }
+  __device__ __forceinline__ void init(const IgemmArgs& a) {
+    g = range_start(a, unit(a));
+    g_end = range_start(a, unit(a) + 1);
+    tile = (int)(g / a.ts);
+    s0 = (int)(g - (int64_t)tile * a.ts);
+    const int64_t left = g_end - g;
+    s1 = left < (int64_t)(a.ts - s0) ? s0 + (int)left : a.ts;
+    const int mgn = a.mtiles * a.group;
+    px = tile / mgn;
+    mg = tile - px * mgn;
+    pt = px / a.tiles_h;
+    ph = px - pt * a.tiles_h;
+  }
+  __device__ __forceinline__ bool valid(const IgemmArgs&) const { return g < g_end; }
+  __device__ __forceinline__ void next(const IgemmArgs& a) {
+    g += s1 - s0;
+    ++tile;
+    s0 = 0;
+    const int64_t left = g_end - g;
+    s1 = left < (int64_t)a.ts ? (int)left : a.ts;
+    if (++mg == a.mtiles * a.group) {
+      mg = 0;
+      ++px;
+      if (++ph == a.tiles_h) {
+        ph = 0;
+        ++pt;
+      }
+    }
+  }
+  // group and first output channel (within the group) of the channel tile (of the pair's 256)
+  __device__ __forceinline__ void channel_tile(const IgemmArgs& a, int& grp, int& m0) const {
+    if (a.group == 1) {
+      grp = 0;
+      m0 = (mg * 128) << a.pair;
+    } else {
+      grp = mg / a.mtiles;
+      m0 = ((mg - grp * a.mtiles) * 128) << a.pair;
+    }
+  }
+  // first image and output row of pixel sub-tile j of the current pair tile; a pair tile past the
+  // last sub-tile gets an image index past the batch (its loads are zero-filled, nothing is stored)
+  __device__ __forceinline__ bool sub_tile(const IgemmArgs& a, int j, int& n0, int& p0) const {
+    const int sub = 2 * px + j;
+    const int spt = sub / a.tiles_h;
+    n0 = spt * a.tn;
+    p0 = (sub - spt * a.tiles_h) * a.th;
+    if (sub < a.tiles_px) return true;
+    n0 = a.N;
+    p0 = 0;
+    return false;
+  }
+  __device__ __forceinline__ void stage_range(const IgemmArgs&, int& a0, int& a1) const {
+    a0 = s0;
+    a1 = s1;
+  }
+  // 0: the whole tile; 1: a later part of a tile another CTA finishes (hand the accumulators
+  // over); 2: the first part of a tile whose later parts other CTAs computed (add theirs, finish)
+  __device__ __forceinline__ int kind(const IgemmArgs& a) const { return s0 > 0 ? 1 : (s1 < a.ts ? 2 : 0); }
+};
+
+template <bool SPLIT>
+struct WorkIterOf { using type = SegIter; };
+template <>
+struct WorkIterOf<true> { using type = TileIter<true>; };
 
 constexpr int kMaxStages = 8;
 
@@ -766,7 +955,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 // Persistent kernel: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...; the two TMEM
 // accumulators alternate so that the epilogue of one tile overlaps the MMAs of the next.
 // EPI: 0 = TMA-store epilogue, 1 = copy epilogue (NCHW, any shape), 2 = channels-last output
-template <int KB, bool HALO, int EW, int EPI, bool SPLIT>
+template <int KB, bool HALO, int EW, int EPI, bool SPLIT, bool PAIR = false>
 __global__ void __launch_bounds__(64 + 32 * EW, 1)
 igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
              const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmYr,
@@ -777,11 +966,18 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   __shared__ __align__(8) uint64_t acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int abort_flag;
+  __shared__ volatile int sk_ready;
+  __shared__ __align__(8) uint64_t sk_bar;    // completion of the bulk copies of a hand-over
+  __shared__ __align__(8) uint64_t meet_bar;  // meeting point of the epilogue warps (hand-overs)
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   // ring of stages; a stage holds one activation tile followed by `taps` weight tiles
   const uint32_t ring_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  // CTA pairs: rank 0 issues the MMAs of both and owns the barriers the two producers and the two
+  // epilogues report to
+  uint32_t rank = 0;
+  if constexpr (PAIR) asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < a.stages; ++s) {
@@ -790,8 +986,10 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(smem_u32(&acc_full[s]), 1);
-      mbar_init(smem_u32(&acc_empty[s]), EW);  // one arrival per epilogue warp
+      mbar_init(smem_u32(&acc_empty[s]), PAIR ? 2 * EW : EW);  // one arrival per epilogue warp (of both CTAs)
     }
+    mbar_init(smem_u32(&sk_bar), 1);
+    mbar_init(smem_u32(&meet_bar), EW);
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -803,7 +1001,8 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();  // the partner's barriers must exist before anything arrives on them
+  else __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = tmem_slot;
 
@@ -828,48 +1027,77 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     bool ok = true;
     const uint32_t depth = (uint32_t)a.stages;
     const int groups_per_row = a.S / a.taps;  // 1 in halo mode (taps == S), S otherwise (taps == 1)
-    TileIter<SPLIT> it;
+    typename WorkIterOf<SPLIT>::type it;
+    const int stages_per_block = a.R * groups_per_row;
     for (it.init(a); it.valid(a) && ok; it.next(a)) {
       int grp, m0;
       it.channel_tile(a, grp, m0);
-      const int n0 = it.pt * a.tn;
-      const int p0 = it.ph * a.th;
+      int n0 = it.pt * a.tn;
+      int p0 = it.ph * a.th;
+      if constexpr (PAIR) {  // this CTA's half of the pair tile: weight rows and pixel sub-tile `rank`
+        m0 += (int)rank * 128;
+        it.sub_tile(a, (int)rank, n0, p0);
+      }
       const int h_base = p0 * a.stride_h - a.pad_h;
-      int cb0, cb1;
-      it.block_range(a, cb0, cb1);
-      for (int cb = cb0; cb < cb1 && ok; ++cb) {
-        int acol = cb * KB;  // column of w' for tap (r, s): (r*S + s)*cw + cb*KB
-        for (int r = 0; r < a.R && ok; ++r) {
-          for (int sg = 0; sg < groups_per_row; ++sg) {
-            if (!mbar_wait(smem_u32(&empty_bar[ring.idx]), ring.phase ^ 1u, &abort_flag, 64)) {
-              ok = false;
-              break;
-            }
-            const uint32_t fb = smem_u32(&full_bar[ring.idx]);
-            const uint32_t sbase = ring_base + ring.idx * a.stage_bytes;
-            if (elect_one()) {
-              mbar_expect_tx(fb, a.b_bytes + (uint32_t)a.taps * a.a_bytes);
-              if (a.nchw) {
-                // x itself, (pixel, channel, image): blocks of 64 pixels x KB channels, pixels contiguous
-                for (int j = 0; j < a.nblk; ++j)
-                  tma_load_3d(sbase + (uint32_t)j * (uint32_t)(KB * 128), &tmB, fb, p0 * a.Q + 64 * j,
-                              grp * a.cg + cb * KB, n0);
-              } else {
-                tma_load_5d(sbase, &tmB, fb, cb * KB, grp, (HALO ? 0 : sg * a.dil_w) - a.pad_w,
-                            h_base + r * a.dil_h, n0);
-              }
-              for (int t = 0; t < a.taps; ++t)
-                tma_load_3d(sbase + a.b_alloc + (uint32_t)t * a.a_bytes, &tmA, fb, acol + t * a.cw, m0, grp);
-            }
-            __syncwarp();
-            acol += a.taps * a.cw;
-            ring.advance(depth);
-            ++issued;
+      int s0, s1;
+      it.stage_range(a, s0, s1);
+      // stage s of a tile = (channel block cb, kernel row r, tap group sg), sg fastest
+      int cb = s0 / stages_per_block;
+      int r = (s0 - cb * stages_per_block) / groups_per_row;
+      int sg = s0 - cb * stages_per_block - r * groups_per_row;
+      int tap0 = (r * groups_per_row + sg) * a.taps;  // first tap (r*S + s) of the stage
+      for (int st = s0; st < s1; ++st) {
+        if (!mbar_wait(smem_u32(&empty_bar[ring.idx]), ring.phase ^ 1u, &abort_flag, 64)) {
+          ok = false;
+          break;
+        }
+        const uint32_t sbase = ring_base + ring.idx * a.stage_bytes;
+        if constexpr (PAIR) {
+          // both CTAs' copies are counted on the first CTA's barrier, which expects the bytes of both
+          const uint32_t fb = cluster_addr(smem_u32(&full_bar[ring.idx]), 0);
+          if (lane == 0 && rank == 0)
+            mbar_expect_tx(smem_u32(&full_bar[ring.idx]), 2u * (a.b_bytes + (uint32_t)a.taps * a.a_bytes));
+          if (lane == 0)
+            tma_load_5d_pair(sbase, &tmB, fb, cb * KB, grp, (HALO ? 0 : sg * a.dil_w) - a.pad_w, h_base + r * a.dil_h, n0);
+          if (lane == 8) tma_load_4d_pair(sbase + a.b_alloc, &tmA, fb, cb * KB, m0, tap0, grp);
+        } else {
+        const uint32_t fb = smem_u32(&full_bar[ring.idx]);
+        // A thread gets a bulk-tensor copy under way only every few hundred clocks, whatever its
+        // size (measured), so a stage is few, large copies issued by different lanes at once:
+        // lane 0 announces the bytes and fetches the activation tile, lane 8 fetches the weight
+        // tiles of all taps of the stage as one box (the 1x1 mode's 64-pixel blocks: one lane each).
+        if (lane == 0) mbar_expect_tx(fb, a.b_bytes + (uint32_t)a.taps * a.a_bytes);
+        if (a.nchw) {
+          // x itself, (pixel, channel, image): blocks of 64 pixels x KB channels, pixels contiguous
+          if (lane < a.nblk)
+            tma_load_3d(sbase + (uint32_t)lane * (uint32_t)(KB * 128), &tmB, fb, p0 * a.Q + 64 * lane,
+                        grp * a.cg + cb * KB, n0);
+        } else if (lane == 0) {
+          tma_load_5d(sbase, &tmB, fb, cb * KB, grp, (HALO ? 0 : sg * a.dil_w) - a.pad_w, h_base + r * a.dil_h, n0);
+        }
+        if (lane == 8) tma_load_4d(sbase + a.b_alloc, &tmA, fb, cb * KB, m0, tap0, grp);
+        }
+        __syncwarp();
+        tap0 += a.taps;
+        if (++sg == groups_per_row) {
+          sg = 0;
+          if (++r == a.R) {
+            r = 0;
+            ++cb;
+            tap0 = 0;
           }
         }
+        ring.advance(depth);
+        ++issued;
       }
     }
-    if (abort_flag && lane == 0) {
+    if (PAIR && rank != 0) {
+      // (its copies are counted on the partner's barriers: after giving up it just waits a while)
+      if (abort_flag && lane == 0) {
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 2000000ull) __nanosleep(1000);
+      }
+    } else if (abort_flag && lane == 0) {
       // let the copies that were issued land before the CTA's shared memory goes away
       const uint32_t first = issued > depth ? issued - depth : 0;
       for (uint32_t it = first; it < issued; ++it) {
@@ -881,8 +1109,8 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       }
     }
     __syncwarp();
-  } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
+  } else if (warp == 1 && (!PAIR || rank == 0)) {
+    // ---------------- MMA issuer (of a pair: the first CTA's, for both) ----------------
     // Warp-uniform loop; one elected lane issues tcgen05.mma and tcgen05.commit (always the same
     // lane: a commit tracks the MMAs of the thread that executes it).
     Ring ring;
@@ -895,15 +1123,12 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const uint64_t desc_hi = a.desc_hi;
     const uint32_t idesc = a.idesc;
     const uint32_t do_mma = 1u;
-    const int groups_per_row = a.S / a.taps;
     uint32_t ready = mbar_test_wait(smem_u32(&full_bar[0]), 0u);
-    const int units = SPLIT ? (a.total_tiles << a.ks_log2) : a.total_tiles;
-    for (int unit = blockIdx.x; unit < units && ok; unit += gridDim.x, ++lt) {  // only count and slice matter here
-      int groups_per_tile = a.cblocks * a.R * groups_per_row;
-      if constexpr (SPLIT) {  // the slice is the fastest index of a unit
-        const int sl = unit & ((1 << a.ks_log2) - 1);
-        groups_per_tile = ((((sl + 1) * a.cblocks) >> a.ks_log2) - ((sl * a.cblocks) >> a.ks_log2)) * a.R * groups_per_row;
-      }
+    typename WorkIterOf<SPLIT>::type it;
+    for (it.init(a); it.valid(a) && ok; it.next(a), ++lt) {  // only the number of stages of an item matters here
+      int s0, s1;
+      it.stage_range(a, s0, s1);
+      const int groups_per_tile = s1 - s0;
       const uint32_t buf = lt & 1u;
       // the epilogue must have drained this accumulator (two tiles ago)
       if (!mbar_wait(smem_u32(&acc_empty[buf]), ((lt >> 1) & 1u) ^ 1u, &abort_flag, 64)) {
@@ -926,23 +1151,26 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         ring.advance(depth);
         // all taps but the last: MMAs only
         for (int t = 0; t + 1 < a.taps; ++t) {
-          issue_mmas<ksteps>(d_tmem, adesc, bdesc, idesc, acc, do_mma, a.b_kstep);
+          issue_mmas<ksteps, PAIR>(d_tmem, adesc, bdesc, idesc, acc, do_mma, a.b_kstep);
           acc = 1;
           adesc += (uint64_t)(a.a_bytes >> 4);
           bdesc += (uint64_t)(tap_step >> 4);
         }
         // last tap: poll the NEXT stage's barrier first and read the answer after the MMAs and the
         // commit have been issued, so that the poll's latency hides behind them
-        ready = issue_stage<ksteps>(smem_u32(&full_bar[ring.idx]), ring.phase, d_tmem, adesc, bdesc, idesc, acc, e_bar,
+        ready = issue_stage<ksteps, PAIR>(smem_u32(&full_bar[ring.idx]), ring.phase, d_tmem, adesc, bdesc, idesc, acc, e_bar,
                                     e_bar, 0u, do_mma, a.b_kstep);
         acc = 1;
       }
       if (ok) {
-        if (elect_one()) umma_commit(smem_u32(&acc_full[buf]));  // accumulator complete
+        if (elect_one()) {  // accumulator complete
+          if constexpr (PAIR) umma_commit_pair(smem_u32(&acc_full[buf]));
+          else umma_commit(smem_u32(&acc_full[buf]));
+        }
         __syncwarp();
       }
     }
-  } else {
+  } else if (warp >= 2) {
     // ---------------- epilogue (warps 2..9) ----------------
     // Warp w may read TMEM lanes 32*(w%4)..+31; the EW/4 warps of a lane quarter take the units of
     // a tile in turn.
@@ -961,12 +1189,12 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const uint32_t row_off = (uint32_t)lane * 128u + (((uint32_t)lane & 7u) << 4);
     uint32_t unit_ctr = 0, stage_sel = 0;
     uint32_t lt = 0;
-    TileIter<SPLIT> it;
+    uint32_t sk_phase = 0, meet_phase = 0;
+    typename WorkIterOf<SPLIT>::type it;
     for (it.init(a); it.valid(a); it.next(a), ++lt) {
       int grp, m0;
       it.channel_tile(a, grp, m0);
-      const int n0 = it.pt * a.tn;
-      const int p0 = it.ph * a.th;
+      if constexpr (PAIR) m0 += (int)rank * 128;  // this CTA's tensor memory holds its own 128 channels
       const int kin = m0 + row;
       const bool kvalid = kin < a.kg;
       const int k = grp * a.kg + (kvalid ? kin : 0);
@@ -974,9 +1202,90 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       const uint32_t buf = lt & 1u;
       if (!mbar_wait(smem_u32(&acc_full[buf]), (lt >> 1) & 1u, &abort_flag, 256)) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t t_addr = tmem_base + buf * 256u + ((uint32_t)(quarter * 32) << 16);
+      const uint32_t t_tile = tmem_base + buf * 256u + ((uint32_t)(quarter * 32) << 16);
       const bool quarter_live = m0 + quarter * 32 < a.kg;  // any real output channel in this warp's lanes?
+      // the barrier the accumulator is handed back on (of a pair: the first CTA's)
+      const uint32_t acc_empty_bar = PAIR ? cluster_addr(smem_u32(&acc_empty[buf]), 0) : smem_u32(&acc_empty[buf]);
 
+      if constexpr (!SPLIT) {
+        const int kind = a.sk_split ? it.kind(a) : 0;
+        const size_t slot_elems = (size_t)a.sk_cols32 * 32 * 128;
+        // slots and flags are per CTA; the parts of a tile come from the following work units
+        // (the CTA of the same rank in the following pairs)
+        const int unit = SegIter::unit(a);
+        if (kind == 1) {
+          // a later part of a tile that another CTA finishes: hand the accumulators over
+          if (quarter_live) sk_hand_over(t_tile, quarter, half, kPerQuarter, a.sk_cols32, a.sk_part + (size_t)blockIdx.x * slot_elems);
+          __threadfence();
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          if (!epi_sync(smem_u32(&meet_bar), meet_phase, &abort_flag)) break;
+          if (ew == 0 && lane == 0) {
+            __threadfence();
+            asm volatile("st.release.gpu.global.b32 [%0], %1;" ::"l"(a.sk_flags + blockIdx.x), "r"(1) : "memory");
+          }
+          __syncwarp();
+          if (lane == 0) {
+            if constexpr (PAIR) mbar_arrive_cluster(acc_empty_bar);
+            else mbar_arrive(acc_empty_bar);
+          }
+          continue;
+        }
+        if (kind == 2) {
+          // the first part of a tile whose later parts belong to the next units: wait for theirs
+          // (they computed them first of all), add them, then finish the tile as usual
+          const int64_t tile_end = (int64_t)(it.tile + 1) * a.ts;
+          int count = 0;
+          while (unit + 1 + count < SegIter::units(a) && SegIter::range_start(a, unit + 1 + count) < tile_end) ++count;
+          const int first_slot = ((unit + 1) << a.pair) + (int)rank;
+          const int slot_step = 1 << a.pair;
+          if (ew == 0 && lane == 0) {
+            int good = 1;
+            for (int i = 0; i < count && good; ++i) {
+              const int* f = a.sk_flags + first_slot + i * slot_step;
+              const uint64_t t0 = global_timer_ns();
+              for (uint32_t spin = 0;; ++spin) {
+                int v;
+                asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(f) : "memory");
+                if (v != 0) break;
+                if ((spin & 255u) == 255u && (abort_flag || global_timer_ns() - t0 > kWaitLimitNs)) {
+                  abort_flag = 1;
+                  good = 0;
+                  break;
+                }
+                __nanosleep(128);
+              }
+            }
+            sk_ready = good;
+          }
+          if (!epi_sync(smem_u32(&meet_bar), meet_phase, &abort_flag)) break;
+          if (!sk_ready) break;
+          {
+            // the ring is idle: this tile is the CTA's last piece of work and its MMAs are complete
+            int piece32 = (int)(((uint32_t)a.stages * a.stage_bytes) >> 14);  // 16 KB per 32 columns
+            if (piece32 > a.sk_cols32) piece32 = a.sk_cols32;
+            if (!sk_take_over(t_tile, quarter, half, kPerQuarter, a.sk_cols32, quarter_live, a.sk_part, slot_elems,
+                              first_slot, slot_step, count, ring_base, piece32, smem_u32(&sk_bar), sk_phase,
+                              smem_u32(&meet_bar), meet_phase, ew == 0 && lane == 0, &abort_flag))
+              break;
+          }
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          if (!epi_sync(smem_u32(&meet_bar), meet_phase, &abort_flag)) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          // every part has been read: lower the flags for the next launch
+          if (ew == 0)
+            for (int i = lane; i < count; i += 32) a.sk_flags[first_slot + i * slot_step] = 0;
+        }
+      }
+
+      // the pixel sub-tiles of the tile: one, or the two of a CTA pair (side by side in the accumulator)
+#pragma unroll 1
+      for (int sub = 0; sub < (PAIR ? 2 : 1); ++sub) {
+      int n0 = it.pt * a.tn;
+      int p0 = it.ph * a.th;
+      if constexpr (PAIR) {
+        if (!it.sub_tile(a, sub, n0, p0)) break;  // (only the last pair tile can lack its second sub-tile)
+      }
+      const uint32_t t_addr = t_tile + (uint32_t)(sub * a.ncols_sub);
       if constexpr (EPI == 0) {
         // ---- staged epilogue: TMEM -> registers -> swizzled fp16 tile in smem -> TMA store ----
         // (taken when Q % 8 == 0, hence P*Q % 8 == 0, and a tile holds one image: every staged run
@@ -1049,10 +1358,6 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             while (!linear && wc >= a.Q) { wc -= a.Q; ++hr; }
           }
         }
-        // this warp has read its lanes of the accumulator: hand the buffer back to the MMA issuer
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
       } else {
         // ---- direct epilogue: each thread stores runs of its own channel plane ----
         {
@@ -1145,10 +1450,14 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             }
           }
         }
-        // this warp has read its lanes of the accumulator: hand the buffer back to the MMA issuer
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
+      }
+      }  // sub-tiles
+      // this warp has read its lanes of the accumulator: hand the buffer back to the MMA issuer
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) {
+        if constexpr (PAIR) mbar_arrive_cluster(acc_empty_bar);
+        else mbar_arrive(acc_empty_bar);
       }
     }
     // the shared-memory tiles of outstanding stores must stay intact until they have been read,
@@ -1157,7 +1466,9 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   }
 
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
+  // (a pair leaves together: the first CTA's MMAs read the partner's shared memory and write its tensor memory)
+  if constexpr (PAIR) cluster_sync_all();
+  else __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
@@ -1183,6 +1494,35 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
 
 inline size_t round_up_sz(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Launches a kernel of CTA pairs (clusters of two).  p.grid pairs are wanted, but never more than
+// can be resident at once: a persistent kernel must not leave a pair waiting for a second round.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pair(void (*kernel)(KArgs...), IgemmPlan& p, int sms, bool cooperative, dim3 block,
+                        cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = p.smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeCooperative;
+  attr[1].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = cooperative ? 2 : 1;
+  if (p.pair_fit == 0) {
+    int n = 0;
+    cfg.gridDim = dim3((unsigned)(2 * (sms / 2)));
+    p.pair_fit = (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) == cudaSuccess && n > 0) ? n : sms / 2;
+    (void)cudaGetLastError();
+  }
+  const int fit = p.pair_fit < p.grid ? p.pair_fit : p.grid;
+  cfg.gridDim = dim3((unsigned)(2 * fit));
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 }  // namespace
 
 int sm_count() {
@@ -1198,7 +1538,32 @@ int sm_count() {
   return n;
 }
 
+namespace {
+bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_max);
+}
+
+// The plan of a layer: the single-CTA form, or CTA pairs where they were asked for and the layer
+// has more than 128 output channels per group.
 bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
+  ConvGeom gs = g;
+  gs.no_pair = 1;
+  IgemmPlan single{};
+  const bool ok_single = make_plan_impl(gs, &single, false, 64);
+  if (!g.no_pair && g.kg > 128) {
+    IgemmPlan pair{};
+    bool ok_pair = make_plan_impl(g, &pair, true, 64);
+    if (ok_pair && pair.kb == 64 && pair.stages < 3) ok_pair = make_plan_impl(g, &pair, true, 32);
+    if (ok_pair) {  // asked for (HGC_FLAG_CTA_PAIRS) and possible
+      *out = pair;
+      return true;
+    }
+  }
+  if (ok_single) *out = single;
+  return ok_single;
+}
+
+namespace {
+bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_max) {
   IgemmPlan p{};
   if (g.group > 1 && (g.cg % 8) != 0) return false;  // group stride of x' must be 16-byte aligned
   p.x_nhwc = g.x_nhwc;
@@ -1284,8 +1649,12 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
     p.kb = g.cg > 32 ? 64 : (g.cg > 16 ? 32 : 16);
     // stride-1 layers with three or more taps per kernel row and at least two 64-channel blocks:
     // 32-channel stages halve a stage (one activation tile + S weight tiles) so that the ring
-    // is four or five deep instead of two; measured 3-5 % faster on 3x3 layers of 128-512 channels
-    if (p.kb == 64 && g.stride_h == 1 && g.stride_w == 1 && g.s >= 3 && g.cg >= 128) p.kb = 32;
+    // is four or five deep instead of two; measured 3-5 % faster on 3x3 layers of 128-512 channels.
+    // (CTA pairs keep 64: a copy engine handles about one row of a box per clock whatever the row's
+    // width (measured), and with 64-byte rows the rows of a stage take as long as its MMAs; their
+    // activation half-tiles are small enough for three 64-channel stages.)
+    if (!want_pair && p.kb == 64 && g.stride_h == 1 && g.stride_w == 1 && g.s >= 3 && g.cg >= 128) p.kb = 32;
+    if (p.kb > kb_max) p.kb = kb_max;
     p.cblocks = (g.cg + p.kb - 1) / p.kb;
     p.cw = p.cblocks * p.kb;
     p.c_pad = (g.c + 7) / 8 * 8;
@@ -1323,17 +1692,49 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   const double a_bytes_mma = 32.0 * (g.kg < 128 ? g.kg : 128);
   // ks: log2 of the number of CTAs that share the reduction of a tile (each then writes fp32
   // partial sums, added by a second kernel): main loop / 2^ks, an epilogue of twice the bytes
-  auto tile_clk = [&](int64_t brow, int64_t cols, int ks) {
+  // clocks of one MMA step in the main loop of a tile of `cols` accumulator columns
+  auto mma_clk = [&](int64_t brow, int64_t cols) {
     const double ncols = (double)((cols + 15) / 16 * 16);
     const double brows = p.nchw ? (double)((cols + 63) / 64 * 64) : (double)brow;
     const double t_l2 = (a_bytes_mma + brows * p.kb * 2.0 / mps) / 30.0;
-    const double t_tensor = ncols / 2.0;
+    // the tensor pipe needs N/2 clocks for a step of N columns, but never less than about 86
+    // (measured: back-to-back steps of 64 to 170 columns all take 86 clocks)
+    const double t_tensor = ncols / 2.0 > 86.0 ? ncols / 2.0 : 86.0;
     const double t_issue = 45.0 + 400.0 / mps;
     double t = t_tensor > t_l2 ? t_tensor : t_l2;
     if (t_issue > t) t = t_issue;
-    const double main_loop = mpt / (double)(1 << ks) * t;
-    const double epilogue = (600.0 + 10.0 * ncols) * (ks > 0 ? 2.0 : 1.0);
+    return t;
+  };
+  auto epilogue_clk = [&](int64_t cols) { return 600.0 + 10.0 * (double)((cols + 15) / 16 * 16); };
+  auto tile_clk = [&](int64_t brow, int64_t cols, int ks) {
+    const double main_loop = mpt / (double)(1 << ks) * mma_clk(brow, cols);
+    const double epilogue = epilogue_clk(cols) * (ks > 0 ? 2.0 : 1.0);
     return (main_loop > epilogue ? main_loop : epilogue) + 300.0;
+  };
+  // Contiguous ranges of ring stages per CTA (kernels without reduction slices).  Whole tiles per
+  // CTA when that balances; otherwise equal ranges, with the tiles that straddle a boundary
+  // reduced by several CTAs (a hand-over of fp32 accumulators through the workspace).
+  const int ts_est = p.cblocks * p.eff_r * (p.halo ? 1 : p.eff_s);  // ring stages per tile
+  auto shared_plan = [&](int64_t tiles, double t_mma, int64_t cols, int units, int* grid_out, double* cost_out) {
+    const double stage_clk = mps * t_mma;
+    const int64_t total = tiles * ts_est;
+    // a range is at least 4 stages and 24 MMA steps long, and a tile is shared by at most 4 CTAs
+    int64_t min_stages = (int64_t)(24.0 / mps + 0.999);
+    if (min_stages < 4) min_stages = 4;
+    int64_t grid = total / min_stages;
+    if (grid > units) grid = units;
+    if (grid > 4 * tiles) grid = 4 * tiles;
+    if (grid < 1) grid = 1;
+    const double per_cta = (double)((total + grid - 1) / grid);
+    const double tiles_per_cta = (double)tiles / (double)grid;
+    const double main_loop = per_cta * stage_clk;
+    const double epi = tiles_per_cta * epilogue_clk(cols);
+    // a hand-over: the accumulators of a part go to the workspace (beside the next tile's MMAs) and
+    // from there into the finishing CTA's idle operand ring by bulk copy, 16 KB per 32 columns
+    const double parts = tiles >= grid ? 1.0 : (double)grid / (double)tiles;  // accumulators added per shared tile
+    const double hand_over = 5000.0 + parts * (1500.0 + 15.0 * (double)cols);  // (measured: 3 to 4 us for 240 columns)
+    *grid_out = (int)grid;
+    *cost_out = (main_loop > epi ? main_loop : epi) + 300.0 * (tiles_per_cta > 1.0 ? tiles_per_cta : 1.0) + hand_over;
   };
   // the second kernel of a split reduction: a launch plus reading the slices and writing y
   auto finish_clk = [&](int ks) {
@@ -1344,7 +1745,8 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   // the split kernel exists for 64-channel stages of stride-1 layers without the direct-x mode
   const bool can_split = p.kb == 64 && p.halo && !p.nchw && !p.y_nhwc;
   double best = 1e300;
-  int best_th = 0, best_tn = 0, best_ks = 0;
+  int best_th = 0, best_tn = 0, best_ks = 0, best_shared = 0, best_grid = 0;
+  const bool can_share = !g.no_split && sms <= kMaxGrid;
   for (int th = 1; th <= g.p; ++th) {
     if ((int64_t)th * p.pitch - junk > 256 || (int64_t)th * (p.patch ? 1 : g.stride_h) > 256) break;
     if (p.vhalo && g.stride_h > 1 && th > 1) break;
@@ -1363,25 +1765,109 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
         if (ks > 0 && (!can_split || (p.cblocks >> ks) < 2 || mpt / (1 << ks) < 24.0 || 4 * tiles > sms)) break;
         const int64_t units = tiles << ks;
         const int64_t waves = (units + sms - 1) / sms;
-        const double cost = (double)waves * tile_clk((int64_t)tn * th * p.pitch, cols, ks) + finish_clk(ks) +
-                            1e-3 * (double)units;
+        double cost = (double)waves * tile_clk((int64_t)tn * th * p.pitch, cols, ks) + finish_clk(ks) +
+                      1e-3 * (double)units;
+        if (can_share && tiles % sms != 0) cost *= 1e3;  // shared tiles were asked for (HGC_FLAG_SHARED_TILES)
         if (cost < best - 1e-9 ||
-            (cost < best + 1e-9 && ks == best_ks && (int64_t)tn * th > (int64_t)best_tn * best_th)) {
+            (cost < best + 1e-9 && ks == best_ks && !best_shared && (int64_t)tn * th > (int64_t)best_tn * best_th)) {
           best = cost;
           best_th = th;
           best_tn = tn;
           best_ks = ks;
+          best_shared = 0;
+          best_grid = (int)(tiles < sms ? tiles : sms);
+        }
+      }
+      if (can_share && tiles % sms != 0) {
+        int grid_s = 0;
+        double cost_s = 0.0;
+        shared_plan(tiles, mma_clk((int64_t)tn * th * p.pitch, cols), cols, sms, &grid_s, &cost_s);
+        if (grid_s > 1 && cost_s < best - 1e-9) {
+          best = cost_s;
+          best_th = th;
+          best_tn = tn;
+          best_ks = 0;
+          best_shared = 1;
+          best_grid = grid_s;
         }
       }
     }
   }
   if (best_th == 0) return false;
+  p.est_clk = best;
+  // CTA pairs (tcgen05 cta_group::2) for layers with more than 128 output channels per group: a
+  // tile is 256 channels x two pixel sub-tiles of at most 128 accumulator columns each.  Every
+  // CTA then reads 128 weight rows and HALF of the activation tile from its own shared memory per
+  // MMA step (and fetches only those): the single-CTA kernel is bound by shared-memory traffic
+  // (operand reads of the tensor core + ring refills: about 150 clocks per 240-column step
+  // against 120 of tensor time, measured), the pair is not.
+  p.pair = 0;
+  p.ncols_sub = 0;
+  const int pairs = sms / 2;
+  if (want_pair && (p.nchw || p.window || p.patch || pairs < 1)) return false;
+  if (want_pair) {
+    const int64_t mgp = (int64_t)((g.kg + 255) / 256) * g.group;
+    double best_pair = 1e300;
+    int pth = 0, ptn = 0, pshared = 0, pgrid = 0;
+    for (int th = 1; th <= g.p; ++th) {
+      if ((int64_t)th * p.pitch - junk > 128 || (int64_t)th * g.stride_h > 256) break;
+      const int tn_hi = th == g.p ? g.n : 1;
+      for (int tn = 1; tn <= tn_hi; ++tn) {
+        const int64_t cols = (int64_t)tn * th * p.pitch - junk;
+        if (cols > (tn > 1 ? 120 : 128)) break;
+        const int64_t subs = (int64_t)((g.n + tn - 1) / tn) * ((g.p + th - 1) / th);
+        const int64_t tiles = (subs + 1) / 2 * mgp;
+        const double ncols = (double)(2 * ((cols + 7) / 8 * 8));
+        double t = ncols / 2.0 > 86.0 ? ncols / 2.0 : 86.0;
+        const double t_issue = 45.0 + 400.0 / mps;
+        if (t_issue > t) t = t_issue;
+        const double main_loop = mpt * t * 1.03;
+        const double epi = 600.0 + 10.0 * ncols;
+        const int64_t waves = (tiles + pairs - 1) / pairs;
+        double cost = (double)waves * ((main_loop > epi ? main_loop : epi) + 300.0) + 1e-3 * (double)tiles;
+        if (can_share && tiles % pairs != 0) cost *= 1e3;
+        if (cost < best_pair - 1e-9 || (cost < best_pair + 1e-9 && !pshared && (int64_t)tn * th > (int64_t)ptn * pth)) {
+          best_pair = cost;
+          pth = th;
+          ptn = tn;
+          pshared = 0;
+          pgrid = (int)(tiles < pairs ? tiles : pairs);
+        }
+        if (can_share && tiles % pairs != 0) {
+          int grid_s = 0;
+          double cost_s = 0.0;
+          shared_plan(tiles, t * 1.03, (int64_t)ncols, pairs, &grid_s, &cost_s);
+          if (grid_s > 1 && cost_s < best_pair - 1e-9) {
+            best_pair = cost_s;
+            pth = th;
+            ptn = tn;
+            pshared = 1;
+            pgrid = grid_s;
+          }
+        }
+      }
+    }
+    if (pth == 0) return false;
+    p.pair = 1;
+    p.est_clk = best_pair;
+    best_th = pth;
+    best_tn = ptn;
+    best_shared = pshared;
+    best_grid = pgrid;
+    best_ks = 0;
+  }
   p.th = best_th;
   p.tn = best_tn;
   p.tiles_h = (g.p + p.th - 1) / p.th;
   p.tiles_n = (g.n + p.tn - 1) / p.tn;
   p.ncols = (p.tn * p.th * p.pitch - junk + 15) / 16 * 16;
-  const int64_t total = (int64_t)p.tiles_n * p.tiles_h * mg;
+  int64_t total = (int64_t)p.tiles_n * p.tiles_h * mg;
+  if (p.pair) {
+    p.ncols_sub = (p.tn * p.th * p.pitch - junk + 7) / 8 * 8;
+    p.ncols = 2 * p.ncols_sub;
+    p.mtiles = (g.kg + 255) / 256;
+    total = ((int64_t)p.tiles_n * p.tiles_h + 1) / 2 * p.mtiles * g.group;
+  }
   if (total > 0x7fffffffLL) return false;
   p.total_tiles = (int32_t)total;
   // weight tile rows: 128, or 64 when the layer has at most 64 output channels per group (the MMA
@@ -1392,7 +1878,7 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   const uint32_t box_rows = (uint32_t)(p.tn * p.th * p.pitch);
   p.b_bytes = box_rows * p.kb * 2u;
   // rows the MMA may touch: the last tap starts (S-1)*dil rows in and reads ncols rows
-  uint32_t rows = (uint32_t)(p.halo ? (g.s - 1) * g.dil_w : 0) + (uint32_t)p.ncols;
+  uint32_t rows = (uint32_t)(p.halo ? (g.s - 1) * g.dil_w : 0) + (uint32_t)(p.pair ? p.ncols_sub : p.ncols);
   if (rows < box_rows) rows = box_rows;
   p.b_alloc = (uint32_t)round_up_sz((size_t)rows * p.kb * 2u, 1024);
   // the epilogue stages fp16 tiles for TMA stores when every staged run of pixels starts on a
@@ -1421,6 +1907,10 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
     if (p.tma_store && mpt * 130.0 < 600.0 + 10.0 * p.ncols && p.tn * p.th * ((g.q + kPassElems - 1) / kPassElems) > 2)
       p.epi_warps = kEpilogueWarpsWide;
   }
+  p.sk_split = best_shared;
+  p.grid = best_grid;
+  p.sk_cols32 = (p.ncols + 31) / 32;
+  if (p.pair) p.epi_warps = kEpilogueWarps;
   // split reduction (chosen with the tile shape above): fp32 partials, copy-style epilogue
   p.ks_log2 = best_ks;
   if (p.ks_log2 > 0) {
@@ -1439,7 +1929,7 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
     p.pitch = p.dense_rows ? p.dense_pitch : (p.halo ? g.q + (g.s - 1) * g.dil_w : g.q);
     const uint32_t box_rows2 = (uint32_t)(p.tn * (p.vhalo ? (p.th - 1) * g.stride_h + g.r : p.th) * p.pitch);
     p.b_bytes = box_rows2 * p.kb * 2u;
-    uint32_t rows2 = (uint32_t)(p.halo ? (g.s - 1) * g.dil_w : 0) + (uint32_t)p.ncols;
+    uint32_t rows2 = (uint32_t)(p.halo ? (g.s - 1) * g.dil_w : 0) + (uint32_t)(p.pair ? p.ncols_sub : p.ncols);
     if (rows2 < box_rows2) rows2 = box_rows2;
     p.b_alloc = (uint32_t)round_up_sz((size_t)rows2 * p.kb * 2u, 1024);
     if (p.dense_rows) {
@@ -1464,6 +1954,9 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
       p.vhalo = 0;
       p.eff_r = g.r;
       p.eff_s = 1;
+    } else if (p.pair) {
+      p.ncols_sub = (p.tn * p.th * g.q + 7) / 8 * 8;
+      p.ncols = 2 * p.ncols_sub;
     } else {
       p.ncols = (p.tn * p.th * g.q + 15) / 16 * 16;
     }
@@ -1474,9 +1967,17 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
   // more than half of an SM's shared memory: at most one CTA per SM, so that the kernel can take
   // all 512 TMEM columns without ever waiting for another CTA to free them
   if (p.smem_bytes < 120u * 1024u) p.smem_bytes = 120u * 1024u;
-  // workspace: status word, re-laid-out weights, NHWC input
+  // ring stages per tile as the kernel walks them; equal ranges need the stage count the cost
+  // model assumed (the ring fitted with the taps of a kernel row sharing a stage)
+  p.ts = p.cblocks * p.eff_r * (p.eff_s / p.taps);
+  if (p.sk_split && p.ts != ts_est) {
+    p.sk_split = 0;
+    const int units = p.pair ? sms / 2 : sms;
+    p.grid = (int)(p.total_tiles < units ? p.total_tiles : units);
+  }
+  // workspace: header (status word, hand-over flags), re-laid-out weights, NHWC input
   p.ws_status_off = 0;
-  p.ws_w_off = 256;
+  p.ws_w_off = kWsHeaderBytes;
   p.ws_x_off = p.ws_w_off + round_up_sz((size_t)g.k * p.eff_r * p.eff_s * p.cw * 2, 256);
   p.ws_part_off = 0;
   p.ws_total = p.ws_x_off + ((p.nchw || p.x_nhwc) ? 0
@@ -1487,9 +1988,15 @@ bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
     p.ws_part_off = p.ws_total;
     p.ws_total += round_up_sz(((size_t)g.n * g.k * g.p * g.q * 4) << p.ks_log2, 256);
   }
+  p.ws_sk_off = 0;
+  if (p.sk_split) {  // one hand-over slot per CTA: [sk_cols32 * 32 columns][128 lanes] fp32
+    p.ws_sk_off = p.ws_total;
+    p.ws_total += (size_t)(p.grid << p.pair) * p.sk_cols32 * 32 * 128 * 4;
+  }
   *out = p;
   return true;
 }
+}  // namespace
 
 // The 5-D map (channel in group, group, W, H, N) over a channels-last activation tensor at `base`:
 // the NHWC copy in the workspace, or the caller's x itself when it is channels-last already.
@@ -1519,12 +2026,16 @@ bool igemm_encode_maps(const ConvGeom& g, IgemmPlan* p, void* ws) {
                                : p->kb == 32 ? CU_TENSOR_MAP_SWIZZLE_64B
                                              : CU_TENSOR_MAP_SWIZZLE_32B;
   {
-    const cuuint64_t kred = (cuuint64_t)p->eff_r * p->eff_s * p->cw;
-    cuuint64_t dims[3] = {kred, (cuuint64_t)g.kg, (cuuint64_t)g.group};
-    cuuint64_t strides[2] = {kred * 2, kred * 2 * (cuuint64_t)g.kg};
-    cuuint32_t box[3] = {(cuuint32_t)p->kb, (cuuint32_t)p->a_rows, 1};
-    cuuint32_t es[3] = {1, 1, 1};
-    if (enc(&p->tmA, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, base + p->ws_w_off, dims, strides, box, es,
+    // w'[group][K/g][tap][cw] as (channel of the tap, output channel, tap, group): one box holds
+    // the kb-channel slices of `taps` consecutive taps for 128 (64) output channels, tap-major in
+    // shared memory, i.e. one K-major weight tile per tap
+    const cuuint64_t ntaps = (cuuint64_t)p->eff_r * p->eff_s;
+    const cuuint64_t kred = ntaps * p->cw;
+    cuuint64_t dims[4] = {(cuuint64_t)p->cw, (cuuint64_t)g.kg, ntaps, (cuuint64_t)g.group};
+    cuuint64_t strides[3] = {kred * 2, (cuuint64_t)p->cw * 2, kred * 2 * (cuuint64_t)g.kg};
+    cuuint32_t box[4] = {(cuuint32_t)p->kb, (cuuint32_t)p->a_rows, (cuuint32_t)p->taps, 1};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    if (enc(&p->tmA, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, base + p->ws_w_off, dims, strides, box, es,
             CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return false;
@@ -1654,7 +2165,7 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
   a.total_tiles = p.total_tiles; a.stages = p.stages; a.taps = p.taps; a.stage_bytes = p.stage_bytes;
   a.a_bytes = p.a_bytes; a.b_bytes = p.b_bytes; a.b_alloc = p.b_alloc;
   // instruction descriptor: D = f32, A = B = f16, both K-major, N >> 3 at bit 17, M >> 4 at bit 24
-  a.idesc = (1u << 4) | ((uint32_t)(p.ncols >> 3) << 17) | ((128u >> 4) << 24);
+  a.idesc = (1u << 4) | ((uint32_t)(p.ncols >> 3) << 17) | (((p.pair ? 256u : 128u) >> 4) << 24);
   if (p.nchw) a.idesc |= 1u << 16;  // activation operand is pixel-major (MN-major)
   // shared-memory descriptor: 8-row groups are 8 * row bytes apart; descriptor version 1;
   // swizzle mode 2 = 128 B, 4 = 64 B, 6 = 32 B
@@ -1689,10 +2200,19 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
   a.y_tma = (p.y_nhwc && p.tma_store) ? 1 : 0;
   a.y_full_w = p.y_full_w;
   a.y_rpu = p.y_rpu > 0 ? p.y_rpu : 1;
+  a.ts = p.ts;
+  a.pair = p.pair;
+  a.ncols_sub = p.ncols_sub;
+  a.sk_split = p.sk_split;
+  a.sk_cols32 = p.sk_cols32;
+  a.sk_part = p.sk_split ? reinterpret_cast<float*>(static_cast<char*>(ws) + p.ws_sk_off) : nullptr;
+  a.sk_flags = reinterpret_cast<int*>(static_cast<char*>(ws) + p.ws_status_off + kWsFlagsOff);
   float* partials = p.ks_log2 > 0 ? reinterpret_cast<float*>(static_cast<char*>(ws) + p.ws_part_off) : nullptr;
   const int sms = sm_count();
   const int64_t units = (int64_t)p.total_tiles << p.ks_log2;
-  dim3 grid((unsigned)(units < sms ? units : sms));
+  dim3 grid((unsigned)(p.ks_log2 > 0 ? (units < sms ? units : sms) : p.grid));
+  // CTAs that share a tile wait for one another: all of them must be resident together
+  const bool cooperative = p.sk_split != 0;
   int* status = reinterpret_cast<int*>(static_cast<char*>(ws) + p.ws_status_off);
   cudaError_t err = cudaSuccess;
   // four instantiations per (kb, halo): TMA-store epilogue with 8 or 16 epilogue warps, copy
@@ -1703,8 +2223,9 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
     err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV, EWV, EPIV, SPLITV>,                                \
                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);            \
     if (err == cudaSuccess)                                                                                \
-      err = launch_kernel(igemm_kernel<KBV, HALOV, EWV, EPIV, SPLITV>, grid, dim3(64 + 32 * EWV),          \
-                          p.smem_bytes, stream, p.tmA, p.tmB, p.tmY, p.tmYr, a, bias, y, partials, status); \
+      err = launch_kernel_coop(cooperative, igemm_kernel<KBV, HALOV, EWV, EPIV, SPLITV>, grid,             \
+                               dim3(64 + 32 * EWV), p.smem_bytes, stream, p.tmA, p.tmB, p.tmY, p.tmYr, a,  \
+                               bias, y, partials, status);                                                 \
   } while (0)
 #define HGC_LAUNCH_IGEMM(KBV, HALOV)                                                              \
   do {                                                                                            \
@@ -1714,6 +2235,30 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
     else if (p.epi_warps == kEpilogueWarpsWide) HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 16, 0, false);    \
     else HGC_LAUNCH_IGEMM_EW(KBV, HALOV, 8, 0, false);                                            \
   } while (0)
+  // CTA pairs: launched as clusters of two, 8 epilogue warps, the three epilogue kinds
+#define HGC_LAUNCH_PAIR_EPI(KBV, HALOV, EPIV)                                                                  \
+  do {                                                                                                       \
+    err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV, 8, EPIV, false, true>,                               \
+                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);              \
+    if (err == cudaSuccess)                                                                                  \
+      err = launch_pair(igemm_kernel<KBV, HALOV, 8, EPIV, false, true>, p, sms, cooperative, dim3(64 + 32 * 8), \
+                        stream, p.tmA, p.tmB, p.tmY, p.tmYr, a, bias, y, partials, status);                  \
+  } while (0)
+#define HGC_LAUNCH_PAIR(KBV, HALOV)                                \
+  do {                                                             \
+    if (p.y_nhwc) HGC_LAUNCH_PAIR_EPI(KBV, HALOV, 2);              \
+    else if (!p.tma_store) HGC_LAUNCH_PAIR_EPI(KBV, HALOV, 1);     \
+    else HGC_LAUNCH_PAIR_EPI(KBV, HALOV, 0);                       \
+  } while (0)
+  if (p.pair) {
+    if (p.kb == 64) {
+      if (p.halo) HGC_LAUNCH_PAIR(64, true); else HGC_LAUNCH_PAIR(64, false);
+    } else if (p.kb == 32) {
+      if (p.halo) HGC_LAUNCH_PAIR(32, true); else HGC_LAUNCH_PAIR(32, false);
+    } else {
+      err = cudaErrorInvalidValue;  // (the planner pairs CTAs only with 32- or 64-channel stages)
+    }
+  } else
   if (p.ks_log2 > 0) {
     HGC_LAUNCH_IGEMM_EW(64, true, 8, 1, true);  // the one instantiation with a split reduction
   } else
@@ -1726,6 +2271,8 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
   }
 #undef HGC_LAUNCH_IGEMM_EW
 #undef HGC_LAUNCH_IGEMM
+#undef HGC_LAUNCH_PAIR_EPI
+#undef HGC_LAUNCH_PAIR
   if (err != cudaSuccess) return err;
   count_launch();
   if (p.ks_log2 > 0) {

@@ -57,6 +57,8 @@ int make_geom(const hgc_conv_params* p, hgc::ConvGeom* g) {
   g->p = (int32_t)P; g->q = (int32_t)Q;
   g->cg = p->c / p->group; g->kg = p->k / p->group;
   g->x_nhwc = 0; g->y_nhwc = 0;  // this entry point takes NCHW tensors only
+  g->no_split = 1;               // whole tiles per CTA: no hand-over slots in the fixed array
+  g->no_pair = 1;
   return HGC_OK;
 }
 
@@ -79,7 +81,7 @@ extern "C" int hgc_conv_forward_static(const hgc_conv_params* p, const void* x, 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // the array keeps whatever the previous call left: the status word must start at zero (the
   // re-layout kernels rewrite every byte of the weight and input copies, padding included)
-  if (cudaMemsetAsync(ws + plan.ws_status_off, 0, 256, st) != cudaSuccess) return HGC_CUDA_ERROR;
+  if (cudaMemsetAsync(ws + plan.ws_status_off, 0, hgc::kWsHeaderBytes, st) != cudaSuccess) return HGC_CUDA_ERROR;
   if (!hgc::igemm_encode_maps(g, &plan, ws)) return HGC_CUDA_ERROR;
   const __half* xh = static_cast<const __half*>(x);
   const __half* wh = static_cast<const __half*>(w);

@@ -113,7 +113,8 @@ def test_planner_paths():
 
 def test_plan_info_reports_tiling_and_activation_source():
     """The planner runs on the host: its choices can be checked without a GPU."""
-    keys = {"path", "kb", "halo", "tn", "th", "pitch", "ncols", "tiles", "stages", "taps", "x_source", "k_slices"}
+    keys = {"path", "kb", "halo", "tn", "th", "pitch", "ncols", "tiles", "stages", "taps", "x_source", "k_slices",
+            "grid", "shared_tiles", "pair"}
     cases = [
         # (n, c, h, w, k, r, s, pad, stride), x_source
         ((16, 256, 56, 56, 256, 3, 3, 1, 1), 0),   # NHWC copy of x
@@ -135,7 +136,8 @@ def test_plan_info_reports_tiling_and_activation_source():
         assert info["tn"] * info["th"] * info["pitch"] - (info["pitch"] - d.output_dims()[3]) <= 256
         d.close()
     fc = hgc.ConvDesc.inner_product(64, 4096, 4096)
-    assert fc.plan_info()["k_slices"] in (2, 4, 8) and fc.plan_info()["tn"] == 64   # few tiles: split reduction
+    info = fc.plan_info()   # few tiles: several CTAs share the reduction of a tile, one way or the other
+    assert (info["k_slices"] in (2, 4, 8) or info["shared_tiles"] == 1) and info["tn"] == 64, info
     fc.close()
     dw = hgc.ConvDesc(2, 32, 14, 14, 32, 3, 3, 1, 1, 1, 1, 1, 1, 32)
     assert dw.plan_info()["kb"] == 0   # not the tensor-core path: zeros

@@ -78,13 +78,88 @@ def test_igemm_mode(hgc, oracle, name, a, source):
     if source is not None:
         assert d.plan_info()["x_source"] == source, (name, d.plan_info())
     if "reduction split" in name:
-        assert d.plan_info()["k_slices"] > 1, d.plan_info()
+        # several CTAs per tile: reduction slices with a second pass, or CTAs that hand their
+        # accumulators over inside the one launch
+        assert d.plan_info()["k_slices"] > 1 or d.plan_info()["shared_tiles"] == 1, d.plan_info()
     d.close()
     for relu, bias, registered in ((True, b, True), (False, None, False)):
         ref = oracle.conv_fast(P, x, w, bias, relu)
         got, path = run_layer(hgc, a, x, w, bias, relu, register_weights=registered)
         assert path == hgc.HGC_PATH_IGEMM
         check_close(got, ref, what=f"{name} relu={relu}")
+
+
+SCHED_CASES = [
+    # (id, params, flags by name, what the plan must report)
+    ("pairs 3x3 c128 k256 24x24 (TMA-store epilogue)", params_dict(3, 128, 24, 24, 256, 3, 3, 1, 1), ("pairs",), {"pair": 1}),
+    ("pairs 3x3 c96 k384 13x13 (copy epilogue, second CTA of the last channel pair idle)",
+     params_dict(3, 96, 13, 13, 384, 3, 3, 1, 1), ("pairs",), {"pair": 1}),
+    ("pairs 3x3 c64 k520 7x7 (several images per sub-tile, odd number of sub-tiles, ragged channels)",
+     params_dict(7, 64, 7, 7, 520, 3, 3, 1, 1), ("pairs",), {"pair": 1}),
+    ("pairs 3x3 stride 2 c96 k256 (one tap per stage)", params_dict(2, 96, 15, 15, 256, 3, 3, 1, 1, 2, 2), ("pairs",), {"pair": 1}),
+    ("pairs 1x1 14x14 c256 k1024", params_dict(4, 256, 14, 14, 1024, 1, 1), ("pairs",), {"pair": 1}),
+    ("pairs grouped 3x3 g2 c128 k512", params_dict(2, 128, 12, 12, 512, 3, 3, 1, 1, 1, 1, 1, 1, 2), ("pairs",), {"pair": 1}),
+    ("pairs k128: not eligible, single CTAs", params_dict(2, 64, 16, 16, 128, 3, 3, 1, 1), ("pairs",), {"pair": 0}),
+    ("shared 3x3 c256 k256 56x56 n2 (tiles over 148 CTAs: ranges end inside tiles)",
+     params_dict(2, 256, 56, 56, 256, 3, 3, 1, 1), ("shared",), {"shared_tiles": 1}),
+    ("shared 3x3 c512 k512 14x14 n3 (a tile over several CTAs)", params_dict(3, 512, 14, 14, 512, 3, 3, 1, 1), ("shared",),
+     {"shared_tiles": 1}),
+    ("shared 1x1 5x5 c4096 k96 (inner-product shape, many CTAs per tile)", params_dict(3, 4096, 5, 5, 96, 1, 1), ("shared",),
+     {"shared_tiles": 1}),
+    ("shared 1x1 direct 28x28 c512 k384", params_dict(3, 512, 28, 28, 384, 1, 1), ("shared",), {"shared_tiles": 1}),
+    ("pairs + shared 3x3 c256 k256 28x28 n5", params_dict(5, 256, 28, 28, 256, 3, 3, 1, 1), ("pairs", "shared"),
+     {"pair": 1, "shared_tiles": 1}),
+    ("pairs + shared 3x3 c512 k512 14x14 n3", params_dict(3, 512, 14, 14, 512, 3, 3, 1, 1), ("pairs", "shared"),
+     {"pair": 1, "shared_tiles": 1}),
+]
+
+
+@pytest.mark.parametrize("name,a,flag_names,want", SCHED_CASES, ids=[c[0] for c in SCHED_CASES])
+def test_scheduling_flags(hgc, oracle, name, a, flag_names, want):
+    """CTA pairs (cta_group::2) and tiles shared by several CTAs are opt-in schedules of the same
+    layer: the plan must report them where asked for, and the results must match the oracle."""
+    flags = (hgc.HGC_FLAG_CTA_PAIRS if "pairs" in flag_names else 0) | (hgc.HGC_FLAG_SHARED_TILES if "shared" in flag_names else 0)
+    rng = np.random.default_rng(zlib.crc32(name.encode()))
+    x, w, b = workloads.random_layer_tensors(rng, a["n"], a["c"], a["h"], a["w"], a["k"], a["r"], a["s"], a["group"])
+    P = oracle.ConvParams(**a)
+    d = hgc.ConvDesc(flags=flags, **a)
+    assert d.path() == hgc.HGC_PATH_IGEMM, name
+    info = d.plan_info()
+    d.close()
+    for key, value in want.items():
+        assert info[key] == value, (name, info)
+    for relu, bias in ((True, b), (False, None)):
+        ref = oracle.conv_fast(P, x, w, bias, relu)
+        first = None
+        for rep in range(2):   # twice: the second launch finds the first one's hand-over flags lowered again
+            got, _ = run_layer(hgc, a, x, w, bias, relu, flags=flags, register_weights=True)
+            check_close(got, ref, what=f"{name} relu={relu} rep={rep}")
+            if first is None:
+                first = got
+            else:
+                assert np.array_equal(first.view(np.uint16), got.view(np.uint16)), "the schedule must be deterministic"
+
+
+def test_scheduling_flags_channels_last(hgc, oracle):
+    """The same schedules with channels-last activations on both sides."""
+    from gpu_util import to_dev, to_host
+    import torch
+    a = params_dict(3, 128, 20, 20, 256, 3, 3, 1, 1)
+    rng = np.random.default_rng(99)
+    x, w, b = workloads.random_layer_tensors(rng, a["n"], a["c"], a["h"], a["w"], a["k"], 3, 3, 1)
+    ref = oracle.conv_fast(oracle.ConvParams(**a), x, w, b, True)
+    for extra in (hgc.HGC_FLAG_CTA_PAIRS, hgc.HGC_FLAG_SHARED_TILES, hgc.HGC_FLAG_CTA_PAIRS | hgc.HGC_FLAG_SHARED_TILES):
+        d = hgc.ConvDesc(flags=hgc.HGC_FLAG_X_NHWC | hgc.HGC_FLAG_Y_NHWC | extra, **a)
+        d.ensure_workspace()
+        xd = to_dev(np.ascontiguousarray(x.transpose(0, 2, 3, 1)))
+        wd, bd = to_dev(w), to_dev(b)
+        y = torch.full((3, 20, 20, 256), float("nan"), dtype=torch.float16, device="cuda")
+        d.set_weights(wd)
+        hgc.conv_forward(d, xd, wd, bd, y, True)
+        torch.cuda.synchronize()
+        assert d.last_device_status() == hgc.HGC_OK
+        check_close(to_host(y).transpose(0, 3, 1, 2), ref, what=f"channels-last flags {extra}")
+        d.close()
 
 
 def test_same_descriptor_new_tensors(hgc, oracle):
