@@ -143,21 +143,31 @@ int hgc_conv_forward_host(hgc_conv_desc* d, const void* x, const void* w, const 
  * way to obtain the scratch buffer that hgc_conv_set_workspace wants.
  *
  * What it does: runs the tensor-core path (HGC_PATH_IGEMM) of hgc_conv_forward with its scratch
- * (status word, re-laid-out weights, NHWC copy of x) in a 32 MiB array that is part of the
- * library image: every device that loads the library holds those 32 MiB until the process exits.
- * It takes the layer description directly; no descriptor object, no workspace, no weight
- * registration (the weights are re-laid-out on every call).  x, w, y: device pointers (required),
- * bias: device pointer or NULL, all 16-byte aligned; everything is queued on `stream`.
+ * (status word, re-laid-out weights, NHWC copy of x, fp32 partial sums of a split reduction) in a
+ * 32 MiB array that is part of the library image: every device that loads the library holds
+ * those 32 MiB until the process exits.  It takes the layer description directly; no descriptor
+ * object, no workspace, no weight registration (the weights are re-laid-out on every call).
+ * p->flags must be 0 or scheduling flags only (those are ignored): NCHW tensors.  x, w, y: device
+ * pointers (required), bias: device pointer or NULL, all 16-byte aligned; everything is queued on
+ * `stream`.
  *
  * It calls no cudaMalloc, cudaFree or other allocating routine.  The first call on each device
  * looks up the array's device address (cudaGetSymbolAddress, with that device current); make
- * that first call outside any stream capture.
+ * that first call outside any stream capture.  With the CUDA runtime's default lazy module
+ * loading the array itself is only backed by device memory when that first call loads the
+ * module, so a caller that may not grow the device footprint later makes one warm-up call per
+ * device at start-up (any small layer), or runs with CUDA_MODULE_LOADING=EAGER; on a device with
+ * less than 32 MiB free that first call fails with HGC_CUDA_ERROR.  The looked-up address is
+ * kept per device ordinal for the life of the process: after cudaDeviceReset it is stale, and
+ * this entry point must not be used again in that process.
  *
  * Limits and errors: HGC_UNSUPPORTED if the layer is not one the tensor-core path takes (fewer
- * than 9 channels per group, very wide rows ...: use hgc_conv_forward); HGC_NO_WORKSPACE if the
- * layer needs more than the 32 MiB (256 B + K*R*S*c_w*2 + N*H*W*c_pad*2 bytes, channels rounded
- * up); HGC_INVALID_ARG / HGC_BAD_ALIGNMENT as for hgc_conv_forward; HGC_CUDA_ERROR.  A
- * device-side timeout cannot be read back through this entry point.
+ * than 9 channels per group unless it is an image stem, very wide rows ...: use hgc_conv_forward)
+ * or if p->flags asks for channels-last tensors or the direct path; HGC_NO_WORKSPACE if the layer
+ * needs more than the 32 MiB (1 KiB + K*R*S*c_w*2 + N*H*W*c_pad*2 bytes, channels rounded up,
+ * + slices*N*K*P*Q*4 for the few layers whose reduction is split into 2, 4 or 8 slices: inner
+ * products, tiny planes); HGC_INVALID_ARG / HGC_BAD_ALIGNMENT as for hgc_conv_forward;
+ * HGC_CUDA_ERROR.  A device-side timeout cannot be read back through this entry point.
  *
  * All calls on a device share the one array, and it keeps the previous call's contents (the
  * call clears the part that must start at zero).  Two calls whose GPU work overlaps - different

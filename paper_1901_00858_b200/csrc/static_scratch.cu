@@ -48,6 +48,9 @@ int make_geom(const hgc_conv_params* p, hgc::ConvGeom* g) {
   const int64_t Q = floor_div_pos((int64_t)p->w + 2 * p->pad_w - (int64_t)p->dil_w * (p->s - 1) - 1, p->stride_w) + 1;
   if (P < 1 || Q < 1) return HGC_INVALID_ARG;
   if (P > 0x7fffffffLL || Q > 0x7fffffffLL) return HGC_UNSUPPORTED;
+  // NCHW tensors and the planner's tensor-core path only: a caller that sets a layout flag would
+  // otherwise get a tensor in the wrong layout back with HGC_OK
+  if (p->flags & (HGC_FLAG_X_NHWC | HGC_FLAG_Y_NHWC | HGC_FLAG_FORCE_DIRECT)) return HGC_UNSUPPORTED;
   g->n = p->n; g->c = p->c; g->h = p->h; g->w = p->w;
   g->k = p->k; g->r = p->r; g->s = p->s;
   g->pad_h = p->pad_h; g->pad_w = p->pad_w;
@@ -57,7 +60,8 @@ int make_geom(const hgc_conv_params* p, hgc::ConvGeom* g) {
   g->p = (int32_t)P; g->q = (int32_t)Q;
   g->cg = p->c / p->group; g->kg = p->k / p->group;
   g->x_nhwc = 0; g->y_nhwc = 0;  // this entry point takes NCHW tensors only
-  g->no_split = 1;               // whole tiles per CTA: no hand-over slots in the fixed array
+  // the scheduling flags are ignored: whole tiles on single CTAs (no hand-over slots in the fixed array)
+  g->no_split = 1;
   g->no_pair = 1;
   return HGC_OK;
 }
@@ -79,8 +83,10 @@ extern "C" int hgc_conv_forward_static(const hgc_conv_params* p, const void* x, 
   char* ws = static_cast<char*>(scratch_for_current_device());
   if (ws == nullptr) return HGC_CUDA_ERROR;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // the array keeps whatever the previous call left: the status word must start at zero (the
-  // re-layout kernels rewrite every byte of the weight and input copies, padding included)
+  // the array keeps whatever the previous call left: the header (status word, hand-over flags)
+  // must start at zero; the re-layout kernels rewrite every byte of the weight and input copies
+  // that the tensor-core kernel reads, padding included, and a reduction slice writes every
+  // partial sum before the second pass reads it
   if (cudaMemsetAsync(ws + plan.ws_status_off, 0, hgc::kWsHeaderBytes, st) != cudaSuccess) return HGC_CUDA_ERROR;
   if (!hgc::igemm_encode_maps(g, &plan, ws)) return HGC_CUDA_ERROR;
   const __half* xh = static_cast<const __half*>(x);

@@ -17,24 +17,82 @@ def to_host(t):
     return t.cpu().view(torch.int16).numpy().view(np.float16)
 
 
+GUARD_BYTES = 4096
+GUARD_BYTE = 0x7E     # 0x7E7E is a binary16 NaN: a guarded buffer starts out NaN-filled
+
+
+def guarded(nbytes):
+    """A device buffer of `nbytes` bytes (rounded up to 256) between two guard bands filled with a
+    fixed byte pattern, all of it inside one allocation.  Returns (whole, inner)."""
+    import torch
+    inner = (int(nbytes) + 255) // 256 * 256
+    whole = torch.full((inner + 2 * GUARD_BYTES,), GUARD_BYTE, dtype=torch.uint8, device="cuda")
+    return whole, whole[GUARD_BYTES:GUARD_BYTES + inner]
+
+
+def check_guards(whole, what=""):
+    """The bands before and after a guarded buffer still hold the pattern: nothing was stored
+    outside the buffer."""
+    n = whole.numel()
+    assert bool((whole[:GUARD_BYTES] == GUARD_BYTE).all()), f"{what}: bytes BEFORE the buffer were overwritten"
+    assert bool((whole[n - GUARD_BYTES:] == GUARD_BYTE).all()), f"{what}: bytes AFTER the buffer were overwritten"
+
+
+def guarded_output(shape):
+    """A NaN-filled float16 output tensor of `shape` between guard bands.  Returns (whole, y)."""
+    import torch
+    count = int(np.prod(shape))
+    whole, inner = guarded(count * 2)
+    return whole, inner[:count * 2].view(torch.float16).view(*shape)
+
+
+def attach_guarded_workspace(d, host=False):
+    """Attaches a workspace between guard bands (its bytes start out as the NaN pattern, so a read
+    of something the library never wrote shows up in the result).  Returns the whole buffer or None."""
+    need = d.host_workspace_bytes() if host else d.workspace_bytes()
+    if need == 0:
+        return None
+    whole, inner = guarded(need)
+    d.set_workspace(inner)
+    return whole
+
+
 def run_layer(hgc, args, x, w, b, relu, flags=0, register_weights=False):
-    """args: dict of hgc_conv_params fields (without flags).  Returns (y float16 ndarray, path)."""
+    """args: dict of hgc_conv_params fields (without flags).  Returns (y float16 ndarray, path).
+    The output and the workspace sit between guard bands that must survive the call."""
     import torch
     d = hgc.ConvDesc(flags=flags, **args)
     n, k, p, q = d.output_dims()
-    d.ensure_workspace()
+    ws_whole = attach_guarded_workspace(d)
     xd, wd, bd = to_dev(x), to_dev(w), to_dev(b)
     # canary-filled output: an element the kernel does not write stays NaN and fails the check
-    y = torch.full((n, k, p, q), float("nan"), dtype=torch.float16, device="cuda")
+    y_whole, y = guarded_output((n, k, p, q))
     if register_weights:
         d.set_weights(wd)
     hgc.conv_forward(d, xd, wd, bd, y, relu)
     torch.cuda.synchronize()
     assert d.last_device_status() == hgc.HGC_OK
+    check_guards(y_whole, f"y of {args}")
+    if ws_whole is not None:
+        check_guards(ws_whole, f"workspace of {args}")
     path = d.path()
     out = to_host(y)
     d.close()
     return out, path
+
+
+def max_ulp_error(got, ref, floor=2.0 ** -6):
+    """Largest distance in binary16 units in the last place between got and ref over the outputs
+    with |ref| >= floor (below that an absolute error of a rounding tie is many ulps)."""
+    g = got.ravel().view(np.uint16).astype(np.int32)
+    r = ref.ravel().view(np.uint16).astype(np.int32)
+    big = np.abs(ref.ravel().astype(np.float32)) >= floor
+    if not big.any():
+        return 0
+    # sign-magnitude -> a monotonic integer scale
+    gm = np.where(g & 0x8000, -(g & 0x7FFF), g & 0x7FFF)
+    rm = np.where(r & 0x8000, -(r & 0x7FFF), r & 0x7FFF)
+    return int(np.abs(gm - rm)[big].max())
 
 
 def check_close(got, ref, what=""):

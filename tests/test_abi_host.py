@@ -172,3 +172,38 @@ def test_batchnorm_entry_points_validate_their_arguments():
     assert L.hgc_bn_fold(None, None, f, f, None, None, 0.0, 4, 9, ok_ptr, ok_ptr, None) == hgc.HGC_INVALID_ARG
     assert L.hgc_bn_fold(ok_ptr, None, f, f, None, None, 0.0, 0, 9, ok_ptr, ok_ptr, None) == hgc.HGC_INVALID_ARG
     assert L.hgc_bn_fold(ok_ptr, None, f, f, None, None, -1.0, 4, 9, ok_ptr, ok_ptr, None) == hgc.HGC_INVALID_ARG
+
+
+def test_static_entry_point_refuses_layouts_it_does_not_have():
+    """hgc_conv_forward_static takes NCHW tensors on the tensor-core path only: a layout flag or the
+    direct-path flag is refused before anything is queued (no GPU needed: the pointers are never
+    dereferenced), where silently ignoring it would hand back a tensor in the wrong layout."""
+    L = hgc.lib()
+    ptr = ctypes.c_void_p(0x10000)
+    for flags in (hgc.HGC_FLAG_X_NHWC, hgc.HGC_FLAG_Y_NHWC, hgc.HGC_FLAG_X_NHWC | hgc.HGC_FLAG_Y_NHWC,
+                  hgc.HGC_FLAG_FORCE_DIRECT):
+        p = hgc.hgc_conv_params(1, 32, 8, 8, 32, 3, 3, 1, 1, 1, 1, 1, 1, 1, flags)
+        assert L.hgc_conv_forward_static(ctypes.byref(p), ptr, ptr, None, ptr, 0, None) == hgc.HGC_UNSUPPORTED
+    p = hgc.hgc_conv_params(1, 32, 8, 8, 32, 3, 3, 1, 1, 1, 1, 1, 1, 1, 0)
+    assert L.hgc_conv_forward_static(ctypes.byref(p), None, ptr, None, ptr, 0, None) == hgc.HGC_INVALID_ARG
+    assert L.hgc_conv_forward_static(ctypes.byref(p), ctypes.c_void_p(0x10002), ptr, None, ptr, 0, None) == hgc.HGC_BAD_ALIGNMENT
+    bad = hgc.hgc_conv_params(1, 32, 8, 8, 32, 3, 3, 1, 1, 0, 1, 1, 1, 1, 0)     # stride 0
+    assert L.hgc_conv_forward_static(ctypes.byref(bad), ptr, ptr, None, ptr, 0, None) == hgc.HGC_INVALID_ARG
+
+
+def test_scheduling_flags_change_the_plan_not_the_layer():
+    """HGC_FLAG_CTA_PAIRS / HGC_FLAG_SHARED_TILES are opt-in schedules: off by default, reported by
+    the plan when set and applicable, and never a different output shape or path."""
+    args = (16, 256, 56, 56, 256, 3, 3, 1, 1, 1, 1, 1, 1, 1)
+    base = hgc.ConvDesc(*args)
+    assert base.plan_info()["pair"] == 0 and base.plan_info()["shared_tiles"] == 0
+    pairs = hgc.ConvDesc(*args, flags=hgc.HGC_FLAG_CTA_PAIRS)
+    info = pairs.plan_info()
+    assert info["pair"] == 1 and info["ncols"] % 16 == 0 and info["ncols"] <= 256 and info["grid"] <= 74
+    shared = hgc.ConvDesc(*args, flags=hgc.HGC_FLAG_SHARED_TILES)
+    assert shared.plan_info()["shared_tiles"] == 1 and shared.plan_info()["grid"] == 148
+    assert shared.workspace_bytes() > base.workspace_bytes()          # hand-over slots
+    for d in (pairs, shared):
+        assert d.output_dims() == base.output_dims() and d.path() == base.path()
+    # a layer with 128 output channels has nothing to pair
+    assert hgc.ConvDesc(16, 128, 112, 112, 128, 3, 3, 1, 1, flags=hgc.HGC_FLAG_CTA_PAIRS).plan_info()["pair"] == 0

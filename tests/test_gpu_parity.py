@@ -7,11 +7,19 @@ import numpy as np
 import pytest
 
 from paper_1901_00858_b200 import workloads
-from gpu_util import check_close, layer_args, params_dict, run_layer, sample_coords, to_dev, to_host
+from gpu_util import (attach_guarded_workspace, check_close, check_guards, guarded_output, layer_args, max_ulp_error,
+                      params_dict, run_layer, sample_coords, to_dev, to_host)
 
 pytestmark = pytest.mark.gpu
 F16 = np.float16
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+# Beyond the tolerance, a correct kernel differs from the fp64 oracle only where its fp32 sum falls
+# on the other side of a binary16 rounding boundary: by one unit in the last place, on a fraction
+# of the outputs that grows with the reduction length (measured: 0.03 % at 27 terms, 0.3 % at
+# 1152, 0.5 % at 2304, about 1 % at 4608).  A dropped tap, a wrong padding column, binary16
+# accumulation or a double rounding moves many outputs by many units, so both numbers are asserted.
+MIN_BIT_IDENTICAL = 0.985
+MAX_ULP = 1
 
 
 @pytest.fixture(scope="module")
@@ -153,7 +161,9 @@ def test_configs_whole_tensor(hgc, oracle, cfg, batch):
         assert float(np.abs(ref.astype(np.float64)).max()) < 65504
         got, _ = run_layer(hgc, a, x, w, b, l.relu, register_weights=True)
         err, same = check_close(got, ref, what=f"{wl.name}/{l.name}")
-        assert same > 0.98, (wl.name, l.name, same)   # beyond rare 1-ulp rounding ties means a bug
+        ulp = max_ulp_error(got, ref)
+        print(f"{wl.name}/{l.name}: bit-identical {same:.5f}, max error {ulp} ulp, {err:.2e} abs")
+        assert same >= MIN_BIT_IDENTICAL and ulp <= MAX_ULP, (wl.name, l.name, same, ulp)
 
 
 def _unique_layers(wl):
@@ -166,76 +176,68 @@ def _unique_layers(wl):
     return out
 
 
-@pytest.mark.parametrize("cfg,batch", [(2, 16), (3, 32), (4, 64)])
-def test_configs_full_size_sampled(hgc, oracle, cfg, batch):
-    """Full-size layers in the configuration the bench times (planner's path, registered
-    weights); the oracle evaluates a sample of outputs one by one: corners, borders, first and
-    last image/channel, and 16k random points per layer.  Every output must also be finite and,
-    with ReLU, non-negative (an unwritten element stays NaN)."""
+def _whole_tensor_layer(hgc, oracle, a, x, w, b, relu, flags, what):
+    """One full-size layer in the configuration the bench times (planner's path, registered
+    weights, guarded output and workspace): EVERY output element against the oracle."""
     import torch
+    d = hgc.ConvDesc(flags=flags, **a)
+    n, k, p, q = d.output_dims()
+    ws_whole = attach_guarded_workspace(d)
+    x_cl, y_cl = bool(flags & hgc.HGC_FLAG_X_NHWC), bool(flags & hgc.HGC_FLAG_Y_NHWC)
+    xd = to_dev(np.ascontiguousarray(x.transpose(0, 2, 3, 1)) if x_cl else x)
+    wd, bd = to_dev(w), to_dev(b)
+    y_whole, y = guarded_output((n, p, q, k) if y_cl else (n, k, p, q))
+    d.set_weights(wd)
+    hgc.conv_forward(d, xd, wd, bd, y, relu)
+    torch.cuda.synchronize()
+    assert d.last_device_status() == hgc.HGC_OK
+    check_guards(y_whole, what + " (y)")
+    if ws_whole is not None:
+        check_guards(ws_whole, what + " (workspace)")
+    got = to_host(y)
+    if y_cl:
+        got = np.ascontiguousarray(got.transpose(0, 3, 1, 2))
+    info = d.plan_info()
+    d.close()
+    del xd, wd, bd, y, y_whole, ws_whole
+    ref = oracle.conv_fast(oracle.ConvParams(**a), x, w, b, relu)
+    assert float(np.abs(ref.astype(np.float32)).max()) < 65504
+    err, same = check_close(got, ref, what=what)
+    ulp = max_ulp_error(got, ref)
+    print(f"{what}: {got.size} outputs, bit-identical {same:.5f}, max error {ulp} ulp, {err:.2e} abs")
+    assert same >= MIN_BIT_IDENTICAL and ulp <= MAX_ULP, (what, same, ulp, info)
+
+
+@pytest.mark.parametrize("cfg,batch", [(2, 16), (3, 32), (4, 64)])
+def test_configs_full_size_whole_tensor(hgc, oracle, cfg, batch):
+    """The three throughput configurations at full size, in the launch configuration the bench
+    times: every unique layer, every output element against the oracle (the tile plans for
+    several images per tile, multi-wave schedules and wide epilogues only occur here)."""
     wl = workloads.workload(cfg, batch)
-    rng = np.random.default_rng(99 + cfg)
     for li, l in _unique_layers(wl):
         x, w, b = workloads.make_tensors(cfg, batch, li, l)
-        a = layer_args(batch, l)
-        d = hgc.ConvDesc(**a)
-        n, k, p, q = d.output_dims()
-        assert (n, k, p, q) == (batch, l.k, l.out, l.out)
-        d.ensure_workspace()
-        xd, wd, bd = to_dev(x), to_dev(w), to_dev(b)
-        y = torch.full((n, k, p, q), float("nan"), dtype=torch.float16, device="cuda")
-        d.set_weights(wd)
-        hgc.conv_forward(d, xd, wd, bd, y, l.relu)
-        torch.cuda.synchronize()
-        assert d.last_device_status() == hgc.HGC_OK
-        assert bool(torch.isfinite(y).all()), f"{wl.name}/{l.name}: non-finite output"
-        if l.relu:
-            assert float(y.min()) >= 0.0
-        coords = sample_coords(rng, n, k, p, q)
-        ref = oracle.conv_points(oracle.ConvParams(**a), x, w, b, l.relu, coords)
-        ct = torch.from_numpy(coords).cuda()
-        got = to_host(y[ct[:, 0], ct[:, 1], ct[:, 2], ct[:, 3]])
-        check_close(got, ref, what=f"{wl.name}/{l.name}")
-        d.close()
-        del xd, wd, bd, y
+        _whole_tensor_layer(hgc, oracle, layer_args(batch, l), x, w, b, l.relu, 0, f"{wl.name}/{l.name}")
 
 
-@pytest.mark.parametrize("cfg,batch", [(2, 16), (4, 64)])
-def test_configs_full_size_channels_last_sampled(hgc, oracle, cfg, batch):
+@pytest.mark.parametrize("cfg,batch", [(2, 16), (3, 32), (4, 64)])
+def test_configs_full_size_channels_last_whole_tensor(hgc, oracle, cfg, batch):
     """The bench's channels-last leg at full size: every layer that takes the flags reads
-    x[N][H][W][C] and writes y[N][P][Q][K]; sampled outputs against the oracle as above."""
-    import torch
+    x[N][H][W][C] and writes y[N][P][Q][K]; every output element against the oracle."""
     wl = workloads.workload(cfg, batch)
-    rng = np.random.default_rng(199 + cfg)
     for li, l in _unique_layers(wl):
         a = layer_args(batch, l)
-        d, fl = None, 0
+        flags = None
         for fl in (hgc.HGC_FLAG_X_NHWC | hgc.HGC_FLAG_Y_NHWC, hgc.HGC_FLAG_Y_NHWC):
             try:
-                d = hgc.ConvDesc(flags=fl, **a)
+                hgc.ConvDesc(flags=fl, **a).close()
+                flags = fl
                 break
             except hgc.HgcError:
-                d = None
-        if d is None:
+                pass
+        if flags is None:
             continue
         x, w, b = workloads.make_tensors(cfg, batch, li, l)
-        n, k, p, q = d.output_dims()
-        d.ensure_workspace()
-        xin = np.ascontiguousarray(x.transpose(0, 2, 3, 1)) if fl & hgc.HGC_FLAG_X_NHWC else x
-        xd, wd, bd = to_dev(xin), to_dev(w), to_dev(b)
-        y = torch.full((n, p, q, k), float("nan"), dtype=torch.float16, device="cuda")
-        d.set_weights(wd)
-        hgc.conv_forward(d, xd, wd, bd, y, l.relu)
-        torch.cuda.synchronize()
-        assert d.last_device_status() == hgc.HGC_OK
-        assert bool(torch.isfinite(y).all()), f"{wl.name}/{l.name}: non-finite output"
-        coords = sample_coords(rng, n, k, p, q)
-        ref = oracle.conv_points(oracle.ConvParams(**a), x, w, b, l.relu, coords)
-        ct = torch.from_numpy(coords).cuda()
-        got = to_host(y[ct[:, 0], ct[:, 2], ct[:, 3], ct[:, 1]])
-        check_close(got, ref, what=f"{wl.name}/{l.name} channels-last")
-        d.close()
-        del xd, wd, bd, y
+        _whole_tensor_layer(hgc, oracle, a, x, w, b, l.relu, flags, f"{wl.name}/{l.name} channels-last")
 
 
 @pytest.mark.parametrize("kind", ["tensor cores", "channels-last", "depthwise", "depthwise channels-last",
