@@ -227,6 +227,9 @@ int hgc_conv_set_weights(hgc_conv_desc* d, const void* w, void* stream);
 
 /* Reads the device status word of the descriptor's last forward (synchronises `stream`
    work that was queued by this descriptor).  *status is HGC_OK or HGC_DEVICE_TIMEOUT.
+   Reading a raised word clears it.  Until then every forward of the tensor-core path on this
+   descriptor returns at once without touching y (its CTAs find the word raised): after a
+   timeout, read the status before using the descriptor again.
    Channels-last depthwise layers share one status word per process (set by any of them,
    cleared when read). */
 int hgc_conv_last_device_status(hgc_conv_desc* d, int32_t* status);
@@ -313,6 +316,25 @@ int hgc_batchnorm_forward(const void* x, void* y, int32_t n, int32_t c, int64_t 
  */
 int hgc_bn_fold(const void* w, const void* bias, const float* mean, const float* var, const float* gamma,
                 const float* beta, float eps, int32_t k, int64_t per_k, void* w_out, void* b_out, void* stream);
+
+/*
+ * Test hooks for the failure-detection path (Section 3.2 of the paper keeps scalars and control on
+ * the host; a device-side wait that cannot be interrupted from the host therefore has to end by
+ * itself).  Every wait of the TMA-fed kernels (tensor-core path, channels-last depthwise) on a
+ * barrier, a copy or another CTA is bounded by wall-clock time: 2 s by default.  When one runs
+ * out, the CTA stops taking work, lets its outstanding copies land, frees its tensor memory and
+ * raises the descriptor's status word (hgc_conv_last_device_status reports HGC_DEVICE_TIMEOUT);
+ * CTAs and launches that find the word raised return at once, so every later forward on that
+ * descriptor is skipped until the status has been read (which clears it).
+ * hgc_debug_set_wait_limit_ns: the limit in nanoseconds for all later launches in this process
+ * (0 restores the default); synchronous (it writes a device variable of the current device).
+ * hgc_debug_drop_copies: index >= 0: in later launches the first CTA announces its index-th
+ * copy (tensor-core path: ring stage; depthwise: tile) but never issues it, so the wait for it
+ * runs out; -1 switches the hook off.  Nothing faults or traps: the kernel returns through the
+ * path described above.  Errors: HGC_CUDA_ERROR.  Host-side state, not thread-safe.
+ */
+int hgc_debug_set_wait_limit_ns(uint64_t ns);
+int hgc_debug_drop_copies(int32_t index);
 
 /*
  * Launch overlap (off by default).  With enabled != 0 the library launches its kernels with the

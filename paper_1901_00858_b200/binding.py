@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.hgc_weights_repack.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, vp]
         L.hgc_kernel_launch_count.argtypes = [ctypes.POINTER(ctypes.c_uint64)]
         L.hgc_set_launch_overlap.argtypes = [ctypes.c_int]
+        L.hgc_debug_set_wait_limit_ns.argtypes = [ctypes.c_uint64]
+        L.hgc_debug_drop_copies.argtypes = [i32]
         L.hgc_status_string.argtypes = [ctypes.c_int]
         L.hgc_status_string.restype = ctypes.c_char_p
         for name in ("hgc_conv_desc_create", "hgc_conv_desc_destroy", "hgc_conv_forward",
@@ -82,7 +84,8 @@ def lib() -> ctypes.CDLL:
                      "hgc_conv_set_workspace", "hgc_conv_set_weights", "hgc_conv_last_device_status",
                      "hgc_layout_nchw_to_nhwc", "hgc_layout_nhwc_to_nchw", "hgc_weights_repack",
                      "hgc_kernel_launch_count", "hgc_inner_product_desc_create", "hgc_cast_f32_to_f16",
-                     "hgc_set_launch_overlap", "hgc_batchnorm_forward", "hgc_bn_fold"):
+                     "hgc_set_launch_overlap", "hgc_batchnorm_forward", "hgc_bn_fold",
+                     "hgc_debug_set_wait_limit_ns", "hgc_debug_drop_copies"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -281,6 +284,16 @@ def weights_repack(src, dst, k, c_per_group, r, s, group, c_pad, stream=None):
 def set_launch_overlap(enabled: bool) -> None:
     """hgc_set_launch_overlap: programmatic dependent launch of the library's kernels on/off."""
     _check(lib().hgc_set_launch_overlap(int(bool(enabled))), "hgc_set_launch_overlap")
+
+
+def debug_set_wait_limit_ns(ns: int) -> None:
+    """hgc_debug_set_wait_limit_ns: limit of the device-side waits (0 = the default of 2 s)."""
+    _check(lib().hgc_debug_set_wait_limit_ns(int(ns)), "hgc_debug_set_wait_limit_ns")
+
+
+def debug_drop_copies(index: int) -> None:
+    """hgc_debug_drop_copies: the first CTA of later launches never issues its index-th copy (-1: off)."""
+    _check(lib().hgc_debug_drop_copies(int(index)), "hgc_debug_drop_copies")
 
 
 def kernel_launch_count() -> int:

@@ -8,6 +8,8 @@
 namespace hgc {
 static std::atomic<uint64_t> g_launches{0};
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+static std::atomic<int> g_debug_drop{-1};
+int debug_drop_copies() { return g_debug_drop.load(std::memory_order_relaxed); }
 static std::atomic<bool> g_launch_overlap{false};
 bool launch_overlap_enabled() { return g_launch_overlap.load(std::memory_order_relaxed); }
 void set_launch_overlap(bool on) { g_launch_overlap.store(on, std::memory_order_relaxed); }
@@ -379,6 +381,17 @@ int hgc_bn_fold(const void* w, const void* bias, const float* mean, const float*
                                               var, gamma, beta, eps, k, per_k, static_cast<__half*>(w_out),
                                               static_cast<__half*>(b_out), static_cast<cudaStream_t>(stream));
   return err == cudaSuccess ? HGC_OK : HGC_CUDA_ERROR;
+}
+
+int hgc_debug_set_wait_limit_ns(uint64_t ns) {
+  if (hgc::igemm_set_wait_limit_ns(ns) != cudaSuccess) return HGC_CUDA_ERROR;
+  if (hgc::depthwise_nhwc_tma_set_wait_limit_ns(ns) != cudaSuccess) return HGC_CUDA_ERROR;
+  return HGC_OK;
+}
+
+int hgc_debug_drop_copies(int32_t index) {
+  hgc::g_debug_drop.store(index < 0 ? -1 : index, std::memory_order_relaxed);
+  return HGC_OK;
 }
 
 int hgc_set_launch_overlap(int enabled) {

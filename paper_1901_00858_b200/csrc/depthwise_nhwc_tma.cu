@@ -22,6 +22,9 @@ namespace {
 constexpr int kRowsPerThread = 8;
 
 __device__ int g_dw_tma_status = 0;
+// limit of a wait for a copy, in ns of %globaltimer (hgc_debug_set_wait_limit_ns shortens it)
+constexpr uint64_t kDwWaitLimitNs = 2000000000ull;
+__device__ uint64_t g_dw_wait_limit_ns = kDwWaitLimitNs;
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count) {
@@ -39,13 +42,19 @@ __device__ __forceinline__ bool bar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// about two seconds at most (try_wait itself suspends for a while per attempt)
-__device__ __forceinline__ bool bar_wait_bounded(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < (1u << 22); ++i) {
+// two seconds at most (try_wait itself suspends for a while per attempt)
+__device__ __noinline__ bool bar_wait_bounded(uint32_t bar, uint32_t parity) {
+  uint64_t t0 = 0;
+  for (uint32_t i = 0;; ++i) {
     if (bar_try_wait(bar, parity)) return true;
     if (i > 64) __nanosleep(256);
+    if ((i & 63u) == 63u) {
+      uint64_t t;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+      if (t0 == 0) t0 = t;
+      else if (t - t0 > g_dw_wait_limit_ns) return false;
+    }
   }
-  return false;
 }
 __device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int w0,
                                               int h0, int n) {
@@ -61,6 +70,7 @@ struct DwTmaArgs {
   int32_t cblocks, row_tiles, col_tiles, th, tw;  // th x tw = output rows x columns per tile
   int64_t tiles;
   uint32_t tile_bytes;
+  int32_t dbg_drop;  // test hook: the first block announces its dbg_drop-th copy but never issues it (-1: none)
 };
 
 template <int CB>
@@ -96,11 +106,14 @@ depthwise3x3_nhwc_tma_kernel(const __grid_constant__ CUtensorMap tmX, DwTmaArgs 
     n = (int)(t % a.n);
     cb = (int)(t / a.n);
   };
+  uint32_t issued = 0;  // (thread 0's count of announced copies)
   auto issue = [&](int64_t t, uint32_t slot) {
     int cb, n, rt, ct;
     decode(t, cb, n, rt, ct);
     const uint32_t bar = smem_addr(&full[slot]);
     bar_expect_tx(bar, a.tile_bytes);
+    // test hook: announced but never issued, so that the wait for it runs out
+    if (a.dbg_drop >= 0 && blockIdx.x == 0 && issued++ == (uint32_t)a.dbg_drop) return;
     tma_load_tile(buf0 + slot * a.tile_bytes, &tmX, bar, cb * CB, ct * a.tw - a.pad_w, rt * a.th - a.pad_h, n);
   };
 
@@ -235,6 +248,11 @@ bool depthwise3x3_nhwc_tma_supported(const ConvGeom& g) {
   return true;
 }
 
+cudaError_t depthwise_nhwc_tma_set_wait_limit_ns(uint64_t ns) {
+  const uint64_t v = ns == 0 ? kDwWaitLimitNs : ns;
+  return cudaMemcpyToSymbol(g_dw_wait_limit_ns, &v, sizeof(v));
+}
+
 int depthwise_nhwc_tma_status() {
   int v = 0;
   if (cudaMemcpyFromSymbol(&v, g_dw_tma_status, sizeof(int)) != cudaSuccess) return -1;
@@ -271,6 +289,7 @@ cudaError_t launch_depthwise3x3_nhwc_tma(const ConvGeom& g, const __half* x, con
   a.tiles = (int64_t)a.cblocks * g.n * a.row_tiles * a.col_tiles;
   const int ih = a.th + 2, kIW = a.tw + 2;
   a.tile_bytes = (uint32_t)(ih * kIW * cb * 2);
+  a.dbg_drop = debug_drop_copies();
   CUtensorMap tm;
   cuuint64_t dims[4] = {(cuuint64_t)g.c, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.n};
   cuuint64_t strides[3] = {(cuuint64_t)g.c * 2, (cuuint64_t)g.c * 2 * g.w, (cuuint64_t)g.c * 2 * g.w * g.h};

@@ -30,6 +30,12 @@ constexpr int kMaxGrid = 192;
 
 void count_launch();  // bumps the process-wide kernel launch counter
 
+// Test hooks (hgc_debug_*): the limit of the device-side waits, and the index of a copy that the
+// first CTA of the next TMA-fed launches announces but never issues (-1: none).
+int debug_drop_copies();
+cudaError_t igemm_set_wait_limit_ns(uint64_t ns);
+cudaError_t depthwise_nhwc_tma_set_wait_limit_ns(uint64_t ns);
+
 // Programmatic dependent launch: a kernel launched with this helper may be scheduled while the
 // kernel before it in the stream is still draining; every kernel of this library therefore
 // executes grid_dependency_wait() before its first access to global memory (it returns when the

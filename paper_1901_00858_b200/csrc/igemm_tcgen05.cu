@@ -43,7 +43,9 @@ constexpr int kPassElems = 64;               // output pixels per channel staged
 // one warp's staging tile: 32 channels x 64 pixels (or 64 pixels x 32 channels, or 32 rows of 32
 // floats): 4 KB, 1024-byte aligned
 constexpr uint32_t kWarpStageBytes = 4096u;
-constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s per wait
+constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s per wait unless the debug hook shortens it
+// the limit of every device-side wait of this file, in ns of %globaltimer (hgc_debug_set_wait_limit_ns)
+__device__ uint64_t g_wait_limit_ns = kWaitLimitNs;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -107,7 +109,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
       const uint64_t t = global_timer_ns();
       if (t0 == 0) {
         t0 = t;
-      } else if (t - t0 > kWaitLimitNs) {
+      } else if (t - t0 > g_wait_limit_ns) {
         *abort_flag = 1;
         return false;
       }
@@ -781,6 +783,7 @@ struct IgemmArgs {
   // sk_split = 1: equal ranges; a tile that straddles a boundary is reduced by two or more CTAs:
   // the CTA that holds the tile's first stage finishes it, the others hand over their fp32
   // accumulators through `sk_part` (one slot per CTA, [column][128 lanes]) and raise `sk_flags`.
+  int32_t dbg_drop;     // test hook: stage of the first CTA whose copies are left out (-1: none)
   int32_t ts;           // ring stages per tile: cblocks * R * (S / taps)
   // CTA pairs (clusters of two, tcgen05 cta_group::2): a tile is 256 output channels x two pixel
   // sub-tiles of tn x th; CTA r of the pair fetches weight rows r*128.. and pixel sub-tile r, its
@@ -1052,7 +1055,12 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           break;
         }
         const uint32_t sbase = ring_base + ring.idx * a.stage_bytes;
-        if constexpr (PAIR) {
+        // test hook: the first CTA announces the bytes of its `dbg_drop`-th stage but never fetches
+        // them, so that the wait for that stage runs out (hgc_debug_drop_copies)
+        const bool drop = a.dbg_drop >= 0 && blockIdx.x == 0 && issued == (uint32_t)a.dbg_drop;
+        if (drop) {
+          if (lane == 0) mbar_expect_tx(smem_u32(&full_bar[ring.idx]), (PAIR ? 2u : 1u) * (a.b_bytes + (uint32_t)a.taps * a.a_bytes));
+        } else if constexpr (PAIR) {
           // both CTAs' copies are counted on the first CTA's barrier, which expects the bytes of both
           const uint32_t fb = cluster_addr(smem_u32(&full_bar[ring.idx]), 0);
           if (lane == 0 && rank == 0)
@@ -1104,7 +1112,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         const uint32_t bar = smem_u32(&full_bar[it % depth]);
         const uint64_t t0 = global_timer_ns();
         while (!mbar_try_wait(bar, (it / depth) & 1u)) {
-          if (global_timer_ns() - t0 > kWaitLimitNs) break;
+          if (global_timer_ns() - t0 > g_wait_limit_ns) break;
         }
       }
     }
@@ -1247,7 +1255,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 int v;
                 asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(f) : "memory");
                 if (v != 0) break;
-                if ((spin & 255u) == 255u && (abort_flag || global_timer_ns() - t0 > kWaitLimitNs)) {
+                if ((spin & 255u) == 255u && (abort_flag || global_timer_ns() - t0 > g_wait_limit_ns)) {
                   abort_flag = 1;
                   good = 0;
                   break;
@@ -1524,6 +1532,11 @@ cudaError_t launch_pair(void (*kernel)(KArgs...), IgemmPlan& p, int sms, bool co
 }
 
 }  // namespace
+
+cudaError_t igemm_set_wait_limit_ns(uint64_t ns) {
+  const uint64_t v = ns == 0 ? kWaitLimitNs : ns;
+  return cudaMemcpyToSymbol(g_wait_limit_ns, &v, sizeof(v));
+}
 
 int sm_count() {
   static int n = 0;
@@ -2200,6 +2213,7 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
   a.y_tma = (p.y_nhwc && p.tma_store) ? 1 : 0;
   a.y_full_w = p.y_full_w;
   a.y_rpu = p.y_rpu > 0 ? p.y_rpu : 1;
+  a.dbg_drop = debug_drop_copies();
   a.ts = p.ts;
   a.pair = p.pair;
   a.ncols_sub = p.ncols_sub;
