@@ -7,8 +7,10 @@ A step is one pass of the whole path over one batch of a workload: every layer o
 network shape, each with its own resident input, weights, bias and output (the layers'
 inputs are generated independently, so the working set is far larger than L2 and no L2
 flush is needed between steps).  The step is captured once as a CUDA graph and the K timed
-steps replay it (--no-graph: eager launches); per-layer times come from a separate eager pass
-with an event pair around every layer.  Prints ONE JSON line (rank 0).
+steps replay it (--no-graph: eager launches); per-layer times come from capturing every
+distinct layer alone as a graph over rotating buffer sets.  The line also carries, under
+`workloads`, the other throughput configurations (graph replay, per-path figures) and the
+batch-1 workloads.  Prints ONE JSON line (rank 0).
 
 N > 1 (under torchrun): the path has no exchange step; every rank runs an independent
 replica on its own batch ("weak" scaling) and the line reports the aggregate.
@@ -215,6 +217,208 @@ def run_reference(args, wl):
 
 # ---- the CUDA arm ----------------------------------------------------------------------------
 
+def layer_roof(batch, l, peaks, tensor_key):
+    return max(layer_flops(batch, l) / (peaks[tensor_key] * 1e12), layer_bytes(batch, l) / (peaks["hbm_gbs"] * 1e9))
+
+
+def choose_regime(timed_seconds, clocks):
+    """Which measured tensor peak a timed region is compared with: the burst figure when the
+    region is shorter than a second and the clock sampler saw no power capping, else the
+    sustained one (MEASURED_PEAKS.json holds both)."""
+    capped = bool(clocks) and "sw_power_cap" in (clocks.get("reasons") or [])
+    return "sustained" if (timed_seconds >= 1.0 or capped) else "burst"
+
+
+def _geo(batch, l):
+    return (batch, l.c, l.h, l.h, l.k, l.r, l.r, l.pad, l.pad, l.stride, l.stride, l.dil, l.dil, l.group)
+
+
+def build_state(hgc, torch, layers, batch, gen, channels_last=False):
+    """Resident tensors, one set per layer (weights registered once: steady-state inference).
+    channels_last: every layer that can takes both layout flags; a layer that cannot read
+    channels-last input (3-channel stems) takes the output flag alone."""
+    state, n_in, n_out = [], 0, 0
+    for l in layers:
+        fl = 0
+        if channels_last:
+            d = None
+            for fl in (hgc.HGC_FLAG_X_NHWC | hgc.HGC_FLAG_Y_NHWC, hgc.HGC_FLAG_Y_NHWC, 0):
+                try:
+                    d = hgc.ConvDesc(*_geo(batch, l), fl)
+                    break
+                except hgc.HgcError:
+                    continue
+            n_in += 1 if fl & hgc.HGC_FLAG_X_NHWC else 0
+            n_out += 1 if fl & hgc.HGC_FLAG_Y_NHWC else 0
+        else:
+            d = hgc.ConvDesc(*_geo(batch, l))
+        d.ensure_workspace()
+        x = torch.empty((batch, l.c, l.h, l.h), dtype=torch.float16, device="cuda")
+        x.uniform_(l.x_lo, 1.0, generator=gen)
+        w = torch.empty((l.k, l.c // l.group, l.r, l.r), dtype=torch.float16, device="cuda")
+        w.normal_(0.0, float(np.sqrt(2.0 / l.fan_in())), generator=gen)
+        b = torch.empty((l.k,), dtype=torch.float16, device="cuda")
+        b.uniform_(-0.1, 0.1, generator=gen)
+        y = torch.empty((batch, l.k, l.out, l.out), dtype=torch.float16, device="cuda")
+        d.set_weights(w)
+        state.append((d, x, w, b, y, l))
+    torch.cuda.synchronize()
+    return state, n_in, n_out
+
+
+def capture_step(hgc, torch, state, side):
+    """The whole step as one CUDA graph on stream `side`.  Returns (graph, launches per step)."""
+    graph = torch.cuda.CUDAGraph()
+    c0 = hgc.kernel_launch_count()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for (d, x, w, b, y, l) in state:
+                hgc.conv_forward(d, x, w, b, y, l.relu, side)
+    per_step = hgc.kernel_launch_count() - c0
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        for _ in range(3):
+            graph.replay()
+    torch.cuda.synchronize()
+    return graph, per_step
+
+
+def time_replays(torch, graph, side, steps):
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(side):
+        t0.record(side)
+        for _ in range(steps):
+            graph.replay()
+        t1.record(side)
+    torch.cuda.synchronize()
+    return t0.elapsed_time(t1) / steps
+
+
+def time_layers_as_graphs(hgc, torch, state, batch, side, replays=7):
+    """Per-layer device times without launch gaps: every distinct layer shape is captured alone as
+    a CUDA graph of `calls` forwards that rotate over enough (x, y) buffer sets to keep the
+    footprint above twice the L2 size (at most 12 sets), and the graph is replayed `replays` times
+    between events.  For layers whose input goes through the NCHW->NHWC layout pass, the pass
+    is timed on its own the same way.  Returns {shape key: {"ms", "ms_min", "layout_ms", "sets"}}."""
+    out = {}
+    l2 = 126 << 20
+    for (d, x, w, b, y, l) in state:
+        key = (l.c, l.h, l.k, l.r, l.stride, l.pad, l.dil, l.group, l.relu)
+        if key in out:
+            continue
+        per_set = (x.numel() + y.numel()) * 2
+        sets = int(min(12, max(3, -(-2 * l2 // per_set))))
+        xs = [x] + [torch.empty_like(x).copy_(x) for _ in range(sets - 1)]
+        ys = [y] + [torch.empty_like(y) for _ in range(sets - 1)]
+        calls = max(sets, 24 // sets * sets)
+
+        def timed(fn):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                for i in range(sets):
+                    fn(i)
+                torch.cuda.synchronize()
+                with torch.cuda.graph(g, stream=side):
+                    for i in range(calls):
+                        fn(i % sets)
+            torch.cuda.synchronize()
+            samples = []
+            for _ in range(replays + 1):
+                samples.append(time_replays(torch, g, side, 1) / calls)
+            samples = samples[1:]
+            return statistics.median(samples), min(samples)
+
+        med, mn = timed(lambda i: hgc.conv_forward(d, xs[i], w, b, ys[i], l.relu, side))
+        layout_ms = None
+        info = d.plan_info() if d.path() == hgc.HGC_PATH_IGEMM else None
+        if info is not None and info["x_source"] == 0 and not (d.params.flags & hgc.HGC_FLAG_X_NHWC) and l.c % 8 == 0:
+            xt = torch.empty((batch, l.h, l.h, l.c), dtype=torch.float16, device="cuda")
+            layout_ms, _ = timed(lambda i: hgc.layout_nchw_to_nhwc(xs[i], xt, batch, l.c, l.h, l.h, l.c, side))
+            del xt
+        out[key] = {"ms": med, "ms_min": mn, "layout_ms": layout_ms, "sets": sets}
+        del xs, ys
+    return out
+
+
+def summarize(hgc, state, batch, layer_t, peaks, regime):
+    """Per path and for the whole step: achieved TFLOP/s and GB/s from the per-layer graph times
+    (a layer's layout pass counted with its path, and listed separately as `layout`)."""
+    tensor_key = "bf16_tflops" if regime == "burst" else "bf16_tflops_sustained"
+    by_path, layout = {}, {"ms": 0.0, "bytes": 0.0, "launches": 0}
+    rows = []
+    for (d, x, w, b, y, l) in state:
+        key = (l.c, l.h, l.k, l.r, l.stride, l.pad, l.dil, l.group, l.relu)
+        t = layer_t[key]
+        p = hgc.PATH_NAMES[d.path()]
+        e = by_path.setdefault(p, {"ms": 0.0, "flops": 0.0, "bytes": 0.0, "launches": 0, "roof_s": 0.0})
+        e["ms"] += t["ms"]
+        e["flops"] += layer_flops(batch, l)
+        e["bytes"] += layer_bytes(batch, l)
+        e["launches"] += 1
+        e["roof_s"] += layer_roof(batch, l, peaks, tensor_key)
+        if t["layout_ms"] is not None:
+            layout["ms"] += t["layout_ms"]
+            layout["bytes"] += 4.0 * x.numel()          # 2 bytes read + 2 written per element
+            layout["launches"] += 1
+        rows.append({"name": l.name, "path": p, "ms": t["ms"], "ms_min": t["ms_min"], "layout_ms": t["layout_ms"],
+                     "tflops": layer_flops(batch, l) / (t["ms"] * 1e-3) / 1e12,
+                     "gbs": layer_bytes(batch, l) / (t["ms"] * 1e-3) / 1e9,
+                     "roof_frac": layer_roof(batch, l, peaks, tensor_key) * 1e3 / t["ms"]})
+    per_path = {}
+    for k, v in by_path.items():
+        tf = v["flops"] / (v["ms"] * 1e-3) / 1e12
+        gb = v["bytes"] / (v["ms"] * 1e-3) / 1e9
+        per_path[k] = {"ms_per_step": v["ms"], "layers": v["launches"], "tflops": tf, "gbs": gb,
+                       "frac_of_tensor_peak": tf / peaks[tensor_key], "frac_of_hbm_peak": gb / peaks["hbm_gbs"],
+                       "roofline_frac": v["roof_s"] * 1e3 / v["ms"]}
+    if layout["launches"]:
+        gb = layout["bytes"] / (layout["ms"] * 1e-3) / 1e9
+        per_path["layout"] = {"ms_per_step": layout["ms"], "layers": layout["launches"], "gbs": gb,
+                              "frac_of_hbm_peak": gb / peaks["hbm_gbs"],
+                              "note": "the NCHW->NHWC pass of the layers that need one, timed alone; its time is "
+                                      "also inside those layers' path"}
+    total_ms = sum(v["ms"] for v in by_path.values())
+    t_roof = sum(v["roof_s"] for v in by_path.values())
+    return by_path, per_path, rows, total_ms, t_roof
+
+
+def measure_extra(hgc, torch, name, steps, peaks, side, rank):
+    """One more workload for the JSON line's `workloads` object: graph replay of the step, and
+    per-path figures from per-layer graph times."""
+    wl = workloads.by_name(name)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(4321 + rank)
+    state, _, _ = build_state(hgc, torch, wl.expanded(), wl.batch, gen)
+    for _ in range(3):
+        for (d, x, w, b, y, l) in state:
+            hgc.conv_forward(d, x, w, b, y, l.relu, side)
+    torch.cuda.synchronize()
+    graph, per_step = capture_step(hgc, torch, state, side)
+    host0 = time.time()
+    ms = time_replays(torch, graph, side, steps)
+    secs = time.time() - host0
+    flops = sum(layer_flops(wl.batch, l) for (_, _, _, _, _, l) in state)
+    out = {"ms_per_step": ms, "steps": steps, "tflops": flops / (ms * 1e-3) / 1e12,
+           "images_per_s": wl.batch / (ms * 1e-3), "launches_per_step": per_step, "launch": "cuda_graph",
+           "layers": len(state), "batch": wl.batch}
+    if wl.batch > 1:
+        regime = choose_regime(secs, None)
+        layer_t = time_layers_as_graphs(hgc, torch, state, wl.batch, side)
+        _, per_path, _, total_ms, t_roof = summarize(hgc, state, wl.batch, layer_t, peaks, regime)
+        tensor_key = "bf16_tflops" if regime == "burst" else "bf16_tflops_sustained"
+        t_roof_step = sum(layer_roof(wl.batch, l, peaks, tensor_key) for (_, _, _, _, _, l) in state)
+        out["roofline_config"] = {"t_roof_ms": t_roof_step * 1e3, "frac": t_roof_step * 1e3 / ms, "regime": regime,
+                                  "note": "sum over layers of max(flops / tensor peak, bytes / HBM peak), divided by "
+                                          "the graph-replayed step time"}
+        out["per_path"] = per_path
+        out["sum_of_layer_ms"] = total_ms
+    for (d, *_rest) in state:
+        d.close()
+    del state, graph
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args, wl):
     import torch
     import torch.distributed as dist
@@ -237,47 +441,15 @@ def run_ours(args, wl):
         if not layers:
             raise SystemExit(f"--only {args.only}: no such layer in {wl.name}")
     batch = args.batch if args.batch else wl.batch
+    subset = bool(args.only or args.batch)
 
-    # resident tensors, one set per layer (weights registered once: steady-state inference)
     gen = torch.Generator(device="cuda")
     gen.manual_seed(1234 + rank)
-    state = []
-    n_cl_in = n_cl_out = 0
-    for li, l in enumerate(layers):
-        geo = (batch, l.c, l.h, l.h, l.k, l.r, l.r, l.pad, l.pad, l.stride, l.stride, l.dil, l.dil, l.group)
-        if args.layout == "channels_last":
-            # every layer that can takes both flags; a layer that cannot read channels-last input
-            # (3-channel stems) takes the output flag alone; the buffers keep their sizes
-            d = None
-            for fl in (hgc.HGC_FLAG_X_NHWC | hgc.HGC_FLAG_Y_NHWC, hgc.HGC_FLAG_Y_NHWC, 0):
-                try:
-                    d = hgc.ConvDesc(*geo, fl)
-                    break
-                except hgc.HgcError:
-                    continue
-            n_cl_in += 1 if fl & hgc.HGC_FLAG_X_NHWC else 0
-            n_cl_out += 1 if fl & hgc.HGC_FLAG_Y_NHWC else 0
-        else:
-            d = hgc.ConvDesc(*geo)
-        d.ensure_workspace()
-        x = torch.empty((batch, l.c, l.h, l.h), dtype=torch.float16, device="cuda")
-        x.uniform_(l.x_lo, 1.0, generator=gen)
-        w = torch.empty((l.k, l.c // l.group, l.r, l.r), dtype=torch.float16, device="cuda")
-        w.normal_(0.0, float(np.sqrt(2.0 / l.fan_in())), generator=gen)
-        b = torch.empty((l.k,), dtype=torch.float16, device="cuda")
-        b.uniform_(-0.1, 0.1, generator=gen)
-        y = torch.empty((batch, l.k, l.out, l.out), dtype=torch.float16, device="cuda")
-        d.set_weights(w)
-        state.append((d, x, w, b, y, l))
-    torch.cuda.synchronize()
+    state, n_cl_in, n_cl_out = build_state(hgc, torch, layers, batch, gen, args.layout == "channels_last")
 
-    def one_step(events=None):
-        for i, (d, x, w, b, y, l) in enumerate(state):
-            if events is not None:
-                events[i][0].record(stream)
+    def one_step():
+        for (d, x, w, b, y, l) in state:
             hgc.conv_forward(d, x, w, b, y, l.relu, stream)
-            if events is not None:
-                events[i][1].record(stream)
 
     def barrier():
         if world > 1:
@@ -301,18 +473,7 @@ def run_ours(args, wl):
     if not args.no_graph:
         try:
             side.wait_stream(stream)
-            graph = torch.cuda.CUDAGraph()
-            c0 = hgc.kernel_launch_count()
-            with torch.cuda.stream(side):
-                with torch.cuda.graph(graph, stream=side):
-                    for (d, x, w, b, y, l) in state:
-                        hgc.conv_forward(d, x, w, b, y, l.relu, side)
-            launches_per_step = hgc.kernel_launch_count() - c0
-            torch.cuda.synchronize()
-            with torch.cuda.stream(side):
-                for _ in range(3):
-                    graph.replay()
-            torch.cuda.synchronize()
+            graph, launches_per_step = capture_step(hgc, torch, state, side)
         except Exception as exc:  # capture not possible: say why and time eager launches
             graph = None
             graph_err = repr(exc)
@@ -336,68 +497,33 @@ def run_ours(args, wl):
     launches = (launches_per_step * args.steps) if graph is not None else hgc.kernel_launch_count() - launches0
     total_ms = t_start.elapsed_time(t_end)
     ms_per_step = total_ms / args.steps
+    clocks = sampler.stop((host_t0, host_t1)) if rank == 0 else None
 
-    # per-layer device times: a separate pass of eager launches with an event pair around every
-    # layer (average over its steps).  Short layers include some launch latency here, so the
-    # per-kernel roofline fractions derived from them are on the low side.
-    lsteps = max(1, min(args.steps, 20))
-    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in state]
-          for _ in range(lsteps)]
-    e_start, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    e_start.record(stream)
-    for s in range(lsteps):
-        one_step(ev[s])
-    e_end.record(stream)
-    barrier()
-    eager_ms = e_start.elapsed_time(e_end) / lsteps
-    layer_ms = [sum(ev[s][i][0].elapsed_time(ev[s][i][1]) for s in range(lsteps)) / lsteps
-                for i in range(len(state))]
+    # per-layer device times without launch gaps: every distinct layer captured alone as a graph
+    layer_t = time_layers_as_graphs(hgc, torch, state, batch, side) if not args.no_graph else None
 
     # ---- the same step with channels-last activations (HGC_FLAG_X_NHWC / HGC_FLAG_Y_NHWC) --------
     # Not the headline (the metric is NCHW in, NCHW out): what a stack of layers that keeps its
     # activations channels-last between layers pays per step.  Layers that cannot take a flag
-    # (3-channel stems on the input side, depthwise layers) keep NCHW on that side.
+    # (3-channel stems on the input side) keep NCHW on that side.
     nhwc = None
     if not args.no_graph and args.layout == "nchw":
         try:
-            nstate, n_in, n_out = [], 0, 0
-            for (d0, x, w, b, y, l) in state:
-                geo = (batch, l.c, l.h, l.h, l.k, l.r, l.r, l.pad, l.pad, l.stride, l.stride, l.dil, l.dil, l.group)
-                d = None
-                for fl in (hgc.HGC_FLAG_X_NHWC | hgc.HGC_FLAG_Y_NHWC, hgc.HGC_FLAG_Y_NHWC, 0):
-                    try:
-                        d = hgc.ConvDesc(*geo, fl)
-                        break
-                    except hgc.HgcError:
-                        continue
-                d.ensure_workspace()
-                d.set_weights(w)
-                n_in += 1 if fl & hgc.HGC_FLAG_X_NHWC else 0
-                n_out += 1 if fl & hgc.HGC_FLAG_Y_NHWC else 0
-                nstate.append((d, x, w, b, y, l))   # same buffers: only the interpretation of x and y changes
-            gl = torch.cuda.CUDAGraph()
+            gen2 = torch.Generator(device="cuda")
+            gen2.manual_seed(99 + rank)
+            nstate, n_in, n_out = build_state(hgc, torch, layers, batch, gen2, True)
             for (d, x, w, b, y, l) in nstate:
                 hgc.conv_forward(d, x, w, b, y, l.relu, side)
             torch.cuda.synchronize()
-            with torch.cuda.stream(side):
-                with torch.cuda.graph(gl, stream=side):
-                    for (d, x, w, b, y, l) in nstate:
-                        hgc.conv_forward(d, x, w, b, y, l.relu, side)
-                torch.cuda.synchronize()
-                for _ in range(3):
-                    gl.replay()
-                n0, n1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                torch.cuda.synchronize()
-                n0.record(side)
-                for _ in range(args.steps):
-                    gl.replay()
-                n1.record(side)
-            torch.cuda.synchronize()
-            nms = n0.elapsed_time(n1) / args.steps
+            gl, _ = capture_step(hgc, torch, nstate, side)
+            nms = time_replays(torch, gl, side, args.steps)
             nhwc = {"ms_per_step": nms, "layers_with_channels_last_input": n_in,
                     "layers_with_channels_last_output": n_out, "layers": len(nstate),
                     "note": "same layers, activations channels-last where the layer takes the flag; this rank"}
+            for (d, *_r) in nstate:
+                d.close()
+            del nstate, gl
+            torch.cuda.empty_cache()
         except Exception as exc:
             nhwc = {"error": repr(exc)}
 
@@ -407,6 +533,7 @@ def run_ours(args, wl):
     h2d = d2h = 0
     for (d, x, w, b, y, l) in (state if not args.no_e2e else []):
         d.ensure_workspace(host=True)
+        d.set_weights(w)
         hx = torch.empty(x.shape, dtype=torch.float16).pin_memory()
         hx.copy_(x.cpu())
         hw = w.cpu().pin_memory()
@@ -442,7 +569,17 @@ def run_ours(args, wl):
         barrier()
         e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
-    clocks = sampler.stop((host_t0, host_t1)) if rank == 0 else None
+    # ---- the other workloads (single GPU, whole workloads only) ------------------------------
+    extras = None
+    if world == 1 and not subset and not args.no_graph and not args.no_extra and args.layout == "nchw":
+        extras = {}
+        big = [n for n in ("vgg16_n16", "mobilenet_v1_n32", "resnet50_n64") if n != wl.name]
+        small = [n for n in ("vgg16_n1", "mobilenet_v1_n1") if n != wl.name]
+        for name in big + small:
+            try:
+                extras[name] = measure_extra(hgc, torch, name, 50, peaks, side, rank)
+            except Exception as exc:
+                extras[name] = {"error": repr(exc)}
 
     # ---- max over ranks ---------------------------------------------------------------------
     if world > 1:
@@ -458,37 +595,39 @@ def run_ours(args, wl):
     e2e = aggregate([step_flops] * world, [batch] * world, e2e_ms * 1e-3)
 
     if rank == 0:
-        # dominant kernel path by time in the timed region
-        by_path = {}
-        for (d, x, w, b, y, l), ms in zip(state, layer_ms):
-            p = hgc.PATH_NAMES[d.path()]
-            e = by_path.setdefault(p, {"ms": 0.0, "flops": 0.0, "bytes": 0.0, "launches": 0})
-            e["ms"] += ms
-            e["flops"] += layer_flops(batch, l)
-            e["bytes"] += layer_bytes(batch, l)
-            e["launches"] += 1
-        dom = max(by_path, key=lambda k: by_path[k]["ms"])
-        e = by_path[dom]
-        hbm_bound = e["bytes"] / (peaks["hbm_gbs"] * 1e9) > e["flops"] / (peaks["bf16_tflops_sustained"] * 1e12)
-        if dom == "depthwise" or hbm_bound:
-            roof = {"bound": "hbm", "kernel": dom, "achieved": e["bytes"] / (e["ms"] * 1e-3) / 1e9,
-                    "peak": peaks["hbm_gbs"], "unit": "GB/s"}
-        else:
-            roof = {"bound": "tensor", "kernel": dom, "achieved": e["flops"] / (e["ms"] * 1e-3) / 1e12,
-                    "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"}
-        roof["frac"] = roof["achieved"] / roof["peak"]
-        roof["traffic"] = measured_traffic(wl.name, dom, bool(args.only or args.batch))
-        roof["peak_source"] = peaks["source"]
-        roof["share_of_step"] = e["ms"] / sum(layer_ms)
-        roof["avg_launch_ms"] = e["ms"] / e["launches"]
-        t_roof = sum(layer_roof_seconds(batch, l, peaks) for l in layers)
+        regime = choose_regime(total_ms * 1e-3, clocks)
+        tensor_key = "bf16_tflops" if regime == "burst" else "bf16_tflops_sustained"
+        t_roof_step = sum(layer_roof(batch, l, peaks, tensor_key) for l in layers)
+        roof, per_path, rows = None, None, None
+        if layer_t is not None:
+            by_path, per_path, rows, sum_layer_ms, _ = summarize(hgc, state, batch, layer_t, peaks, regime)
+            # dominant kernel path by time; its achieved rate from the per-layer graph times
+            dom = max(by_path, key=lambda k: by_path[k]["ms"])
+            e = by_path[dom]
+            hbm_bound = e["bytes"] / (peaks["hbm_gbs"] * 1e9) > e["flops"] / (peaks[tensor_key] * 1e12)
+            if dom == "depthwise" or hbm_bound:
+                ach = e["bytes"] / (e["ms"] * 1e-3) / 1e9
+                roof = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": ach / peaks["hbm_gbs"]}
+            else:
+                ach = e["flops"] / (e["ms"] * 1e-3) / 1e12
+                roof = {"bound": "tensor", "kernel": dom, "achieved": ach, "peak": peaks[tensor_key], "unit": "TFLOP/s",
+                        "frac": ach / peaks[tensor_key], "frac_burst": ach / peaks["bf16_tflops"],
+                        "frac_sustained": ach / peaks["bf16_tflops_sustained"], "regime": regime,
+                        "frac_of_step": (e["flops"] / (ms_per_step * 1e-3) / 1e12) / peaks[tensor_key]}
+            roof["traffic"] = measured_traffic(wl.name, dom, subset)
+            roof["peak_source"] = peaks["source"]
+            roof["share_of_step"] = e["ms"] / sum_layer_ms
+            roof["avg_launch_ms"] = e["ms"] / e["launches"]
+            roof["timing"] = ("every distinct layer captured alone as a CUDA graph over rotating buffer sets "
+                              "(median of 7 replays); a layer's layout pass is counted with its kernel")
         cpu = cpu_baseline(wl) if world == 1 and not args.no_cpu_baseline else None
         line = {
             "metric": "conv_forward_tflops", "value": agg["tflops"], "unit": "TFLOP/s", "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16 (f32 accumulate)",
             "data": "synthetic",
-            "config": {"workload": wl.name if not (args.only or args.batch) else f"{wl.name} (subset: only={args.only or 'all'}, batch={batch})",
+            "config": {"workload": wl.name if not subset else f"{wl.name} (subset: only={args.only or 'all'}, batch={batch})",
                        "layers": len(layers), "batch_per_gpu": batch,
                        "l2": "inputs larger than L2 (every layer has its own tensors)",
                        "launch": "cuda_graph" if graph is not None else "eager",
@@ -497,34 +636,30 @@ def run_ours(args, wl):
                                      "channels-last activations)"} if args.layout == "channels_last" else {})},
             "images_per_s": agg["images_per_s"],
             "roofline": roof,
-            "roofline_config": {"t_roof_ms": t_roof * 1e3, "frac": t_roof * 1e3 / (sum(layer_ms)),
-                                "note": "sum over layers of max(flops/tensor peak, bytes/HBM peak) / sum of layer times"},
-            "per_path": {k: {"ms_per_step": v["ms"], "launches_per_step": v["launches"],
-                             "tflops": v["flops"] / (v["ms"] * 1e-3) / 1e12,
-                             "gbs": v["bytes"] / (v["ms"] * 1e-3) / 1e9} for k, v in by_path.items()},
+            "roofline_config": {"t_roof_ms": t_roof_step * 1e3, "frac": t_roof_step * 1e3 / ms_per_step, "regime": regime,
+                                "frac_burst": sum(layer_roof(batch, l, peaks, "bf16_tflops") for l in layers) * 1e3 / ms_per_step,
+                                "frac_sustained": sum(layer_roof(batch, l, peaks, "bf16_tflops_sustained") for l in layers) * 1e3 / ms_per_step,
+                                "note": "sum over layers of max(flops / tensor peak, bytes / HBM peak), divided by the "
+                                        "timed step (ms_per_step); regime = which measured tensor peak applies: burst "
+                                        "for a timed region under a second without power capping, else sustained"},
+            "per_path": per_path,
             "e2e": {"value": e2e["tflops"], "unit": "TFLOP/s", "ms_per_step": e2e_ms, "steps": e2e_steps,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "images_per_s": e2e["images_per_s"]},
             "gpu_launches": launches,
             "clocks": clocks,
         }
-        line["eager"] = {"ms_per_step": eager_ms, "tflops": step_flops / (eager_ms * 1e-3) / 1e12,
-                         "steps": lsteps,
-                         "note": "the same step as eager launches with an event pair around every layer "
-                                 "(source of the per-layer and per-kernel times), this rank"}
         if graph_err is not None:
             line["graph_error"] = graph_err
         if nhwc is not None:
             if "ms_per_step" in nhwc:
                 nhwc["tflops"] = step_flops / (nhwc["ms_per_step"] * 1e-3) / 1e12
             line["channels_last"] = nhwc
+        if extras is not None:
+            line["workloads"] = extras
         if cpu is not None:
             line["cpu_baseline"] = cpu
-        if args.layers:
-            line["layers"] = [{"name": l.name, "path": hgc.PATH_NAMES[d.path()], "ms": ms,
-                               "tflops": layer_flops(batch, l) / (ms * 1e-3) / 1e12,
-                               "gbs": layer_bytes(batch, l) / (ms * 1e-3) / 1e9,
-                               "roof_frac": layer_roof_seconds(batch, l, peaks) * 1e3 / ms}
-                              for (d, x, w, b, y, l), ms in zip(state, layer_ms)]
+        if args.layers and rows is not None:
+            line["layers"] = rows
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -660,6 +795,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of replaying the step as a CUDA graph")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
+    ap.add_argument("--no-extra", action="store_true", help="skip the other workloads of the `workloads` object")
     ap.add_argument("--only", default="", help="comma-separated layer names: run just these layers (profiling)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling on a small case)")
     args = ap.parse_args()

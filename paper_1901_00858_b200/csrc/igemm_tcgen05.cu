@@ -873,44 +873,70 @@ struct TileIter {
 // The work items of one CTA when the stages of all tiles are dealt out as contiguous ranges (see
 // IgemmArgs::sk_split): item = (tile, stages [s0, s1) of it).  Only the first item of a CTA can
 // start inside a tile and only the last one can end inside a tile.
+template <bool SHARED>
 struct SegIter {
   int tile, mg, px, pt, ph;  // px: pixel tile (pair of sub-tiles for CTA pairs); pt, ph: its image and row tile (single CTAs)
   int s0, s1;
-  int64_t g, g_end;  // position in the global stage sequence, end of this unit's range
+  int64_t g, g_end;  // shared tiles: position in the global stage sequence, end of this unit's range
+  int stride, d_mg, d_px, d_pt, d_ph;  // whole tiles: step between this unit's tiles and its decomposition
   // work units: CTAs, or CTA pairs
   __device__ __forceinline__ static int unit(const IgemmArgs& a) { return (int)blockIdx.x >> a.pair; }
   __device__ __forceinline__ static int units(const IgemmArgs& a) { return (int)gridDim.x >> a.pair; }
   __device__ __forceinline__ static int64_t range_start(const IgemmArgs& a, int u) {
-    if (a.sk_split) return (int64_t)a.total_tiles * a.ts * u / units(a);
-    return ((int64_t)a.total_tiles * u / units(a)) * a.ts;
+    return (int64_t)a.total_tiles * a.ts * u / units(a);
   }
+  // Whole tiles (sk_split = 0): unit u takes tiles u, u + units, ...  Tiles that run at the same
+  // time are then neighbours in x and y, which is what the memory system likes (contiguous ranges
+  // per CTA measured 10 to 50 % slower on the memory-bound layers).  Shared tiles (sk_split = 1):
+  // a contiguous range of the stage sequence, which may begin and end inside a tile.
   __device__ __forceinline__ void init(const IgemmArgs& a) {
-    g = range_start(a, unit(a));
-    g_end = range_start(a, unit(a) + 1);
-    tile = (int)(g / a.ts);
-    s0 = (int)(g - (int64_t)tile * a.ts);
-    const int64_t left = g_end - g;
-    s1 = left < (int64_t)(a.ts - s0) ? s0 + (int)left : a.ts;
     const int mgn = a.mtiles * a.group;
+    if constexpr (SHARED) {
+      g = range_start(a, unit(a));
+      g_end = range_start(a, unit(a) + 1);
+      tile = (int)(g / a.ts);
+      s0 = (int)(g - (int64_t)tile * a.ts);
+      const int64_t left = g_end - g;
+      s1 = left < (int64_t)(a.ts - s0) ? s0 + (int)left : a.ts;
+      stride = 1;
+    } else {
+      tile = unit(a);
+      stride = units(a);
+      s0 = 0;
+      s1 = a.ts;
+      g = 0;
+      g_end = 0;
+    }
     px = tile / mgn;
     mg = tile - px * mgn;
     pt = px / a.tiles_h;
     ph = px - pt * a.tiles_h;
+    d_px = stride / mgn;
+    d_mg = stride - d_px * mgn;
+    d_pt = d_px / a.tiles_h;
+    d_ph = d_px - d_pt * a.tiles_h;
   }
-  __device__ __forceinline__ bool valid(const IgemmArgs&) const { return g < g_end; }
+  __device__ __forceinline__ bool valid(const IgemmArgs& a) const { return SHARED ? g < g_end : tile < a.total_tiles; }
   __device__ __forceinline__ void next(const IgemmArgs& a) {
-    g += s1 - s0;
-    ++tile;
-    s0 = 0;
-    const int64_t left = g_end - g;
-    s1 = left < (int64_t)a.ts ? (int)left : a.ts;
-    if (++mg == a.mtiles * a.group) {
-      mg = 0;
+    if constexpr (SHARED) {
+      g += s1 - s0;
+      s0 = 0;
+      const int64_t left = g_end - g;
+      s1 = left < (int64_t)a.ts ? (int)left : a.ts;
+    }
+    tile += stride;
+    mg += d_mg;
+    px += d_px;
+    ph += d_ph;
+    pt += d_pt;
+    if (mg >= a.mtiles * a.group) {
+      mg -= a.mtiles * a.group;
       ++px;
-      if (++ph == a.tiles_h) {
-        ph = 0;
-        ++pt;
-      }
+      ++ph;
+    }
+    if (ph >= a.tiles_h) {
+      ph -= a.tiles_h;
+      ++pt;
     }
   }
   // group and first output channel (within the group) of the channel tile (of the pair's 256)
@@ -935,19 +961,21 @@ struct SegIter {
     p0 = 0;
     return false;
   }
-  __device__ __forceinline__ void stage_range(const IgemmArgs&, int& a0, int& a1) const {
-    a0 = s0;
-    a1 = s1;
+  __device__ __forceinline__ void stage_range(const IgemmArgs& a, int& a0, int& a1) const {
+    a0 = SHARED ? s0 : 0;
+    a1 = SHARED ? s1 : a.ts;
   }
   // 0: the whole tile; 1: a later part of a tile another CTA finishes (hand the accumulators
   // over); 2: the first part of a tile whose later parts other CTAs computed (add theirs, finish)
-  __device__ __forceinline__ int kind(const IgemmArgs& a) const { return s0 > 0 ? 1 : (s1 < a.ts ? 2 : 0); }
+  __device__ __forceinline__ int kind(const IgemmArgs& a) const {
+    return SHARED ? (s0 > 0 ? 1 : (s1 < a.ts ? 2 : 0)) : 0;
+  }
 };
 
-template <bool SPLIT>
-struct WorkIterOf { using type = SegIter; };
-template <>
-struct WorkIterOf<true> { using type = TileIter<true>; };
+template <bool SPLIT, bool SHARED>
+struct WorkIterOf { using type = SegIter<SHARED>; };
+template <bool SHARED>
+struct WorkIterOf<true, SHARED> { using type = TileIter<true>; };
 
 constexpr int kMaxStages = 8;
 
@@ -958,7 +986,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 // Persistent kernel: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...; the two TMEM
 // accumulators alternate so that the epilogue of one tile overlaps the MMAs of the next.
 // EPI: 0 = TMA-store epilogue, 1 = copy epilogue (NCHW, any shape), 2 = channels-last output
-template <int KB, bool HALO, int EW, int EPI, bool SPLIT, bool PAIR = false>
+template <int KB, bool HALO, int EW, int EPI, bool SPLIT, bool PAIR = false, bool SHARED = false>
 __global__ void __launch_bounds__(64 + 32 * EW, 1)
 igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
              const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmYr,
@@ -1030,7 +1058,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     bool ok = true;
     const uint32_t depth = (uint32_t)a.stages;
     const int groups_per_row = a.S / a.taps;  // 1 in halo mode (taps == S), S otherwise (taps == 1)
-    typename WorkIterOf<SPLIT>::type it;
+    typename WorkIterOf<SPLIT, SHARED>::type it;
     const int stages_per_block = a.R * groups_per_row;
     for (it.init(a); it.valid(a) && ok; it.next(a)) {
       int grp, m0;
@@ -1045,9 +1073,12 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       int s0, s1;
       it.stage_range(a, s0, s1);
       // stage s of a tile = (channel block cb, kernel row r, tap group sg), sg fastest
-      int cb = s0 / stages_per_block;
-      int r = (s0 - cb * stages_per_block) / groups_per_row;
-      int sg = s0 - cb * stages_per_block - r * groups_per_row;
+      int cb = 0, r = 0, sg = 0;
+      if (SHARED || SPLIT) {  // (whole tiles start at stage 0)
+        cb = s0 / stages_per_block;
+        r = (s0 - cb * stages_per_block) / groups_per_row;
+        sg = s0 - cb * stages_per_block - r * groups_per_row;
+      }
       int tap0 = (r * groups_per_row + sg) * a.taps;  // first tap (r*S + s) of the stage
       for (int st = s0; st < s1; ++st) {
         if (!mbar_wait(smem_u32(&empty_bar[ring.idx]), ring.phase ^ 1u, &abort_flag, 64)) {
@@ -1132,7 +1163,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const uint32_t idesc = a.idesc;
     const uint32_t do_mma = 1u;
     uint32_t ready = mbar_test_wait(smem_u32(&full_bar[0]), 0u);
-    typename WorkIterOf<SPLIT>::type it;
+    typename WorkIterOf<SPLIT, SHARED>::type it;
     for (it.init(a); it.valid(a) && ok; it.next(a), ++lt) {  // only the number of stages of an item matters here
       int s0, s1;
       it.stage_range(a, s0, s1);
@@ -1198,7 +1229,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     uint32_t unit_ctr = 0, stage_sel = 0;
     uint32_t lt = 0;
     uint32_t sk_phase = 0, meet_phase = 0;
-    typename WorkIterOf<SPLIT>::type it;
+    typename WorkIterOf<SPLIT, SHARED>::type it;
     for (it.init(a); it.valid(a); it.next(a), ++lt) {
       int grp, m0;
       it.channel_tile(a, grp, m0);
@@ -1215,12 +1246,12 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       // the barrier the accumulator is handed back on (of a pair: the first CTA's)
       const uint32_t acc_empty_bar = PAIR ? cluster_addr(smem_u32(&acc_empty[buf]), 0) : smem_u32(&acc_empty[buf]);
 
-      if constexpr (!SPLIT) {
-        const int kind = a.sk_split ? it.kind(a) : 0;
+      if constexpr (!SPLIT && SHARED) {
+        const int kind = it.kind(a);
         const size_t slot_elems = (size_t)a.sk_cols32 * 32 * 128;
         // slots and flags are per CTA; the parts of a tile come from the following work units
         // (the CTA of the same rank in the following pairs)
-        const int unit = SegIter::unit(a);
+        const int unit = SegIter<SHARED>::unit(a);
         if (kind == 1) {
           // a later part of a tile that another CTA finishes: hand the accumulators over
           if (quarter_live) sk_hand_over(t_tile, quarter, half, kPerQuarter, a.sk_cols32, a.sk_part + (size_t)blockIdx.x * slot_elems);
@@ -1243,7 +1274,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           // (they computed them first of all), add them, then finish the tile as usual
           const int64_t tile_end = (int64_t)(it.tile + 1) * a.ts;
           int count = 0;
-          while (unit + 1 + count < SegIter::units(a) && SegIter::range_start(a, unit + 1 + count) < tile_end) ++count;
+          while (unit + 1 + count < SegIter<SHARED>::units(a) && SegIter<SHARED>::range_start(a, unit + 1 + count) < tile_end) ++count;
           const int first_slot = ((unit + 1) << a.pair) + (int)rank;
           const int slot_step = 1 << a.pair;
           if (ew == 0 && lane == 0) {
@@ -1759,7 +1790,7 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
   const bool can_split = p.kb == 64 && p.halo && !p.nchw && !p.y_nhwc;
   double best = 1e300;
   int best_th = 0, best_tn = 0, best_ks = 0, best_shared = 0, best_grid = 0;
-  const bool can_share = !g.no_split && sms <= kMaxGrid;
+  const bool can_share = !g.no_split && sms <= kMaxGrid && p.kb >= 32;
   for (int th = 1; th <= g.p; ++th) {
     if ((int64_t)th * p.pitch - junk > 256 || (int64_t)th * (p.patch ? 1 : g.stride_h) > 256) break;
     if (p.vhalo && g.stride_h > 1 && th > 1) break;
@@ -1923,7 +1954,7 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
   p.sk_split = best_shared;
   p.grid = best_grid;
   p.sk_cols32 = (p.ncols + 31) / 32;
-  if (p.pair) p.epi_warps = kEpilogueWarps;
+  if (p.pair || p.sk_split) p.epi_warps = kEpilogueWarps;
   // split reduction (chosen with the tile shape above): fp32 partials, copy-style epilogue
   p.ks_log2 = best_ks;
   if (p.ks_log2 > 0) {
@@ -2237,9 +2268,24 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
     err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV, EWV, EPIV, SPLITV>,                                \
                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);            \
     if (err == cudaSuccess)                                                                                \
-      err = launch_kernel_coop(cooperative, igemm_kernel<KBV, HALOV, EWV, EPIV, SPLITV>, grid,             \
-                               dim3(64 + 32 * EWV), p.smem_bytes, stream, p.tmA, p.tmB, p.tmY, p.tmYr, a,  \
+      err = launch_kernel(igemm_kernel<KBV, HALOV, EWV, EPIV, SPLITV>, grid, dim3(64 + 32 * EWV),          \
+                          p.smem_bytes, stream, p.tmA, p.tmB, p.tmY, p.tmYr, a, bias, y, partials, status); \
+  } while (0)
+  // tiles shared between CTAs: their own instantiations (8 epilogue warps), launched cooperatively
+#define HGC_LAUNCH_SHARED_EPI(KBV, HALOV, EPIV)                                                            \
+  do {                                                                                                     \
+    err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV, 8, EPIV, false, false, true>,                      \
+                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);            \
+    if (err == cudaSuccess)                                                                                \
+      err = launch_kernel_coop(true, igemm_kernel<KBV, HALOV, 8, EPIV, false, false, true>, grid,          \
+                               dim3(64 + 32 * 8), p.smem_bytes, stream, p.tmA, p.tmB, p.tmY, p.tmYr, a,    \
                                bias, y, partials, status);                                                 \
+  } while (0)
+#define HGC_LAUNCH_SHARED(KBV, HALOV)                                \
+  do {                                                               \
+    if (p.y_nhwc) HGC_LAUNCH_SHARED_EPI(KBV, HALOV, 2);              \
+    else if (!p.tma_store) HGC_LAUNCH_SHARED_EPI(KBV, HALOV, 1);     \
+    else HGC_LAUNCH_SHARED_EPI(KBV, HALOV, 0);                       \
   } while (0)
 #define HGC_LAUNCH_IGEMM(KBV, HALOV)                                                              \
   do {                                                                                            \
@@ -2252,11 +2298,19 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
   // CTA pairs: launched as clusters of two, 8 epilogue warps, the three epilogue kinds
 #define HGC_LAUNCH_PAIR_EPI(KBV, HALOV, EPIV)                                                                  \
   do {                                                                                                       \
-    err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV, 8, EPIV, false, true>,                               \
-                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);              \
-    if (err == cudaSuccess)                                                                                  \
-      err = launch_pair(igemm_kernel<KBV, HALOV, 8, EPIV, false, true>, p, sms, cooperative, dim3(64 + 32 * 8), \
-                        stream, p.tmA, p.tmB, p.tmY, p.tmYr, a, bias, y, partials, status);                  \
+    if (cooperative) {                                                                                       \
+      err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV, 8, EPIV, false, true, true>,                       \
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);            \
+      if (err == cudaSuccess)                                                                                \
+        err = launch_pair(igemm_kernel<KBV, HALOV, 8, EPIV, false, true, true>, p, sms, true,                \
+                          dim3(64 + 32 * 8), stream, p.tmA, p.tmB, p.tmY, p.tmYr, a, bias, y, partials, status); \
+    } else {                                                                                                 \
+      err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV, 8, EPIV, false, true, false>,                      \
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);            \
+      if (err == cudaSuccess)                                                                                \
+        err = launch_pair(igemm_kernel<KBV, HALOV, 8, EPIV, false, true, false>, p, sms, false,              \
+                          dim3(64 + 32 * 8), stream, p.tmA, p.tmB, p.tmY, p.tmYr, a, bias, y, partials, status); \
+    }                                                                                                        \
   } while (0)
 #define HGC_LAUNCH_PAIR(KBV, HALOV)                                \
   do {                                                             \
@@ -2271,6 +2325,14 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
       if (p.halo) HGC_LAUNCH_PAIR(32, true); else HGC_LAUNCH_PAIR(32, false);
     } else {
       err = cudaErrorInvalidValue;  // (the planner pairs CTAs only with 32- or 64-channel stages)
+    }
+  } else if (p.sk_split) {
+    if (p.kb == 64) {
+      if (p.halo) HGC_LAUNCH_SHARED(64, true); else HGC_LAUNCH_SHARED(64, false);
+    } else if (p.kb == 32) {
+      if (p.halo) HGC_LAUNCH_SHARED(32, true); else HGC_LAUNCH_SHARED(32, false);
+    } else {
+      err = cudaErrorInvalidValue;  // (the planner shares tiles only with 32- or 64-channel stages)
     }
   } else
   if (p.ks_log2 > 0) {
@@ -2287,6 +2349,8 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
 #undef HGC_LAUNCH_IGEMM
 #undef HGC_LAUNCH_PAIR_EPI
 #undef HGC_LAUNCH_PAIR
+#undef HGC_LAUNCH_SHARED_EPI
+#undef HGC_LAUNCH_SHARED
   if (err != cudaSuccess) return err;
   count_launch();
   if (p.ks_log2 > 0) {
