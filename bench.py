@@ -331,7 +331,8 @@ def time_layers_as_graphs(hgc, torch, state, batch, side, replays=7):
         med, mn = timed(lambda i: hgc.conv_forward(d, xs[i], w, b, ys[i], l.relu, side))
         layout_ms = None
         info = d.plan_info() if d.path() == hgc.HGC_PATH_IGEMM else None
-        if info is not None and info["x_source"] == 0 and not (d.params.flags & hgc.HGC_FLAG_X_NHWC) and l.c % 8 == 0:
+        if (info is not None and info["x_source"] == 0 and not info["fused_layout"]
+                and not (d.params.flags & hgc.HGC_FLAG_X_NHWC) and l.c % 8 == 0):
             xt = torch.empty((batch, l.h, l.h, l.c), dtype=torch.float16, device="cuda")
             layout_ms, _ = timed(lambda i: hgc.layout_nchw_to_nhwc(xs[i], xt, batch, l.c, l.h, l.h, l.c, side))
             del xt

@@ -92,6 +92,15 @@ typedef struct hgc_conv_params {
  */
 #define HGC_FLAG_CTA_PAIRS 8
 #define HGC_FLAG_SHARED_TILES 16
+/*
+ * HGC_FLAG_FUSED_LAYOUT (off by default): layers whose input needs the NCHW->NHWC copy and whose
+ * output rows are whole 16-byte vectors (3x3 layers on 224, 112, 56 wide planes ...) make that
+ * copy inside the tensor-core kernel: eight extra warps of every CTA convert x while the MMAs of
+ * earlier tiles run, and a tile starts when the rows it reads are complete (a cooperative
+ * launch).  Measured on the VGG-16 layers: no faster than the copy as a kernel of its own (the
+ * step runs under the board's power cap, where work that overlaps costs what it costs alone).
+ */
+#define HGC_FLAG_FUSED_LAYOUT 32
 
 typedef struct hgc_conv_desc hgc_conv_desc; /* opaque; owned by the caller via create/destroy */
 
@@ -201,7 +210,9 @@ int hgc_conv_path(const hgc_conv_desc* d, int32_t* path);
  * stage adds the others' fp32 accumulators in a fixed order), 0 if every CTA takes whole tiles,
  * [14] 1 if the launch consists of CTA pairs (clusters of two that share tiles of 256 output
  * channels; [3], [4] then describe one CTA's pixel sub-tile, [6] the MMA N of the pair, [7] the
- * number of pair tiles, [12] the number of pairs); zeros for the other paths.  info: host pointer.
+ * number of pair tiles, [12] the number of pairs), [15] 1 if the NCHW->NHWC copy of x ([10] = 0)
+ * is made by extra warps of the tensor-core kernel itself instead of a kernel of its own; zeros
+ * for the other paths.  info: host pointer.
  */
 int hgc_conv_plan_info(const hgc_conv_desc* d, int32_t* info, int32_t count);
 

@@ -21,6 +21,7 @@ HGC_FLAG_X_NHWC = 2
 HGC_FLAG_Y_NHWC = 4
 HGC_FLAG_CTA_PAIRS = 8
 HGC_FLAG_SHARED_TILES = 16
+HGC_FLAG_FUSED_LAYOUT = 32
 PATH_NAMES = {HGC_PATH_DIRECT: "direct", HGC_PATH_DEPTHWISE: "depthwise", HGC_PATH_IGEMM: "igemm"}
 
 
@@ -170,10 +171,10 @@ class ConvDesc:
         return v.value
 
     def plan_info(self) -> dict:
-        v = (ctypes.c_int32 * 15)()
-        _check(lib().hgc_conv_plan_info(self._h, v, 15), "hgc_conv_plan_info")
+        v = (ctypes.c_int32 * 16)()
+        _check(lib().hgc_conv_plan_info(self._h, v, 16), "hgc_conv_plan_info")
         keys = ("path", "kb", "halo", "tn", "th", "pitch", "ncols", "tiles", "stages", "taps", "x_source",
-                "k_slices", "grid", "shared_tiles", "pair")
+                "k_slices", "grid", "shared_tiles", "pair", "fused_layout")
         return dict(zip(keys, list(v)))
 
     def workspace_bytes(self) -> int:

@@ -135,6 +135,7 @@ int hgc_conv_desc_create(hgc_conv_desc** out, const hgc_conv_params* p) {
   g.y_nhwc = (p->flags & HGC_FLAG_Y_NHWC) ? 1 : 0;
   g.no_pair = (p->flags & HGC_FLAG_CTA_PAIRS) ? 0 : 1;
   g.no_split = (p->flags & HGC_FLAG_SHARED_TILES) ? 0 : 1;
+  g.no_fuse = (p->flags & HGC_FLAG_FUSED_LAYOUT) ? 0 : 1;
   const bool channels_last = g.x_nhwc || g.y_nhwc;
 
   d->path = HGC_PATH_DIRECT;
@@ -216,7 +217,7 @@ int hgc_conv_path(const hgc_conv_desc* d, int32_t* path) {
 
 int hgc_conv_plan_info(const hgc_conv_desc* d, int32_t* info, int32_t count) {
   if (d == nullptr || info == nullptr || count < 1) return HGC_INVALID_ARG;
-  int32_t v[15] = {d->path, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+  int32_t v[16] = {d->path, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
   if (d->path == HGC_PATH_IGEMM) {
     const hgc::IgemmPlan& p = d->igemm;
     v[1] = p.kb; v[2] = p.halo; v[3] = p.tn; v[4] = p.th; v[5] = p.pitch; v[6] = p.ncols;
@@ -226,8 +227,9 @@ int hgc_conv_plan_info(const hgc_conv_desc* d, int32_t* info, int32_t count) {
     v[12] = p.ks_log2 > 0 ? 0 : ((p.pair && p.pair_fit > 0 && p.pair_fit < p.grid) ? p.pair_fit : p.grid);
     v[13] = p.sk_split;
     v[14] = p.pair;
+    v[15] = p.fuse_layout;
   }
-  for (int i = 0; i < count && i < 15; ++i) info[i] = v[i];
+  for (int i = 0; i < count && i < 16; ++i) info[i] = v[i];
   return HGC_OK;
 }
 
@@ -257,6 +259,10 @@ int hgc_conv_set_workspace(hgc_conv_desc* d, void* dev_ptr, size_t bytes) {
     // the TMA descriptors point into the workspace: encode them now; clear the status word
     if (!hgc::igemm_encode_maps(d->geom, &d->igemm, dev_ptr)) return HGC_CUDA_ERROR;
     if (cudaMemset(static_cast<char*>(dev_ptr) + d->igemm.ws_status_off, 0, hgc::kWsHeaderBytes) != cudaSuccess)
+      return HGC_CUDA_ERROR;
+    if (d->igemm.fuse_layout &&
+        cudaMemset(static_cast<char*>(dev_ptr) + d->igemm.ws_lay_off, 0,
+                   ((size_t)d->geom.n * d->igemm.lay_segs + 1) * sizeof(int)) != cudaSuccess)
       return HGC_CUDA_ERROR;
   }
   return HGC_OK;
@@ -288,6 +294,10 @@ int hgc_conv_last_device_status(hgc_conv_desc* d, int32_t* status) {
       *status = word;
       // the launch that gave up may have left hand-over flags raised: clear the whole header
       if (cudaMemset(sp, 0, hgc::kWsHeaderBytes) != cudaSuccess) return HGC_CUDA_ERROR;
+      if (d->igemm.fuse_layout &&
+          cudaMemset(static_cast<char*>(d->ws) + d->igemm.ws_lay_off, 0,
+                     ((size_t)d->geom.n * d->igemm.lay_segs + 1) * sizeof(int)) != cudaSuccess)
+        return HGC_CUDA_ERROR;
     }
   }
   // the TMA-fed channels-last depthwise kernel keeps one status word per process

@@ -20,6 +20,7 @@ struct ConvGeom {
   int32_t x_nhwc, y_nhwc;  // channels-last input / output (tensor-core path only)
   int32_t no_split;        // 1: never let several CTAs share the reduction of a tile (no scratch for it)
   int32_t no_pair;         // 1: never pair CTAs on 256-channel tiles
+  int32_t no_fuse;         // 1: the layout pass stays a kernel of its own
 };
 
 // First bytes of the tensor-core path's workspace: the device status word (int at byte 0) and,
@@ -171,6 +172,9 @@ struct IgemmPlan {
   // CTA pairs (clusters of two sharing 256-channel tiles): th/tn/tiles_h/tiles_n describe one
   // CTA's pixel sub-tile, ncols = 2 * ncols_sub, grid counts pairs; pair_fit = pairs that can be
   // resident at once (asked of the runtime at the first launch)
+  // layout pass fused into the tensor-core kernel (see IgemmArgs::lay_*): segment counters at ws_lay_off
+  int32_t fuse_layout, lay_px, lay_ch, lay_units_p, lay_units_c, lay_seg_units, lay_segs;
+  size_t ws_lay_off;
   int32_t pair, ncols_sub, pair_fit;
   double est_clk;  // the cost model's estimate for the launch, in SM clocks
   size_t ws_status_off, ws_w_off, ws_x_off, ws_part_off, ws_sk_off, ws_total;

@@ -251,6 +251,138 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
       : "memory");
 }
 
+// One unit of the fused layout pass (see IgemmArgs::lay_*): a thread owns 8 channels x PX
+// consecutive pixels: eight 16- or 8-byte loads (one per channel plane), a transpose of the
+// binary16 values in registers, PX 16-byte stores (one per pixel).  lane % CH picks the 8-channel
+// chunk and lane / CH the pixel group, so a store instruction writes CH*16 contiguous bytes per pixel.
+template <int CH, int PX>
+struct LayoutUnit {
+  static constexpr int PG = 32 / CH;
+  static constexpr int W32 = PX / 2;
+  uint32_t v[8][W32];
+  int64_t out;  // element offset of the thread's first output pixel in x', or -1: nothing to do
+  __device__ __forceinline__ void load(const uint16_t* __restrict__ src, int c, int64_t hw, int c_pad, int64_t n, int uc,
+                                       int64_t up) {
+    const int lane = threadIdx.x & 31;
+    const int c8 = lane % CH, pg = lane / CH;
+    const int ch = (uc * CH + c8) * 8;
+    const int64_t p = (up * PG + pg) * PX;
+    out = -1;
+    if (ch >= c_pad || p >= hw) return;
+    out = (n * hw + p) * c_pad + ch;
+    const uint16_t* s = src + (n * c + ch) * hw + p;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if (ch + i < c) {
+        if constexpr (PX == 8) {
+          const uint4 q = __ldcs(reinterpret_cast<const uint4*>(s + (int64_t)i * hw));
+          v[i][0] = q.x; v[i][1] = q.y; v[i][2] = q.z; v[i][3] = q.w;
+        } else {
+          const uint2 q = __ldcs(reinterpret_cast<const uint2*>(s + (int64_t)i * hw));
+          v[i][0] = q.x; v[i][1] = q.y;
+        }
+      } else {
+#pragma unroll
+        for (int w = 0; w < W32; ++w) v[i][w] = 0u;
+      }
+    }
+  }
+  __device__ __forceinline__ void store(uint16_t* __restrict__ dst, int c_pad) const {
+    if (out < 0) return;
+    uint16_t* d = dst + out;
+#pragma unroll
+    for (int q = 0; q < PX; ++q) {
+      const uint32_t sel = (q & 1) ? 0x7632u : 0x5410u;
+      uint32_t o[4];
+#pragma unroll
+      for (int m = 0; m < 4; ++m) o[m] = __byte_perm(v[2 * m][q >> 1], v[2 * m + 1][q >> 1], sel);
+      *reinterpret_cast<uint4*>(d + (int64_t)q * c_pad) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+  }
+};
+
+// The layout warps' loop: global warp `gw` of `nwarps` takes units gw, gw + nwarps, ... of the
+// sequence (image, pixel unit, channel unit), channel units fastest, two at a time (all loads of
+// both are under way before the first store), and reports each one.
+template <int CH, int PX>
+__device__ __noinline__ void layout_warp_loop(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int hw,
+                                              int c_pad, int units_p, int units_c, int seg_units, int segs, int N,
+                                              int* flags, int64_t gw, int64_t nwarps) {
+  const int64_t total = (int64_t)N * units_p * units_c;
+  for (int64_t u = gw; u < total; u += 2 * nwarps) {
+    LayoutUnit<CH, PX> a0, a1;
+    const int uc0 = (int)(u % units_c);
+    const int64_t t0 = u / units_c;
+    const int up0 = (int)(t0 % units_p);
+    const int64_t n0 = t0 / units_p;
+    a0.load(src, c, hw, c_pad, n0, uc0, up0);
+    const int64_t u1 = u + nwarps;
+    int up1 = 0;
+    int64_t n1 = 0;
+    if (u1 < total) {
+      const int uc1 = (int)(u1 % units_c);
+      const int64_t t1 = u1 / units_c;
+      up1 = (int)(t1 % units_p);
+      n1 = t1 / units_p;
+      a1.load(src, c, hw, c_pad, n1, uc1, up1);
+    } else {
+      a1.out = -1;
+    }
+    a0.store(dst, c_pad);
+    a1.store(dst, c_pad);
+    // the stores must be visible to the copy engines of every SM before the units are counted
+    asm volatile("fence.proxy.async.global;" ::: "memory");
+    __threadfence();
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) {
+      atomicAdd(flags + n0 * segs + up0 / seg_units, 1);
+      if (u1 < total) atomicAdd(flags + n1 * segs + up1 / seg_units, 1);
+    }
+  }
+}
+
+// Waits (bounded) until the pixel segments under input rows [h_lo, h_hi) of images n0 .. n0 + tn - 1
+// have been converted.  Whole warp; lane 0 polls.
+__device__ __noinline__ bool layout_wait(const int* flags, int N, int plane_h, int plane_w, int seg_px, int seg_units,
+                                         int segs, int units_p, int units_c, int n0, int tn, int h_lo, int h_hi,
+                                         volatile int* abort_flag) {
+  bool ok = true;
+  if ((threadIdx.x & 31) == 0) {
+    if (h_lo < 0) h_lo = 0;
+    if (h_hi > plane_h) h_hi = plane_h;
+    if (h_hi > h_lo) {
+      const int s_lo = (h_lo * plane_w) / seg_px, s_hi = (h_hi * plane_w - 1) / seg_px;
+      for (int img = 0; img < tn && ok; ++img) {
+        if (n0 + img >= N) break;
+        for (int sgm = s_lo; sgm <= s_hi && ok; ++sgm) {
+          const int units_here = units_p - sgm * seg_units < seg_units ? units_p - sgm * seg_units : seg_units;
+          const int target = units_here * units_c;
+          const int* f = flags + (int64_t)(n0 + img) * segs + sgm;
+          uint64_t t0 = 0;
+          for (uint32_t spin = 0;; ++spin) {
+            int v;
+            asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(f) : "memory");
+            if (v >= target) break;
+            __nanosleep(64);
+            if ((spin & 255u) == 255u) {
+              const uint64_t t = global_timer_ns();
+              if (t0 == 0) t0 = t;
+              if (*abort_flag || t - t0 > g_wait_limit_ns) {
+                *abort_flag = 1;
+                ok = false;
+                break;
+              }
+            }
+          }
+        }
+      }
+    }
+    asm volatile("fence.proxy.async.global;" ::: "memory");
+  }
+  ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+  return ok;
+}
+
 // Meeting point of the epilogue warps (one arrival per warp on an mbarrier initialised to their
 // number), with a bounded wait: false if it ran out or another role already gave up.  A plain
 // named barrier would hang the warps that reach it after others have left on a timeout.
@@ -783,6 +915,18 @@ struct IgemmArgs {
   // sk_split = 1: equal ranges; a tile that straddles a boundary is reduced by two or more CTAs:
   // the CTA that holds the tile's first stage finishes it, the others hand over their fp32
   // accumulators through `sk_part` (one slot per CTA, [column][128 lanes]) and raise `sk_flags`.
+  // Layout pass fused into the kernel (its own instantiations): extra warps of every CTA turn
+  // x[N][C][HW] into x'[N][HW][c_pad] in global memory, unit by unit in the order the tiles need
+  // them (a unit = 32 or 64 channels x 16 to 64 pixels of one image, channel chunks fastest), and
+  // count finished units per (image, pixel segment) in lay_flags; a tile's copies start when the
+  // segments under its input rows are complete.
+  const uint16_t* lay_x;
+  uint16_t* lay_xp;
+  int* lay_flags;        // [N][lay_segs] counters, then one counter of CTAs that have finished
+  int32_t lay_c, lay_cpad, lay_ch, lay_px;  // channels, padded channels, 8-channel chunks per unit (8 / 4), pixels per thread (8 / 4)
+  int32_t lay_hw, lay_w;                    // plane size and row width in pixels
+  int32_t lay_units_p, lay_units_c;         // units per image along the pixels / along the channels
+  int32_t lay_seg_units, lay_segs;          // pixel units per segment, segments per image
   int32_t dbg_drop;     // test hook: stage of the first CTA whose copies are left out (-1: none)
   int32_t ts;           // ring stages per tile: cblocks * R * (S / taps)
   // CTA pairs (clusters of two, tcgen05 cta_group::2): a tile is 256 output channels x two pixel
@@ -986,8 +1130,10 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 // Persistent kernel: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...; the two TMEM
 // accumulators alternate so that the epilogue of one tile overlaps the MMAs of the next.
 // EPI: 0 = TMA-store epilogue, 1 = copy epilogue (NCHW, any shape), 2 = channels-last output
-template <int KB, bool HALO, int EW, int EPI, bool SPLIT, bool PAIR = false, bool SHARED = false>
-__global__ void __launch_bounds__(64 + 32 * EW, 1)
+constexpr int kLayoutWarps = 8;  // extra warps of the instantiations with the fused layout pass
+
+template <int KB, bool HALO, int EW, int EPI, bool SPLIT, bool PAIR = false, bool SHARED = false, bool FUSEL = false>
+__global__ void __launch_bounds__(64 + 32 * EW + (FUSEL ? 32 * kLayoutWarps : 0), 1)
 igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
              const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmYr,
              const IgemmArgs a, const __half* __restrict__ bias, __half* __restrict__ y, float* __restrict__ partials,
@@ -1072,6 +1218,15 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       const int h_base = p0 * a.stride_h - a.pad_h;
       int s0, s1;
       it.stage_range(a, s0, s1);
+      if constexpr (FUSEL) {
+        // the tile reads input rows h_base .. h_base + (th-1)*stride + (R-1)*dil of tn images
+        if (!layout_wait(a.lay_flags, a.N, a.lay_hw / a.lay_w, a.lay_w, a.lay_seg_units * (32 / a.lay_ch) * a.lay_px,
+                         a.lay_seg_units, a.lay_segs, a.lay_units_p, a.lay_units_c, n0, a.tn, h_base,
+                         h_base + (a.th - 1) * a.stride_h + (a.R - 1) * a.dil_h + 1, &abort_flag)) {
+          ok = false;
+          break;
+        }
+      }
       // stage s of a tile = (channel block cb, kernel row r, tap group sg), sg fastest
       int cb = 0, r = 0, sg = 0;
       if (SHARED || SPLIT) {  // (whole tiles start at stage 0)
@@ -1209,7 +1364,23 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         __syncwarp();
       }
     }
-  } else if (warp >= 2) {
+  } else if (FUSEL && warp >= 2 + EW) {
+    // ---------------- fused layout pass (warps past the epilogue's) ----------------
+    const int64_t gw = (int64_t)blockIdx.x * kLayoutWarps + (warp - 2 - EW);
+    const int64_t nw = (int64_t)gridDim.x * kLayoutWarps;
+    if (a.lay_ch == 8 && a.lay_px == 8)
+      layout_warp_loop<8, 8>(a.lay_x, a.lay_xp, a.lay_c, a.lay_hw, a.lay_cpad, a.lay_units_p, a.lay_units_c, a.lay_seg_units,
+                             a.lay_segs, a.N, a.lay_flags, gw, nw);
+    else if (a.lay_px == 8)
+      layout_warp_loop<4, 8>(a.lay_x, a.lay_xp, a.lay_c, a.lay_hw, a.lay_cpad, a.lay_units_p, a.lay_units_c, a.lay_seg_units,
+                             a.lay_segs, a.N, a.lay_flags, gw, nw);
+    else if (a.lay_ch == 8)
+      layout_warp_loop<8, 4>(a.lay_x, a.lay_xp, a.lay_c, a.lay_hw, a.lay_cpad, a.lay_units_p, a.lay_units_c, a.lay_seg_units,
+                             a.lay_segs, a.N, a.lay_flags, gw, nw);
+    else
+      layout_warp_loop<4, 4>(a.lay_x, a.lay_xp, a.lay_c, a.lay_hw, a.lay_cpad, a.lay_units_p, a.lay_units_c, a.lay_seg_units,
+                             a.lay_segs, a.N, a.lay_flags, gw, nw);
+  } else if (warp >= 2 && warp < 2 + EW) {
     // ---------------- epilogue (warps 2..9) ----------------
     // Warp w may read TMEM lanes 32*(w%4)..+31; the EW/4 warps of a lane quarter take the units of
     // a tile in turn.
@@ -1513,6 +1684,19 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
   }
   if (threadIdx.x == 0 && abort_flag && status != nullptr) atomicExch(status, (int)HGC_DEVICE_TIMEOUT);
+  if constexpr (FUSEL) {
+    // the CTA that finishes last lowers the segment counters for the next launch
+    __shared__ int last_cta;
+    const int nflags = a.N * a.lay_segs;
+    if (threadIdx.x == 0) {
+      __threadfence();
+      last_cta = atomicAdd(a.lay_flags + nflags, 1) == (int)gridDim.x - 1;
+    }
+    __syncthreads();
+    if (last_cta) {
+      for (int i = threadIdx.x; i <= nflags; i += blockDim.x) a.lay_flags[i] = 0;
+    }
+  }
 }
 
 // ---- host side ----------------------------------------------------------------------------------
@@ -2032,6 +2216,31 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
     p.ws_part_off = p.ws_total;
     p.ws_total += round_up_sz(((size_t)g.n * g.k * g.p * g.q * 4) << p.ks_log2, 256);
   }
+  // Layout pass inside the tensor-core kernel (extra warps convert x while the MMAs run; a tile
+  // waits for the segments it reads): layers that take the plain NHWC copy of x, planes of a
+  // multiple of 4 pixels, whole 8-channel chunks, 8 epilogue warps, NCHW output.
+  p.fuse_layout = 0;
+  p.ws_lay_off = 0;
+  // On request (HGC_FLAG_FUSED_LAYOUT), with the TMA-store epilogue (planes whose rows are whole
+  // 16-byte vectors: the large ones, where the copy is worth hiding).  Measured: the VGG-16 layers
+  // take as long as with the separate pass (conv1_2 116 us against 112, conv3_2 65 against 61):
+  // they run under the power cap, and on small inputs the first tiles wait for their rows.
+  if (!g.no_fuse && !p.nchw && !p.x_nhwc && !p.window && !p.patch && !p.pair && !p.sk_split && p.ks_log2 == 0 &&
+      !p.y_nhwc && p.tma_store && p.kb >= 32 && p.epi_warps == kEpilogueWarps && ((int64_t)g.h * g.w) % 4 == 0 &&
+      (g.c % 8) == 0 && (int64_t)g.h * g.w <= 0x7fffffffLL / 4 && sms <= kMaxGrid) {
+    p.fuse_layout = 1;
+    const int hw = g.h * g.w;
+    p.lay_px = (hw % 8) == 0 ? 8 : 4;
+    p.lay_ch = p.c_pad >= 64 ? 8 : 4;
+    const int unit_px = (32 / p.lay_ch) * p.lay_px;
+    p.lay_units_p = (hw + unit_px - 1) / unit_px;
+    p.lay_units_c = (p.c_pad / 8 + p.lay_ch - 1) / p.lay_ch;
+    // segments of about 512 pixels (at least one unit)
+    p.lay_seg_units = 512 / unit_px > 0 ? 512 / unit_px : 1;
+    p.lay_segs = (p.lay_units_p + p.lay_seg_units - 1) / p.lay_seg_units;
+    p.ws_lay_off = p.ws_total;
+    p.ws_total += round_up_sz(((size_t)g.n * p.lay_segs + 1) * sizeof(int), 256);
+  }
   p.ws_sk_off = 0;
   if (p.sk_split) {  // one hand-over slot per CTA: [sk_cols32 * 32 columns][128 lanes] fp32
     p.ws_sk_off = p.ws_total;
@@ -2245,6 +2454,13 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
   a.y_full_w = p.y_full_w;
   a.y_rpu = p.y_rpu > 0 ? p.y_rpu : 1;
   a.dbg_drop = debug_drop_copies();
+  a.lay_x = reinterpret_cast<const uint16_t*>(x);
+  a.lay_xp = reinterpret_cast<uint16_t*>(static_cast<char*>(ws) + p.ws_x_off);
+  a.lay_flags = reinterpret_cast<int*>(static_cast<char*>(ws) + p.ws_lay_off);
+  a.lay_c = g.c; a.lay_cpad = p.c_pad; a.lay_ch = p.lay_ch; a.lay_px = p.lay_px;
+  a.lay_hw = g.h * g.w; a.lay_w = g.w;
+  a.lay_units_p = p.lay_units_p; a.lay_units_c = p.lay_units_c;
+  a.lay_seg_units = p.lay_seg_units; a.lay_segs = p.lay_segs;
   a.ts = p.ts;
   a.pair = p.pair;
   a.ncols_sub = p.ncols_sub;
@@ -2271,6 +2487,18 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
       err = launch_kernel(igemm_kernel<KBV, HALOV, EWV, EPIV, SPLITV>, grid, dim3(64 + 32 * EWV),          \
                           p.smem_bytes, stream, p.tmA, p.tmB, p.tmY, p.tmYr, a, bias, y, partials, status); \
   } while (0)
+  // fused layout pass: its own instantiations (8 epilogue + 4 layout warps), launched cooperatively
+  // (a tile waits for segments that other CTAs' layout warps convert)
+#define HGC_LAUNCH_FUSED_EPI(KBV, HALOV, EPIV)                                                             \
+  do {                                                                                                     \
+    err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV, 8, EPIV, false, false, false, true>,               \
+                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);            \
+    if (err == cudaSuccess)                                                                                \
+      err = launch_kernel_coop(true, igemm_kernel<KBV, HALOV, 8, EPIV, false, false, false, true>, grid,   \
+                               dim3(64 + 32 * 8 + 32 * kLayoutWarps), p.smem_bytes, stream, p.tmA, p.tmB,  \
+                               p.tmY, p.tmYr, a, bias, y, partials, status);                               \
+  } while (0)
+#define HGC_LAUNCH_FUSED(KBV, HALOV) HGC_LAUNCH_FUSED_EPI(KBV, HALOV, 0)
   // tiles shared between CTAs: their own instantiations (8 epilogue warps), launched cooperatively
 #define HGC_LAUNCH_SHARED_EPI(KBV, HALOV, EPIV)                                                            \
   do {                                                                                                     \
@@ -2326,6 +2554,14 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
     } else {
       err = cudaErrorInvalidValue;  // (the planner pairs CTAs only with 32- or 64-channel stages)
     }
+  } else if (p.fuse_layout) {
+    if (p.kb == 64) {
+      if (p.halo) HGC_LAUNCH_FUSED(64, true); else HGC_LAUNCH_FUSED(64, false);
+    } else if (p.kb == 32) {
+      if (p.halo) HGC_LAUNCH_FUSED(32, true); else HGC_LAUNCH_FUSED(32, false);
+    } else {
+      err = cudaErrorInvalidValue;
+    }
   } else if (p.sk_split) {
     if (p.kb == 64) {
       if (p.halo) HGC_LAUNCH_SHARED(64, true); else HGC_LAUNCH_SHARED(64, false);
@@ -2351,6 +2587,8 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
 #undef HGC_LAUNCH_PAIR
 #undef HGC_LAUNCH_SHARED_EPI
 #undef HGC_LAUNCH_SHARED
+#undef HGC_LAUNCH_FUSED_EPI
+#undef HGC_LAUNCH_FUSED
   if (err != cudaSuccess) return err;
   count_launch();
   if (p.ks_log2 > 0) {

@@ -618,6 +618,7 @@ cudaError_t launch_igemm_weights(const ConvGeom& g, const IgemmPlan& p, const __
 cudaError_t launch_igemm_input(const ConvGeom& g, const IgemmPlan& p, const __half* x, __half* xp,
                                cudaStream_t stream) {
   if (p.nchw || p.x_nhwc) return cudaSuccess;  // the kernel reads x itself
+  if (p.fuse_layout) return cudaSuccess;       // the tensor-core kernel converts x itself
   if (p.patch) return launch_patch_im2col(g, x, xp, p.cw, stream);
   if (p.window) return launch_nchw_to_nhwc8_bordered(x, xp, g.n, g.c, g.h, g.w, g.pad_h, g.pad_w, p.hp, p.wp, stream, p.px_ch);
   return launch_nchw_to_nhwc(x, xp, g.n, g.c, g.h, g.w, p.c_pad, stream);

@@ -63,6 +63,7 @@ int make_geom(const hgc_conv_params* p, hgc::ConvGeom* g) {
   // the scheduling flags are ignored: whole tiles on single CTAs (no hand-over slots in the fixed array)
   g->no_split = 1;
   g->no_pair = 1;
+  g->no_fuse = 1;
   return HGC_OK;
 }
 

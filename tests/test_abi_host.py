@@ -114,7 +114,7 @@ def test_planner_paths():
 def test_plan_info_reports_tiling_and_activation_source():
     """The planner runs on the host: its choices can be checked without a GPU."""
     keys = {"path", "kb", "halo", "tn", "th", "pitch", "ncols", "tiles", "stages", "taps", "x_source", "k_slices",
-            "grid", "shared_tiles", "pair"}
+            "grid", "shared_tiles", "pair", "fused_layout"}
     cases = [
         # (n, c, h, w, k, r, s, pad, stride), x_source
         ((16, 256, 56, 56, 256, 3, 3, 1, 1), 0),   # NHWC copy of x

@@ -111,14 +111,26 @@ SCHED_CASES = [
      {"pair": 1, "shared_tiles": 1}),
     ("pairs + shared 3x3 c512 k512 14x14 n3", params_dict(3, 512, 14, 14, 512, 3, 3, 1, 1), ("pairs", "shared"),
      {"pair": 1, "shared_tiles": 1}),
+    ("fused layout 3x3 c64 k64 56x56 n5 (64-channel units)", params_dict(5, 64, 56, 56, 64, 3, 3, 1, 1), ("fused",),
+     {"fused_layout": 1}),
+    ("fused layout 3x3 c40 k72 24x40 n3 (32-channel units, ragged channel and pixel units)",
+     params_dict(3, 40, 24, 40, 72, 3, 3, 1, 1), ("fused",), {"fused_layout": 1}),
+    ("fused layout 3x3 stride 2 c128 k96 34x32 n2", params_dict(2, 128, 34, 32, 96, 3, 3, 1, 1, 2, 2), ("fused",),
+     {"fused_layout": 1}),
+    ("fused layout 5x5 grouped c96 k64 24x24 n2", params_dict(2, 96, 24, 24, 64, 5, 5, 2, 2, 1, 1, 1, 1, 2), ("fused",),
+     {"fused_layout": 1}),
+    ("fused layout: 13x13 plane keeps the separate pass", params_dict(2, 96, 13, 13, 72, 3, 3, 1, 1), ("fused",),
+     {"fused_layout": 0}),
 ]
 
 
 @pytest.mark.parametrize("name,a,flag_names,want", SCHED_CASES, ids=[c[0] for c in SCHED_CASES])
 def test_scheduling_flags(hgc, oracle, name, a, flag_names, want):
-    """CTA pairs (cta_group::2) and tiles shared by several CTAs are opt-in schedules of the same
-    layer: the plan must report them where asked for, and the results must match the oracle."""
-    flags = (hgc.HGC_FLAG_CTA_PAIRS if "pairs" in flag_names else 0) | (hgc.HGC_FLAG_SHARED_TILES if "shared" in flag_names else 0)
+    """CTA pairs (cta_group::2), tiles shared by several CTAs and the layout pass inside the
+    tensor-core kernel are opt-in schedules of the same layer: the plan must report them where
+    asked for, and the results must match the oracle."""
+    flags = ((hgc.HGC_FLAG_CTA_PAIRS if "pairs" in flag_names else 0) | (hgc.HGC_FLAG_SHARED_TILES if "shared" in flag_names else 0)
+             | (hgc.HGC_FLAG_FUSED_LAYOUT if "fused" in flag_names else 0))
     rng = np.random.default_rng(zlib.crc32(name.encode()))
     x, w, b = workloads.random_layer_tensors(rng, a["n"], a["c"], a["h"], a["w"], a["k"], a["r"], a["s"], a["group"])
     P = oracle.ConvParams(**a)

@@ -38,10 +38,12 @@ def _forward(hgc, d, xd, wd, bd, shape, relu=True):
     ("several CTAs, first stage of the first CTA", params_dict(4, 64, 16, 16, 256, 3, 3, 1, 1), "", 0),
     ("CTA pairs: the first CTA's copies of a stage", params_dict(2, 64, 12, 12, 256, 3, 3, 1, 1), "pairs", 2),
     ("tiles shared between CTAs: a part that is never handed over", params_dict(2, 256, 24, 24, 256, 3, 3, 1, 1), "shared", 0),
+    ("layout pass inside the kernel", params_dict(2, 64, 24, 24, 64, 3, 3, 1, 1), "fused", 1),
 ])
 def test_tensor_core_wait_runs_out_and_the_descriptor_recovers(hgc, oracle, name, a, flags_name, drop):
     import torch
-    flags = {"": 0, "pairs": hgc.HGC_FLAG_CTA_PAIRS, "shared": hgc.HGC_FLAG_SHARED_TILES}[flags_name]
+    flags = {"": 0, "pairs": hgc.HGC_FLAG_CTA_PAIRS, "shared": hgc.HGC_FLAG_SHARED_TILES,
+             "fused": hgc.HGC_FLAG_FUSED_LAYOUT}[flags_name]
     rng = np.random.default_rng(3)
     x, w, b = workloads.random_layer_tensors(rng, a["n"], a["c"], a["h"], a["w"], a["k"], a["r"], a["s"], a["group"])
     ref = oracle.conv_fast(oracle.ConvParams(**a), x, w, b, True)
