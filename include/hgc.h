@@ -329,6 +329,35 @@ int hgc_bn_fold(const void* w, const void* bias, const float* mean, const float*
                 const float* beta, float eps, int32_t k, int64_t per_k, void* w_out, void* b_out, void* stream);
 
 /*
+ * A depthwise-separable block as one kernel (Section 3.3: nothing is converted or stored between
+ * layers that the engine itself chains): the 3x3 depthwise layer (group = C, pad 1, stride 1 or
+ * 2, + bias, optional ReLU, rounded once to binary16 as the layer's output would be) followed by
+ * the 1x1 pointwise layer C -> K (+ bias, optional ReLU).  The depthwise result is never written
+ * to memory: extra warps of the tensor-core kernel compute it tile by tile straight into the
+ * shared-memory stages that the MMAs of the pointwise layer read.
+ *   x: [N][H][W][C] channels-last (C a multiple of 8, at least 16); w_dw: [C][1][3][3];
+ *   w_pw: [K][C][1][1]; y: [N][K][P][Q], or [N][P][Q][K] with HGC_FLAG_Y_NHWC in p->flags
+ *   (P, Q: the depthwise layer's output plane; hgc_conv_output_dims reports N, K, P, Q).
+ * The descriptor is used with hgc_conv_workspace_bytes / hgc_conv_set_workspace /
+ * hgc_conv_last_device_status / hgc_conv_desc_destroy like a layer descriptor, and with
+ * hgc_dwpw_set_weights (optional: prepares both weight tensors once) and hgc_dwpw_forward
+ * (device pointers, 16-byte aligned, bias pointers may be NULL; queued on `stream`).
+ * Errors: HGC_INVALID_ARG (NULL, sizes < 1, stride other than 1 or 2, other flags, a layer
+ * descriptor passed to hgc_dwpw_* or a block descriptor to hgc_conv_forward), HGC_UNSUPPORTED
+ * (C not a multiple of 8 or below 16), HGC_BAD_ALIGNMENT, HGC_NO_WORKSPACE, HGC_CUDA_ERROR.
+ */
+typedef struct hgc_dwpw_params {
+  int32_t n, c, h, w;   /* input, channels-last */
+  int32_t k;            /* output channels of the pointwise layer */
+  int32_t stride;       /* of the depthwise layer: 1 or 2 */
+  int32_t flags;        /* 0 or HGC_FLAG_Y_NHWC */
+} hgc_dwpw_params;
+int hgc_dwpw_desc_create(hgc_conv_desc** out, const hgc_dwpw_params* p);
+int hgc_dwpw_set_weights(hgc_conv_desc* d, const void* w_dw, const void* w_pw, void* stream);
+int hgc_dwpw_forward(hgc_conv_desc* d, const void* x, const void* w_dw, const void* bias_dw, const void* w_pw,
+                     const void* bias_pw, void* y, int relu_dw, int relu_pw, void* stream);
+
+/*
  * Test hooks for the failure-detection path (Section 3.2 of the paper keeps scalars and control on
  * the host; a device-side wait that cannot be interrupted from the host therefore has to end by
  * itself).  Every wait of the TMA-fed kernels (tensor-core path, channels-last depthwise) on a

@@ -31,6 +31,10 @@ class HgcError(RuntimeError):
         super().__init__(f"{where}: {status_string(status)} (hgc_status {status})")
 
 
+class hgc_dwpw_params(ctypes.Structure):
+    _fields_ = [(f, ctypes.c_int32) for f in ("n", "c", "h", "w", "k", "stride", "flags")]
+
+
 class hgc_conv_params(ctypes.Structure):
     _fields_ = [(f, ctypes.c_int32) for f in (
         "n", "c", "h", "w", "k", "r", "s", "pad_h", "pad_w", "stride_h", "stride_w",
@@ -75,6 +79,9 @@ def lib() -> ctypes.CDLL:
         L.hgc_weights_repack.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, vp]
         L.hgc_kernel_launch_count.argtypes = [ctypes.POINTER(ctypes.c_uint64)]
         L.hgc_set_launch_overlap.argtypes = [ctypes.c_int]
+        L.hgc_dwpw_desc_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(hgc_dwpw_params)]
+        L.hgc_dwpw_set_weights.argtypes = [vp, vp, vp, vp]
+        L.hgc_dwpw_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_int, ctypes.c_int, vp]
         L.hgc_debug_set_wait_limit_ns.argtypes = [ctypes.c_uint64]
         L.hgc_debug_drop_copies.argtypes = [i32]
         L.hgc_status_string.argtypes = [ctypes.c_int]
@@ -86,7 +93,8 @@ def lib() -> ctypes.CDLL:
                      "hgc_layout_nchw_to_nhwc", "hgc_layout_nhwc_to_nchw", "hgc_weights_repack",
                      "hgc_kernel_launch_count", "hgc_inner_product_desc_create", "hgc_cast_f32_to_f16",
                      "hgc_set_launch_overlap", "hgc_batchnorm_forward", "hgc_bn_fold",
-                     "hgc_debug_set_wait_limit_ns", "hgc_debug_drop_copies"):
+                     "hgc_debug_set_wait_limit_ns", "hgc_debug_drop_copies", "hgc_dwpw_desc_create",
+                     "hgc_dwpw_set_weights", "hgc_dwpw_forward"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -212,6 +220,30 @@ class ConvDesc:
         v = ctypes.c_int32()
         _check(lib().hgc_conv_last_device_status(self._h, ctypes.byref(v)), "hgc_conv_last_device_status")
         return v.value
+
+
+class DwPwDesc(ConvDesc):
+    """hgc_dwpw_desc_create: a 3x3 depthwise layer (stride 1 or 2, pad 1) and the 1x1 pointwise layer
+    behind it as one kernel; x channels-last.  Shares workspace / status / output_dims / close with
+    ConvDesc."""
+
+    def __init__(self, n, c, h, w, k, stride=1, flags=0):
+        self.block_params = hgc_dwpw_params(n, c, h, w, k, stride, flags)
+        self.params = hgc_conv_params(n, c, h, w, k, 1, 1, 0, 0, 1, 1, 1, 1, 1, flags)
+        self._h = ctypes.c_void_p()
+        self._ws = None
+        _check(lib().hgc_dwpw_desc_create(ctypes.byref(self._h), ctypes.byref(self.block_params)),
+               "hgc_dwpw_desc_create")
+
+    def set_weights(self, w_dw, w_pw, stream=None):
+        _check(lib().hgc_dwpw_set_weights(self._h, _ptr(w_dw), _ptr(w_pw), _stream(stream)), "hgc_dwpw_set_weights")
+
+
+def dwpw_forward(desc: DwPwDesc, x, w_dw, bias_dw, w_pw, bias_pw, y, relu_dw: bool, relu_pw: bool, stream=None):
+    """hgc_dwpw_forward: x [N,H,W,C] channels-last, w_dw [C,1,3,3], w_pw [K,C,1,1], y [N,K,P,Q] (or
+    [N,P,Q,K] with HGC_FLAG_Y_NHWC): CUDA fp16 tensors; biases may be None."""
+    _check(lib().hgc_dwpw_forward(desc.handle, _ptr(x), _ptr(w_dw), _ptr(bias_dw), _ptr(w_pw), _ptr(bias_pw), _ptr(y),
+                                  int(bool(relu_dw)), int(bool(relu_pw)), _stream(stream)), "hgc_dwpw_forward")
 
 
 def conv_forward(desc: ConvDesc, x, w, bias, y, relu: bool, stream=None):

@@ -24,6 +24,12 @@ struct hgc_conv_desc {
   size_t ws_bytes;
   const void* registered_w;
   hgc::IgemmPlan igemm;
+  // depthwise + pointwise block (hgc_dwpw_desc_create): geom / igemm describe the pointwise layer
+  // on the depthwise layer's output plane; the depthwise layer itself:
+  bool is_dwpw;
+  int32_t dw_h, dw_w, dw_stride;
+  size_t ws_dw_off;             // depthwise weights as [9][C] in the workspace
+  const void* registered_w_dw;
 };
 
 namespace {
@@ -170,6 +176,7 @@ int hgc_conv_desc_destroy(hgc_conv_desc* d) {
 int hgc_conv_forward(hgc_conv_desc* d, const void* x, const void* w, const void* bias, void* y,
                      int relu, void* stream) {
   if (d == nullptr || x == nullptr || w == nullptr || y == nullptr) return HGC_INVALID_ARG;
+  if (d->is_dwpw) return HGC_INVALID_ARG;  // a block descriptor: hgc_dwpw_forward
   if (misaligned(x) || misaligned(w) || misaligned(y) || (bias != nullptr && misaligned(bias)))
     return HGC_BAD_ALIGNMENT;
   if (d->ws_needed > 0 && (d->ws == nullptr || d->ws_bytes < d->ws_needed)) return HGC_NO_WORKSPACE;
@@ -179,6 +186,7 @@ int hgc_conv_forward(hgc_conv_desc* d, const void* x, const void* w, const void*
 int hgc_conv_forward_host(hgc_conv_desc* d, const void* x, const void* w, const void* bias, void* y,
                           int relu, void* stream) {
   if (d == nullptr || x == nullptr || w == nullptr || y == nullptr) return HGC_INVALID_ARG;
+  if (d->is_dwpw) return HGC_INVALID_ARG;
   const HostStaging s = host_staging(d);
   if (d->ws == nullptr || d->ws_bytes < s.total) return HGC_NO_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -252,6 +260,7 @@ int hgc_conv_set_workspace(hgc_conv_desc* d, void* dev_ptr, size_t bytes) {
   d->ws = dev_ptr;
   d->ws_bytes = dev_ptr ? bytes : 0;
   d->registered_w = nullptr;
+  d->registered_w_dw = nullptr;
   d->igemm.maps_ready = false;
   d->igemm.y_mapped = nullptr;
   d->igemm.x_mapped = nullptr;
@@ -270,6 +279,7 @@ int hgc_conv_set_workspace(hgc_conv_desc* d, void* dev_ptr, size_t bytes) {
 
 int hgc_conv_set_weights(hgc_conv_desc* d, const void* w, void* stream) {
   if (d == nullptr || w == nullptr) return HGC_INVALID_ARG;
+  if (d->is_dwpw) return HGC_INVALID_ARG;  // hgc_dwpw_set_weights
   if (misaligned(w)) return HGC_BAD_ALIGNMENT;
   if (d->ws_needed > 0 && (d->ws == nullptr || d->ws_bytes < d->ws_needed)) return HGC_NO_WORKSPACE;
   if (d->path == HGC_PATH_IGEMM) {
@@ -340,6 +350,97 @@ int hgc_weights_repack(const void* src, void* dst, int32_t k, int32_t c_per_grou
   cudaError_t err = hgc::launch_weights_repack(static_cast<const __half*>(src), static_cast<__half*>(dst), k,
                                               c_per_group, r, s, group, c_pad,
                                               static_cast<cudaStream_t>(stream));
+  return err == cudaSuccess ? HGC_OK : HGC_CUDA_ERROR;
+}
+
+int hgc_dwpw_desc_create(hgc_conv_desc** out, const hgc_dwpw_params* p) {
+  if (out == nullptr) return HGC_INVALID_ARG;
+  *out = nullptr;
+  if (p == nullptr) return HGC_INVALID_ARG;
+  if (p->n < 1 || p->c < 1 || p->h < 1 || p->w < 1 || p->k < 1) return HGC_INVALID_ARG;
+  if (p->stride != 1 && p->stride != 2) return HGC_INVALID_ARG;
+  if (p->flags & ~HGC_FLAG_Y_NHWC) return HGC_INVALID_ARG;
+  // the depthwise layer: 3x3, pad 1; its output plane is the pointwise layer's plane
+  const int64_t P = out_extent(p->h, 3, 1, p->stride, 1);
+  const int64_t Q = out_extent(p->w, 3, 1, p->stride, 1);
+  if (P < 1 || Q < 1) return HGC_INVALID_ARG;
+  hgc_conv_desc* d = new (std::nothrow) hgc_conv_desc();
+  if (d == nullptr) return HGC_CUDA_ERROR;
+  hgc_conv_params& cp = d->params;
+  cp.n = p->n; cp.c = p->c; cp.h = (int32_t)P; cp.w = (int32_t)Q; cp.k = p->k; cp.r = 1; cp.s = 1;
+  cp.pad_h = 0; cp.pad_w = 0; cp.stride_h = 1; cp.stride_w = 1; cp.dil_h = 1; cp.dil_w = 1; cp.group = 1;
+  cp.flags = HGC_FLAG_X_NHWC | (p->flags & HGC_FLAG_Y_NHWC);
+  hgc::ConvGeom& g = d->geom;
+  g.n = p->n; g.c = p->c; g.h = (int32_t)P; g.w = (int32_t)Q; g.k = p->k; g.r = 1; g.s = 1;
+  g.pad_h = 0; g.pad_w = 0; g.stride_h = 1; g.stride_w = 1; g.dil_h = 1; g.dil_w = 1; g.group = 1;
+  g.p = (int32_t)P; g.q = (int32_t)Q; g.cg = p->c; g.kg = p->k;
+  g.x_nhwc = 1;
+  g.y_nhwc = (p->flags & HGC_FLAG_Y_NHWC) ? 1 : 0;
+  g.no_pair = 1; g.no_split = 1; g.no_fuse = 1;
+  g.dw_stride = p->stride;
+  // the tensor-core plan of the pointwise layer over a channels-last input that is never stored:
+  // whole 8-channel chunks, 32- or 64-channel stages, whole tiles on single CTAs
+  if ((p->c % 8) != 0 || !hgc::igemm_make_plan(g, &d->igemm) || d->igemm.kb < 32 || d->igemm.ks_log2 > 0 ||
+      !d->igemm.x_nhwc || d->igemm.dw_in_bytes == 0) {
+    delete d;
+    return HGC_UNSUPPORTED;
+  }
+  d->path = HGC_PATH_IGEMM;
+  d->is_dwpw = true;
+  d->dw_h = p->h; d->dw_w = p->w; d->dw_stride = p->stride;
+  d->ws_dw_off = round_up(d->igemm.ws_total, 256);
+  d->ws_needed = d->ws_dw_off + round_up((size_t)9 * p->c * 2, 256);
+  d->ws = nullptr;
+  d->ws_bytes = 0;
+  d->registered_w = nullptr;
+  d->registered_w_dw = nullptr;
+  *out = d;
+  return HGC_OK;
+}
+
+int hgc_dwpw_set_weights(hgc_conv_desc* d, const void* w_dw, const void* w_pw, void* stream) {
+  if (d == nullptr || w_dw == nullptr || w_pw == nullptr || !d->is_dwpw) return HGC_INVALID_ARG;
+  if (misaligned(w_dw) || misaligned(w_pw)) return HGC_BAD_ALIGNMENT;
+  if (d->ws == nullptr || d->ws_bytes < d->ws_needed) return HGC_NO_WORKSPACE;
+  char* ws = static_cast<char*>(d->ws);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (hgc::launch_igemm_weights(d->geom, d->igemm, static_cast<const __half*>(w_pw),
+                                reinterpret_cast<__half*>(ws + d->igemm.ws_w_off), st) != cudaSuccess)
+    return HGC_CUDA_ERROR;
+  if (hgc::launch_depthwise_weights_to_taps(static_cast<const __half*>(w_dw), reinterpret_cast<__half*>(ws + d->ws_dw_off),
+                                            d->geom.c, st) != cudaSuccess)
+    return HGC_CUDA_ERROR;
+  d->registered_w = w_pw;
+  d->registered_w_dw = w_dw;
+  return HGC_OK;
+}
+
+int hgc_dwpw_forward(hgc_conv_desc* d, const void* x, const void* w_dw, const void* bias_dw, const void* w_pw,
+                     const void* bias_pw, void* y, int relu_dw, int relu_pw, void* stream) {
+  if (d == nullptr || x == nullptr || w_dw == nullptr || w_pw == nullptr || y == nullptr || !d->is_dwpw)
+    return HGC_INVALID_ARG;
+  if (misaligned(x) || misaligned(w_dw) || misaligned(w_pw) || misaligned(y) || (bias_dw != nullptr && misaligned(bias_dw)) ||
+      (bias_pw != nullptr && misaligned(bias_pw)))
+    return HGC_BAD_ALIGNMENT;
+  if (d->ws == nullptr || d->ws_bytes < d->ws_needed) return HGC_NO_WORKSPACE;
+  char* ws = static_cast<char*>(d->ws);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (d->registered_w != w_pw || d->registered_w_dw != w_dw) {  // weights not prepared in advance: re-lay them out now
+    if (hgc::launch_igemm_weights(d->geom, d->igemm, static_cast<const __half*>(w_pw),
+                                  reinterpret_cast<__half*>(ws + d->igemm.ws_w_off), st) != cudaSuccess)
+      return HGC_CUDA_ERROR;
+    if (hgc::launch_depthwise_weights_to_taps(static_cast<const __half*>(w_dw), reinterpret_cast<__half*>(ws + d->ws_dw_off),
+                                              d->geom.c, st) != cudaSuccess)
+      return HGC_CUDA_ERROR;
+  }
+  hgc::DwBlock dw{};
+  dw.x = static_cast<const __half*>(x);
+  dw.w9 = reinterpret_cast<const __half*>(ws + d->ws_dw_off);
+  dw.bias = static_cast<const __half*>(bias_dw);
+  dw.h = d->dw_h; dw.w = d->dw_w; dw.c = d->geom.c; dw.stride = d->dw_stride; dw.relu = relu_dw ? 1 : 0;
+  const cudaError_t err = hgc::launch_igemm(d->geom, d->igemm, ws, static_cast<const __half*>(x),
+                                            static_cast<const __half*>(bias_pw), static_cast<__half*>(y), relu_pw, st, &dw);
+  if (err == cudaErrorInvalidConfiguration || err == cudaErrorInvalidValue) return HGC_UNSUPPORTED;
   return err == cudaSuccess ? HGC_OK : HGC_CUDA_ERROR;
 }
 

@@ -21,6 +21,7 @@ struct ConvGeom {
   int32_t no_split;        // 1: never let several CTAs share the reduction of a tile (no scratch for it)
   int32_t no_pair;         // 1: never pair CTAs on 256-channel tiles
   int32_t no_fuse;         // 1: the layout pass stays a kernel of its own
+  int32_t dw_stride;       // > 0: the pointwise layer of a depthwise + pointwise block; the depthwise layer's stride
 };
 
 // First bytes of the tensor-core path's workspace: the device status word (int at byte 0) and,
@@ -175,6 +176,9 @@ struct IgemmPlan {
   // layout pass fused into the tensor-core kernel (see IgemmArgs::lay_*): segment counters at ws_lay_off
   int32_t fuse_layout, lay_px, lay_ch, lay_units_p, lay_units_c, lay_seg_units, lay_segs;
   size_t ws_lay_off;
+  // depthwise + pointwise block: the depthwise layer's input tile in shared memory
+  int32_t dw_in_h, dw_in_w;
+  uint32_t dw_in_bytes, dw_in_alloc;
   int32_t pair, ncols_sub, pair_fit;
   double est_clk;  // the cost model's estimate for the launch, in SM clocks
   size_t ws_status_off, ws_w_off, ws_x_off, ws_part_off, ws_sk_off, ws_total;
@@ -196,7 +200,17 @@ int sm_count();
 
 bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out);
 bool igemm_encode_maps(const ConvGeom& g, IgemmPlan* p, void* ws);
+// The 3x3 depthwise layer in front of a pointwise layer when both run as one kernel: the
+// tensor-core kernel computes its activation tiles from x (channels-last) instead of fetching them.
+struct DwBlock {
+  const __half* x;     // [N][h][w][c]
+  const __half* w9;    // depthwise weights as [9 taps][c]
+  const __half* bias;  // [c] or nullptr
+  int32_t h, w, c, stride, relu;
+};
 cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half* x, const __half* bias, __half* y,
-                         int relu, cudaStream_t stream);
+                         int relu, cudaStream_t stream, const DwBlock* dw = nullptr);
+// w[c][3][3] -> w9[9][c]
+cudaError_t launch_depthwise_weights_to_taps(const __half* w, __half* w9, int32_t c, cudaStream_t stream);
 
 }  // namespace hgc

@@ -927,6 +927,19 @@ struct IgemmArgs {
   int32_t lay_hw, lay_w;                    // plane size and row width in pixels
   int32_t lay_units_p, lay_units_c;         // units per image along the pixels / along the channels
   int32_t lay_seg_units, lay_segs;          // pixel units per segment, segments per image
+  // Depthwise + pointwise block in one kernel (its own instantiations): the layer the kernel sees
+  // is the 1x1 convolution; its activation tiles are not fetched but COMPUTED: eight extra warps
+  // apply the 3x3 depthwise layer (stride dw_stride, pad 1, + bias, optional ReLU, one rounding to
+  // binary16) to the channels-last input dw_x[N][dw_h][dw_w][dw_c] and write the results straight
+  // into the ring stages in the swizzled K-major layout the MMA reads.
+  const uint16_t* dw_x;
+  const uint16_t* dw_w9;   // depthwise weights re-laid-out as [9 taps][dw_c]
+  const uint16_t* dw_b;    // depthwise bias [dw_c] or nullptr
+  int32_t dw_h, dw_wd, dw_c, dw_stride, dw_relu;
+  // its input tiles ([tn][dw_in_h][dw_in_w][KB], fetched by TMA with the zero padding as
+  // out-of-bounds fill) alternate between two buffers behind the epilogue's staging tiles
+  int32_t dw_in_h, dw_in_w;
+  uint32_t dw_in_bytes, dw_in_alloc;
   int32_t dbg_drop;     // test hook: stage of the first CTA whose copies are left out (-1: none)
   int32_t ts;           // ring stages per tile: cblocks * R * (S / taps)
   // CTA pairs (clusters of two, tcgen05 cta_group::2): a tile is 256 output channels x two pixel
@@ -1130,10 +1143,51 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 // Persistent kernel: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...; the two TMEM
 // accumulators alternate so that the epilogue of one tile overlaps the MMAs of the next.
 // EPI: 0 = TMA-store epilogue, 1 = copy epilogue (NCHW, any shape), 2 = channels-last output
-constexpr int kLayoutWarps = 8;  // extra warps of the instantiations with the fused layout pass
+// Depthwise + pointwise blocks: two horizontally adjacent outputs of the 3x3 depthwise layer
+// (stride SD) for 8 channels, from an input tile in shared memory: 3 rows x (SD + 3) columns of
+// 16 bytes, `row_bytes` between rows and `px_bytes` between columns; fp32 accumulation.
+template <int SD>
+__device__ __forceinline__ void dw_pair(uint32_t src0, uint32_t row_bytes, uint32_t px_bytes, const uint32_t (&wv)[9][4],
+                                        float (&acc)[2][8]) {
+#pragma unroll
+  for (int r = 0; r < 3; ++r) {
+#pragma unroll
+    for (int col = 0; col < SD + 3; ++col) {
+      uint32_t u[4];
+      asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                   : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3])
+                   : "r"(src0 + (uint32_t)r * row_bytes + (uint32_t)col * px_bytes));
+      uint16_t xl[4], xh[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) asm("mov.b32 {%0, %1}, %2;" : "=h"(xl[j]), "=h"(xh[j]) : "r"(u[j]));
+      if (col < 3) {  // tap (r, col) of the first output
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          uint16_t wl, wh;
+          asm("mov.b32 {%0, %1}, %2;" : "=h"(wl), "=h"(wh) : "r"(wv[r * 3 + col][j]));
+          asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(acc[0][2 * j]) : "h"(xl[j]), "h"(wl));
+          asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(acc[0][2 * j + 1]) : "h"(xh[j]), "h"(wh));
+        }
+      }
+      if (col >= SD) {  // tap (r, col - SD) of the second output
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          uint16_t wl, wh;
+          asm("mov.b32 {%0, %1}, %2;" : "=h"(wl), "=h"(wh) : "r"(wv[r * 3 + col - SD][j]));
+          asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(acc[1][2 * j]) : "h"(xl[j]), "h"(wl));
+          asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(acc[1][2 * j + 1]) : "h"(xh[j]), "h"(wh));
+        }
+      }
+    }
+  }
+}
 
-template <int KB, bool HALO, int EW, int EPI, bool SPLIT, bool PAIR = false, bool SHARED = false, bool FUSEL = false>
-__global__ void __launch_bounds__(64 + 32 * EW + (FUSEL ? 32 * kLayoutWarps : 0), 1)
+constexpr int kLayoutWarps = 8;  // extra warps of the instantiations with the fused layout pass
+constexpr int kDwWarps = 8;      // extra warps of the depthwise + pointwise instantiations
+
+template <int KB, bool HALO, int EW, int EPI, bool SPLIT, bool PAIR = false, bool SHARED = false, bool FUSEL = false,
+          bool DWPW = false>
+__global__ void __launch_bounds__(64 + 32 * EW + (FUSEL ? 32 * kLayoutWarps : 0) + (DWPW ? 32 * kDwWarps : 0), 1)
 igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
              const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmYr,
              const IgemmArgs a, const __half* __restrict__ bias, __half* __restrict__ y, float* __restrict__ partials,
@@ -1146,6 +1200,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   __shared__ volatile int sk_ready;
   __shared__ __align__(8) uint64_t sk_bar;    // completion of the bulk copies of a hand-over
   __shared__ __align__(8) uint64_t meet_bar;  // meeting point of the epilogue warps (hand-overs)
+  __shared__ __align__(8) uint64_t in_full[2], in_empty[2];  // depthwise input tiles (depthwise + pointwise blocks)
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -1158,12 +1213,16 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < a.stages; ++s) {
-      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&full_bar[s]), DWPW ? 1 + kDwWarps : 1);  // (the weight copy + one arrival per depthwise warp)
       mbar_init(smem_u32(&empty_bar[s]), 1);
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(smem_u32(&acc_full[s]), 1);
       mbar_init(smem_u32(&acc_empty[s]), PAIR ? 2 * EW : EW);  // one arrival per epilogue warp (of both CTAs)
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&in_full[b]), 1);
+      mbar_init(smem_u32(&in_empty[b]), kDwWarps);
     }
     mbar_init(smem_u32(&sk_bar), 1);
     mbar_init(smem_u32(&meet_bar), EW);
@@ -1246,6 +1305,24 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         const bool drop = a.dbg_drop >= 0 && blockIdx.x == 0 && issued == (uint32_t)a.dbg_drop;
         if (drop) {
           if (lane == 0) mbar_expect_tx(smem_u32(&full_bar[ring.idx]), (PAIR ? 2u : 1u) * (a.b_bytes + (uint32_t)a.taps * a.a_bytes));
+        } else if constexpr (DWPW) {
+          // the activation tile of the stage is computed by the depthwise warps from an input tile
+          // (with its one-pixel border) that is fetched here, beside the pointwise weights
+          const uint32_t fb = smem_u32(&full_bar[ring.idx]);
+          if (lane == 0) {
+            mbar_expect_tx(fb, (uint32_t)a.taps * a.a_bytes);
+            tma_load_4d(sbase + a.b_alloc, &tmA, fb, cb * KB, m0, tap0, grp);
+          }
+          const uint32_t ib = issued & 1u;
+          if (!mbar_wait(smem_u32(&in_empty[ib]), ((issued >> 1) & 1u) ^ 1u, &abort_flag, 64)) {
+            ok = false;
+            break;
+          }
+          if (lane == 0) {
+            const uint32_t in_base = ring_base + (uint32_t)a.stages * a.stage_bytes + (uint32_t)(EW * a.nbuf) * kWarpStageBytes;
+            mbar_expect_tx(smem_u32(&in_full[ib]), a.dw_in_bytes);
+            tma_load_5d(in_base + ib * a.dw_in_alloc, &tmB, smem_u32(&in_full[ib]), cb * KB, 0, -1, p0 * a.dw_stride - 1, n0);
+          }
         } else if constexpr (PAIR) {
           // both CTAs' copies are counted on the first CTA's barrier, which expects the bytes of both
           const uint32_t fb = cluster_addr(smem_u32(&full_bar[ring.idx]), 0);
@@ -1362,6 +1439,95 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           else umma_commit(smem_u32(&acc_full[buf]));
         }
         __syncwarp();
+      }
+    }
+  } else if (DWPW && warp >= 2 + EW) {
+    // ---------------- depthwise warps: compute the activation tiles of the 1x1 layer ----------------
+    // A stage holds [pixel of the tile][KB channels], 16-byte chunks of 8 channels swizzled by the
+    // pixel row as the copy engine would have written them.  The input tile of the stage lies in
+    // shared memory as [image][row][column][KB] with a zero border.  Thread dt owns chunk
+    // dt % (KB/8) of every (256 / (KB/8))-th pair of horizontally adjacent output pixels: the pair
+    // shares its input columns (3 rows x 4 or 5 columns of 16 bytes for two outputs), and the
+    // threads of a warp read consecutive chunks: no bank conflicts.
+    constexpr int CPR = KB / 8;                     // chunks per pixel
+    constexpr int PASS = kDwWarps * 32 / CPR;       // pairs per pass of the 256 threads
+    const int dt = (warp - 2 - EW) * 32 + lane;
+    const int chunk = dt % CPR;
+    const int slot = dt / CPR;
+    Ring ring;
+    uint32_t produced = 0;
+    bool ok = true;
+    const uint32_t depth = (uint32_t)a.stages;
+    const int pairs_per_row = (a.Q + 1) >> 1;
+    const int pairs_total = a.tn * a.th * pairs_per_row;
+    const int sd = a.dw_stride;
+    const uint32_t in_base = ring_base + (uint32_t)a.stages * a.stage_bytes + (uint32_t)(EW * a.nbuf) * kWarpStageBytes;
+    typename WorkIterOf<SPLIT, SHARED>::type it;
+    for (it.init(a); it.valid(a) && ok; it.next(a)) {
+      for (int cb = 0; cb < a.cblocks && ok; ++cb, ++produced) {
+        const int c0 = cb * KB + chunk * 8;
+        const bool cvalid = c0 < a.dw_c;            // (dw_c is a multiple of 8)
+        // this thread's 8 channels: the nine taps' weights (packed pairs) and the bias
+        uint32_t wv[9][4];
+        float bv[8];
+#pragma unroll
+        for (int t = 0; t < 9; ++t) {
+          const uint4 q = cvalid ? __ldg(reinterpret_cast<const uint4*>(a.dw_w9 + (int64_t)t * a.dw_c + c0)) : make_uint4(0, 0, 0, 0);
+          wv[t][0] = q.x; wv[t][1] = q.y; wv[t][2] = q.z; wv[t][3] = q.w;
+        }
+        {
+          const uint4 q = (cvalid && a.dw_b != nullptr) ? __ldg(reinterpret_cast<const uint4*>(a.dw_b + c0)) : make_uint4(0, 0, 0, 0);
+          const uint32_t u[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            bv[2 * j] = __half2float(__ushort_as_half((uint16_t)(u[j] & 0xffffu)));
+            bv[2 * j + 1] = __half2float(__ushort_as_half((uint16_t)(u[j] >> 16)));
+          }
+        }
+        const uint32_t ib = produced & 1u;
+        if (!mbar_wait(smem_u32(&in_full[ib]), (produced >> 1) & 1u, &abort_flag, 32) ||
+            !mbar_wait(smem_u32(&empty_bar[ring.idx]), ring.phase ^ 1u, &abort_flag, 32)) {
+          ok = false;
+          break;
+        }
+        const uint32_t sbase = ring_base + ring.idx * a.stage_bytes;
+        const uint32_t tile_in = in_base + ib * a.dw_in_alloc + (uint32_t)chunk * 16u;
+        for (int pr = slot; pr < pairs_total; pr += PASS) {
+          const int rowi = pr / pairs_per_row;               // (image, output row) of the tile
+          const int wc = (pr - rowi * pairs_per_row) * 2;    // first output column of the pair
+          const int img = rowi / a.th, hr = rowi - img * a.th;
+          float acc[2][8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) acc[0][j] = acc[1][j] = bv[j];
+          const uint32_t src0 = tile_in + (uint32_t)(((img * a.dw_in_h + hr * sd) * a.dw_in_w + wc * sd) * (KB * 2));
+          if (sd == 1) dw_pair<1>(src0, (uint32_t)(a.dw_in_w * KB * 2), (uint32_t)(KB * 2), wv, acc);
+          else dw_pair<2>(src0, (uint32_t)(a.dw_in_w * KB * 2), (uint32_t)(KB * 2), wv, acc);
+          const int row = rowi * a.Q + wc;                   // row of the stage = accumulator column
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            if (wc + e < a.Q) {
+              uint32_t o[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                o[j] = a.dw_relu ? pack_f16x2<true>(acc[e][2 * j], acc[e][2 * j + 1]) : pack_f16x2<false>(acc[e][2 * j], acc[e][2 * j + 1]);
+              // row of KB*2 bytes; the swizzle of the copy engine XORs the 16-byte chunk index with
+              // address bits 7..9 (128-byte rows: the row index; 64-byte rows: the row index / 2)
+              const uint32_t rr = (uint32_t)(row + e);
+              const uint32_t sw = KB == 64 ? (rr & 7u) : ((rr >> 1) & 3u);
+              const uint32_t dst = sbase + rr * (uint32_t)(KB * 2) + (((uint32_t)chunk ^ sw) << 4);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3])
+                           : "memory");
+            }
+          }
+        }
+        // the tensor core reads the stage through the async proxy
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(smem_u32(&full_bar[ring.idx]));
+          mbar_arrive(smem_u32(&in_empty[ib]));   // (this warp has read its part of the input tile)
+        }
+        ring.advance(depth);
       }
     }
   } else if (FUSEL && warp >= 2 + EW) {
@@ -1985,6 +2151,12 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
       // several images per tile: image boundaries need not fall on multiples of 8 columns, and an
       // 8-column accumulator read that starts in the tile must end inside the 256-column buffer
       if (cols > (tn > 1 ? 248 : 256) || tn > 256) break;
+      if (g.dw_stride > 0) {
+        // depthwise + pointwise block: the depthwise layer's input tile (one-pixel border) of a
+        // 64- / 32-channel block, twice, must fit beside the ring: at most 48 KB each
+        const int64_t in_h = (int64_t)(th - 1) * g.dw_stride + 3, in_w = (int64_t)(g.q - 1) * g.dw_stride + 3;
+        if (in_h > 256 || in_w > 256 || tn * in_h * in_w * p.kb * 2 > 48 * 1024) break;
+      }
       const int64_t tiles = (int64_t)((g.n + tn - 1) / tn) * ((g.p + th - 1) / th) * mg;
       for (int ks = 0; ks <= 3; ++ks) {
         // a slice keeps at least two channel blocks and a main loop of 24 MMAs; only layers whose
@@ -2138,7 +2310,7 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
   p.sk_split = best_shared;
   p.grid = best_grid;
   p.sk_cols32 = (p.ncols + 31) / 32;
-  if (p.pair || p.sk_split) p.epi_warps = kEpilogueWarps;
+  if (p.pair || p.sk_split || g.dw_stride > 0) p.epi_warps = kEpilogueWarps;
   // split reduction (chosen with the tile shape above): fp32 partials, copy-style epilogue
   p.ks_log2 = best_ks;
   if (p.ks_log2 > 0) {
@@ -2148,7 +2320,17 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
   const size_t stage_buf_bytes = (size_t)p.epi_warps * kWarpStageBytes;
   // rings: B two or three deep, A with what is left (each A stage feeds kb/16 MMAs).  227 KB per
   // CTA minus alignment slack, static barriers and the two epilogue staging buffers.
-  const size_t budget_all = 232448u - 1024u - 512u;
+  size_t budget_all = 232448u - 1024u - 512u;
+  p.dw_in_h = p.dw_in_w = 0;
+  p.dw_in_bytes = p.dw_in_alloc = 0;
+  if (g.dw_stride > 0) {
+    p.dw_in_h = (p.th - 1) * g.dw_stride + 3;
+    p.dw_in_w = (g.q - 1) * g.dw_stride + 3;
+    p.dw_in_bytes = (uint32_t)((size_t)p.tn * p.dw_in_h * p.dw_in_w * p.kb * 2);
+    // (a pair of outputs at the end of a row reads up to two pixels past the tile)
+    p.dw_in_alloc = (uint32_t)round_up_sz((size_t)p.dw_in_bytes + 2u * p.kb * 2u, 1024);
+    budget_all -= 2u * p.dw_in_alloc;
+  }
   const size_t budget = budget_all - stage_buf_bytes;
   // ring of stages: one activation tile + `taps` weight tiles each, at least two deep; if the
   // S taps of a kernel row do not fit twice, fall back to one tap (and its own tile) per stage
@@ -2191,7 +2373,7 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
   }
   // a second staging tile per epilogue warp (its store overlaps the next unit) if memory is left
   p.nbuf = ((size_t)p.stages * p.stage_bytes + 2u * stage_buf_bytes <= budget_all) ? 2 : 1;
-  p.smem_bytes = (size_t)p.stages * p.stage_bytes + (size_t)p.nbuf * stage_buf_bytes + 1024;
+  p.smem_bytes = (size_t)p.stages * p.stage_bytes + (size_t)p.nbuf * stage_buf_bytes + 2u * p.dw_in_alloc + 1024;
   // more than half of an SM's shared memory: at most one CTA per SM, so that the kernel can take
   // all 512 TMEM columns without ever waiting for another CTA to free them
   if (p.smem_bytes < 120u * 1024u) p.smem_bytes = 120u * 1024u;
@@ -2268,6 +2450,22 @@ bool encode_nhwc_map(const ConvGeom& g, IgemmPlan* p, void* base) {
   cuuint32_t es[5] = {1, 1, (cuuint32_t)g.stride_w, (cuuint32_t)g.stride_h, 1};
   return enc(&p->tmB, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
              sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Depthwise + pointwise block: the 5-D map (channel, -, W, H, N) over the block's channels-last
+// input; a box is the input tile of one pixel tile and channel block with its one-pixel border
+// (zero padding = out-of-bounds fill), dense in shared memory.
+bool encode_dw_input_map(const DwBlock& dw, int n, IgemmPlan* p) {
+  PFN_cuTensorMapEncodeTiled_v12000 enc = encode_fn();
+  if (enc == nullptr) return false;
+  const cuuint64_t pix = (cuuint64_t)dw.c * 2;
+  cuuint64_t dims[5] = {(cuuint64_t)dw.c, 1, (cuuint64_t)dw.w, (cuuint64_t)dw.h, (cuuint64_t)n};
+  cuuint64_t strides[4] = {pix, pix, pix * dw.w, pix * dw.w * dw.h};
+  cuuint32_t box[5] = {(cuuint32_t)p->kb, 1, (cuuint32_t)p->dw_in_w, (cuuint32_t)p->dw_in_h, (cuuint32_t)p->tn};
+  cuuint32_t es[5] = {1, 1, 1, 1, 1};
+  return enc(&p->tmB, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, const_cast<__half*>(dw.x), dims, strides, box, es,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // Encodes the two tensor maps over the workspace tensors.  Returns false on failure.
@@ -2398,10 +2596,16 @@ bool igemm_encode_y_maps(const ConvGeom& g, IgemmPlan* p, void* y) {
 }
 
 cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half* x, const __half* bias, __half* y,
-                         int relu, cudaStream_t stream) {
+                         int relu, cudaStream_t stream, const DwBlock* dw) {
   if (!p.maps_ready) return cudaErrorInvalidValue;
+  if (dw != nullptr && (!p.x_nhwc || p.pair || p.sk_split || p.ks_log2 > 0 || p.fuse_layout || p.kb < 32))
+    return cudaErrorInvalidValue;
   if (p.nchw && p.x_mapped != x && !igemm_encode_x_map(g, &p, x)) return cudaErrorInvalidValue;
-  if (p.x_nhwc && p.x_mapped != x) {
+  if (dw != nullptr && p.x_mapped != x) {  // the block's input tiles come from x (channels-last) with their border
+    if (p.dw_in_bytes == 0 || !encode_dw_input_map(*dw, g.n, &p)) return cudaErrorInvalidValue;
+    p.x_mapped = x;
+  }
+  if (dw == nullptr && p.x_nhwc && p.x_mapped != x) {
     if (!encode_nhwc_map(g, &p, const_cast<__half*>(x))) return cudaErrorInvalidValue;
     p.x_mapped = x;
   }
@@ -2454,6 +2658,13 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
   a.y_full_w = p.y_full_w;
   a.y_rpu = p.y_rpu > 0 ? p.y_rpu : 1;
   a.dbg_drop = debug_drop_copies();
+  if (dw != nullptr) {
+    a.dw_x = reinterpret_cast<const uint16_t*>(dw->x);
+    a.dw_w9 = reinterpret_cast<const uint16_t*>(dw->w9);
+    a.dw_b = reinterpret_cast<const uint16_t*>(dw->bias);
+    a.dw_h = dw->h; a.dw_wd = dw->w; a.dw_c = dw->c; a.dw_stride = dw->stride; a.dw_relu = dw->relu;
+    a.dw_in_h = p.dw_in_h; a.dw_in_w = p.dw_in_w; a.dw_in_bytes = p.dw_in_bytes; a.dw_in_alloc = p.dw_in_alloc;
+  }
   a.lay_x = reinterpret_cast<const uint16_t*>(x);
   a.lay_xp = reinterpret_cast<uint16_t*>(static_cast<char*>(ws) + p.ws_x_off);
   a.lay_flags = reinterpret_cast<int*>(static_cast<char*>(ws) + p.ws_lay_off);
@@ -2486,6 +2697,22 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
     if (err == cudaSuccess)                                                                                \
       err = launch_kernel(igemm_kernel<KBV, HALOV, EWV, EPIV, SPLITV>, grid, dim3(64 + 32 * EWV),          \
                           p.smem_bytes, stream, p.tmA, p.tmB, p.tmY, p.tmYr, a, bias, y, partials, status); \
+  } while (0)
+  // depthwise + pointwise block: its own instantiations (8 epilogue + 8 depthwise warps)
+#define HGC_LAUNCH_DWPW_EPI(KBV, EPIV)                                                                     \
+  do {                                                                                                     \
+    err = cudaFuncSetAttribute(igemm_kernel<KBV, true, 8, EPIV, false, false, false, false, true>,         \
+                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);            \
+    if (err == cudaSuccess)                                                                                \
+      err = launch_kernel(igemm_kernel<KBV, true, 8, EPIV, false, false, false, false, true>, grid,        \
+                          dim3(64 + 32 * 8 + 32 * kDwWarps), p.smem_bytes, stream, p.tmA, p.tmB, p.tmY,    \
+                          p.tmYr, a, bias, y, partials, status);                                           \
+  } while (0)
+#define HGC_LAUNCH_DWPW(KBV)                                   \
+  do {                                                         \
+    if (p.y_nhwc) HGC_LAUNCH_DWPW_EPI(KBV, 2);                 \
+    else if (!p.tma_store) HGC_LAUNCH_DWPW_EPI(KBV, 1);        \
+    else HGC_LAUNCH_DWPW_EPI(KBV, 0);                          \
   } while (0)
   // fused layout pass: its own instantiations (8 epilogue + 4 layout warps), launched cooperatively
   // (a tile waits for segments that other CTAs' layout warps convert)
@@ -2546,7 +2773,9 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
     else if (!p.tma_store) HGC_LAUNCH_PAIR_EPI(KBV, HALOV, 1);     \
     else HGC_LAUNCH_PAIR_EPI(KBV, HALOV, 0);                       \
   } while (0)
-  if (p.pair) {
+  if (dw != nullptr) {
+    if (p.kb == 64) HGC_LAUNCH_DWPW(64); else HGC_LAUNCH_DWPW(32);
+  } else if (p.pair) {
     if (p.kb == 64) {
       if (p.halo) HGC_LAUNCH_PAIR(64, true); else HGC_LAUNCH_PAIR(64, false);
     } else if (p.kb == 32) {
@@ -2589,6 +2818,8 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
 #undef HGC_LAUNCH_SHARED
 #undef HGC_LAUNCH_FUSED_EPI
 #undef HGC_LAUNCH_FUSED
+#undef HGC_LAUNCH_DWPW_EPI
+#undef HGC_LAUNCH_DWPW
   if (err != cudaSuccess) return err;
   count_launch();
   if (p.ks_log2 > 0) {

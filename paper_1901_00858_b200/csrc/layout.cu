@@ -615,6 +615,20 @@ cudaError_t launch_igemm_weights(const ConvGeom& g, const IgemmPlan& p, const __
   return launch_weights_repack(w, wp, g.k, g.cg, g.r, g.s, g.group, p.cw, stream, p.y_perm);
 }
 
+__global__ void __launch_bounds__(256)
+depthwise_weights_to_taps_kernel(const uint16_t* __restrict__ w, uint16_t* __restrict__ w9, int c) {
+  grid_dependency_wait();
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;  // index into w9: tap * c + channel
+  if (i < 9 * c) w9[i] = w[(i % c) * 9 + i / c];
+}
+
+cudaError_t launch_depthwise_weights_to_taps(const __half* w, __half* w9, int32_t c, cudaStream_t stream) {
+  launch_kernel(depthwise_weights_to_taps_kernel, dim3((unsigned)((9 * c + 255) / 256)), dim3(256), 0, stream,
+                reinterpret_cast<const uint16_t*>(w), reinterpret_cast<uint16_t*>(w9), (int)c);
+  count_launch();
+  return cudaGetLastError();
+}
+
 cudaError_t launch_igemm_input(const ConvGeom& g, const IgemmPlan& p, const __half* x, __half* xp,
                                cudaStream_t stream) {
   if (p.nchw || p.x_nhwc) return cudaSuccess;  // the kernel reads x itself
