@@ -383,6 +383,61 @@ def summarize(hgc, state, batch, layer_t, peaks, regime):
     return by_path, per_path, rows, total_ms, t_roof
 
 
+def measure_block_chain(hgc, torch, steps, side, rank):
+    """MobileNet-v1 at batch 32 as a channels-last chain: the stem, then the 13 depthwise +
+    pointwise blocks each as ONE kernel (hgc_dwpw_forward).  Same shapes, tensors per block."""
+    wl = workloads.by_name("mobilenet_v1_n32")
+    layers = wl.expanded()
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(777 + rank)
+    n = wl.batch
+    stem = layers[0]
+    calls = []
+    d0 = hgc.ConvDesc(*_geo(n, stem), hgc.HGC_FLAG_Y_NHWC)
+    d0.ensure_workspace()
+    x0 = torch.empty((n, stem.c, stem.h, stem.h), dtype=torch.float16, device="cuda").uniform_(0, 1, generator=gen)
+    w0 = torch.empty((stem.k, stem.c, stem.r, stem.r), dtype=torch.float16, device="cuda").normal_(0, 0.27, generator=gen)
+    b0 = torch.zeros(stem.k, dtype=torch.float16, device="cuda")
+    y0 = torch.empty((n, stem.out, stem.out, stem.k), dtype=torch.float16, device="cuda")
+    d0.set_weights(w0)
+    calls.append(lambda st: hgc.conv_forward(d0, x0, w0, b0, y0, True, st))
+    keep = [d0]
+    flops = layer_flops(n, stem)
+    for i in range(1, len(layers), 2):
+        dw, pw = layers[i], layers[i + 1]
+        d = hgc.DwPwDesc(n, dw.c, dw.h, dw.h, pw.k, dw.stride, hgc.HGC_FLAG_Y_NHWC)
+        d.ensure_workspace()
+        x = torch.empty((n, dw.h, dw.h, dw.c), dtype=torch.float16, device="cuda").uniform_(0, 1, generator=gen)
+        w_dw = torch.empty((dw.c, 1, 3, 3), dtype=torch.float16, device="cuda").normal_(0, 0.47, generator=gen)
+        w_pw = torch.empty((pw.k, dw.c, 1, 1), dtype=torch.float16, device="cuda").normal_(0, float(np.sqrt(2.0 / dw.c)), generator=gen)
+        b_dw = torch.zeros(dw.c, dtype=torch.float16, device="cuda")
+        b_pw = torch.zeros(pw.k, dtype=torch.float16, device="cuda")
+        y = torch.empty((n, pw.out, pw.out, pw.k), dtype=torch.float16, device="cuda")
+        d.set_weights(w_dw, w_pw)
+        calls.append(lambda st, d=d, x=x, w_dw=w_dw, b_dw=b_dw, w_pw=w_pw, b_pw=b_pw, y=y:
+                     hgc.dwpw_forward(d, x, w_dw, b_dw, w_pw, b_pw, y, True, True, st))
+        keep.append(d)
+        flops += layer_flops(n, dw) + layer_flops(n, pw)
+    for c in calls:
+        c(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    c0 = hgc.kernel_launch_count()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            for c in calls:
+                c(side)
+    per_step = hgc.kernel_launch_count() - c0
+    torch.cuda.synchronize()
+    ms = time_replays(torch, g, side, steps)
+    ms = time_replays(torch, g, side, steps)
+    for d in keep:
+        d.close()
+    return {"ms_per_step": ms, "steps": steps, "tflops": flops / (ms * 1e-3) / 1e12, "images_per_s": n / (ms * 1e-3),
+            "launches_per_step": per_step, "launch": "cuda_graph",
+            "note": "channels-last chain: stem + 13 depthwise+pointwise blocks, one kernel per block (hgc_dwpw_forward)"}
+
+
 def measure_extra(hgc, torch, name, steps, peaks, side, rank):
     """One more workload for the JSON line's `workloads` object: graph replay of the step, and
     per-path figures from per-layer graph times."""
@@ -413,6 +468,21 @@ def measure_extra(hgc, torch, name, steps, peaks, side, rank):
                                           "the graph-replayed step time"}
         out["per_path"] = per_path
         out["sum_of_layer_ms"] = total_ms
+        try:   # the same step with channels-last activations
+            gen2 = torch.Generator(device="cuda")
+            gen2.manual_seed(99 + rank)
+            nstate, n_in, n_out = build_state(hgc, torch, wl.expanded(), wl.batch, gen2, True)
+            for (d, x, w, b, y, l) in nstate:
+                hgc.conv_forward(d, x, w, b, y, l.relu, side)
+            torch.cuda.synchronize()
+            gl, _ = capture_step(hgc, torch, nstate, side)
+            out["channels_last"] = {"ms_per_step": time_replays(torch, gl, side, steps), "layers_with_channels_last_input": n_in,
+                                    "layers_with_channels_last_output": n_out}
+            for (d, *_r) in nstate:
+                d.close()
+            del nstate, gl
+        except Exception as exc:
+            out["channels_last"] = {"error": repr(exc)}
     for (d, *_rest) in state:
         d.close()
     del state, graph
@@ -581,6 +651,10 @@ def run_ours(args, wl):
                 extras[name] = measure_extra(hgc, torch, name, 50, peaks, side, rank)
             except Exception as exc:
                 extras[name] = {"error": repr(exc)}
+        try:
+            extras["mobilenet_v1_n32_block_kernels"] = measure_block_chain(hgc, torch, 50, side, rank)
+        except Exception as exc:
+            extras["mobilenet_v1_n32_block_kernels"] = {"error": repr(exc)}
 
     # ---- max over ranks ---------------------------------------------------------------------
     if world > 1:

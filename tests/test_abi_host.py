@@ -207,3 +207,33 @@ def test_scheduling_flags_change_the_plan_not_the_layer():
         assert d.output_dims() == base.output_dims() and d.path() == base.path()
     # a layer with 128 output channels has nothing to pair
     assert hgc.ConvDesc(16, 128, 112, 112, 128, 3, 3, 1, 1, flags=hgc.HGC_FLAG_CTA_PAIRS).plan_info()["pair"] == 0
+
+
+def test_block_descriptor_validation():
+    """hgc_dwpw_desc_create: argument checks and planning run on the host."""
+    L = hgc.lib()
+    h = ctypes.c_void_p()
+    ok = hgc.hgc_dwpw_params(32, 512, 14, 14, 512, 1, hgc.HGC_FLAG_Y_NHWC)
+    assert L.hgc_dwpw_desc_create(ctypes.byref(h), ctypes.byref(ok)) == hgc.HGC_OK
+    n, k, p, q = (ctypes.c_int32() for _ in range(4))
+    assert L.hgc_conv_output_dims(h, ctypes.byref(n), ctypes.byref(k), ctypes.byref(p), ctypes.byref(q)) == hgc.HGC_OK
+    assert (n.value, k.value, p.value, q.value) == (32, 512, 14, 14)
+    ptr = ctypes.c_void_p(0x10000)
+    # a block descriptor is not a layer descriptor, and needs its workspace
+    assert L.hgc_conv_forward(h, ptr, ptr, None, ptr, 0, None) == hgc.HGC_INVALID_ARG
+    assert L.hgc_conv_set_weights(h, ptr, None) == hgc.HGC_INVALID_ARG
+    assert L.hgc_dwpw_forward(h, ptr, ptr, None, ptr, None, ptr, 1, 1, None) == hgc.HGC_NO_WORKSPACE
+    assert L.hgc_dwpw_forward(h, None, ptr, None, ptr, None, ptr, 1, 1, None) == hgc.HGC_INVALID_ARG
+    assert L.hgc_conv_desc_destroy(h) == hgc.HGC_OK
+    s2 = hgc.hgc_dwpw_params(2, 64, 15, 17, 128, 2, 0)           # stride 2 on an odd plane: 8 x 9 outputs
+    assert L.hgc_dwpw_desc_create(ctypes.byref(h), ctypes.byref(s2)) == hgc.HGC_OK
+    assert L.hgc_conv_output_dims(h, ctypes.byref(n), ctypes.byref(k), ctypes.byref(p), ctypes.byref(q)) == hgc.HGC_OK
+    assert (p.value, q.value) == (8, 9)
+    assert L.hgc_conv_desc_destroy(h) == hgc.HGC_OK
+    for bad, want in [(hgc.hgc_dwpw_params(1, 32, 8, 8, 32, 3, 0), hgc.HGC_INVALID_ARG),      # stride 3
+                      (hgc.hgc_dwpw_params(1, 32, 8, 8, 32, 1, hgc.HGC_FLAG_X_NHWC), hgc.HGC_INVALID_ARG),  # other flags
+                      (hgc.hgc_dwpw_params(0, 32, 8, 8, 32, 1, 0), hgc.HGC_INVALID_ARG),
+                      (hgc.hgc_dwpw_params(1, 12, 8, 8, 32, 1, 0), hgc.HGC_UNSUPPORTED)]:     # 12 channels
+        assert L.hgc_dwpw_desc_create(ctypes.byref(h), ctypes.byref(bad)) == want
+    layer = hgc.ConvDesc(1, 32, 8, 8, 32, 3, 3, 1, 1)
+    assert L.hgc_dwpw_forward(layer.handle, ptr, ptr, None, ptr, None, ptr, 1, 1, None) == hgc.HGC_INVALID_ARG
