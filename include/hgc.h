@@ -77,21 +77,25 @@ typedef struct hgc_conv_params {
 #define HGC_FLAG_X_NHWC 2
 #define HGC_FLAG_Y_NHWC 4
 /*
- * Scheduling choices of the tensor-core path, off by default, for measurement and tests (the
- * result is the same layer within the tolerance; the summation order over the input channels
- * changes).  Both were built to lift what looked like the limits of the single-CTA kernel; on the
- * measured layers, which run under the board's power cap, neither made a layer faster by more
- * than a few per cent, so the planner does not choose them by itself.
- * HGC_FLAG_CTA_PAIRS: layers with more than 128 output channels per group may be launched as CTA
- * pairs (clusters of two SMs that share tiles of 256 output channels through tcgen05
- * cta_group::2: each CTA fetches its own 128 weight rows and half of the activation tile).
+ * Scheduling choices of the tensor-core path (the result is the same layer within the tolerance;
+ * the summation order over the input channels changes).
+ * HGC_FLAG_CTA_PAIRS (off unless set): layers with more than 128 output channels per group may be
+ * launched as CTA pairs (clusters of two SMs that share tiles of 256 output channels through
+ * tcgen05 cta_group::2: each CTA fetches its own 128 weight rows and half of the activation
+ * tile).  Measured on the VGG-16 layers: within a few per cent of the single-CTA kernel either
+ * way, so the planner does not choose it by itself.
  * HGC_FLAG_SHARED_TILES: the ring stages of all tiles are dealt out in equal contiguous ranges,
  * so that every CTA (or pair) gets the same amount of work; a tile that straddles a boundary is
  * reduced by several CTAs inside the one launch (fp32 hand-over through the workspace, added in
- * a fixed order: deterministic).  Such a launch is cooperative.
+ * a fixed order: deterministic).  Such a launch is cooperative.  Without the flag the planner
+ * takes this schedule only where its cost model expects a gain (long tiles, at least 2.5 per
+ * CTA, a last wave that is mostly empty: VGG-16's 256-channel layers on 56x56 planes at batch
+ * 16, 61 -> 56 us); with it, wherever the tiles do not fill whole waves.
+ * HGC_FLAG_WHOLE_TILES: never (smaller workspace; ordinary launch).  Wins over the flag above.
  */
 #define HGC_FLAG_CTA_PAIRS 8
 #define HGC_FLAG_SHARED_TILES 16
+#define HGC_FLAG_WHOLE_TILES 64
 /*
  * HGC_FLAG_FUSED_LAYOUT (off by default): layers whose input needs the NCHW->NHWC copy and whose
  * output rows are whole 16-byte vectors (3x3 layers on 224, 112, 56 wide planes ...) make that

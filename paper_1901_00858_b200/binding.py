@@ -22,6 +22,7 @@ HGC_FLAG_Y_NHWC = 4
 HGC_FLAG_CTA_PAIRS = 8
 HGC_FLAG_SHARED_TILES = 16
 HGC_FLAG_FUSED_LAYOUT = 32
+HGC_FLAG_WHOLE_TILES = 64
 PATH_NAMES = {HGC_PATH_DIRECT: "direct", HGC_PATH_DEPTHWISE: "depthwise", HGC_PATH_IGEMM: "igemm"}
 
 

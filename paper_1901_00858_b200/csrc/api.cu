@@ -140,7 +140,7 @@ int hgc_conv_desc_create(hgc_conv_desc** out, const hgc_conv_params* p) {
   g.x_nhwc = (p->flags & HGC_FLAG_X_NHWC) ? 1 : 0;
   g.y_nhwc = (p->flags & HGC_FLAG_Y_NHWC) ? 1 : 0;
   g.no_pair = (p->flags & HGC_FLAG_CTA_PAIRS) ? 0 : 1;
-  g.no_split = (p->flags & HGC_FLAG_SHARED_TILES) ? 0 : 1;
+  g.no_split = (p->flags & HGC_FLAG_WHOLE_TILES) ? 1 : ((p->flags & HGC_FLAG_SHARED_TILES) ? 0 : 2);  // 2: the planner's cost model decides
   g.no_fuse = (p->flags & HGC_FLAG_FUSED_LAYOUT) ? 0 : 1;
   const bool channels_last = g.x_nhwc || g.y_nhwc;
 

@@ -18,7 +18,7 @@ struct ConvGeom {
   int32_t p, q;    // output plane
   int32_t cg, kg;  // channels per group: C/group, K/group
   int32_t x_nhwc, y_nhwc;  // channels-last input / output (tensor-core path only)
-  int32_t no_split;        // 1: never let several CTAs share the reduction of a tile (no scratch for it)
+  int32_t no_split;        // 1: never let several CTAs share the reduction of a tile (no scratch for it); 0: wherever possible; 2: where the cost model expects a gain
   int32_t no_pair;         // 1: never pair CTAs on 256-channel tiles
   int32_t no_fuse;         // 1: the layout pass stays a kernel of its own
   int32_t dw_stride;       // > 0: the pointwise layer of a depthwise + pointwise block; the depthwise layer's stride

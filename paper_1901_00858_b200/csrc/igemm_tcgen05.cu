@@ -396,12 +396,14 @@ __device__ __forceinline__ bool epi_sync(uint32_t bar, uint32_t& phase, volatile
 }
 
 // A tile reduced by several CTAs (IgemmArgs::sk_split).  The accumulators travel as fp32 in the
-// order [column][128 lanes]: a warp's 32 lanes are 128 contiguous bytes per column.
-// sk_hand_over: this warp's lane quarter, column chunks `first`, `first + step`, ... -> slot.
-__device__ __noinline__ void sk_hand_over(uint32_t t_addr, int quarter, int first, int step, int cols32, float* slot) {
+// order [column][128 lanes]: a warp's 32 lanes are 128 contiguous bytes per column.  (Moving them
+// with the bulk copy engine through the warp's 4 KB staging tiles was measured slower: two copies
+// in flight per warp do not hide their latency.)
+// sk_hand_over: this warp's lane quarter of the accumulator -> slot.
+__device__ __noinline__ void sk_hand_over(uint32_t t_addr, int quarter, int cols32, float* slot) {
   const int lane = threadIdx.x & 31;
   float* dst = slot + quarter * 32 + lane;
-  for (int c = first; c < cols32; c += step) {
+  for (int c = 0; c < cols32; ++c) {
     uint32_t v[32];
     tmem_ld32(t_addr + (uint32_t)(c * 32), v);
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -410,50 +412,32 @@ __device__ __noinline__ void sk_hand_over(uint32_t t_addr, int quarter, int firs
   }
 }
 
-// sk_take_over: adds the slots of CTAs first_cta, first_cta + cta_step, ... (count of them, in that
-// order: the sum does not depend on timing) to this CTA's accumulator, in place.  The tile is the
-// CTA's last piece of work, so the operand ring is idle: each slot is fetched into it with bulk
-// copies (pieces of `piece32` 32-column chunks, as many as the ring holds) and added from there.
-// Called by all epilogue warps, which meet on `meet_bar`; `leader` issues the copies.  False after a
-// wait that ran out.
-__device__ __noinline__ bool sk_take_over(uint32_t t_addr, int quarter, int first, int step, int cols32, bool live,
-                                          const float* slots, size_t slot_elems, int first_cta, int cta_step, int count,
-                                          uint32_t ring, int piece32, uint32_t copy_bar, uint32_t& copy_phase,
-                                          uint32_t meet_bar, uint32_t& meet_phase, bool leader, volatile int* abort_flag) {
+// sk_preload: the sum of the slots first_slot, first_slot + slot_step, ... (count of them, in that
+// order: the sum does not depend on timing) -> this warp's lane quarter of an accumulator that the
+// MMAs of the tile's first part then add to.  A column of a warp is 128 contiguous bytes of a
+// slot: one coalesced load per column, 32 in flight.
+__device__ __noinline__ void sk_preload(uint32_t t_addr, int quarter, int cols32, const float* slots, size_t slot_elems,
+                                        int first_slot, int slot_step, int count) {
   const int lane = threadIdx.x & 31;
-  for (int i = 0; i < count; ++i) {
-    const float* slot = slots + (size_t)(first_cta + i * cta_step) * slot_elems;
-    for (int c0 = 0; c0 < cols32; c0 += piece32) {
-      const int nc = cols32 - c0 < piece32 ? cols32 - c0 : piece32;
-      // the previous piece has been added by everybody before it is overwritten
-      if (!epi_sync(meet_bar, meet_phase, abort_flag)) return false;
-      if (leader) {
-        const uint32_t bytes = (uint32_t)nc * 32u * 128u * 4u;
-        mbar_expect_tx(copy_bar, bytes);
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(ring),
-                     "l"(slot + (size_t)c0 * 32 * 128), "r"(bytes), "r"(copy_bar)
-                     : "memory");
-      }
-      if (!mbar_wait(copy_bar, copy_phase, abort_flag, 32)) return false;
-      copy_phase ^= 1u;
-      if (live) {
-        for (int c = first; c < nc; c += step) {
-          uint32_t v[32];
-          tmem_ld32(t_addr + (uint32_t)((c0 + c) * 32), v);
-          const uint32_t src = ring + (uint32_t)(c * 32 * 128 + quarter * 32 + lane) * 4u;
-          float add[32];
+  for (int c = 0; c < cols32; ++c) {
+    const float* src = slots + (size_t)first_slot * slot_elems + (size_t)c * 32 * 128 + quarter * 32 + lane;
+    float v[32];
 #pragma unroll
-          for (int j = 0; j < 32; ++j) asm volatile("ld.shared.f32 %0, [%1];" : "=f"(add[j]) : "r"(src + (uint32_t)j * 512u));
-          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+    for (int j = 0; j < 32; ++j) v[j] = __ldcg(src + (size_t)j * 128);
+    for (int i = 1; i < count; ++i) {
+      src += (size_t)slot_step * slot_elems;
+      float w[32];
 #pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + add[j]);
-          tmem_st32(t_addr + (uint32_t)((c0 + c) * 32), v);
-        }
-      }
+      for (int j = 0; j < 32; ++j) w[j] = __ldcg(src + (size_t)j * 128);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] += w[j];
     }
+    uint32_t u[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) u[j] = __float_as_uint(v[j]);
+    tmem_st32(t_addr + (uint32_t)(c * 32), u);
   }
   asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-  return true;
 }
 
 // two fp32 -> packed fp16x2 (round to nearest even), lo = first value; optional ReLU in the convert
@@ -1197,9 +1181,10 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   __shared__ __align__(8) uint64_t acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int abort_flag;
-  __shared__ volatile int sk_ready;
-  __shared__ __align__(8) uint64_t sk_bar;    // completion of the bulk copies of a hand-over
-  __shared__ __align__(8) uint64_t meet_bar;  // meeting point of the epilogue warps (hand-overs)
+  __shared__ __align__(8) uint64_t sk_bar;    // shared tiles: the partial sums of the unit's last tile are in its accumulator
+  __shared__ __align__(8) uint64_t meet_bar;  // shared tiles: meeting point of all epilogue warps,
+  __shared__ __align__(8) uint64_t ho_bar;    //   of the warps that hand accumulators over (the first of each lane quarter),
+  __shared__ __align__(8) uint64_t pl_bar;    //   of the warps that fetch partial sums (the second of each lane quarter)
   __shared__ __align__(8) uint64_t in_full[2], in_empty[2];  // depthwise input tiles (depthwise + pointwise blocks)
 
   const int warp = threadIdx.x >> 5;
@@ -1224,8 +1209,10 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       mbar_init(smem_u32(&in_full[b]), 1);
       mbar_init(smem_u32(&in_empty[b]), kDwWarps);
     }
-    mbar_init(smem_u32(&sk_bar), 1);
+    mbar_init(smem_u32(&sk_bar), PAIR ? EW : EW / 2);  // one arrival per fetching warp (of both CTAs)
     mbar_init(smem_u32(&meet_bar), EW);
+    mbar_init(smem_u32(&ho_bar), EW / 2);
+    mbar_init(smem_u32(&pl_bar), EW / 2);
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -1409,6 +1396,18 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t d_tmem = tmem_base + buf * 256u;
       uint32_t acc = 0;
+      if constexpr (!SPLIT && SHARED) {
+        if (it.kind(a) == 2) {
+          // the first part of a tile whose later parts other units computed: the epilogue warps
+          // have put the sum of those parts into the accumulator (see there); add to it
+          if (!mbar_wait(smem_u32(&sk_bar), 0u, &abort_flag, 64)) {
+            ok = false;
+            break;
+          }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          acc = 1;
+        }
+      }
       for (int gi = 0; gi < groups_per_tile; ++gi) {
         if (!ready && !mbar_wait(smem_u32(&full_bar[ring.idx]), ring.phase, &abort_flag)) {
           ok = false;
@@ -1565,9 +1564,75 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const uint32_t row_off = (uint32_t)lane * 128u + (((uint32_t)lane & 7u) << 4);
     uint32_t unit_ctr = 0, stage_sel = 0;
     uint32_t lt = 0;
-    uint32_t sk_phase = 0, meet_phase = 0;
+    uint32_t meet_phase = 0, ho_phase = 0, pl_phase = 0;
+    // Shared tiles: when this unit's range ends inside a tile whose first stage it holds, it
+    // finishes that tile (its last item), and the following units computed the tile's later parts
+    // first of all.  The sum of their partial accumulators is put into the tile's accumulator
+    // BEFORE its MMAs start (which then add to it), while the MMAs of the items before run: by the
+    // second warp of every lane quarter, at the top of the item before the last (of the first item
+    // when there are at most two: that accumulator has not been used yet).  Handing over (the
+    // unit's first item, when its range begins inside a tile) is the first warps' work, so that a
+    // unit's hand-over never waits for its own fetch: no chain of waits through the units.
+    int fin_item = -1, fin_tile = 0;
+    if constexpr (!SPLIT && SHARED) {
+      const int u = SegIter<SHARED>::unit(a);
+      const int64_t g_beg = SegIter<SHARED>::range_start(a, u), g_end = SegIter<SHARED>::range_start(a, u + 1);
+      fin_tile = (int)(g_end / a.ts);
+      if (g_end > g_beg && g_end % a.ts != 0 && (int64_t)fin_tile * a.ts >= g_beg) fin_item = fin_tile - (int)(g_beg / a.ts);
+    }
     typename WorkIterOf<SPLIT, SHARED>::type it;
     for (it.init(a); it.valid(a); it.next(a), ++lt) {
+      if constexpr (!SPLIT && SHARED) {
+        if (fin_item >= 0 && (int)lt == (fin_item >= 2 ? fin_item - 1 : 0)) {
+          // every warp has drained the accumulator's previous tile, two items back
+          if (fin_item >= 2 && !epi_sync(smem_u32(&meet_bar), meet_phase, &abort_flag)) break;
+          if (half == 1) {
+            const int unit = SegIter<SHARED>::unit(a);
+            const size_t slot_elems = (size_t)a.sk_cols32 * 32 * 128;
+            const int64_t tile_end = (int64_t)(fin_tile + 1) * a.ts;
+            int count = 0;
+            while (unit + 1 + count < SegIter<SHARED>::units(a) && SegIter<SHARED>::range_start(a, unit + 1 + count) < tile_end) ++count;
+            const int first_slot = ((unit + 1) << a.pair) + (int)rank;
+            const int slot_step = 1 << a.pair;
+            int good = 1;
+            if (lane == 0) {
+              for (int i = 0; i < count && good; ++i) {
+                const int* f = a.sk_flags + first_slot + i * slot_step;
+                const uint64_t t0 = global_timer_ns();
+                for (uint32_t spin = 0;; ++spin) {
+                  int v;
+                  asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(f) : "memory");
+                  if (v != 0) break;
+                  if ((spin & 255u) == 255u && (abort_flag || global_timer_ns() - t0 > g_wait_limit_ns)) {
+                    abort_flag = 1;
+                    good = 0;
+                    break;
+                  }
+                  __nanosleep(128);
+                }
+              }
+            }
+            good = __shfl_sync(0xffffffffu, good, 0);
+            if (!good) break;
+            const int mgn = a.mtiles * a.group;
+            const int mg_f = fin_tile % mgn;
+            const int m0_f = (((a.group == 1 ? mg_f : mg_f % a.mtiles) * 128) << a.pair) + (PAIR ? (int)rank * 128 : 0);
+            if (m0_f + quarter * 32 < a.kg)
+              sk_preload(tmem_base + (uint32_t)(fin_item & 1) * 256u + ((uint32_t)(quarter * 32) << 16), quarter, a.sk_cols32,
+                         a.sk_part, slot_elems, first_slot, slot_step, count);
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+              if constexpr (PAIR) mbar_arrive_cluster(cluster_addr(smem_u32(&sk_bar), 0));
+              else mbar_arrive(smem_u32(&sk_bar));
+            }
+            // every part has been read by the four warps: lower the flags for the next launch
+            if (!epi_sync(smem_u32(&pl_bar), pl_phase, &abort_flag)) break;
+            if (quarter == 0)
+              for (int i = lane; i < count; i += 32) a.sk_flags[first_slot + i * slot_step] = 0;
+          }
+        }
+      }
       int grp, m0;
       it.channel_tile(a, grp, m0);
       if constexpr (PAIR) m0 += (int)rank * 128;  // this CTA's tensor memory holds its own 128 channels
@@ -1588,16 +1653,17 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         const size_t slot_elems = (size_t)a.sk_cols32 * 32 * 128;
         // slots and flags are per CTA; the parts of a tile come from the following work units
         // (the CTA of the same rank in the following pairs)
-        const int unit = SegIter<SHARED>::unit(a);
         if (kind == 1) {
           // a later part of a tile that another CTA finishes: hand the accumulators over
-          if (quarter_live) sk_hand_over(t_tile, quarter, half, kPerQuarter, a.sk_cols32, a.sk_part + (size_t)blockIdx.x * slot_elems);
-          __threadfence();
-          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-          if (!epi_sync(smem_u32(&meet_bar), meet_phase, &abort_flag)) break;
-          if (ew == 0 && lane == 0) {
+          if (half == 0) {
+            if (quarter_live) sk_hand_over(t_tile, quarter, a.sk_cols32, a.sk_part + (size_t)blockIdx.x * slot_elems);
             __threadfence();
-            asm volatile("st.release.gpu.global.b32 [%0], %1;" ::"l"(a.sk_flags + blockIdx.x), "r"(1) : "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            if (!epi_sync(smem_u32(&ho_bar), ho_phase, &abort_flag)) break;
+            if (ew == 0 && lane == 0) {
+              __threadfence();
+              asm volatile("st.release.gpu.global.b32 [%0], %1;" ::"l"(a.sk_flags + blockIdx.x), "r"(1) : "memory");
+            }
           }
           __syncwarp();
           if (lane == 0) {
@@ -1605,51 +1671,6 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             else mbar_arrive(acc_empty_bar);
           }
           continue;
-        }
-        if (kind == 2) {
-          // the first part of a tile whose later parts belong to the next units: wait for theirs
-          // (they computed them first of all), add them, then finish the tile as usual
-          const int64_t tile_end = (int64_t)(it.tile + 1) * a.ts;
-          int count = 0;
-          while (unit + 1 + count < SegIter<SHARED>::units(a) && SegIter<SHARED>::range_start(a, unit + 1 + count) < tile_end) ++count;
-          const int first_slot = ((unit + 1) << a.pair) + (int)rank;
-          const int slot_step = 1 << a.pair;
-          if (ew == 0 && lane == 0) {
-            int good = 1;
-            for (int i = 0; i < count && good; ++i) {
-              const int* f = a.sk_flags + first_slot + i * slot_step;
-              const uint64_t t0 = global_timer_ns();
-              for (uint32_t spin = 0;; ++spin) {
-                int v;
-                asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(f) : "memory");
-                if (v != 0) break;
-                if ((spin & 255u) == 255u && (abort_flag || global_timer_ns() - t0 > g_wait_limit_ns)) {
-                  abort_flag = 1;
-                  good = 0;
-                  break;
-                }
-                __nanosleep(128);
-              }
-            }
-            sk_ready = good;
-          }
-          if (!epi_sync(smem_u32(&meet_bar), meet_phase, &abort_flag)) break;
-          if (!sk_ready) break;
-          {
-            // the ring is idle: this tile is the CTA's last piece of work and its MMAs are complete
-            int piece32 = (int)(((uint32_t)a.stages * a.stage_bytes) >> 14);  // 16 KB per 32 columns
-            if (piece32 > a.sk_cols32) piece32 = a.sk_cols32;
-            if (!sk_take_over(t_tile, quarter, half, kPerQuarter, a.sk_cols32, quarter_live, a.sk_part, slot_elems,
-                              first_slot, slot_step, count, ring_base, piece32, smem_u32(&sk_bar), sk_phase,
-                              smem_u32(&meet_bar), meet_phase, ew == 0 && lane == 0, &abort_flag))
-              break;
-          }
-          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-          if (!epi_sync(smem_u32(&meet_bar), meet_phase, &abort_flag)) break;
-          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          // every part has been read: lower the flags for the next launch
-          if (ew == 0)
-            for (int i = lane; i < count; i += 32) a.sk_flags[first_slot + i * slot_step] = 0;
         }
       }
 
@@ -2147,7 +2168,10 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
   const bool can_split = p.kb == 64 && p.halo && !p.nchw && !p.y_nhwc;
   double best = 1e300;
   int best_th = 0, best_tn = 0, best_ks = 0, best_shared = 0, best_grid = 0;
-  const bool can_share = !g.no_split && sms <= kMaxGrid && p.kb >= 32;
+  // shared tiles: asked for (no_split == 0: taken wherever tiles do not fill whole waves), or left
+  // to this cost model (no_split == 2)
+  const bool can_share = g.no_split != 1 && sms <= kMaxGrid && p.kb >= 32;
+  const bool force_share = g.no_split == 0;
   for (int th = 1; th <= g.p; ++th) {
     if ((int64_t)th * p.pitch - junk > 256 || (int64_t)th * (p.patch ? 1 : g.stride_h) > 256) break;
     if (p.vhalo && g.stride_h > 1 && th > 1) break;
@@ -2174,7 +2198,7 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
         const int64_t waves = (units + sms - 1) / sms;
         double cost = (double)waves * tile_clk((int64_t)tn * th * p.pitch, cols, ks) + finish_clk(ks) +
                       1e-3 * (double)units;
-        if (can_share && tiles % sms != 0) cost *= 1e3;  // shared tiles were asked for (HGC_FLAG_SHARED_TILES)
+        if (force_share && can_share && tiles % sms != 0) cost *= 1e3;  // shared tiles were asked for (HGC_FLAG_SHARED_TILES)
         if (cost < best - 1e-9 ||
             (cost < best + 1e-9 && ks == best_ks && !best_shared && (int64_t)tn * th > (int64_t)best_tn * best_th)) {
           best = cost;
@@ -2189,6 +2213,15 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
         int grid_s = 0;
         double cost_s = 0.0;
         shared_plan(tiles, mma_clk((int64_t)tn * th * p.pitch, cols), cols, sms, &grid_s, &cost_s);
+        if (!force_share) {
+          // Measured (VGG-16, batch 16): a unit hands its first partial tile over and fetches the
+          // partial sums of its last one beside the MMAs of the tiles between them, which takes
+          // whole tiles in between (at least 2.5 tiles per unit); the contiguous ranges cost some
+          // locality in L2 and the hand-overs some time, together about 10k clocks per launch
+          // (conv3_2: 3.03 waves of 11 us tiles, 61.3 -> 55.6 us; conv2_2, conv4_x: slower).
+          cost_s = (double)tiles / (double)sms * tile_clk((int64_t)tn * th * p.pitch, cols, 0) + 10000.0;
+          if (2 * tiles < 5 * (int64_t)sms || grid_s != sms || ts_est < 16) grid_s = 0;
+        }
         if (grid_s > 1 && cost_s < best - 1e-9) {
           best = cost_s;
           best_th = th;

@@ -192,11 +192,19 @@ def test_static_entry_point_refuses_layouts_it_does_not_have():
 
 
 def test_scheduling_flags_change_the_plan_not_the_layer():
-    """HGC_FLAG_CTA_PAIRS / HGC_FLAG_SHARED_TILES are opt-in schedules: off by default, reported by
-    the plan when set and applicable, and never a different output shape or path."""
+    """HGC_FLAG_CTA_PAIRS is opt-in; shared tiles are the planner's choice (this layer: 3.03 waves of
+    long tiles), forced by HGC_FLAG_SHARED_TILES and forbidden by HGC_FLAG_WHOLE_TILES; the plan
+    reports them, and none changes the output shape or the path."""
     args = (16, 256, 56, 56, 256, 3, 3, 1, 1, 1, 1, 1, 1, 1)
-    base = hgc.ConvDesc(*args)
+    auto = hgc.ConvDesc(*args)
+    assert auto.plan_info()["pair"] == 0 and auto.plan_info()["shared_tiles"] == 1
+    base = hgc.ConvDesc(*args, flags=hgc.HGC_FLAG_WHOLE_TILES)
     assert base.plan_info()["pair"] == 0 and base.plan_info()["shared_tiles"] == 0
+    assert hgc.ConvDesc(*args, flags=hgc.HGC_FLAG_WHOLE_TILES | hgc.HGC_FLAG_SHARED_TILES).plan_info()["shared_tiles"] == 0
+    # layers whose tiles are short, or fewer than 2.5 per CTA, keep whole tiles unless asked
+    small = (16, 512, 28, 28, 512, 3, 3, 1, 1, 1, 1, 1, 1, 1)
+    assert hgc.ConvDesc(*small).plan_info()["shared_tiles"] == 0
+    assert hgc.ConvDesc(*small, flags=hgc.HGC_FLAG_SHARED_TILES).plan_info()["shared_tiles"] == 1
     pairs = hgc.ConvDesc(*args, flags=hgc.HGC_FLAG_CTA_PAIRS)
     info = pairs.plan_info()
     assert info["pair"] == 1 and info["ncols"] % 16 == 0 and info["ncols"] <= 256 and info["grid"] <= 74
