@@ -164,6 +164,8 @@ struct IgemmPlan {
   void* y_mapped;  // output pointer tmY/tmYr were encoded for
   uint32_t a_bytes, b_bytes, b_alloc;
   int32_t a_rows;  // rows of a weight tile in shared memory (128, or 64 for layers of <= 64 channels per group)
+  int32_t fine_units;  // TMA-store epilogue works in units of 32 pixels (else 64)
+  int32_t dup_log2;  // log2 of the number of copies of the layer's weight rows in w' and in a weight tile (0, 1, 2)
   size_t smem_bytes;
   int32_t ks_log2;  // log2 of the number of reduction slices a tile is split into (0 = none)
   // work distribution of the kernels without reduction slices: `grid` CTAs take contiguous ranges

@@ -885,6 +885,8 @@ struct IgemmArgs {
   int32_t tma_store;  // 1: the epilogue stages fp16 tiles in shared memory and stores them with TMA
   int32_t rem;        // (th*Q) % 64: width of the last staged pass of a full tile (0 = none)
   int32_t nbuf;       // staging tiles per epilogue warp (1 or 2)
+  int32_t dup_log2;   // log2 of the number of copies of the layer's rows in a weight tile (0, 1, 2)
+  int32_t fine_units; // TMA-store epilogue: units of 32 pixels instead of 64
   // split reduction (its own kernel instantiation): the channel blocks of a tile are dealt out to
   // 2^ks_log2 CTAs, each of which writes its fp32 partial sums to its own slice of `partials`; a
   // second kernel adds the slices in a fixed order (+ bias, ReLU, rounding)
@@ -1555,7 +1557,15 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const int half = ew >> 2;  // which of the quarter's warps this is
     // accumulator lane = output channel within the tile (interleaved within the warp's 32 when the
     // staged channels-last epilogue runs: see convert_store_pixels)
-    const int row = quarter * 32 + ((EPI == 2 && a.y_tma) ? ((lane & 3) << 3) + (lane >> 2) : lane);
+    // Replicated weight rows (layers of 64 or 32 output channels, TMA-store epilogue): lane
+    // quarters 2 and 3 (1, 2 and 3) hold the same channels as quarter 0 and 1 (0), because the
+    // weight tile holds the layer's rows two (four) times; the replicas take different pixels, so
+    // that every epilogue warp has work although the layer fills only part of the MMA's 128 rows.
+    const int rep_q = EPI == 0 ? (4 >> a.dup_log2) : 4;  // lane quarters per replica
+    const int cq = quarter & (rep_q - 1);                // the quarter's place among the channels
+    const int half_eff = EPI == 0 ? (quarter / rep_q) * kPerQuarter + half : half;  // which of the warps that share the channels
+    const int per_eff = EPI == 0 ? (kPerQuarter << a.dup_log2) : kPerQuarter;
+    const int row = cq * 32 + ((EPI == 2 && a.y_tma) ? ((lane & 3) << 3) + (lane >> 2) : lane);
     uint16_t* yb = reinterpret_cast<uint16_t*>(y);
     const uint32_t stage_base = ring_base + (uint32_t)a.stages * a.stage_bytes;
     const bool relu = a.relu != 0;
@@ -1565,6 +1575,8 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     uint32_t unit_ctr = 0, stage_sel = 0;
     uint32_t lt = 0;
     uint32_t meet_phase = 0, ho_phase = 0, pl_phase = 0;
+    float bv = 0.f;
+    int bias_k = -1;
     // Shared tiles: when this unit's range ends inside a tile whose first stage it holds, it
     // finishes that tile (its last item), and the following units computed the tile's later parts
     // first of all.  The sum of their partial accumulators is put into the tile's accumulator
@@ -1639,12 +1651,18 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       const int kin = m0 + row;
       const bool kvalid = kin < a.kg;
       const int k = grp * a.kg + (kvalid ? kin : 0);
-      const float bv = (bias != nullptr && kvalid) ? __half2float(__ldg(bias + k)) : 0.f;
+      // (fetched again only when the channel changes: a load from global memory at the head of
+      //  every tile's epilogue costs several hundred clocks, a third of a short tile's epilogue)
+      const int bias_key = kvalid ? k : -2;
+      if (bias_key != bias_k) {
+        bv = (bias != nullptr && kvalid) ? __half2float(__ldg(bias + k)) : 0.f;
+        bias_k = bias_key;
+      }
       const uint32_t buf = lt & 1u;
       if (!mbar_wait(smem_u32(&acc_full[buf]), (lt >> 1) & 1u, &abort_flag, 256)) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t t_tile = tmem_base + buf * 256u + ((uint32_t)(quarter * 32) << 16);
-      const bool quarter_live = m0 + quarter * 32 < a.kg;  // any real output channel in this warp's lanes?
+      const bool quarter_live = m0 + cq * 32 < a.kg;  // any real output channel in this warp's lanes?
       // the barrier the accumulator is handed back on (of a pair: the first CTA's)
       const uint32_t acc_empty_bar = PAIR ? cluster_addr(smem_u32(&acc_empty[buf]), 0) : smem_u32(&acc_empty[buf]);
 
@@ -1696,10 +1714,12 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           const bool last_row_tile = p0 + a.th >= a.P;
           // (row, column) of the unit's first pixel, kept up to date without divisions
           const bool linear = a.pitch == a.Q;  // no junk columns: accumulator columns are consecutive pixels
-          int hr = 0, wc = half * kPassElems;
+          // pixels per unit: 64, or 32 where the replicas would otherwise leave warps without a unit
+          const int upx = a.fine_units ? 32 : kPassElems;
+          int hr = 0, wc = half_eff * upx;
           while (!linear && wc >= a.Q) { wc -= a.Q; ++hr; }
-          for (int e_lo = half * kPassElems; e_lo < e_valid; e_lo += kPerQuarter * kPassElems, ++unit_ctr) {
-            const int e_hi = e_lo + kPassElems < e_valid ? e_lo + kPassElems : e_valid;
+          for (int e_lo = half_eff * upx; e_lo < e_valid; e_lo += per_eff * upx, ++unit_ctr) {
+            const int e_hi = e_lo + upx < e_valid ? e_lo + upx : e_valid;
             const uint32_t sbuf = my_stage + stage_sel * kWarpStageBytes;
             stage_sel = a.nbuf == 2 ? stage_sel ^ 1u : 0u;
             int uh = hr, uw = wc;  // walks through this unit
@@ -1746,12 +1766,12 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) {
-              const bool full_box = (e_hi - e_lo == kPassElems) || last_row_tile;  // past P*Q the store is clipped
-              tma_store_4d(full_box ? &tmY : &tmYr, sbuf, p0 * a.Q + e_lo, m0 + quarter * 32, grp, n0);
+              const bool full_box = !a.fine_units && ((e_hi - e_lo == kPassElems) || last_row_tile);  // past P*Q the store is clipped
+              tma_store_4d(full_box ? &tmY : &tmYr, sbuf, p0 * a.Q + e_lo, m0 + cq * 32, grp, n0);
               asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             }
             // first pixel of this warp's next unit
-            wc += kPerQuarter * kPassElems;
+            wc += per_eff * upx;
             while (!linear && wc >= a.Q) { wc -= a.Q; ++hr; }
           }
         }
@@ -2314,7 +2334,8 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
   // still reads 128 rows: the upper 64 come from whatever follows in shared memory and land in
   // accumulator lanes that no epilogue warp reads; half the tile bytes, one more ring stage)
   p.a_rows = g.kg <= 64 ? 64 : 128;
-  p.a_bytes = (uint32_t)p.a_rows * p.kb * 2u;
+  p.dup_log2 = 0;
+  p.fine_units = 0;
   const uint32_t box_rows = (uint32_t)(p.tn * p.th * p.pitch);
   p.b_bytes = box_rows * p.kb * 2u;
   // rows the MMA may touch: the last tap starts (S-1)*dil rows in and reads ncols rows
@@ -2349,6 +2370,22 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
   }
   p.sk_split = best_shared;
   p.grid = best_grid;
+  // Layers of exactly 64 output channels and a short reduction whose tiles are bound by the
+  // epilogue (the wide epilogue was chosen): the weight tensor is laid out twice, one copy after the
+  // other, the weight tile is 128 rows again, and all lane quarters hold real channels (see the kernel).
+  if (p.epi_warps == kEpilogueWarpsWide && !p.y_nhwc && p.tma_store && g.group == 1 && best_ks == 0 && !best_shared &&
+      !want_pair && g.dw_stride == 0 && g.kg == 64 && mpt <= 8.0) {
+    // (measured: VGG conv1_1 47.5 -> 41.1 us, 1x1 layers 32 -> 64 and 64 -> 64 channels 7 % faster;
+    //  with a longer reduction the doubled weight traffic costs more than the epilogue gains, and
+    //  four copies of a 32-channel layer were slower than one)
+    p.dup_log2 = 1;
+    p.a_rows = 128;
+    // a tile's units of 64 pixels x 32 channels are fewer than the warps that can now take them:
+    // units of 32 pixels (stored through the remainder map, whose box is then 32 pixels)
+    const int px = p.th * g.q;
+    if (px % 32 == 0 && ((px + 63) / 64) * (g.kg / 32) < p.epi_warps) p.fine_units = 1;
+  }
+  p.a_bytes = (uint32_t)p.a_rows * p.kb * 2u;
   p.sk_cols32 = (p.ncols + 31) / 32;
   if (p.pair || p.sk_split || g.dw_stride > 0) p.epi_warps = kEpilogueWarps;
   // split reduction (chosen with the tile shape above): fp32 partials, copy-style epilogue
@@ -2428,7 +2465,7 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
   // workspace: header (status word, hand-over flags), re-laid-out weights, NHWC input
   p.ws_status_off = 0;
   p.ws_w_off = kWsHeaderBytes;
-  p.ws_x_off = p.ws_w_off + round_up_sz((size_t)g.k * p.eff_r * p.eff_s * p.cw * 2, 256);
+  p.ws_x_off = p.ws_w_off + round_up_sz(((size_t)g.k << p.dup_log2) * p.eff_r * p.eff_s * p.cw * 2, 256);
   p.ws_part_off = 0;
   p.ws_total = p.ws_x_off + ((p.nchw || p.x_nhwc) ? 0
                                     : round_up_sz(p.patch    ? (size_t)g.n * g.p * g.q * p.cw * 2
@@ -2522,7 +2559,7 @@ bool igemm_encode_maps(const ConvGeom& g, IgemmPlan* p, void* ws) {
     // shared memory, i.e. one K-major weight tile per tap
     const cuuint64_t ntaps = (cuuint64_t)p->eff_r * p->eff_s;
     const cuuint64_t kred = ntaps * p->cw;
-    cuuint64_t dims[4] = {(cuuint64_t)p->cw, (cuuint64_t)g.kg, ntaps, (cuuint64_t)g.group};
+    cuuint64_t dims[4] = {(cuuint64_t)p->cw, (cuuint64_t)g.kg << p->dup_log2, ntaps, (cuuint64_t)g.group};  // (replicas: group == 1)
     cuuint64_t strides[3] = {kred * 2, (cuuint64_t)p->cw * 2, kred * 2 * (cuuint64_t)g.kg};
     cuuint32_t box[4] = {(cuuint32_t)p->kb, (cuuint32_t)p->a_rows, (cuuint32_t)p->taps, 1};
     cuuint32_t es[4] = {1, 1, 1, 1};
@@ -2625,7 +2662,7 @@ bool igemm_encode_y_maps(const ConvGeom& g, IgemmPlan* p, void* y) {
   cuuint64_t strides[3] = {pq * 2, pq * 2 * (cuuint64_t)g.kg, pq * 2 * (cuuint64_t)g.k};
   cuuint32_t es[4] = {1, 1, 1, 1};
   for (int i = 0; i < 2; ++i) {
-    cuuint32_t box[4] = {(cuuint32_t)((i == 0 || p->rem == 0) ? kPassElems : p->rem), 32, 1, 1};
+    cuuint32_t box[4] = {(cuuint32_t)(i == 0 ? kPassElems : (p->fine_units ? 32 : (p->rem == 0 ? kPassElems : p->rem))), 32, 1, 1};
     if (enc(i == 0 ? &p->tmY : &p->tmYr, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, y, dims, strides, box, es,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -2692,6 +2729,8 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
   a.tma_store = p.tma_store;
   a.rem = p.rem;
   a.nbuf = p.nbuf;
+  a.dup_log2 = p.dup_log2;
+  a.fine_units = p.fine_units;
   a.ks_log2 = p.ks_log2;
   a.part_stride = (int64_t)g.n * g.k * g.p * g.q;
   a.y_tma = (p.y_nhwc && p.tma_store) ? 1 : 0;

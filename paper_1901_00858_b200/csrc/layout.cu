@@ -610,9 +610,17 @@ cudaError_t launch_weights_repack_patch(const __half* src, __half* dst, int32_t 
 // The two preparation steps of the tensor-core path, dispatched on the plan's mode.
 cudaError_t launch_igemm_weights(const ConvGeom& g, const IgemmPlan& p, const __half* w, __half* wp,
                                  cudaStream_t stream) {
-  if (p.patch) return launch_weights_repack_patch(w, wp, g.k, g.c, g.r, g.s, p.cw, stream, p.y_perm);
-  if (p.window) return launch_weights_repack_window(w, wp, g.k, g.c, g.r, g.s, p.kw_pix, stream, p.y_perm, p.px_ch);
-  return launch_weights_repack(w, wp, g.k, g.cg, g.r, g.s, g.group, p.cw, stream, p.y_perm);
+  // (replicated rows: the whole re-laid-out tensor once per replica, one copy after the other)
+  const size_t copy_elems = (size_t)g.k * p.eff_r * p.eff_s * p.cw;
+  for (int i = 0; i < (1 << p.dup_log2); ++i) {
+    __half* dst = wp + (size_t)i * copy_elems;
+    cudaError_t e;
+    if (p.patch) e = launch_weights_repack_patch(w, dst, g.k, g.c, g.r, g.s, p.cw, stream, p.y_perm);
+    else if (p.window) e = launch_weights_repack_window(w, dst, g.k, g.c, g.r, g.s, p.kw_pix, stream, p.y_perm, p.px_ch);
+    else e = launch_weights_repack(w, dst, g.k, g.cg, g.r, g.s, g.group, p.cw, stream, p.y_perm);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 __global__ void __launch_bounds__(256)
