@@ -215,8 +215,13 @@ int hgc_conv_path(const hgc_conv_desc* d, int32_t* path);
  * [14] 1 if the launch consists of CTA pairs (clusters of two that share tiles of 256 output
  * channels; [3], [4] then describe one CTA's pixel sub-tile, [6] the MMA N of the pair, [7] the
  * number of pair tiles, [12] the number of pairs), [15] 1 if the NCHW->NHWC copy of x ([10] = 0)
- * is made by extra warps of the tensor-core kernel itself instead of a kernel of its own; zeros
- * for the other paths.  info: host pointer.
+ * is made by extra warps of the tensor-core kernel itself instead of a kernel of its own, [16] 1
+ * if a layer of 64 output channels runs as row pairs: accumulator lanes 64..127 of the 128-row MMA
+ * hold the odd output rows ([4] then counts row pairs per tile, [7] tiles of two output rows, [9]
+ * and the kernel's taps are those of a kernel with one more row), [17] the number of copies of the
+ * layer's weight rows in a weight tile (2 for epilogue-bound layers of 64 output channels: lane
+ * quarters 2 and 3 then hold the same channels as 0 and 1 and take other pixels; else 1); zeros
+ * for the other paths.  info: host pointer; at most 18 values are written.
  */
 int hgc_conv_plan_info(const hgc_conv_desc* d, int32_t* info, int32_t count);
 

@@ -22,6 +22,7 @@ struct ConvGeom {
   int32_t no_pair;         // 1: never pair CTAs on 256-channel tiles
   int32_t no_fuse;         // 1: the layout pass stays a kernel of its own
   int32_t dw_stride;       // > 0: the pointwise layer of a depthwise + pointwise block; the depthwise layer's stride
+  int32_t rowpair;         // planner-internal: this is the re-stated form of a 64-channel layer (IgemmPlan::rowpair)
 };
 
 // First bytes of the tensor-core path's workspace: the device status word (int at byte 0) and,
@@ -165,6 +166,12 @@ struct IgemmPlan {
   uint32_t a_bytes, b_bytes, b_alloc;
   int32_t a_rows;  // rows of a weight tile in shared memory (128, or 64 for layers of <= 64 channels per group)
   int32_t fine_units;  // TMA-store epilogue works in units of 32 pixels (else 64)
+  // Row pairs: a stride-1 layer of 64 output channels with R kernel rows is run as a layer of 128
+  // "channels" (output row parity x channel), R + 1 kernel rows and stride 2 along H on P/2 rows:
+  // accumulator lanes 64..127 hold the odd output rows, so no lane of the 128-row MMA is idle
+  // (3x3: 12 MMA steps per two output rows instead of 18).  The plan's shapes are those of the
+  // re-stated layer; w' holds the R + 1 shifted copies of the kernel rows (zero where a row has none).
+  int32_t rowpair;
   int32_t dup_log2;  // log2 of the number of copies of the layer's weight rows in w' and in a weight tile (0, 1, 2)
   size_t smem_bytes;
   int32_t ks_log2;  // log2 of the number of reduction slices a tile is split into (0 = none)

@@ -887,6 +887,7 @@ struct IgemmArgs {
   int32_t nbuf;       // staging tiles per epilogue warp (1 or 2)
   int32_t dup_log2;   // log2 of the number of copies of the layer's rows in a weight tile (0, 1, 2)
   int32_t fine_units; // TMA-store epilogue: units of 32 pixels instead of 64
+  int32_t rowpair;    // lanes 64..127 hold the odd output rows of the layer's 64 channels (IgemmPlan::rowpair)
   // split reduction (its own kernel instantiation): the channel blocks of a tile are dealt out to
   // 2^ks_log2 CTAs, each of which writes its fp32 partial sums to its own slice of `partials`; a
   // second kernel adds the slices in a fixed order (+ bias, ReLU, rounding)
@@ -1561,10 +1562,14 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     // quarters 2 and 3 (1, 2 and 3) hold the same channels as quarter 0 and 1 (0), because the
     // weight tile holds the layer's rows two (four) times; the replicas take different pixels, so
     // that every epilogue warp has work although the layer fills only part of the MMA's 128 rows.
-    const int rep_q = EPI == 0 ? (4 >> a.dup_log2) : 4;  // lane quarters per replica
-    const int cq = quarter & (rep_q - 1);                // the quarter's place among the channels
-    const int half_eff = EPI == 0 ? (quarter / rep_q) * kPerQuarter + half : half;  // which of the warps that share the channels
-    const int per_eff = EPI == 0 ? (kPerQuarter << a.dup_log2) : kPerQuarter;
+    // Row pairs: quarters 2 and 3 hold the same channels too, but of the odd output rows; the
+    // two halves do not share pixels, they store to rows 2 * p0 and 2 * p0 + 1.
+    const int rep_q = EPI == 0 ? (a.rowpair ? 2 : (4 >> a.dup_log2)) : 4;  // lane quarters per replica
+    const int cq = quarter & (rep_q - 1);                                  // the quarter's place among the channels
+    const bool split_px = EPI == 0 && !a.rowpair;
+    const int half_eff = split_px ? (quarter / rep_q) * kPerQuarter + half : half;  // which of the warps that share the pixels
+    const int per_eff = split_px ? (kPerQuarter << a.dup_log2) : kPerQuarter;
+    const int odd_row = (EPI == 0 && a.rowpair) ? (quarter >> 1) : 0;
     const int row = cq * 32 + ((EPI == 2 && a.y_tma) ? ((lane & 3) << 3) + (lane >> 2) : lane);
     uint16_t* yb = reinterpret_cast<uint16_t*>(y);
     const uint32_t stage_base = ring_base + (uint32_t)a.stages * a.stage_bytes;
@@ -1649,7 +1654,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       it.channel_tile(a, grp, m0);
       if constexpr (PAIR) m0 += (int)rank * 128;  // this CTA's tensor memory holds its own 128 channels
       const int kin = m0 + row;
-      const bool kvalid = kin < a.kg;
+      const bool kvalid = kin < (a.rowpair ? 64 : a.kg);
       const int k = grp * a.kg + (kvalid ? kin : 0);
       // (fetched again only when the channel changes: a load from global memory at the head of
       //  every tile's epilogue costs several hundred clocks, a third of a short tile's epilogue)
@@ -1662,7 +1667,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       if (!mbar_wait(smem_u32(&acc_full[buf]), (lt >> 1) & 1u, &abort_flag, 256)) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t t_tile = tmem_base + buf * 256u + ((uint32_t)(quarter * 32) << 16);
-      const bool quarter_live = m0 + cq * 32 < a.kg;  // any real output channel in this warp's lanes?
+      const bool quarter_live = m0 + cq * 32 < (a.rowpair ? 64 : a.kg);  // any real output channel in this warp's lanes?
       // the barrier the accumulator is handed back on (of a pair: the first CTA's)
       const uint32_t acc_empty_bar = PAIR ? cluster_addr(smem_u32(&acc_empty[buf]), 0) : smem_u32(&acc_empty[buf]);
 
@@ -1766,8 +1771,9 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) {
-              const bool full_box = !a.fine_units && ((e_hi - e_lo == kPassElems) || last_row_tile);  // past P*Q the store is clipped
-              tma_store_4d(full_box ? &tmY : &tmYr, sbuf, p0 * a.Q + e_lo, m0 + cq * 32, grp, n0);
+              // past P*Q the store is clipped (row pairs: the next row of y belongs to other warps)
+              const bool full_box = !a.fine_units && ((e_hi - e_lo == kPassElems) || (last_row_tile && !a.rowpair));
+              tma_store_4d(full_box ? &tmY : &tmYr, sbuf, (a.rowpair ? 2 * p0 + odd_row : p0) * a.Q + e_lo, m0 + cq * 32, grp, n0);
               asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             }
             // first pixel of this warp's next unit
@@ -1979,7 +1985,38 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
 
 // The plan of a layer: the single-CTA form, or CTA pairs where they were asked for and the layer
 // has more than 128 output channels per group.
+// The layer that a row-pair plan (IgemmPlan::rowpair) runs in place of layer g: 128 "channels"
+// (parity of the output row x the 64 channels), R + 1 kernel rows, stride 2 along H, P/2 rows.
+static ConvGeom rowpair_geom(const ConvGeom& g) {
+  ConvGeom r = g;
+  r.k = r.kg = 128;
+  r.r = g.r + 1;
+  r.stride_h = 2;
+  r.p = g.p / 2;
+  r.rowpair = 1;
+  return r;
+}
+static inline ConvGeom effective_geom(const ConvGeom& g, const IgemmPlan& p) { return p.rowpair ? rowpair_geom(g) : g; }
+
 bool igemm_make_plan(const ConvGeom& g, IgemmPlan* out) {
+  // Row pairs: stride-1 layers of exactly 64 output channels with at least two kernel rows and a
+  // wide, even output plane, NCHW output through the TMA-store epilogue (VGG-16 conv1_2: the
+  // kernel 77 -> ... us).  Narrow planes would need several row pairs per tile, whose rows of
+  // one parity are not contiguous in y: not built.
+  if (!g.rowpair && g.group == 1 && g.kg == 64 && g.cg >= 16 && g.r >= 2 && g.stride_h == 1 && g.stride_w == 1 &&
+      g.dil_h == 1 && g.dil_w == 1 && !g.y_nhwc && g.dw_stride == 0 && (g.p % 2) == 0 && (g.q % 8) == 0 && g.q >= 112 &&
+      g.q + (g.s - 1) <= 256) {
+    ConvGeom g2 = rowpair_geom(g);
+    g2.no_pair = 1;
+    g2.no_split = 1;
+    IgemmPlan rp{};
+    if (make_plan_impl(g2, &rp, false, 64, false) && rp.th == 1 && rp.tn == 1 && rp.tma_store && rp.halo && !rp.nchw &&
+        rp.ks_log2 == 0 && !rp.fuse_layout) {
+      rp.rowpair = 1;
+      *out = rp;
+      return true;
+    }
+  }
   ConvGeom gs = g;
   gs.no_pair = 1;
   IgemmPlan single{};
@@ -2102,7 +2139,7 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
     p.c_pad = (g.c + 7) / 8 * 8;
     p.eff_r = g.r; p.eff_s = g.s; p.eff_pad_h = g.pad_h; p.eff_pad_w = g.pad_w;
     // stride 1: the S taps of a kernel row read one shared tile, shifted by s*dil pixels
-    p.halo = (g.stride_h == 1 && g.stride_w == 1) ? 1 : 0;
+    p.halo = ((g.stride_h == 1 || g.rowpair) && g.stride_w == 1) ? 1 : 0;  // (row pairs: one row of columns per tile)
   }
   // 1x1, stride 1, unpadded layers on planes of a multiple of 8 pixels read x as it is (no NHWC
   // copy): the activation operand is then pixel-major ("MN-major") in shared memory
@@ -2195,6 +2232,7 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
   for (int th = 1; th <= g.p; ++th) {
     if ((int64_t)th * p.pitch - junk > 256 || (int64_t)th * (p.patch ? 1 : g.stride_h) > 256) break;
     if (p.vhalo && g.stride_h > 1 && th > 1) break;
+    if (g.rowpair && th > 1) break;
     if (p.nchw && th != g.p && ((int64_t)th * g.q) % 8 != 0) continue;  // tiles must start on 16-byte boundaries of x
     const int tn_hi = (th == g.p && !p.nchw && !p.vhalo) ? g.n : 1;  // several images only when a tile holds whole planes
     for (int tn = 1; tn <= tn_hi; ++tn) {
@@ -2546,7 +2584,8 @@ bool encode_dw_input_map(const DwBlock& dw, int n, IgemmPlan* p) {
 }
 
 // Encodes the two tensor maps over the workspace tensors.  Returns false on failure.
-bool igemm_encode_maps(const ConvGeom& g, IgemmPlan* p, void* ws) {
+bool igemm_encode_maps(const ConvGeom& g_layer, IgemmPlan* p, void* ws) {
+  const ConvGeom g = effective_geom(g_layer, *p);
   PFN_cuTensorMapEncodeTiled_v12000 enc = encode_fn();
   if (enc == nullptr) return false;
   char* base = static_cast<char*>(ws);
@@ -2672,8 +2711,9 @@ bool igemm_encode_y_maps(const ConvGeom& g, IgemmPlan* p, void* y) {
   return true;
 }
 
-cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half* x, const __half* bias, __half* y,
+cudaError_t launch_igemm(const ConvGeom& g_layer, IgemmPlan& p, void* ws, const __half* x, const __half* bias, __half* y,
                          int relu, cudaStream_t stream, const DwBlock* dw) {
+  const ConvGeom g = effective_geom(g_layer, p);
   if (!p.maps_ready) return cudaErrorInvalidValue;
   if (dw != nullptr && (!p.x_nhwc || p.pair || p.sk_split || p.ks_log2 > 0 || p.fuse_layout || p.kb < 32))
     return cudaErrorInvalidValue;
@@ -2686,7 +2726,7 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
     if (!encode_nhwc_map(g, &p, const_cast<__half*>(x))) return cudaErrorInvalidValue;
     p.x_mapped = x;
   }
-  if (p.tma_store && p.y_mapped != y && !igemm_encode_y_maps(g, &p, y)) return cudaErrorInvalidValue;
+  if (p.tma_store && p.y_mapped != y && !igemm_encode_y_maps(g_layer, &p, y)) return cudaErrorInvalidValue;  // (y is the layer's)
   IgemmArgs a{};
   a.N = g.n; a.K = g.k; a.P = g.p; a.Q = g.q;
   a.kg = g.kg; a.group = g.group;
@@ -2731,6 +2771,7 @@ cudaError_t launch_igemm(const ConvGeom& g, IgemmPlan& p, void* ws, const __half
   a.nbuf = p.nbuf;
   a.dup_log2 = p.dup_log2;
   a.fine_units = p.fine_units;
+  a.rowpair = p.rowpair;
   a.ks_log2 = p.ks_log2;
   a.part_stride = (int64_t)g.n * g.k * g.p * g.q;
   a.y_tma = (p.y_nhwc && p.tma_store) ? 1 : 0;

@@ -607,9 +607,44 @@ cudaError_t launch_weights_repack_patch(const __half* src, __half* dst, int32_t 
   return cudaGetLastError();
 }
 
+// Row pairs (IgemmPlan::rowpair): w[k][c][r][s] (k < 64) -> w'[half * 64 + k][r'][s][c_pad] with
+// r' = r + half, r' in [0, R]; rows r' that a half does not have are zero.  One thread per 8 channels.
+__global__ void weights_repack_rowpair_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int cg, int r,
+                                              int s, int c_pad) {
+  grid_dependency_wait();
+  const int64_t vecs_per_k = (int64_t)(r + 1) * s * (c_pad / 8);
+  const int64_t total = 128 * vecs_per_k;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int kk = (int)(i / vecs_per_k);
+    const int64_t rem = i % vecs_per_k;
+    const int t = (int)(rem / (c_pad / 8));  // tap r' * s + column
+    const int cv = (int)(rem % (c_pad / 8));
+    const int half = kk >> 6, k = kk & 63;
+    const int rr = t / s - half, ss = t % s;
+    uint32_t o[4] = {0, 0, 0, 0};
+    if (rr >= 0 && rr < r) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int ch = cv * 8 + j;
+        uint32_t v = 0;
+        if (ch < cg) v = src[(((int64_t)k * cg + ch) * r + rr) * s + ss];
+        o[j >> 1] |= v << ((j & 1) * 16);
+      }
+    }
+    *reinterpret_cast<uint4*>(dst + ((int64_t)kk * (r + 1) * s + t) * c_pad + cv * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
 // The two preparation steps of the tensor-core path, dispatched on the plan's mode.
 cudaError_t launch_igemm_weights(const ConvGeom& g, const IgemmPlan& p, const __half* w, __half* wp,
                                  cudaStream_t stream) {
+  if (p.rowpair) {
+    const int64_t total = (int64_t)128 * (g.r + 1) * g.s * (p.cw / 8);
+    launch_kernel(weights_repack_rowpair_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, stream,
+                  reinterpret_cast<const uint16_t*>(w), reinterpret_cast<uint16_t*>(wp), g.cg, g.r, g.s, p.cw);
+    count_launch();
+    return cudaGetLastError();
+  }
   // (replicated rows: the whole re-laid-out tensor once per replica, one copy after the other)
   const size_t copy_elems = (size_t)g.k * p.eff_r * p.eff_s * p.cw;
   for (int i = 0; i < (1 << p.dup_log2); ++i) {

@@ -114,7 +114,7 @@ def test_planner_paths():
 def test_plan_info_reports_tiling_and_activation_source():
     """The planner runs on the host: its choices can be checked without a GPU."""
     keys = {"path", "kb", "halo", "tn", "th", "pitch", "ncols", "tiles", "stages", "taps", "x_source", "k_slices",
-            "grid", "shared_tiles", "pair", "fused_layout"}
+            "grid", "shared_tiles", "pair", "fused_layout", "row_pairs", "replicas"}
     cases = [
         # (n, c, h, w, k, r, s, pad, stride), x_source
         ((16, 256, 56, 56, 256, 3, 3, 1, 1), 0),   # NHWC copy of x
@@ -215,6 +215,24 @@ def test_scheduling_flags_change_the_plan_not_the_layer():
         assert d.output_dims() == base.output_dims() and d.path() == base.path()
     # a layer with 128 output channels has nothing to pair
     assert hgc.ConvDesc(16, 128, 112, 112, 128, 3, 3, 1, 1, flags=hgc.HGC_FLAG_CTA_PAIRS).plan_info()["pair"] == 0
+
+
+def test_64_channel_layers_fill_the_mma():
+    """Layers of 64 output channels leave half of the 128-row MMA idle.  Wide stride-1 layers with
+    several kernel rows run as row pairs (odd output rows in the upper lanes: tiles of two rows, one
+    more kernel row); epilogue-bound ones with a short reduction hold their weight rows twice."""
+    rp = hgc.ConvDesc(16, 64, 224, 224, 64, 3, 3, 1, 1).plan_info()
+    assert rp["row_pairs"] == 1 and rp["th"] == 1 and rp["tiles"] == 16 * 112 and rp["replicas"] == 1
+    # not: odd output height, narrow planes, strides, channels-last output, other channel counts
+    for args, kw in [((16, 64, 223, 224, 64, 3, 3, 1, 1), {}), ((64, 64, 56, 56, 64, 3, 3, 1, 1), {}),
+                     ((16, 64, 224, 224, 64, 3, 3, 1, 1, 2, 2), {}), ((16, 64, 224, 224, 128, 3, 3, 1, 1), {}),
+                     ((16, 64, 224, 224, 64, 3, 3, 1, 1), {"flags": hgc.HGC_FLAG_Y_NHWC}),
+                     ((16, 64, 224, 224, 64, 1, 1, 0, 0), {})]:
+        assert hgc.ConvDesc(*args, **kw).plan_info()["row_pairs"] == 0, args
+    assert hgc.ConvDesc(16, 3, 224, 224, 64, 3, 3, 1, 1).plan_info()["replicas"] == 2     # stem: 6 MMAs per tile
+    assert hgc.ConvDesc(32, 32, 112, 112, 64, 1, 1, 0, 0).plan_info()["replicas"] == 2    # 1x1, 32 channels in
+    assert hgc.ConvDesc(64, 256, 56, 56, 64, 1, 1, 0, 0).plan_info()["replicas"] == 1     # long reduction
+    assert hgc.ConvDesc(16, 64, 112, 112, 128, 3, 3, 1, 1).plan_info()["replicas"] == 1
 
 
 def test_block_descriptor_validation():

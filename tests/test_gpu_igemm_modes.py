@@ -65,6 +65,19 @@ CASES = [
     ("stem 3x3 c4 stride 2 dilated (patches)", params_dict(2, 4, 30, 30, 20, 3, 3, 2, 2, 2, 2, 2, 2), X_PATCHES),
     ("stem 5x5 c2 stride 3 (patches, generic expansion)", params_dict(2, 2, 29, 35, 20, 5, 5, 2, 2, 3, 3), X_PATCHES),
     ("stem 1x1 c8 stride 2 (patches)", params_dict(2, 8, 18, 18, 16, 1, 1, 0, 0, 2, 2), X_PATCHES),
+    # 64 output channels: odd output rows in the upper accumulator lanes (row pairs) ...
+    ("row pairs 3x3 c16 112 wide", params_dict(2, 16, 10, 112, 64, 3, 3, 1, 1), X_NHWC_COPY),
+    ("row pairs 3x3 c64 224 wide, two images", params_dict(2, 64, 6, 224, 64, 3, 3, 1, 1), X_NHWC_COPY),
+    ("row pairs 2x3 c32 120 wide, pad 1", params_dict(3, 32, 9, 120, 64, 2, 3, 1, 1), X_NHWC_COPY),
+    ("row pairs 5x1 c24 unpadded columns, pad 2 rows", params_dict(1, 24, 8, 136, 64, 5, 1, 2, 0), X_NHWC_COPY),
+    ("row pairs 3x3 c40 without padding (channel tail)", params_dict(2, 40, 12, 130, 64, 3, 3, 0, 0), X_NHWC_COPY),
+    ("row pairs 4x3 c64 248 wide (250 columns)", params_dict(1, 64, 7, 248, 64, 4, 3, 1, 1), X_NHWC_COPY),
+    # ... or, for epilogue-bound layers, the weight rows twice (replicas that take other pixels)
+    ("replicas 1x1 c32 112x112 k64", params_dict(2, 32, 112, 112, 64, 1, 1), X_DIRECT),
+    ("replicas 1x1 c64 56x56 k64", params_dict(8, 64, 56, 56, 64, 1, 1), X_DIRECT),
+    ("replicas stem 3x3 c3 224 wide k64 (32-pixel units)", params_dict(2, 3, 12, 224, 64, 3, 3, 1, 1), X_WINDOWS),
+    ("replicas 1x1 c32 27x72 k64 (64-pixel units, ragged tiles)", params_dict(8, 32, 27, 72, 64, 1, 1), X_DIRECT),
+    ("replicas stem 3x3 c3 200 wide k64 (64-pixel units, ragged)", params_dict(2, 3, 20, 200, 64, 3, 3, 1, 1), X_WINDOWS),
 ]
 
 
@@ -77,6 +90,10 @@ def test_igemm_mode(hgc, oracle, name, a, source):
     assert d.path() == hgc.HGC_PATH_IGEMM, name
     if source is not None:
         assert d.plan_info()["x_source"] == source, (name, d.plan_info())
+    if name.startswith("row pairs"):
+        assert d.plan_info()["row_pairs"] == 1, d.plan_info()
+    if name.startswith("replicas"):
+        assert d.plan_info()["replicas"] == 2, d.plan_info()
     if "reduction split" in name:
         # several CTAs per tile: reduction slices with a second pass, or CTAs that hand their
         # accumulators over inside the one launch
