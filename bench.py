@@ -498,6 +498,8 @@ def run_ours(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.launch_overlap:
+        hgc.set_launch_overlap(True)
     if not torch.cuda.is_available():
         raise SystemExit("bench.py: no CUDA device; the CUDA path has no CPU fallback")
     torch.cuda.set_device(local)
@@ -871,6 +873,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of replaying the step as a CUDA graph")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     ap.add_argument("--no-extra", action="store_true", help="skip the other workloads of the `workloads` object")
+    ap.add_argument("--launch-overlap", action="store_true",
+                    help="launch the library's kernels with programmatic stream serialization (hgc_set_launch_overlap)")
     ap.add_argument("--only", default="", help="comma-separated layer names: run just these layers (profiling)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling on a small case)")
     args = ap.parse_args()

@@ -391,8 +391,12 @@ int hgc_debug_drop_copies(int32_t index);
  * kernel of the stream is still draining, and waits, before it touches global memory, until that
  * kernel has completed.  Results are the same either way.  Measured on B200: with eager launches
  * the gap between dependent kernels shrinks (a VGG-16 step 0.776 -> 0.757 ms, ResNet-50 1.76 ->
- * 1.69 ms); a step replayed as a CUDA graph gets slower with programmatic edges (0.657 -> 0.737
- * ms), which is why it is off unless asked for.  Applies to all later launches of this process.
+ * 1.69 ms); a step replayed as a CUDA graph gets slower when layout passes sit between the
+ * tensor-core kernels (NCHW layers: 0.605 -> 0.696 ms; 0.665 ms when the tensor-core kernel
+ * releases its dependents only after its last MMA) and 2 % faster when it consists of tensor-core
+ * kernels only (channels-last chain: 0.514 -> 0.504 ms), which is why it is off unless asked for
+ * (`python bench.py --launch-overlap` repeats the measurement).  Applies to all later launches
+ * of this process.
  * Always returns HGC_OK.
  */
 int hgc_set_launch_overlap(int enabled);
