@@ -605,9 +605,10 @@ __device__ __noinline__ void epilogue_copy(uint32_t t_addr, uint32_t sbuf, int f
   const int rows_valid = (P - p0) < th ? (P - p0) : th;
   const int cols_need = (rows_valid - 1) * pitch + Q;  // columns of one image up to its last real pixel
   const int img_cols = th * pitch;
-  // pairs of columns can be copied as 4-byte words when columns are pixels (no junk) and every
-  // image's first pixel and every channel plane start on a 4-byte boundary
-  const bool words = pitch == Q && (pq & 1) == 0 && ((p0 * Q) & 1) == 0 && (cols_need & 1) == 0;
+  // pairs of columns can be copied as 4-byte words when rows (with their junk columns, if any) are
+  // an even number of columns long, so that a pair never straddles a row end, and every image's
+  // first pixel and every channel plane start on a 4-byte boundary
+  const bool words = (Q & 1) == 0 && (pitch & 1) == 0 && (pq & 1) == 0 && ((p0 * Q) & 1) == 0 && (cols_need & 1) == 0;
   const uint32_t row_off = (uint32_t)lane * 128u;
   int unit = 0;
   for (int img = 0; img < tn; ++img) {
@@ -642,8 +643,11 @@ __device__ __noinline__ void epilogue_copy(uint32_t t_addr, uint32_t sbuf, int f
       // ---- staging tile -> y (lane = column) ----
       if (words) {
         const int col = 2 * lane;  // columns col, col + 1 of the unit
-        if (col < ncol) {          // ncol is even here
-          uint16_t* dst = yimg + (int64_t)p0 * Q + c0 + col;
+        const int cabs = c0 + col;
+        const int hr = cabs / pitch;
+        const int wc = cabs - hr * pitch;
+        if (col < ncol && wc < Q) {  // ncol is even here; junk columns come in pairs too
+          uint16_t* dst = yimg + (int64_t)(p0 + hr) * Q + wc;
           const uint32_t chunk = (uint32_t)col >> 3, within = ((uint32_t)col & 7u) * 2u;
 #pragma unroll 4
           for (int r = 0; r < kvalid_rows; ++r) {
