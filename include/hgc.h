@@ -386,17 +386,19 @@ int hgc_debug_set_wait_limit_ns(uint64_t ns);
 int hgc_debug_drop_copies(int32_t index);
 
 /*
- * Launch overlap (off by default).  With enabled != 0 the library launches its kernels with the
- * programmatic stream serialization attribute: a kernel may be scheduled while the previous
- * kernel of the stream is still draining, and waits, before it touches global memory, until that
- * kernel has completed.  Results are the same either way.  Measured on B200: with eager launches
- * the gap between dependent kernels shrinks (a VGG-16 step 0.776 -> 0.757 ms, ResNet-50 1.76 ->
- * 1.69 ms); a step replayed as a CUDA graph gets slower when layout passes sit between the
- * tensor-core kernels (NCHW layers: 0.605 -> 0.696 ms; 0.665 ms when the tensor-core kernel
- * releases its dependents only after its last MMA) and 2 % faster when it consists of tensor-core
- * kernels only (channels-last chain: 0.514 -> 0.504 ms), which is why it is off unless asked for
- * (`python bench.py --launch-overlap` repeats the measurement).  Applies to all later launches
- * of this process.
+ * Launch overlap.  The persistent tensor-core kernels are always launched with the programmatic
+ * stream serialization attribute: such a kernel may be scheduled while the previous kernel of
+ * the stream is still draining, and waits, before it touches global memory, until that kernel
+ * has completed; so its set-up overlaps the tail of the kernel before it, and where one
+ * tensor-core kernel follows another its CTAs start as the previous kernel's leave.  Results are
+ * the same either way.  Measured on B200, steps replayed as CUDA graphs: ResNet-50 channels-last
+ * 1.065 -> 1.018 ms, MobileNet channels-last 0.332 -> 0.321 ms, NCHW steps unchanged.
+ * With enabled != 0 EVERY kernel of the library is launched that way (off by default): with
+ * eager launches the gap between dependent kernels shrinks (a VGG-16 step 0.776 -> 0.757 ms,
+ * ResNet-50 1.76 -> 1.69 ms), but a step replayed as a CUDA graph gets slower when layout passes
+ * sit between the tensor-core kernels (NCHW VGG-16 layers: 0.605 -> 0.696 ms), which is why it
+ * is off unless asked for (`python bench.py --launch-overlap` repeats the measurement).
+ * Applies to all later launches of this process.
  * Always returns HGC_OK.
  */
 int hgc_set_launch_overlap(int enabled);

@@ -50,8 +50,8 @@ bool launch_overlap_enabled();
 void set_launch_overlap(bool on);
 
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
-                                 Args... args) {
+inline cudaError_t launch_kernel_attr(bool overlap, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                      cudaStream_t stream, Args... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
@@ -61,8 +61,24 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = launch_overlap_enabled() ? 1 : 0;
+  cfg.numAttrs = overlap ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                 Args... args) {
+  return launch_kernel_attr(launch_overlap_enabled(), kernel, grid, block, smem, stream, args...);
+}
+// The persistent tensor-core kernel is always launched with the attribute: its set-up (barriers,
+// tensor memory) then overlaps the tail of the kernel before it, and where one tensor-core kernel
+// follows another (channels-last chains, 1x1 layers that read x in place) its CTAs start as the
+// previous kernel's CTAs leave.  Measured, steps replayed as CUDA graphs: ResNet-50 channels-last
+// 1.065 -> 1.018 ms, MobileNet channels-last 0.332 -> 0.321 ms, NCHW steps unchanged (VGG-16
+// 0.596, ResNet-50 1.295 -> 1.287, MobileNet 0.326 ms).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                            cudaStream_t stream, Args... args) {
+  return launch_kernel_attr(true, kernel, grid, block, smem, stream, args...);
 }
 
 // The same with the cooperative attribute when `cooperative` is set: the launch waits until every

@@ -2819,7 +2819,7 @@ cudaError_t launch_igemm(const ConvGeom& g_layer, IgemmPlan& p, void* ws, const 
     err = cudaFuncSetAttribute(igemm_kernel<KBV, HALOV, EWV, EPIV, SPLITV>,                                \
                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);            \
     if (err == cudaSuccess)                                                                                \
-      err = launch_kernel(igemm_kernel<KBV, HALOV, EWV, EPIV, SPLITV>, grid, dim3(64 + 32 * EWV),          \
+      err = launch_kernel_overlapped(igemm_kernel<KBV, HALOV, EWV, EPIV, SPLITV>, grid, dim3(64 + 32 * EWV), \
                           p.smem_bytes, stream, p.tmA, p.tmB, p.tmY, p.tmYr, a, bias, y, partials, status); \
   } while (0)
   // depthwise + pointwise block: its own instantiations (8 epilogue + 8 depthwise warps)
@@ -2828,7 +2828,7 @@ cudaError_t launch_igemm(const ConvGeom& g_layer, IgemmPlan& p, void* ws, const 
     err = cudaFuncSetAttribute(igemm_kernel<KBV, true, 8, EPIV, false, false, false, false, true>,         \
                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);            \
     if (err == cudaSuccess)                                                                                \
-      err = launch_kernel(igemm_kernel<KBV, true, 8, EPIV, false, false, false, false, true>, grid,        \
+      err = launch_kernel_overlapped(igemm_kernel<KBV, true, 8, EPIV, false, false, false, false, true>, grid, \
                           dim3(64 + 32 * 8 + 32 * kDwWarps), p.smem_bytes, stream, p.tmA, p.tmB, p.tmY,    \
                           p.tmYr, a, bias, y, partials, status);                                           \
   } while (0)
