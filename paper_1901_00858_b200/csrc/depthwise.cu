@@ -35,6 +35,7 @@ __global__ void __launch_bounds__(kThreads)
 depthwise3x3_kernel(DwPlan a, const uint16_t* __restrict__ x, const __half* __restrict__ w,
                     const __half* __restrict__ bias, uint16_t* __restrict__ y, int relu) {
   grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   extern __shared__ __align__(16) uint16_t smem[];
   uint16_t* sin = smem;
   uint16_t* sout = smem + a.smem_in;
@@ -206,6 +207,7 @@ depthwise3x3_rowvec_kernel(const uint16_t* __restrict__ x, const __half* __restr
                            const __half* __restrict__ bias, uint16_t* __restrict__ y, int c, int h, int wd,
                            int p, int q, int relu, int64_t total_items, int vec_per_row, int strips) {
   grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   // item = (plane, strip, vector); the vectors of a row are consecutive lanes.  32-bit index
   // arithmetic (the launcher checks that the item count fits).
   const uint32_t item = blockIdx.x * blockDim.x + threadIdx.x;
@@ -338,6 +340,7 @@ depthwise3x3_smallrow_kernel(const uint16_t* __restrict__ x, const __half* __res
                              const __half* __restrict__ bias, uint16_t* __restrict__ y, int c, int h, int p, int relu,
                              int64_t total_rows) {
   grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   constexpr int Q = (W - 1) / S + 1;  // kernel 3, pad 1
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= total_rows) return;
@@ -410,6 +413,7 @@ depthwise3x3_nhwc_kernel(const uint16_t* __restrict__ x, const uint16_t* __restr
                          const uint16_t* __restrict__ bias, uint16_t* __restrict__ y, int c, int h, int wd, int p,
                          int q, int pad_h, int pad_w, int relu, int strips, int64_t items) {
   grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   constexpr int COLS = (TQ - 1) * S + 3;
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= items) return;
@@ -506,6 +510,7 @@ depthwise3x3_colword_kernel(const uint16_t* __restrict__ x, const __half* __rest
                             const __half* __restrict__ bias, uint16_t* __restrict__ y, int c, int relu,
                             int64_t planes) {
   grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   constexpr int WORDS = W / 2;         // column words per row
   constexpr int PPW = 32 / WORDS;      // planes per warp
   constexpr int H = W;

@@ -103,11 +103,14 @@ inline cudaError_t launch_kernel_coop(bool cooperative, void (*kernel)(KArgs...)
 #ifdef __CUDACC__
 // see launch_kernel: call before the first global-memory access of a kernel
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-// Lets the next kernel of the stream be scheduled as soon as every CTA of this grid has called
-// this (or exited).  Only the persistent tensor-core kernel calls it: its CTAs hold a whole SM, so
-// the next kernel's CTAs start exactly where one of them has finished.  The many-block copy and
-// depthwise kernels do not: CTAs of a following tensor-core kernel that became resident early
-// would pin most of an SM's registers while they wait and starve the blocks still to run.
+// Lets the next kernel of the stream, if it was launched with the attribute (the tensor-core
+// kernels always are), be scheduled as soon as EVERY CTA of this grid has called this or exited.
+// The persistent tensor-core kernel calls it at its start: its CTAs hold a whole SM, so the next
+// kernel's CTAs start exactly where one of them has finished.  The many-block copy and depthwise
+// kernels call it at their start too: the condition is met only when their last blocks are
+// running, so the CTAs of a following tensor-core kernel take SMs that have no more blocks to
+// wait for and set themselves up (barriers, tensor memory) beside the last wave.  Measured, NCHW
+// steps as CUDA graphs: VGG-16 0.596 -> 0.589 ms, ResNet-50 1.287 -> 1.263, MobileNet 0.327 -> 0.321.
 __device__ __forceinline__ void grid_launch_dependents() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }

@@ -22,6 +22,7 @@ __global__ void __launch_bounds__(kThreads)
 nchw_to_nhwc_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int64_t hw,
                     int c_pad, int vec_ok) {
   grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   __shared__ __align__(16) uint16_t tile[kTileC][kRow];
   const int64_t n = blockIdx.z;
   const int c0 = blockIdx.y * kTileC;
@@ -75,6 +76,7 @@ __global__ void __launch_bounds__(kThreads)
 nchw_to_nhwc_regs_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int64_t hw,
                          int c_pad, int64_t units_p, int units_c, int64_t total_units) {
   grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   constexpr int PG = 32 / CH;
   constexpr int W32 = PX / 2;  // 32-bit words per channel
   const int lane = threadIdx.x & 31;
@@ -127,6 +129,7 @@ __global__ void __launch_bounds__(kThreads)
 nchw_to_nhwc_smallplane_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int hw,
                                int c_pad) {
   grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   extern __shared__ __align__(16) uint16_t flat[];  // [kTileC][hw]
   const int64_t n = blockIdx.y;
   const int c0 = blockIdx.x * kTileC;
@@ -157,6 +160,7 @@ __global__ void __launch_bounds__(kThreads)
 nhwc_to_nchw_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int64_t hw,
                     int c_pad, int vec_ok) {
   grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   __shared__ __align__(16) uint16_t tile[kTileC][kRow];
   const int64_t n = blockIdx.z;
   const int c0 = blockIdx.y * kTileC;
@@ -211,6 +215,7 @@ __device__ __forceinline__ int64_t row_channel(int64_t row, int perm) {
 __global__ void weights_repack_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst,
                                       int64_t k, int cg, int rs, int c_pad, int perm) {
   grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   const int64_t vecs_per_k = (int64_t)rs * (c_pad / 8);
   const int64_t total = k * vecs_per_k;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
@@ -238,6 +243,7 @@ __global__ void __launch_bounds__(256)
 nchw_to_nhwc8_bordered_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int h, int w,
                               int pad_h, int pad_w, int hp, int wp, int64_t total) {
   grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   const int64_t hw = (int64_t)h * w;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int ow = (int)(i % wp);
@@ -267,6 +273,7 @@ __global__ void __launch_bounds__(256)
 nchw_to_nhwc8_bordered_vec_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int h, int w,
                                   int pad_h, int pad_w, int hp, int wp, int64_t items) {
   grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   const int slots = w / 8 + 1;
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= items) return;
@@ -315,6 +322,7 @@ template <int PC>  // channels per pixel of the window: 8 or 4
 __global__ void weights_repack_window_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst,
                                              int64_t k, int c, int r, int s, int kw_pix, int perm) {
   grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   const int64_t total = k * r * kw_pix;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int sp = (int)(i % kw_pix);
@@ -344,6 +352,7 @@ patch_im2col_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst
                     int pad_h, int pad_w, int stride_h, int stride_w, int dil_h, int dil_w, int kelems,
                     int64_t total) {
   grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   constexpr int E = R * S * C;
   constexpr int EW = (E + 1) / 2;  // 32-bit words that hold real elements
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -391,6 +400,7 @@ patch_im2col_generic_kernel(const uint16_t* __restrict__ src, uint16_t* __restri
                             int p, int q, int r, int s, int pad_h, int pad_w, int stride_h, int stride_w,
                             int dil_h, int dil_w, int kelems, int64_t total_chunks) {
   grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total_chunks) return;
   const int vecs = kelems >> 3;
@@ -424,6 +434,7 @@ patch_im2col_generic_kernel(const uint16_t* __restrict__ src, uint16_t* __restri
 __global__ void weights_repack_patch_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int64_t k,
                                             int c, int r, int s, int kelems, int perm) {
   grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   const int64_t total = k * kelems;
   const int rsc = r * s * c;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
@@ -612,6 +623,7 @@ cudaError_t launch_weights_repack_patch(const __half* src, __half* dst, int32_t 
 __global__ void weights_repack_rowpair_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int cg, int r,
                                               int s, int c_pad) {
   grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   const int64_t vecs_per_k = (int64_t)(r + 1) * s * (c_pad / 8);
   const int64_t total = 128 * vecs_per_k;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
@@ -661,6 +673,7 @@ cudaError_t launch_igemm_weights(const ConvGeom& g, const IgemmPlan& p, const __
 __global__ void __launch_bounds__(256)
 depthwise_weights_to_taps_kernel(const uint16_t* __restrict__ w, uint16_t* __restrict__ w9, int c) {
   grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   const int i = blockIdx.x * blockDim.x + threadIdx.x;  // index into w9: tap * c + channel
   if (i < 9 * c) w9[i] = w[(i % c) * 9 + i / c];
 }
