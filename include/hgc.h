@@ -386,6 +386,26 @@ int hgc_debug_set_wait_limit_ns(uint64_t ns);
 int hgc_debug_drop_copies(int32_t index);
 
 /*
+ * Checked build.  The library can be built with -DHGC_DEBUG (libhgc_debug.so beside libhgc.so,
+ * `python -m paper_1901_00858_b200.build` builds both).  In that build every global-memory access
+ * that a kernel addresses by hand (the layout, depthwise and direct kernels; the copy and
+ * channels-last epilogues, bias loads, partial sums and hand-overs of the tensor-core kernel)
+ * is tested against the byte ranges of the call in progress: x, w, bias, y and the workspace, as
+ * the descriptor's shapes give them (the copy engine's accesses are clipped to their tensor maps
+ * by the hardware).  An access outside is recorded and SKIPPED: nothing faults.
+ * hgc_debug_checked_build: 1 in the checked build, else 0.
+ * hgc_debug_violations: synchronises the device, then writes the number of accesses outside every
+ * range since the last call (0 in the ordinary build) and, of the first one, the source line of
+ * its test, its address and size (host pointers; all but count may be NULL); clears the record.
+ * hgc_debug_shrink_ranges: test hook: the ranges registered by later calls end `bytes` early, so
+ * that the last accesses of correct kernels count as violations (and are skipped) although the
+ * memory is there; 0 switches it off.  Errors: HGC_INVALID_ARG, HGC_CUDA_ERROR.
+ */
+int hgc_debug_checked_build(void);
+int hgc_debug_violations(int32_t* count, int32_t* line, uint64_t* addr, uint64_t* bytes);
+int hgc_debug_shrink_ranges(int64_t bytes);
+
+/*
  * Launch overlap.  The persistent tensor-core kernels are always launched with the programmatic
  * stream serialization attribute: such a kernel may be scheduled while the previous kernel of
  * the stream is still draining, and waits, before it touches global memory, until that kernel

@@ -12,6 +12,7 @@ from typing import Optional
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libhgc.so")
+DEBUG_LIB_PATH = os.path.join(HERE, "libhgc_debug.so")   # the checked build (-DHGC_DEBUG)
 
 HGC_OK, HGC_INVALID_ARG, HGC_UNSUPPORTED, HGC_BAD_ALIGNMENT, HGC_NO_WORKSPACE, HGC_CUDA_ERROR, \
     HGC_DEVICE_TIMEOUT = range(7)
@@ -85,6 +86,8 @@ def lib() -> ctypes.CDLL:
         L.hgc_dwpw_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_int, ctypes.c_int, vp]
         L.hgc_debug_set_wait_limit_ns.argtypes = [ctypes.c_uint64]
         L.hgc_debug_drop_copies.argtypes = [i32]
+        L.hgc_debug_violations.argtypes = [i32p, i32p, ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64)]
+        L.hgc_debug_shrink_ranges.argtypes = [ctypes.c_int64]
         L.hgc_status_string.argtypes = [ctypes.c_int]
         L.hgc_status_string.restype = ctypes.c_char_p
         for name in ("hgc_conv_desc_create", "hgc_conv_desc_destroy", "hgc_conv_forward",
@@ -95,7 +98,8 @@ def lib() -> ctypes.CDLL:
                      "hgc_kernel_launch_count", "hgc_inner_product_desc_create", "hgc_cast_f32_to_f16",
                      "hgc_set_launch_overlap", "hgc_batchnorm_forward", "hgc_bn_fold",
                      "hgc_debug_set_wait_limit_ns", "hgc_debug_drop_copies", "hgc_dwpw_desc_create",
-                     "hgc_dwpw_set_weights", "hgc_dwpw_forward"):
+                     "hgc_dwpw_set_weights", "hgc_dwpw_forward", "hgc_debug_checked_build", "hgc_debug_violations",
+                     "hgc_debug_shrink_ranges"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -328,6 +332,35 @@ def debug_set_wait_limit_ns(ns: int) -> None:
 def debug_drop_copies(index: int) -> None:
     """hgc_debug_drop_copies: the first CTA of later launches never issues its index-th copy (-1: off)."""
     _check(lib().hgc_debug_drop_copies(int(index)), "hgc_debug_drop_copies")
+
+
+def use_checked_build() -> None:
+    """Makes this process load libhgc_debug.so (the -DHGC_DEBUG build) instead of libhgc.so; call it
+    before anything else touches the library."""
+    global LIB_PATH
+    if _lib is not None:
+        raise RuntimeError("the library is loaded already")
+    LIB_PATH = DEBUG_LIB_PATH
+
+
+def debug_checked_build() -> bool:
+    """hgc_debug_checked_build: True when the loaded library tests its hand-addressed accesses."""
+    return bool(lib().hgc_debug_checked_build())
+
+
+def debug_violations() -> dict:
+    """hgc_debug_violations: accesses outside the call's tensors since the last call, and the first
+    one's source line, address and size; clears the record (synchronises the device)."""
+    count, line = ctypes.c_int32(), ctypes.c_int32()
+    addr, nbytes = ctypes.c_uint64(), ctypes.c_uint64()
+    _check(lib().hgc_debug_violations(ctypes.byref(count), ctypes.byref(line), ctypes.byref(addr), ctypes.byref(nbytes)),
+           "hgc_debug_violations")
+    return {"count": count.value, "line": line.value, "addr": addr.value, "bytes": nbytes.value}
+
+
+def debug_shrink_ranges(nbytes: int) -> None:
+    """hgc_debug_shrink_ranges: later calls register their tensors `nbytes` short (test hook; 0 = off)."""
+    _check(lib().hgc_debug_shrink_ranges(int(nbytes)), "hgc_debug_shrink_ranges")
 
 
 def kernel_launch_count() -> int:

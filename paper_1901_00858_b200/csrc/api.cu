@@ -11,6 +11,21 @@ void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 static std::atomic<int> g_debug_drop{-1};
 int debug_drop_copies() { return g_debug_drop.load(std::memory_order_relaxed); }
 static std::atomic<bool> g_launch_overlap{false};
+static std::atomic<long long> g_debug_shrink{0};
+void debug_add_range(DebugRanges* r, const void* p, size_t bytes) {
+  if (p == nullptr || bytes == 0 || r->count >= DebugRanges::kMax) return;
+  const uint64_t cut = (uint64_t)g_debug_shrink.load(std::memory_order_relaxed);
+  r->lo[r->count] = (uint64_t)(uintptr_t)p;
+  r->hi[r->count] = r->lo[r->count] + (bytes > cut ? bytes - cut : 0);
+  ++r->count;
+}
+void debug_set_call_ranges(const DebugRanges& r, cudaStream_t stream) {
+  if (!kCheckedBuild) return;
+  layout_debug_set_ranges(r, stream);
+  igemm_debug_set_ranges(r, stream);
+  depthwise_debug_set_ranges(r, stream);
+  direct_debug_set_ranges(r, stream);
+}
 bool launch_overlap_enabled() { return g_launch_overlap.load(std::memory_order_relaxed); }
 void set_launch_overlap(bool on) { g_launch_overlap.store(on, std::memory_order_relaxed); }
 }  // namespace hgc
@@ -68,9 +83,23 @@ HostStaging host_staging(const hgc_conv_desc* d) {
   return s;
 }
 
+// Checked build: the byte ranges that the kernels of one forward call may touch.
+void debug_register_ranges(const hgc::ConvGeom& g, const void* x, const void* w, const void* bias, const void* y,
+                           const void* ws, size_t ws_bytes, cudaStream_t stream) {
+  if (!hgc::kCheckedBuild) return;
+  hgc::DebugRanges r{};
+  hgc::debug_add_range(&r, x, (size_t)g.n * g.c * g.h * g.w * 2);
+  hgc::debug_add_range(&r, w, (size_t)g.k * g.cg * g.r * g.s * 2);
+  hgc::debug_add_range(&r, bias, (size_t)g.k * 2);
+  hgc::debug_add_range(&r, y, (size_t)g.n * g.k * g.p * g.q * 2);
+  hgc::debug_add_range(&r, ws, ws_bytes);
+  hgc::debug_set_call_ranges(r, stream);
+}
+
 int forward_impl(hgc_conv_desc* d, const void* x, const void* w, const void* bias, void* y,
                  int relu, cudaStream_t stream) {
   const hgc::ConvGeom& g = d->geom;
+  debug_register_ranges(g, x, w, bias, y, d->ws, d->ws_needed, stream);
   const __half* xh = static_cast<const __half*>(x);
   const __half* wh = static_cast<const __half*>(w);
   const __half* bh = static_cast<const __half*>(bias);
@@ -427,6 +456,18 @@ int hgc_dwpw_forward(hgc_conv_desc* d, const void* x, const void* w_dw, const vo
   if (d->ws == nullptr || d->ws_bytes < d->ws_needed) return HGC_NO_WORKSPACE;
   char* ws = static_cast<char*>(d->ws);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (hgc::kCheckedBuild) {
+    const hgc::ConvGeom& g = d->geom;  // the pointwise layer on the depthwise layer's output plane
+    hgc::DebugRanges r{};
+    hgc::debug_add_range(&r, x, (size_t)g.n * g.c * d->dw_h * d->dw_w * 2);
+    hgc::debug_add_range(&r, w_dw, (size_t)g.c * 9 * 2);
+    hgc::debug_add_range(&r, bias_dw, (size_t)g.c * 2);
+    hgc::debug_add_range(&r, w_pw, (size_t)g.k * g.c * 2);
+    hgc::debug_add_range(&r, bias_pw, (size_t)g.k * 2);
+    hgc::debug_add_range(&r, y, (size_t)g.n * g.k * g.p * g.q * 2);
+    hgc::debug_add_range(&r, ws, d->ws_needed);
+    hgc::debug_set_call_ranges(r, st);
+  }
   if (d->registered_w != w_pw || d->registered_w_dw != w_dw) {  // weights not prepared in advance: re-lay them out now
     if (hgc::launch_igemm_weights(d->geom, d->igemm, static_cast<const __half*>(w_pw),
                                   reinterpret_cast<__half*>(ws + d->igemm.ws_w_off), st) != cudaSuccess)
@@ -504,6 +545,35 @@ int hgc_debug_set_wait_limit_ns(uint64_t ns) {
 
 int hgc_debug_drop_copies(int32_t index) {
   hgc::g_debug_drop.store(index < 0 ? -1 : index, std::memory_order_relaxed);
+  return HGC_OK;
+}
+
+int hgc_debug_checked_build(void) { return hgc::kCheckedBuild ? 1 : 0; }
+
+int hgc_debug_violations(int32_t* count, int32_t* line, uint64_t* addr, uint64_t* bytes) {
+  if (count == nullptr) return HGC_INVALID_ARG;
+  if (cudaDeviceSynchronize() != cudaSuccess) return HGC_CUDA_ERROR;
+  hgc::DebugViolation v[4];
+  hgc::layout_debug_read(&v[0]);
+  hgc::igemm_debug_read(&v[1]);
+  hgc::depthwise_debug_read(&v[2]);
+  hgc::direct_debug_read(&v[3]);
+  int32_t total = 0;
+  const hgc::DebugViolation* first = nullptr;
+  for (const hgc::DebugViolation& e : v) {
+    total += e.count;
+    if (e.count > 0 && first == nullptr) first = &e;
+  }
+  *count = total;
+  if (line != nullptr) *line = first != nullptr ? first->line : 0;
+  if (addr != nullptr) *addr = first != nullptr ? first->addr : 0;
+  if (bytes != nullptr) *bytes = first != nullptr ? first->bytes : 0;
+  return HGC_OK;
+}
+
+int hgc_debug_shrink_ranges(int64_t bytes) {
+  if (bytes < 0) return HGC_INVALID_ARG;
+  hgc::g_debug_shrink.store(bytes, std::memory_order_relaxed);
   return HGC_OK;
 }
 

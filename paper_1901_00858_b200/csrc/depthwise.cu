@@ -13,6 +13,7 @@
 #include "hgc_internal.h"
 
 namespace hgc {
+HGC_DEBUG_STATE(depthwise)
 namespace {
 
 constexpr int kThreads = 256;
@@ -80,7 +81,7 @@ depthwise3x3_kernel(DwPlan a, const uint16_t* __restrict__ x, const __half* __re
       const int64_t ge = gbase + (int64_t)v * 8;
       uint4 val;
       if (ge + 8 <= a.x_elems) {
-        val = __ldg(reinterpret_cast<const uint4*>(x + ge));
+        HGC_CHECKED_LOAD(val, reinterpret_cast<const uint4*>(x + ge), __ldg(reinterpret_cast<const uint4*>(x + ge)));
       } else {
         uint32_t o[4] = {0, 0, 0, 0};
         for (int j = 0; j < 8; ++j)
@@ -182,10 +183,10 @@ depthwise3x3_kernel(DwPlan a, const uint16_t* __restrict__ x, const __half* __re
     for (int v = threadIdx.x; v < nvec; v += kThreads) {
       const int e = v * 8;
       if (e >= lo && e + 8 <= hi) {
-        *reinterpret_cast<uint4*>(y + gbase + e) = *reinterpret_cast<const uint4*>(sout + e);
+        HGC_CHECKED_STORE(reinterpret_cast<uint4*>(y + gbase + e), *reinterpret_cast<uint4*>(y + gbase + e) = *reinterpret_cast<const uint4*>(sout + e));
       } else {
         for (int j = 0; j < 8; ++j)
-          if (e + j >= lo && e + j < hi) y[gbase + e + j] = sout[e + j];
+          if (e + j >= lo && e + j < hi) HGC_CHECKED_STORE(y + gbase + e + j, y[gbase + e + j] = sout[e + j]);
       }
     }
   }
@@ -250,8 +251,8 @@ depthwise3x3_rowvec_kernel(const uint16_t* __restrict__ x, const __half* __restr
     if (S == 2) rb[i] = make_uint4(0, 0, 0, 0);
     if (rv) {
       const uint4* src = reinterpret_cast<const uint4*>(xp + (int64_t)ih * wd) + (int64_t)v * S;
-      ra[i] = __ldg(src);
-      if (S == 2 && (v * 2 + 1) * 8 < wd) rb[i] = __ldg(src + 1);  // the row may end after the first vector
+      HGC_CHECKED_LOAD(ra[i], src, __ldg(src));
+      if (S == 2 && (v * 2 + 1) * 8 < wd) HGC_CHECKED_LOAD(rb[i], src + 1, __ldg(src + 1));  // the row may end after the first vector
     }
     // halo pixels that no neighbouring lane holds (warp boundary inside a row)
     left[i] = 0;
@@ -318,7 +319,7 @@ depthwise3x3_rowvec_kernel(const uint16_t* __restrict__ x, const __half* __restr
     if (live && pr < p) {
       uint16_t* dst = yp + (int64_t)pr * q + (int64_t)v * 8;
       if ((q & 7) == 0) {
-        *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
+        HGC_CHECKED_STORE(reinterpret_cast<uint4*>(dst), *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]));
       } else {  // q % 8 == 4: rows are 8-byte aligned and the last vector of a row is half full
         reinterpret_cast<uint2*>(dst)[0] = make_uint2(o[0], o[1]);
         if (v * 8 + 8 <= q) reinterpret_cast<uint2*>(dst)[1] = make_uint2(o[2], o[3]);
@@ -363,12 +364,17 @@ depthwise3x3_smallrow_kernel(const uint16_t* __restrict__ x, const __half* __res
     if constexpr ((W & 1) == 0) {
 #pragma unroll
       for (int e = 0; e < W / 2; ++e) {
-        const uint32_t v = rv ? __ldg(reinterpret_cast<const uint32_t*>(xr) + e) : 0u;
+        uint32_t v = 0u;
+        if (rv) HGC_CHECKED_LOAD(v, reinterpret_cast<const uint32_t*>(xr) + e, __ldg(reinterpret_cast<const uint32_t*>(xr) + e));
         asm("mov.b32 {%0, %1}, %2;" : "=h"(in[rr][1 + 2 * e]), "=h"(in[rr][2 + 2 * e]) : "r"(v));
       }
     } else {
 #pragma unroll
-      for (int e = 0; e < W; ++e) in[rr][1 + e] = rv ? __ldg(xr + e) : (uint16_t)0;
+      for (int e = 0; e < W; ++e) {
+        uint16_t v = 0;
+        if (rv) HGC_CHECKED_LOAD(v, xr + e, __ldg(xr + e));
+        in[rr][1 + e] = v;
+      }
     }
   }
   float f[Q + 1];
@@ -394,8 +400,8 @@ depthwise3x3_smallrow_kernel(const uint16_t* __restrict__ x, const __half* __res
     if constexpr ((Q & 1) == 0) {
       reinterpret_cast<uint32_t*>(yr)[j >> 1] = o;
     } else {
-      yr[j] = (uint16_t)(o & 0xffffu);
-      if (j + 1 < Q) yr[j + 1] = (uint16_t)(o >> 16);
+      HGC_CHECKED_STORE(yr + j, yr[j] = (uint16_t)(o & 0xffffu));
+      if (j + 1 < Q) HGC_CHECKED_STORE(yr + j + 1, yr[j + 1] = (uint16_t)(o >> 16));
     }
   }
 }
@@ -437,8 +443,9 @@ depthwise3x3_nhwc_kernel(const uint16_t* __restrict__ x, const uint16_t* __restr
     for (int cc = 0; cc < COLS; ++cc) {
       const int iw = iw0 + cc;
       const bool v = rv && iw >= 0 && iw < wd;
-      in[rr][cc] = v ? __ldg(reinterpret_cast<const uint4*>(x + ((img * h + ih) * wd + iw) * c) + oc)
-                     : make_uint4(0u, 0u, 0u, 0u);
+      in[rr][cc] = make_uint4(0u, 0u, 0u, 0u);
+      if (v) HGC_CHECKED_LOAD(in[rr][cc], reinterpret_cast<const uint4*>(x + ((img * h + ih) * wd + iw) * c) + oc,
+                              __ldg(reinterpret_cast<const uint4*>(x + ((img * h + ih) * wd + iw) * c) + oc));
     }
   }
   // weights w[ch][9] of the 8 channels: 144 contiguous bytes, element ch*9 + tap
@@ -494,7 +501,8 @@ depthwise3x3_nhwc_kernel(const uint16_t* __restrict__ x, const uint16_t* __restr
       else
         asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(ov[j]) : "f"(acc[2 * j + 1]), "f"(acc[2 * j]));
     }
-    reinterpret_cast<uint4*>(y + ((img * p + pr) * q + q0 + o) * c)[oc] = make_uint4(ov[0], ov[1], ov[2], ov[3]);
+    HGC_CHECKED_STORE(reinterpret_cast<uint4*>(y + ((img * p + pr) * q + q0 + o) * c) + oc,
+                      reinterpret_cast<uint4*>(y + ((img * p + pr) * q + q0 + o) * c)[oc] = make_uint4(ov[0], ov[1], ov[2], ov[3]));
   }
 }
 
@@ -527,7 +535,10 @@ depthwise3x3_colword_kernel(const uint16_t* __restrict__ x, const __half* __rest
   const uint32_t* xp = reinterpret_cast<const uint32_t*>(x) + (live ? plane : 0) * (H * WORDS) + e;
   uint32_t v[H];
 #pragma unroll
-  for (int r = 0; r < H; ++r) v[r] = live ? __ldg(xp + r * WORDS) : 0u;
+  for (int r = 0; r < H; ++r) {
+    v[r] = 0u;
+    if (live) HGC_CHECKED_LOAD(v[r], xp + r * WORDS, __ldg(xp + r * WORDS));
+  }
   // per row: (pixel left of the word, pixel right of it)
   uint32_t lr[H];
 #pragma unroll
@@ -585,7 +596,7 @@ depthwise3x3_colword_kernel(const uint16_t* __restrict__ x, const __half* __rest
       asm("cvt.rn.relu.f16x2.f32 %0, %1, %2;" : "=r"(o) : "f"(a1), "f"(a0));
     else
       asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(o) : "f"(a1), "f"(a0));
-    if (live) yp[p * WORDS] = o;
+    if (live) HGC_CHECKED_STORE(yp + p * WORDS, yp[p * WORDS] = o);
   }
 }
 

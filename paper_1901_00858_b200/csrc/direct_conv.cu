@@ -9,6 +9,7 @@
 #include "hgc_internal.h"
 
 namespace hgc {
+HGC_DEBUG_STATE(direct)
 namespace {
 
 constexpr int kThreads = 128;
@@ -66,7 +67,9 @@ direct_conv_kernel(ConvGeom g, const __half* __restrict__ x, const __half* __res
         const int ih = ih0 + r * g.dil_h;
         const int iw = iw0 + s * g.dil_w;
         if (ih >= 0 && ih < g.h && iw >= 0 && iw < g.w) {
-          const float xv = __half2float(__ldg(xg + (int64_t)cc * plane + (int64_t)ih * g.w + iw));
+          float xv = 0.f;
+          if (HGC_ADDR_OK(xg + (int64_t)cc * plane + (int64_t)ih * g.w + iw, sizeof(__half)))
+            xv = __half2float(__ldg(xg + (int64_t)cc * plane + (int64_t)ih * g.w + iw));
 #pragma unroll
           for (int i = 0; i < KT; ++i) acc[i] = fmaf(xv, ws[i][t], acc[i]);
         }
@@ -90,7 +93,7 @@ direct_conv_kernel(ConvGeom g, const __half* __restrict__ x, const __half* __res
         float v = acc[i];
         if (bias != nullptr) v += __half2float(bias[k]);
         if (relu) v = fmaxf(v, 0.f);
-        y[((int64_t)n * g.k + k) * pq + pix] = __float2half_rn(v);
+        if (HGC_ADDR_OK(y + ((int64_t)n * g.k + k) * pq + pix, sizeof(__half))) y[((int64_t)n * g.k + k) * pq + pix] = __float2half_rn(v);
       }
     }
   }

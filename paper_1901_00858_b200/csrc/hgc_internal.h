@@ -116,6 +116,97 @@ __device__ __forceinline__ void grid_launch_dependents() {
 }
 #endif
 
+// ---------------------------------------------------------------------------------------------
+// Checked build (-DHGC_DEBUG, libhgc_debug.so): every global-memory access that a kernel of this
+// library addresses by hand (everything but the copy engine's tensor-map accesses, which the
+// hardware clips to the map's bounds) goes through dbg_load / dbg_store below, which test the
+// address range against the tensors of the call in progress (x, w, bias, y, workspace; set by the
+// entry points before they launch) and, when it lies outside, record it and SKIP the access:
+// nothing faults, the caller reads the record (hgc_debug_violations).  In the ordinary build
+// the helpers are the plain accesses.
+struct DebugRanges {
+  static constexpr int kMax = 8;
+  uint64_t lo[kMax], hi[kMax];  // valid bytes [lo, hi)
+  int32_t count;
+};
+struct DebugViolation {
+  int32_t count;  // accesses outside every range since the record was last read
+  int32_t line;   // source line of the first one
+  uint64_t addr, bytes;
+};
+#ifdef HGC_DEBUG
+constexpr bool kCheckedBuild = true;
+#else
+constexpr bool kCheckedBuild = false;
+#endif
+// all translation units at once (api.cu); a table without entries switches the test off
+void debug_set_call_ranges(const DebugRanges& r, cudaStream_t stream);
+// appends [p, p + bytes) shortened by the test hook's cut (hgc_debug_shrink_ranges)
+void debug_add_range(DebugRanges* r, const void* p, size_t bytes);
+// per translation unit: sets the ranges for the launches that follow on `stream`; reads and clears the record
+void layout_debug_set_ranges(const DebugRanges& r, cudaStream_t stream);
+void igemm_debug_set_ranges(const DebugRanges& r, cudaStream_t stream);
+void depthwise_debug_set_ranges(const DebugRanges& r, cudaStream_t stream);
+void direct_debug_set_ranges(const DebugRanges& r, cudaStream_t stream);
+void layout_debug_read(DebugViolation* v);
+void igemm_debug_read(DebugViolation* v);
+void depthwise_debug_read(DebugViolation* v);
+void direct_debug_read(DebugViolation* v);
+
+#ifdef __CUDACC__
+// Defines the translation unit's range table and record, the device-side test and the two host
+// functions declared above (NAME = layout, igemm, depthwise, direct).
+#ifdef HGC_DEBUG
+#define HGC_DEBUG_STATE(NAME)                                                                              \
+  namespace {                                                                                              \
+  __device__ DebugRanges g_dbg_ranges;                                                                     \
+  __device__ DebugViolation g_dbg_violation;                                                               \
+  __device__ __noinline__ bool dbg_addr_ok(const void* p, size_t bytes, int line) {                        \
+    const uint64_t a = (uint64_t)(uintptr_t)p;                                                             \
+    if (g_dbg_ranges.count == 0) return true;                                                              \
+    for (int i = 0; i < g_dbg_ranges.count; ++i)                                                           \
+      if (a >= g_dbg_ranges.lo[i] && a + bytes <= g_dbg_ranges.hi[i]) return true;                         \
+    if (atomicAdd(&g_dbg_violation.count, 1) == 0) {                                                       \
+      g_dbg_violation.line = line;                                                                         \
+      g_dbg_violation.addr = a;                                                                            \
+      g_dbg_violation.bytes = bytes;                                                                       \
+    }                                                                                                      \
+    return false;                                                                                          \
+  }                                                                                                        \
+  }                                                                                                        \
+  void NAME##_debug_set_ranges(const DebugRanges& r, cudaStream_t stream) {                                \
+    cudaMemcpyToSymbolAsync(g_dbg_ranges, &r, sizeof(DebugRanges), 0, cudaMemcpyHostToDevice, stream);     \
+  }                                                                                                        \
+  void NAME##_debug_read(DebugViolation* v) {                                                              \
+    cudaMemcpyFromSymbol(v, g_dbg_violation, sizeof(DebugViolation));                                      \
+    const DebugViolation zero{};                                                                           \
+    cudaMemcpyToSymbol(g_dbg_violation, &zero, sizeof(DebugViolation));                                    \
+  }
+#define HGC_ADDR_OK(p, bytes) dbg_addr_ok((p), (bytes), __LINE__)
+#else
+#define HGC_DEBUG_STATE(NAME)                                                       \
+  void NAME##_debug_set_ranges(const DebugRanges&, cudaStream_t) {}                 \
+  void NAME##_debug_read(DebugViolation* v) { *v = DebugViolation{}; }
+#define HGC_ADDR_OK(p, bytes) true
+#endif
+// checked accesses (the plain access in the ordinary build): PTR is the typed pointer that is
+// accessed, ACCESS the expression that reads it / STMT the statement that writes it
+#define HGC_CHECKED_LOAD(VAR, PTR, ACCESS)              \
+  do {                                                  \
+    if (HGC_ADDR_OK((PTR), sizeof(*(PTR)))) {           \
+      VAR = ACCESS;                                     \
+    } else {                                            \
+      VAR = {};                                         \
+    }                                                   \
+  } while (0)
+#define HGC_CHECKED_STORE(PTR, STMT)                    \
+  do {                                                  \
+    if (HGC_ADDR_OK((PTR), sizeof(*(PTR)))) {           \
+      STMT;                                             \
+    }                                                   \
+  } while (0)
+#endif
+
 // Each launcher enqueues on `stream` and returns the launch error (cudaSuccess if fine).
 cudaError_t launch_direct_conv(const ConvGeom& g, const __half* x, const __half* w,
                                const __half* bias, __half* y, int relu, cudaStream_t stream);

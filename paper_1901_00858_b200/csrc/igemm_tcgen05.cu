@@ -35,6 +35,7 @@
 #include "hgc_internal.h"
 
 namespace hgc {
+HGC_DEBUG_STATE(igemm)
 namespace {
 
 constexpr int kEpilogueWarps = 8;       // two per TMEM lane quarter (the default)
@@ -275,10 +276,12 @@ struct LayoutUnit {
     for (int i = 0; i < 8; ++i) {
       if (ch + i < c) {
         if constexpr (PX == 8) {
-          const uint4 q = __ldcs(reinterpret_cast<const uint4*>(s + (int64_t)i * hw));
+          uint4 q;
+          HGC_CHECKED_LOAD(q, reinterpret_cast<const uint4*>(s + (int64_t)i * hw), __ldcs(reinterpret_cast<const uint4*>(s + (int64_t)i * hw)));
           v[i][0] = q.x; v[i][1] = q.y; v[i][2] = q.z; v[i][3] = q.w;
         } else {
-          const uint2 q = __ldcs(reinterpret_cast<const uint2*>(s + (int64_t)i * hw));
+          uint2 q;
+          HGC_CHECKED_LOAD(q, reinterpret_cast<const uint2*>(s + (int64_t)i * hw), __ldcs(reinterpret_cast<const uint2*>(s + (int64_t)i * hw)));
           v[i][0] = q.x; v[i][1] = q.y;
         }
       } else {
@@ -296,7 +299,8 @@ struct LayoutUnit {
       uint32_t o[4];
 #pragma unroll
       for (int m = 0; m < 4; ++m) o[m] = __byte_perm(v[2 * m][q >> 1], v[2 * m + 1][q >> 1], sel);
-      *reinterpret_cast<uint4*>(d + (int64_t)q * c_pad) = make_uint4(o[0], o[1], o[2], o[3]);
+      HGC_CHECKED_STORE(reinterpret_cast<uint4*>(d + (int64_t)q * c_pad),
+                        *reinterpret_cast<uint4*>(d + (int64_t)q * c_pad) = make_uint4(o[0], o[1], o[2], o[3]));
     }
   }
 };
@@ -408,7 +412,7 @@ __device__ __noinline__ void sk_hand_over(uint32_t t_addr, int quarter, int cols
     tmem_ld32(t_addr + (uint32_t)(c * 32), v);
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-    for (int j = 0; j < 32; ++j) __stcg(dst + (size_t)(c * 32 + j) * 128, __uint_as_float(v[j]));
+    for (int j = 0; j < 32; ++j) HGC_CHECKED_STORE(dst + (size_t)(c * 32 + j) * 128, __stcg(dst + (size_t)(c * 32 + j) * 128, __uint_as_float(v[j])));
   }
 }
 
@@ -423,12 +427,12 @@ __device__ __noinline__ void sk_preload(uint32_t t_addr, int quarter, int cols32
     const float* src = slots + (size_t)first_slot * slot_elems + (size_t)c * 32 * 128 + quarter * 32 + lane;
     float v[32];
 #pragma unroll
-    for (int j = 0; j < 32; ++j) v[j] = __ldcg(src + (size_t)j * 128);
+    for (int j = 0; j < 32; ++j) HGC_CHECKED_LOAD(v[j], src + (size_t)j * 128, __ldcg(src + (size_t)j * 128));
     for (int i = 1; i < count; ++i) {
       src += (size_t)slot_step * slot_elems;
       float w[32];
 #pragma unroll
-      for (int j = 0; j < 32; ++j) w[j] = __ldcg(src + (size_t)j * 128);
+      for (int j = 0; j < 32; ++j) HGC_CHECKED_LOAD(w[j], src + (size_t)j * 128, __ldcg(src + (size_t)j * 128));
 #pragma unroll
       for (int j = 0; j < 32; ++j) v[j] += w[j];
     }
@@ -653,7 +657,7 @@ __device__ __noinline__ void epilogue_copy(uint32_t t_addr, uint32_t sbuf, int f
           for (int r = 0; r < kvalid_rows; ++r) {
             uint32_t w;
             asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w) : "r"(sbuf + (uint32_t)r * 128u + ((chunk ^ ((uint32_t)r & 7u)) << 4) + within));
-            *reinterpret_cast<uint32_t*>(dst + (int64_t)r * pq) = w;
+            HGC_CHECKED_STORE(reinterpret_cast<uint32_t*>(dst + (int64_t)r * pq), *reinterpret_cast<uint32_t*>(dst + (int64_t)r * pq) = w);
           }
         }
       } else {
@@ -670,7 +674,7 @@ __device__ __noinline__ void epilogue_copy(uint32_t t_addr, uint32_t sbuf, int f
             for (int r = 0; r < kvalid_rows; ++r) {
               uint16_t w;
               asm volatile("ld.shared.b16 %0, [%1];" : "=h"(w) : "r"(sbuf + (uint32_t)r * 128u + ((chunk ^ ((uint32_t)r & 7u)) << 4) + within));
-              dst[(int64_t)r * pq] = w;
+              HGC_CHECKED_STORE(dst + (int64_t)r * pq, dst[(int64_t)r * pq] = w);
             }
           }
         }
@@ -696,7 +700,7 @@ __device__ __noinline__ void epilogue_columns(uint32_t t_addr, int first_unit, i
         if (c0 + j < nimg) {
           float f = __uint_as_float(v[j]) + bv;
           if (relu) f = fmaxf(f, 0.f);
-          yb[(int64_t)(n0 + c0 + j) * K + k0 + lane] = __half_as_ushort(__float2half_rn(f));
+          HGC_CHECKED_STORE(yb + (int64_t)(n0 + c0 + j) * K + k0 + lane, yb[(int64_t)(n0 + c0 + j) * K + k0 + lane] = __half_as_ushort(__float2half_rn(f)));
         }
       }
     }
@@ -724,7 +728,7 @@ __device__ __noinline__ void epilogue_partial(uint32_t t_addr, uint32_t sbuf, in
       if (lane < kvalid_rows) {
 #pragma unroll
         for (int j = 0; j < 32; ++j)
-          if (c0 + j < nimg) part[(int64_t)(n0 + c0 + j) * K + k0 + lane] = __uint_as_float(v[j]);
+          if (c0 + j < nimg) HGC_CHECKED_STORE(part + (int64_t)(n0 + c0 + j) * K + k0 + lane, part[(int64_t)(n0 + c0 + j) * K + k0 + lane] = __uint_as_float(v[j]));
       }
     }
     __syncwarp();
@@ -772,7 +776,7 @@ __device__ __noinline__ void epilogue_partial(uint32_t t_addr, uint32_t sbuf, in
         for (int r = 0; r < kvalid_rows; ++r) {
           uint32_t w;
           asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w) : "r"(sbuf + (uint32_t)r * 128u + ((chunk ^ ((uint32_t)r & 7u)) << 4) + within));
-          dst[(int64_t)r * pq] = __uint_as_float(w);
+          HGC_CHECKED_STORE(dst + (int64_t)r * pq, dst[(int64_t)r * pq] = __uint_as_float(w));
         }
       }
     }
@@ -788,9 +792,13 @@ splitk_finish_kernel(const float* __restrict__ part, int slices, int64_t stride,
   grid_dependency_wait();
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     float acc = bias != nullptr ? __half2float(__ldg(bias + (int)((i / pq) % K))) : 0.f;
-    for (int sidx = 0; sidx < slices; ++sidx) acc += __ldcs(part + sidx * stride + i);
+    for (int sidx = 0; sidx < slices; ++sidx) {
+      float pv;
+      HGC_CHECKED_LOAD(pv, part + sidx * stride + i, __ldcs(part + sidx * stride + i));
+      acc += pv;
+    }
     if (relu) acc = fmaxf(acc, 0.f);
-    y[i] = __half_as_ushort(__float2half_rn(acc));
+    HGC_CHECKED_STORE(y + i, y[i] = __half_as_ushort(__float2half_rn(acc)));
   }
 }
 
@@ -825,8 +833,8 @@ __device__ __noinline__ void epilogue_nhwc(uint32_t t_addr, int first_unit, int 
             const float f0 = __uint_as_float(v[j]) + bv, f1 = __uint_as_float(v[j + 1]) + bv;
             const uint32_t o = relu ? pack_f16x2<true>(f0, f1) : pack_f16x2<false>(f0, f1);
             if (kvalid) {
-              dst[(int64_t)j * K] = (uint16_t)(o & 0xffffu);
-              if (j + 1 < ncol) dst[(int64_t)(j + 1) * K] = (uint16_t)(o >> 16);
+              HGC_CHECKED_STORE(dst + (int64_t)j * K, dst[(int64_t)j * K] = (uint16_t)(o & 0xffffu));
+              if (j + 1 < ncol) HGC_CHECKED_STORE(dst + (int64_t)(j + 1) * K, dst[(int64_t)(j + 1) * K] = (uint16_t)(o >> 16));
             }
           }
         }
@@ -1664,7 +1672,10 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       //  every tile's epilogue costs several hundred clocks, a third of a short tile's epilogue)
       const int bias_key = kvalid ? k : -2;
       if (bias_key != bias_k) {
-        bv = (bias != nullptr && kvalid) ? __half2float(__ldg(bias + k)) : 0.f;
+        bv = 0.f;
+        if (bias != nullptr && kvalid) {
+          if (HGC_ADDR_OK(bias + k, sizeof(__half))) bv = __half2float(__ldg(bias + k));
+        }
         bias_k = bias_key;
       }
       const uint32_t buf = lt & 1u;

@@ -10,6 +10,7 @@
 #include "hgc_internal.h"
 
 namespace hgc {
+HGC_DEBUG_STATE(layout)
 namespace {
 
 constexpr int kTileC = 64;
@@ -37,7 +38,10 @@ nchw_to_nhwc_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst
       const int ch = c0 + row;
       const int64_t p = p0 + v * 8;
       uint4 val = make_uint4(0, 0, 0, 0);
-      if (ch < c && p < hw) val = *reinterpret_cast<const uint4*>(s + (int64_t)ch * hw + p);  // hw % 8 == 0
+      if (ch < c && p < hw) {  // hw % 8 == 0
+        const uint4* sp = reinterpret_cast<const uint4*>(s + (int64_t)ch * hw + p);
+        HGC_CHECKED_LOAD(val, sp, *sp);
+      }
       *reinterpret_cast<uint4*>(&tile[row][v * 8]) = val;
     }
   } else {
@@ -45,7 +49,9 @@ nchw_to_nhwc_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst
       const int row = i / kTileP, col = i % kTileP;
       const int ch = c0 + row;
       const int64_t p = p0 + col;
-      tile[row][col] = (ch < c && p < hw) ? s[(int64_t)ch * hw + p] : (uint16_t)0;
+      uint16_t e = 0;
+      if (ch < c && p < hw) HGC_CHECKED_LOAD(e, s + (int64_t)ch * hw + p, s[(int64_t)ch * hw + p]);
+      tile[row][col] = e;
     }
   }
   __syncthreads();
@@ -59,7 +65,8 @@ nchw_to_nhwc_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst
 #pragma unroll
       for (int j = 0; j < 4; ++j)
         o[j] = (uint32_t)tile[cv * 8 + 2 * j][px] | ((uint32_t)tile[cv * 8 + 2 * j + 1][px] << 16);
-      *reinterpret_cast<uint4*>(d + p * c_pad + ch) = make_uint4(o[0], o[1], o[2], o[3]);
+      HGC_CHECKED_STORE(reinterpret_cast<uint4*>(d + p * c_pad + ch),
+                        *reinterpret_cast<uint4*>(d + p * c_pad + ch) = make_uint4(o[0], o[1], o[2], o[3]));
     }
   }
 }
@@ -98,10 +105,12 @@ nchw_to_nhwc_regs_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict_
     for (int i = 0; i < 8; ++i) {
       if (ch + i < c) {
         if constexpr (PX == 8) {
-          const uint4 q = __ldcs(reinterpret_cast<const uint4*>(s + (int64_t)i * hw));
+          uint4 q;
+          HGC_CHECKED_LOAD(q, reinterpret_cast<const uint4*>(s + (int64_t)i * hw), __ldcs(reinterpret_cast<const uint4*>(s + (int64_t)i * hw)));
           v[i][0] = q.x; v[i][1] = q.y; v[i][2] = q.z; v[i][3] = q.w;
         } else {
-          const uint2 q = __ldcs(reinterpret_cast<const uint2*>(s + (int64_t)i * hw));
+          uint2 q;
+          HGC_CHECKED_LOAD(q, reinterpret_cast<const uint2*>(s + (int64_t)i * hw), __ldcs(reinterpret_cast<const uint2*>(s + (int64_t)i * hw)));
           v[i][0] = q.x; v[i][1] = q.y;
         }
       } else {
@@ -116,7 +125,8 @@ nchw_to_nhwc_regs_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict_
       uint32_t o[4];
 #pragma unroll
       for (int m = 0; m < 4; ++m) o[m] = __byte_perm(v[2 * m][q >> 1], v[2 * m + 1][q >> 1], sel);
-      *reinterpret_cast<uint4*>(d + (int64_t)q * c_pad) = make_uint4(o[0], o[1], o[2], o[3]);
+      HGC_CHECKED_STORE(reinterpret_cast<uint4*>(d + (int64_t)q * c_pad),
+                        *reinterpret_cast<uint4*>(d + (int64_t)q * c_pad) = make_uint4(o[0], o[1], o[2], o[3]));
     }
   }
 }
@@ -138,8 +148,16 @@ nchw_to_nhwc_smallplane_kernel(const uint16_t* __restrict__ src, uint16_t* __res
   const uint16_t* s = src + (n * c + c0) * (int64_t)hw;
   const int nvec = span >> 3;
   for (int v = threadIdx.x; v < nvec; v += kThreads)
-    reinterpret_cast<uint4*>(flat)[v] = __ldg(reinterpret_cast<const uint4*>(s) + v);
-  for (int e = (nvec << 3) + threadIdx.x; e < span; e += kThreads) flat[e] = s[e];
+  {
+      uint4 q;
+      HGC_CHECKED_LOAD(q, reinterpret_cast<const uint4*>(s) + v, __ldg(reinterpret_cast<const uint4*>(s) + v));
+      reinterpret_cast<uint4*>(flat)[v] = q;
+    }
+  for (int e = (nvec << 3) + threadIdx.x; e < span; e += kThreads) {
+    uint16_t q;
+    HGC_CHECKED_LOAD(q, s + e, s[e]);
+    flat[e] = q;
+  }
   __syncthreads();
   uint16_t* d = dst + n * (int64_t)hw * c_pad;
   const int cvecs = (c_pad - c0 < kTileC ? c_pad - c0 : kTileC) >> 3;  // 16-byte vectors per pixel in this tile
@@ -151,7 +169,8 @@ nchw_to_nhwc_smallplane_kernel(const uint16_t* __restrict__ src, uint16_t* __res
       const int ch = cv * 8 + j;
       if (ch < nch) o[j >> 1] |= (uint32_t)flat[ch * hw + px] << ((j & 1) * 16);
     }
-    *reinterpret_cast<uint4*>(d + (int64_t)px * c_pad + c0 + cv * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+    HGC_CHECKED_STORE(reinterpret_cast<uint4*>(d + (int64_t)px * c_pad + c0 + cv * 8),
+                      *reinterpret_cast<uint4*>(d + (int64_t)px * c_pad + c0 + cv * 8) = make_uint4(o[0], o[1], o[2], o[3]));
   }
 }
 
@@ -188,14 +207,15 @@ nhwc_to_nchw_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst
       const int ch = c0 + row;
       const int64_t p = p0 + v * 8;
       if (ch < c && p < hw)
-        *reinterpret_cast<uint4*>(d + (int64_t)ch * hw + p) = *reinterpret_cast<const uint4*>(&tile[row][v * 8]);
+        HGC_CHECKED_STORE(reinterpret_cast<uint4*>(d + (int64_t)ch * hw + p),
+                          *reinterpret_cast<uint4*>(d + (int64_t)ch * hw + p) = *reinterpret_cast<const uint4*>(&tile[row][v * 8]));
     }
   } else {
     for (int i = threadIdx.x; i < kTileC * kTileP; i += kThreads) {
       const int row = i / kTileP, col = i % kTileP;
       const int ch = c0 + row;
       const int64_t p = p0 + col;
-      if (ch < c && p < hw) d[(int64_t)ch * hw + p] = tile[row][col];
+      if (ch < c && p < hw) HGC_CHECKED_STORE(d + (int64_t)ch * hw + p, d[(int64_t)ch * hw + p] = tile[row][col]);
     }
   }
 }
@@ -229,10 +249,15 @@ __global__ void weights_repack_kernel(const uint16_t* __restrict__ src, uint16_t
     for (int j = 0; j < 8; ++j) {
       const int ch = cv * 8 + j;
       uint32_t v = 0;
-      if (ch < cg) v = src[(row_channel(kk, perm) * cg + ch) * rs + t];
+      if (ch < cg) {
+        uint16_t e;
+        HGC_CHECKED_LOAD(e, src + (row_channel(kk, perm) * cg + ch) * rs + t, src[(row_channel(kk, perm) * cg + ch) * rs + t]);
+        v = e;
+      }
       o[j >> 1] |= v << ((j & 1) * 16);
     }
-    *reinterpret_cast<uint4*>(dst + (kk * rs + t) * c_pad + cv * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+    HGC_CHECKED_STORE(reinterpret_cast<uint4*>(dst + (kk * rs + t) * c_pad + cv * 8),
+                      *reinterpret_cast<uint4*>(dst + (kk * rs + t) * c_pad + cv * 8) = make_uint4(o[0], o[1], o[2], o[3]));
   }
 }
 
@@ -258,8 +283,8 @@ nchw_to_nhwc8_bordered_kernel(const uint16_t* __restrict__ src, uint16_t* __rest
       for (int ch = 0; ch < PC; ++ch)
         if (ch < c) o[ch >> 1] |= (uint32_t)s[ch * hw] << ((ch & 1) * 16);
     }
-    if (PC == 8) *reinterpret_cast<uint4*>(dst + i * 8) = make_uint4(o[0], o[1], o[2], o[3]);
-    else *reinterpret_cast<uint2*>(dst + i * 4) = make_uint2(o[0], o[1]);
+    if (PC == 8) HGC_CHECKED_STORE(reinterpret_cast<uint4*>(dst + i * 8), *reinterpret_cast<uint4*>(dst + i * 8) = make_uint4(o[0], o[1], o[2], o[3]));
+    else HGC_CHECKED_STORE(reinterpret_cast<uint2*>(dst + i * 4), *reinterpret_cast<uint2*>(dst + i * 4) = make_uint2(o[0], o[1]));
   }
 }
 
@@ -283,8 +308,8 @@ nchw_to_nhwc8_bordered_vec_kernel(const uint16_t* __restrict__ src, uint16_t* __
   const int64_t n = t / hp;
   uint16_t* drow = dst + (n * hp + oh) * (int64_t)wp * PC;
   auto store_px = [&](int ow, uint32_t o0, uint32_t o1, uint32_t o2, uint32_t o3) {
-    if (PC == 8) *reinterpret_cast<uint4*>(drow + (int64_t)ow * 8) = make_uint4(o0, o1, o2, o3);
-    else *reinterpret_cast<uint2*>(drow + (int64_t)ow * 4) = make_uint2(o0, o1);
+    if (PC == 8) HGC_CHECKED_STORE(reinterpret_cast<uint4*>(drow + (int64_t)ow * 8), *reinterpret_cast<uint4*>(drow + (int64_t)ow * 8) = make_uint4(o0, o1, o2, o3));
+    else HGC_CHECKED_STORE(reinterpret_cast<uint2*>(drow + (int64_t)ow * 4), *reinterpret_cast<uint2*>(drow + (int64_t)ow * 4) = make_uint2(o0, o1));
   };
   if (slot == slots - 1) {  // the zero columns of this row
     for (int ow = 0; ow < pad_w; ++ow) store_px(ow, 0u, 0u, 0u, 0u);
@@ -336,8 +361,8 @@ __global__ void weights_repack_window_kernel(const uint16_t* __restrict__ src, u
         if (ch < c)
           o[ch >> 1] |= (uint32_t)src[((row_channel(kk, perm) * c + ch) * r + rr) * s + sp] << ((ch & 1) * 16);
     }
-    if (PC == 8) *reinterpret_cast<uint4*>(dst + i * 8) = make_uint4(o[0], o[1], o[2], o[3]);
-    else *reinterpret_cast<uint2*>(dst + i * 4) = make_uint2(o[0], o[1]);
+    if (PC == 8) HGC_CHECKED_STORE(reinterpret_cast<uint4*>(dst + i * 8), *reinterpret_cast<uint4*>(dst + i * 8) = make_uint4(o[0], o[1], o[2], o[3]));
+    else HGC_CHECKED_STORE(reinterpret_cast<uint2*>(dst + i * 4), *reinterpret_cast<uint2*>(dst + i * 4) = make_uint2(o[0], o[1]));
   }
 }
 
@@ -389,7 +414,7 @@ patch_im2col_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst
       uint32_t a[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) a[j] = (4 * v + j) < EW ? o[(4 * v + j) < EW ? 4 * v + j : 0] : 0u;
-      d[v] = make_uint4(a[0], a[1], a[2], a[3]);
+      HGC_CHECKED_STORE(d + v, d[v] = make_uint4(a[0], a[1], a[2], a[3]));
     }
   }
 }
@@ -427,7 +452,7 @@ patch_im2col_generic_kernel(const uint16_t* __restrict__ src, uint16_t* __restri
         o[j >> 1] |= (uint32_t)__ldg(xn + ch * hw + (int64_t)ih * w + iw) << ((j & 1) * 16);
     }
   }
-  *reinterpret_cast<uint4*>(dst + i * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+  HGC_CHECKED_STORE(reinterpret_cast<uint4*>(dst + i * 8), *reinterpret_cast<uint4*>(dst + i * 8) = make_uint4(o[0], o[1], o[2], o[3]));
 }
 
 // w[k][c][r][s] -> w'[k][kelems], element (r*S + s)*C + ch; zeros from R*S*C on
@@ -446,7 +471,7 @@ __global__ void weights_repack_patch_kernel(const uint16_t* __restrict__ src, ui
       const int tap = e / c;
       v = src[(row_channel(kk, perm) * c + ch) * (r * s) + tap];
     }
-    dst[i] = v;
+    HGC_CHECKED_STORE(dst + i, dst[i] = v);
   }
 }
 
@@ -643,7 +668,8 @@ __global__ void weights_repack_rowpair_kernel(const uint16_t* __restrict__ src, 
         o[j >> 1] |= v << ((j & 1) * 16);
       }
     }
-    *reinterpret_cast<uint4*>(dst + ((int64_t)kk * (r + 1) * s + t) * c_pad + cv * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+    HGC_CHECKED_STORE(reinterpret_cast<uint4*>(dst + ((int64_t)kk * (r + 1) * s + t) * c_pad + cv * 8),
+                      *reinterpret_cast<uint4*>(dst + ((int64_t)kk * (r + 1) * s + t) * c_pad + cv * 8) = make_uint4(o[0], o[1], o[2], o[3]));
   }
 }
 
@@ -675,7 +701,7 @@ depthwise_weights_to_taps_kernel(const uint16_t* __restrict__ w, uint16_t* __res
   grid_dependency_wait();
   grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
   const int i = blockIdx.x * blockDim.x + threadIdx.x;  // index into w9: tap * c + channel
-  if (i < 9 * c) w9[i] = w[(i % c) * 9 + i / c];
+  if (i < 9 * c) HGC_CHECKED_STORE(w9 + i, w9[i] = w[(i % c) * 9 + i / c]);
 }
 
 cudaError_t launch_depthwise_weights_to_taps(const __half* w, __half* w9, int32_t c, cudaStream_t stream) {

@@ -88,6 +88,15 @@ extern "C" int hgc_conv_forward_static(const hgc_conv_params* p, const void* x, 
   // must start at zero; the re-layout kernels rewrite every byte of the weight and input copies
   // that the tensor-core kernel reads, padding included, and a reduction slice writes every
   // partial sum before the second pass reads it
+  if (hgc::kCheckedBuild) {
+    hgc::DebugRanges r{};
+    hgc::debug_add_range(&r, x, (size_t)g.n * g.c * g.h * g.w * 2);
+    hgc::debug_add_range(&r, w, (size_t)g.k * g.cg * g.r * g.s * 2);
+    hgc::debug_add_range(&r, bias, (size_t)g.k * 2);
+    hgc::debug_add_range(&r, y, (size_t)g.n * g.k * g.p * g.q * 2);
+    hgc::debug_add_range(&r, ws, plan.ws_total);
+    hgc::debug_set_call_ranges(r, st);
+  }
   if (cudaMemsetAsync(ws + plan.ws_status_off, 0, hgc::kWsHeaderBytes, st) != cudaSuccess) return HGC_CUDA_ERROR;
   if (!hgc::igemm_encode_maps(g, &plan, ws)) return HGC_CUDA_ERROR;
   const __half* xh = static_cast<const __half*>(x);
