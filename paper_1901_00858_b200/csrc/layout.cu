@@ -419,6 +419,73 @@ patch_im2col_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst
   }
 }
 
+// The same for 3x3 kernels with stride 2 and padding 1 along W on rows of an even number of pixels
+// (the stems of MobileNet-like networks): output pixel oq reads input pixels 2oq-1, 2oq, 2oq+1 of
+// three rows.  A warp owns 32 consecutive output pixels of ONE output row; a lane loads the aligned
+// 4-byte word (2oq, 2oq+1) per row and channel and takes pixel 2oq-1 from its left neighbour's word
+// by shuffle: 9 loads per thread instead of 27 two-byte ones (the MobileNet stem, 32x3x224x224: 36.5 -> 33.8 us with its tensor-core kernel).
+template <int C>
+__global__ void __launch_bounds__(256)
+patch_im2col_s2_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int h, int w, int p, int q,
+                       int pad_h, int stride_h, int kelems, int warps_per_row, int64_t total_warps) {
+  grid_dependency_wait();
+  grid_launch_dependents();  // a tensor-core kernel that follows may set itself up beside this one
+  constexpr int E = 9 * C;
+  constexpr int EW = (E + 1) / 2;
+  const int lane = threadIdx.x & 31;
+  const int64_t gw = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (gw >= total_warps) return;
+  const int wr = (int)(gw % warps_per_row);
+  const int64_t row = gw / warps_per_row;  // (image, output row)
+  const int op = (int)(row % p);
+  const int64_t n = row / p;
+  const int oq = wr * 32 + lane;
+  const bool live = oq < q;
+  const int64_t hw = (int64_t)h * w;
+  const uint16_t* xn = src + n * C * hw;
+  uint32_t o[EW];
+#pragma unroll
+  for (int e = 0; e < EW; ++e) o[e] = 0u;
+#pragma unroll
+  for (int r = 0; r < 3; ++r) {
+    const int ih = op * stride_h - pad_h + r;
+    const bool rv = ih >= 0 && ih < h;  // (the same for the whole warp)
+#pragma unroll
+    for (int ch = 0; ch < C; ++ch) {
+      const uint16_t* xr = xn + ch * hw + (int64_t)ih * w;
+      uint32_t word = 0u;
+      if (rv && live) HGC_CHECKED_LOAD(word, reinterpret_cast<const uint32_t*>(xr + 2 * oq), __ldg(reinterpret_cast<const uint32_t*>(xr + 2 * oq)));
+      uint32_t left = __shfl_up_sync(0xffffffffu, word, 1) >> 16;
+      if (lane == 0) {
+        left = 0u;
+        if (rv && live && oq > 0) {
+          uint16_t e;
+          HGC_CHECKED_LOAD(e, xr + 2 * oq - 1, __ldg(xr + 2 * oq - 1));
+          left = e;
+        }
+      }
+      const uint32_t px[3] = {left, word & 0xffffu, word >> 16};
+#pragma unroll
+      for (int sx = 0; sx < 3; ++sx) {
+        const int e = (r * 3 + sx) * C + ch;
+        o[e >> 1] |= px[sx] << ((e & 1) * 16);
+      }
+    }
+  }
+  if (!live) return;
+  uint4* d = reinterpret_cast<uint4*>(dst + ((row * q) + oq) * kelems);
+  const int vecs = kelems >> 3;
+#pragma unroll
+  for (int v = 0; v < 8; ++v) {
+    if (v < vecs) {
+      uint32_t a[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) a[j] = (4 * v + j) < EW ? o[(4 * v + j) < EW ? 4 * v + j : 0] : 0u;
+      HGC_CHECKED_STORE(d + v, d[v] = make_uint4(a[0], a[1], a[2], a[3]));
+    }
+  }
+}
+
 // any R, S, C with R*S*C <= 64: one thread per 8-element chunk of an output pixel's patch
 __global__ void __launch_bounds__(256)
 patch_im2col_generic_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int c, int h, int w,
@@ -608,7 +675,21 @@ cudaError_t launch_patch_im2col(const ConvGeom& g, const __half* src, __half* ds
   const uint16_t* s16 = reinterpret_cast<const uint16_t*>(src);
   uint16_t* d16 = reinterpret_cast<uint16_t*>(dst);
   const int64_t pixels = (int64_t)g.n * g.p * g.q;
-  if (g.r == 3 && g.s == 3 && (g.c == 3 || g.c == 1 || g.c == 4)) {
+  if (g.r == 3 && g.s == 3 && (g.c == 3 || g.c == 1 || g.c == 4) && g.stride_w == 2 && g.pad_w == 1 && g.dil_h == 1 &&
+      g.dil_w == 1 && (g.w % 2) == 0 && g.q == g.w / 2) {
+    // (even rows: every row of x starts on a 4-byte boundary)
+    const int wpr = (g.q + 31) / 32;
+    const int64_t warps = (int64_t)g.n * g.p * wpr;
+    const int64_t blocks = (warps + 7) / 8;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+#define HGC_PATCH_S2(CV)                                                                                        \
+  launch_kernel(patch_im2col_s2_kernel<CV>, dim3((unsigned)blocks), dim3(256), 0, stream, s16, d16, g.h, g.w, g.p, g.q, \
+                g.pad_h, g.stride_h, kelems, wpr, warps)
+    if (g.c == 3) HGC_PATCH_S2(3);
+    else if (g.c == 1) HGC_PATCH_S2(1);
+    else HGC_PATCH_S2(4);
+#undef HGC_PATCH_S2
+  } else if (g.r == 3 && g.s == 3 && (g.c == 3 || g.c == 1 || g.c == 4)) {
     const int64_t blocks = (pixels + 255) / 256;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
 #define HGC_PATCH(CV)                                                                                         \

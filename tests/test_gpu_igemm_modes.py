@@ -62,6 +62,8 @@ CASES = [
     ("stem 3x3 c3 stride 1, 256 wide (rows too wide for the dense form)", params_dict(1, 3, 6, 256, 16, 3, 3, 1, 1), X_WINDOWS),
     ("stem 3x3 c3 stride 2 (patches)", params_dict(2, 3, 64, 48, 32, 3, 3, 1, 1, 2, 2), X_PATCHES),
     ("stem 3x3 c1 stride 2 (patches)", params_dict(3, 1, 33, 31, 24, 3, 3, 1, 1, 2, 2), X_PATCHES),
+    ("stem 3x3 c4 stride 2, 44 wide (patches from aligned words)", params_dict(2, 4, 30, 44, 16, 3, 3, 1, 1, 2, 2), X_PATCHES),
+    ("stem 3x3 c1 stride 2 x 1, 70 wide, pad 2 x 1 (patches from aligned words)", params_dict(3, 1, 21, 70, 24, 3, 3, 2, 1, 1, 2), X_PATCHES),
     ("stem 3x3 c4 stride 2 dilated (patches)", params_dict(2, 4, 30, 30, 20, 3, 3, 2, 2, 2, 2, 2, 2), X_PATCHES),
     ("stem 5x5 c2 stride 3 (patches, generic expansion)", params_dict(2, 2, 29, 35, 20, 5, 5, 2, 2, 3, 3), X_PATCHES),
     ("stem 1x1 c8 stride 2 (patches)", params_dict(2, 8, 18, 18, 16, 1, 1, 0, 0, 2, 2), X_PATCHES),
