@@ -276,6 +276,7 @@ struct IgemmPlan {
   uint32_t a_bytes, b_bytes, b_alloc;
   int32_t a_rows;  // rows of a weight tile in shared memory (128, or 64 for layers of <= 64 channels per group)
   int32_t fine_units;  // TMA-store epilogue works in units of 32 pixels (else 64)
+  int32_t nacc;        // depthwise + pointwise blocks: 128-channel tiles (accumulators) that share a pixel tile's depthwise result: 1, 2, 4
   // Row pairs: a stride-1 layer of 64 output channels with R kernel rows is run as a layer of 128
   // "channels" (output row parity x channel), R + 1 kernel rows and stride 2 along H on P/2 rows:
   // accumulator lanes 64..127 hold the odd output rows, so no lane of the 128-row MMA is idle

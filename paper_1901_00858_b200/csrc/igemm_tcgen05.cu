@@ -900,6 +900,9 @@ struct IgemmArgs {
   int32_t dup_log2;   // log2 of the number of copies of the layer's rows in a weight tile (0, 1, 2)
   int32_t fine_units; // TMA-store epilogue: units of 32 pixels instead of 64
   int32_t rowpair;    // lanes 64..127 hold the odd output rows of the layer's 64 channels (IgemmPlan::rowpair)
+  int32_t nacc;       // depthwise + pointwise blocks: channel tiles (accumulators) per pixel tile: 1, 2 or 4
+  int32_t mshift;     // log2 of the channel tiles that one work item covers (pairs: 1; nacc: 0, 1, 2)
+  int32_t acc_stride; // accumulator columns between the channel tiles of an item (nacc > 1: 512 / nacc)
   // split reduction (its own kernel instantiation): the channel blocks of a tile are dealt out to
   // 2^ks_log2 CTAs, each of which writes its fp32 partial sums to its own slice of `partials`; a
   // second kernel adds the slices in a fixed order (+ bias, ReLU, rounding)
@@ -1099,10 +1102,10 @@ struct SegIter {
   __device__ __forceinline__ void channel_tile(const IgemmArgs& a, int& grp, int& m0) const {
     if (a.group == 1) {
       grp = 0;
-      m0 = (mg * 128) << a.pair;
+      m0 = (mg * 128) << a.mshift;
     } else {
       grp = mg / a.mtiles;
-      m0 = ((mg - grp * a.mtiles) * 128) << a.pair;
+      m0 = ((mg - grp * a.mtiles) * 128) << a.mshift;
     }
   }
   // first image and output row of pixel sub-tile j of the current pair tile; a pair tile past the
@@ -1306,15 +1309,16 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         // them, so that the wait for that stage runs out (hgc_debug_drop_copies)
         const bool drop = a.dbg_drop >= 0 && blockIdx.x == 0 && issued == (uint32_t)a.dbg_drop;
         if (drop) {
-          if (lane == 0) mbar_expect_tx(smem_u32(&full_bar[ring.idx]), (PAIR ? 2u : 1u) * (a.b_bytes + (uint32_t)a.taps * a.a_bytes));
+          if (lane == 0) mbar_expect_tx(smem_u32(&full_bar[ring.idx]), (PAIR ? 2u : 1u) * (a.b_bytes + (uint32_t)((DWPW ? a.nacc : 1) * a.taps) * a.a_bytes));
         } else if constexpr (DWPW) {
           // the activation tile of the stage is computed by the depthwise warps from an input tile
           // (with its one-pixel border) that is fetched here, beside the pointwise weights
           const uint32_t fb = smem_u32(&full_bar[ring.idx]);
-          if (lane == 0) {
-            mbar_expect_tx(fb, (uint32_t)a.taps * a.a_bytes);
-            tma_load_4d(sbase + a.b_alloc, &tmA, fb, cb * KB, m0, tap0, grp);
-          }
+          // the weight tiles of the item's channel tiles (one per accumulator), behind one another
+          if (lane == 0) mbar_expect_tx(fb, (uint32_t)(a.nacc * a.taps) * a.a_bytes);
+          __syncwarp();
+          if (lane < a.nacc)
+            tma_load_4d(sbase + a.b_alloc + (uint32_t)(lane * a.taps) * a.a_bytes, &tmA, fb, cb * KB, m0 + lane * 128, tap0, grp);
           const uint32_t ib = issued & 1u;
           if (!mbar_wait(smem_u32(&in_empty[ib]), ((issued >> 1) & 1u) ^ 1u, &abort_flag, 64)) {
             ok = false;
@@ -1402,9 +1406,12 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       int s0, s1;
       it.stage_range(a, s0, s1);
       const int groups_per_tile = s1 - s0;
-      const uint32_t buf = lt & 1u;
+      // two accumulators take turns; a block kernel with several channel tiles per pixel tile has
+      // one set of them, which the epilogue must have drained before the next tile starts
+      const bool one_set = DWPW && a.nacc > 1;
+      const uint32_t buf = one_set ? 0u : (lt & 1u);
       // the epilogue must have drained this accumulator (two tiles ago)
-      if (!mbar_wait(smem_u32(&acc_empty[buf]), ((lt >> 1) & 1u) ^ 1u, &abort_flag, 64)) {
+      if (!mbar_wait(smem_u32(&acc_empty[buf]), ((one_set ? lt : (lt >> 1)) & 1u) ^ 1u, &abort_flag, 64)) {
         ok = false;
         break;
       }
@@ -1434,16 +1441,24 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         uint64_t bdesc = a.desc_hi_b | (uint64_t)((sbase & 0x3FFFFu) >> 4);
         uint64_t adesc = desc_hi | (uint64_t)(((sbase + a.b_alloc) & 0x3FFFFu) >> 4);
         ring.advance(depth);
+        if constexpr (DWPW) {
+          // further channel tiles of the item: the same activation tile against their weight tiles
+          for (int ci = 0; ci + 1 < a.nacc; ++ci) {
+            issue_mmas<ksteps, PAIR>(d_tmem + (uint32_t)(ci * a.acc_stride), adesc, bdesc, idesc, acc, do_mma, a.b_kstep);
+            adesc += (uint64_t)(((uint32_t)a.taps * a.a_bytes) >> 4);
+          }
+        }
+        const uint32_t d_last = DWPW ? d_tmem + (uint32_t)((a.nacc - 1) * a.acc_stride) : d_tmem;
         // all taps but the last: MMAs only
         for (int t = 0; t + 1 < a.taps; ++t) {
-          issue_mmas<ksteps, PAIR>(d_tmem, adesc, bdesc, idesc, acc, do_mma, a.b_kstep);
+          issue_mmas<ksteps, PAIR>(d_last, adesc, bdesc, idesc, acc, do_mma, a.b_kstep);
           acc = 1;
           adesc += (uint64_t)(a.a_bytes >> 4);
           bdesc += (uint64_t)(tap_step >> 4);
         }
         // last tap: poll the NEXT stage's barrier first and read the answer after the MMAs and the
         // commit have been issued, so that the poll's latency hides behind them
-        ready = issue_stage<ksteps, PAIR>(smem_u32(&full_bar[ring.idx]), ring.phase, d_tmem, adesc, bdesc, idesc, acc, e_bar,
+        ready = issue_stage<ksteps, PAIR>(smem_u32(&full_bar[ring.idx]), ring.phase, d_last, adesc, bdesc, idesc, acc, e_bar,
                                     e_bar, 0u, do_mma, a.b_kstep);
         acc = 1;
       }
@@ -1662,9 +1677,13 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           }
         }
       }
-      int grp, m0;
-      it.channel_tile(a, grp, m0);
-      if constexpr (PAIR) m0 += (int)rank * 128;  // this CTA's tensor memory holds its own 128 channels
+      int grp, m0_item;
+      it.channel_tile(a, grp, m0_item);
+      if constexpr (PAIR) m0_item += (int)rank * 128;  // this CTA's tensor memory holds its own 128 channels
+      // (block kernels with several channel tiles per pixel tile come back here for each of them)
+      int ci = 0;
+    next_channel_tile:
+      const int m0 = m0_item + ci * 128;
       const int kin = m0 + row;
       const bool kvalid = kin < (a.rowpair ? 64 : a.kg);
       const int k = grp * a.kg + (kvalid ? kin : 0);
@@ -1678,10 +1697,13 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         }
         bias_k = bias_key;
       }
-      const uint32_t buf = lt & 1u;
-      if (!mbar_wait(smem_u32(&acc_full[buf]), (lt >> 1) & 1u, &abort_flag, 256)) break;
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t t_tile = tmem_base + buf * 256u + ((uint32_t)(quarter * 32) << 16);
+      const bool one_set = DWPW && a.nacc > 1;  // (see the MMA issuer)
+      const uint32_t buf = one_set ? 0u : (lt & 1u);
+      if (ci == 0) {
+        if (!mbar_wait(smem_u32(&acc_full[buf]), (one_set ? lt : (lt >> 1)) & 1u, &abort_flag, 256)) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      }
+      const uint32_t t_tile = tmem_base + buf * 256u + (uint32_t)(DWPW ? ci * a.acc_stride : 0) + ((uint32_t)(quarter * 32) << 16);
       const bool quarter_live = m0 + cq * 32 < (a.rowpair ? 64 : a.kg);  // any real output channel in this warp's lanes?
       // the barrier the accumulator is handed back on (of a pair: the first CTA's)
       const uint32_t acc_empty_bar = PAIR ? cluster_addr(smem_u32(&acc_empty[buf]), 0) : smem_u32(&acc_empty[buf]);
@@ -1890,6 +1912,9 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         }
       }
       }  // sub-tiles
+      if constexpr (DWPW) {
+        if (++ci < a.nacc) goto next_channel_tile;
+      }
       // this warp has read its lanes of the accumulator: hand the buffer back to the MMA issuer
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
@@ -2369,12 +2394,64 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
     best_grid = pgrid;
     best_ks = 0;
   }
+  // Depthwise + pointwise blocks: the depthwise warps, not the MMAs, bound a stage (about 33 clocks
+  // per pixel of a 64-channel block, measured), and every 128-channel tile of the pointwise layer
+  // that is computed from its own pass repeats that work.  So a work item covers up to four
+  // channel tiles (accumulators of 512 / nacc columns, one set: the epilogue is not overlapped)
+  // that share the depthwise result, and the pixel tile is chosen together with their number.
+  p.nacc = 1;
+  if (g.dw_stride > 0) {
+    double best_blk = 1e300;
+    int bth = 0, btn = 0, bna = 1;
+    for (int th = 1; th <= g.p; ++th) {
+      const int64_t in_h = (int64_t)(th - 1) * g.dw_stride + 3, in_w = (int64_t)(g.q - 1) * g.dw_stride + 3;
+      if ((int64_t)th * g.q > 256 || in_h > 256 || in_w > 256) break;
+      const int tn_hi = th == g.p ? g.n : 1;
+      for (int tn = 1; tn <= tn_hi; ++tn) {
+        const int64_t px = (int64_t)tn * th * g.q;
+        if (px > (tn > 1 ? 248 : 256) || tn * in_h * in_w * p.kb * 2 > 48 * 1024) break;
+        for (int na = 1; na <= 4; na *= 2) {
+          if (na > 1 && (px > 512 / na || (int64_t)(na / 2) * 128 >= g.kg)) break;
+          {
+            // two ring stages (activation tile + na weight tiles), both input tiles and the
+            // epilogue's staging tiles must fit into shared memory
+            const size_t stage = round_up_sz((size_t)((px + 15) / 16 * 16) * p.kb * 2, 1024) + (size_t)na * 128 * p.kb * 2;
+            const size_t in_tile = round_up_sz((size_t)tn * in_h * in_w * p.kb * 2 + 2u * p.kb * 2u, 1024);
+            if (2 * stage + 2 * in_tile + (size_t)kEpilogueWarps * kWarpStageBytes > 232448u - 1024u - 512u) break;
+          }
+          const int64_t tiles = (int64_t)((g.n + tn - 1) / tn) * ((g.p + th - 1) / th) * ((p.mtiles + na - 1) / na);
+          const double waves = (double)((tiles + sms - 1) / sms);
+          const double t_dw = 33.0 * (double)px * (p.kb / 64.0);
+          const double t_mma = (double)na * (p.kb / 16.0) * ((double)px / 2.0 > 58.0 ? (double)px / 2.0 : 58.0);
+          const double units = (double)((px + 63) / 64);
+          const double t_epi = 2000.0 * units * (na > 1 ? 2.0 * na : 1.0);  // (one set of accumulators: not hidden)
+          const double cost = waves * ((double)p.cblocks * (t_dw > t_mma ? t_dw : t_mma) + t_epi + 4000.0);
+          if (cost < best_blk) {
+            best_blk = cost;
+            bth = th; btn = tn; bna = na;
+          }
+        }
+      }
+    }
+    if (bth == 0) return false;
+    best_th = bth;
+    best_tn = btn;
+    best_ks = 0;
+    best_shared = 0;
+    p.nacc = bna;
+    const int64_t tiles = (int64_t)((g.n + btn - 1) / btn) * ((g.p + bth - 1) / bth) * ((p.mtiles + bna - 1) / bna);
+    best_grid = (int)(tiles < sms ? tiles : sms);
+  }
   p.th = best_th;
   p.tn = best_tn;
   p.tiles_h = (g.p + p.th - 1) / p.th;
   p.tiles_n = (g.n + p.tn - 1) / p.tn;
   p.ncols = (p.tn * p.th * p.pitch - junk + 15) / 16 * 16;
   int64_t total = (int64_t)p.tiles_n * p.tiles_h * mg;
+  if (p.nacc > 1) {  // (blocks: one group, so mg == mtiles)
+    p.mtiles = (p.mtiles + p.nacc - 1) / p.nacc;
+    total = (int64_t)p.tiles_n * p.tiles_h * p.mtiles * g.group;
+  }
   if (p.pair) {
     p.ncols_sub = (p.tn * p.th * p.pitch - junk + 7) / 8 * 8;
     p.ncols = 2 * p.ncols_sub;
@@ -2483,7 +2560,7 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
       p.b_bytes = (uint32_t)p.nblk * (uint32_t)p.kb * 128u;
       p.b_alloc = p.b_bytes;
     }
-    p.stage_bytes = p.b_alloc + (uint32_t)p.taps * p.a_bytes;
+    p.stage_bytes = p.b_alloc + (uint32_t)(p.nacc > 1 ? p.nacc : 1) * (uint32_t)p.taps * p.a_bytes;
     p.stages = (int)(budget / p.stage_bytes);
     if (p.stages > 8) p.stages = 8;
     if (p.stages >= 2) break;
@@ -2787,6 +2864,9 @@ cudaError_t launch_igemm(const ConvGeom& g_layer, IgemmPlan& p, void* ws, const 
   a.dup_log2 = p.dup_log2;
   a.fine_units = p.fine_units;
   a.rowpair = p.rowpair;
+  a.nacc = p.nacc > 0 ? p.nacc : 1;
+  a.acc_stride = a.nacc > 1 ? 512 / a.nacc : 0;
+  a.mshift = p.pair + (a.nacc == 4 ? 2 : (a.nacc == 2 ? 1 : 0));
   a.ks_log2 = p.ks_log2;
   a.part_stride = (int64_t)g.n * g.k * g.p * g.q;
   a.y_tma = (p.y_nhwc && p.tma_store) ? 1 : 0;
