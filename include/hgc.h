@@ -105,6 +105,17 @@ typedef struct hgc_conv_params {
  * step runs under the board's power cap, where work that overlaps costs what it costs alone).
  */
 #define HGC_FLAG_FUSED_LAYOUT 32
+/*
+ * 1x1, stride-1, unpadded layers read x (NCHW) as it is when a channel's plane is a multiple of 8
+ * pixels (the copy engine fetches pixel-major tiles); other planes take the NHWC copy of x first.
+ * HGC_FLAG_GATHER_X (off by default): planes of a multiple of 4 pixels and at most 256 (14x14),
+ * with C a multiple of 64, start on 8-byte boundaries only, which no tensor map can describe;
+ * with this flag eight extra warps of the tensor-core kernel gather the pixel-major tile
+ * themselves with 8-byte asynchronous copies (plan [10] = 4) and no copy of x is made.  Measured
+ * (B200): slower than the layout pass plus the plain kernel (64 x 1024 -> 256 on 14x14: 24.8 us
+ * against 21.2; 256 -> 1024: 32.1 against 23.1), so it is not the planner's choice.
+ */
+#define HGC_FLAG_GATHER_X 128
 
 typedef struct hgc_conv_desc hgc_conv_desc; /* opaque; owned by the caller via create/destroy */
 
@@ -205,7 +216,8 @@ int hgc_conv_path(const hgc_conv_desc* d, int32_t* path);
  * as pixel-major tiles; channels-last x, which includes every input with a 1x1 plane), 2 = a
  * zero-bordered 8-channel NHWC copy read through
  * overlapping windows (few input channels), 3 = an expanded copy holding, per output pixel, the
- * values under the kernel (few input channels, strided), [11] the number of CTAs that share
+ * values under the kernel (few input channels, strided), 4 = x itself, gathered by extra warps of
+ * the kernel (1x1 layers on small planes, see HGC_FLAG_GATHER_X), [11] the number of CTAs that share
  * the reduction of one tile (1, or 2 / 4 / 8 for layers with very few tiles, e.g. inner products:
  * each CTA writes fp32 partial sums and a second kernel adds them in a fixed order), [12] the
  * number of CTAs of the launch when the ring stages of all tiles are dealt out as contiguous

@@ -24,6 +24,7 @@ HGC_FLAG_CTA_PAIRS = 8
 HGC_FLAG_SHARED_TILES = 16
 HGC_FLAG_FUSED_LAYOUT = 32
 HGC_FLAG_WHOLE_TILES = 64
+HGC_FLAG_GATHER_X = 128
 PATH_NAMES = {HGC_PATH_DIRECT: "direct", HGC_PATH_DEPTHWISE: "depthwise", HGC_PATH_IGEMM: "igemm"}
 
 

@@ -171,6 +171,7 @@ int hgc_conv_desc_create(hgc_conv_desc** out, const hgc_conv_params* p) {
   g.no_pair = (p->flags & HGC_FLAG_CTA_PAIRS) ? 0 : 1;
   g.no_split = (p->flags & HGC_FLAG_WHOLE_TILES) ? 1 : ((p->flags & HGC_FLAG_SHARED_TILES) ? 0 : 2);  // 2: the planner's cost model decides
   g.no_fuse = (p->flags & HGC_FLAG_FUSED_LAYOUT) ? 0 : 1;
+  g.no_gather = (p->flags & HGC_FLAG_GATHER_X) ? 0 : 1;
   const bool channels_last = g.x_nhwc || g.y_nhwc;
 
   d->path = HGC_PATH_DIRECT;
@@ -259,7 +260,7 @@ int hgc_conv_plan_info(const hgc_conv_desc* d, int32_t* info, int32_t count) {
     const hgc::IgemmPlan& p = d->igemm;
     v[1] = p.kb; v[2] = p.halo; v[3] = p.tn; v[4] = p.th; v[5] = p.pitch; v[6] = p.ncols;
     v[7] = p.total_tiles; v[8] = p.stages; v[9] = p.taps;
-    v[10] = (p.nchw || p.x_nhwc) ? 1 : (p.window ? 2 : (p.patch ? 3 : 0));
+    v[10] = p.gather ? 4 : ((p.nchw || p.x_nhwc) ? 1 : (p.window ? 2 : (p.patch ? 3 : 0)));
     v[11] = 1 << p.ks_log2;
     v[12] = p.ks_log2 > 0 ? 0 : ((p.pair && p.pair_fit > 0 && p.pair_fit < p.grid) ? p.pair_fit : p.grid);
     v[13] = p.sk_split;
@@ -407,7 +408,7 @@ int hgc_dwpw_desc_create(hgc_conv_desc** out, const hgc_dwpw_params* p) {
   g.p = (int32_t)P; g.q = (int32_t)Q; g.cg = p->c; g.kg = p->k;
   g.x_nhwc = 1;
   g.y_nhwc = (p->flags & HGC_FLAG_Y_NHWC) ? 1 : 0;
-  g.no_pair = 1; g.no_split = 1; g.no_fuse = 1;
+  g.no_pair = 1; g.no_split = 1; g.no_fuse = 1; g.no_gather = 1;
   g.dw_stride = p->stride;
   // the tensor-core plan of the pointwise layer over a channels-last input that is never stored:
   // whole 8-channel chunks, 32- or 64-channel stages, whole tiles on single CTAs

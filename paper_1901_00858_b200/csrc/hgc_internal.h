@@ -21,6 +21,7 @@ struct ConvGeom {
   int32_t no_split;        // 1: never let several CTAs share the reduction of a tile (no scratch for it); 0: wherever possible; 2: where the cost model expects a gain
   int32_t no_pair;         // 1: never pair CTAs on 256-channel tiles
   int32_t no_fuse;         // 1: the layout pass stays a kernel of its own
+  int32_t no_gather;       // 1: 1x1 layers on small planes keep the separate layout pass (never gathered by the kernel's own warps)
   int32_t dw_stride;       // > 0: the pointwise layer of a depthwise + pointwise block; the depthwise layer's stride
   int32_t rowpair;         // planner-internal: this is the re-stated form of a 64-channel layer (IgemmPlan::rowpair)
 };
@@ -276,6 +277,7 @@ struct IgemmPlan {
   uint32_t a_bytes, b_bytes, b_alloc;
   int32_t a_rows;  // rows of a weight tile in shared memory (128, or 64 for layers of <= 64 channels per group)
   int32_t fine_units;  // TMA-store epilogue works in units of 32 pixels (else 64)
+  int32_t gather;      // 1x1 layer on planes of a multiple of 4 pixels read from x (NCHW) by the kernel's extra warps (a form of nchw)
   int32_t nacc;        // depthwise + pointwise blocks: 128-channel tiles (accumulators) that share a pixel tile's depthwise result: 1, 2, 4
   // Row pairs: a stride-1 layer of 64 output channels with R kernel rows is run as a layer of 128
   // "channels" (output row parity x channel), R + 1 kernel rows and stride 2 along H on P/2 rows:

@@ -901,6 +901,10 @@ struct IgemmArgs {
   int32_t fine_units; // TMA-store epilogue: units of 32 pixels instead of 64
   int32_t rowpair;    // lanes 64..127 hold the odd output rows of the layer's 64 channels (IgemmPlan::rowpair)
   int32_t nacc;       // depthwise + pointwise blocks: channel tiles (accumulators) per pixel tile: 1, 2 or 4
+  // 1x1 layers on planes that start on 8-byte boundaries only: the extra warps gather the
+  // pixel-major activation tile from x (NCHW) themselves
+  int32_t gather, g_hw, g_c;
+  const uint16_t* g_x;
   int32_t mshift;     // log2 of the channel tiles that one work item covers (pairs: 1; nacc: 0, 1, 2)
   int32_t acc_stride; // accumulator columns between the channel tiles of an item (nacc > 1: 512 / nacc)
   // split reduction (its own kernel instantiation): the channel blocks of a tile are dealt out to
@@ -1216,7 +1220,8 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < a.stages; ++s) {
-      mbar_init(smem_u32(&full_bar[s]), DWPW ? 1 + kDwWarps : 1);  // (the weight copy + one arrival per depthwise warp)
+      // (the weight copy + one arrival per depthwise / gathering warp)
+      mbar_init(smem_u32(&full_bar[s]), DWPW ? 1 + kDwWarps : 1);
       mbar_init(smem_u32(&empty_bar[s]), 1);
     }
     for (int s = 0; s < 2; ++s) {
@@ -1320,11 +1325,11 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           if (lane < a.nacc)
             tma_load_4d(sbase + a.b_alloc + (uint32_t)(lane * a.taps) * a.a_bytes, &tmA, fb, cb * KB, m0 + lane * 128, tap0, grp);
           const uint32_t ib = issued & 1u;
-          if (!mbar_wait(smem_u32(&in_empty[ib]), ((issued >> 1) & 1u) ^ 1u, &abort_flag, 64)) {
+          if (!a.gather && !mbar_wait(smem_u32(&in_empty[ib]), ((issued >> 1) & 1u) ^ 1u, &abort_flag, 64)) {
             ok = false;
             break;
           }
-          if (lane == 0) {
+          if (lane == 0 && !a.gather) {
             const uint32_t in_base = ring_base + (uint32_t)a.stages * a.stage_bytes + (uint32_t)(EW * a.nbuf) * kWarpStageBytes;
             mbar_expect_tx(smem_u32(&in_full[ib]), a.dw_in_bytes);
             tma_load_5d(in_base + ib * a.dw_in_alloc, &tmB, smem_u32(&in_full[ib]), cb * KB, 0, -1, p0 * a.dw_stride - 1, n0);
@@ -1492,6 +1497,69 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const int sd = a.dw_stride;
     const uint32_t in_base = ring_base + (uint32_t)a.stages * a.stage_bytes + (uint32_t)(EW * a.nbuf) * kWarpStageBytes;
     typename WorkIterOf<SPLIT, SHARED>::type it;
+    if (a.gather) {
+      // ---- 1x1 layer on NCHW planes of a multiple of 4 pixels: the stage is the pixel-major tile
+      // [64-pixel block][KB channel rows of 128 bytes], 128-byte swizzle, as the copy engine writes
+      // it for planes it can address.  The KB planes of a stage follow one another in x, so the
+      // stage is one contiguous run of 8-byte pieces (4 pixels of a channel); a thread copies every
+      // 256th of them with cp.async.  Where a piece goes does not depend on the stage: the offsets
+      // are computed once.  Up to three stages' copies are in flight; the oldest is waited for,
+      // made visible to the tensor core's proxy and reported on its barrier.
+      constexpr int kMaxPieces = 16;                      // per thread: KB * 64 pieces at most (planes of <= 256 pixels)
+      const int pieces_pc = a.g_hw >> 2;                 // pieces per channel
+      const int pieces = KB * pieces_pc;                  // per stage
+      uint32_t doff[kMaxPieces];
+#pragma unroll
+      for (int i = 0; i < kMaxPieces; ++i) {
+        const int pc = dt + i * (kDwWarps * 32);
+        const int cl = pc / pieces_pc, px = (pc - cl * pieces_pc) << 2;  // channel row, first pixel of the piece
+        doff[i] = (uint32_t)(px >> 6) * (uint32_t)(KB * 128) + (uint32_t)cl * 128u +
+                  (((uint32_t)((px & 63) >> 3) ^ ((uint32_t)cl & 7u)) << 4) + (uint32_t)(px & 4) * 2u;
+      }
+      // stages whose copies are in flight, oldest first (at most depth - 1, and at most 3)
+      const int max_fly = (int)depth - 1 < 3 ? (int)depth - 1 : 3;
+      int fly_idx[3] = {0, 0, 0};
+      int fly = 0;
+      auto retire_oldest = [&]() {  // wait for the oldest stage's copies, publish it, report it
+        if (fly == 3) asm volatile("cp.async.wait_group 2;" ::: "memory");
+        else if (fly == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
+        else asm volatile("cp.async.wait_group 0;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&full_bar[fly_idx[0]]));
+        fly_idx[0] = fly_idx[1];
+        fly_idx[1] = fly_idx[2];
+        --fly;
+      };
+      for (it.init(a); it.valid(a) && ok; it.next(a)) {
+        const int n0 = it.pt * a.tn;
+        for (int cb = 0; cb < a.cblocks && ok; ++cb) {
+          if (fly == max_fly) retire_oldest();
+          if (!mbar_wait(smem_u32(&empty_bar[ring.idx]), ring.phase ^ 1u, &abort_flag, 32)) {
+            ok = false;
+            break;
+          }
+          const uint32_t sbase = ring_base + ring.idx * a.stage_bytes;
+          const uint16_t* src = a.g_x + ((int64_t)n0 * a.g_c + (int64_t)cb * KB) * a.g_hw + (int64_t)dt * 4;
+#pragma unroll
+          for (int i = 0; i < kMaxPieces; ++i) {
+            if (dt + i * (kDwWarps * 32) < pieces) {
+              const uint16_t* sp = src + (int64_t)i * (kDwWarps * 32 * 4);
+              if (HGC_ADDR_OK(sp, 8))
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(sbase + doff[i]), "l"(sp) : "memory");
+            }
+          }
+          asm volatile("cp.async.commit_group;" ::: "memory");
+          fly_idx[fly++] = (int)ring.idx;
+          ring.advance(depth);
+        }
+      }
+      if (ok) {
+        while (fly > 0) retire_oldest();
+      } else {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+      }
+    } else
     for (it.init(a); it.valid(a) && ok; it.next(a)) {
       for (int cb = 0; cb < a.cblocks && ok; ++cb, ++produced) {
         const int c0 = cb * KB + chunk * 8;
@@ -2187,6 +2255,20 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
             g.pad_w == 0 && g.group == 1 && ((int64_t)g.h * g.w) % 8 == 0)
                ? 1
                : 0;
+  // The same layers on small planes of a multiple of 4 pixels (14x14), on request
+  // (HGC_FLAG_GATHER_X): a channel's plane starts on an 8-byte boundary only, which no tensor map
+  // can describe, so extra warps of the kernel gather the pixel-major tile themselves with 8-byte
+  // asynchronous copies (the kernel of the depthwise + pointwise blocks, whose extra warps produce
+  // the activation tile too).  A tile is one whole plane; whole 64-channel blocks only (nothing
+  // fills channels past the last one).  Measured slower than the layout pass + plain kernel
+  // (64 x 1024 -> 256 on 14x14: 24.8 us against 21.2; with the copies left out 13.6), hence opt-in.
+  p.gather = 0;
+  if (!p.nchw && !p.x_nhwc && !p.window && !p.patch && g.r == 1 && g.s == 1 && g.stride_h == 1 && g.stride_w == 1 &&
+      g.pad_h == 0 && g.pad_w == 0 && g.group == 1 && g.dw_stride == 0 && !g.rowpair && !want_pair && p.kb == 64 &&
+      (g.c % 64) == 0 && ((int64_t)g.h * g.w) % 4 == 0 && (int64_t)g.h * g.w <= 256 && !g.no_gather) {
+    p.nchw = 1;
+    p.gather = 1;
+  }
   p.pitch = p.dense_rows ? p.dense_pitch : (p.halo ? g.q + (g.s - 1) * g.dil_w : g.q);
   p.tw = g.q;
   const int box_w = (p.halo && !p.vhalo) ? p.pitch : ((p.window || p.patch) ? g.q : g.q * g.stride_w);
@@ -2267,13 +2349,14 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
   int best_th = 0, best_tn = 0, best_ks = 0, best_shared = 0, best_grid = 0;
   // shared tiles: asked for (no_split == 0: taken wherever tiles do not fill whole waves), or left
   // to this cost model (no_split == 2)
-  const bool can_share = g.no_split != 1 && sms <= kMaxGrid && p.kb >= 32;
+  const bool can_share = g.no_split != 1 && sms <= kMaxGrid && p.kb >= 32 && !p.gather;
   const bool force_share = g.no_split == 0;
   for (int th = 1; th <= g.p; ++th) {
     if ((int64_t)th * p.pitch - junk > 256 || (int64_t)th * (p.patch ? 1 : g.stride_h) > 256) break;
     if (p.vhalo && g.stride_h > 1 && th > 1) break;
     if (g.rowpair && th > 1) break;
     if (p.nchw && th != g.p && ((int64_t)th * g.q) % 8 != 0) continue;  // tiles must start on 16-byte boundaries of x
+    if (p.gather && th != g.p) continue;
     const int tn_hi = (th == g.p && !p.nchw && !p.vhalo) ? g.n : 1;  // several images only when a tile holds whole planes
     for (int tn = 1; tn <= tn_hi; ++tn) {
       const int64_t cols = (int64_t)tn * th * p.pitch - junk;
@@ -2517,7 +2600,7 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
   }
   p.a_bytes = (uint32_t)p.a_rows * p.kb * 2u;
   p.sk_cols32 = (p.ncols + 31) / 32;
-  if (p.pair || p.sk_split || g.dw_stride > 0) p.epi_warps = kEpilogueWarps;
+  if (p.pair || p.sk_split || g.dw_stride > 0 || p.gather) p.epi_warps = kEpilogueWarps;
   // split reduction (chosen with the tile shape above): fp32 partials, copy-style epilogue
   p.ks_log2 = best_ks;
   if (p.ks_log2 > 0) {
@@ -2809,7 +2892,7 @@ cudaError_t launch_igemm(const ConvGeom& g_layer, IgemmPlan& p, void* ws, const 
   if (!p.maps_ready) return cudaErrorInvalidValue;
   if (dw != nullptr && (!p.x_nhwc || p.pair || p.sk_split || p.ks_log2 > 0 || p.fuse_layout || p.kb < 32))
     return cudaErrorInvalidValue;
-  if (p.nchw && p.x_mapped != x && !igemm_encode_x_map(g, &p, x)) return cudaErrorInvalidValue;
+  if (p.nchw && !p.gather && p.x_mapped != x && !igemm_encode_x_map(g, &p, x)) return cudaErrorInvalidValue;
   if (dw != nullptr && p.x_mapped != x) {  // the block's input tiles come from x (channels-last) with their border
     if (p.dw_in_bytes == 0 || !encode_dw_input_map(*dw, g.n, &p)) return cudaErrorInvalidValue;
     p.x_mapped = x;
@@ -2880,6 +2963,10 @@ cudaError_t launch_igemm(const ConvGeom& g_layer, IgemmPlan& p, void* ws, const 
     a.dw_h = dw->h; a.dw_wd = dw->w; a.dw_c = dw->c; a.dw_stride = dw->stride; a.dw_relu = dw->relu;
     a.dw_in_h = p.dw_in_h; a.dw_in_w = p.dw_in_w; a.dw_in_bytes = p.dw_in_bytes; a.dw_in_alloc = p.dw_in_alloc;
   }
+  a.gather = p.gather;
+  a.g_x = reinterpret_cast<const uint16_t*>(x);
+  a.g_hw = g.h * g.w;
+  a.g_c = g.c;
   a.lay_x = reinterpret_cast<const uint16_t*>(x);
   a.lay_xp = reinterpret_cast<uint16_t*>(static_cast<char*>(ws) + p.ws_x_off);
   a.lay_flags = reinterpret_cast<int*>(static_cast<char*>(ws) + p.ws_lay_off);
@@ -2988,7 +3075,7 @@ cudaError_t launch_igemm(const ConvGeom& g_layer, IgemmPlan& p, void* ws, const 
     else if (!p.tma_store) HGC_LAUNCH_PAIR_EPI(KBV, HALOV, 1);     \
     else HGC_LAUNCH_PAIR_EPI(KBV, HALOV, 0);                       \
   } while (0)
-  if (dw != nullptr) {
+  if (dw != nullptr || p.gather) {
     if (p.kb == 64) HGC_LAUNCH_DWPW(64); else HGC_LAUNCH_DWPW(32);
   } else if (p.pair) {
     if (p.kb == 64) {

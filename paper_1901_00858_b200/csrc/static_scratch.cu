@@ -64,6 +64,7 @@ int make_geom(const hgc_conv_params* p, hgc::ConvGeom* g) {
   g->no_split = 1;
   g->no_pair = 1;
   g->no_fuse = 1;
+  g->no_gather = 1;
   return HGC_OK;
 }
 
@@ -74,7 +75,7 @@ inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) &
 extern "C" int hgc_conv_forward_static(const hgc_conv_params* p, const void* x, const void* w, const void* bias,
                                        void* y, int relu, void* stream) {
   if (x == nullptr || w == nullptr || y == nullptr) return HGC_INVALID_ARG;
-  hgc::ConvGeom g;
+  hgc::ConvGeom g{};  // (fields this entry point never sets, the block and row-pair markers, must be zero)
   const int rc = make_geom(p, &g);
   if (rc != HGC_OK) return rc;
   if (misaligned(x) || misaligned(w) || misaligned(y) || (bias != nullptr && misaligned(bias))) return HGC_BAD_ALIGNMENT;

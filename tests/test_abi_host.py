@@ -217,6 +217,22 @@ def test_scheduling_flags_change_the_plan_not_the_layer():
     assert hgc.ConvDesc(16, 128, 112, 112, 128, 3, 3, 1, 1, flags=hgc.HGC_FLAG_CTA_PAIRS).plan_info()["pair"] == 0
 
 
+def test_gather_flag_replaces_the_layout_pass_on_small_planes():
+    """1x1 layers on 14x14 planes (8-byte plane starts) take the NHWC copy of x unless
+    HGC_FLAG_GATHER_X asks the kernel's own warps to fetch x: then no copy is planned."""
+    args = (64, 1024, 14, 14, 256, 1, 1, 0, 0, 1, 1, 1, 1, 1)
+    plain = hgc.ConvDesc(*args)
+    gather = hgc.ConvDesc(*args, flags=hgc.HGC_FLAG_GATHER_X)
+    assert plain.plan_info()["x_source"] == 0 and gather.plan_info()["x_source"] == 4
+    assert gather.plan_info()["th"] == 14 and gather.plan_info()["tn"] == 1          # a tile is one plane
+    assert gather.workspace_bytes() + 2 * 64 * 1024 * 14 * 14 <= plain.workspace_bytes()
+    assert gather.output_dims() == plain.output_dims() and gather.path() == plain.path()
+    # planes the copy engine can address, odd planes and ragged channel blocks are not gathered
+    for other in ((2, 64, 16, 16, 64), (2, 64, 7, 7, 64), (2, 96, 14, 14, 64), (2, 64, 20, 20, 64)):
+        d = hgc.ConvDesc(*other, 1, 1, flags=hgc.HGC_FLAG_GATHER_X)
+        assert d.plan_info()["x_source"] != 4, other
+
+
 def test_64_channel_layers_fill_the_mma():
     """Layers of 64 output channels leave half of the 128-row MMA idle.  Wide stride-1 layers with
     several kernel rows run as row pairs (odd output rows in the upper lanes: tiles of two rows, one

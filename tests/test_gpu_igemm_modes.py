@@ -140,16 +140,28 @@ SCHED_CASES = [
      {"fused_layout": 1}),
     ("fused layout: 13x13 plane keeps the separate pass", params_dict(2, 96, 13, 13, 72, 3, 3, 1, 1), ("fused",),
      {"fused_layout": 0}),
+    # 1x1 layers on planes that start on 8-byte boundaries: x gathered by the kernel's own warps
+    ("gather 1x1 14x14 c256 k256 n3 (several stages in flight, two channel tiles)", params_dict(3, 256, 14, 14, 256, 1, 1),
+     ("gather",), {"x_source": 4}),
+    ("gather 1x1 14x14 c1024 k72 n2 (ring laps, ragged channel tile)", params_dict(2, 1024, 14, 14, 72, 1, 1), ("gather",),
+     {"x_source": 4}),
+    ("gather 1x1 10x10 c192 k130 n5", params_dict(5, 192, 10, 10, 130, 1, 1), ("gather",), {"x_source": 4}),
+    ("gather 1x1 2x2 c64 k16 n2 (one piece per channel)", params_dict(2, 64, 2, 2, 16, 1, 1), ("gather",), {"x_source": 4}),
+    ("gather 1x1 12x21 c64 k64 n2 (252 pixels: all 256 accumulator columns)", params_dict(2, 64, 12, 21, 64, 1, 1), ("gather",),
+     {"x_source": 4}),
+    ("gather: 16-byte planes go through the copy engine", params_dict(2, 64, 16, 15, 64, 1, 1), ("gather",), {"x_source": 1}),
+    ("gather: 7x7 planes keep the layout pass", params_dict(2, 64, 7, 7, 64, 1, 1), ("gather",), {"x_source": 0}),
+    ("gather: c96 keeps the layout pass", params_dict(2, 96, 14, 14, 64, 1, 1), ("gather",), {"x_source": 0}),
 ]
 
 
 @pytest.mark.parametrize("name,a,flag_names,want", SCHED_CASES, ids=[c[0] for c in SCHED_CASES])
 def test_scheduling_flags(hgc, oracle, name, a, flag_names, want):
-    """CTA pairs (cta_group::2), tiles shared by several CTAs and the layout pass inside the
-    tensor-core kernel are opt-in schedules of the same layer: the plan must report them where
+    """CTA pairs (cta_group::2), tiles shared by several CTAs, the layout pass inside the
+    tensor-core kernel and x gathered by the kernel's own warps are opt-in schedules of the same layer: the plan must report them where
     asked for, and the results must match the oracle."""
     flags = ((hgc.HGC_FLAG_CTA_PAIRS if "pairs" in flag_names else 0) | (hgc.HGC_FLAG_SHARED_TILES if "shared" in flag_names else 0)
-             | (hgc.HGC_FLAG_FUSED_LAYOUT if "fused" in flag_names else 0))
+             | (hgc.HGC_FLAG_FUSED_LAYOUT if "fused" in flag_names else 0) | (hgc.HGC_FLAG_GATHER_X if "gather" in flag_names else 0))
     rng = np.random.default_rng(zlib.crc32(name.encode()))
     x, w, b = workloads.random_layer_tensors(rng, a["n"], a["c"], a["h"], a["w"], a["k"], a["r"], a["s"], a["group"])
     P = oracle.ConvParams(**a)
