@@ -1750,7 +1750,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       if constexpr (PAIR) m0_item += (int)rank * 128;  // this CTA's tensor memory holds its own 128 channels
       // (block kernels with several channel tiles per pixel tile come back here for each of them)
       int ci = 0;
-    next_channel_tile:
+    [[maybe_unused]] next_channel_tile:
       const int m0 = m0_item + ci * 128;
       const int kin = m0 + row;
       const bool kvalid = kin < (a.rowpair ? 64 : a.kg);
