@@ -232,8 +232,11 @@ int hgc_conv_path(const hgc_conv_desc* d, int32_t* path);
  * hold the odd output rows ([4] then counts row pairs per tile, [7] tiles of two output rows, [9]
  * and the kernel's taps are those of a kernel with one more row), [17] the number of copies of the
  * layer's weight rows in a weight tile (2 for epilogue-bound layers of 64 output channels: lane
- * quarters 2 and 3 then hold the same channels as 0 and 1 and take other pixels; else 1); zeros
- * for the other paths.  info: host pointer; at most 18 values are written.
+ * quarters 2 and 3 then hold the same channels as 0 and 1 and take other pixels; else 1), [18] how
+ * the epilogue writes y: 1 = staged tiles sent by the copy engine (tensor map over y), 2 = tiles of
+ * whole planes of a 1x1 layer, one bulk copy per block of 32 channels (contiguous in y), 0 = plain
+ * stores from a staging tile; zeros for the other paths.  info: host pointer; at most 19 values
+ * are written.
  */
 int hgc_conv_plan_info(const hgc_conv_desc* d, int32_t* info, int32_t count);
 

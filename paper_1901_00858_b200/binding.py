@@ -185,10 +185,10 @@ class ConvDesc:
         return v.value
 
     def plan_info(self) -> dict:
-        v = (ctypes.c_int32 * 18)()
-        _check(lib().hgc_conv_plan_info(self._h, v, 18), "hgc_conv_plan_info")
+        v = (ctypes.c_int32 * 19)()
+        _check(lib().hgc_conv_plan_info(self._h, v, 19), "hgc_conv_plan_info")
         keys = ("path", "kb", "halo", "tn", "th", "pitch", "ncols", "tiles", "stages", "taps", "x_source",
-                "k_slices", "grid", "shared_tiles", "pair", "fused_layout", "row_pairs", "replicas")
+                "k_slices", "grid", "shared_tiles", "pair", "fused_layout", "row_pairs", "replicas", "y_store")
         return dict(zip(keys, list(v)))
 
     def workspace_bytes(self) -> int:

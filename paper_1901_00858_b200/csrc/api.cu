@@ -255,7 +255,7 @@ int hgc_conv_path(const hgc_conv_desc* d, int32_t* path) {
 
 int hgc_conv_plan_info(const hgc_conv_desc* d, int32_t* info, int32_t count) {
   if (d == nullptr || info == nullptr || count < 1) return HGC_INVALID_ARG;
-  int32_t v[18] = {d->path, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+  int32_t v[19] = {d->path, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
   if (d->path == HGC_PATH_IGEMM) {
     const hgc::IgemmPlan& p = d->igemm;
     v[1] = p.kb; v[2] = p.halo; v[3] = p.tn; v[4] = p.th; v[5] = p.pitch; v[6] = p.ncols;
@@ -268,8 +268,9 @@ int hgc_conv_plan_info(const hgc_conv_desc* d, int32_t* info, int32_t count) {
     v[15] = p.fuse_layout;
     v[16] = p.rowpair;
     v[17] = 1 << p.dup_log2;
+    v[18] = p.plane_store ? 2 : (p.tma_store ? 1 : 0);
   }
-  for (int i = 0; i < count && i < 18; ++i) info[i] = v[i];
+  for (int i = 0; i < count && i < 19; ++i) info[i] = v[i];
   return HGC_OK;
 }
 

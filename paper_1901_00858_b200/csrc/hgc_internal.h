@@ -277,6 +277,8 @@ struct IgemmPlan {
   uint32_t a_bytes, b_bytes, b_alloc;
   int32_t a_rows;  // rows of a weight tile in shared memory (128, or 64 for layers of <= 64 channels per group)
   int32_t fine_units;  // TMA-store epilogue works in units of 32 pixels (else 64)
+  int32_t plane_store; // whole-plane tiles leave as one bulk copy per 32-channel block
+  uint32_t plane_bytes;  //   bytes of a lane quarter's staging tile
   int32_t gather;      // 1x1 layer on planes of a multiple of 4 pixels read from x (NCHW) by the kernel's extra warps (a form of nchw)
   int32_t nacc;        // depthwise + pointwise blocks: 128-channel tiles (accumulators) that share a pixel tile's depthwise result: 1, 2, 4
   // Row pairs: a stride-1 layer of 64 output channels with R kernel rows is run as a layer of 128

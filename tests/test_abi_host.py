@@ -114,7 +114,7 @@ def test_planner_paths():
 def test_plan_info_reports_tiling_and_activation_source():
     """The planner runs on the host: its choices can be checked without a GPU."""
     keys = {"path", "kb", "halo", "tn", "th", "pitch", "ncols", "tiles", "stages", "taps", "x_source", "k_slices",
-            "grid", "shared_tiles", "pair", "fused_layout", "row_pairs", "replicas"}
+            "grid", "shared_tiles", "pair", "fused_layout", "row_pairs", "replicas", "y_store"}
     cases = [
         # (n, c, h, w, k, r, s, pad, stride), x_source
         ((16, 256, 56, 56, 256, 3, 3, 1, 1), 0),   # NHWC copy of x
@@ -231,6 +231,18 @@ def test_gather_flag_replaces_the_layout_pass_on_small_planes():
     for other in ((2, 64, 16, 16, 64), (2, 64, 7, 7, 64), (2, 96, 14, 14, 64), (2, 64, 20, 20, 64)):
         d = hgc.ConvDesc(*other, 1, 1, flags=hgc.HGC_FLAG_GATHER_X)
         assert d.plan_info()["x_source"] != 4, other
+
+
+def test_plan_reports_how_the_output_is_written():
+    """[18] of the plan: staged tiles through a tensor map (rows of whole 16-byte vectors), whole
+    planes of a 1x1 layer as bulk copies (14x14, 32-channel blocks contiguous in y), else plain stores."""
+    assert hgc.ConvDesc(16, 64, 56, 56, 64, 3, 3, 1, 1).plan_info()["y_store"] == 1
+    assert hgc.ConvDesc(64, 256, 14, 14, 1024, 1, 1, 0, 0).plan_info()["y_store"] == 2
+    assert hgc.ConvDesc(64, 256, 14, 14, 256, 3, 3, 1, 1).plan_info()["y_store"] == 0      # junk columns between rows
+    assert hgc.ConvDesc(64, 512, 7, 7, 2048, 1, 1, 0, 0).plan_info()["y_store"] == 0       # 98-byte planes
+    assert hgc.ConvDesc(64, 256, 14, 14, 1000, 1, 1, 0, 0).plan_info()["y_store"] == 0     # K % 32 != 0
+    assert hgc.ConvDesc(2, 256, 14, 14, 1024, 1, 1, 0, 0).plan_info()["y_store"] == 0      # few images: tiles of a few rows
+    assert hgc.ConvDesc(64, 256, 14, 14, 1024, 1, 1, 0, 0, flags=hgc.HGC_FLAG_Y_NHWC).plan_info()["y_store"] == 1
 
 
 def test_64_channel_layers_fill_the_mma():

@@ -183,6 +183,38 @@ def test_scheduling_flags(hgc, oracle, name, a, flag_names, want):
                 assert np.array_equal(first.view(np.uint16), got.view(np.uint16)), "the schedule must be deterministic"
 
 
+PLANE_CASES = [
+    # (name, layer, flags, plan keys): tiles of whole output planes of 1x1 layers leave as one bulk copy per 32-channel block
+    ("14x14 c64 k256 n40", params_dict(40, 64, 14, 14, 256, 1, 1), 0, {"y_store": 2, "th": 14, "tn": 1}),
+    ("10x10 c128 k160 n48 (ragged last group of columns)", params_dict(48, 128, 10, 10, 160, 1, 1), 0, {"y_store": 2, "tn": 1}),
+    ("2x2 c64 k32 n70 (several images per tile, last tile short)", params_dict(70, 64, 2, 2, 32, 1, 1), 0, {"y_store": 2}),
+    ("6x6 c64 k64 n120 stride 2 from 12x12", params_dict(120, 64, 12, 12, 64, 1, 1, 0, 0, 2, 2), 0, {"y_store": 2, "th": 6}),
+    ("6x6 c64 k96 n200 (two images per tile)", params_dict(200, 64, 6, 6, 96, 1, 1), 0, {"y_store": 2, "tn": 2}),
+    ("14x14 c256 k256 n20, x gathered by the kernel's warps", params_dict(20, 256, 14, 14, 256, 1, 1), "gather", {"y_store": 2, "x_source": 4}),
+    ("k72: channel blocks are not whole, copy epilogue", params_dict(40, 64, 14, 14, 72, 1, 1), 0, {"y_store": 0}),
+    ("7x7: planes of 98 bytes, copy epilogue", params_dict(64, 64, 7, 7, 64, 1, 1), 0, {"y_store": 0}),
+    ("3x3 on 14x14: junk columns between rows, copy epilogue", params_dict(64, 64, 14, 14, 64, 3, 3, 1, 1), 0, {"y_store": 0}),
+]
+
+
+@pytest.mark.parametrize("name,a,flags,want", PLANE_CASES, ids=[c[0] for c in PLANE_CASES])
+def test_whole_plane_epilogue(hgc, oracle, name, a, flags, want):
+    """Whole-tensor comparison of the layers whose tiles are written as bulk copies, and of their
+    neighbours that must keep the copy epilogue; the output buffer is NaN-filled with guard bands."""
+    fl = hgc.HGC_FLAG_GATHER_X if flags == "gather" else flags
+    rng = np.random.default_rng(zlib.crc32(name.encode()))
+    x, w, b = workloads.random_layer_tensors(rng, a["n"], a["c"], a["h"], a["w"], a["k"], a["r"], a["s"], a["group"])
+    d = hgc.ConvDesc(flags=fl, **a)
+    info = d.plan_info()
+    d.close()
+    for key, value in want.items():
+        assert info[key] == value, (name, info)
+    for relu, bias in ((True, b), (False, None)):
+        ref = oracle.conv_fast(oracle.ConvParams(**a), x, w, bias, relu)
+        got, _ = run_layer(hgc, a, x, w, bias, relu, flags=fl)
+        check_close(got, ref, what=f"{name} relu={relu}")
+
+
 def test_scheduling_flags_channels_last(hgc, oracle):
     """The same schedules with channels-last activations on both sides."""
     from gpu_util import to_dev, to_host
