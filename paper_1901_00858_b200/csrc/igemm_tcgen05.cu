@@ -895,7 +895,7 @@ struct IgemmArgs {
   int32_t cg;          // channels per group (nchw: channel coordinate of the tile)
   int32_t relu;
   int32_t tma_store;  // 1: the epilogue stages fp16 tiles in shared memory and stores them with TMA
-  int32_t plane_store;  // 1: whole-plane tiles leave as one bulk copy per 32-channel block (epilogue_planes)
+  int32_t plane_store;  // 1, 2: whole-plane tiles leave as one bulk copy per 32-channel block (epilogue_planes: its mode)
   uint32_t plane_bytes; //    bytes of a lane quarter's staging tile
   int32_t rem;        // (th*Q) % 64: width of the last staged pass of a full tile (0 = none)
   int32_t nbuf;       // staging tiles per epilogue warp (1 or 2)
@@ -1193,30 +1193,39 @@ __device__ __forceinline__ void dw_pair(uint32_t src0, uint32_t row_bytes, uint3
 
 // Whole-plane epilogue: tiles that hold whole output planes (of one or several images) of a 1x1
 // layer (accumulator columns are the planes' pixels) whose 32-channel blocks are runs of
-// 32 * P*Q contiguous, 16-byte aligned halves in y (K % 32 == 0, P*Q % 4 == 0).  The two warps of a lane quarter convert
-// alternate groups of 32 columns into ONE staging tile that is the memory image of the block
-// ([32 channels][P*Q], rows 8-byte aligned: 8-byte stores, no bank conflicts within a half warp),
-// meet on a named barrier, and one lane sends the block with a single bulk copy.  (The copy
-// epilogue's stores, 128 bytes per instruction and channel row, cost a 14x14 layer of 1024
-// output channels 8.9 of its 22.7 us: measured with the stores left out.)
-__device__ __noinline__ void epilogue_planes(uint32_t t_addr, uint32_t qstage, int half, int tn, int N, int K, int pq, int n0,
-                                             int k0, float bv, bool relu, uint16_t* yb) {
+// 32 * P*Q contiguous, 16-byte aligned halves in y (K % 32 == 0).  The block is built in a staging
+// tile that is its memory image ([32 channels][P*Q], a lane writes its channel's row: 8-byte
+// stores when P*Q % 4 == 0, which are conflict-free within a half warp, else 2-byte stores) and
+// leaves with a single bulk copy.  One image per tile (mode 1): the two warps of a lane quarter
+// convert alternate groups of 32 columns into one tile, meet on a named barrier, and one lane
+// sends it.  Several images per tile (mode 2): the warps take alternate images, each with a
+// staging tile of its own, and need not meet.  (The copy epilogue's stores, 128 bytes per
+// instruction and channel row, cost a 14x14 layer of 1024 output channels 8.9 of its 22.7 us:
+// measured with the stores left out.)
+__device__ __noinline__ void epilogue_planes(uint32_t t_addr, uint32_t qstage, int half, int mode, int tn, int N, int K, int pq,
+                                             int n0, int k0, float bv, bool relu, uint16_t* yb) {
   const int lane = threadIdx.x & 31;
   const int quarter = (threadIdx.x >> 5) & 3;
-  const uint32_t row = qstage + (uint32_t)lane * (uint32_t)(pq * 2);
+  const bool shared_tile = mode == 1;
+  const uint32_t tile_bytes = (uint32_t)(((32 * pq * 2) + 127) & ~127);
+  const uint32_t tile = shared_tile ? qstage : qstage + (uint32_t)half * tile_bytes;
+  const uint32_t row = tile + (uint32_t)lane * (uint32_t)(pq * 2);
+  const bool wide = (pq & 3) == 0;
   auto quarter_sync = [&]() {  // the two warps of this lane quarter (named barriers 1..4)
     if (quarter == 0) asm volatile("bar.sync 1, 64;" ::: "memory");
     else if (quarter == 1) asm volatile("bar.sync 2, 64;" ::: "memory");
     else if (quarter == 2) asm volatile("bar.sync 3, 64;" ::: "memory");
     else asm volatile("bar.sync 4, 64;" ::: "memory");
   };
-  for (int img = 0; img < tn; ++img) {
+  const bool sender = lane == 0 && (half == 0 || !shared_tile);
+  for (int img = shared_tile ? 0 : half; img < tn; img += shared_tile ? 1 : 2) {
     if (n0 + img >= N) break;
     // the staging tile's previous copy must have read it
-    if (half == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-    quarter_sync();
-    for (int c0 = half * 32; c0 < pq; c0 += 64) {
-      const int ncol = pq - c0 < 32 ? pq - c0 : 32;  // a multiple of 4
+    if (sender) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+    if (shared_tile) quarter_sync();
+    else __syncwarp();
+    for (int c0 = shared_tile ? half * 32 : 0; c0 < pq; c0 += shared_tile ? 64 : 32) {
+      const int ncol = pq - c0 < 32 ? pq - c0 : 32;
       const uint32_t tcol = t_addr + (uint32_t)(img * pq + c0);
       uint32_t v[32];
       if (ncol == 32) {
@@ -1227,25 +1236,39 @@ __device__ __noinline__ void epilogue_planes(uint32_t t_addr, uint32_t qstage, i
           if (c * 8 < ncol) tmem_ld8(tcol + (uint32_t)(c * 8), &v[8 * c]);
       }
       asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      if (wide) {  // (ncol is a multiple of 4)
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        if (4 * j < ncol) {
-          const float f0 = __uint_as_float(v[4 * j]) + bv, f1 = __uint_as_float(v[4 * j + 1]) + bv;
-          const float f2 = __uint_as_float(v[4 * j + 2]) + bv, f3 = __uint_as_float(v[4 * j + 3]) + bv;
-          const uint32_t o0 = relu ? pack_f16x2<true>(f0, f1) : pack_f16x2<false>(f0, f1);
-          const uint32_t o1 = relu ? pack_f16x2<true>(f2, f3) : pack_f16x2<false>(f2, f3);
-          asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(row + (uint32_t)((c0 + 4 * j) * 2)), "r"(o0), "r"(o1) : "memory");
+        for (int j = 0; j < 8; ++j) {
+          if (4 * j < ncol) {
+            const float f0 = __uint_as_float(v[4 * j]) + bv, f1 = __uint_as_float(v[4 * j + 1]) + bv;
+            const float f2 = __uint_as_float(v[4 * j + 2]) + bv, f3 = __uint_as_float(v[4 * j + 3]) + bv;
+            const uint32_t o0 = relu ? pack_f16x2<true>(f0, f1) : pack_f16x2<false>(f0, f1);
+            const uint32_t o1 = relu ? pack_f16x2<true>(f2, f3) : pack_f16x2<false>(f2, f3);
+            asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(row + (uint32_t)((c0 + 4 * j) * 2)), "r"(o0), "r"(o1) : "memory");
+          }
+        }
+      } else {  // rows of the tile start on 2-byte boundaries (7x7 planes: 98 bytes)
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          if (2 * j < ncol) {
+            const float f0 = __uint_as_float(v[2 * j]) + bv, f1 = __uint_as_float(v[2 * j + 1]) + bv;
+            const uint32_t o = relu ? pack_f16x2<true>(f0, f1) : pack_f16x2<false>(f0, f1);
+            asm volatile("st.shared.b16 [%0], %1;" ::"r"(row + (uint32_t)((c0 + 2 * j) * 2)), "h"((uint16_t)(o & 0xffffu)) : "memory");
+            if (2 * j + 1 < ncol)
+              asm volatile("st.shared.b16 [%0], %1;" ::"r"(row + (uint32_t)((c0 + 2 * j + 1) * 2)), "h"((uint16_t)(o >> 16)) : "memory");
+          }
         }
       }
     }
     // the copy engine reads the tile through the async proxy
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    quarter_sync();
-    if (half == 0 && lane == 0) {
+    if (shared_tile) quarter_sync();
+    else __syncwarp();
+    if (sender) {
       uint16_t* dst = yb + ((int64_t)(n0 + img) * K + k0) * pq;
       const uint32_t bytes = (uint32_t)(32 * pq * 2);
       if (HGC_ADDR_OK(dst, bytes)) {
-        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(qstage), "r"(bytes) : "memory");
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(tile), "r"(bytes) : "memory");
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
       }
     }
@@ -2038,8 +2061,8 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             } else if constexpr (EPI == 3) {
               // whole-plane tiles (instantiations of their own: the other kernels' code stays as it is)
               if (quarter_live)
-                epilogue_planes(t_addr, stage_base + (uint32_t)quarter * a.plane_bytes, half, a.tn, a.N, a.K, a.P * a.Q, n0,
-                                grp * a.kg + m0 + quarter * 32, bv, relu, yb);
+                epilogue_planes(t_addr, stage_base + (uint32_t)quarter * a.plane_bytes, half, a.plane_store, a.tn, a.N, a.K, a.P * a.Q,
+                                n0, grp * a.kg + m0 + quarter * 32, bv, relu, yb);
             } else if (quarter_live) {
               const int kleft = a.kg - (m0 + quarter * 32);
               epilogue_copy(t_addr, my_stage, half, kPerQuarter, a.tn, a.th, a.pitch, a.N, a.K, a.P, a.Q, n0, p0,
@@ -2685,10 +2708,11 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
     // (1x1 layers: no junk columns between the rows of a tile.  With them, 3x3 layers on 14x14, the
     //  row-by-row accumulator loads made this form slower than the copy epilogue: 22.1 against 20.7 us.)
     if (!p.tma_store && !p.y_nhwc && p.ks_log2 == 0 && !p.pair && !p.sk_split && g.group == 1 && g.dw_stride == 0 && g.r == 1 &&
-        g.s == 1 && p.th == g.p && !p.patch && !p.window && pq > 1 && pq <= 256 && (pq % 4) == 0 && (g.k % 32) == 0 &&
+        g.s == 1 && p.th == g.p && !p.patch && !p.window && pq > 1 && pq <= 256 && (g.k % 32) == 0 &&
         p.epi_warps == kEpilogueWarps) {
-      p.plane_store = 1;
-      p.plane_bytes = (uint32_t)round_up_sz((size_t)(32 * pq * 2), 128);
+      // one image per tile: the two warps of a lane quarter share a staging tile; several: one each
+      p.plane_store = p.tn == 1 ? 1 : 2;
+      p.plane_bytes = (uint32_t)round_up_sz((size_t)(32 * pq * 2), 128) * (uint32_t)p.plane_store;
     }
   }
   const size_t stage_buf_bytes = p.plane_store ? (size_t)4 * p.plane_bytes : (size_t)p.epi_warps * kWarpStageBytes;

@@ -235,11 +235,11 @@ def test_gather_flag_replaces_the_layout_pass_on_small_planes():
 
 def test_plan_reports_how_the_output_is_written():
     """[18] of the plan: staged tiles through a tensor map (rows of whole 16-byte vectors), whole
-    planes of a 1x1 layer as bulk copies (14x14, 32-channel blocks contiguous in y), else plain stores."""
+    planes of a 1x1 layer as bulk copies (14x14, 7x7: 32-channel blocks contiguous in y), else plain stores."""
     assert hgc.ConvDesc(16, 64, 56, 56, 64, 3, 3, 1, 1).plan_info()["y_store"] == 1
     assert hgc.ConvDesc(64, 256, 14, 14, 1024, 1, 1, 0, 0).plan_info()["y_store"] == 2
     assert hgc.ConvDesc(64, 256, 14, 14, 256, 3, 3, 1, 1).plan_info()["y_store"] == 0      # junk columns between rows
-    assert hgc.ConvDesc(64, 512, 7, 7, 2048, 1, 1, 0, 0).plan_info()["y_store"] == 0       # 98-byte planes
+    assert hgc.ConvDesc(64, 512, 7, 7, 2048, 1, 1, 0, 0).plan_info()["y_store"] == 2       # four images per tile
     assert hgc.ConvDesc(64, 256, 14, 14, 1000, 1, 1, 0, 0).plan_info()["y_store"] == 0     # K % 32 != 0
     assert hgc.ConvDesc(2, 256, 14, 14, 1024, 1, 1, 0, 0).plan_info()["y_store"] == 0      # few images: tiles of a few rows
     assert hgc.ConvDesc(64, 256, 14, 14, 1024, 1, 1, 0, 0, flags=hgc.HGC_FLAG_Y_NHWC).plan_info()["y_store"] == 1

@@ -44,6 +44,7 @@ CHILD = textwrap.dedent(r'''
         ("grouped", params_dict(1, 96, 27, 27, 256, 5, 5, 2, 2, 1, 1, 1, 1, 2), 0),
         ("x gathered by the kernel's warps", params_dict(3, 128, 14, 14, 72, 1, 1), hgc.HGC_FLAG_GATHER_X),
         ("whole planes as bulk copies", params_dict(40, 64, 14, 14, 96, 1, 1), 0),
+        ("whole planes as bulk copies, several images per tile", params_dict(33, 64, 7, 7, 256, 1, 1), 0),
         # depthwise kernels (rows of whole vectors, column words, small rows, general), direct kernel
         ("depthwise 112x112", params_dict(2, 32, 112, 112, 32, 3, 3, 1, 1, 1, 1, 1, 1, 32), 0),
         ("depthwise 56x56 stride 2", params_dict(2, 64, 56, 56, 64, 3, 3, 1, 1, 2, 2, 1, 1, 64), 0),

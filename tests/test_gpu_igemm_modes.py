@@ -192,7 +192,12 @@ PLANE_CASES = [
     ("6x6 c64 k96 n200 (two images per tile)", params_dict(200, 64, 6, 6, 96, 1, 1), 0, {"y_store": 2, "tn": 2}),
     ("14x14 c256 k256 n20, x gathered by the kernel's warps", params_dict(20, 256, 14, 14, 256, 1, 1), "gather", {"y_store": 2, "x_source": 4}),
     ("k72: channel blocks are not whole, copy epilogue", params_dict(40, 64, 14, 14, 72, 1, 1), 0, {"y_store": 0}),
-    ("7x7: planes of 98 bytes, copy epilogue", params_dict(64, 64, 7, 7, 64, 1, 1), 0, {"y_store": 0}),
+    ("7x7 c512 k256 n64 (98-byte planes: 2-byte staging stores, one image per tile)", params_dict(64, 512, 7, 7, 256, 1, 1), 0,
+     {"y_store": 2, "tn": 1}),
+    ("7x7 c64 k2048 n33 (four images per tile, the last tile short)", params_dict(33, 64, 7, 7, 2048, 1, 1), 0, {"y_store": 2, "tn": 4}),
+    ("3x3 planes c64 k32 n130", params_dict(130, 64, 3, 3, 32, 1, 1), 0, {"y_store": 2}),
+    ("1x2 planes c64 k64 n300 (eight images per tile)", params_dict(300, 64, 1, 2, 64, 1, 1), 0, {"y_store": 2, "tn": 8}),
+    ("7x7 c64 k64 n64: tiles of four rows, copy epilogue", params_dict(64, 64, 7, 7, 64, 1, 1), 0, {"y_store": 0}),
     ("3x3 on 14x14: junk columns between rows, copy epilogue", params_dict(64, 64, 14, 14, 64, 3, 3, 1, 1), 0, {"y_store": 0}),
 ]
 
