@@ -112,8 +112,9 @@ typedef struct hgc_conv_params {
  * with C a multiple of 64, start on 8-byte boundaries only, which no tensor map can describe;
  * with this flag eight extra warps of the tensor-core kernel gather the pixel-major tile
  * themselves with 8-byte asynchronous copies (plan [10] = 4) and no copy of x is made.  Measured
- * (B200): slower than the layout pass plus the plain kernel (64 x 1024 -> 256 on 14x14: 24.8 us
- * against 21.2; 256 -> 1024: 32.1 against 23.1), so it is not the planner's choice.
+ * (B200, against the layout pass plus the plain kernel): 64 x 1024 -> 256 on 14x14 19.1 us against
+ * 20.3; 256 -> 1024 21.8 against 18.4; 32 x 512 -> 512 12.5 against 12.3: it pays only where x is
+ * large and the output small, so it is not the planner's choice.
  */
 #define HGC_FLAG_GATHER_X 128
 

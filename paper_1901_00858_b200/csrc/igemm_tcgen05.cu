@@ -2352,8 +2352,9 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
   // can describe, so extra warps of the kernel gather the pixel-major tile themselves with 8-byte
   // asynchronous copies (the kernel of the depthwise + pointwise blocks, whose extra warps produce
   // the activation tile too).  A tile is one whole plane; whole 64-channel blocks only (nothing
-  // fills channels past the last one).  Measured slower than the layout pass + plain kernel
-  // (64 x 1024 -> 256 on 14x14: 24.8 us against 21.2; with the copies left out 13.6), hence opt-in.
+  // fills channels past the last one).  Measured against the layout pass + plain kernel: 64 x 1024
+  // -> 256 on 14x14 19.1 us against 20.3, 256 -> 1024 21.8 against 18.4 (with the copies left out
+  // 13.6 and 25.8 before the whole-plane epilogue): a gain only where x is large and y small, hence opt-in.
   p.gather = 0;
   if (!p.nchw && !p.x_nhwc && !p.window && !p.patch && g.r == 1 && g.s == 1 && g.stride_h == 1 && g.stride_w == 1 &&
       g.pad_h == 0 && g.pad_w == 0 && g.group == 1 && g.dw_stride == 0 && !g.rowpair && !want_pair && p.kb == 64 &&
