@@ -1192,7 +1192,7 @@ __device__ __forceinline__ void dw_pair(uint32_t src0, uint32_t row_bytes, uint3
 }
 
 // Whole-plane epilogue: tiles that hold whole output planes (of one or several images) of a 1x1
-// layer (accumulator columns are the planes' pixels) whose 32-channel blocks are runs of
+// or strided layer (accumulator columns are the planes' pixels) whose 32-channel blocks are runs of
 // 32 * P*Q contiguous, 16-byte aligned halves in y (K % 32 == 0).  The block is built in a staging
 // tile that is its memory image ([32 channels][P*Q], a lane writes its channel's row: 8-byte
 // stores when P*Q % 4 == 0, which are conflict-free within a half warp, else 2-byte stores) and
@@ -2708,9 +2708,10 @@ bool make_plan_impl(const ConvGeom& g, IgemmPlan* out, bool want_pair, int kb_ma
     const int64_t pq = (int64_t)g.p * g.q;
     // (1x1 layers: no junk columns between the rows of a tile.  With them, 3x3 layers on 14x14, the
     //  row-by-row accumulator loads made this form slower than the copy epilogue: 22.1 against 20.7 us.)
-    if (!p.tma_store && !p.y_nhwc && p.ks_log2 == 0 && !p.pair && !p.sk_split && g.group == 1 && g.dw_stride == 0 && g.r == 1 &&
-        g.s == 1 && p.th == g.p && !p.patch && !p.window && pq > 1 && pq <= 256 && (g.k % 32) == 0 &&
-        p.epi_warps == kEpilogueWarps) {
+    //  Strided layers never share a tile between taps, so their columns are pixels as well.
+    const bool linear_cols = (g.r == 1 && g.s == 1) || !p.halo;
+    if (!p.tma_store && !p.y_nhwc && p.ks_log2 == 0 && !p.pair && !p.sk_split && g.group == 1 && g.dw_stride == 0 && linear_cols &&
+        p.th == g.p && !p.patch && !p.window && pq > 1 && pq <= 256 && (g.k % 32) == 0 && p.epi_warps == kEpilogueWarps) {
       // one image per tile: the two warps of a lane quarter share a staging tile; several: one each
       p.plane_store = p.tn == 1 ? 1 : 2;
       p.plane_bytes = (uint32_t)round_up_sz((size_t)(32 * pq * 2), 128) * (uint32_t)p.plane_store;

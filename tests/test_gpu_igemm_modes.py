@@ -191,6 +191,10 @@ PLANE_CASES = [
     ("6x6 c64 k64 n120 stride 2 from 12x12", params_dict(120, 64, 12, 12, 64, 1, 1, 0, 0, 2, 2), 0, {"y_store": 2, "th": 6}),
     ("6x6 c64 k96 n200 (two images per tile)", params_dict(200, 64, 6, 6, 96, 1, 1), 0, {"y_store": 2, "tn": 2}),
     ("14x14 c256 k256 n20, x gathered by the kernel's warps", params_dict(20, 256, 14, 14, 256, 1, 1), "gather", {"y_store": 2, "x_source": 4}),
+    ("3x3 stride 2, 12x12 -> 6x6, c64 k64 n40 (taps do not share a tile: columns are pixels)",
+     params_dict(40, 64, 12, 12, 64, 3, 3, 1, 1, 2, 2), 0, {"y_store": 2, "halo": 0}),
+    ("3x3 stride 2, 14x14 -> 7x7, c64 k64 n150 (two images per tile)", params_dict(150, 64, 14, 14, 64, 3, 3, 1, 1, 2, 2), 0,
+     {"y_store": 2, "tn": 2}),
     ("k72: channel blocks are not whole, copy epilogue", params_dict(40, 64, 14, 14, 72, 1, 1), 0, {"y_store": 0}),
     ("7x7 c512 k256 n64 (98-byte planes: 2-byte staging stores, one image per tile)", params_dict(64, 512, 7, 7, 256, 1, 1), 0,
      {"y_store": 2, "tn": 1}),
