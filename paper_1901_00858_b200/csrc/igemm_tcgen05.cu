@@ -1197,33 +1197,31 @@ __device__ __forceinline__ void dw_pair(uint32_t src0, uint32_t row_bytes, uint3
 // tile that is its memory image ([32 channels][P*Q], a lane writes its channel's row: 8-byte
 // stores when P*Q % 4 == 0, which are conflict-free within a half warp, else 2-byte stores) and
 // leaves with a single bulk copy.  One image per tile (mode 1): the two warps of a lane quarter
-// convert alternate groups of 32 columns into one tile, meet on a named barrier, and one lane
-// sends it.  Several images per tile (mode 2): the warps take alternate images, each with a
+// convert alternate groups of 32 columns into one tile, meet, and one lane sends it.  Several images per tile (mode 2): the warps take alternate images, each with a
 // staging tile of its own, and need not meet.  (The copy epilogue's stores, 128 bytes per
 // instruction and channel row, cost a 14x14 layer of 1024 output channels 8.9 of its 22.7 us:
 // measured with the stores left out.)
-__device__ __noinline__ void epilogue_planes(uint32_t t_addr, uint32_t qstage, int half, int mode, int tn, int N, int K, int pq,
-                                             int n0, int k0, float bv, bool relu, uint16_t* yb) {
+// The meetings are on an mbarrier of the quarter with a bounded wait (a named barrier would hang a
+// warp whose partner has left on a timeout); returns the barrier's next phase, or ~0 after giving up.
+__device__ __noinline__ uint32_t epilogue_planes(uint32_t t_addr, uint32_t qstage, int half, int mode, int tn, int N, int K, int pq,
+                                                 int n0, int k0, float bv, bool relu, uint16_t* yb, uint32_t qbar, uint32_t phase,
+                                                 volatile int* abort_flag) {
   const int lane = threadIdx.x & 31;
-  const int quarter = (threadIdx.x >> 5) & 3;
   const bool shared_tile = mode == 1;
   const uint32_t tile_bytes = (uint32_t)(((32 * pq * 2) + 127) & ~127);
   const uint32_t tile = shared_tile ? qstage : qstage + (uint32_t)half * tile_bytes;
   const uint32_t row = tile + (uint32_t)lane * (uint32_t)(pq * 2);
   const bool wide = (pq & 3) == 0;
-  auto quarter_sync = [&]() {  // the two warps of this lane quarter (named barriers 1..4)
-    if (quarter == 0) asm volatile("bar.sync 1, 64;" ::: "memory");
-    else if (quarter == 1) asm volatile("bar.sync 2, 64;" ::: "memory");
-    else if (quarter == 2) asm volatile("bar.sync 3, 64;" ::: "memory");
-    else asm volatile("bar.sync 4, 64;" ::: "memory");
-  };
   const bool sender = lane == 0 && (half == 0 || !shared_tile);
   for (int img = shared_tile ? 0 : half; img < tn; img += shared_tile ? 1 : 2) {
     if (n0 + img >= N) break;
     // the staging tile's previous copy must have read it
     if (sender) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-    if (shared_tile) quarter_sync();
-    else __syncwarp();
+    if (shared_tile) {
+      if (!epi_sync(qbar, phase, abort_flag)) return ~0u;
+    } else {
+      __syncwarp();
+    }
     for (int c0 = shared_tile ? half * 32 : 0; c0 < pq; c0 += shared_tile ? 64 : 32) {
       const int ncol = pq - c0 < 32 ? pq - c0 : 32;
       const uint32_t tcol = t_addr + (uint32_t)(img * pq + c0);
@@ -1262,8 +1260,11 @@ __device__ __noinline__ void epilogue_planes(uint32_t t_addr, uint32_t qstage, i
     }
     // the copy engine reads the tile through the async proxy
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    if (shared_tile) quarter_sync();
-    else __syncwarp();
+    if (shared_tile) {
+      if (!epi_sync(qbar, phase, abort_flag)) return ~0u;
+    } else {
+      __syncwarp();
+    }
     if (sender) {
       uint16_t* dst = yb + ((int64_t)(n0 + img) * K + k0) * pq;
       const uint32_t bytes = (uint32_t)(32 * pq * 2);
@@ -1273,6 +1274,7 @@ __device__ __noinline__ void epilogue_planes(uint32_t t_addr, uint32_t qstage, i
       }
     }
   }
+  return phase;
 }
 
 constexpr int kLayoutWarps = 8;  // extra warps of the instantiations with the fused layout pass
@@ -1295,6 +1297,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   __shared__ __align__(8) uint64_t ho_bar;    //   of the warps that hand accumulators over (the first of each lane quarter),
   __shared__ __align__(8) uint64_t pl_bar;    //   of the warps that fetch partial sums (the second of each lane quarter)
   __shared__ __align__(8) uint64_t in_full[2], in_empty[2];  // depthwise input tiles (depthwise + pointwise blocks)
+  __shared__ __align__(8) uint64_t q_bar[4];  // whole-plane epilogue: meeting point of the two warps of a lane quarter
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -1320,6 +1323,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       mbar_init(smem_u32(&in_empty[b]), kDwWarps);
     }
     mbar_init(smem_u32(&sk_bar), PAIR ? EW : EW / 2);  // one arrival per fetching warp (of both CTAs)
+    for (int q = 0; q < 4; ++q) mbar_init(smem_u32(&q_bar[q]), EW / 4);
     mbar_init(smem_u32(&meet_bar), EW);
     mbar_init(smem_u32(&ho_bar), EW / 2);
     mbar_init(smem_u32(&pl_bar), EW / 2);
@@ -1761,7 +1765,8 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const uint32_t row_off = (uint32_t)lane * 128u + (((uint32_t)lane & 7u) << 4);
     uint32_t unit_ctr = 0, stage_sel = 0;
     uint32_t lt = 0;
-    uint32_t meet_phase = 0, ho_phase = 0, pl_phase = 0;
+    uint32_t meet_phase = 0, ho_phase = 0, pl_phase = 0, q_phase = 0;
+    bool gave_up = false;  // (a meeting of the whole-plane epilogue ran out of time)
     float bv = 0.f;
     int bias_k = -1;
     // Shared tiles: when this unit's range ends inside a tile whose first stage it holds, it
@@ -2060,9 +2065,12 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                                kleft < 32 ? kleft : 32, bv, relu, yb);
             } else if constexpr (EPI == 3) {
               // whole-plane tiles (instantiations of their own: the other kernels' code stays as it is)
-              if (quarter_live)
-                epilogue_planes(t_addr, stage_base + (uint32_t)quarter * a.plane_bytes, half, a.plane_store, a.tn, a.N, a.K, a.P * a.Q,
-                                n0, grp * a.kg + m0 + quarter * 32, bv, relu, yb);
+              if (quarter_live) {
+                q_phase = epilogue_planes(t_addr, stage_base + (uint32_t)quarter * a.plane_bytes, half, a.plane_store, a.tn, a.N, a.K,
+                                          a.P * a.Q, n0, grp * a.kg + m0 + quarter * 32, bv, relu, yb, smem_u32(&q_bar[quarter]),
+                                          q_phase, &abort_flag);
+                if (q_phase == ~0u) gave_up = true;
+              }
             } else if (quarter_live) {
               const int kleft = a.kg - (m0 + quarter * 32);
               epilogue_copy(t_addr, my_stage, half, kPerQuarter, a.tn, a.th, a.pitch, a.N, a.K, a.P, a.Q, n0, p0,
@@ -2072,6 +2080,7 @@ igemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         }
       }
       }  // sub-tiles
+      if (gave_up) break;
       if constexpr (DWPW) {
         if (++ci < a.nacc) goto next_channel_tile;
       }

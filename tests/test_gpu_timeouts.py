@@ -39,11 +39,13 @@ def _forward(hgc, d, xd, wd, bd, shape, relu=True):
     ("CTA pairs: the first CTA's copies of a stage", params_dict(2, 64, 12, 12, 256, 3, 3, 1, 1), "pairs", 2),
     ("tiles shared between CTAs: a part that is never handed over", params_dict(2, 256, 24, 24, 256, 3, 3, 1, 1), "shared", 0),
     ("layout pass inside the kernel", params_dict(2, 64, 24, 24, 64, 3, 3, 1, 1), "fused", 1),
+    ("whole-plane epilogue (the warps of a lane quarter meet on a bounded barrier)", params_dict(40, 64, 14, 14, 256, 1, 1), "", 0),
+    ("x gathered by the kernel's own warps: the weight copy of a later stage", params_dict(20, 256, 14, 14, 256, 1, 1), "gather", 1),
 ])
 def test_tensor_core_wait_runs_out_and_the_descriptor_recovers(hgc, oracle, name, a, flags_name, drop):
     import torch
     flags = {"": 0, "pairs": hgc.HGC_FLAG_CTA_PAIRS, "shared": hgc.HGC_FLAG_SHARED_TILES,
-             "fused": hgc.HGC_FLAG_FUSED_LAYOUT}[flags_name]
+             "fused": hgc.HGC_FLAG_FUSED_LAYOUT, "gather": hgc.HGC_FLAG_GATHER_X}[flags_name]
     rng = np.random.default_rng(3)
     x, w, b = workloads.random_layer_tensors(rng, a["n"], a["c"], a["h"], a["w"], a["k"], a["r"], a["s"], a["group"])
     ref = oracle.conv_fast(oracle.ConvParams(**a), x, w, b, True)
